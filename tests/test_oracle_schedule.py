@@ -1,0 +1,143 @@
+"""Pins for the oracle's Algorithm-1 bookkeeping: grouping, order, delayed LR,
+memory model.  None of these needs a GPU."""
+import os
+
+import numpy as np
+import pytest
+
+import synth
+from oracle import hift_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "paper_figures.txt")
+
+
+def _golden():
+    out = {}
+    for line in open(GOLD):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        kv = line.split("|")[0]
+        k, v = kv.split("=")
+        out[k.strip()] = float(v)
+    return out
+
+
+def test_k_formula_grid():
+    # paper, Notation: k = n/m if m | n else floor(n/m)+1  == ceil(n/m)
+    for n in range(1, 60):
+        for m in range(1, n + 1):
+            k = O.num_groups(n, m)
+            assert k == -(-n // m)
+            groups = O.build_groups(n, m)
+            assert len(groups) == k
+            assert sum(groups, []) == list(range(n))            # a partition, in order
+            assert all(len(g) == m for g in groups[:-1])
+            assert 1 <= len(groups[-1]) <= m
+
+
+def test_llama_units_and_groups_match_paper():
+    g = _golden()
+    cfg, gc, _ = synth.config_llama_7b()
+    assert cfg.n_units == g["llama7b_units_n"]
+    assert len(O.build_groups(cfg.n_units, 1)) == g["llama7b_groups_k_at_m1"]
+
+
+def test_split_grouping_gpt2_large():
+    cfg, gc, _ = synth.config_gpt2_large()
+    groups = O.build_groups(cfg.n_units, gc.layers_per_group, gc.split_emb_head)
+    assert len(groups) == 20
+    assert groups[0] == [0] and groups[-1] == [37]
+    assert groups[1] == [1, 2] and groups[18] == [35, 36]
+
+
+def test_orders():
+    k = 20
+    assert O.group_order(k, 0) == list(range(k))
+    assert O.group_order(k, 1) == list(range(k))[::-1]
+    r1 = O.group_order(k, 2, seed=2401)
+    r2 = O.group_order(k, 2, seed=2401)
+    assert r1 == r2 and sorted(r1) == list(range(k)) and r1 != list(range(k))
+    assert O.group_order(k, 2, seed=7) != r1
+
+
+def test_splitmix64_published_vector():
+    # first outputs of SplitMix64 seeded with 1234567 (reference vector of the
+    # public-domain implementation by S. Vigna)
+    s = 1234567
+    outs = []
+    for _ in range(3):
+        s, z = O.splitmix64(s)
+        outs.append(z)
+    assert outs == [6457827717110365317, 3203168211198807973, 9817491932198370423]
+
+
+def test_queue_walk_equals_fixed_partition_when_m_divides_n():
+    # Algorithm 1 c-d: pop m from the head, push to the tail.
+    for n, m in [(6, 1), (6, 2), (6, 3), (34, 1), (34, 2), (12, 4)]:
+        for order in (0, 1):
+            groups = O.build_groups(n, m)
+            seq = O.group_order(len(groups), order)
+            walk = O.queue_walk(n, m, order, 3 * len(groups))
+            for t, e in enumerate(walk):
+                assert sorted(e) == groups[seq[t % len(groups)]]
+
+
+def test_random_order_fixed_across_cycles_and_active_sequence():
+    cfg, gc, oc = synth.config_tiny_fp32()
+    gc = synth.GroupCfg(layers_per_group=1, order=2, order_seed=5)
+    orc = O.HiFTOracle(cfg, gc, oc, synth.init_params(cfg, 0))
+    perm = O.group_order(6, 2, 5)
+    seq = []
+    for t in range(18):
+        seq.append(orc.active_group())
+        orc.t += 1
+    assert seq == perm * 3
+
+
+def test_delayed_lr_constant_within_cycle():
+    # last branch of Algorithm 1: the schedule moves only after all groups were updated
+    k, C, lr0 = 14, 3, 2e-5
+    lrs = [O.lr_for_cycle(lr0, 1, t // k, C) for t in range(k * C)]
+    for c in range(C):
+        chunk = lrs[c * k:(c + 1) * k]
+        assert len(set(chunk)) == 1
+    assert lrs[0] == lr0
+    assert lrs[k] == pytest.approx(lr0 * 2 / 3, rel=1e-15)
+    assert lrs[2 * k] == pytest.approx(lr0 / 3, rel=1e-15)
+    assert all(O.lr_for_cycle(lr0, 0, c, C) == lr0 for c in range(5))
+    assert O.lr_for_cycle(lr0, 1, 7, 3) == 0.0
+
+
+def test_memory_model_against_paper():
+    g = _golden()
+    z1 = g["zeta1_7b_fp32_G"]
+    # zeta1 itself: 7e9 parameters * 4 bytes in GiB
+    assert 7e9 * 4 / 2**30 == pytest.approx(z1, abs=0.005)
+    assert O.zeta_fpft(z1) == pytest.approx(g["zeta_fpft_7b_G"], abs=1e-9)
+    zh = O.zeta_hift(z1, 34)
+    assert zh == pytest.approx((34 + 3) / 34 * z1, rel=1e-15)
+    assert O.zeta_fpft(z1) - zh == pytest.approx((3 * 34 - 3) / 34 * z1, rel=1e-12)
+    # The printed worked value does not follow from the printed equations; the
+    # oracle follows the equations.  Keep the discrepancy visible:
+    assert zh == pytest.approx(28.38, abs=0.005)
+    assert abs(zh - g["zeta_hift_printed_G"]) > 2.0
+    assert g["zeta_fpft_7b_G"] - g["zeta_hift_printed_G"] == pytest.approx(g["zeta_saving_printed_G"], abs=0.005)
+    # k = 1 degenerates to full fine-tuning
+    assert O.zeta_hift(z1, 1) == pytest.approx(O.zeta_fpft(z1))
+
+
+def test_peak_trainable_fraction():
+    cfg, gc, _ = synth.config_llama_7b()
+    up = synth.count_params(cfg)
+    assert sum(up) == 6_738_415_616
+    groups = O.build_groups(cfg.n_units, 1)
+    frac = O.peak_trainable_fraction(up, groups)
+    assert frac == pytest.approx(202_383_360 / 6_738_415_616)
+    assert 0.029 < frac < 0.031
+    # names listed by the oracle agree with the synthetic tensor catalogue
+    for cfgf in (synth.config_tiny_fp32, synth.config_roberta_base, synth.config_gpt2_large, synth.config_llama_7b):
+        c = cfgf()[0]
+        cat = synth.unit_tensors(c)
+        for u in range(c.n_units):
+            assert [n for n, _, _ in cat[u]] == O.tensor_names_of_unit(c, u)
