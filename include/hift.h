@@ -1,0 +1,226 @@
+/*
+ * hift.h -- C ABI of the B200 hierarchical fine-tuning (HiFT) training step.
+ *
+ * One context = one model on one GPU.  A call to hift_step() performs one
+ * iteration of the paper's Algorithm 1: select the active group (steps c-g),
+ * full forward pass (h), move that group's optimizer state to the GPU (i),
+ * back-propagate only as far down as the group and form weight gradients only
+ * inside it (the "Backpropagation" step), update the group with the chosen
+ * optimizer, clear gradients, move the state back to host memory (k), and
+ * advance the learning-rate schedule once every full cycle of groups (final
+ * branch of Algorithm 1).  Only the active group's parameters change
+ * (Eq. 2-3: the binary mask beta_i).
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers on the context's GPU, "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer it
+ *     passes in; the library never frees or keeps them past the call.
+ *   - Everything the context allocates (device and pinned host memory) is
+ *     released by hift_destroy().
+ *   - Every function returns a hift_status (or a plain value for getters);
+ *     nothing aborts, throws, or traps on the device.
+ *   - A context is not thread-safe.  Work is issued on the CUDA stream given to
+ *     hift_create() plus copy streams the context owns.
+ *   - Row-major everywhere.  Linear weights are [out_features, in_features].
+ */
+#ifndef HIFT_H_
+#define HIFT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hift_ctx hift_ctx;
+
+typedef enum {
+  HIFT_OK = 0,
+  HIFT_ERR_CFG = 1,          /* invalid or unsupported configuration / argument      */
+  HIFT_ERR_OOM_DEVICE = 2,   /* cudaMalloc failed                                    */
+  HIFT_ERR_OOM_PINNED = 3,   /* pinned host allocation failed                        */
+  HIFT_ERR_INPUT = 4,        /* token id or label out of range, NULL pointer         */
+  HIFT_ERR_NONFINITE = 5,    /* the loss of the step was NaN/Inf (update was applied) */
+  HIFT_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up                   */
+  HIFT_ERR_CUDA = 7          /* any other CUDA runtime/driver error                  */
+} hift_status;
+
+/* Model description.  Units (the paper's "layers", Section "Hierarchical
+ * Training": the embedding is the bottom layer, the head the top layer):
+ * unit 0 = all embeddings, units 1..n_blocks = transformer blocks,
+ * unit n_blocks+1 = head (final norm + LM matrix, or classifier). */
+typedef struct {
+  int32_t arch;        /* 0 pre-LN causal decoder (GELU, learned positions)
+                          1 post-LN bidirectional encoder + classifier on token 0
+                          2 LLaMA-style (RMSNorm, RoPE, SwiGLU, no biases)          */
+  int32_t n_blocks, d_model, n_heads, d_ffn, vocab;
+  int32_t max_pos;     /* rows of the learned position table (arch 0,1)            */
+  int32_t n_classes;   /* arch 1 only                                              */
+  int32_t causal;      /* 1: attention masks keys after the query                  */
+  int32_t tie_head;    /* 1: LM head shares tok_emb; the matrix belongs to unit 0  */
+  int32_t dtype;       /* 0: fp32 params+activations; 1: bf16 with fp32 master     */
+  int32_t batch, seq;  /* fixed per context                                        */
+  double  norm_eps, rope_base;
+} hift_model_cfg;
+
+/* Grouping and order (paper: Notation paragraph; Algorithm 1 "UpdateStrategy"). */
+typedef struct {
+  int32_t layers_per_group;  /* m: consecutive units per group, last group short   */
+  int32_t split_emb_head;    /* 1: embedding | blocks in chunks of m | head        */
+  int32_t order;             /* 0 bottom2up, 1 top2down, 2 random (shuffled once)  */
+  uint64_t order_seed;       /* seed of the one-time shuffle                       */
+} hift_group_cfg;
+
+/* Optimizer P and schedule eta_t of Algorithm 1's "Require" list; state residency
+ * per its steps i and k ("MoveOptimizerState2GPU/2CPU") and the adapted mixed
+ * precision of Section "Mixing Precision" (only the active group's fp32 master
+ * is on the GPU). */
+typedef struct {
+  int32_t kind;              /* 0 AdamW, 1 AdaGrad, 2 SGD with momentum            */
+  int32_t sched;             /* 0 constant, 1 linear decay lr*(1 - cycle/total)    */
+  int32_t total_cycles;      /* horizon of the linear schedule                     */
+  int32_t offload_state;     /* 1: inactive groups' master+state in pinned host    */
+  int32_t prefetch_groups;   /* 0: one state slot, H2D issued after the forward
+                                   (the paper's order); 1: two slots, H2D issued at
+                                   step start and overlapped with the previous D2H  */
+  double lr, beta1, beta2, eps, weight_decay, momentum;
+} hift_opt_cfg;
+
+/* Build a context.  `cuda_stream` is a cudaStream_t (NULL = default stream).
+ * Parameters start as zeros; fill them with hift_set_param() or
+ * hift_init_synthetic().  Fails with HIFT_ERR_OOM_* and leaves *out NULL if the
+ * device or pinned memory cannot be had. */
+hift_status hift_create(const hift_model_cfg *model, const hift_group_cfg *groups,
+                        const hift_opt_cfg *opt, void *cuda_stream, hift_ctx **out);
+void hift_destroy(hift_ctx *ctx);
+
+/* One iteration of Algorithm 1 on the group hift_active_group() names.
+ * tokens_dev: int32 [batch, seq].  labels_dev: int32 [batch, seq] (arch 0, 2;
+ * -1 = position ignored) or int32 [batch] (arch 1).  The mean cross-entropy of
+ * the batch, computed before the update, is written to *loss_host.  Returns
+ * after the loss is on the host; state write-back may still be in flight.
+ * An out-of-range token id is clamped on the device and reported as
+ * HIFT_ERR_INPUT after the step has run. */
+hift_status hift_step(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *labels_dev,
+                      float *loss_host);
+/* Same, with the batch in host memory (validated on the host, then copied to
+ * the GPU inside the call; invalid input is rejected before anything runs). */
+hift_status hift_step_host(hift_ctx *ctx, const int32_t *tokens_host, const int32_t *labels_host,
+                           float *loss_host);
+
+int32_t hift_active_group(const hift_ctx *ctx);   /* group the NEXT hift_step trains */
+int32_t hift_num_groups(const hift_ctx *ctx);     /* k                               */
+int64_t hift_step_count(const hift_ctx *ctx);     /* t, steps taken so far           */
+double  hift_current_lr(const hift_ctx *ctx);     /* lr the NEXT step will use       */
+/* Units of group g: writes the first and last unit id (inclusive). */
+hift_status hift_group_units(const hift_ctx *ctx, int32_t g, int32_t *unit_lo, int32_t *unit_hi);
+/* Force the group trained by the next steps (depth sweeps); -1 restores the schedule. */
+hift_status hift_force_group(hift_ctx *ctx, int32_t g);
+
+/* High-water mark, in bytes, of all device memory the context holds. */
+size_t hift_peak_hbm_bytes(const hift_ctx *ctx);
+/* Bytes of pinned host memory the context holds. */
+size_t hift_pinned_host_bytes(const hift_ctx *ctx);
+
+/* ---- parameter / gradient access (tests and checkpoints) ---------------- */
+int32_t hift_num_tensors(const hift_ctx *ctx);
+/* name_out: at least 64 bytes.  A vector has rows = 1. */
+hift_status hift_tensor_info(const hift_ctx *ctx, int32_t tensor, char *name_out,
+                             int32_t *unit, int64_t *rows, int64_t *cols);
+/* fp32 master values of one tensor, host memory, `n` = rows*cols elements.
+ * set: also refreshes the bf16 model copy (round to nearest even). */
+hift_status hift_set_param(hift_ctx *ctx, int32_t tensor, const float *src_host, size_t n);
+hift_status hift_get_param(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t n);
+/* The value the forward pass reads (bf16 widened to fp32, or the fp32 itself). */
+hift_status hift_get_model_param(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t n);
+/* Optimizer state `which` (0: first moment / accumulator / momentum, 1: second moment). */
+hift_status hift_get_state(hift_ctx *ctx, int32_t tensor, int32_t which, float *dst_host, size_t n);
+/* fp32 gradient of a tensor of the group trained by the LAST step. */
+hift_status hift_get_grad(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t n);
+/* Fill every parameter on the device: matrices N(0, std^2) from a counter-based
+ * hash of (seed, element index), gains 1, biases 0; optimizer state zero. */
+hift_status hift_init_synthetic(hift_ctx *ctx, uint64_t seed, double std);
+
+/* ---- instrumentation ------------------------------------------------------ */
+/* Kernel classes for hift_profile(). */
+enum { HIFT_K_GEMM_FWD = 0, HIFT_K_GEMM_DX = 1, HIFT_K_GEMM_DW = 2, HIFT_K_ATTN_FWD = 3,
+       HIFT_K_ATTN_BWD = 4, HIFT_K_NORM = 5, HIFT_K_ELEMWISE = 6, HIFT_K_CE = 7,
+       HIFT_K_EMBED = 8, HIFT_K_OPT = 9, HIFT_K_REDUCE = 10, HIFT_K_NUM = 11 };
+/* on=1: bracket every kernel launch of the following steps with CUDA events on
+ * the launching stream and accumulate per class; on=0 stops.  Resets counters. */
+hift_status hift_profile_enable(hift_ctx *ctx, int32_t on);
+/* Accumulated since enable: launches, device milliseconds and algorithmic work
+ * (flops for GEMM/attention classes, bytes for the others). */
+hift_status hift_profile(hift_ctx *ctx, int32_t kernel_class, int64_t *launches,
+                         double *millis, double *work);
+/* Kernel launches issued by the last hift_step (all classes). */
+int64_t hift_last_step_launches(const hift_ctx *ctx);
+/* Bytes paged host->device and device->host by the last step. */
+hift_status hift_last_step_paging(const hift_ctx *ctx, size_t *h2d_bytes, size_t *d2h_bytes);
+
+/* ---- the group-local fused optimizer on caller-owned flat buffers --------
+ * One streaming pass over n elements (the update Algorithm 1 applies to the
+ * active group once "UpdateOptimizerParameter" has pointed P at theta_s).  All
+ * pointers are device pointers, 16-byte aligned.  master/grad/s0/s1 are fp32;
+ * s1 is used by AdamW only (may be NULL otherwise); param_bf16 may be NULL
+ * (fp32 configs).  tau >= 1 is the number of updates this group has had,
+ * including this one (bias correction).  Launches on `cuda_stream`, does not
+ * synchronise. */
+hift_status hift_opt_step(int32_t kind, size_t n, void *param_bf16_dev, float *master_dev,
+                          const float *grad_dev, float *s0_dev, float *s1_dev,
+                          double lr, double beta1, double beta2, double eps,
+                          double weight_decay, double momentum, int64_t tau,
+                          void *cuda_stream);
+
+/* ---- single kernels on caller-owned device buffers (per-kernel parity) ----
+ * These are the pieces of Algorithm 1's "ForwardPropagation"/"Backpropagation"
+ * steps.  dtype 0: fp32 operands, 1: bf16 operands.  All launch on `cuda_stream`
+ * and do not synchronise. */
+/* form 0: y[M,N]  = x[M,K] * w[N,K]^T (+ bias[N]);             out has operand type
+ * form 1: dx[M,K] = dy[M,N] * w[N,K];                          out has operand type
+ * form 2: dw[N,K] = dy[M,N]^T * x[M,K];                        out is fp32
+ * residual_dev (forms 0,1; optional): fp32 [M, out cols]; when given the output
+ * is fp32 too (the residual stream is kept in fp32).
+ * `path`: 0 = pick automatically, 1 = force the CUDA-core kernel, 2 = force the
+ * tcgen05 tensor-core kernel (bf16 only; HIFT_ERR_CFG if the shape is not eligible). */
+hift_status hift_k_linear(int32_t form, int32_t dtype, int32_t path, int64_t M, int64_t N, int64_t K,
+                          const void *a_dev, const void *b_dev, void *out_dev,
+                          const void *bias_dev, const float *residual_dev, void *cuda_stream);
+/* qkv[T,3d] (q|k|v column blocks, head h at columns h*d_h) -> o[T,d], lse[B,H,S] fp32. */
+hift_status hift_k_attention_fwd(int32_t dtype, int32_t batch, int32_t seq, int32_t n_heads,
+                                 int32_t d_head, int32_t causal, const void *qkv_dev, void *o_dev,
+                                 float *lse_dev, void *cuda_stream);
+/* -> dqkv[T,3d]; dsum_dev is fp32 scratch of batch*seq*n_heads elements. */
+hift_status hift_k_attention_bwd(int32_t dtype, int32_t batch, int32_t seq, int32_t n_heads,
+                                 int32_t d_head, int32_t causal, const void *qkv_dev,
+                                 const void *o_dev, const float *lse_dev, const void *do_dev,
+                                 void *dqkv_dev, float *dsum_dev, void *cuda_stream);
+/* kind 0 LayerNorm (gain, bias), 1 RMSNorm (gain).  x is the fp32 residual stream in every
+ * dtype; gain/bias/y have the operand type.  stats: fp32 [2*rows] (mean|rstd). */
+hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,
+                            const float *x_dev, const void *gain_dev, const void *bias_dev,
+                            void *y_dev, float *stats_dev, void *cuda_stream);
+/* dx = norm_bwd(dy) (+ add).  dy and gain have the operand type; x, add and dx are fp32
+ * (residual stream and its gradient).  dx may be NULL (skipped).  dgain/dbias fp32 [cols]
+ * may be NULL (skipped); partial_dev: fp32 scratch of 2*64*cols elements, needed when
+ * dgain != NULL. */
+hift_status hift_k_norm_bwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols,
+                            const void *dy_dev, const float *x_dev, const float *stats_dev,
+                            const void *gain_dev, const float *add_dev, float *dx_dev,
+                            float *dgain_dev, float *dbias_dev, float *partial_dev,
+                            void *cuda_stream);
+/* Softmax cross-entropy over rows of logits[rows, ld] (columns >= vocab are
+ * padding).  Overwrites logits with d loss / d logits.  loss_dev: 4 fp32 words,
+ * [0] = mean loss over rows with label >= 0, [1] = that row count (int32 bits),
+ * [2] = 1 (int32) if a label was >= vocab.  rowloss_dev: fp32 scratch [rows]. */
+hift_status hift_k_cross_entropy(int32_t dtype, int64_t rows, int64_t vocab, int64_t ld,
+                                 void *logits_dev, const int32_t *labels_dev, float *rowloss_dev,
+                                 float *loss_dev, void *cuda_stream);
+
+const char *hift_strerror(hift_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIFT_H_ */

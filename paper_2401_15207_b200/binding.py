@@ -1,0 +1,312 @@
+"""ctypes binding of include/hift.h: same names, argument marshalling only.
+
+torch is used for device memory (tensors whose data_ptr() is handed to the
+library) and for the CUDA stream; nothing is computed in Python.  There is no
+CPU fallback: if libhift.so is missing or no CUDA device is present the calls
+raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libhift.so")
+_lib = None
+
+KERNEL_CLASSES = ["gemm_fwd", "gemm_dx", "gemm_dw", "attn_fwd", "attn_bwd", "norm", "elementwise",
+                  "cross_entropy", "embedding", "optimizer", "reduce"]
+
+STATUS_NAMES = {0: "HIFT_OK", 1: "HIFT_ERR_CFG", 2: "HIFT_ERR_OOM_DEVICE", 3: "HIFT_ERR_OOM_PINNED",
+                4: "HIFT_ERR_INPUT", 5: "HIFT_ERR_NONFINITE", 6: "HIFT_ERR_TIMEOUT", 7: "HIFT_ERR_CUDA"}
+
+
+class HiftError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().hift_strerror(status).decode() if _lib is not None else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({msg})")
+
+
+class ModelCfgC(C.Structure):
+    _fields_ = [("arch", C.c_int32), ("n_blocks", C.c_int32), ("d_model", C.c_int32),
+                ("n_heads", C.c_int32), ("d_ffn", C.c_int32), ("vocab", C.c_int32),
+                ("max_pos", C.c_int32), ("n_classes", C.c_int32), ("causal", C.c_int32),
+                ("tie_head", C.c_int32), ("dtype", C.c_int32), ("batch", C.c_int32),
+                ("seq", C.c_int32), ("norm_eps", C.c_double), ("rope_base", C.c_double)]
+
+
+class GroupCfgC(C.Structure):
+    _fields_ = [("layers_per_group", C.c_int32), ("split_emb_head", C.c_int32),
+                ("order", C.c_int32), ("order_seed", C.c_uint64)]
+
+
+class OptCfgC(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("sched", C.c_int32), ("total_cycles", C.c_int32),
+                ("offload_state", C.c_int32), ("prefetch_groups", C.c_int32),
+                ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
+                ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double)]
+
+
+# name -> (restype, argtypes); mirrors include/hift.h one to one
+def _prototypes():
+    vp, i32, i64, f64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_double, C.c_size_t
+    pf = C.POINTER(C.c_float)
+    return {
+        "hift_strerror": (C.c_char_p, [C.c_int]),
+        "hift_create": (C.c_int, [C.POINTER(ModelCfgC), C.POINTER(GroupCfgC), C.POINTER(OptCfgC), vp, C.POINTER(vp)]),
+        "hift_destroy": (None, [vp]),
+        "hift_step": (C.c_int, [vp, vp, vp, pf]),
+        "hift_step_host": (C.c_int, [vp, vp, vp, pf]),
+        "hift_active_group": (i32, [vp]),
+        "hift_num_groups": (i32, [vp]),
+        "hift_step_count": (i64, [vp]),
+        "hift_current_lr": (f64, [vp]),
+        "hift_group_units": (C.c_int, [vp, i32, C.POINTER(i32), C.POINTER(i32)]),
+        "hift_force_group": (C.c_int, [vp, i32]),
+        "hift_peak_hbm_bytes": (sz, [vp]),
+        "hift_pinned_host_bytes": (sz, [vp]),
+        "hift_num_tensors": (i32, [vp]),
+        "hift_tensor_info": (C.c_int, [vp, i32, C.c_char_p, C.POINTER(i32), C.POINTER(i64), C.POINTER(i64)]),
+        "hift_set_param": (C.c_int, [vp, i32, vp, sz]),
+        "hift_get_param": (C.c_int, [vp, i32, vp, sz]),
+        "hift_get_model_param": (C.c_int, [vp, i32, vp, sz]),
+        "hift_get_grad": (C.c_int, [vp, i32, vp, sz]),
+        "hift_get_state": (C.c_int, [vp, i32, i32, vp, sz]),
+        "hift_init_synthetic": (C.c_int, [vp, C.c_uint64, f64]),
+        "hift_profile_enable": (C.c_int, [vp, i32]),
+        "hift_profile": (C.c_int, [vp, i32, C.POINTER(i64), C.POINTER(f64), C.POINTER(f64)]),
+        "hift_last_step_launches": (i64, [vp]),
+        "hift_last_step_paging": (C.c_int, [vp, C.POINTER(sz), C.POINTER(sz)]),
+        "hift_opt_step": (C.c_int, [i32, sz, vp, vp, vp, vp, vp, f64, f64, f64, f64, f64, f64, i64, vp]),
+        "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
+        "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
+        "hift_k_attention_bwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+        "hift_k_norm_fwd": (C.c_int, [i32, i32, i64, i64, f64, vp, vp, vp, vp, vp, vp]),
+        "hift_k_norm_bwd": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
+        "hift_k_cross_entropy": (C.c_int, [i32, i64, i64, i64, vp, vp, vp, vp, vp]),
+    }
+
+
+def load_library(path: Optional[str] = None):
+    """dlopen libhift.so and declare the prototypes of include/hift.h."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(f"{p} not found: build it with `python -m paper_2401_15207_b200.build`")
+    L = C.CDLL(p)
+    for name, (res, args) in _prototypes().items():
+        f = getattr(L, name)
+        f.restype = res
+        f.argtypes = args
+    if path is None:
+        _lib = L
+    return L
+
+
+def lib():
+    return load_library()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise HiftError(status, where)
+
+
+def _stream_ptr() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+class HiFT:
+    """One model on one GPU; mirrors hift_create / hift_step / getters."""
+
+    def __init__(self, model, groups, opt, stream: Optional[int] = None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("HiFT needs a CUDA device; there is no CPU fallback")
+        self.model, self.groups_cfg, self.opt = model, groups, opt
+        m = ModelCfgC(model.arch, model.n_blocks, model.d_model, model.n_heads, model.d_ffn,
+                      model.vocab, model.max_pos, model.n_classes, model.causal, model.tie_head,
+                      model.dtype, model.batch, model.seq, model.norm_eps, model.rope_base)
+        g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed)
+        o = OptCfgC(opt.kind, opt.sched, opt.total_cycles, opt.offload_state, opt.prefetch_groups,
+                    opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
+        self._h = C.c_void_p()
+        self._stream = _stream_ptr() if stream is None else stream
+        _check(lib().hift_create(C.byref(m), C.byref(g), C.byref(o), self._stream, C.byref(self._h)), "hift_create")
+        self._names: Dict[str, int] = {}
+        self._info: List[Tuple[str, int, int, int]] = []
+        buf = C.create_string_buffer(64)
+        for i in range(lib().hift_num_tensors(self._h)):
+            u, r, c = C.c_int32(), C.c_int64(), C.c_int64()
+            _check(lib().hift_tensor_info(self._h, i, buf, C.byref(u), C.byref(r), C.byref(c)), "hift_tensor_info")
+            name = buf.value.decode()
+            self._names[name] = i
+            self._info.append((name, u.value, r.value, c.value))
+
+    # -- lifetime
+    def close(self):
+        if self._h:
+            lib().hift_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the step
+    def step(self, tokens, labels) -> float:
+        """tokens/labels: int32 CUDA tensors.  Returns the loss (before the update)."""
+        loss = C.c_float()
+        st = lib().hift_step(self._h, tokens.data_ptr(), labels.data_ptr(), C.byref(loss))
+        _check(st, "hift_step")
+        return loss.value
+
+    def step_host(self, tokens: np.ndarray, labels: np.ndarray) -> float:
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        labels = np.ascontiguousarray(labels, dtype=np.int32)
+        loss = C.c_float()
+        st = lib().hift_step_host(self._h, tokens.ctypes.data, labels.ctypes.data, C.byref(loss))
+        _check(st, "hift_step_host")
+        return loss.value
+
+    # -- getters
+    def active_group(self) -> int:
+        return lib().hift_active_group(self._h)
+
+    def num_groups(self) -> int:
+        return lib().hift_num_groups(self._h)
+
+    def step_count(self) -> int:
+        return lib().hift_step_count(self._h)
+
+    def current_lr(self) -> float:
+        return lib().hift_current_lr(self._h)
+
+    def group_units(self, g: int) -> Tuple[int, int]:
+        lo, hi = C.c_int32(), C.c_int32()
+        _check(lib().hift_group_units(self._h, g, C.byref(lo), C.byref(hi)), "hift_group_units")
+        return lo.value, hi.value
+
+    def force_group(self, g: int):
+        _check(lib().hift_force_group(self._h, g), "hift_force_group")
+
+    def peak_hbm_bytes(self) -> int:
+        return lib().hift_peak_hbm_bytes(self._h)
+
+    def pinned_host_bytes(self) -> int:
+        return lib().hift_pinned_host_bytes(self._h)
+
+    def tensor_names(self) -> List[str]:
+        return [n for n, _, _, _ in self._info]
+
+    def tensor_info(self, name: str) -> Tuple[int, Tuple[int, int]]:
+        n, u, r, c = self._info[self._names[name]]
+        return u, (r, c)
+
+    def _numel(self, name: str) -> int:
+        _, _, r, c = self._info[self._names[name]]
+        return r * c
+
+    def set_param(self, name: str, value: np.ndarray):
+        a = np.ascontiguousarray(value, dtype=np.float32)
+        _check(lib().hift_set_param(self._h, self._names[name], a.ctypes.data, a.size), "hift_set_param")
+
+    def set_params(self, params: Dict[str, np.ndarray]):
+        for k, v in params.items():
+            self.set_param(k, v)
+
+    def _get(self, fn, where: str, name: str, *extra) -> np.ndarray:
+        n = self._numel(name)
+        out = np.empty(n, dtype=np.float32)
+        _check(fn(self._h, self._names[name], *extra, out.ctypes.data, n), where)
+        _, _, r, c = self._info[self._names[name]]
+        return out.reshape(r, c)
+
+    def get_param(self, name: str) -> np.ndarray:
+        return self._get(lib().hift_get_param, "hift_get_param", name)
+
+    def get_model_param(self, name: str) -> np.ndarray:
+        return self._get(lib().hift_get_model_param, "hift_get_model_param", name)
+
+    def get_grad(self, name: str) -> np.ndarray:
+        return self._get(lib().hift_get_grad, "hift_get_grad", name)
+
+    def get_state(self, name: str, which: int) -> np.ndarray:
+        return self._get(lib().hift_get_state, "hift_get_state", name, which)
+
+    def init_synthetic(self, seed: int, std: float = 0.02):
+        _check(lib().hift_init_synthetic(self._h, seed, std), "hift_init_synthetic")
+
+    # -- instrumentation
+    def profile_enable(self, on: bool):
+        _check(lib().hift_profile_enable(self._h, 1 if on else 0), "hift_profile_enable")
+
+    def profile(self) -> Dict[str, Dict[str, float]]:
+        out = {}
+        for i, name in enumerate(KERNEL_CLASSES):
+            n, ms, w = C.c_int64(), C.c_double(), C.c_double()
+            _check(lib().hift_profile(self._h, i, C.byref(n), C.byref(ms), C.byref(w)), "hift_profile")
+            out[name] = {"launches": n.value, "ms": ms.value, "work": w.value}
+        return out
+
+    def last_step_launches(self) -> int:
+        return lib().hift_last_step_launches(self._h)
+
+    def last_step_paging(self) -> Tuple[int, int]:
+        a, b = C.c_size_t(), C.c_size_t()
+        _check(lib().hift_last_step_paging(self._h, C.byref(a), C.byref(b)), "hift_last_step_paging")
+        return a.value, b.value
+
+
+# ---------------------------------------------------------------- free functions
+def _st(stream):
+    return _stream_ptr() if stream is None else stream
+
+
+def opt_step(kind, n, param_bf16, master, grad, s0, s1, lr, beta1=0.9, beta2=0.999, eps=1e-8,
+             weight_decay=0.0, momentum=0.9, tau=1, stream=None):
+    _check(lib().hift_opt_step(kind, n, _ptr(param_bf16), _ptr(master), _ptr(grad), _ptr(s0), _ptr(s1),
+                               lr, beta1, beta2, eps, weight_decay, momentum, tau, _st(stream)), "hift_opt_step")
+
+
+def k_linear(form, dtype, M, N, K, a, b, out, bias=None, residual=None, path=0, stream=None):
+    _check(lib().hift_k_linear(form, dtype, path, M, N, K, _ptr(a), _ptr(b), _ptr(out), _ptr(bias),
+                               _ptr(residual), _st(stream)), "hift_k_linear")
+
+
+def k_attention_fwd(dtype, B, S, H, dh, causal, qkv, o, lse, stream=None):
+    _check(lib().hift_k_attention_fwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _st(stream)),
+           "hift_k_attention_fwd")
+
+
+def k_attention_bwd(dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, stream=None):
+    _check(lib().hift_k_attention_bwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout),
+                                      _ptr(dqkv), _ptr(dsum), _st(stream)), "hift_k_attention_bwd")
+
+
+def k_norm_fwd(dtype, kind, rows, cols, eps, x, gain, bias, y, stats, stream=None):
+    _check(lib().hift_k_norm_fwd(dtype, kind, rows, cols, eps, _ptr(x), _ptr(gain), _ptr(bias), _ptr(y),
+                                 _ptr(stats), _st(stream)), "hift_k_norm_fwd")
+
+
+def k_norm_bwd(dtype, kind, rows, cols, dy, x, stats, gain, add, dx, dgain, dbias, partial, stream=None):
+    _check(lib().hift_k_norm_bwd(dtype, kind, rows, cols, _ptr(dy), _ptr(x), _ptr(stats), _ptr(gain), _ptr(add),
+                                 _ptr(dx), _ptr(dgain), _ptr(dbias), _ptr(partial), _st(stream)), "hift_k_norm_bwd")
+
+
+def k_cross_entropy(dtype, rows, vocab, ld, logits, labels, rowloss, loss, stream=None):
+    _check(lib().hift_k_cross_entropy(dtype, rows, vocab, ld, _ptr(logits), _ptr(labels), _ptr(rowloss),
+                                      _ptr(loss), _st(stream)), "hift_k_cross_entropy")

@@ -1,0 +1,18 @@
+// Tensor-core (tcgen05 / TMEM / TMA) bf16 GEMM: host interface.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "gemm_args.h"
+
+namespace hift {
+
+// Resolves the driver entry point used to encode TMA descriptors and opts the kernels into
+// large dynamic shared memory.  0 on success; anything else means the tensor-core path is
+// unavailable and gemm_tc_eligible() answers false.
+int gemm_tc_init();
+// True when the operands are bf16 in one of the three supported major-ness combinations,
+// 16-byte aligned with 16-byte-multiple leading dimensions.
+bool gemm_tc_eligible(const GemmArgs& g);
+cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g);
+
+}  // namespace hift

@@ -1,0 +1,1090 @@
+// Engine and C entry points of the hierarchical fine-tuning step (see include/hift.h).
+//
+// One hift_step = one iteration of the paper's Algorithm 1:
+//   select group (c-g)  ->  forward (h)  ->  state to GPU (i)  ->  backward truncated at the
+//   group + update + clear gradients  ->  state to host (k)  ->  delayed learning rate.
+// Activations below the group's lowest unit are not kept (two ping-pong buffers); above it only
+// what activation gradients need is kept; inside it the GEMM inputs are kept too.
+#include "hift.h"
+
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <string>
+#include <vector>
+
+#include "gemm_tc.h"
+#include "launchers.cuh"
+
+using namespace hift;
+
+namespace {
+
+constexpr size_t kAlignElems = 128;   // every tensor starts on a multiple of 128 elements
+
+// Per-block activation slots.  Residual-stream tensors are fp32 in every configuration;
+// GEMM operands have the parameter type (bf16 or fp32).
+//   pre-norm blocks:  XIN x (stream) | H1 norm1(x) | QKV | O | LSE | X2 x + attn (stream) |
+//                     H2 norm2(x2) | A pre-activation | U activation output
+//   post-LN blocks:   XIN x (stream) + XINA operand copy | QKV | O | LSE | X2 y = x + attn (stream) |
+//                     H2 x1 = LN1(y) operand copy + H2R stream copy | A | U | Z z = x1 + ffn (stream)
+enum Slot { S_XIN = 0, S_XINA, S_H1, S_QKV, S_O, S_LSE, S_X2, S_ST1, S_H2, S_H2R, S_A, S_U, S_Z, S_ST2, S_NUM };
+
+struct TensorRec {
+  char name[64];
+  int unit;
+  int64_t rows, cols;
+  size_t numel, off;
+  int init_kind;   // 0 normal, 1 ones, 2 zeros
+};
+struct GroupRec {
+  int unit_lo, unit_hi;
+  size_t off, numel;      // span in the flat parameter buffer (padded)
+  int64_t tau;            // updates so far
+  char* blob;             // pinned host: [master][s0][s1]
+  size_t blob_bytes;
+};
+struct BlockIdx {          // tensor indices of one block, -1 if absent
+  int n1_g, n1_b, w_qkv, b_qkv, w_o, b_o, n2_g, n2_b, w_fc1, b_fc1, w_fc2, b_fc2;
+};
+struct ProfRec { int cls; cudaEvent_t e0, e1; double work; };
+
+}  // namespace
+
+struct hift_ctx {
+  hift_model_cfg m;
+  hift_group_cfg gc;
+  hift_opt_cfg oc;
+  cudaStream_t st = nullptr, st_h2d = nullptr, st_d2h = nullptr;
+  int es = 2;                       // bytes per parameter / GEMM-operand element
+  int L = 0, d = 0, f = 0, fa = 0, H = 0, dh = 0, T = 0, B = 0, S = 0, V = 0, Vp = 0;
+  int n_state = 2;
+  bool mixed = true, offload = false;
+  std::vector<TensorRec> tens;
+  std::vector<std::vector<int>> unit_tens;
+  std::vector<GroupRec> groups;
+  std::vector<int> order;
+  std::vector<BlockIdx> bidx;
+  int t_tok = -1, t_pos = -1, t_eg = -1, t_eb = -1, t_fg = -1, t_fb = -1, t_wh = -1, t_wc = -1, t_bc = -1;
+  size_t total = 0, max_group = 0;
+  int64_t t = 0;
+  int forced = -1, last_group = -1;
+
+  // device memory
+  std::vector<void*> dev_allocs;
+  size_t dev_bytes = 0, pinned_bytes = 0;
+  char* params = nullptr;           // [total] of element type
+  float* master_all = nullptr;      // non-offload mixed mode
+  float* s0_all = nullptr; float* s1_all = nullptr;
+  char* slot[2] = {nullptr, nullptr};   // offload staging: [master][s0][s1] per slot
+  int n_slots = 1;
+  float* grad = nullptr;            // [max_group]
+  char* arena = nullptr; size_t arena_cap = 0, arena_off = 0, arena_fixed = 0;
+  cudaEvent_t ev_h2d[2], ev_opt[2], ev_d2h[2], ev_fwd;
+  bool events_made = false;
+  bool d2h_pending[2] = {false, false};
+  // fixed work buffers
+  int32_t *tok_dev = nullptr, *lab_dev = nullptr;
+  float *dxa = nullptr, *dxb = nullptr;             // residual-stream gradients (fp32)
+  char *dxa_a = nullptr, *dxb_a = nullptr;          // the same, rounded once to the operand type
+  char *dt1 = nullptr, *dqkv = nullptr, *dbig = nullptr, *dsw = nullptr;
+  float *x_final = nullptr, *emb_e = nullptr, *pp[2] = {nullptr, nullptr};
+  char *x_final_a = nullptr, *ppa[2] = {nullptr, nullptr};
+  char *xf = nullptr, *logits = nullptr;
+  float *stf = nullptr, *st_e = nullptr, *dsum = nullptr, *partial = nullptr, *rowloss = nullptr, *rope_cs = nullptr;
+  float* scal = nullptr;            // device: [0] loss, [1] nvalid(int), [2] bad(int)
+  float* scal_host = nullptr;       // pinned mirror
+  std::vector<std::vector<char*>> slots;   // [block][slot]; entry L holds the scratch copies
+  // instrumentation
+  bool prof_on = false;
+  std::vector<cudaEvent_t> ev_pool; size_t ev_used = 0;
+  std::vector<ProfRec> prof_recs;
+  int64_t prof_launches[HIFT_K_NUM]; double prof_ms[HIFT_K_NUM], prof_work[HIFT_K_NUM];
+  int64_t step_launches = 0;
+  size_t step_h2d = 0, step_d2h = 0;
+  cudaError_t first_err = cudaSuccess;
+
+  // ---- helpers
+  void note(cudaError_t e) { if (e != cudaSuccess && first_err == cudaSuccess) first_err = e; }
+  void* P(int ti) const { return params + tens[ti].off * es; }
+  void* Pn(int ti) const { return ti < 0 ? nullptr : P(ti); }
+  float* G(int ti) const { return grad + (tens[ti].off - groups[last_group].off); }
+  void pre(int cls, double work) {
+    ++step_launches;
+    if (!prof_on) return;
+    if (ev_used + 2 > ev_pool.size()) {
+      for (int i = 0; i < 256; ++i) { cudaEvent_t e; note(cudaEventCreate(&e)); ev_pool.push_back(e); }
+    }
+    ProfRec r{cls, ev_pool[ev_used], ev_pool[ev_used + 1], work};
+    ev_used += 2;
+    note(cudaEventRecord(r.e0, st));
+    prof_recs.push_back(r);
+  }
+  void post() {
+    note(cudaGetLastError());
+    if (prof_on) note(cudaEventRecord(prof_recs.back().e1, st));
+  }
+  void prof_collect() {
+    for (auto& r : prof_recs) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess) {
+        prof_launches[r.cls]++; prof_ms[r.cls] += ms; prof_work[r.cls] += r.work;
+      }
+    }
+    prof_recs.clear();
+    ev_used = 0;
+  }
+};
+
+#define LAUNCH(cls, work, ...) do { c->pre(cls, work); __VA_ARGS__; c->post(); } while (0)
+
+namespace {
+
+// ------------------------------------------------------------------ schedule (host, integers)
+// SplitMix64 (Steele, Lea, Flood 2014): the one-time shuffle of the "random" strategy.
+uint64_t splitmix64_next(uint64_t& s) {
+  s += 0x9E3779B97F4A7C15ull;
+  uint64_t z = s;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+std::vector<int> make_order(int k, int order, uint64_t seed) {
+  std::vector<int> o(k);
+  for (int i = 0; i < k; ++i) o[i] = i;
+  if (order == 1) std::reverse(o.begin(), o.end());
+  if (order == 2) {
+    uint64_t s = seed;
+    for (int i = k - 1; i > 0; --i) {
+      const int j = (int)(splitmix64_next(s) % (uint64_t)(i + 1));
+      std::swap(o[i], o[j]);
+    }
+  }
+  return o;
+}
+double lr_for_cycle(const hift_opt_cfg& oc, int64_t cycle) {
+  if (oc.sched == 0) return oc.lr;
+  const double fct = 1.0 - (double)cycle / (double)oc.total_cycles;
+  return oc.lr * (fct > 0.0 ? fct : 0.0);
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int add_tensor(hift_ctx* c, int unit, const std::string& name, int64_t rows, int64_t cols, int kind) {
+  TensorRec r;
+  memset(&r, 0, sizeof(r));
+  snprintf(r.name, sizeof(r.name), "%s", name.c_str());
+  r.unit = unit; r.rows = rows; r.cols = cols; r.numel = (size_t)rows * cols; r.init_kind = kind;
+  r.off = c->total;
+  c->total = align_up(c->total + r.numel, kAlignElems);
+  c->tens.push_back(r);
+  c->unit_tens[unit].push_back((int)c->tens.size() - 1);
+  return (int)c->tens.size() - 1;
+}
+
+void build_layout(hift_ctx* c) {
+  const hift_model_cfg& m = c->m;
+  const int L = m.n_blocks, d = m.d_model, f = m.d_ffn, V = m.vocab;
+  c->unit_tens.assign(L + 2, {});
+  c->t_tok = add_tensor(c, 0, "tok_emb", V, d, 0);
+  if (m.arch != 2) c->t_pos = add_tensor(c, 0, "pos_emb", m.max_pos, d, 0);
+  if (m.arch == 1) {
+    c->t_eg = add_tensor(c, 0, "emb_ln_g", 1, d, 1);
+    c->t_eb = add_tensor(c, 0, "emb_ln_b", 1, d, 2);
+  }
+  c->bidx.resize(L);
+  for (int i = 0; i < L; ++i) {
+    const std::string p = "b" + std::to_string(i) + ".";
+    BlockIdx& b = c->bidx[i];
+    const int u = i + 1;
+    if (m.arch == 2) {
+      b.n1_g = add_tensor(c, u, p + "rms1_g", 1, d, 1); b.n1_b = -1;
+      b.w_qkv = add_tensor(c, u, p + "w_qkv", 3 * d, d, 0); b.b_qkv = -1;
+      b.w_o = add_tensor(c, u, p + "w_o", d, d, 0); b.b_o = -1;
+      b.n2_g = add_tensor(c, u, p + "rms2_g", 1, d, 1); b.n2_b = -1;
+      b.w_fc1 = add_tensor(c, u, p + "w_gu", 2 * f, d, 0); b.b_fc1 = -1;
+      b.w_fc2 = add_tensor(c, u, p + "w_down", d, f, 0); b.b_fc2 = -1;
+    } else {
+      b.n1_g = add_tensor(c, u, p + "ln1_g", 1, d, 1); b.n1_b = add_tensor(c, u, p + "ln1_b", 1, d, 2);
+      b.w_qkv = add_tensor(c, u, p + "w_qkv", 3 * d, d, 0); b.b_qkv = add_tensor(c, u, p + "b_qkv", 1, 3 * d, 2);
+      b.w_o = add_tensor(c, u, p + "w_o", d, d, 0); b.b_o = add_tensor(c, u, p + "b_o", 1, d, 2);
+      b.n2_g = add_tensor(c, u, p + "ln2_g", 1, d, 1); b.n2_b = add_tensor(c, u, p + "ln2_b", 1, d, 2);
+      b.w_fc1 = add_tensor(c, u, p + "w_fc1", f, d, 0); b.b_fc1 = add_tensor(c, u, p + "b_fc1", 1, f, 2);
+      b.w_fc2 = add_tensor(c, u, p + "w_fc2", d, f, 0); b.b_fc2 = add_tensor(c, u, p + "b_fc2", 1, d, 2);
+    }
+  }
+  const int hu = L + 1;
+  if (m.arch == 1) {
+    c->t_wc = add_tensor(c, hu, "w_cls", m.n_classes, d, 0);
+    c->t_bc = add_tensor(c, hu, "b_cls", 1, m.n_classes, 2);
+  } else {
+    if (m.arch == 2) c->t_fg = add_tensor(c, hu, "rmsf_g", 1, d, 1);
+    else { c->t_fg = add_tensor(c, hu, "lnf_g", 1, d, 1); c->t_fb = add_tensor(c, hu, "lnf_b", 1, d, 2); }
+    if (!m.tie_head) c->t_wh = add_tensor(c, hu, "w_head", V, d, 0);
+  }
+  // groups: consecutive chunks of m units (paper, Notation), or embedding | chunks | head
+  const int n = L + 2, mm = c->gc.layers_per_group;
+  std::vector<std::pair<int, int>> spans;
+  if (c->gc.split_emb_head) {
+    spans.push_back({0, 0});
+    for (int u = 1; u <= L; u += mm) spans.push_back({u, std::min(u + mm - 1, L)});
+    spans.push_back({n - 1, n - 1});
+  } else {
+    for (int u = 0; u < n; u += mm) spans.push_back({u, std::min(u + mm - 1, n - 1)});
+  }
+  for (auto& sp : spans) {
+    GroupRec g;
+    memset(&g, 0, sizeof(g));
+    g.unit_lo = sp.first; g.unit_hi = sp.second;
+    const int t_first = c->unit_tens[sp.first].front();
+    const int t_last = c->unit_tens[sp.second].back();
+    g.off = c->tens[t_first].off;
+    g.numel = align_up(c->tens[t_last].off + c->tens[t_last].numel, kAlignElems) - g.off;
+    c->max_group = std::max(c->max_group, g.numel);
+    c->groups.push_back(g);
+  }
+  c->order = make_order((int)c->groups.size(), c->gc.order, c->gc.order_seed);
+}
+
+hift_status dev_alloc(hift_ctx* c, void** p, size_t bytes) {
+  *p = nullptr;
+  if (bytes == 0) bytes = 256;
+  cudaError_t e = cudaMalloc(p, bytes);
+  if (e != cudaSuccess) { cudaGetLastError(); return HIFT_ERR_OOM_DEVICE; }
+  c->dev_allocs.push_back(*p);
+  c->dev_bytes += bytes;
+  return HIFT_OK;
+}
+
+char* arena_take(hift_ctx* c, size_t bytes) {
+  const size_t o = c->arena_off;
+  c->arena_off = align_up(o + bytes, 256);
+  return c->arena ? c->arena + o : (char*)(uintptr_t)o;
+}
+
+// Lowest level at which a slot must outlive the forward pass: 1 = activation gradients need
+// it, 2 = only weight gradients need it, 3 = never (forward scratch), 99 = unused by the arch.
+int slot_min_level(int arch, int s) {
+  if (arch == 1) {
+    switch (s) {
+      case S_XIN: return 3; case S_XINA: return 2; case S_H1: return 99; case S_QKV: return 1;
+      case S_O: return 1; case S_LSE: return 1; case S_X2: return 1; case S_ST1: return 1;
+      case S_H2: return 2; case S_H2R: return 3; case S_A: return 1; case S_U: return 2;
+      case S_Z: return 1; case S_ST2: return 1;
+    }
+  } else {
+    switch (s) {
+      case S_XIN: return 1; case S_XINA: return 99; case S_H1: return 2; case S_QKV: return 1;
+      case S_O: return 1; case S_LSE: return 1; case S_X2: return 1; case S_ST1: return 1;
+      case S_H2: return 2; case S_H2R: return 99; case S_A: return 1; case S_U: return 2;
+      case S_Z: return 99; case S_ST2: return 1;
+    }
+  }
+  return 99;
+}
+size_t slot_bytes(const hift_ctx* c, int s) {
+  const size_t T = c->T, d = c->d, es = c->es;
+  switch (s) {
+    case S_XIN: case S_X2: case S_Z: case S_H2R: return T * d * sizeof(float);
+    case S_XINA: case S_H1: case S_O: case S_H2: return T * d * es;
+    case S_QKV: return T * 3 * d * es;
+    case S_A: return T * (size_t)c->fa * es;
+    case S_U: return T * (size_t)c->f * es;
+    case S_LSE: return (size_t)c->B * c->H * c->S * sizeof(float);
+    case S_ST1: case S_ST2: return 2 * T * sizeof(float);
+  }
+  return 0;
+}
+int level_of_block(const hift_ctx* c, int g, int i) {
+  const int u = i + 1;
+  if (u < c->groups[g].unit_lo) return 0;
+  return u <= c->groups[g].unit_hi ? 2 : 1;
+}
+// Assign the per-block activation slots for a step that trains group g.  Returns the arena
+// bytes used.  With assign == false only sizes are computed.
+size_t plan_slots(hift_ctx* c, int g, bool assign) {
+  c->arena_off = c->arena_fixed;
+  for (int i = 0; i < c->L; ++i) {
+    const int lvl = level_of_block(c, g, i);
+    for (int s = 0; s < S_NUM; ++s) {
+      const int need = slot_min_level(c->m.arch, s);
+      if (need == 99) { if (assign) c->slots[i][s] = nullptr; continue; }
+      if (lvl >= need) {
+        char* p = arena_take(c, slot_bytes(c, s));
+        if (assign) c->slots[i][s] = p;
+      } else if (assign) {
+        c->slots[i][s] = (s == S_XIN) ? (char*)c->pp[i & 1] : (s == S_XINA) ? c->ppa[i & 1] : c->slots[c->L][s];
+      }
+    }
+  }
+  return c->arena_off;
+}
+
+// ------------------------------------------------------------------ thin launch helpers
+void gemm(hift_ctx* c, int cls, int M, int N, int K, const void* a, int64_t sam, int64_t sak,
+          const void* b, int64_t sbk, int64_t sbn, void* out, int64_t ldc, const void* bias,
+          const float* residual, int64_t ldr, bool out_f32) {
+  GemmArgs g{M, N, K, a, sam, sak, b, sbk, sbn, out, ldc, bias, residual, ldr, out_f32};
+  const double work = 2.0 * M * (double)N * K;
+  if (c->mixed && gemm_tc_eligible(g)) {
+    LAUNCH(cls, work, c->note(gemm_tc_launch(c->st, g)));
+    return;
+  }
+  LAUNCH(cls, work, launch_gemm_simt(c->st, c->mixed ? 1 : 0, g));
+}
+// y[M,N] = x[M,K] w[N,K]^T + bias (+ residual).  to_stream: the output (and the residual) is
+// the fp32 residual stream.
+void linear_fwd(hift_ctx* c, int M, int N, int K, const void* x, int64_t ldx, const void* w,
+                void* y, int64_t ldy, const void* bias, const float* res, int64_t ldr, bool to_stream) {
+  gemm(c, HIFT_K_GEMM_FWD, M, N, K, x, ldx, 1, w, 1, K, y, ldy, bias, res, ldr, to_stream);
+}
+// dx[M,K] = dy[M,N] w[N,K] (+ residual)
+void linear_dx(hift_ctx* c, int M, int N, int K, const void* dy, int64_t ldy, const void* w,
+               void* dx, int64_t ldx, const float* res, int64_t ldr, bool to_stream) {
+  gemm(c, HIFT_K_GEMM_DX, M, K, N, dy, ldy, 1, w, K, 1, dx, ldx, nullptr, res, ldr, to_stream);
+}
+// dw[N,K] = dy[M,N]^T x[M,K]   (fp32 out)
+void linear_dw(hift_ctx* c, int M, int N, int K, const void* dy, int64_t ldy, const void* x,
+               int64_t ldx, float* dw) {
+  gemm(c, HIFT_K_GEMM_DW, N, K, M, dy, 1, ldy, x, ldx, 1, dw, K, nullptr, nullptr, 0, true);
+}
+void norm_fwd(hift_ctx* c, const float* x, int tg, int tb, void* y_a, float* y_r, float* stats) {
+  const int kind = c->m.arch == 2 ? 1 : 0;
+  LAUNCH(HIFT_K_NORM, (double)c->T * c->d * (4 + c->es + (y_r ? 4 : 0)),
+         launch_norm_fwd(c->st, c->mixed, kind, c->T, c->d, (float)c->m.norm_eps, x, c->P(tg),
+                         c->Pn(tb), y_a, y_r, stats));
+}
+void norm_bwd_dx(hift_ctx* c, const void* dy, bool dy_f32, const float* x, const float* stats, int tg,
+                 const float* add, float* dx_r, void* dx_a) {
+  const int kind = c->m.arch == 2 ? 1 : 0;
+  const double bytes = (double)c->T * c->d * ((dy_f32 ? 4 : c->es) + 4 + (add ? 4 : 0) + 4 + (dx_a ? c->es : 0));
+  LAUNCH(HIFT_K_NORM, bytes,
+         launch_norm_bwd_dx(c->st, c->mixed, kind, dy_f32, c->T, c->d, dy, x, stats, c->P(tg), add, dx_r, dx_a));
+}
+void norm_bwd_params(hift_ctx* c, const void* dy, bool dy_f32, const float* x, const float* stats, int tg, int tb) {
+  const int mode = c->m.arch == 2 ? 2 : 1;
+  LAUNCH(HIFT_K_REDUCE, (double)c->T * c->d * ((dy_f32 ? 4 : c->es) + 4),
+         launch_colreduce(c->st, c->mixed && !dy_f32, mode, c->T, c->d, dy, c->d, x, stats, c->partial,
+                          c->G(tg), tb >= 0 ? c->G(tb) : nullptr));
+  ++c->step_launches;   // two kernels per call
+}
+void bias_grad(hift_ctx* c, const void* dy, bool dy_f32, int64_t rows, int cols, int64_t ld, int tb) {
+  if (tb < 0) return;
+  LAUNCH(HIFT_K_REDUCE, (double)rows * cols * (dy_f32 ? 4 : c->es),
+         launch_colreduce(c->st, c->mixed && !dy_f32, 0, rows, cols, dy, ld, nullptr, nullptr, c->partial,
+                          c->G(tb), nullptr));
+  ++c->step_launches;
+}
+void attn_fwd(hift_ctx* c, const void* qkv, void* o, float* lse) {
+  const double work = 4.0 * c->B * c->H * (double)c->S * c->S * c->dh * (c->m.causal ? 0.5 : 1.0);
+  LAUNCH(HIFT_K_ATTN_FWD, work,
+         launch_attention_fwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse));
+}
+void attn_bwd(hift_ctx* c, const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv) {
+  const double work = 10.0 * c->B * c->H * (double)c->S * c->S * c->dh * (c->m.causal ? 0.5 : 1.0);
+  LAUNCH(HIFT_K_ATTN_BWD, work,
+         launch_attention_bwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse,
+                              dout, dqkv, c->dsum));
+  ++c->step_launches;
+}
+void rope(hift_ctx* c, void* qkv, float sign) {
+  const size_t n = (size_t)c->T * c->H * (c->dh / 2);
+  LAUNCH(HIFT_K_ELEMWISE, 8.0 * n * c->es,
+         if (c->mixed) rope_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>((bf16*)qkv, c->rope_cs, c->T, c->S, c->H, c->dh, sign);
+         else rope_kernel<float><<<grid_for(n, 256), 256, 0, c->st>>>((float*)qkv, c->rope_cs, c->T, c->S, c->H, c->dh, sign));
+}
+void act_fwd(hift_ctx* c, const void* a, void* u) {
+  const size_t n = (size_t)c->T * c->f;
+  if (c->m.arch == 2) {
+    LAUNCH(HIFT_K_ELEMWISE, 3.0 * n * c->es,
+           if (c->mixed) swiglu_fwd_kernel<bf16><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const bf16*)a, (bf16*)u, c->T, c->f);
+           else swiglu_fwd_kernel<float><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const float*)a, (float*)u, c->T, c->f));
+  } else {
+    LAUNCH(HIFT_K_ELEMWISE, 2.0 * n * c->es,
+           if (c->mixed) gelu_fwd_kernel<bf16><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const bf16*)a, (bf16*)u, n / 8);
+           else gelu_fwd_kernel<float><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const float*)a, (float*)u, n / 8));
+  }
+}
+// GELU: du (in c->dbig, [T,f]) *= gelu'(a) in place.
+// SwiGLU: ds (in c->dsw, [T,f]) -> dgu in c->dbig [T,2f].
+void act_bwd(hift_ctx* c, const void* a) {
+  const size_t n = (size_t)c->T * c->f;
+  if (c->m.arch == 2) {
+    LAUNCH(HIFT_K_ELEMWISE, 5.0 * n * c->es,
+           if (c->mixed) swiglu_bwd_kernel<bf16><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const bf16*)c->dsw, (const bf16*)a, (bf16*)c->dbig, c->T, c->f);
+           else swiglu_bwd_kernel<float><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const float*)c->dsw, (const float*)a, (float*)c->dbig, c->T, c->f));
+  } else {
+    LAUNCH(HIFT_K_ELEMWISE, 3.0 * n * c->es,
+           if (c->mixed) gelu_bwd_kernel<bf16><<<grid_for(n / 8, 256), 256, 0, c->st>>>((bf16*)c->dbig, (const bf16*)a, n / 8);
+           else gelu_bwd_kernel<float><<<grid_for(n / 8, 256), 256, 0, c->st>>>((float*)c->dbig, (const float*)a, n / 8));
+  }
+}
+
+// ------------------------------------------------------------------ forward
+// x_r / x_a: the block input on the residual stream and (post-LN only) its operand copy.
+void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float* xo_r, char* xo_a) {
+  const BlockIdx& b = c->bidx[i];
+  std::vector<char*>& s = c->slots[i];
+  const int T = c->T, d = c->d, f = c->f, fa = c->fa;
+  float* x2 = (float*)s[S_X2];
+  if (c->m.arch == 1) {
+    float* x1r = (float*)s[S_H2R];
+    float* z = (float*)s[S_Z];
+    linear_fwd(c, T, 3 * d, d, x_a, d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
+    attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
+    linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);             // y
+    norm_fwd(c, x2, b.n1_g, b.n1_b, s[S_H2], x1r, (float*)s[S_ST1]);                                 // x1
+    linear_fwd(c, T, f, d, s[S_H2], d, c->P(b.w_fc1), s[S_A], f, c->Pn(b.b_fc1), nullptr, 0, false);
+    act_fwd(c, s[S_A], s[S_U]);
+    linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), z, d, c->Pn(b.b_fc2), x1r, d, true);           // z
+    norm_fwd(c, z, b.n2_g, b.n2_b, xo_a, xo_r, (float*)s[S_ST2]);
+    return;
+  }
+  norm_fwd(c, x_r, b.n1_g, b.n1_b, s[S_H1], nullptr, (float*)s[S_ST1]);
+  linear_fwd(c, T, 3 * d, d, s[S_H1], d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
+  if (c->m.arch == 2) rope(c, s[S_QKV], 1.0f);
+  attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
+  linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);
+  norm_fwd(c, x2, b.n2_g, b.n2_b, s[S_H2], nullptr, (float*)s[S_ST2]);
+  linear_fwd(c, T, fa, d, s[S_H2], d, c->P(b.w_fc1), s[S_A], fa, c->Pn(b.b_fc1), nullptr, 0, false);
+  act_fwd(c, s[S_A], s[S_U]);
+  linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
+}
+
+// ------------------------------------------------------------------ backward
+// On entry c->dxa (fp32; pre-norm blocks also c->dxa_a) holds the gradient of the block output;
+// on exit (need_dx) the gradient of the block input, in the same buffers.
+void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool on, bool need_dx) {
+  const BlockIdx& b = c->bidx[i];
+  std::vector<char*>& s = c->slots[i];
+  const int T = c->T, d = c->d, f = c->f, fa = c->fa;
+  char* dact_in = c->m.arch == 2 ? c->dsw : c->dbig;    // gradient w.r.t. the activation output
+  float* x2 = (float*)s[S_X2];
+  if (c->m.arch == 1) {
+    float* z = (float*)s[S_Z];
+    if (on) norm_bwd_params(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, b.n2_b);
+    norm_bwd_dx(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, nullptr, c->dxb, c->dxb_a);          // dz
+    linear_dx(c, T, d, f, c->dxb_a, d, c->P(b.w_fc2), c->dbig, f, nullptr, 0, false);               // du
+    if (on) { linear_dw(c, T, d, f, c->dxb_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxb, true, T, d, d, b.b_fc2); }
+    act_bwd(c, s[S_A]);                                                                             // da
+    linear_dx(c, T, f, d, c->dbig, f, c->P(b.w_fc1), c->dxa, d, c->dxb, d, true);                   // dx1
+    if (on) { linear_dw(c, T, f, d, c->dbig, f, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, f, f, b.b_fc1); }
+    if (on) norm_bwd_params(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, b.n1_b);
+    norm_bwd_dx(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, nullptr, c->dxb, c->dxb_a);         // dy
+    linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                  // do
+    if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); }
+    attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
+    if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, x_a, d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); }
+    if (need_dx) linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dxa, d, c->dxb, d, true);
+    return;
+  }
+  linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);                 // du / ds
+  if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxa, true, T, d, d, b.b_fc2); }
+  act_bwd(c, s[S_A]);                                                                               // da in dbig [T,fa]
+  linear_dx(c, T, fa, d, c->dbig, fa, c->P(b.w_fc1), c->dt1, d, nullptr, 0, false);                 // dh2
+  if (on) { linear_dw(c, T, fa, d, c->dbig, fa, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, fa, fa, b.b_fc1); }
+  if (on) norm_bwd_params(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, b.n2_b);
+  norm_bwd_dx(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, c->dxa, c->dxb, c->dxb_a);            // dx2
+  linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                    // do
+  if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); }
+  attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
+  if (c->m.arch == 2) rope(c, c->dqkv, -1.0f);
+  linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dt1, d, nullptr, 0, false);           // dh1
+  if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, s[S_H1], d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); }
+  if (on) norm_bwd_params(c, c->dt1, false, x_r, (float*)s[S_ST1], b.n1_g, b.n1_b);
+  if (need_dx) norm_bwd_dx(c, c->dt1, false, x_r, (float*)s[S_ST1], b.n1_g, c->dxb, c->dxa, c->dxa_a);
+}
+
+void issue_h2d(hift_ctx* c, int g, int sl, bool after_forward) {
+  GroupRec& gr = c->groups[g];
+  if (after_forward) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_fwd, 0));
+  if (c->d2h_pending[sl]) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_d2h[sl], 0));
+  // slot layout follows the blob: consecutive planes of gr.numel floats
+  c->note(cudaMemcpyAsync(c->slot[sl], gr.blob, gr.blob_bytes, cudaMemcpyHostToDevice, c->st_h2d));
+  c->note(cudaEventRecord(c->ev_h2d[sl], c->st_h2d));
+  c->step_h2d = gr.blob_bytes;
+}
+
+hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
+  const hift_model_cfg& m = c->m;
+  const int L = c->L, T = c->T, d = c->d, V = c->V, Vp = c->Vp, B = c->B, S = c->S;
+  const int k = (int)c->groups.size();
+  const int g = c->forced >= 0 ? c->forced : c->order[c->t % k];
+  GroupRec& gr = c->groups[g];
+  const int lo = gr.unit_lo, hi = gr.unit_hi;
+  const double lr = lr_for_cycle(c->oc, c->t / k);
+  c->last_group = g;
+  c->step_launches = 0; c->step_h2d = 0; c->step_d2h = 0;
+  c->first_err = cudaSuccess;
+  const int sl = c->n_slots == 2 ? (int)(c->t & 1) : 0;
+  auto active = [&](int u) { return u >= lo && u <= hi; };
+
+  plan_slots(c, g, true);
+  if (c->arena_off > c->arena_cap) return HIFT_ERR_CFG;
+
+  if (c->offload && c->oc.prefetch_groups) issue_h2d(c, g, sl, false);
+
+  // "Clear gradients": the group's span of the gradient buffer starts at zero
+  c->note(cudaMemsetAsync(c->grad, 0, gr.numel * sizeof(float), c->st));
+  c->note(cudaMemsetAsync(c->scal, 0, 4 * sizeof(float), c->st));
+  int* bad = (int*)(c->scal + 2);
+  int* nvalid = (int*)(c->scal + 1);
+
+  // ---------------- forward (Algorithm 1, step h)
+  std::vector<float*> chain_r(L + 1);
+  std::vector<char*> chain_a(L + 1, nullptr);
+  for (int i = 0; i < L; ++i) { chain_r[i] = (float*)c->slots[i][S_XIN]; chain_a[i] = c->slots[i][S_XINA]; }
+  chain_r[L] = c->x_final; chain_a[L] = c->x_final_a;
+  {
+    float* x0 = m.arch == 1 ? c->emb_e : chain_r[0];
+    LAUNCH(HIFT_K_EMBED, (double)T * d * (c->es * (c->t_pos >= 0 ? 2 : 1) + 4),
+           if (c->mixed) embed_fwd_kernel<bf16><<<T, norm_threads(d), 0, c->st>>>(tok, (const bf16*)c->P(c->t_tok), (const bf16*)c->Pn(c->t_pos), x0, S, d, V, bad);
+           else embed_fwd_kernel<float><<<T, norm_threads(d), 0, c->st>>>(tok, (const float*)c->P(c->t_tok), (const float*)c->Pn(c->t_pos), x0, S, d, V, bad));
+    if (m.arch == 1) norm_fwd(c, c->emb_e, c->t_eg, c->t_eb, chain_a[0], chain_r[0], c->st_e);
+  }
+  for (int i = 0; i < L; ++i) forward_block(c, i, chain_r[i], chain_a[i], chain_r[i + 1], chain_a[i + 1]);
+  if (m.arch == 1) {
+    const int C = m.n_classes;
+    // pooled = first token of every sequence: rows of the last block's output with stride S*d
+    linear_fwd(c, B, C, d, c->x_final_a, (int64_t)S * d, c->P(c->t_wc), c->logits, C, c->P(c->t_bc), nullptr, 0, false);
+    LAUNCH(HIFT_K_CE, 2.0 * B * C * c->es,
+           launch_cross_entropy(c->st, c->mixed, B, C, C, c->logits, lab, c->rowloss, nvalid, bad, c->scal));
+    c->step_launches += 2;
+  } else {
+    norm_fwd(c, c->x_final, c->t_fg, c->t_fb, c->xf, nullptr, c->stf);
+    const int tw = m.tie_head ? c->t_tok : c->t_wh;
+    linear_fwd(c, T, V, d, c->xf, d, c->P(tw), c->logits, Vp, nullptr, nullptr, 0, false);
+    LAUNCH(HIFT_K_CE, 4.0 * T * (double)V * c->es,
+           launch_cross_entropy(c->st, c->mixed, T, V, Vp, c->logits, lab, c->rowloss, nvalid, bad, c->scal));
+    c->step_launches += 2;
+  }
+  if (c->offload && !c->oc.prefetch_groups) {
+    // the paper's order: optimizer state moves to the GPU after the forward pass (step i)
+    c->note(cudaEventRecord(c->ev_fwd, c->st));
+    issue_h2d(c, g, sl, true);
+  }
+
+  // ---------------- backward, truncated at the group ("Backpropagation")
+  const bool head_on = active(L + 1);
+  bool done = false;
+  if (m.arch == 1) {
+    const int C = m.n_classes;
+    if (head_on) {
+      // dWc[C,d] = dlogits^T pooled ; pooled rows have stride S*d
+      gemm(c, HIFT_K_GEMM_DW, C, d, B, c->logits, 1, C, c->x_final_a, (int64_t)S * d, 1, c->G(c->t_wc), d, nullptr, nullptr, 0, true);
+      bias_grad(c, c->logits, false, B, C, C, c->t_bc);
+    }
+    if (lo == L + 1) done = true;
+    else {
+      c->note(cudaMemsetAsync(c->dxa, 0, (size_t)T * d * sizeof(float), c->st));
+      // dx[b*S,:] = dlogits[b,:] Wc
+      gemm(c, HIFT_K_GEMM_DX, B, d, C, c->logits, C, 1, c->P(c->t_wc), d, 1, c->dxa, (int64_t)S * d, nullptr, nullptr, 0, true);
+    }
+  } else {
+    const int tw = m.tie_head ? c->t_tok : c->t_wh;
+    const bool w_on = m.tie_head ? active(0) : head_on;
+    if (w_on) linear_dw(c, T, V, d, c->logits, Vp, c->xf, d, c->G(tw));
+    linear_dx(c, T, V, d, c->logits, Vp, c->P(tw), c->dt1, d, nullptr, 0, false);
+    if (head_on) norm_bwd_params(c, c->dt1, false, c->x_final, c->stf, c->t_fg, c->t_fb);
+    if (lo == L + 1) done = true;
+    else norm_bwd_dx(c, c->dt1, false, c->x_final, c->stf, c->t_fg, nullptr, c->dxa, c->dxa_a);
+  }
+  if (!done) {
+    for (int i = L - 1; i >= 0; --i) {
+      const int u = i + 1;
+      if (u < lo) break;
+      backward_block(c, i, chain_r[i], chain_a[i], active(u), u > lo);
+      if (u == lo) break;
+    }
+  }
+  if (active(0)) {
+    const float* src = c->dxa;
+    if (m.arch == 1) {
+      norm_bwd_params(c, c->dxa, true, c->emb_e, c->st_e, c->t_eg, c->t_eb);
+      norm_bwd_dx(c, c->dxa, true, c->emb_e, c->st_e, c->t_eg, nullptr, c->dxb, nullptr);
+      src = c->dxb;
+    }
+    LAUNCH(HIFT_K_EMBED, (double)T * d * 12,
+           embed_bwd_tok_kernel<<<T, 128, T * sizeof(int), c->st>>>(tok, src, c->G(c->t_tok), T, d, V));
+    if (c->t_pos >= 0) {
+      LAUNCH(HIFT_K_EMBED, (double)T * d * 4 + (double)S * d * 4,
+             embed_bwd_pos_kernel<<<S, 128, 0, c->st>>>(src, c->G(c->t_pos), B, S, d));
+    }
+  }
+
+  // ---------------- group-local optimizer (Algorithm 1: P now points at theta_s only)
+  gr.tau += 1;
+  float *mst, *s0, *s1;
+  void* pbf = nullptr;
+  if (c->offload) {
+    float* base = (float*)c->slot[sl];
+    if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
+    else { mst = (float*)c->params + gr.off; s0 = base; s1 = base + gr.numel; }
+    c->note(cudaStreamWaitEvent(c->st, c->ev_h2d[sl], 0));
+  } else {
+    if (c->mixed) { mst = c->master_all + gr.off; pbf = c->params + gr.off * c->es; }
+    else mst = (float*)c->params + gr.off;
+    s0 = c->s0_all + gr.off;
+    s1 = c->s1_all ? c->s1_all + gr.off : nullptr;
+  }
+  const OptScalars hs = make_opt_scalars(c->oc.kind, lr, c->oc.beta1, c->oc.beta2, c->oc.eps,
+                                         c->oc.weight_decay, c->oc.momentum, gr.tau);
+  const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : 20.0) + (pbf ? 2.0 : 0.0));
+  LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs));
+
+  // ---------------- state back to the host (step k)
+  if (c->offload) {
+    c->note(cudaEventRecord(c->ev_opt[sl], c->st));
+    c->note(cudaStreamWaitEvent(c->st_d2h, c->ev_opt[sl], 0));
+    c->note(cudaMemcpyAsync(gr.blob, c->slot[sl], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st_d2h));
+    c->note(cudaEventRecord(c->ev_d2h[sl], c->st_d2h));
+    c->d2h_pending[sl] = true;
+    c->step_d2h = gr.blob_bytes;
+  }
+
+  c->note(cudaMemcpyAsync(c->scal_host, c->scal, 4 * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  c->note(cudaStreamSynchronize(c->st));
+  c->prof_collect();
+  c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
+  if (c->first_err != cudaSuccess) return HIFT_ERR_CUDA;
+  const float loss = c->scal_host[0];
+  int bad_h;
+  memcpy(&bad_h, &c->scal_host[2], sizeof(int));
+  if (loss_host) *loss_host = loss;
+  if (bad_h) return HIFT_ERR_INPUT;
+  if (!isfinite(loss)) return HIFT_ERR_NONFINITE;
+  return HIFT_OK;
+}
+
+void sync_all(hift_ctx* c) {
+  cudaStreamSynchronize(c->st);
+  if (c->st_h2d) cudaStreamSynchronize(c->st_h2d);
+  if (c->st_d2h) cudaStreamSynchronize(c->st_d2h);
+}
+
+int group_of_unit(const hift_ctx* c, int u) {
+  for (size_t g = 0; g < c->groups.size(); ++g)
+    if (u >= c->groups[g].unit_lo && u <= c->groups[g].unit_hi) return (int)g;
+  return -1;
+}
+// where the fp32 master / state plane `plane` (0 master, 1 s0, 2 s1) of tensor ti lives
+float* plane_ptr(hift_ctx* c, int ti, int plane, bool* on_host) {
+  const TensorRec& r = c->tens[ti];
+  const int g = group_of_unit(c, r.unit);
+  const GroupRec& gr = c->groups[g];
+  *on_host = false;
+  if (plane == 0 && !c->mixed) return (float*)c->params + r.off;
+  if (c->offload) {
+    *on_host = true;
+    const int pl = c->mixed ? plane : plane - 1;
+    return (float*)gr.blob + (size_t)pl * gr.numel + (r.off - gr.off);
+  }
+  if (plane == 0) return c->master_all + r.off;
+  if (plane == 1) return c->s0_all + r.off;
+  return c->s1_all ? c->s1_all + r.off : nullptr;
+}
+
+}  // namespace
+
+// ====================================================================== C entry points
+extern "C" {
+
+const char* hift_strerror(hift_status s) {
+  switch (s) {
+    case HIFT_OK: return "ok";
+    case HIFT_ERR_CFG: return "invalid or unsupported configuration";
+    case HIFT_ERR_OOM_DEVICE: return "out of device memory";
+    case HIFT_ERR_OOM_PINNED: return "out of pinned host memory";
+    case HIFT_ERR_INPUT: return "invalid input (token id / label out of range or NULL pointer)";
+    case HIFT_ERR_NONFINITE: return "non-finite loss";
+    case HIFT_ERR_TIMEOUT: return "device-side wait timed out";
+    case HIFT_ERR_CUDA: return "CUDA error";
+  }
+  return "unknown";
+}
+
+void hift_destroy(hift_ctx* c) {
+  if (!c) return;
+  sync_all(c);
+  for (void* p : c->dev_allocs) cudaFree(p);
+  for (auto& g : c->groups) if (g.blob) cudaFreeHost(g.blob);
+  if (c->scal_host) cudaFreeHost(c->scal_host);
+  for (auto e : c->ev_pool) cudaEventDestroy(e);
+  if (c->events_made) {
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(c->ev_h2d[i]); cudaEventDestroy(c->ev_opt[i]); cudaEventDestroy(c->ev_d2h[i]); }
+    cudaEventDestroy(c->ev_fwd);
+  }
+  if (c->st_h2d) cudaStreamDestroy(c->st_h2d);
+  if (c->st_d2h) cudaStreamDestroy(c->st_d2h);
+  delete c;
+}
+
+hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const hift_opt_cfg* oc,
+                        void* cuda_stream, hift_ctx** out) {
+  if (!out) return HIFT_ERR_CFG;
+  *out = nullptr;
+  if (!m || !gc || !oc) return HIFT_ERR_CFG;
+  // ---- validation
+  if (m->arch < 0 || m->arch > 2 || m->n_blocks < 1 || m->d_model < 8 || m->n_heads < 1 ||
+      m->d_ffn < 8 || m->vocab < 2 || m->batch < 1 || m->seq < 1)
+    return HIFT_ERR_CFG;
+  if (m->d_model % 8 || m->d_ffn % 8 || m->d_model % m->n_heads) return HIFT_ERR_CFG;
+  if (!attention_head_ok(m->d_model / m->n_heads)) return HIFT_ERR_CFG;
+  if (m->dtype != 0 && m->dtype != 1) return HIFT_ERR_CFG;
+  if (m->arch != 2 && m->max_pos < m->seq) return HIFT_ERR_CFG;
+  if (m->arch == 1 && (m->n_classes < 2 || m->tie_head)) return HIFT_ERR_CFG;
+  // the embedding-gradient kernel keeps one occurrence list of <= batch*seq ints in shared memory
+  if ((int64_t)m->batch * m->seq > 8192) return HIFT_ERR_CFG;
+  if (gc->layers_per_group < 1 || gc->order < 0 || gc->order > 2) return HIFT_ERR_CFG;
+  if (oc->kind < 0 || oc->kind > 2 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
+  if (oc->sched == 1 && oc->total_cycles < 1) return HIFT_ERR_CFG;
+  if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
+
+  hift_ctx* c = new hift_ctx();
+  c->m = *m; c->gc = *gc; c->oc = *oc;
+  c->st = (cudaStream_t)cuda_stream;
+  c->mixed = m->dtype == 1;
+  c->es = c->mixed ? 2 : 4;
+  c->L = m->n_blocks; c->d = m->d_model; c->f = m->d_ffn; c->fa = m->arch == 2 ? 2 * m->d_ffn : m->d_ffn;
+  c->H = m->n_heads; c->dh = m->d_model / m->n_heads; c->B = m->batch; c->S = m->seq; c->T = m->batch * m->seq;
+  c->V = m->vocab; c->Vp = (int)align_up(m->vocab, 128);
+  c->n_state = oc->kind == 0 ? 2 : 1;
+  c->offload = oc->offload_state != 0;
+  c->n_slots = (c->offload && oc->prefetch_groups) ? 2 : 1;
+  memset(c->prof_launches, 0, sizeof(c->prof_launches));
+  memset(c->prof_ms, 0, sizeof(c->prof_ms));
+  memset(c->prof_work, 0, sizeof(c->prof_work));
+  build_layout(c);
+
+  hift_status rc = HIFT_OK;
+  auto fail = [&](hift_status s) { hift_destroy(c); return s; };
+  for (int i = 0; i < 2; ++i) {
+    cudaEventCreateWithFlags(&c->ev_h2d[i], cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&c->ev_opt[i], cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&c->ev_d2h[i], cudaEventDisableTiming);
+  }
+  cudaEventCreateWithFlags(&c->ev_fwd, cudaEventDisableTiming);
+  c->events_made = true;
+  if (cudaStreamCreateWithFlags(&c->st_h2d, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
+  if (cudaStreamCreateWithFlags(&c->st_d2h, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
+
+  // ---- parameters, gradients, optimizer state
+  const size_t planes = (size_t)(c->mixed ? 1 : 0) + c->n_state;
+  if ((rc = dev_alloc(c, (void**)&c->params, c->total * c->es)) != HIFT_OK) return fail(rc);
+  cudaMemsetAsync(c->params, 0, c->total * c->es, c->st);
+  if ((rc = dev_alloc(c, (void**)&c->grad, c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
+  if (c->offload) {
+    for (int s = 0; s < c->n_slots; ++s) {
+      if ((rc = dev_alloc(c, (void**)&c->slot[s], planes * c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->slot[s], 0, planes * c->max_group * sizeof(float), c->st);
+    }
+    for (auto& g : c->groups) {
+      g.blob_bytes = planes * g.numel * sizeof(float);
+      if (cudaHostAlloc((void**)&g.blob, g.blob_bytes, cudaHostAllocDefault) != cudaSuccess) {
+        cudaGetLastError();
+        g.blob = nullptr;
+        return fail(HIFT_ERR_OOM_PINNED);
+      }
+      memset(g.blob, 0, g.blob_bytes);
+      c->pinned_bytes += g.blob_bytes;
+    }
+  } else {
+    if (c->mixed) {
+      if ((rc = dev_alloc(c, (void**)&c->master_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->master_all, 0, c->total * sizeof(float), c->st);
+    }
+    if ((rc = dev_alloc(c, (void**)&c->s0_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
+    cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
+    if (c->n_state == 2) {
+      if ((rc = dev_alloc(c, (void**)&c->s1_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
+    }
+  }
+  if (cudaHostAlloc((void**)&c->scal_host, 4 * sizeof(float), cudaHostAllocDefault) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
+
+  // ---- activation arena: fixed work buffers, one scratch copy of every slot, then the
+  //      per-group kept activations (sized for the worst group)
+  const size_t T = c->T, d = c->d, es = c->es;
+  c->slots.assign(c->L + 1, std::vector<char*>(S_NUM, nullptr));
+  for (int pass = 0; pass < 2; ++pass) {
+    c->arena_off = 0;
+    c->tok_dev = (int32_t*)arena_take(c, T * sizeof(int32_t));
+    c->lab_dev = (int32_t*)arena_take(c, T * sizeof(int32_t));
+    c->dxa = (float*)arena_take(c, T * d * 4); c->dxb = (float*)arena_take(c, T * d * 4);
+    c->dxa_a = arena_take(c, T * d * es); c->dxb_a = arena_take(c, T * d * es); c->dt1 = arena_take(c, T * d * es);
+    c->dqkv = arena_take(c, T * 3 * d * es);
+    c->dbig = arena_take(c, T * (size_t)c->fa * es);
+    c->dsw = m->arch == 2 ? arena_take(c, T * (size_t)c->f * es) : nullptr;
+    c->x_final = (float*)arena_take(c, T * d * 4);
+    c->pp[0] = (float*)arena_take(c, T * d * 4); c->pp[1] = (float*)arena_take(c, T * d * 4);
+    if (m->arch == 1) {
+      c->x_final_a = arena_take(c, T * d * es);
+      c->ppa[0] = arena_take(c, T * d * es); c->ppa[1] = arena_take(c, T * d * es);
+      c->emb_e = (float*)arena_take(c, T * d * 4);
+      c->st_e = (float*)arena_take(c, 2 * T * sizeof(float));
+      c->logits = arena_take(c, (size_t)c->B * m->n_classes * es);
+    } else {
+      c->xf = arena_take(c, T * d * es);
+      c->stf = (float*)arena_take(c, 2 * T * sizeof(float));
+      c->logits = arena_take(c, T * (size_t)c->Vp * es);
+    }
+    c->dsum = (float*)arena_take(c, T * c->H * sizeof(float));
+    const size_t maxcols = std::max<size_t>(std::max<size_t>(3 * d, c->fa), 8);
+    c->partial = (float*)arena_take(c, 2 * kColChunks * maxcols * sizeof(float));
+    c->rowloss = (float*)arena_take(c, T * sizeof(float));
+    c->scal = (float*)arena_take(c, 4 * sizeof(float));
+    if (m->arch == 2) c->rope_cs = (float*)arena_take(c, 2 * (size_t)c->S * (c->dh / 2) * sizeof(float));
+    for (int s = 0; s < S_NUM; ++s)
+      c->slots[c->L][s] = (slot_min_level(m->arch, s) == 99 || s == S_XIN || s == S_XINA)
+                              ? nullptr : arena_take(c, slot_bytes(c, s));
+    c->arena_fixed = c->arena_off;
+    if (pass == 0) {
+      size_t worst = c->arena_fixed;
+      for (size_t g = 0; g < c->groups.size(); ++g) worst = std::max(worst, plan_slots(c, (int)g, false));
+      c->arena_cap = worst;
+      if ((rc = dev_alloc(c, (void**)&c->arena, c->arena_cap)) != HIFT_OK) return fail(rc);
+    }
+  }
+  if (m->arch == 2) {
+    const int half = c->dh / 2;
+    std::vector<float> cs(2 * (size_t)c->S * half);
+    for (int p = 0; p < c->S; ++p)
+      for (int j = 0; j < half; ++j) {
+        const double ang = (double)p * pow(m->rope_base, -2.0 * j / (double)c->dh);
+        cs[(size_t)p * half + j] = (float)cos(ang);
+        cs[(size_t)c->S * half + (size_t)p * half + j] = (float)sin(ang);
+      }
+    cudaMemcpyAsync(c->rope_cs, cs.data(), cs.size() * sizeof(float), cudaMemcpyHostToDevice, c->st);
+    cudaStreamSynchronize(c->st);
+  }
+  if (cudaStreamSynchronize(c->st) != cudaSuccess) return fail(HIFT_ERR_CUDA);
+  gemm_tc_init();   // if unavailable, gemm_tc_eligible() answers false and CUDA cores are used
+  *out = c;
+  return HIFT_OK;
+}
+
+hift_status hift_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
+  if (!c || !tok || !lab) return HIFT_ERR_INPUT;
+  return do_step(c, tok, lab, loss_host);
+}
+
+hift_status hift_step_host(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
+  if (!c || !tok || !lab) return HIFT_ERR_INPUT;
+  const size_t nlab = c->m.arch == 1 ? c->B : c->T;
+  for (int i = 0; i < c->T; ++i) if (tok[i] < 0 || tok[i] >= c->V) return HIFT_ERR_INPUT;
+  const int nl = c->m.arch == 1 ? c->m.n_classes : c->V;
+  for (size_t i = 0; i < nlab; ++i) if (lab[i] >= nl) return HIFT_ERR_INPUT;
+  cudaMemcpyAsync(c->tok_dev, tok, c->T * sizeof(int32_t), cudaMemcpyHostToDevice, c->st);
+  cudaMemcpyAsync(c->lab_dev, lab, nlab * sizeof(int32_t), cudaMemcpyHostToDevice, c->st);
+  return do_step(c, c->tok_dev, c->lab_dev, loss_host);
+}
+
+int32_t hift_active_group(const hift_ctx* c) {
+  if (c->forced >= 0) return c->forced;
+  return c->order[c->t % (int64_t)c->groups.size()];
+}
+int32_t hift_num_groups(const hift_ctx* c) { return (int32_t)c->groups.size(); }
+int64_t hift_step_count(const hift_ctx* c) { return c->t; }
+double hift_current_lr(const hift_ctx* c) { return lr_for_cycle(c->oc, c->t / (int64_t)c->groups.size()); }
+hift_status hift_group_units(const hift_ctx* c, int32_t g, int32_t* lo, int32_t* hi) {
+  if (g < 0 || g >= (int)c->groups.size()) return HIFT_ERR_CFG;
+  *lo = c->groups[g].unit_lo; *hi = c->groups[g].unit_hi;
+  return HIFT_OK;
+}
+hift_status hift_force_group(hift_ctx* c, int32_t g) {
+  if (g < -1 || g >= (int)c->groups.size()) return HIFT_ERR_CFG;
+  c->forced = g;
+  return HIFT_OK;
+}
+size_t hift_peak_hbm_bytes(const hift_ctx* c) { return c->dev_bytes; }
+size_t hift_pinned_host_bytes(const hift_ctx* c) { return c->pinned_bytes; }
+
+int32_t hift_num_tensors(const hift_ctx* c) { return (int32_t)c->tens.size(); }
+hift_status hift_tensor_info(const hift_ctx* c, int32_t ti, char* name, int32_t* unit, int64_t* rows, int64_t* cols) {
+  if (ti < 0 || ti >= (int)c->tens.size()) return HIFT_ERR_CFG;
+  const TensorRec& r = c->tens[ti];
+  if (name) memcpy(name, r.name, 64);
+  if (unit) *unit = r.unit;
+  if (rows) *rows = r.rows;
+  if (cols) *cols = r.cols;
+  return HIFT_OK;
+}
+
+hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) {
+  if (ti < 0 || ti >= (int)c->tens.size() || !src || n != c->tens[ti].numel) return HIFT_ERR_CFG;
+  sync_all(c);
+  bool on_host;
+  float* mp = plane_ptr(c, ti, 0, &on_host);
+  if (on_host) memcpy(mp, src, n * sizeof(float));
+  else if (cudaMemcpy(mp, src, n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return HIFT_ERR_CUDA;
+  if (c->mixed) {
+    // stage the fp32 values in the gradient buffer (any tensor fits in the largest group)
+    if (cudaMemcpy(c->grad, src, n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return HIFT_ERR_CUDA;
+    cast_from_f32_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>(c->grad, (bf16*)c->P(ti), n);
+    if (cudaStreamSynchronize(c->st) != cudaSuccess) return HIFT_ERR_CUDA;
+  }
+  return HIFT_OK;
+}
+hift_status hift_get_param(hift_ctx* c, int32_t ti, float* dst, size_t n) {
+  if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
+  sync_all(c);
+  bool on_host;
+  float* mp = plane_ptr(c, ti, 0, &on_host);
+  if (on_host) memcpy(dst, mp, n * sizeof(float));
+  else if (cudaMemcpy(dst, mp, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
+  return HIFT_OK;
+}
+hift_status hift_get_model_param(hift_ctx* c, int32_t ti, float* dst, size_t n) {
+  if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
+  sync_all(c);
+  if (!c->mixed) return cudaMemcpy(dst, c->P(ti), n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+  float* tmp = nullptr;
+  if (cudaMalloc((void**)&tmp, n * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return HIFT_ERR_OOM_DEVICE; }
+  cast_to_f32_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>((const bf16*)c->P(ti), tmp, n);
+  cudaError_t e = cudaMemcpyAsync(dst, tmp, n * sizeof(float), cudaMemcpyDeviceToHost, c->st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->st);
+  cudaFree(tmp);
+  return e == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_get_state(hift_ctx* c, int32_t ti, int32_t which, float* dst, size_t n) {
+  if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
+  if (which < 0 || which >= c->n_state) return HIFT_ERR_CFG;
+  sync_all(c);
+  bool on_host;
+  float* sp = plane_ptr(c, ti, 1 + which, &on_host);
+  if (!sp) return HIFT_ERR_CFG;
+  if (on_host) memcpy(dst, sp, n * sizeof(float));
+  else if (cudaMemcpy(dst, sp, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
+  return HIFT_OK;
+}
+hift_status hift_get_grad(hift_ctx* c, int32_t ti, float* dst, size_t n) {
+  if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
+  if (c->last_group < 0 || group_of_unit(c, c->tens[ti].unit) != c->last_group) return HIFT_ERR_CFG;
+  sync_all(c);
+  return cudaMemcpy(dst, c->G(ti), n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+
+hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
+  sync_all(c);
+  const size_t planes = (size_t)(c->mixed ? 1 : 0) + c->n_state;
+  for (size_t g = 0; g < c->groups.size(); ++g) {
+    GroupRec& gr = c->groups[g];
+    if (c->offload) cudaMemsetAsync(c->slot[0], 0, planes * gr.numel * sizeof(float), c->st);
+    for (int u = gr.unit_lo; u <= gr.unit_hi; ++u) {
+      for (int ti : c->unit_tens[u]) {
+        const TensorRec& r = c->tens[ti];
+        float* mp = nullptr;
+        if (c->mixed) mp = c->offload ? (float*)c->slot[0] + (r.off - gr.off) : c->master_all + r.off;
+        const uint64_t sd = seed * 0x9E3779B97F4A7C15ull + (uint64_t)ti * 0xD1B54A32D192ED03ull;
+        if (c->mixed) init_tensor_kernel<bf16><<<grid_for(r.numel, 256), 256, 0, c->st>>>((bf16*)c->P(ti), mp, r.numel, r.init_kind, (float)stdv, sd);
+        else init_tensor_kernel<float><<<grid_for(r.numel, 256), 256, 0, c->st>>>((float*)c->P(ti), nullptr, r.numel, r.init_kind, (float)stdv, sd);
+      }
+    }
+    if (c->offload) {
+      cudaMemcpyAsync(gr.blob, c->slot[0], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st);
+      if (cudaStreamSynchronize(c->st) != cudaSuccess) return HIFT_ERR_CUDA;
+    }
+    gr.tau = 0;
+  }
+  if (!c->offload) {
+    cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
+    if (c->s1_all) cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
+  }
+  return cudaStreamSynchronize(c->st) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+
+hift_status hift_profile_enable(hift_ctx* c, int32_t on) {
+  sync_all(c);
+  c->prof_on = on != 0;
+  memset(c->prof_launches, 0, sizeof(c->prof_launches));
+  memset(c->prof_ms, 0, sizeof(c->prof_ms));
+  memset(c->prof_work, 0, sizeof(c->prof_work));
+  return HIFT_OK;
+}
+hift_status hift_profile(hift_ctx* c, int32_t cls, int64_t* launches, double* ms, double* work) {
+  if (cls < 0 || cls >= HIFT_K_NUM) return HIFT_ERR_CFG;
+  if (launches) *launches = c->prof_launches[cls];
+  if (ms) *ms = c->prof_ms[cls];
+  if (work) *work = c->prof_work[cls];
+  return HIFT_OK;
+}
+int64_t hift_last_step_launches(const hift_ctx* c) { return c->step_launches; }
+hift_status hift_last_step_paging(const hift_ctx* c, size_t* h2d, size_t* d2h) {
+  if (h2d) *h2d = c->step_h2d;
+  if (d2h) *d2h = c->step_d2h;
+  return HIFT_OK;
+}
+
+// ---------------------------------------------------------------- optimizer on flat buffers
+hift_status hift_opt_step(int32_t kind, size_t n, void* param_bf16, float* master, const float* grad,
+                          float* s0, float* s1, double lr, double b1, double b2, double eps,
+                          double wd, double mu, int64_t tau, void* stream) {
+  if (kind < 0 || kind > 2 || !master || !grad || !s0 || (kind == 0 && !s1) || tau < 1) return HIFT_ERR_CFG;
+  const uintptr_t al = (uintptr_t)master | (uintptr_t)grad | (uintptr_t)s0 | (uintptr_t)s1 | (uintptr_t)param_bf16;
+  if (al & 15) return HIFT_ERR_CFG;
+  const OptScalars h = make_opt_scalars(kind, lr, b1, b2, eps, wd, mu, tau);
+  launch_fused_opt((cudaStream_t)stream, kind, n, param_bf16, master, grad, s0, s1, h);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- single kernels
+hift_status hift_k_linear(int32_t form, int32_t dtype, int32_t path, int64_t M, int64_t N, int64_t K,
+                          const void* a, const void* b, void* out, const void* bias,
+                          const float* residual, void* stream) {
+  if (form < 0 || form > 2 || dtype < 0 || dtype > 1 || M < 1 || N < 1 || K < 1) return HIFT_ERR_CFG;
+  const bool f32o = residual != nullptr;
+  GemmArgs g;
+  if (form == 0) g = GemmArgs{(int)M, (int)N, (int)K, a, K, 1, b, 1, K, out, N, bias, residual, N, f32o};
+  else if (form == 1) g = GemmArgs{(int)M, (int)K, (int)N, a, N, 1, b, K, 1, out, K, nullptr, residual, K, f32o};
+  else g = GemmArgs{(int)N, (int)K, (int)M, a, 1, N, b, K, 1, out, K, nullptr, nullptr, 0, true};
+  const bool tc_ok = dtype == 1 && gemm_tc_init() == 0 && gemm_tc_eligible(g);
+  if (path == 2 && !tc_ok) return HIFT_ERR_CFG;
+  if (path != 1 && tc_ok) {
+    if (gemm_tc_launch((cudaStream_t)stream, g) != cudaSuccess) return HIFT_ERR_CUDA;
+    return HIFT_OK;
+  }
+  launch_gemm_simt((cudaStream_t)stream, dtype, g);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_attention_fwd(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
+                                 const void* qkv, void* o, float* lse, void* stream) {
+  if (!attention_head_ok(dh) || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
+  launch_attention_fwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_attention_bwd(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
+                                 const void* qkv, const void* o, const float* lse, const void* dout,
+                                 void* dqkv, float* dsum, void* stream) {
+  if (!attention_head_ok(dh) || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
+  launch_attention_bwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,
+                            const float* x, const void* gain, const void* bias, void* y, float* stats,
+                            void* stream) {
+  if (cols % 8 || kind < 0 || kind > 1 || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
+  launch_norm_fwd((cudaStream_t)stream, dtype, kind, rows, (int)cols, (float)eps, x, gain, bias, y, nullptr, stats);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_norm_bwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, const void* dy,
+                            const float* x, const float* stats, const void* gain, const float* add,
+                            float* dx, float* dgain, float* dbias, float* partial, void* stream) {
+  if (cols % 8 || kind < 0 || kind > 1 || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
+  if (dgain && !partial) return HIFT_ERR_CFG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dx) launch_norm_bwd_dx(st, dtype, kind, false, rows, (int)cols, dy, x, stats, gain, add, dx, nullptr);
+  if (dgain) launch_colreduce(st, dtype == 1, kind == 0 ? 1 : 2, rows, (int)cols, dy, cols, x, stats, partial, dgain, dbias);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_cross_entropy(int32_t dtype, int64_t rows, int64_t vocab, int64_t ld, void* logits,
+                                 const int32_t* labels, float* rowloss, float* loss, void* stream) {
+  if (dtype < 0 || dtype > 1 || ld < vocab) return HIFT_ERR_CFG;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaMemsetAsync(loss, 0, 4 * sizeof(float), st);
+  launch_cross_entropy(st, dtype, rows, vocab, ld, logits, labels, rowloss, (int*)(loss + 1), (int*)(loss + 2), loss);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+
+}  // extern "C"

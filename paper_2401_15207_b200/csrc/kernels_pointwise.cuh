@@ -1,0 +1,542 @@
+// Bandwidth-bound kernels of the training step: embedding, LayerNorm/RMSNorm, GELU/SwiGLU,
+// RoPE, softmax cross-entropy, column reductions (bias and gain gradients), the fused
+// group-local optimizer, and small utilities.  All reductions have a fixed order.
+//
+// The residual stream and its gradient are fp32 in every configuration; P / T below is the
+// parameter and GEMM-operand type (bf16 or fp32).
+#pragma once
+#include "common.cuh"
+
+namespace hift {
+
+// ------------------------------------------------------------------ utilities
+template <typename T>
+__global__ void cast_from_f32_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) dst[i] = from_f<T>(src[i]);
+}
+template <typename T>
+__global__ void cast_to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) dst[i] = to_f(src[i]);
+}
+
+// Counter-based synthetic weights: element i of stream `seed` is a Box-Muller normal built
+// from the two 32-bit halves of a SplitMix64-style finaliser of (seed, i).
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+template <typename T>
+__global__ void init_tensor_kernel(T* __restrict__ param, float* __restrict__ master, size_t n,
+                                   int kind, float stdv, uint64_t seed) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) {
+    float v;
+    if (kind == 0) {
+      uint64_t h = mix64(seed + 0x9E3779B97F4A7C15ull * (uint64_t)(i + 1));
+      float u1 = ((uint32_t)(h >> 32) + 1.0f) * (1.0f / 4294967808.0f);
+      float u2 = (uint32_t)h * (1.0f / 4294967296.0f);
+      v = stdv * sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+    } else {
+      v = kind == 1 ? 1.0f : 0.0f;
+    }
+    if (master) master[i] = v;
+    param[i] = from_f<T>(v);
+  }
+}
+
+// ------------------------------------------------------------------ embedding
+// x[t,:] = tok[id[t],:] (+ pos[t mod S,:]), written to the fp32 residual stream.
+// One block per token row.  An id outside [0, vocab) is clamped (never gathered out of
+// bounds) and reported through *bad.
+template <typename T>
+__global__ void embed_fwd_kernel(const int32_t* __restrict__ ids, const T* __restrict__ tok,
+                                 const T* __restrict__ pos, float* __restrict__ x, int S, int d,
+                                 int vocab, int* __restrict__ bad) {
+  const int t = blockIdx.x;
+  int id = ids[t];
+  if (id < 0 || id >= vocab) {
+    if (threadIdx.x == 0) *bad = 1;
+    id = id < 0 ? 0 : vocab - 1;
+  }
+  const T* tr = tok + (size_t)id * d;
+  const T* pr = pos ? pos + (size_t)(t % S) * d : nullptr;
+  float* xr = x + (size_t)t * d;
+  for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
+    float a[8];
+    load8(tr + c, a);
+    if (pr) {
+      float b[8];
+      load8(pr + c, b);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] += b[i];
+    }
+    store8(xr + c, a);
+  }
+}
+
+// grad_tok[id,:] += sum over positions t with ids[t] == id of dx[t,:], occurrences added in
+// increasing t.  Block t does the work for id = ids[t] only if t is the first occurrence, so
+// every gradient row has one writer and a fixed summation order (no atomics).
+__global__ void embed_bwd_tok_kernel(const int32_t* __restrict__ ids, const float* __restrict__ dx,
+                                     float* __restrict__ grad_tok, int Ttot, int d, int vocab) {
+  extern __shared__ int occ[];                       // positions of this id, in order
+  __shared__ int n_occ;
+  __shared__ int warp_cnt[32];
+  const int t0 = blockIdx.x;
+  const int id = ids[t0];
+  if (id < 0 || id >= vocab) return;                 // reported by the forward pass
+  int found = 0;
+  for (int t = threadIdx.x; t < t0; t += blockDim.x) found |= (ids[t] == id);
+  if (__syncthreads_or(found)) return;
+  if (threadIdx.x == 0) n_occ = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  // ordered compaction, one blockDim-sized chunk at a time
+  for (int base = t0; base < Ttot; base += blockDim.x) {
+    const int t = base + threadIdx.x;
+    const int hit = (t < Ttot) && (ids[t] == id);
+    const unsigned bal = __ballot_sync(0xffffffffu, hit);
+    if (lane == 0) warp_cnt[w] = __popc(bal);
+    __syncthreads();
+    int off = n_occ;
+    for (int i = 0; i < w; ++i) off += warp_cnt[i];
+    if (hit) occ[off + __popc(bal & ((1u << lane) - 1u))] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int tot = 0;
+      for (int i = 0; i < nw; ++i) tot += warp_cnt[i];
+      n_occ += tot;
+    }
+    __syncthreads();
+  }
+  const int n = n_occ;
+  float* gr = grad_tok + (size_t)id * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float acc = 0.f;
+    for (int i = 0; i < n; ++i) acc += dx[(size_t)occ[i] * d + c];
+    gr[c] += acc;
+  }
+}
+
+// grad_pos[s,:] = sum over batch rows b of dx[b*S+s,:]
+__global__ void embed_bwd_pos_kernel(const float* __restrict__ dx, float* __restrict__ grad_pos,
+                                     int B, int S, int d) {
+  const int s = blockIdx.x;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float acc = 0.f;
+    for (int b = 0; b < B; ++b) acc += dx[((size_t)b * S + s) * d + c];
+    grad_pos[(size_t)s * d + c] = acc;
+  }
+}
+
+// ------------------------------------------------------------------ norms
+// KIND 0: LayerNorm y = (x-mean)*rstd*g + b; KIND 1: RMSNorm y = x*rstd*g.
+// stats[row] = mean (0 for RMSNorm), stats[rows+row] = rstd.  cols % 8 == 0.
+// y_a (type P) feeds the next GEMM; y_r (fp32, optional) continues the residual stream.
+template <typename P, int KIND>
+__global__ void norm_fwd_kernel(const float* __restrict__ x, const P* __restrict__ gain,
+                                const P* __restrict__ bias, P* __restrict__ y_a,
+                                float* __restrict__ y_r, float* __restrict__ stats, int64_t rows,
+                                int cols, float eps) {
+  __shared__ float red[33];
+  const int64_t row = blockIdx.x;
+  const float* xr = x + row * cols;
+  float mean = 0.f;
+  if (KIND == 0) {
+    float s = 0.f;
+    for (int c = threadIdx.x * 8; c < cols; c += blockDim.x * 8) {
+      float v[8];
+      load8(xr + c, v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s += v[i];
+    }
+    mean = block_sum(s, red) / cols;
+  }
+  float q = 0.f;
+  for (int c = threadIdx.x * 8; c < cols; c += blockDim.x * 8) {
+    float v[8];
+    load8(xr + c, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q += (v[i] - mean) * (v[i] - mean);
+  }
+  const float var = block_sum(q, red) / cols;
+  const float rstd = 1.0f / sqrtf(var + eps);
+  if (threadIdx.x == 0) {
+    stats[row] = mean;
+    stats[rows + row] = rstd;
+  }
+  for (int c = threadIdx.x * 8; c < cols; c += blockDim.x * 8) {
+    float v[8], g[8];
+    load8(xr + c, v);
+    load8(gain + c, g);
+    if (KIND == 0) {
+      float b[8];
+      load8(bias + c, b);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = (v[i] - mean) * rstd * g[i] + b[i];
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = v[i] * rstd * g[i];
+    }
+    store8(y_a + row * cols + c, v);
+    if (y_r) store8(y_r + row * cols + c, v);
+  }
+}
+
+// dx = norm_bwd(dy; x, stats, gain) (+ add).  One block per row.  dy is either a GEMM
+// output (type P) or a residual-stream gradient (fp32).  dx_r: fp32 stream gradient;
+// dx_a (optional): the same values rounded once to the GEMM-operand type.
+template <typename DY, typename P, int KIND>
+__global__ void norm_bwd_dx_kernel(const DY* __restrict__ dy, const float* __restrict__ x,
+                                   const float* __restrict__ stats, const P* __restrict__ gain,
+                                   const float* __restrict__ add, float* __restrict__ dx_r,
+                                   P* __restrict__ dx_a, int64_t rows, int cols) {
+  __shared__ float red[33];
+  const int64_t row = blockIdx.x;
+  const float mean = stats[row], rstd = stats[rows + row];
+  const DY* dyr = dy + row * cols;
+  const float* xr = x + row * cols;
+  float s1 = 0.f, s2 = 0.f;
+  for (int c = threadIdx.x * 8; c < cols; c += blockDim.x * 8) {
+    float a[8], v[8], g[8];
+    load8(dyr + c, a);
+    load8(xr + c, v);
+    load8(gain + c, g);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float dxh = a[i] * g[i];
+      if (KIND == 0) {
+        s1 += dxh;
+        s2 += dxh * (v[i] - mean) * rstd;
+      } else {
+        s2 += dxh * v[i];
+      }
+    }
+  }
+  if (KIND == 0) s1 = block_sum(s1, red) / cols;
+  s2 = block_sum(s2, red) / cols;
+  const float* ar = add ? add + row * cols : nullptr;
+  for (int c = threadIdx.x * 8; c < cols; c += blockDim.x * 8) {
+    float a[8], v[8], g[8], o[8];
+    load8(dyr + c, a);
+    load8(xr + c, v);
+    load8(gain + c, g);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float dxh = a[i] * g[i];
+      if (KIND == 0) {
+        const float xh = (v[i] - mean) * rstd;
+        o[i] = rstd * (dxh - s1 - xh * s2);
+      } else {
+        o[i] = rstd * dxh - v[i] * rstd * rstd * rstd * s2;
+      }
+    }
+    if (ar) {
+      float r[8];
+      load8(ar + c, r);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[i] += r[i];
+    }
+    if (dx_r) store8(dx_r + row * cols + c, o);
+    if (dx_a) store8(dx_a + row * cols + c, o);
+  }
+}
+
+// ------------------------------------------------------------------ column reductions
+// Stage 1: partial[chunk][col] over a slab of rows.  MODE 0: sum dy (bias gradient).
+// MODE 1: LayerNorm: p0 = sum dy*xhat, p1 = sum dy.  MODE 2: RMSNorm: p0 = sum dy*x*rstd.
+// Block = 32 x 8 threads over 32 columns; grid = (ceil(cols/32), n_chunks).
+// partial layout: [2][n_chunks][cols].  x is the fp32 residual stream.  With fp32 dy the
+// sums run in double: these sums cancel heavily and the fp32 configuration is held to 1e-5.
+constexpr int kColChunks = 64;
+template <typename T> struct ColAcc { typedef float type; };
+template <> struct ColAcc<float> { typedef double type; };
+template <typename DY, int MODE>
+__global__ void colreduce_stage1_kernel(const DY* __restrict__ dy, int64_t ld,
+                                        const float* __restrict__ x, const float* __restrict__ stats,
+                                        float* __restrict__ partial, int64_t rows, int cols) {
+  typedef typename ColAcc<DY>::type acc_t;
+  __shared__ acc_t sh0[8][33], sh1[8][33];
+  const int col = blockIdx.x * 32 + threadIdx.x;
+  const int nch = gridDim.y;
+  const int64_t per = (rows + nch - 1) / nch;
+  const int64_t r0 = (int64_t)blockIdx.y * per;
+  const int64_t r1 = r0 + per < rows ? r0 + per : rows;
+  acc_t a0 = 0, a1 = 0;
+  if (col < cols) {
+    for (int64_t r = r0 + threadIdx.y; r < r1; r += 8) {
+      const float g = to_f(dy[r * ld + col]);
+      if (MODE == 0) {
+        a0 += g;
+      } else if (MODE == 1) {
+        const float xh = (x[r * cols + col] - stats[r]) * stats[rows + r];
+        a0 += (acc_t)g * xh;
+        a1 += g;
+      } else {
+        a0 += (acc_t)g * (x[r * cols + col] * stats[rows + r]);
+      }
+    }
+  }
+  sh0[threadIdx.y][threadIdx.x] = a0;
+  sh1[threadIdx.y][threadIdx.x] = a1;
+  __syncthreads();
+  if (threadIdx.y == 0 && col < cols) {
+    acc_t t0 = 0, t1 = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      t0 += sh0[i][threadIdx.x];
+      t1 += sh1[i][threadIdx.x];
+    }
+    partial[((size_t)0 * nch + blockIdx.y) * cols + col] = (float)t0;
+    if (MODE == 1) partial[((size_t)1 * nch + blockIdx.y) * cols + col] = (float)t1;
+  }
+}
+// Stage 2: out0[col] = sum_chunk partial[0][chunk][col] (and out1 likewise from plane 1).
+__global__ void colreduce_stage2_kernel(const float* __restrict__ partial, int nch, int cols,
+                                        float* __restrict__ out0, float* __restrict__ out1) {
+  const int col = blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= cols) return;
+  double t0 = 0.0, t1 = 0.0;
+  for (int c = 0; c < nch; ++c) {
+    t0 += partial[((size_t)c) * cols + col];
+    if (out1) t1 += partial[((size_t)nch + c) * cols + col];
+  }
+  out0[col] = (float)t0;
+  if (out1) out1[col] = (float)t1;
+}
+
+// ------------------------------------------------------------------ activations
+__device__ __forceinline__ float gelu_f(float a) {
+  return 0.5f * a * (1.0f + erff(a * 0.70710678118654752440f));
+}
+__device__ __forceinline__ float gelu_grad_f(float a) {
+  const float cdf = 0.5f * (1.0f + erff(a * 0.70710678118654752440f));
+  const float pdf = expf(-0.5f * a * a) * 0.39894228040143267794f;
+  return cdf + a * pdf;
+}
+template <typename T>
+__global__ void gelu_fwd_kernel(const T* __restrict__ a, T* __restrict__ u, size_t n8) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n8; i += stride) {
+    float v[8];
+    load8(a + i * 8, v);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = gelu_f(v[j]);
+    store8(u + i * 8, v);
+  }
+}
+// du <- du * gelu'(a), in place
+template <typename T>
+__global__ void gelu_bwd_kernel(T* __restrict__ du, const T* __restrict__ a, size_t n8) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n8; i += stride) {
+    float v[8], g[8];
+    load8(a + i * 8, v);
+    load8(du + i * 8, g);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) g[j] *= gelu_grad_f(v[j]);
+    store8(du + i * 8, g);
+  }
+}
+// s[t,j] = silu(gu[t,j]) * gu[t,f+j];  f % 8 == 0
+template <typename T>
+__global__ void swiglu_fwd_kernel(const T* __restrict__ gu, T* __restrict__ s, int64_t rows, int f) {
+  const size_t f8 = f / 8, n8 = (size_t)rows * f8;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n8; i += stride) {
+    const size_t r = i / f8, c = (i % f8) * 8;
+    float g[8], u[8];
+    load8(gu + r * 2 * f + c, g);
+    load8(gu + r * 2 * f + f + c, u);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) g[j] = g[j] / (1.0f + expf(-g[j])) * u[j];
+    store8(s + r * f + c, g);
+  }
+}
+// dgu[t,j] = ds*up*sig*(1+g(1-sig)); dgu[t,f+j] = ds*g*sig
+template <typename T>
+__global__ void swiglu_bwd_kernel(const T* __restrict__ ds, const T* __restrict__ gu,
+                                  T* __restrict__ dgu, int64_t rows, int f) {
+  const size_t f8 = f / 8, n8 = (size_t)rows * f8;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n8; i += stride) {
+    const size_t r = i / f8, c = (i % f8) * 8;
+    float g[8], u[8], d[8], o0[8], o1[8];
+    load8(gu + r * 2 * f + c, g);
+    load8(gu + r * 2 * f + f + c, u);
+    load8(ds + r * f + c, d);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float sig = 1.0f / (1.0f + expf(-g[j]));
+      o0[j] = d[j] * u[j] * sig * (1.0f + g[j] * (1.0f - sig));
+      o1[j] = d[j] * g[j] * sig;
+    }
+    store8(dgu + r * 2 * f + c, o0);
+    store8(dgu + r * 2 * f + f + c, o1);
+  }
+}
+
+// ------------------------------------------------------------------ RoPE
+// In place on the q and k column blocks of qkv[T,3d]: pair (j, j+half) of every head rotated
+// by angle(pos, j) (sign = +1) or its inverse (sign = -1).  cs: [S, half] cos | [S, half] sin.
+template <typename T>
+__global__ void rope_kernel(T* __restrict__ qkv, const float* __restrict__ cs, int64_t Ttot, int S,
+                            int H, int dh, float sign) {
+  const int half = dh / 2;
+  const size_t n = (size_t)Ttot * H * half;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  const int d = H * dh;
+  for (; i < n; i += stride) {
+    const int j = i % half;
+    const int h = (i / half) % H;
+    const size_t t = i / ((size_t)half * H);
+    const int pos = t % S;
+    const float c = cs[(size_t)pos * half + j];
+    const float s = sign * cs[(size_t)S * half + (size_t)pos * half + j];
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {          // q then k
+      T* p = qkv + t * 3 * d + (size_t)part * d + (size_t)h * dh;
+      const float x1 = to_f(p[j]), x2 = to_f(p[j + half]);
+      p[j] = from_f<T>(x1 * c - x2 * s);
+      p[j + half] = from_f<T>(x1 * s + x2 * c);
+    }
+  }
+}
+
+// ------------------------------------------------------------------ softmax cross-entropy
+// nvalid[0] = number of labels >= 0  (single block)
+__global__ void count_valid_kernel(const int32_t* __restrict__ labels, int64_t n, int* nvalid) {
+  __shared__ float red[33];
+  float c = 0.f;
+  for (int64_t i = threadIdx.x; i < n; i += blockDim.x) c += labels[i] >= 0 ? 1.f : 0.f;
+  c = block_sum(c, red);
+  if (threadIdx.x == 0) nvalid[0] = (int)(c + 0.5f);
+}
+// One block per row.  rowloss[row] = lse - logit[label] (0 if ignored); logits overwritten by
+// (softmax - onehot)/nvalid, zeros for ignored rows and padding columns.  A label >= vocab sets
+// *bad = 1 and the row is treated as ignored.
+template <typename T>
+__global__ void cross_entropy_kernel(T* __restrict__ logits, const int32_t* __restrict__ labels,
+                                     float* __restrict__ rowloss, const int* __restrict__ nvalid,
+                                     int* __restrict__ bad, int64_t vocab, int64_t ld) {
+  __shared__ float red[33];
+  const int64_t row = blockIdx.x;
+  T* lr = logits + row * ld;
+  int label = labels[row];
+  if (label >= vocab) {
+    if (threadIdx.x == 0) *bad = 1;
+    label = -1;
+  }
+  if (label < 0) {
+    for (int64_t c = threadIdx.x; c < ld; c += blockDim.x) lr[c] = from_f<T>(0.f);
+    if (threadIdx.x == 0) rowloss[row] = 0.f;
+    return;
+  }
+  float mx = -INFINITY;
+  for (int64_t c = threadIdx.x; c < vocab; c += blockDim.x) mx = fmaxf(mx, to_f(lr[c]));
+  mx = block_max(mx, red);
+  float se = 0.f;
+  for (int64_t c = threadIdx.x; c < vocab; c += blockDim.x) se += expf(to_f(lr[c]) - mx);
+  se = block_sum(se, red);
+  const float lse = mx + logf(se);
+  const float inv_n = 1.0f / (float)nvalid[0];
+  if (threadIdx.x == 0) rowloss[row] = lse - to_f(lr[label]);
+  __syncthreads();
+  for (int64_t c = threadIdx.x; c < ld; c += blockDim.x) {
+    float g = 0.f;
+    if (c < vocab) {
+      g = expf(to_f(lr[c]) - lse);
+      if (c == label) g -= 1.0f;
+      g *= inv_n;
+    }
+    lr[c] = from_f<T>(g);
+  }
+}
+// loss = sum(rowloss)/nvalid  (single block, fixed order)
+__global__ void loss_reduce_kernel(const float* __restrict__ rowloss, int64_t rows,
+                                   const int* __restrict__ nvalid, float* __restrict__ loss) {
+  __shared__ float red[33];
+  float s = 0.f;
+  for (int64_t i = threadIdx.x; i < rows; i += blockDim.x) s += rowloss[i];
+  s = block_sum(s, red);
+  if (threadIdx.x == 0) loss[0] = s / (float)nvalid[0];
+}
+
+// ------------------------------------------------------------------ fused group optimizer
+// One streaming pass over the group's flat buffers: 128-bit loads/stores, 4 elements per
+// thread per iteration.  KIND 0 AdamW, 1 AdaGrad, 2 SGD-momentum.  Scalars precomputed on the
+// host in double: decay = 1 - lr*wd, omb1 = 1-beta1, omb2 = 1-beta2, c1 = 1/(1-beta1^tau),
+// c2 = 1/(1-beta2^tau).  IEEE sqrt and division.
+struct OptScalars {
+  float lr, beta1, beta2, eps, decay, omb1, omb2, c1, c2, mu;
+};
+template <int KIND>
+__device__ __forceinline__ void opt_update(float& th, float g, float& s0, float& s1,
+                                           const OptScalars& h) {
+  if (KIND == 0) {
+    th = th * h.decay;
+    s0 = h.beta1 * s0 + h.omb1 * g;
+    s1 = h.beta2 * s1 + h.omb2 * g * g;
+    const float mhat = s0 * h.c1;
+    const float vhat = s1 * h.c2;
+    th = th - __fdiv_rn(h.lr * mhat, __fsqrt_rn(vhat) + h.eps);
+  } else if (KIND == 1) {
+    s0 = s0 + g * g;
+    th = th - __fdiv_rn(h.lr * g, __fsqrt_rn(s0) + h.eps);
+  } else {
+    s0 = h.mu * s0 + g;
+    th = th - h.lr * s0;
+  }
+}
+template <int KIND, bool HAS_BF16>
+__global__ void __launch_bounds__(256)
+fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const float* __restrict__ grad,
+                 float* __restrict__ s0, float* __restrict__ s1, size_t n, OptScalars h) {
+  const size_t n4 = n / 4;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (; i < n4; i += stride) {
+    float4 th = reinterpret_cast<const float4*>(master)[i];
+    const float4 g = __ldcs(reinterpret_cast<const float4*>(grad) + i);
+    float4 a = reinterpret_cast<const float4*>(s0)[i];
+    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (KIND == 0) b = reinterpret_cast<const float4*>(s1)[i];
+    opt_update<KIND>(th.x, g.x, a.x, b.x, h);
+    opt_update<KIND>(th.y, g.y, a.y, b.y, h);
+    opt_update<KIND>(th.z, g.z, a.z, b.z, h);
+    opt_update<KIND>(th.w, g.w, a.w, b.w, h);
+    reinterpret_cast<float4*>(master)[i] = th;
+    reinterpret_cast<float4*>(s0)[i] = a;
+    if (KIND == 0) reinterpret_cast<float4*>(s1)[i] = b;
+    if (HAS_BF16) {
+      uint2 pk;
+      __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y), hi = __floats2bfloat162_rn(th.z, th.w);
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(param)[i] = pk;
+    }
+  }
+  // ragged tail (n not a multiple of 4)
+  const size_t t = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) {
+    float th = master[t], a = s0[t], b = (KIND == 0) ? s1[t] : 0.f;
+    opt_update<KIND>(th, grad[t], a, b, h);
+    master[t] = th;
+    s0[t] = a;
+    if (KIND == 0) s1[t] = b;
+    if (HAS_BF16) param[t] = __float2bfloat16_rn(th);
+  }
+}
+
+}  // namespace hift

@@ -1,0 +1,173 @@
+// Host-side launch wrappers: pick the template instance for the dtype / head size and the
+// grid.  Shared by the training-step engine and the single-kernel C entry points.
+#pragma once
+#include "gemm_args.h"
+#include "kernels_attention.cuh"
+#include "kernels_gemm_simt.cuh"
+#include "kernels_pointwise.cuh"
+
+namespace hift {
+
+inline int grid_for(size_t n, int block, int max_blocks = 148 * 16) {
+  size_t g = (n + block - 1) / block;
+  if (g < 1) g = 1;
+  if (g > (size_t)max_blocks) g = max_blocks;
+  return (int)g;
+}
+inline int norm_threads(int cols) {
+  int t = ((cols / 8 + 31) / 32) * 32;
+  if (t < 32) t = 32;
+  if (t > 256) t = 256;
+  return t;
+}
+
+// ---- GEMM (CUDA cores) ----------------------------------------------------------
+inline void launch_gemm_simt(cudaStream_t st, int dtype, const GemmArgs& g) {
+  dim3 grid((g.N + 63) / 64, (g.M + 63) / 64);
+  if (dtype == 0) {
+    gemm_simt_kernel<float, float><<<grid, 256, 0, st>>>(
+        g.M, g.N, g.K, (const float*)g.a, g.sam, g.sak, (const float*)g.b, g.sbk, g.sbn,
+        (float*)g.c, g.ldc, (const float*)g.bias, g.residual, g.ldr);
+  } else if (g.out_f32) {
+    gemm_simt_kernel<bf16, float><<<grid, 256, 0, st>>>(
+        g.M, g.N, g.K, (const bf16*)g.a, g.sam, g.sak, (const bf16*)g.b, g.sbk, g.sbn,
+        (float*)g.c, g.ldc, (const bf16*)g.bias, g.residual, g.ldr);
+  } else {
+    gemm_simt_kernel<bf16, bf16><<<grid, 256, 0, st>>>(
+        g.M, g.N, g.K, (const bf16*)g.a, g.sam, g.sak, (const bf16*)g.b, g.sbk, g.sbn,
+        (bf16*)g.c, g.ldc, (const bf16*)g.bias, nullptr, 0);
+  }
+}
+
+// ---- attention ------------------------------------------------------------------
+inline bool attention_head_ok(int dh) { return dh == 8 || dh == 16 || dh == 32 || dh == 64 || dh == 128; }
+
+template <typename T, int DH>
+inline void attention_fwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv,
+                               void* o, float* lse) {
+  dim3 grid((S + kAttRows - 1) / kAttRows, H, B);
+  attention_fwd_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, (T*)o, lse, S, H, causal,
+                                                    1.0f / sqrtf((float)DH));
+}
+template <typename T, int DH>
+inline void attention_bwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv,
+                               const void* o, const float* lse, const void* dout, void* dqkv,
+                               float* dsum) {
+  dim3 grid((S + kAttRows - 1) / kAttRows, H, B);
+  const float scale = 1.0f / sqrtf((float)DH);
+  attention_bwd_dq_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, (const T*)o, lse,
+                                                       (const T*)dout, (T*)dqkv, dsum, S, H, causal, scale);
+  attention_bwd_dkv_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, lse, (const T*)dout, dsum,
+                                                        (T*)dqkv, S, H, causal, scale);
+}
+#define HIFT_DH_SWITCH(dh, CALL)            \
+  switch (dh) {                             \
+    case 8: { CALL(8); break; }             \
+    case 16: { CALL(16); break; }           \
+    case 32: { CALL(32); break; }           \
+    case 64: { CALL(64); break; }           \
+    case 128: { CALL(128); break; }         \
+    default: break;                         \
+  }
+inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
+                                 const void* qkv, void* o, float* lse) {
+#define CALL_F(D)                                                              \
+  if (dtype == 0) attention_fwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse); \
+  else attention_fwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse)
+  HIFT_DH_SWITCH(dh, CALL_F)
+#undef CALL_F
+}
+inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
+                                 const void* qkv, const void* o, const float* lse, const void* dout,
+                                 void* dqkv, float* dsum) {
+#define CALL_B(D)                                                                              \
+  if (dtype == 0) attention_bwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum); \
+  else attention_bwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum)
+  HIFT_DH_SWITCH(dh, CALL_B)
+#undef CALL_B
+}
+
+// ---- norms ----------------------------------------------------------------------
+// dtype 0: parameters fp32; 1: parameters / GEMM operands bf16.  x and y_r are fp32.
+inline void launch_norm_fwd(cudaStream_t st, int dtype, int kind, int64_t rows, int cols, float eps,
+                            const float* x, const void* gain, const void* bias, void* y_a, float* y_r,
+                            float* stats) {
+  const int th = norm_threads(cols);
+#define NF(P, K) norm_fwd_kernel<P, K><<<(unsigned)rows, th, 0, st>>>(x, (const P*)gain, (const P*)bias, (P*)y_a, y_r, stats, rows, cols, eps)
+  if (dtype == 0) { if (kind == 0) NF(float, 0); else NF(float, 1); }
+  else { if (kind == 0) NF(bf16, 0); else NF(bf16, 1); }
+#undef NF
+}
+// dy_f32: dy is an fp32 stream gradient (else it has the operand type)
+inline void launch_norm_bwd_dx(cudaStream_t st, int dtype, int kind, bool dy_f32, int64_t rows, int cols,
+                               const void* dy, const float* x, const float* stats, const void* gain,
+                               const float* add, float* dx_r, void* dx_a) {
+  const int th = norm_threads(cols);
+#define NB(DY, P, K) norm_bwd_dx_kernel<DY, P, K><<<(unsigned)rows, th, 0, st>>>((const DY*)dy, x, stats, (const P*)gain, add, dx_r, (P*)dx_a, rows, cols)
+  if (dtype == 0) { if (kind == 0) NB(float, float, 0); else NB(float, float, 1); }
+  else if (dy_f32) { if (kind == 0) NB(float, bf16, 0); else NB(float, bf16, 1); }
+  else { if (kind == 0) NB(bf16, bf16, 0); else NB(bf16, bf16, 1); }
+#undef NB
+}
+// mode 0: out0 = colsum(dy) ; 1: out0 = sum dy*xhat, out1 = sum dy ; 2: out0 = sum dy*x*rstd
+// dy_bf16: dy has type bf16 (else fp32); x is fp32.
+inline int colreduce_chunks(int64_t rows) {
+  int c = (int)((rows + 31) / 32);
+  if (c < 1) c = 1;
+  if (c > kColChunks) c = kColChunks;
+  return c;
+}
+inline void launch_colreduce(cudaStream_t st, bool dy_bf16, int mode, int64_t rows, int cols,
+                             const void* dy, int64_t ld, const float* x, const float* stats,
+                             float* partial, float* out0, float* out1) {
+  const int nch = colreduce_chunks(rows);
+  dim3 grid((cols + 31) / 32, nch), block(32, 8);
+#define CR(T, M) colreduce_stage1_kernel<T, M><<<grid, block, 0, st>>>((const T*)dy, ld, x, stats, partial, rows, cols)
+  if (!dy_bf16) { if (mode == 0) CR(float, 0); else if (mode == 1) CR(float, 1); else CR(float, 2); }
+  else { if (mode == 0) CR(bf16, 0); else if (mode == 1) CR(bf16, 1); else CR(bf16, 2); }
+#undef CR
+  colreduce_stage2_kernel<<<(cols + 127) / 128, 128, 0, st>>>(partial, nch, cols, out0,
+                                                             mode == 1 ? out1 : nullptr);
+}
+
+// ---- cross-entropy --------------------------------------------------------------
+inline void launch_cross_entropy(cudaStream_t st, int dtype, int64_t rows, int64_t vocab, int64_t ld,
+                                 void* logits, const int32_t* labels, float* rowloss, int* nvalid,
+                                 int* bad, float* loss) {
+  count_valid_kernel<<<1, 256, 0, st>>>(labels, rows, nvalid);
+  const int th = vocab >= 4096 ? 512 : (vocab >= 256 ? 128 : 32);
+  if (dtype == 0)
+    cross_entropy_kernel<float><<<(unsigned)rows, th, 0, st>>>((float*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+  else
+    cross_entropy_kernel<bf16><<<(unsigned)rows, th, 0, st>>>((bf16*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+  loss_reduce_kernel<<<1, 256, 0, st>>>(rowloss, rows, nvalid, loss);
+}
+
+// ---- optimizer ------------------------------------------------------------------
+inline OptScalars make_opt_scalars(int kind, double lr, double b1, double b2, double eps, double wd,
+                                   double mu, int64_t tau) {
+  OptScalars h;
+  h.lr = (float)lr; h.beta1 = (float)b1; h.beta2 = (float)b2; h.eps = (float)eps;
+  h.decay = (float)(1.0 - lr * wd);
+  h.omb1 = (float)(1.0 - b1); h.omb2 = (float)(1.0 - b2);
+  h.c1 = 1.f; h.c2 = 1.f;
+  if (kind == 0) {
+    h.c1 = (float)(1.0 / (1.0 - pow(b1, (double)tau)));
+    h.c2 = (float)(1.0 / (1.0 - pow(b2, (double)tau)));
+  }
+  h.mu = (float)mu;
+  return h;
+}
+inline void launch_fused_opt(cudaStream_t st, int kind, size_t n, void* param_bf16, float* master,
+                             const float* grad, float* s0, float* s1, const OptScalars& h) {
+  if (n == 0) return;
+  const int block = 256;
+  int grid = grid_for((n + 3) / 4, block, 148 * 8);
+#define OPT(K)                                                                                         \
+  if (param_bf16) fused_opt_kernel<K, true><<<grid, block, 0, st>>>((bf16*)param_bf16, master, grad, s0, s1, n, h); \
+  else fused_opt_kernel<K, false><<<grid, block, 0, st>>>(nullptr, master, grad, s0, s1, n, h)
+  if (kind == 0) { OPT(0); } else if (kind == 1) { OPT(1); } else { OPT(2); }
+#undef OPT
+}
+
+}  // namespace hift

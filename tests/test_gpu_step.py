@@ -1,0 +1,127 @@
+"""Whole-step parity of the CUDA library against the fp64 oracle (through the C ABI)."""
+import numpy as np
+import pytest
+
+import synth
+from gpu_util import lockstep
+
+pytestmark = pytest.mark.gpu
+
+FP32_LOSS, FP32_GRAD = 1e-5, 1e-5
+BF16_LOSS, BF16_GRAD = 1e-2, 2e-2
+
+
+def mini(arch, dtype, **kw):
+    base = dict(arch=arch, n_blocks=3, d_model=64, n_heads=4, d_ffn=128, vocab=203, max_pos=48,
+                n_classes=2 if arch == 1 else 0, causal=0 if arch == 1 else 1, tie_head=0,
+                norm_eps=1e-6 if arch == 2 else 1e-5, dtype=dtype, batch=3, seq=40, init_std=0.08)
+    base.update(kw)
+    return synth.ModelCfg(**base)
+
+
+def test_config1_tiny_fp32_full_cycle():
+    cfg, gc, oc = synth.config_tiny_fp32()
+    rep = lockstep(cfg, gc, oc, 6, "uniform", FP32_LOSS, FP32_GRAD, perturb=0.0, check_update=1e-3, resync=True)
+    assert [g for _, g, _, _, _ in rep] == [0, 1, 2, 3, 4, 5]
+
+
+def test_config1_second_cycle_bias_correction():
+    cfg, gc, oc = synth.config_tiny_fp32()
+    lockstep(cfg, gc, oc, 8, "uniform", FP32_LOSS, FP32_GRAD, perturb=0.05, check_update=1e-3, resync=True)
+
+
+@pytest.mark.parametrize("arch", [0, 1, 2])
+@pytest.mark.parametrize("order", [0, 1, 2])
+def test_mini_fp32_all_archs_orders(arch, order):
+    cfg = mini(arch, synth.DTYPE_FP32, tie_head=1 if arch == 0 else 0)
+    gc = synth.GroupCfg(layers_per_group=1, order=order, order_seed=11)
+    oc = synth.OptCfg(kind=order, lr=1e-3, weight_decay=0.01, eps=1e-8, sched=1, total_cycles=3)
+    lockstep(cfg, gc, oc, 7, "zipf", FP32_LOSS, FP32_GRAD, check_update=2e-3, resync=True)
+
+
+@pytest.mark.parametrize("arch", [0, 1, 2])
+def test_mini_fp32_grouped_and_split(arch):
+    cfg = mini(arch, synth.DTYPE_FP32, n_blocks=4)
+    lockstep(cfg, synth.GroupCfg(layers_per_group=2, split_emb_head=1, order=2, order_seed=3),
+             synth.OptCfg(kind=0, lr=1e-3), 4, "zipf", FP32_LOSS, FP32_GRAD, resync=True)
+    lockstep(cfg, synth.GroupCfg(layers_per_group=4, split_emb_head=0, order=1),
+             synth.OptCfg(kind=2, lr=1e-3), 2, "zipf", FP32_LOSS, FP32_GRAD, resync=True)
+    # one group holding every unit: the ordinary full-parameter step
+    lockstep(cfg, synth.GroupCfg(layers_per_group=6), synth.OptCfg(kind=1, lr=1e-2, eps=1e-10), 2, "zipf",
+             FP32_LOSS, FP32_GRAD, resync=True)
+
+
+@pytest.mark.parametrize("arch", [0, 1, 2])
+@pytest.mark.parametrize("offload,prefetch", [(0, 0), (1, 0), (1, 1)])
+def test_mini_bf16_paging_modes(arch, offload, prefetch):
+    cfg = mini(arch, synth.DTYPE_BF16, tie_head=1 if arch == 0 else 0)
+    gc = synth.GroupCfg(layers_per_group=1, order=0)
+    oc = synth.OptCfg(kind=0, lr=1e-3, weight_decay=0.01, offload_state=offload, prefetch_groups=prefetch)
+    lockstep(cfg, gc, oc, 7, "zipf", BF16_LOSS, BF16_GRAD, resync=True)
+
+
+@pytest.mark.parametrize("kind", [1, 2])
+def test_mini_bf16_gpt2_style_groups(kind):
+    cfg = mini(0, synth.DTYPE_BF16, n_blocks=4, tie_head=1, d_model=128, n_heads=2, d_ffn=256)
+    gc = synth.GroupCfg(layers_per_group=2, split_emb_head=1, order=2, order_seed=2401)
+    oc = synth.OptCfg(kind=kind, lr=1e-2 if kind == 1 else 1e-3, eps=1e-10, momentum=0.9)
+    lockstep(cfg, gc, oc, 5, "zipf", BF16_LOSS, BF16_GRAD, resync=True)
+
+
+def test_free_running_trajectories_stay_close():
+    """No resynchronisation: the two trajectories only share the initial weights."""
+    cfg = mini(0, synth.DTYPE_BF16, tie_head=1)
+    lockstep(cfg, synth.GroupCfg(1), synth.OptCfg(kind=2, lr=1e-3), 10, "zipf", BF16_LOSS, 2 * BF16_GRAD)
+
+
+def test_head_dim_128_llama_shape_miniature():
+    cfg = mini(2, synth.DTYPE_BF16, n_blocks=2, d_model=256, n_heads=2, d_ffn=344, vocab=1000, batch=2, seq=72)
+    lockstep(cfg, synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-4), 4, "zipf", BF16_LOSS, BF16_GRAD, resync=True)
+
+
+def test_invalid_inputs_are_reported_not_faulted():
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError
+    cfg, gc, oc = synth.config_tiny_fp32()
+    with pytest.raises(HiftError):
+        HiFT(cfg.scaled(d_model=130), gc, oc)            # not a multiple of 8
+    with pytest.raises(HiftError):
+        HiFT(cfg.scaled(max_pos=8), gc, oc)              # position table shorter than seq
+    h = HiFT(cfg, gc, oc)
+    h.set_params(synth.init_params(cfg, 0))
+    tok, lab = synth.lm_batch(cfg, 0, 0, "uniform")
+    bad = tok.copy()
+    bad[0, 0] = cfg.vocab + 5
+    with pytest.raises(HiftError) as e:
+        h.step_host(bad, lab)
+    assert e.value.status == 4 and h.step_count() == 0   # rejected on the host, nothing ran
+    with pytest.raises(HiftError) as e:
+        h.step(torch.from_numpy(bad).cuda(), torch.from_numpy(lab).cuda())
+    assert e.value.status == 4                            # clamped on the device and reported
+    loss = h.step_host(tok, lab)                          # the context is still usable
+    assert np.isfinite(loss)
+    h.close()
+
+
+def test_step_host_matches_step_and_is_deterministic():
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(0, synth.DTYPE_BF16, tie_head=1)
+    gc, oc = synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3)
+    p0 = synth.init_params(cfg, 4)
+    outs = []
+    for mode in ("dev", "host", "dev"):
+        h = HiFT(cfg, gc, oc)
+        h.set_params(p0)
+        losses = []
+        for t in range(5):
+            tok, lab = synth.lm_batch(cfg, 9, t)
+            if mode == "dev":
+                losses.append(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
+            else:
+                losses.append(h.step_host(tok, lab))
+        outs.append((losses, h.get_param("tok_emb"), h.get_param("b0.w_qkv")))
+        h.close()
+    for o in outs[1:]:
+        assert o[0] == outs[0][0]                         # same bits, run to run and across entry points
+        assert np.array_equal(o[1], outs[0][1]) and np.array_equal(o[2], outs[0][2])
