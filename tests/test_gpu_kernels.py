@@ -1,0 +1,228 @@
+"""Per-kernel parity through the C ABI: each kernel against the oracle's fp64 definition of
+the same operation, at shapes that span several tiles and a ragged tail, plus edge cases."""
+import numpy as np
+import pytest
+
+import synth
+from gpu_util import rel_l2
+from oracle import hift_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _t(a, dtype=None):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t if dtype is None else t.to(dtype)
+
+
+def _bf(a):
+    """bf16-rounded fp64 copy of an fp32 array (what the oracle sees of a bf16 operand)."""
+    return O.bf16_round(np.asarray(a, dtype=np.float32)).astype(np.float64)
+
+
+# ------------------------------------------------------------------ optimizer: 1e-6
+@pytest.mark.parametrize("kind", [0, 1, 2])
+@pytest.mark.parametrize("n", [1, 3, 1000, 4099, (1 << 20) + 5])
+def test_fused_optimizer_matches_oracle_1e6(kind, n):
+    import torch
+    from paper_2401_15207_b200 import opt_step
+    master, grad, s0, s1 = synth.flat_optimizer_inputs(n, seed=kind * 100 + 7, warm=True)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01, momentum=0.9)
+    if kind == 1:
+        hp.update(lr=1e-2, eps=1e-10)
+        s0 = np.abs(s0).astype(np.float32) ** 2            # accumulator is non-negative
+    tm, tg, ts0, ts1 = _t(master), _t(grad), _t(s0), _t(s1)
+    tp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    m64, g64, a64, b64 = (x.astype(np.float64) for x in (master, grad, s0, s1))
+    for tau in (3, 4):                                      # two consecutive updates, warm state
+        opt_step(kind, n, tp, tm, tg, ts0, ts1, tau=tau, **hp)
+        if kind == 0:
+            m64, a64, b64 = O.adamw_update(m64, g64, a64, b64, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                           hp["weight_decay"], tau)
+        elif kind == 1:
+            m64, a64 = O.adagrad_update(m64, g64, a64, hp["lr"], hp["eps"])
+        else:
+            m64, a64 = O.sgdm_update(m64, g64, a64, hp["lr"], hp["momentum"])
+    torch.cuda.synchronize()
+    gm = tm.cpu().numpy()
+    assert rel_l2(gm, m64) <= 1e-6
+    assert rel_l2(ts0.cpu().numpy(), a64) <= 1e-6
+    if kind == 0:
+        assert rel_l2(ts1.cpu().numpy(), b64) <= 1e-6
+    # the update itself (theta_new - theta_old): 1e-4 relative plus the rounding of the fp32
+    # value it is stored in (half an ulp of theta per update; the subtraction cancels)
+    delta, delta_ref = gm.astype(np.float64) - master, m64 - master
+    assert np.linalg.norm(delta - delta_ref) <= 1e-4 * np.linalg.norm(delta_ref) + 2 * 6e-8 * np.linalg.norm(master)
+    # the bf16 model copy is the round-to-nearest-even image of the fp32 master, bit for bit
+    assert np.array_equal(tp.float().cpu().numpy(), O.bf16_round(gm))
+
+
+def test_fused_optimizer_fp32_params_and_argument_checks():
+    import torch
+    from paper_2401_15207_b200 import opt_step, HiftError
+    n = 777
+    master, grad, s0, s1 = synth.flat_optimizer_inputs(n, seed=3)
+    tm, tg, ts0, ts1 = _t(master), _t(grad), _t(s0), _t(s1)
+    opt_step(0, n, None, tm, tg, ts0, ts1, lr=1e-3, weight_decay=0.01, tau=1)
+    ref, _, _ = O.adamw_update(master.astype(np.float64), grad.astype(np.float64), 0.0, 0.0, 1e-3, 0.9, 0.999,
+                               1e-8, 0.01, 1)
+    assert rel_l2(tm.cpu().numpy(), ref) <= 1e-6
+    with pytest.raises(HiftError):
+        opt_step(0, n, None, tm, tg, ts0, None, lr=1e-3)         # AdamW needs the second moment
+    with pytest.raises(HiftError):
+        opt_step(0, n - 1, None, tm[1:], tg, ts0, ts1, lr=1e-3)  # misaligned pointer
+    with pytest.raises(HiftError):
+        opt_step(5, n, None, tm, tg, ts0, ts1, lr=1e-3)
+    opt_step(2, 0, None, tm, tg, ts0, None, lr=1e-3)             # empty input is a no-op
+
+
+# ------------------------------------------------------------------ linear layers, three forms
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("M,N,K", [(70, 200, 96), (257, 129, 520), (1, 8, 8)])
+def test_linear_three_forms(dtype, M, N, K):
+    import torch
+    from paper_2401_15207_b200 import k_linear
+    rng = np.random.default_rng(M + N + K)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.1).astype(np.float32)
+    dy = rng.standard_normal((M, N)).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    td = torch.float32 if dtype == 0 else torch.bfloat16
+    tol = 2e-6 if dtype == 0 else 6e-3
+    cvt = (lambda a: a.astype(np.float64)) if dtype == 0 else _bf
+    # forward with bias
+    y = torch.empty((M, N), dtype=td, device="cuda")
+    k_linear(0, dtype, M, N, K, _t(x, td), _t(w, td), y, bias=_t(bias, td))
+    assert rel_l2(y.float().cpu().numpy(), cvt(x) @ cvt(w).T + cvt(bias)) <= tol
+    # forward into the fp32 residual stream
+    y32 = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    k_linear(0, dtype, M, N, K, _t(x, td), _t(w, td), y32, bias=_t(bias, td), residual=_t(res))
+    assert rel_l2(y32.cpu().numpy(), cvt(x) @ cvt(w).T + cvt(bias) + res) <= 2e-6 if dtype == 0 else 2e-3
+    # activation gradient
+    dx = torch.empty((M, K), dtype=td, device="cuda")
+    k_linear(1, dtype, M, N, K, _t(dy, td), _t(w, td), dx)
+    assert rel_l2(dx.float().cpu().numpy(), cvt(dy) @ cvt(w)) <= tol
+    # weight gradient (fp32 out)
+    dw = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    k_linear(2, dtype, M, N, K, _t(dy, td), _t(x, td), dw)
+    assert rel_l2(dw.cpu().numpy(), cvt(dy).T @ cvt(x)) <= 2e-6
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("dtype,dh", [(0, 32), (1, 64), (1, 128), (0, 8)])
+@pytest.mark.parametrize("causal", [0, 1])
+def test_attention_forward_backward(dtype, dh, causal):
+    import torch
+    from paper_2401_15207_b200 import k_attention_fwd, k_attention_bwd
+    B, S, H = 2, 150, 3                                     # S spans tiles of 64/32 with a ragged tail
+    d = H * dh
+    rng = np.random.default_rng(dh + causal)
+    qkv = rng.standard_normal((B * S, 3 * d)).astype(np.float32)
+    do = rng.standard_normal((B * S, d)).astype(np.float32)
+    td = torch.float32 if dtype == 0 else torch.bfloat16
+    cvt = (lambda a: a.astype(np.float64)) if dtype == 0 else _bf
+    q, k, v = (cvt(qkv)[:, i * d:(i + 1) * d].reshape(B, S, H, dh) for i in range(3))
+    o_ref, p = O.attention_fwd(q, k, v, bool(causal))
+    tq = _t(qkv, td)
+    o = torch.empty((B * S, d), dtype=td, device="cuda")
+    lse = torch.empty((B, H, S), dtype=torch.float32, device="cuda")
+    k_attention_fwd(dtype, B, S, H, dh, causal, tq, o, lse)
+    tol = 3e-6 if dtype == 0 else 6e-3
+    assert rel_l2(o.float().cpu().numpy(), o_ref.reshape(B * S, d)) <= tol
+    # log-sum-exp against its definition
+    s = np.einsum("bshe,bthe->bhst", q, k) / np.sqrt(dh)
+    if causal:
+        s = np.where(np.triu(np.ones((S, S), dtype=bool), 1), -np.inf, s)
+    lse_ref = np.log(np.exp(s - s.max(-1, keepdims=True)).sum(-1)) + s.max(-1)
+    assert np.allclose(lse.cpu().numpy(), lse_ref, rtol=1e-5, atol=1e-5)
+    # backward: feed the oracle the same (rounded) o the kernel saved
+    dqkv = torch.empty((B * S, 3 * d), dtype=td, device="cuda")
+    dsum = torch.empty(B * S * H, dtype=torch.float32, device="cuda")
+    k_attention_bwd(dtype, B, S, H, dh, causal, tq, o, lse, _t(do, td), dqkv, dsum)
+    dq, dk, dv = O.attention_bwd(cvt(do).reshape(B, S, H, dh), q, k, v, p)
+    ref = np.concatenate([t.reshape(B * S, d) for t in (dq, dk, dv)], axis=1)
+    tolb = 5e-6 if dtype == 0 else 1.2e-2
+    got = dqkv.float().cpu().numpy()
+    for i in range(3):
+        assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= tolb, i
+
+
+# ------------------------------------------------------------------ norms
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("rows,cols", [(37, 64), (300, 1280), (5, 4096)])
+def test_norm_forward_backward(dtype, kind, rows, cols):
+    import torch
+    from paper_2401_15207_b200 import k_norm_fwd, k_norm_bwd
+    rng = np.random.default_rng(rows + cols)
+    x = (rng.standard_normal((rows, cols)) * 2 + 0.3).astype(np.float32)
+    gain = (1 + 0.1 * rng.standard_normal(cols)).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(cols)).astype(np.float32)
+    dy = rng.standard_normal((rows, cols)).astype(np.float32)
+    add = rng.standard_normal((rows, cols)).astype(np.float32)
+    td = torch.float32 if dtype == 0 else torch.bfloat16
+    cvt = (lambda a: a.astype(np.float64)) if dtype == 0 else _bf
+    eps = 1e-5 if kind == 0 else 1e-6
+    y = torch.empty((rows, cols), dtype=td, device="cuda")
+    stats = torch.empty(2 * rows, dtype=torch.float32, device="cuda")
+    tx, tg, tb = _t(x), _t(gain, td), _t(bias, td)
+    k_norm_fwd(dtype, kind, rows, cols, eps, tx, tg, tb if kind == 0 else None, y, stats)
+    x64 = x.astype(np.float64)
+    if kind == 0:
+        y_ref, cache = O.layernorm_fwd(x64, cvt(gain), cvt(bias), eps)
+    else:
+        y_ref, cache = O.rmsnorm_fwd(x64, cvt(gain), eps)
+    assert rel_l2(y.float().cpu().numpy(), y_ref) <= (2e-6 if dtype == 0 else 4e-3)
+    dx = torch.empty((rows, cols), dtype=torch.float32, device="cuda")
+    dgain = torch.empty(cols, dtype=torch.float32, device="cuda")
+    dbias = torch.empty(cols, dtype=torch.float32, device="cuda")
+    partial = torch.empty(2 * 64 * cols, dtype=torch.float32, device="cuda")
+    k_norm_bwd(dtype, kind, rows, cols, _t(dy, td), tx, stats, tg, _t(add), dx, dgain,
+               dbias if kind == 0 else None, partial)
+    if kind == 0:
+        dx_ref, dg_ref, db_ref = O.layernorm_bwd(cvt(dy), cache, cvt(gain))
+        assert rel_l2(dbias.cpu().numpy(), db_ref) <= 3e-6
+    else:
+        dx_ref, dg_ref = O.rmsnorm_bwd(cvt(dy), cache, cvt(gain))
+    assert rel_l2(dx.cpu().numpy(), dx_ref + add) <= 3e-6
+    assert rel_l2(dgain.cpu().numpy(), dg_ref) <= 5e-6
+
+
+# ------------------------------------------------------------------ cross-entropy
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("rows,vocab,ld", [(64, 512, 512), (33, 50257, 50304), (16, 2, 2)])
+def test_cross_entropy(dtype, rows, vocab, ld):
+    import torch
+    from paper_2401_15207_b200 import k_cross_entropy
+    rng = np.random.default_rng(vocab)
+    logits = (rng.standard_normal((rows, ld)) * 3).astype(np.float32)
+    labels = rng.integers(0, vocab, rows).astype(np.int32)
+    if rows > 8:
+        labels[3] = -1                                       # an ignored row
+    td = torch.float32 if dtype == 0 else torch.bfloat16
+    cvt = (lambda a: a.astype(np.float64)) if dtype == 0 else _bf
+    tl = _t(logits, td)
+    rowloss = torch.empty(rows, dtype=torch.float32, device="cuda")
+    out = torch.zeros(4, dtype=torch.float32, device="cuda")
+    k_cross_entropy(dtype, rows, vocab, ld, tl, _t(labels), rowloss, out)
+    loss_ref, d_ref = O.cross_entropy(cvt(logits)[:, :vocab], labels)
+    o = out.cpu().numpy()
+    assert abs(o[0] - loss_ref) <= 2e-6 * abs(loss_ref)
+    assert o[1:3].view(np.int32).tolist() == [int((labels >= 0).sum()), 0]
+    got = tl.float().cpu().numpy()
+    assert rel_l2(got[:, :vocab], d_ref) <= (3e-6 if dtype == 0 else 4e-3)
+    assert not got[:, vocab:].any()                          # padding columns carry no gradient
+    if rows > 8:
+        assert not got[3].any()
+
+
+def test_cross_entropy_flags_bad_label():
+    import torch
+    from paper_2401_15207_b200 import k_cross_entropy
+    logits = torch.zeros((4, 8), dtype=torch.float32, device="cuda")
+    labels = _t(np.array([1, 9, 2, 3], dtype=np.int32))     # 9 >= vocab
+    out = torch.zeros(4, dtype=torch.float32, device="cuda")
+    k_cross_entropy(0, 4, 8, 8, logits, labels, torch.empty(4, device="cuda"), out)
+    assert out.cpu().numpy()[2:3].view(np.int32)[0] == 1
