@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the hierarchical fine-tuning (HiFT) step on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" = one hift_step: full forward, backward truncated at the active group, fused
+group-local optimizer, optimizer-state paging.  Default workload: the LLaMA-7B-shaped causal LM
+(32 blocks, d 4096, 32 heads, SwiGLU 11008, vocab 32000, batch 4 x seq 512, bf16 with fp32
+master, one block per group plus embedding and head groups, bottom2up, AdamW with inactive-group
+state in pinned host memory).  Prints ONE JSON line on rank 0.
+
+N > 1 runs N independent replicas (one process per GPU, no data-path collective): the step has
+no exchange inside it on one GPU, and the data-parallel variant is not built yet.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import synth
+
+WORKLOADS = {
+    "llama7b": synth.config_llama_7b,
+    "gpt2large": synth.config_gpt2_large,
+    "roberta": synth.config_roberta_base,
+    "tiny": synth.config_tiny_fp32,
+}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg, gcfg, ocfg, max_blocks=1):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: the same widths,
+    vocabulary, batch and sequence length, but only `max_blocks` transformer blocks; one step that
+    trains the top block (forward, backward through head and block, update).  Returns
+    (seconds, sample description, flops of the sample step, threads used)."""
+    from oracle import hift_oracle as O
+    nb = min(max_blocks, cfg.n_blocks)
+    big = cfg.d_model >= 2048
+    # at 7B widths the vocabulary matrices alone are 2 x 131 M fp64 values: sample one block with a
+    # 1024-entry vocabulary and one sequence, and scale by flops
+    small = cfg.scaled(n_blocks=nb, batch=1 if big else cfg.batch, vocab=1024 if big else cfg.vocab)
+    g = synth.GroupCfg(layers_per_group=1, split_emb_head=0, order=synth.ORDER_BOTTOM2UP)
+    p0 = synth.init_params(small, 0)
+    orc = O.HiFTOracle(small, g, ocfg, p0)
+    orc.t = nb                                   # group nb = the top block
+    tok, lab = synth.batch_for(small, 0, 0)
+    t0 = time.perf_counter()
+    orc.step(tok, lab)
+    dt = time.perf_counter() - t0
+    T, d, f, V = small.tokens_per_step, cfg.d_model, cfg.d_ffn, small.vocab
+    ffn = 3 if cfg.arch == synth.ARCH_LLAMA else 2
+    blk = 2.0 * T * (4 * d * d + ffn * d * f) + 4.0 * T * cfg.seq * d * (0.5 if cfg.causal else 1.0)
+    head = 2.0 * T * d * V if cfg.arch != synth.ARCH_POSTLN_ENC else 0.0
+    flops = nb * blk + head + head + 2.0 * blk    # forward, head dX, top block dX + dW
+    try:
+        threads = len(os.sched_getaffinity(0))
+    except Exception:
+        threads = os.cpu_count() or 1
+    desc = (f"fp64 oracle, one step training the top block of a {nb}-block model of the same widths "
+            f"(d={d}, f={f}, vocab {V} of {cfg.vocab}, batch {small.batch} of {cfg.batch} x seq {cfg.seq}); "
+            f"full-model figure extrapolated by flops")
+    return dt, desc, flops, threads
+
+
+def mean_step_flops(cfg, groups):
+    """Algorithmic flops of a HiFT step averaged over one cycle of groups (GEMM + attention)."""
+    T, d, f, V, L = cfg.tokens_per_step, cfg.d_model, cfg.d_ffn, cfg.vocab, cfg.n_blocks
+    ffn = 3 if cfg.arch == synth.ARCH_LLAMA else 2
+    blk_lin = 2.0 * T * (4 * d * d + ffn * d * f)
+    blk_att = 4.0 * T * cfg.seq * d * (0.5 if cfg.causal else 1.0)
+    head = 2.0 * T * d * V if cfg.arch != synth.ARCH_POSTLN_ENC else 0.0
+    fwd = L * (blk_lin + blk_att) + head
+    tot = 0.0
+    for lo, hi in groups:
+        fl = fwd
+        if lo <= L:                                       # something below the head is trained
+            fl += head                                    # head dX
+        head_w = (hi == L + 1 and not cfg.tie_head) or (lo == 0 and cfg.tie_head)
+        if head_w:
+            fl += head                                    # head dW
+        if hi == L + 1 and lo == L + 1 and not head_w:
+            fl += head                                    # dX still needed for the final norm's gain
+        for u in range(max(lo, 1), L + 1):
+            fl += blk_lin + 2.5 * blk_att                 # dX through this block
+            if u <= hi:
+                fl += blk_lin                             # dW inside the group
+        tot += fl
+    return tot / len(groups)
+
+
+# ---------------------------------------------------------------------------- main legs
+def run_reference(args, cfg, gcfg, ocfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    for _ in range(args.warmup_ref + args.steps_ref):
+        dt, desc, flops, threads = oracle_sample(cfg, gcfg, ocfg)
+        times.append(dt)
+    times = times[args.warmup_ref:]
+    dt = float(np.mean(times))
+    groups = [(g[0], g[-1]) for g in __import__("oracle.hift_oracle", fromlist=["x"]).build_groups(
+        cfg.n_units, gcfg.layers_per_group, gcfg.split_emb_head)]
+    full = mean_step_flops(cfg, groups)
+    value = cfg.tokens_per_step / (dt * full / flops)
+    line = {
+        "impl": "reference", "metric": "HiFT step tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps_ref, "warmup": args.warmup_ref, "ms_per_step": dt * full / flops * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "note": "CPU oracle on a bounded sample, extrapolated by flops"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, cfg, gcfg, ocfg):
+    import torch
+    import torch.distributed as dist
+    from paper_2401_15207_b200 import HiFT
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": args.prefetch, "offload_state": args.offload})
+    h = HiFT(cfg, gcfg, ocfg)
+    h.init_synthetic(1234 + rank, cfg.init_std)
+    k = h.num_groups()
+    K, W = args.steps, args.warmup
+    n_batches = 2 * (W + K)
+    host = [synth.batch_for(cfg, 77 + rank, t) for t in range(n_batches)]
+    dev = [(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for a, b in host[:W + K]]
+    groups = [h.group_units(g) for g in range(k)]
+
+    # ---- device-resident leg
+    for t in range(W):
+        h.step(*dev[t])
+    sampler = ClockSampler(local)
+    sampler.start()
+    h.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    launches = 0
+    trained = []
+    e0.record()
+    for t in range(W, W + K):
+        trained.append(h.active_group())
+        h.step(*dev[t])
+        launches += h.last_step_launches()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    prof = h.profile()
+    h.profile_enable(False)
+    clocks = sampler.stop()
+    paging = h.last_step_paging()
+
+    # ---- end-to-end leg: host buffers, copies inside the call
+    for t in range(W):
+        h.step_host(*host[W + K + t])
+    barrier()
+    t0 = time.perf_counter()
+    e0.record()
+    last_loss = 0.0
+    for t in range(K):
+        last_loss = h.step_host(*host[2 * W + K + t])
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    if world > 1:
+        tm = torch.tensor([ms, ms_e2e], device="cuda")
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = tm.tolist()
+    tokens = cfg.tokens_per_step * K * world
+    value = tokens / (ms * 1e-3)
+    e2e_value = tokens / (ms_e2e * 1e-3)
+    peak_hbm = h.peak_hbm_bytes()
+    pinned = h.pinned_host_bytes()
+
+    if rank == 0:
+        peaks = measured_peaks()
+        g = {c: prof[c] for c in ("gemm_fwd", "gemm_dx", "gemm_dw")}
+        g_launch = sum(v["launches"] for v in g.values())
+        g_ms = sum(v["ms"] for v in g.values())
+        g_fl = sum(v["work"] for v in g.values())
+        achieved = g_fl / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0
+        peak = peaks["bf16_tflops_sustained"] if cfg.dtype == 1 else None
+        roof = {"kernel": "linear-layer GEMMs (forward, dX, dW)", "bound": "tensor" if cfg.dtype == 1 else "alu",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": (achieved / peak) if peak else None, "traffic": None,
+                "peak_source": f"bf16 dense sustained, {peaks['source']}",
+                "launches": g_launch, "avg_launch_ms": g_ms / max(g_launch, 1),
+                "by_form": {c: {"launches": v["launches"], "ms": v["ms"],
+                                "tflops": v["work"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0}
+                            for c, v in g.items()}}
+        kernel_share = {c: round(v["ms"], 3) for c, v in prof.items()}
+        opt = prof["optimizer"]
+        opt_gbs = opt["work"] / (opt["ms"] * 1e-3) / 1e9 if opt["ms"] > 0 else 0.0
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            dt, desc, flops, threads = oracle_sample(cfg, gcfg, ocfg)
+            full = mean_step_flops(cfg, groups)
+            cpu = {"value": cfg.tokens_per_step / (dt * full / flops), "unit": "tokens/s", "cores": threads,
+                   "kind": "oracle", "sample": desc, "sample_seconds": dt}
+        line = {
+            "metric": "HiFT step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfg.dtype == 1 else "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "global_batch": cfg.batch * world, "seq_len": cfg.seq,
+                       "groups": k, "groups_trained": trained, "optimizer": ["adamw", "adagrad", "sgdm"][ocfg.kind],
+                       "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups,
+                       "parallelism": "replicas" if world > 1 else "single",
+                       "l2_policy": "inputs larger than L2 (weights + activations of a step exceed 126 MB)"},
+            "peak_hbm_gb": peak_hbm / 1e9, "pinned_host_gb": pinned / 1e9,
+            "paging_bytes_per_step": {"h2d": paging[0], "d2h": paging[1]},
+            "e2e": {"value": e2e_value, "unit": "tokens/s",
+                    "h2d_bytes_per_step": int(host[0][0].nbytes + host[0][1].nbytes) + paging[0],
+                    "d2h_bytes_per_step": 4 + paging[1], "ms_per_step": ms_e2e / K, "last_loss": last_loss},
+            "gpu_launches": int(launches),
+            "roofline": roof,
+            "optimizer_gbs": opt_gbs, "optimizer_frac_of_hbm": opt_gbs / peaks["hbm_gbs"],
+            "kernel_ms": kernel_share,
+            "clocks": clocks,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    h.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=34)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b", choices=sorted(WORKLOADS))
+    ap.add_argument("--prefetch", type=int, default=1)
+    ap.add_argument("--offload", type=int, default=1)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--steps-ref", type=int, default=2)
+    ap.add_argument("--warmup-ref", type=int, default=0)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    cfg, gcfg, ocfg = WORKLOADS[args.workload]()
+    if args.impl == "reference":
+        args.steps_ref = max(1, min(args.steps, args.steps_ref))
+        run_reference(args, cfg, gcfg, ocfg)
+    else:
+        run_ours(args, cfg, gcfg, ocfg)
+
+
+if __name__ == "__main__":
+    main()
