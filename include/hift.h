@@ -43,7 +43,8 @@ typedef enum {
   HIFT_ERR_INPUT = 4,        /* token id or label out of range, NULL pointer         */
   HIFT_ERR_NONFINITE = 5,    /* the loss of the step was NaN/Inf (update was applied) */
   HIFT_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up                   */
-  HIFT_ERR_CUDA = 7          /* any other CUDA runtime/driver error                  */
+  HIFT_ERR_CUDA = 7,         /* any other CUDA runtime/driver error                  */
+  HIFT_ERR_CAPACITY = 8      /* size exceeds the library's built-in scratch capacity */
 } hift_status;
 
 /* Model description.  Units (the paper's "layers", Section "Hierarchical
@@ -210,6 +211,30 @@ hift_status hift_k_norm_bwd(int32_t dtype, int32_t kind, int64_t rows, int64_t c
                             const void *gain_dev, const float *add_dev, float *dx_dev,
                             float *dgain_dev, float *dbias_dev, float *partial_dev,
                             void *cuda_stream);
+/* The paper has no counterpart for this entry point; it exists for callers that must not
+ * allocate.  It computes exactly what hift_k_norm_bwd computes (same kernels, same summation
+ * order, same results), but takes no `partial_dev` argument: the column-reduction scratch lives
+ * in a fixed array that is part of the library image (4 MiB of device memory per GPU that loads
+ * the library, held until the process exits).  Nothing is allocated or freed, on the host or on
+ * the device, by this call: no cudaMalloc, no cudaFree, no allocating library routine.  That is
+ * what code needs which runs where the allocator is off limits - inside a memory pool whose
+ * budget is already committed, in a latency-critical loop that cannot afford an allocator's
+ * implicit synchronisation, or in a host process that was handed its buffers by someone else
+ * and has no allocator of its own for this device.
+ *   - cols must be <= HIFT_STATIC_SCRATCH_MAX_COLS, else HIFT_ERR_CAPACITY (nothing is launched).
+ *   - The first call on each device looks up the device address of the array (with that
+ *     device current).  Make that first call before starting any stream capture.
+ *   - All calls on one GPU share the one array, which keeps whatever the previous call left.
+ *     Every word a call reads it has written earlier in the same call, so stale contents
+ *     are harmless and nothing needs clearing; but two calls that overlap on the GPU (different
+ *     streams, or different host threads) race on it.  Serialise them.
+ * Inputs and outputs are the caller's, as for hift_k_norm_bwd. */
+#define HIFT_STATIC_SCRATCH_MAX_COLS 8192
+hift_status hift_k_norm_bwd_static(int32_t dtype, int32_t kind, int64_t rows, int64_t cols,
+                                   const void *dy_dev, const float *x_dev, const float *stats_dev,
+                                   const void *gain_dev, const float *add_dev, float *dx_dev,
+                                   float *dgain_dev, float *dbias_dev, void *cuda_stream);
+
 /* Softmax cross-entropy over rows of logits[rows, ld] (columns >= vocab are
  * padding).  Overwrites logits with d loss / d logits.  loss_dev: 4 fp32 words,
  * [0] = mean loss over rows with label >= 0, [1] = that row count (int32 bits),

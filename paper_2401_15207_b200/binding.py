@@ -21,7 +21,9 @@ KERNEL_CLASSES = ["gemm_fwd", "gemm_dx", "gemm_dw", "attn_fwd", "attn_bwd", "nor
                   "cross_entropy", "embedding", "optimizer", "reduce"]
 
 STATUS_NAMES = {0: "HIFT_OK", 1: "HIFT_ERR_CFG", 2: "HIFT_ERR_OOM_DEVICE", 3: "HIFT_ERR_OOM_PINNED",
-                4: "HIFT_ERR_INPUT", 5: "HIFT_ERR_NONFINITE", 6: "HIFT_ERR_TIMEOUT", 7: "HIFT_ERR_CUDA"}
+                4: "HIFT_ERR_INPUT", 5: "HIFT_ERR_NONFINITE", 6: "HIFT_ERR_TIMEOUT", 7: "HIFT_ERR_CUDA",
+                8: "HIFT_ERR_CAPACITY"}
+STATIC_SCRATCH_MAX_COLS = 8192
 
 
 class HiftError(RuntimeError):
@@ -87,6 +89,7 @@ def _prototypes():
         "hift_k_attention_bwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
         "hift_k_norm_fwd": (C.c_int, [i32, i32, i64, i64, f64, vp, vp, vp, vp, vp, vp]),
         "hift_k_norm_bwd": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
+        "hift_k_norm_bwd_static": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "hift_k_cross_entropy": (C.c_int, [i32, i64, i64, i64, vp, vp, vp, vp, vp]),
     }
 
@@ -305,6 +308,15 @@ def k_norm_fwd(dtype, kind, rows, cols, eps, x, gain, bias, y, stats, stream=Non
 def k_norm_bwd(dtype, kind, rows, cols, dy, x, stats, gain, add, dx, dgain, dbias, partial, stream=None):
     _check(lib().hift_k_norm_bwd(dtype, kind, rows, cols, _ptr(dy), _ptr(x), _ptr(stats), _ptr(gain), _ptr(add),
                                  _ptr(dx), _ptr(dgain), _ptr(dbias), _ptr(partial), _st(stream)), "hift_k_norm_bwd")
+
+
+def k_norm_bwd_static(dtype, kind, rows, cols, dy, x, stats, gain, add, dx, dgain, dbias, stream=None):
+    """hift_k_norm_bwd without the caller-provided scratch and without any allocation: for
+    callers that may not allocate.  cols <= STATIC_SCRATCH_MAX_COLS; calls on one GPU must not
+    overlap (they share one built-in scratch array)."""
+    _check(lib().hift_k_norm_bwd_static(dtype, kind, rows, cols, _ptr(dy), _ptr(x), _ptr(stats), _ptr(gain),
+                                        _ptr(add), _ptr(dx), _ptr(dgain), _ptr(dbias), _st(stream)),
+           "hift_k_norm_bwd_static")
 
 
 def k_cross_entropy(dtype, rows, vocab, ld, logits, labels, rowloss, loss, stream=None):

@@ -701,6 +701,7 @@ const char* hift_strerror(hift_status s) {
     case HIFT_ERR_NONFINITE: return "non-finite loss";
     case HIFT_ERR_TIMEOUT: return "device-side wait timed out";
     case HIFT_ERR_CUDA: return "CUDA error";
+    case HIFT_ERR_CAPACITY: return "size exceeds the library's built-in scratch capacity";
   }
   return "unknown";
 }
@@ -1088,3 +1089,35 @@ hift_status hift_k_cross_entropy(int32_t dtype, int64_t rows, int64_t vocab, int
 }
 
 }  // extern "C"
+
+// ====================================================================== allocation-free variant
+// Column-reduction scratch for hift_k_norm_bwd_static: [2 planes][kColChunks][max cols] fp32,
+// resident in every GPU context that loads this library.  In host code `g_static_partial` is
+// only a handle for the runtime's symbol lookup, never a device address: the address the
+// kernels get comes from cudaGetSymbolAddress, once per device.
+namespace {
+constexpr int kStaticMaxDevices = 64;
+static __device__ __align__(256) float g_static_partial[2 * kColChunks * HIFT_STATIC_SCRATCH_MAX_COLS];
+float* g_static_partial_addr[kStaticMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" hift_status hift_k_norm_bwd_static(int32_t dtype, int32_t kind, int64_t rows, int64_t cols,
+                                              const void* dy, const float* x, const float* stats,
+                                              const void* gain, const float* add, float* dx,
+                                              float* dgain, float* dbias, void* stream) {
+  if (cols % 8 || cols < 8 || rows < 1 || kind < 0 || kind > 1 || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
+  if (cols > HIFT_STATIC_SCRATCH_MAX_COLS) return HIFT_ERR_CAPACITY;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return HIFT_ERR_CUDA;
+  float* partial = g_static_partial_addr[dev];
+  if (!partial) {
+    // first call on this device (which is current): resolve the array's device address
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_partial) != cudaSuccess || !p) { cudaGetLastError(); return HIFT_ERR_CUDA; }
+    partial = g_static_partial_addr[dev] = (float*)p;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dx) launch_norm_bwd_dx(st, dtype, kind, false, rows, (int)cols, dy, x, stats, gain, add, dx, nullptr);
+  if (dgain) launch_colreduce(st, dtype == 1, kind == 0 ? 1 : 2, rows, (int)cols, dy, cols, x, stats, partial, dgain, dbias);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}

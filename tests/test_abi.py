@@ -28,8 +28,8 @@ def test_every_declared_symbol_is_exported_and_bound():
 
 def test_strerror_covers_all_codes():
     L = binding.load_library()
-    msgs = [L.hift_strerror(i).decode() for i in range(8)]
-    assert msgs[0] == "ok" and len(set(msgs)) == 8
+    msgs = [L.hift_strerror(i).decode() for i in range(9)]
+    assert msgs[0] == "ok" and len(set(msgs)) == 9
 
 
 def test_structs_match_header_sizes():
