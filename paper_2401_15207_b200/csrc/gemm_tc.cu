@@ -1,7 +1,422 @@
+// bf16 GEMM on the Blackwell tensor cores: tcgen05.mma with the accumulator in tensor memory,
+// operands staged in shared memory by TMA (no cluster multicast), an mbarrier ring between a
+// one-thread TMA producer, a one-thread MMA issuer and four epilogue warps.
+//
+//   C[m,n] = sum_k A(m,k) * B(k,n) (+ bias[n]) (+ residual[m,n])
+//
+// The three linear-layer products of the training step differ only in which operand dimension
+// is contiguous in memory, and the tensor core takes both:
+//   forward  y  = x w^T : A K-major  (x[m,k]),   B K-major  (w[n,k])
+//   dX       dx = dy w  : A K-major  (dy[m,k']), B N-major  (w[k',n])
+//   dW       dw = dy^T x: A M-major  (dy[k',m]), B N-major  (x[k',n])
+// so no operand is ever transposed or copied.  "MN-major" tiles are loaded as 64-element-wide
+// TMA boxes (one 128-byte swizzle span along M or N) and described to the MMA with the
+// matching shared-memory descriptor (leading-dimension offset = distance between boxes).
+//
+// Every wait on an mbarrier is bounded: after about a second it records an error code in
+// g_tc_error, and the kernel drains and releases its tensor memory normally.
 #include "gemm_tc.h"
 
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdio.h>
+
+#include <mutex>
+#include <unordered_map>
+
 namespace hift {
-int gemm_tc_init() { return 1; }
-bool gemm_tc_eligible(const GemmArgs&) { return false; }
-cudaError_t gemm_tc_launch(cudaStream_t, const GemmArgs&) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int BM = 128;          // rows of the output tile = MMA M
+constexpr int BK = 64;           // k elements per pipeline stage = one 128-byte swizzle span
+constexpr int UMMA_K = 16;       // k elements per tcgen05.mma (bf16)
+constexpr int kThreads = 192;    // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2-5: epilogue
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
+
+__device__ int g_tc_error = 0;   // 0 ok; 1 producer, 2 MMA issuer, 3 epilogue gave up waiting
+
+template <int BN> struct TileCfg {
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait: false if the phase did not complete within kWaitCycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > kWaitCycles) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_c, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_c), "l"(da), "l"(db), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(addr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Fields in 16-byte units: start address
+// bits [0,14), leading-dimension byte offset [16,30), stride-dimension byte offset [32,46),
+// descriptor version 1 at [46,48), swizzle mode (2 = 128 B) at [61,64).
+//   K-major tile  [rows][64]: 8-row groups are 1024 B apart (stride offset); leading offset unused.
+//   MN-major tile [k][64] boxes: 8-k groups are 1024 B apart (stride offset); the next 64-wide box
+//   along M/N is BK*128 B further (leading offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
+  const uint64_t lbo = mn_major ? (uint64_t)((BK * 128) >> 4) : 1ull;
+  const uint64_t sbo = 1024 >> 4;
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// ------------------------------------------------------------------ kernel
+template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
+               const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr) {
+  typedef TileCfg<BN> Cfg;
+  constexpr int S = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  if (g_tc_error != 0) return;                       // an earlier launch timed out: do nothing
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
+  const uint32_t bar_base = base + S * Cfg::kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  const uint32_t accum_bar = bar_base + 8u * (2 * S);
+  const uint32_t tmem_slot = bar_base + 8u * (2 * S + 1);
+  uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + S * Cfg::kStageBytes + 8 * (2 * S + 1));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+  const int num_kb = (K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_gen;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (one thread)
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (kb / S) & 1;
+        if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); break; }
+        const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
+        mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
+        const int k0 = kb * BK;
+        if (A_MN) {
+#pragma unroll
+          for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * (BK * 128), &tmap_a, full_bar(s), m0 + j * 64, k0);
+        } else {
+          tma_load_2d(sa, &tmap_a, full_bar(s), k0, m0);
+        }
+        if (B_MN) {
+#pragma unroll
+          for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
+        } else {
+          tma_load_2d(sb, &tmap_b, full_bar(s), k0, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (one thread)
+    if (lane == 0) {
+      // instruction descriptor: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
+      // A / B major-ness (bits 15, 16: 1 = MN-major), N/8 at bits 17-22, M/16 at bits 24-28
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                             ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (kb / S) & 1;
+        if (!mbar_wait(full_bar(s), ph)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
+        const uint64_t da = make_desc(sa, A_MN), db = make_desc(sb, B_MN);
+#pragma unroll
+        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+          // advance along k inside the stage: 32 B within the swizzle span (K-major) or
+          // 16 k-rows of 128 B (MN-major); descriptor addresses are in 16-byte units
+          const uint64_t adv_a = A_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
+          const uint64_t adv_b = B_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
+          tc_mma(tmem_base, da + adv_a, db + adv_b, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(empty_bar(s));         // frees the stage once these MMAs have read it
+      }
+      tc_commit(accum_bar);              // accumulator complete (or abandoned: the epilogue is told by g_tc_error)
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp%4) .. +31
+    const int q = warp & 3;
+    const bool ready = mbar_wait(accum_bar, 0);
+    if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 3);
+    tc_fence_after();
+    const bool good = ready && (*(volatile int*)&g_tc_error == 0);
+    const int m = m0 + q * 32 + lane;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    if (good) {
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (n0 + c0 >= N) break;                       // uniform across the warp
+        uint32_t v[32];
+        tmem_ld32(taddr + c0, v);
+        if (m < M) {
+          const int n = n0 + c0;
+          float f[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+          if (n + 32 <= N) {
+            if (bias) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                const uint4 b4 = *reinterpret_cast<const uint4*>(bias + n + j);
+                const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b4);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                  const float2 bf = __bfloat1622float2(hb[t]);
+                  f[j + 2 * t] += bf.x; f[j + 2 * t + 1] += bf.y;
+                }
+              }
+            }
+            if (OUT_F32) {
+              float* crow = reinterpret_cast<float*>(cptr) + (int64_t)m * ldc + n;
+              if (residual) {
+                const float* rrow = residual + (int64_t)m * ldr + n;
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                  const float4 r = *reinterpret_cast<const float4*>(rrow + j);
+                  f[j] += r.x; f[j + 1] += r.y; f[j + 2] += r.z; f[j + 3] += r.w;
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(crow + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+            } else {
+              __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * ldc + n;
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 o;
+                __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) ho[t] = __floats2bfloat162_rn(f[j + 2 * t], f[j + 2 * t + 1]);
+                *reinterpret_cast<uint4*>(crow + j) = o;
+              }
+            }
+          } else {
+            for (int j = 0; j < 32 && n + j < N; ++j) {     // ragged right edge
+              float x = f[j];
+              if (bias) x += __bfloat162float(bias[n + j]);
+              if (OUT_F32) {
+                if (residual) x += residual[(int64_t)m * ldr + n + j];
+                reinterpret_cast<float*>(cptr)[(int64_t)m * ldc + n + j] = x;
+              } else {
+                reinterpret_cast<__nv_bfloat16*>(cptr)[(int64_t)m * ldc + n + j] = __float2bfloat16_rn(x);
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int g_init_state = -1;    // -1 not tried, 0 ok, 1 failed
+std::mutex g_mu;
+
+struct MapKey {
+  const void* p; uint64_t inner, outer, stride; uint32_t box_outer;
+  bool operator==(const MapKey& o) const {
+    return p == o.p && inner == o.inner && outer == o.outer && stride == o.stride && box_outer == o.box_outer;
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    size_t h = (size_t)k.p;
+    h = h * 1000003u ^ k.inner; h = h * 1000003u ^ k.outer; h = h * 1000003u ^ k.stride; h = h * 1000003u ^ k.box_outer;
+    return h;
+  }
+};
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_maps;
+
+// 2-D bf16 tensor [outer][inner] with row pitch `stride_elems`; box = 64 x box_outer, 128-byte swizzle.
+bool get_map(const void* p, uint64_t inner, uint64_t outer, uint64_t stride_elems, uint32_t box_outer, CUtensorMap* out) {
+  MapKey key{p, inner, outer, stride_elems, box_outer};
+  std::lock_guard<std::mutex> lk(g_mu);
+  auto it = g_maps.find(key);
+  if (it != g_maps.end()) { *out = it->second; return true; }
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {stride_elems * 2};
+  cuuint32_t box[2] = {64, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap m;
+  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (g_maps.size() > 65536) g_maps.clear();
+  g_maps[key] = m;
+  *out = m;
+  return true;
+}
+
+template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
+cudaError_t set_smem_attr() {
+  return cudaFuncSetAttribute(gemm_tc_kernel<BN, A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TileCfg<BN>::kSmemBytes);
+}
+template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
+cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& ta, const CUtensorMap& tb) {
+  dim3 grid((g.M + BM - 1) / BM, (g.N + BN - 1) / BN);
+  gemm_tc_kernel<BN, A_MN, B_MN, OUT_F32><<<grid, kThreads, TileCfg<BN>::kSmemBytes, st>>>(
+      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int gemm_tc_init() {
+  std::lock_guard<std::mutex> lk(g_mu);
+  if (g_init_state >= 0) return g_init_state;
+  g_init_state = 1;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return g_init_state;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10) return g_init_state;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    return g_init_state;
+  }
+  g_encode = (EncodeTiledFn)fn;
+  cudaError_t e = cudaSuccess;
+#define SET_ALL(BN)                                                              \
+  if (e == cudaSuccess) e = set_smem_attr<BN, false, false, false>();           \
+  if (e == cudaSuccess) e = set_smem_attr<BN, false, false, true>();            \
+  if (e == cudaSuccess) e = set_smem_attr<BN, false, true, false>();            \
+  if (e == cudaSuccess) e = set_smem_attr<BN, false, true, true>();             \
+  if (e == cudaSuccess) e = set_smem_attr<BN, true, true, true>();
+  SET_ALL(256)
+  SET_ALL(128)
+#undef SET_ALL
+  if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
+  g_init_state = 0;
+  return 0;
+}
+
+// 0: not eligible; 1: forward (A K-major, B K-major); 2: dX (A K-major, B N-major); 3: dW (A M-major, B N-major)
+static int classify(const GemmArgs& g) {
+  if (g_init_state != 0) return 0;
+  if (g.M < 128 || g.N < 64 || g.K < 64) return 0;
+  const bool a_k = g.sak == 1, a_m = g.sam == 1, b_k = g.sbk == 1, b_n = g.sbn == 1;
+  int form = 0;
+  if (a_k && b_k) form = 1; else if (a_k && b_n) form = 2; else if (a_m && b_n) form = 3; else return 0;
+  const int64_t lda = a_k ? g.sam : g.sak, ldb = b_k ? g.sbn : g.sbk;
+  if (lda % 8 || ldb % 8 || g.ldc % (g.out_f32 ? 4 : 8)) return 0;
+  if (((uintptr_t)g.a | (uintptr_t)g.b | (uintptr_t)g.c) & 15) return 0;
+  if (g.bias && ((uintptr_t)g.bias & 15)) return 0;
+  if (g.residual && (!g.out_f32 || ((uintptr_t)g.residual & 15) || g.ldr % 4)) return 0;
+  if (form == 3 && (!g.out_f32 || g.bias || g.residual)) return 0;
+  return form;
+}
+bool gemm_tc_eligible(const GemmArgs& g) { return classify(g) != 0; }
+
+cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
+  const int form = classify(g);
+  if (!form) return cudaErrorInvalidValue;
+  const int bn = g.N >= 256 ? 256 : 128;
+  CUtensorMap ta, tb;
+  bool ok;
+  // K-major operand: tensor [rows = M or N][inner = K]; MN-major operand: tensor [rows = K][inner = M or N]
+  if (form == 3) ok = get_map(g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.sak, BK, &ta);
+  else ok = get_map(g.a, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.sam, BM, &ta);
+  if (form == 1) ok = ok && get_map(g.b, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.sbn, (uint32_t)bn, &tb);
+  else ok = ok && get_map(g.b, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.sbk, BK, &tb);
+  if (!ok) return cudaErrorInvalidValue;
+#define GO(BN)                                                                                     \
+  if (form == 1) return g.out_f32 ? launch_inst<BN, false, false, true>(st, g, ta, tb)             \
+                                  : launch_inst<BN, false, false, false>(st, g, ta, tb);           \
+  if (form == 2) return g.out_f32 ? launch_inst<BN, false, true, true>(st, g, ta, tb)              \
+                                  : launch_inst<BN, false, true, false>(st, g, ta, tb);            \
+  return launch_inst<BN, true, true, true>(st, g, ta, tb);
+  if (bn == 256) { GO(256) } else { GO(128) }
+#undef GO
+}
+
+int gemm_tc_poll_error() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)) != cudaSuccess) return -1;
+  return v;
+}
+
 }  // namespace hift

@@ -14,5 +14,8 @@ int gemm_tc_init();
 // 16-byte aligned with 16-byte-multiple leading dimensions.
 bool gemm_tc_eligible(const GemmArgs& g);
 cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g);
+// 0 if no tensor-core kernel has given up on a bounded wait since the library was loaded, else the
+// code of the first one (1 producer, 2 MMA issuer, 3 epilogue); -1 if the flag cannot be read.
+int gemm_tc_poll_error();
 
 }  // namespace hift

@@ -649,6 +649,7 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
   c->prof_collect();
   c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
   if (c->first_err != cudaSuccess) return HIFT_ERR_CUDA;
+  if (c->mixed && gemm_tc_poll_error() > 0) return HIFT_ERR_TIMEOUT;
   const float loss = c->scal_host[0];
   int bad_h;
   memcpy(&bad_h, &c->scal_host[2], sizeof(int));

@@ -226,3 +226,51 @@ def test_cross_entropy_flags_bad_label():
     out = torch.zeros(4, dtype=torch.float32, device="cuda")
     k_cross_entropy(0, 4, 8, 8, logits, labels, torch.empty(4, device="cuda"), out)
     assert out.cpu().numpy()[2:3].view(np.int32)[0] == 1
+
+
+# ------------------------------------------------------------------ tensor-core GEMM (tcgen05), forced
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 640), (300, 328, 200), (1024, 128, 1096),
+                                   (130, 72, 72)])
+def test_linear_tensor_core_three_forms(M, N, K):
+    import torch
+    from paper_2401_15207_b200 import k_linear
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.1).astype(np.float32)
+    dy = rng.standard_normal((M, N)).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    bf = torch.bfloat16
+    tx, tw, tdy, tb = _t(x, bf), _t(w, bf), _t(dy, bf), _t(bias, bf)
+    # forward, bf16 out with bias
+    y = torch.zeros((M, N), dtype=bf, device="cuda")
+    k_linear(0, 1, M, N, K, tx, tw, y, bias=tb, path=2)
+    ref = _bf(x) @ _bf(w).T + _bf(bias)
+    assert rel_l2(y.float().cpu().numpy(), ref) <= 6e-3
+    # forward into the fp32 residual stream
+    res = rng.standard_normal((M, N)).astype(np.float32)
+    y32 = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    k_linear(0, 1, M, N, K, tx, tw, y32, bias=tb, residual=_t(res), path=2)
+    assert rel_l2(y32.cpu().numpy(), ref + res) <= 1e-5
+    # activation gradient: dx[M,K] = dy[M,N] w[N,K]   (B operand N-major)
+    if K >= 64 and N >= 64:
+        dx = torch.zeros((M, K), dtype=torch.float32, device="cuda")
+        k_linear(1, 1, M, N, K, tdy, tw, dx, residual=torch.zeros((M, K), dtype=torch.float32, device="cuda"), path=2)
+        assert rel_l2(dx.cpu().numpy(), _bf(dy) @ _bf(w)) <= 1e-5
+    # weight gradient: dw[N,K] = dy^T x   (both operands MN-major); needs N >= 128 rows of output
+    if N >= 128:
+        dw = torch.zeros((N, K), dtype=torch.float32, device="cuda")
+        k_linear(2, 1, M, N, K, tdy, tx, dw, path=2)
+        assert rel_l2(dw.cpu().numpy(), _bf(dy).T @ _bf(x)) <= 1e-5
+
+
+def test_tensor_core_path_refuses_ineligible_shapes():
+    import torch
+    from paper_2401_15207_b200 import k_linear, HiftError
+    bf = torch.bfloat16
+    a = torch.zeros((64, 64), dtype=bf, device="cuda")
+    with pytest.raises(HiftError):
+        k_linear(0, 1, 64, 64, 64, a, a, torch.zeros((64, 64), dtype=bf, device="cuda"), path=2)   # M < 128
+    a = torch.zeros((128, 100), dtype=bf, device="cuda")
+    w = torch.zeros((64, 100), dtype=bf, device="cuda")
+    with pytest.raises(HiftError):
+        k_linear(0, 1, 128, 64, 100, a, w, torch.zeros((128, 64), dtype=bf, device="cuda"), path=2)  # ld % 8 != 0
