@@ -316,12 +316,17 @@ def main():
     ap.add_argument("--prefetch", type=int, default=1)
     ap.add_argument("--offload", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--full-param", action="store_true",
+                    help="one group holding every unit, state resident: the ordinary full-parameter step")
     ap.add_argument("--steps-ref", type=int, default=2)
     ap.add_argument("--warmup-ref", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     cfg, gcfg, ocfg = WORKLOADS[args.workload]()
+    if args.full_param:
+        gcfg = synth.GroupCfg(layers_per_group=cfg.n_units, split_emb_head=0, order=synth.ORDER_BOTTOM2UP)
+        args.offload, args.prefetch = 0, 0
     if args.impl == "reference":
         args.steps_ref = max(1, min(args.steps, args.steps_ref))
         run_reference(args, cfg, gcfg, ocfg)

@@ -387,7 +387,7 @@ void attn_bwd(hift_ctx* c, const void* qkv, const void* o, const float* lse, con
   LAUNCH(HIFT_K_ATTN_BWD, work,
          launch_attention_bwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse,
                               dout, dqkv, c->dsum));
-  ++c->step_launches;
+  c->step_launches += attention_use_mma(c->mixed, c->dh) ? 2 : 1;   // dsum, dq, dkv or dq, dkv
 }
 void rope(hift_ctx* c, void* qkv, float sign) {
   const size_t n = (size_t)c->T * c->H * (c->dh / 2);

@@ -1,0 +1,463 @@
+// bf16 attention on the warp-level tensor-core path (mma.sync m16n8k16, fp32 accumulate), for
+// head sizes 64 and 128.  Same mathematics and layout as kernels_attention.cuh:
+//   forward:  o = softmax(q k^T / sqrt(d_h) + causal mask) v, online softmax over 64-key tiles, LSE saved
+//   backward: probabilities recomputed from LSE; one kernel owns query rows (dq), one owns key
+//             rows (dk, dv), so every output has one writer and the result is deterministic.
+// qkv[T,3d] with column blocks q | k | v, head h at columns h*d_h; o, do: [T,d]; lse, dsum: [B,H,S].
+//
+// Shared-memory tiles are [rows][DH] bf16 with the 16-byte chunk index XOR-ed with (row & 7), so
+// that ldmatrix (8 rows x 16 bytes) is bank-conflict free.
+#pragma once
+#include "common.cuh"
+
+namespace hift {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
+}
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// byte offset of element (r, col) in a swizzled [rows][DH] bf16 tile; col % 8 == 0
+template <int DH>
+__device__ __forceinline__ uint32_t swz(int r, int col) {
+  return (uint32_t)((r * (DH / 8) + ((col >> 3) ^ (r & 7))) * 16);
+}
+// Stage ROWS rows of DH bf16 (row pitch `pitch` elements) starting at global row row0; rows at
+// or beyond `rows_total` are zero-filled.  All 128 threads of the block take part.
+template <int ROWS, int DH>
+__device__ __forceinline__ void stage_tile(uint8_t* tile, const bf16* __restrict__ g, int64_t pitch,
+                                           int row0, int rows_total) {
+  constexpr int CH = DH / 8;
+  for (int idx = threadIdx.x; idx < ROWS * CH; idx += blockDim.x) {
+    const int r = idx / CH, c = idx % CH;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row0 + r < rows_total) v = *reinterpret_cast<const uint4*>(g + (int64_t)(row0 + r) * pitch + c * 8);
+    *reinterpret_cast<uint4*>(tile + swz<DH>(r, c * 8)) = v;
+  }
+}
+// A fragment (16 rows x 16 k) of a row-major tile at (r0, c0)
+template <int DH>
+__device__ __forceinline__ void load_a(uint32_t (&a)[4], uint32_t tile, int r0, int c0, int lane) {
+  ldsm_x4(a, tile + swz<DH>(r0 + (lane & 7) + ((lane >> 3) & 1) * 8, c0 + (lane >> 4) * 8));
+}
+// B fragments for two adjacent n8 tiles where B(k, n) = X[n][k] (tile rows are n, k contiguous):
+// r[0], r[1] = b0, b1 of tile n0; r[2], r[3] = b0, b1 of tile n0 + 8
+template <int DH>
+__device__ __forceinline__ void load_b_nk(uint32_t (&r)[4], uint32_t tile, int n0, int k0, int lane) {
+  ldsm_x4(r, tile + swz<DH>(n0 + (lane & 7) + (lane >> 4) * 8, k0 + ((lane >> 3) & 1) * 8));
+}
+// B fragments for two adjacent n8 tiles where B(k, n) = X[k][n] (tile rows are k, n contiguous)
+template <int DH>
+__device__ __forceinline__ void load_b_kn(uint32_t (&r)[4], uint32_t tile, int k0, int n0, int lane) {
+  ldsm_x4_t(r, tile + swz<DH>(k0 + (lane & 7) + ((lane >> 3) & 1) * 8, n0 + (lane >> 4) * 8));
+}
+
+// ------------------------------------------------------------------ forward
+template <int DH>
+__global__ void __launch_bounds__(128)
+attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* __restrict__ lse,
+                    int S, int H, int causal, float scale) {
+  constexpr int BQ = 64, BKV = 64, KS = DH / 16;
+  __shared__ __align__(128) uint8_t sQ[BQ * DH * 2];
+  __shared__ __align__(128) uint8_t sK[BKV * DH * 2];
+  __shared__ __align__(128) uint8_t sV[BKV * DH * 2];
+  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * BQ;
+  const int d = H * DH;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const bf16* qb = qkv + (int64_t)b * S * 3 * d + (int64_t)h * DH;
+  const bf16* kb = qb + d;
+  const bf16* vb = qb + 2 * d;
+  const uint32_t tQ = (uint32_t)__cvta_generic_to_shared(sQ);
+  const uint32_t tK = (uint32_t)__cvta_generic_to_shared(sK);
+  const uint32_t tV = (uint32_t)__cvta_generic_to_shared(sV);
+
+  stage_tile<BQ, DH>(sQ, qb, 3 * d, q0, S);
+  __syncthreads();
+  uint32_t qa[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) load_a<DH>(qa[ks], tQ, warp * 16, ks * 16, lane);
+
+  float oacc[DH / 8][4];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) { oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f; }
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+  const float sl2 = scale * kLog2e;
+  const int row_lo = q0 + warp * 16 + g;              // this thread's rows: row_lo, row_lo + 8
+  const int k_end = causal ? min(S, q0 + BQ) : S;
+
+  for (int k0 = 0; k0 < k_end; k0 += BKV) {
+    __syncthreads();
+    stage_tile<BKV, DH>(sK, kb, 3 * d, k0, S);
+    stage_tile<BKV, DH>(sV, vb, 3 * d, k0, S);
+    __syncthreads();
+    float sacc[BKV / 8][4];
+#pragma unroll
+    for (int i = 0; i < BKV / 8; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < BKV / 16; ++np) {
+        uint32_t bfr[4];
+        load_b_nk<DH>(bfr, tK, np * 16, ks * 16, lane);
+        mma16816(sacc[2 * np], qa[ks], bfr[0], bfr[1]);
+        mma16816(sacc[2 * np + 1], qa[ks], bfr[2], bfr[3]);
+      }
+    }
+    // scale, mask, running max
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int i = 0; i < BKV / 8; ++i) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int col = k0 + i * 8 + 2 * t + (e & 1);
+        const int row = row_lo + (e >> 1) * 8;
+        float v = sacc[i][e] * sl2;
+        if (col >= S || (causal && col > row)) v = -INFINITY;
+        sacc[i][e] = v;
+        mx[e >> 1] = fmaxf(mx[e >> 1], v);
+      }
+    }
+    float corr[2], muse[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+      const float mnew = fmaxf(mrow[r], mx[r]);
+      muse[r] = (mnew == -INFINITY) ? 0.f : mnew;       // a row with nothing visible yet
+      corr[r] = exp2f(mrow[r] - muse[r]);                // exp2(-inf) = 0 on the first tile
+      mrow[r] = mnew;
+      lrow[r] *= corr[r];
+    }
+#pragma unroll
+    for (int i = 0; i < BKV / 8; ++i) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float p = exp2f(sacc[i][e] - muse[e >> 1]);
+        sacc[i][e] = p;
+        lrow[e >> 1] += p;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) {
+      oacc[i][0] *= corr[0]; oacc[i][1] *= corr[0]; oacc[i][2] *= corr[1]; oacc[i][3] *= corr[1];
+    }
+    // O += P V
+#pragma unroll
+    for (int j = 0; j < BKV / 16; ++j) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16(sacc[2 * j][0], sacc[2 * j][1]);
+      pa[1] = pack_bf16(sacc[2 * j][2], sacc[2 * j][3]);
+      pa[2] = pack_bf16(sacc[2 * j + 1][0], sacc[2 * j + 1][1]);
+      pa[3] = pack_bf16(sacc[2 * j + 1][2], sacc[2 * j + 1][3]);
+#pragma unroll
+      for (int np = 0; np < DH / 16; ++np) {
+        uint32_t bfr[4];
+        load_b_kn<DH>(bfr, tV, j * 16, np * 16, lane);
+        mma16816(oacc[2 * np], pa, bfr[0], bfr[1]);
+        mma16816(oacc[2 * np + 1], pa, bfr[2], bfr[3]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
+    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int row = row_lo + r * 8;
+    if (row >= S) continue;
+    const float inv = 1.0f / lrow[r];
+    bf16* orow = o + ((int64_t)b * S + row) * d + (int64_t)h * DH;
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i)
+      *reinterpret_cast<uint32_t*>(orow + i * 8 + 2 * t) = pack_bf16(oacc[i][2 * r] * inv, oacc[i][2 * r + 1] * inv);
+    if (t == 0) lse[((int64_t)b * H + h) * S + row] = (mrow[r] + log2f(lrow[r])) * kLn2;
+  }
+}
+
+// ------------------------------------------------------------------ backward: dsum = rowsum(do * o)
+// one warp per (token, head)
+__global__ void attn_dsum_kernel(const bf16* __restrict__ o, const bf16* __restrict__ dout,
+                                 float* __restrict__ dsum, int B, int S, int H, int DH) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= (int64_t)B * S * H) return;
+  const int h = (int)(w % H);
+  const int64_t tok = w / H;
+  const int b = (int)(tok / S), s = (int)(tok % S);
+  const bf16* po = o + tok * (int64_t)H * DH + (int64_t)h * DH;
+  const bf16* pg = dout + tok * (int64_t)H * DH + (int64_t)h * DH;
+  float acc = 0.f;
+  for (int e = lane * 2; e < DH; e += 64) {
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + e));
+    const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pg + e));
+    acc += a.x * c.x + a.y * c.y;
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) dsum[((int64_t)b * H + h) * S + s] = acc;
+}
+
+// ------------------------------------------------------------------ backward: dq (owner of query rows)
+template <int DH>
+__global__ void __launch_bounds__(128)
+attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse,
+                       const bf16* __restrict__ dout, const float* __restrict__ dsum,
+                       bf16* __restrict__ dqkv, int S, int H, int causal, float scale) {
+  constexpr int BQ = 64, BKV = 32, KS = DH / 16;
+  __shared__ __align__(128) uint8_t sX[BQ * DH * 2];       // q tile, then do tile (fragments are kept in registers)
+  __shared__ __align__(128) uint8_t sK[BKV * DH * 2];
+  __shared__ __align__(128) uint8_t sV[BKV * DH * 2];
+  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * BQ;
+  const int d = H * DH;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const bf16* qb = qkv + (int64_t)b * S * 3 * d + (int64_t)h * DH;
+  const bf16* kb = qb + d;
+  const bf16* vb = qb + 2 * d;
+  const bf16* gb = dout + (int64_t)b * S * d + (int64_t)h * DH;
+  const uint32_t tX = (uint32_t)__cvta_generic_to_shared(sX);
+  const uint32_t tK = (uint32_t)__cvta_generic_to_shared(sK);
+  const uint32_t tV = (uint32_t)__cvta_generic_to_shared(sV);
+
+  uint32_t qa[KS][4], ga[KS][4];
+  stage_tile<BQ, DH>(sX, qb, 3 * d, q0, S);
+  __syncthreads();
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) load_a<DH>(qa[ks], tX, warp * 16, ks * 16, lane);
+  __syncthreads();
+  stage_tile<BQ, DH>(sX, gb, d, q0, S);
+  __syncthreads();
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) load_a<DH>(ga[ks], tX, warp * 16, ks * 16, lane);
+
+  const int row_lo = q0 + warp * 16 + g;
+  float L2[2], Dr[2];
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int row = row_lo + r * 8;
+    const bool ok = row < S;
+    L2[r] = ok ? lse[((int64_t)b * H + h) * S + row] * kLog2e : 0.f;
+    Dr[r] = ok ? dsum[((int64_t)b * H + h) * S + row] : 0.f;
+  }
+  float dq[DH / 8][4];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) { dq[i][0] = dq[i][1] = dq[i][2] = dq[i][3] = 0.f; }
+  const float sl2 = scale * kLog2e;
+  const int k_end = causal ? min(S, q0 + BQ) : S;
+
+  for (int k0 = 0; k0 < k_end; k0 += BKV) {
+    __syncthreads();
+    stage_tile<BKV, DH>(sK, kb, 3 * d, k0, S);
+    stage_tile<BKV, DH>(sV, vb, 3 * d, k0, S);
+    __syncthreads();
+    float sacc[BKV / 8][4], pacc[BKV / 8][4];
+#pragma unroll
+    for (int i = 0; i < BKV / 8; ++i) {
+      sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
+      pacc[i][0] = pacc[i][1] = pacc[i][2] = pacc[i][3] = 0.f;
+    }
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < BKV / 16; ++np) {
+        uint32_t bfr[4];
+        load_b_nk<DH>(bfr, tK, np * 16, ks * 16, lane);
+        mma16816(sacc[2 * np], qa[ks], bfr[0], bfr[1]);
+        mma16816(sacc[2 * np + 1], qa[ks], bfr[2], bfr[3]);
+        load_b_nk<DH>(bfr, tV, np * 16, ks * 16, lane);
+        mma16816(pacc[2 * np], ga[ks], bfr[0], bfr[1]);
+        mma16816(pacc[2 * np + 1], ga[ks], bfr[2], bfr[3]);
+      }
+    }
+    // dS = P * (dP - D), masked entries 0
+#pragma unroll
+    for (int i = 0; i < BKV / 8; ++i) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int col = k0 + i * 8 + 2 * t + (e & 1);
+        const int row = row_lo + (e >> 1) * 8;
+        float ds = 0.f;
+        if (col < S && row < S && !(causal && col > row)) {
+          const float p = exp2f(sacc[i][e] * sl2 - L2[e >> 1]);
+          ds = p * (pacc[i][e] - Dr[e >> 1]);
+        }
+        sacc[i][e] = ds;
+      }
+    }
+    // dQ += dS K
+#pragma unroll
+    for (int j = 0; j < BKV / 16; ++j) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16(sacc[2 * j][0], sacc[2 * j][1]);
+      pa[1] = pack_bf16(sacc[2 * j][2], sacc[2 * j][3]);
+      pa[2] = pack_bf16(sacc[2 * j + 1][0], sacc[2 * j + 1][1]);
+      pa[3] = pack_bf16(sacc[2 * j + 1][2], sacc[2 * j + 1][3]);
+#pragma unroll
+      for (int np = 0; np < DH / 16; ++np) {
+        uint32_t bfr[4];
+        load_b_kn<DH>(bfr, tK, j * 16, np * 16, lane);
+        mma16816(dq[2 * np], pa, bfr[0], bfr[1]);
+        mma16816(dq[2 * np + 1], pa, bfr[2], bfr[3]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int row = row_lo + r * 8;
+    if (row >= S) continue;
+    bf16* out = dqkv + ((int64_t)b * S + row) * 3 * d + (int64_t)h * DH;
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i)
+      *reinterpret_cast<uint32_t*>(out + i * 8 + 2 * t) = pack_bf16(dq[i][2 * r] * scale, dq[i][2 * r + 1] * scale);
+  }
+}
+
+// ------------------------------------------------------------------ backward: dk, dv (owner of key rows)
+// dynamic shared memory: K tile [64][DH], V tile [64][DH], Q tile [32][DH], dO tile [32][DH], L2[32], D[32]
+template <int DH>
+constexpr int attn_dkv_smem_bytes() { return (64 + 64 + 32 + 32) * DH * 2 + 2 * 32 * 4; }
+
+template <int DH>
+__global__ void __launch_bounds__(128)
+attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse,
+                        const bf16* __restrict__ dout, const float* __restrict__ dsum,
+                        bf16* __restrict__ dqkv, int S, int H, int causal, float scale) {
+  constexpr int BKV = 64, BQ = 32, KS = DH / 16;
+  extern __shared__ __align__(128) uint8_t smem_dkv[];
+  uint8_t* sK = smem_dkv;
+  uint8_t* sV = sK + BKV * DH * 2;
+  uint8_t* sQ = sV + BKV * DH * 2;
+  uint8_t* sG = sQ + BQ * DH * 2;
+  float* sL = reinterpret_cast<float*>(sG + BQ * DH * 2);
+  float* sD = sL + BQ;
+  const int b = blockIdx.z, h = blockIdx.y, kr0 = blockIdx.x * BKV;
+  const int d = H * DH;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const bf16* qb = qkv + (int64_t)b * S * 3 * d + (int64_t)h * DH;
+  const bf16* kb = qb + d;
+  const bf16* vb = qb + 2 * d;
+  const bf16* gb = dout + (int64_t)b * S * d + (int64_t)h * DH;
+  const uint32_t tK = (uint32_t)__cvta_generic_to_shared(sK);
+  const uint32_t tV = (uint32_t)__cvta_generic_to_shared(sV);
+  const uint32_t tQ = (uint32_t)__cvta_generic_to_shared(sQ);
+  const uint32_t tG = (uint32_t)__cvta_generic_to_shared(sG);
+
+  stage_tile<BKV, DH>(sK, kb, 3 * d, kr0, S);
+  stage_tile<BKV, DH>(sV, vb, 3 * d, kr0, S);
+
+  float dk[DH / 8][4], dv[DH / 8][4];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) {
+    dk[i][0] = dk[i][1] = dk[i][2] = dk[i][3] = 0.f;
+    dv[i][0] = dv[i][1] = dv[i][2] = dv[i][3] = 0.f;
+  }
+  const float sl2 = scale * kLog2e;
+  const int key_lo = kr0 + warp * 16 + g;             // this thread's key rows: key_lo, key_lo + 8
+  const int q_begin = causal ? (kr0 / BQ) * BQ : 0;
+
+  for (int q0 = q_begin; q0 < S; q0 += BQ) {
+    __syncthreads();
+    stage_tile<BQ, DH>(sQ, qb, 3 * d, q0, S);
+    stage_tile<BQ, DH>(sG, gb, d, q0, S);
+    if (threadIdx.x < BQ) {
+      const int row = q0 + threadIdx.x;
+      const bool ok = row < S;
+      sL[threadIdx.x] = ok ? lse[((int64_t)b * H + h) * S + row] * kLog2e : 0.f;
+      sD[threadIdx.x] = ok ? dsum[((int64_t)b * H + h) * S + row] : 0.f;
+    }
+    __syncthreads();
+    // S^T = K Q^T and dP^T = V dO^T, 16 keys x 32 queries per warp
+    float sacc[BQ / 8][4], pacc[BQ / 8][4];
+#pragma unroll
+    for (int i = 0; i < BQ / 8; ++i) {
+      sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
+      pacc[i][0] = pacc[i][1] = pacc[i][2] = pacc[i][3] = 0.f;
+    }
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      uint32_t ka[4], va[4];
+      load_a<DH>(ka, tK, warp * 16, ks * 16, lane);
+      load_a<DH>(va, tV, warp * 16, ks * 16, lane);
+#pragma unroll
+      for (int np = 0; np < BQ / 16; ++np) {
+        uint32_t bfr[4];
+        load_b_nk<DH>(bfr, tQ, np * 16, ks * 16, lane);
+        mma16816(sacc[2 * np], ka, bfr[0], bfr[1]);
+        mma16816(sacc[2 * np + 1], ka, bfr[2], bfr[3]);
+        load_b_nk<DH>(bfr, tG, np * 16, ks * 16, lane);
+        mma16816(pacc[2 * np], va, bfr[0], bfr[1]);
+        mma16816(pacc[2 * np + 1], va, bfr[2], bfr[3]);
+      }
+    }
+    // P^T and dS^T (masked entries 0); rows are keys, columns are queries
+#pragma unroll
+    for (int i = 0; i < BQ / 8; ++i) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int qc = i * 8 + 2 * t + (e & 1);
+        const int qrow = q0 + qc;
+        const int key = key_lo + (e >> 1) * 8;
+        float p = 0.f, ds = 0.f;
+        if (qrow < S && key < S && !(causal && key > qrow)) {
+          p = exp2f(sacc[i][e] * sl2 - sL[qc]);
+          ds = p * (pacc[i][e] - sD[qc]);
+        }
+        sacc[i][e] = p;
+        pacc[i][e] = ds;
+      }
+    }
+    // dV += P^T dO ; dK += dS^T Q
+#pragma unroll
+    for (int j = 0; j < BQ / 16; ++j) {
+      uint32_t pa[4], da[4];
+      pa[0] = pack_bf16(sacc[2 * j][0], sacc[2 * j][1]);
+      pa[1] = pack_bf16(sacc[2 * j][2], sacc[2 * j][3]);
+      pa[2] = pack_bf16(sacc[2 * j + 1][0], sacc[2 * j + 1][1]);
+      pa[3] = pack_bf16(sacc[2 * j + 1][2], sacc[2 * j + 1][3]);
+      da[0] = pack_bf16(pacc[2 * j][0], pacc[2 * j][1]);
+      da[1] = pack_bf16(pacc[2 * j][2], pacc[2 * j][3]);
+      da[2] = pack_bf16(pacc[2 * j + 1][0], pacc[2 * j + 1][1]);
+      da[3] = pack_bf16(pacc[2 * j + 1][2], pacc[2 * j + 1][3]);
+#pragma unroll
+      for (int np = 0; np < DH / 16; ++np) {
+        uint32_t bfr[4];
+        load_b_kn<DH>(bfr, tG, j * 16, np * 16, lane);
+        mma16816(dv[2 * np], pa, bfr[0], bfr[1]);
+        mma16816(dv[2 * np + 1], pa, bfr[2], bfr[3]);
+        load_b_kn<DH>(bfr, tQ, j * 16, np * 16, lane);
+        mma16816(dk[2 * np], da, bfr[0], bfr[1]);
+        mma16816(dk[2 * np + 1], da, bfr[2], bfr[3]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int key = key_lo + r * 8;
+    if (key >= S) continue;
+    bf16* outk = dqkv + ((int64_t)b * S + key) * 3 * d + d + (int64_t)h * DH;
+    bf16* outv = outk + d;
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) {
+      *reinterpret_cast<uint32_t*>(outk + i * 8 + 2 * t) = pack_bf16(dk[i][2 * r] * scale, dk[i][2 * r + 1] * scale);
+      *reinterpret_cast<uint32_t*>(outv + i * 8 + 2 * t) = pack_bf16(dv[i][2 * r], dv[i][2 * r + 1]);
+    }
+  }
+}
+
+}  // namespace hift

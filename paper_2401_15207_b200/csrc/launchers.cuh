@@ -3,6 +3,7 @@
 #pragma once
 #include "gemm_args.h"
 #include "kernels_attention.cuh"
+#include "kernels_attention_mma.cuh"
 #include "kernels_gemm_simt.cuh"
 #include "kernels_pointwise.cuh"
 
@@ -69,8 +70,36 @@ inline void attention_bwd_inst(cudaStream_t st, int B, int S, int H, int causal,
     case 128: { CALL(128); break; }         \
     default: break;                         \
   }
+// bf16 with head size 64 or 128 goes to the tensor-core kernels
+inline bool attention_use_mma(int dtype, int dh) { return dtype == 1 && (dh == 64 || dh == 128); }
+template <int DH>
+inline void attention_mma_fwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, void* o, float* lse) {
+  dim3 grid((S + 63) / 64, H, B);
+  attn_fwd_mma_kernel<DH><<<grid, 128, 0, st>>>((const bf16*)qkv, (bf16*)o, lse, S, H, causal, 1.0f / sqrtf((float)DH));
+}
+template <int DH>
+inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, const void* o,
+                              const float* lse, const void* dout, void* dqkv, float* dsum) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(attn_bwd_dkv_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_dkv_smem_bytes<DH>());
+    attr_set = true;
+  }
+  const float scale = 1.0f / sqrtf((float)DH);
+  const int64_t warps = (int64_t)B * S * H;
+  attn_dsum_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)dout, dsum, B, S, H, DH);
+  dim3 grid((S + 63) / 64, H, B);
+  attn_bwd_dq_mma_kernel<DH><<<grid, 128, 0, st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum, (bf16*)dqkv, S, H, causal, scale);
+  attn_bwd_dkv_mma_kernel<DH><<<grid, 128, attn_dkv_smem_bytes<DH>(), st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum,
+                                                                           (bf16*)dqkv, S, H, causal, scale);
+}
 inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
                                  const void* qkv, void* o, float* lse) {
+  if (attention_use_mma(dtype, dh)) {
+    if (dh == 64) attention_mma_fwd<64>(st, B, S, H, causal, qkv, o, lse);
+    else attention_mma_fwd<128>(st, B, S, H, causal, qkv, o, lse);
+    return;
+  }
 #define CALL_F(D)                                                              \
   if (dtype == 0) attention_fwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse); \
   else attention_fwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse)
@@ -80,6 +109,11 @@ inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H
 inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
                                  const void* qkv, const void* o, const float* lse, const void* dout,
                                  void* dqkv, float* dsum) {
+  if (attention_use_mma(dtype, dh)) {
+    if (dh == 64) attention_mma_bwd<64>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum);
+    else attention_mma_bwd<128>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum);
+    return;
+  }
 #define CALL_B(D)                                                                              \
   if (dtype == 0) attention_bwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum); \
   else attention_bwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum)
