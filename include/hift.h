@@ -160,6 +160,12 @@ int64_t hift_last_step_launches(const hift_ctx *ctx);
 /* Bytes paged host->device and device->host by the last step. */
 hift_status hift_last_step_paging(const hift_ctx *ctx, size_t *h2d_bytes, size_t *d2h_bytes);
 
+/* Device timeline of the last step's state paging (Algorithm 1 steps i and k), in milliseconds
+ * after the step's first kernel: [0] H2D begin, [1] H2D end, [2] optimizer reaches its wait
+ * for the state, [3] wait over, [4] D2H begin, [5] D2H end.  -1 where offload is off.  Waits
+ * for the copies to finish. */
+hift_status hift_last_step_timeline(hift_ctx *ctx, double *ms6);
+
 /* ---- the group-local fused optimizer on caller-owned flat buffers --------
  * One streaming pass over n elements (the update Algorithm 1 applies to the
  * active group once "UpdateOptimizerParameter" has pointed P at theta_s).  All

@@ -83,6 +83,7 @@ def _prototypes():
         "hift_profile": (C.c_int, [vp, i32, C.POINTER(i64), C.POINTER(f64), C.POINTER(f64)]),
         "hift_last_step_launches": (i64, [vp]),
         "hift_last_step_paging": (C.c_int, [vp, C.POINTER(sz), C.POINTER(sz)]),
+        "hift_last_step_timeline": (C.c_int, [vp, C.POINTER(f64)]),
         "hift_opt_step": (C.c_int, [i32, sz, vp, vp, vp, vp, vp, f64, f64, f64, f64, f64, f64, i64, vp]),
         "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
@@ -272,6 +273,12 @@ class HiFT:
         a, b = C.c_size_t(), C.c_size_t()
         _check(lib().hift_last_step_paging(self._h, C.byref(a), C.byref(b)), "hift_last_step_paging")
         return a.value, b.value
+
+
+    def last_step_timeline(self) -> List[float]:
+        arr = (C.c_double * 6)()
+        _check(lib().hift_last_step_timeline(self._h, arr), "hift_last_step_timeline")
+        return list(arr)
 
 
 # ---------------------------------------------------------------- free functions

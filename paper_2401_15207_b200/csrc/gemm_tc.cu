@@ -413,6 +413,16 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
 #undef GO
 }
 
+const int* gemm_tc_error_device_ptr() {
+  static const int* ptr = nullptr;
+  if (!ptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_tc_error) == cudaSuccess) ptr = (const int*)p;
+    else cudaGetLastError();
+  }
+  return ptr;
+}
+
 int gemm_tc_poll_error() {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)) != cudaSuccess) return -1;

@@ -17,5 +17,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g);
 // 0 if no tensor-core kernel has given up on a bounded wait since the library was loaded, else the
 // code of the first one (1 producer, 2 MMA issuer, 3 epilogue); -1 if the flag cannot be read.
 int gemm_tc_poll_error();
+// Device address of that flag (an int), or nullptr if it cannot be resolved.
+const int* gemm_tc_error_device_ptr();
 
 }  // namespace hift

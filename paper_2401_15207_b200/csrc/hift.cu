@@ -57,7 +57,9 @@ struct hift_ctx {
   hift_model_cfg m;
   hift_group_cfg gc;
   hift_opt_cfg oc;
-  cudaStream_t st = nullptr, st_h2d = nullptr, st_d2h = nullptr;
+  cudaStream_t st = nullptr, st_h2d = nullptr, st_d2h = nullptr;   // compute and copy streams (owned, non-blocking)
+  cudaStream_t caller = nullptr;    // the stream given to hift_create: inputs are ordered after it
+  cudaEvent_t ev_in;
   int es = 2;                       // bytes per parameter / GEMM-operand element
   int L = 0, d = 0, f = 0, fa = 0, H = 0, dh = 0, T = 0, B = 0, S = 0, V = 0, Vp = 0;
   int n_state = 2;
@@ -83,6 +85,8 @@ struct hift_ctx {
   float* grad = nullptr;            // [max_group]
   char* arena = nullptr; size_t arena_cap = 0, arena_off = 0, arena_fixed = 0;
   cudaEvent_t ev_h2d[2], ev_opt[2], ev_d2h[2], ev_fwd;
+  cudaEvent_t tl[7];                // timeline of the last step: start, h2d begin/end, optimizer wait begin/end, d2h begin/end
+  bool tl_valid = false;
   bool events_made = false;
   bool d2h_pending[2] = {false, false};
   // fixed work buffers
@@ -95,7 +99,8 @@ struct hift_ctx {
   char *xf = nullptr, *logits = nullptr;
   float *stf = nullptr, *st_e = nullptr, *dsum = nullptr, *partial = nullptr, *rowloss = nullptr, *rope_cs = nullptr;
   float* scal = nullptr;            // device: [0] loss, [1] nvalid(int), [2] bad(int)
-  float* scal_host = nullptr;       // pinned mirror
+  float* scal_host = nullptr;       // pinned, mapped mirror
+  float* scal_host_dev = nullptr;   // its device-side address
   std::vector<std::vector<char*>> slots;   // [block][slot]; entry L holds the scratch copies
   // instrumentation
   bool prof_on = false;
@@ -502,7 +507,9 @@ void issue_h2d(hift_ctx* c, int g, int sl, bool after_forward) {
   if (after_forward) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_fwd, 0));
   if (c->d2h_pending[sl]) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_d2h[sl], 0));
   // slot layout follows the blob: consecutive planes of gr.numel floats
+  c->note(cudaEventRecord(c->tl[1], c->st_h2d));
   c->note(cudaMemcpyAsync(c->slot[sl], gr.blob, gr.blob_bytes, cudaMemcpyHostToDevice, c->st_h2d));
+  c->note(cudaEventRecord(c->tl[2], c->st_h2d));
   c->note(cudaEventRecord(c->ev_h2d[sl], c->st_h2d));
   c->step_h2d = gr.blob_bytes;
 }
@@ -523,6 +530,10 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
 
   plan_slots(c, g, true);
   if (c->arena_off > c->arena_cap) return HIFT_ERR_CFG;
+  // inputs produced on the caller's stream are visible to the step
+  c->note(cudaEventRecord(c->ev_in, c->caller));
+  c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
+  c->note(cudaEventRecord(c->tl[0], c->st));
 
   if (c->offload && c->oc.prefetch_groups) issue_h2d(c, g, sl, false);
 
@@ -622,7 +633,9 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
     float* base = (float*)c->slot[sl];
     if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
     else { mst = (float*)c->params + gr.off; s0 = base; s1 = base + gr.numel; }
+    c->note(cudaEventRecord(c->tl[3], c->st));
     c->note(cudaStreamWaitEvent(c->st, c->ev_h2d[sl], 0));
+    c->note(cudaEventRecord(c->tl[4], c->st));
   } else {
     if (c->mixed) { mst = c->master_all + gr.off; pbf = c->params + gr.off * c->es; }
     else mst = (float*)c->params + gr.off;
@@ -638,18 +651,25 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
   if (c->offload) {
     c->note(cudaEventRecord(c->ev_opt[sl], c->st));
     c->note(cudaStreamWaitEvent(c->st_d2h, c->ev_opt[sl], 0));
+    c->note(cudaEventRecord(c->tl[5], c->st_d2h));
     c->note(cudaMemcpyAsync(gr.blob, c->slot[sl], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st_d2h));
+    c->note(cudaEventRecord(c->tl[6], c->st_d2h));
     c->note(cudaEventRecord(c->ev_d2h[sl], c->st_d2h));
+    c->tl_valid = true;
     c->d2h_pending[sl] = true;
     c->step_d2h = gr.blob_bytes;
   }
 
-  c->note(cudaMemcpyAsync(c->scal_host, c->scal, 4 * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  // the loss goes to mapped host memory by a kernel store: a copy would queue behind the state transfers
+  publish_scalars_kernel<<<1, 32, 0, c->st>>>(c->scal, c->mixed ? gemm_tc_error_device_ptr() : nullptr, c->scal_host_dev);
+  c->note(cudaGetLastError());
   c->note(cudaStreamSynchronize(c->st));
   c->prof_collect();
   c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
   if (c->first_err != cudaSuccess) return HIFT_ERR_CUDA;
-  if (c->mixed && gemm_tc_poll_error() > 0) return HIFT_ERR_TIMEOUT;
+  int tc_err;
+  memcpy(&tc_err, &c->scal_host[3], sizeof(int));
+  if (tc_err > 0) return HIFT_ERR_TIMEOUT;
   const float loss = c->scal_host[0];
   int bad_h;
   memcpy(&bad_h, &c->scal_host[2], sizeof(int));
@@ -660,7 +680,7 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
 }
 
 void sync_all(hift_ctx* c) {
-  cudaStreamSynchronize(c->st);
+  if (c->st) cudaStreamSynchronize(c->st);
   if (c->st_h2d) cudaStreamSynchronize(c->st_h2d);
   if (c->st_d2h) cudaStreamSynchronize(c->st_d2h);
 }
@@ -717,7 +737,10 @@ void hift_destroy(hift_ctx* c) {
   if (c->events_made) {
     for (int i = 0; i < 2; ++i) { cudaEventDestroy(c->ev_h2d[i]); cudaEventDestroy(c->ev_opt[i]); cudaEventDestroy(c->ev_d2h[i]); }
     cudaEventDestroy(c->ev_fwd);
+    cudaEventDestroy(c->ev_in);
+    for (int i = 0; i < 7; ++i) cudaEventDestroy(c->tl[i]);
   }
+  if (c->st) cudaStreamDestroy(c->st);
   if (c->st_h2d) cudaStreamDestroy(c->st_h2d);
   if (c->st_d2h) cudaStreamDestroy(c->st_d2h);
   delete c;
@@ -746,7 +769,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
 
   hift_ctx* c = new hift_ctx();
   c->m = *m; c->gc = *gc; c->oc = *oc;
-  c->st = (cudaStream_t)cuda_stream;
+  c->caller = (cudaStream_t)cuda_stream;
   c->mixed = m->dtype == 1;
   c->es = c->mixed ? 2 : 4;
   c->L = m->n_blocks; c->d = m->d_model; c->f = m->d_ffn; c->fa = m->arch == 2 ? 2 * m->d_ffn : m->d_ffn;
@@ -768,7 +791,12 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     cudaEventCreateWithFlags(&c->ev_d2h[i], cudaEventDisableTiming);
   }
   cudaEventCreateWithFlags(&c->ev_fwd, cudaEventDisableTiming);
+  for (int i = 0; i < 7; ++i) cudaEventCreate(&c->tl[i]);
   c->events_made = true;
+  cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming);
+  // The step runs on a stream of its own: work in the legacy default stream would order itself after
+  // the state transfers still in flight from the previous step.
+  if (cudaStreamCreateWithFlags(&c->st, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
   if (cudaStreamCreateWithFlags(&c->st_h2d, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
   if (cudaStreamCreateWithFlags(&c->st_d2h, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
@@ -804,7 +832,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
       cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
     }
   }
-  if (cudaHostAlloc((void**)&c->scal_host, 4 * sizeof(float), cudaHostAllocDefault) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
+  if (cudaHostAlloc((void**)&c->scal_host, 4 * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
+  if (cudaHostGetDevicePointer((void**)&c->scal_host_dev, c->scal_host, 0) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
   // ---- activation arena: fixed work buffers, one scratch copy of every slot, then the
   //      per-group kept activations (sized for the worst group)
@@ -919,15 +948,15 @@ hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) 
   sync_all(c);
   bool on_host;
   float* mp = plane_ptr(c, ti, 0, &on_host);
+  // every copy goes through the context's stream, so the cast below is ordered after its input
   if (on_host) memcpy(mp, src, n * sizeof(float));
-  else if (cudaMemcpy(mp, src, n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return HIFT_ERR_CUDA;
+  else if (cudaMemcpyAsync(mp, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
   if (c->mixed) {
     // stage the fp32 values in the gradient buffer (any tensor fits in the largest group)
-    if (cudaMemcpy(c->grad, src, n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return HIFT_ERR_CUDA;
+    if (cudaMemcpyAsync(c->grad, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
     cast_from_f32_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>(c->grad, (bf16*)c->P(ti), n);
-    if (cudaStreamSynchronize(c->st) != cudaSuccess) return HIFT_ERR_CUDA;
   }
-  return HIFT_OK;
+  return cudaStreamSynchronize(c->st) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_get_param(hift_ctx* c, int32_t ti, float* dst, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
@@ -1016,6 +1045,19 @@ int64_t hift_last_step_launches(const hift_ctx* c) { return c->step_launches; }
 hift_status hift_last_step_paging(const hift_ctx* c, size_t* h2d, size_t* d2h) {
   if (h2d) *h2d = c->step_h2d;
   if (d2h) *d2h = c->step_d2h;
+  return HIFT_OK;
+}
+
+hift_status hift_last_step_timeline(hift_ctx* c, double* ms6) {
+  if (!c || !ms6) return HIFT_ERR_CFG;
+  for (int i = 0; i < 6; ++i) ms6[i] = -1.0;
+  if (!c->offload || !c->tl_valid) return HIFT_OK;
+  sync_all(c);
+  for (int i = 0; i < 6; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->tl[0], c->tl[i + 1]) == cudaSuccess) ms6[i] = ms;
+    else cudaGetLastError();
+  }
   return HIFT_OK;
 }
 

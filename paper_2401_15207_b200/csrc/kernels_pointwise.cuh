@@ -473,6 +473,16 @@ __global__ void loss_reduce_kernel(const float* __restrict__ rowloss, int64_t ro
   if (threadIdx.x == 0) loss[0] = s / (float)nvalid[0];
 }
 
+// Copies the step's scalar words (loss, valid count, bad-input flag, and the tensor-core GEMM's
+// timeout flag) into mapped pinned host memory with plain stores, so that the read-back never
+// queues on a copy engine behind the multi-gigabyte optimizer-state transfers.
+__global__ void publish_scalars_kernel(const float* __restrict__ src, const int* __restrict__ tc_error,
+                                       volatile float* dst_mapped_host) {
+  if (threadIdx.x < 3) dst_mapped_host[threadIdx.x] = src[threadIdx.x];
+  if (threadIdx.x == 3) dst_mapped_host[3] = tc_error ? __int_as_float(*tc_error) : 0.f;
+  __threadfence_system();
+}
+
 // ------------------------------------------------------------------ fused group optimizer
 // One streaming pass over the group's flat buffers: 128-bit loads/stores, 4 elements per
 // thread per iteration.  KIND 0 AdamW, 1 AdaGrad, 2 SGD-momentum.  Scalars precomputed on the
