@@ -1,6 +1,7 @@
 // bf16 GEMM on the Blackwell tensor cores: tcgen05.mma with the accumulator in tensor memory,
 // operands staged in shared memory by TMA (no cluster multicast), an mbarrier ring between a
-// one-thread TMA producer, a one-thread MMA issuer and four epilogue warps.
+// one-thread TMA producer, a one-thread MMA issuer and four epilogue warps.  The kernel is
+// persistent (one CTA per SM) with two accumulators, so epilogues overlap the next tile's MMAs.
 //
 //   C[m,n] = sum_k A(m,k) * B(k,n) (+ bias[n]) (+ residual[m,n])
 //
@@ -116,11 +117,19 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
 }
 
 // ------------------------------------------------------------------ kernel
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Persistent: one CTA per SM walks output tiles (m fastest, so CTAs running together share the
+// same B tile through L2).  Two accumulators in tensor memory: while the epilogue warps drain
+// tile i, the MMA thread already accumulates tile i+1.
 template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
-               const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr) {
+               const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
+               int tiles_m, int num_tiles) {
   typedef TileCfg<BN> Cfg;
   constexpr int S = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -130,22 +139,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const uint32_t bar_base = base + S * Cfg::kStageBytes;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
-  const uint32_t accum_bar = bar_base + 8u * (2 * S);
-  const uint32_t tmem_slot = bar_base + 8u * (2 * S + 1);
+  auto acc_full = [&](int a) { return bar_base + 8u * (2 * S + a); };
+  auto acc_empty = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
+  const uint32_t tmem_slot = bar_base + 8u * (2 * S + 4);
   uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + S * Cfg::kStageBytes + 8 * (2 * S + 1));
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + S * Cfg::kStageBytes + 8 * (2 * S + 4));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
   const int num_kb = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(accum_bar, 1);
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(2 * BN) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -156,24 +165,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (warp == 0) {
     // ---------------- TMA producer (one thread)
     if (lane == 0) {
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (kb / S) & 1;
-        if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); break; }
-        const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
-        mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
-        const int k0 = kb * BK;
-        if (A_MN) {
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % S;
+          const uint32_t ph = (it / S) & 1;
+          if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); ok = false; break; }
+          const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
+          mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
+          const int k0 = kb * BK;
+          if (A_MN) {
 #pragma unroll
-          for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * (BK * 128), &tmap_a, full_bar(s), m0 + j * 64, k0);
-        } else {
-          tma_load_2d(sa, &tmap_a, full_bar(s), k0, m0);
-        }
-        if (B_MN) {
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * (BK * 128), &tmap_a, full_bar(s), m0 + j * 64, k0);
+          } else {
+            tma_load_2d(sa, &tmap_a, full_bar(s), k0, m0);
+          }
+          if (B_MN) {
 #pragma unroll
-          for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
-        } else {
-          tma_load_2d(sb, &tmap_b, full_bar(s), k0, n0);
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
+          } else {
+            tma_load_2d(sb, &tmap_b, full_bar(s), k0, n0);
+          }
         }
       }
     }
@@ -184,36 +198,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // A / B major-ness (bits 15, 16: 1 = MN-major), N/8 at bits 17-22, M/16 at bits 24-28
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
                              ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int it = 0, lt = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (kb / S) & 1;
-        if (!mbar_wait(full_bar(s), ph)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+        const int ab = lt & 1;
+        const uint32_t aph = (lt >> 1) & 1;
+        // the epilogue must have drained this accumulator (passes at once on its first use)
+        if (!mbar_wait(acc_empty(ab), aph ^ 1)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
-        const uint64_t da = make_desc(sa, A_MN), db = make_desc(sb, B_MN);
+        const uint32_t tacc = tmem_base + (uint32_t)(ab * BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % S;
+          const uint32_t ph = (it / S) & 1;
+          if (!mbar_wait(full_bar(s), ph)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
+          const uint64_t da = make_desc(sa, A_MN), db = make_desc(sb, B_MN);
 #pragma unroll
-        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-          // advance along k inside the stage: 32 B within the swizzle span (K-major) or
-          // 16 k-rows of 128 B (MN-major); descriptor addresses are in 16-byte units
-          const uint64_t adv_a = A_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
-          const uint64_t adv_b = B_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
-          tc_mma(tmem_base, da + adv_a, db + adv_b, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            // advance along k inside the stage: 32 B within the swizzle span (K-major) or
+            // 16 k-rows of 128 B (MN-major); descriptor addresses are in 16-byte units
+            const uint64_t adv_a = A_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
+            const uint64_t adv_b = B_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
+            tc_mma(tacc, da + adv_a, db + adv_b, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));       // frees the stage once these MMAs have read it
         }
-        tc_commit(empty_bar(s));         // frees the stage once these MMAs have read it
+        tc_commit(acc_full(ab));         // accumulator complete (or abandoned: g_tc_error tells the epilogue)
       }
-      tc_commit(accum_bar);              // accumulator complete (or abandoned: the epilogue is told by g_tc_error)
     }
   } else {
     // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp%4) .. +31
     const int q = warp & 3;
-    const bool ready = mbar_wait(accum_bar, 0);
-    if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 3);
-    tc_fence_after();
-    const bool good = ready && (*(volatile int*)&g_tc_error == 0);
-    const int m = m0 + q * 32 + lane;
-    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-    if (good) {
+    int lt = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++lt) {
+      const int ab = lt & 1;
+      const uint32_t aph = (lt >> 1) & 1;
+      const bool ready = mbar_wait(acc_full(ab), aph);
+      if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 3);
+      tc_fence_after();
+      // one decision for the whole warp: the tensor-memory loads below are warp-collective
+      if (!__all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0)) break;
+      const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+      const int m = m0 + q * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN);
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         if (n0 + c0 >= N) break;                       // uniform across the warp
@@ -275,13 +303,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       }
+      // hand the accumulator back to the MMA thread
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(ab));
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
   }
 }
 
@@ -290,6 +322,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
+int g_num_sms = 148;
 int g_init_state = -1;    // -1 not tried, 0 ok, 1 failed
 std::mutex g_mu;
 
@@ -336,9 +369,11 @@ cudaError_t set_smem_attr() {
 }
 template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& ta, const CUtensorMap& tb) {
-  dim3 grid((g.M + BM - 1) / BM, (g.N + BN - 1) / BN);
+  const int tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+  const int num_tiles = tiles_m * tiles_n;
+  const int grid = num_tiles < g_num_sms ? num_tiles : g_num_sms;
   gemm_tc_kernel<BN, A_MN, B_MN, OUT_F32><<<grid, kThreads, TileCfg<BN>::kSmemBytes, st>>>(
-      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr);
+      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles);
   return cudaGetLastError();
 }
 
@@ -359,6 +394,7 @@ int gemm_tc_init() {
     return g_init_state;
   }
   g_encode = (EncodeTiledFn)fn;
+  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1) g_num_sms = 148;
   cudaError_t e = cudaSuccess;
 #define SET_ALL(BN)                                                              \
   if (e == cudaSuccess) e = set_smem_attr<BN, false, false, false>();           \
