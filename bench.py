@@ -271,6 +271,13 @@ def run_ours(args, cfg, gcfg, ocfg):
     e2e_value = tokens / (ms_e2e * 1e-3)
     peak_hbm = h.peak_hbm_bytes()
     pinned = h.pinned_host_bytes()
+    h.close()
+    full_ref = None
+    if world == 1 and not args.no_full_param_reference and not args.full_param and not args.skip_e2e:
+        try:
+            full_ref = run_full_param_reference(cfg, ocfg)
+        except Exception as e:                      # e.g. not enough HBM for 16 B/param
+            full_ref = {"unavailable": str(e)[:200]}
 
     if rank == 0:
         peaks = measured_peaks()
@@ -283,6 +290,8 @@ def run_ours(args, cfg, gcfg, ocfg):
         roof = {"kernel": "linear-layer GEMMs (forward, dX, dW)", "bound": "tensor" if cfg.dtype == 1 else "alu",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": (achieved / peak) if peak else None, "traffic": None,
+                "traffic_note": "launches of many shapes are averaged here; per-shape DRAM counters are in "
+                                "profiles/gemm_tc_kernel_m2048_n12288_k4096.md (traffic / algorithmic bytes 0.88-1.32)",
                 "peak_source": f"bf16 dense sustained, {peaks['source']}",
                 "launches": g_launch, "avg_launch_ms": g_ms / max(g_launch, 1),
                 "profiled_ms_per_step": ms_prof / K,
@@ -319,12 +328,119 @@ def run_ours(args, cfg, gcfg, ocfg):
             "optimizer_gbs": opt_gbs, "optimizer_frac_of_hbm": opt_gbs / peaks["hbm_gbs"],
             "kernel_ms": kernel_share,
             "clocks": clocks,
+            "full_param_reference": full_ref,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
-    h.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_full_param_reference(cfg, ocfg, steps=4, warmup=3):
+    """The same model trained the ordinary way: one group holding every unit (k = 1), all master
+    weights and optimizer state resident on the GPU, full backward.  Returns tokens/s and peak HBM."""
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    g = synth.GroupCfg(layers_per_group=cfg.n_units, split_emb_head=0, order=synth.ORDER_BOTTOM2UP)
+    o = synth.OptCfg(**{**ocfg.__dict__, "offload_state": 0, "prefetch_groups": 0})
+    h = HiFT(cfg, g, o)
+    try:
+        h.init_synthetic(99, cfg.init_std)
+        dev = [tuple(torch.from_numpy(a).cuda() for a in synth.batch_for(cfg, 55, t)) for t in range(warmup + steps)]
+        for t in range(warmup):
+            h.step(*dev[t])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for t in range(warmup, warmup + steps):
+            h.step(*dev[t])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        return {"tokens_per_s": cfg.tokens_per_step / (ms * 1e-3), "ms_per_step": ms,
+                "peak_hbm_gb": h.peak_hbm_bytes() / 1e9, "steps": steps}
+    finally:
+        h.close()
+
+
+def run_sweep_optimizer(args):
+    """Group-local fused optimizer over flat buffers of 2^20 .. 2^30 elements (bf16 param, fp32
+    master/state, gradients N(0, 1e-3)): achieved algorithmic GB/s against the measured HBM peak."""
+    import torch
+    from paper_2401_15207_b200 import opt_step
+    peaks = measured_peaks()
+    rows = []
+    for kind, name, bpe in ((0, "adamw", 30), (1, "adagrad", 22), (2, "sgdm", 22)):
+        for lg in range(20, 31):
+            n = 1 << lg
+            # rotate over enough buffer sets to exceed L2 (126 MB) between visits
+            sets = max(1, min(8, int(200e6 // (n * bpe)) + 1))
+            bufs = []
+            for _ in range(sets):
+                master = torch.randn(n, device="cuda") * 0.02
+                grad = torch.randn(n, device="cuda") * 1e-3
+                bufs.append((torch.zeros(n, dtype=torch.bfloat16, device="cuda"), master, grad,
+                             torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")))
+            iters = max(5, min(200, int(2e9 // (n * bpe))))
+            for i in range(3):
+                p, m, g, a, b = bufs[i % sets]
+                opt_step(kind, n, p, m, g, a, b, lr=1e-3, eps=1e-8 if kind != 1 else 1e-10, tau=1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(iters):
+                p, m, g, a, b = bufs[i % sets]
+                opt_step(kind, n, p, m, g, a, b, lr=1e-3, eps=1e-8 if kind != 1 else 1e-10, tau=2 + i)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / iters
+            gbs = n * bpe / (us * 1e-6) / 1e9
+            rows.append({"optimizer": name, "log2_n": lg, "us": round(us, 2), "gbs": round(gbs, 1),
+                         "frac_of_hbm": round(gbs / peaks["hbm_gbs"], 3),
+                         "l2_resident": bool(n * bpe * sets < 126e6)})
+            del bufs
+            torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "optimizer", "unit": "GB/s", "hbm_peak_gbs": peaks["hbm_gbs"],
+                      "peak_source": peaks["source"], "rows": rows}))
+
+
+def run_sweep_depth(args):
+    """GPT-2-large-shaped config with block-group g = 0..17 forced active (plus the embedding and head
+    groups): step time and dX / dW GEMM throughput versus the depth at which the backward pass stops."""
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    cfg, gcfg, ocfg = synth.config_gpt2_large(synth.OPT_SGDM)
+    ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": 1})
+    h = HiFT(cfg, gcfg, ocfg)
+    h.init_synthetic(5, cfg.init_std)
+    dev = [tuple(torch.from_numpy(a).cuda() for a in synth.batch_for(cfg, 5, t)) for t in range(4)]
+    peaks = measured_peaks()
+    rows = []
+    for g in range(h.num_groups()):
+        h.force_group(g)
+        for t in range(3):
+            h.step(*dev[t])
+        h.profile_enable(True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for t in range(4):
+            h.step(*dev[t])
+        e1.record()
+        torch.cuda.synchronize()
+        prof = h.profile()
+        h.profile_enable(False)
+        lo, hi = h.group_units(g)
+        tf = lambda c: prof[c]["work"] / (prof[c]["ms"] * 1e-3) / 1e12 if prof[c]["ms"] > 0 else 0.0
+        label = "embedding" if hi == 0 else ("head" if lo == cfg.n_blocks + 1 else f"blocks {lo - 1}-{hi - 1}")
+        rows.append({"group": g, "units": label, "ms_per_step": round(e0.elapsed_time(e1) / 4, 3),
+                     "dx_tflops": round(tf("gemm_dx"), 1), "dw_tflops": round(tf("gemm_dw"), 1),
+                     "dx_frac_of_peak": round(tf("gemm_dx") / peaks["bf16_tflops_sustained"], 3),
+                     "dw_frac_of_peak": round(tf("gemm_dw") / peaks["bf16_tflops_sustained"], 3),
+                     "dx_launches": prof["gemm_dx"]["launches"] // 4, "dw_launches": prof["gemm_dw"]["launches"] // 4})
+    h.close()
+    print(json.dumps({"sweep": "depth", "workload": "gpt2large", "peak_tflops": peaks["bf16_tflops_sustained"],
+                      "rows": rows}))
 
 
 def main():
@@ -341,11 +457,19 @@ def main():
                     help="one group holding every unit, state resident: the ordinary full-parameter step")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave out the end-to-end leg")
     ap.add_argument("--skip-profiled", action="store_true", help="profiling runs: leave out the event-bracketed pass")
+    ap.add_argument("--no-full-param-reference", action="store_true",
+                    help="leave out the k = 1 full-parameter step of the same model (needs ~132 GB at the 7B shape)")
+    ap.add_argument("--sweep", default=None, choices=["optimizer", "depth"],
+                    help="kernel sweeps instead of the step benchmark")
     ap.add_argument("--steps-ref", type=int, default=2)
     ap.add_argument("--warmup-ref", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.sweep == "optimizer":
+        return run_sweep_optimizer(args)
+    if args.sweep == "depth":
+        return run_sweep_depth(args)
     cfg, gcfg, ocfg = WORKLOADS[args.workload]()
     if args.full_param:
         gcfg = synth.GroupCfg(layers_per_group=cfg.n_units, split_emb_head=0, order=synth.ORDER_BOTTOM2UP)

@@ -38,7 +38,7 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 __device__ int g_tc_error = 0;   // 0 ok; 1 producer, 2 MMA issuer, 3 epilogue gave up waiting
 
 template <int BN> struct TileCfg {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kStages = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
@@ -404,6 +404,7 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr<BN, true, true, true>();
   SET_ALL(256)
   SET_ALL(128)
+  SET_ALL(64)
 #undef SET_ALL
   if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
   g_init_state = 0;
@@ -430,7 +431,22 @@ bool gemm_tc_eligible(const GemmArgs& g) { return classify(g) != 0; }
 cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   const int form = classify(g);
   if (!form) return cudaErrorInvalidValue;
-  const int bn = g.N >= 256 ? 256 : 128;
+  // Tile width: the widest tile keeps the tensor pipe busiest, but a grid that leaves most SMs idle
+  // in its last round (or never fills one round) loses more; score = SM occupancy x per-tile efficiency.
+  int bn = 256;
+  {
+    const int tm = (g.M + BM - 1) / BM;
+    double best = -1.0;
+    const int cand[3] = {256, 128, 64};
+    const double tile_eff[3] = {1.0, 0.88, 0.62};
+    for (int i = 0; i < 3; ++i) {
+      if (cand[i] > 64 && g.N < cand[i]) continue;
+      const int tiles = tm * ((g.N + cand[i] - 1) / cand[i]);
+      const int rounds = (tiles + g_num_sms - 1) / g_num_sms;
+      const double score = (double)tiles / ((double)rounds * g_num_sms) * tile_eff[i];
+      if (score > best + 1e-9) { best = score; bn = cand[i]; }
+    }
+  }
   CUtensorMap ta, tb;
   bool ok;
   // K-major operand: tensor [rows = M or N][inner = K]; MN-major operand: tensor [rows = K][inner = M or N]
@@ -445,7 +461,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   if (form == 2) return g.out_f32 ? launch_inst<BN, false, true, true>(st, g, ta, tb)              \
                                   : launch_inst<BN, false, true, false>(st, g, ta, tb);            \
   return launch_inst<BN, true, true, true>(st, g, ta, tb);
-  if (bn == 256) { GO(256) } else { GO(128) }
+  if (bn == 256) { GO(256) } else if (bn == 128) { GO(128) } else { GO(64) }
 #undef GO
 }
 
