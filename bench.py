@@ -184,7 +184,7 @@ def run_reference(args, cfg, gcfg, ocfg):
 def run_ours(args, cfg, gcfg, ocfg):
     import torch
     import torch.distributed as dist
-    from paper_2401_15207_b200 import HiFT
+    from paper_2401_15207_b200 import HiFT, dist_util
 
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -200,11 +200,11 @@ def run_ours(args, cfg, gcfg, ocfg):
 
     ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": args.prefetch, "offload_state": args.offload})
     h = HiFT(cfg, gcfg, ocfg)
-    h.init_synthetic(1234 + rank, cfg.init_std)
+    h.init_synthetic(dist_util.rank_seed(1234, rank), cfg.init_std)
     k = h.num_groups()
     K, W = args.steps, args.warmup
     n_batches = 2 * (W + K)
-    host = [synth.batch_for(cfg, 77 + rank, t) for t in range(n_batches)]
+    host = [synth.batch_for(cfg, dist_util.rank_seed(77, rank), t) for t in range(n_batches)]
     dev = [(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for a, b in host[:W + K]]
     groups = [h.group_units(g) for g in range(k)]
 
@@ -262,10 +262,7 @@ def run_ours(args, cfg, gcfg, ocfg):
         barrier()
         ms_e2e = e0.elapsed_time(e1)
 
-    if world > 1:
-        tm = torch.tensor([ms, ms_e2e], device="cuda")
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = tm.tolist()
+    ms, ms_e2e = dist_util.max_over_ranks([ms, ms_e2e], device="cuda")
     tokens = cfg.tokens_per_step * K * world
     value = tokens / (ms * 1e-3)
     e2e_value = tokens / (ms_e2e * 1e-3)
