@@ -37,13 +37,24 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 
 __device__ int g_tc_error = 0;   // 0 ok; 1 producer, 2 MMA issuer, 3 epilogue gave up waiting
 
-template <int BN> struct TileCfg {
-  static constexpr int kStages = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int kABytes = BM * BK * 2;
-  static constexpr int kBBytes = BN * BK * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-};
+// Tile width BN is a run-time multiple of 32 in [64, 256] (MMA N), chosen per problem so that the
+// grid fills whole rounds of SMs.  Shared memory per stage: A 128 x 64 bf16 (16 KB) plus B, which is
+// BN x 64 bf16 when K-major and ceil(BN/64) boxes of 64 x 64 when N-major.
+constexpr int kABytes = BM * BK * 2;
+constexpr int kSmemBudget = 196608;                 // operand ring
+constexpr int kSmemBytes = kSmemBudget + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kMaxStages = 8;
+constexpr int kAccStride = 256;                     // tensor-memory columns between the two accumulators
+struct TileRt { int bn, b_bytes, stage_bytes, stages; };
+inline TileRt make_tile(int bn, bool b_mn) {
+  TileRt t;
+  t.bn = bn;
+  t.b_bytes = b_mn ? ((bn + 63) / 64) * (BK * 128) : bn * BK * 2;
+  t.stage_bytes = kABytes + t.b_bytes;
+  t.stages = kSmemBudget / t.stage_bytes;
+  if (t.stages > kMaxStages) t.stages = kMaxStages;
+  return t;
+}
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -124,26 +135,26 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Persistent: one CTA per SM walks output tiles (m fastest, so CTAs running together share the
 // same B tile through L2).  Two accumulators in tensor memory: while the epilogue warps drain
 // tile i, the MMA thread already accumulates tile i+1.
-template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
+template <bool A_MN, bool B_MN, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-               int tiles_m, int num_tiles) {
-  typedef TileCfg<BN> Cfg;
-  constexpr int S = Cfg::kStages;
+               int tiles_m, int num_tiles, TileRt tc) {
+  const int BN = tc.bn, S = tc.stages;
+  const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
   if (g_tc_error != 0) return;                       // an earlier launch timed out: do nothing
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
-  const uint32_t bar_base = base + S * Cfg::kStageBytes;
+  const uint32_t bar_base = base + S * kStageBytes;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
   auto acc_full = [&](int a) { return bar_base + 8u * (2 * S + a); };
   auto acc_empty = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
   const uint32_t tmem_slot = bar_base + 8u * (2 * S + 4);
   uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + S * Cfg::kStageBytes + 8 * (2 * S + 4));
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + S * kStageBytes + 8 * (2 * S + 4));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (K + BK - 1) / BK;
@@ -154,7 +165,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(2 * BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(2 * kAccStride) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -165,16 +176,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (warp == 0) {
     // ---------------- TMA producer (one thread)
     if (lane == 0) {
-      int it = 0;
+      int s = 0;
+      uint32_t ph = 0;                   // ring position and its phase, advanced without divisions
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-          const int s = it % S;
-          const uint32_t ph = (it / S) & 1;
+        for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); ok = false; break; }
-          const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
-          mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
+          const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+          mbar_expect_tx(full_bar(s), kStageBytes);
           const int k0 = kb * BK;
           if (A_MN) {
 #pragma unroll
@@ -183,11 +193,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             tma_load_2d(sa, &tmap_a, full_bar(s), k0, m0);
           }
           if (B_MN) {
-#pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
+            for (int j = 0; j * 64 < BN; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
           } else {
             tma_load_2d(sb, &tmap_b, full_bar(s), k0, n0);
           }
+          if (++s == S) { s = 0; ph ^= 1; }
         }
       }
     }
@@ -198,7 +208,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // A / B major-ness (bits 15, 16: 1 = MN-major), N/8 at bits 17-22, M/16 at bits 24-28
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
                              ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-      int it = 0, lt = 0;
+      int s = 0, lt = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
         const int ab = lt & 1;
@@ -206,13 +217,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // the epilogue must have drained this accumulator (passes at once on its first use)
         if (!mbar_wait(acc_empty(ab), aph ^ 1)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
         tc_fence_after();
-        const uint32_t tacc = tmem_base + (uint32_t)(ab * BN);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-          const int s = it % S;
-          const uint32_t ph = (it / S) & 1;
+        const uint32_t tacc = tmem_base + (uint32_t)(ab * kAccStride);
+        for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(s), ph)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + s * Cfg::kStageBytes, sb = sa + Cfg::kABytes;
+          const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
           const uint64_t da = make_desc(sa, A_MN), db = make_desc(sb, B_MN);
 #pragma unroll
           for (int kk = 0; kk < BK / UMMA_K; ++kk) {
@@ -223,6 +232,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             tc_mma(tacc, da + adv_a, db + adv_b, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
           tc_commit(empty_bar(s));       // frees the stage once these MMAs have read it
+          if (++s == S) { s = 0; ph ^= 1; }
         }
         tc_commit(acc_full(ab));         // accumulator complete (or abandoned: g_tc_error tells the epilogue)
       }
@@ -241,7 +251,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!__all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0)) break;
       const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         if (n0 + c0 >= N) break;                       // uniform across the warp
@@ -313,7 +323,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   __syncthreads();
   if (warp == 1) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kAccStride) : "memory");
   }
 }
 
@@ -362,18 +372,19 @@ bool get_map(const void* p, uint64_t inner, uint64_t outer, uint64_t stride_elem
   return true;
 }
 
-template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
+template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr() {
-  return cudaFuncSetAttribute(gemm_tc_kernel<BN, A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              TileCfg<BN>::kSmemBytes);
+  return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kSmemBytes);
 }
-template <int BN, bool A_MN, bool B_MN, bool OUT_F32>
-cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& ta, const CUtensorMap& tb) {
-  const int tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + BN - 1) / BN;
+template <bool A_MN, bool B_MN, bool OUT_F32>
+cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& ta, const CUtensorMap& tb, int bn) {
+  const TileRt tc = make_tile(bn, B_MN);
+  const int tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + bn - 1) / bn;
   const int num_tiles = tiles_m * tiles_n;
   const int grid = num_tiles < g_num_sms ? num_tiles : g_num_sms;
-  gemm_tc_kernel<BN, A_MN, B_MN, OUT_F32><<<grid, kThreads, TileCfg<BN>::kSmemBytes, st>>>(
-      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles);
+  gemm_tc_kernel<A_MN, B_MN, OUT_F32><<<grid, kThreads, kSmemBytes, st>>>(
+      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc);
   return cudaGetLastError();
 }
 
@@ -396,16 +407,11 @@ int gemm_tc_init() {
   g_encode = (EncodeTiledFn)fn;
   if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1) g_num_sms = 148;
   cudaError_t e = cudaSuccess;
-#define SET_ALL(BN)                                                              \
-  if (e == cudaSuccess) e = set_smem_attr<BN, false, false, false>();           \
-  if (e == cudaSuccess) e = set_smem_attr<BN, false, false, true>();            \
-  if (e == cudaSuccess) e = set_smem_attr<BN, false, true, false>();            \
-  if (e == cudaSuccess) e = set_smem_attr<BN, false, true, true>();             \
-  if (e == cudaSuccess) e = set_smem_attr<BN, true, true, true>();
-  SET_ALL(256)
-  SET_ALL(128)
-  SET_ALL(64)
-#undef SET_ALL
+  if (e == cudaSuccess) e = set_smem_attr<false, false, false>();
+  if (e == cudaSuccess) e = set_smem_attr<false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr<false, true, false>();
+  if (e == cudaSuccess) e = set_smem_attr<false, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr<true, true, true>();
   if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
   g_init_state = 0;
   return 0;
@@ -431,20 +437,23 @@ bool gemm_tc_eligible(const GemmArgs& g) { return classify(g) != 0; }
 cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   const int form = classify(g);
   if (!form) return cudaErrorInvalidValue;
-  // Tile width: the widest tile keeps the tensor pipe busiest, but a grid that leaves most SMs idle
-  // in its last round (or never fills one round) loses more; score = SM occupancy x per-tile efficiency.
+  // Tile width: wide tiles keep the tensor pipe busiest (less shared-memory traffic per flop), but a
+  // grid that leaves most SMs idle in its last round loses more.  Score every multiple of 32:
+  // fraction of SM-rounds doing work x a per-tile efficiency that falls with narrower tiles.
   int bn = 256;
   {
     const int tm = (g.M + BM - 1) / BM;
     double best = -1.0;
-    const int cand[3] = {256, 128, 64};
-    const double tile_eff[3] = {1.0, 0.88, 0.62};
-    for (int i = 0; i < 3; ++i) {
-      if (cand[i] > 64 && g.N < cand[i]) continue;
-      const int tiles = tm * ((g.N + cand[i] - 1) / cand[i]);
+    const bool b_mn = form != 1;
+    for (int cand = 256; cand >= 64; cand -= 32) {
+      const int tn = (g.N + cand - 1) / cand;
+      const int tiles = tm * tn;
       const int rounds = (tiles + g_num_sms - 1) / g_num_sms;
-      const double score = (double)tiles / ((double)rounds * g_num_sms) * tile_eff[i];
-      if (score > best + 1e-9) { best = score; bn = cand[i]; }
+      const double useful = (double)g.N / ((double)tn * cand);            // columns of the last tile that exist
+      double tile_eff = (double)cand / (cand + 48.0);                      // narrower tiles: more operand traffic per flop
+      if (b_mn) tile_eff *= (double)cand / (double)(((cand + 63) / 64) * 64);   // N-major B is staged in whole 64-wide boxes
+      const double score = (double)tiles / ((double)rounds * g_num_sms) * useful * tile_eff;
+      if (score > best * 1.08) { best = score; bn = cand; }               // leave a wider tile only for a clear gain
     }
   }
   CUtensorMap ta, tb;
@@ -455,14 +464,11 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   if (form == 1) ok = ok && get_map(g.b, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.sbn, (uint32_t)bn, &tb);
   else ok = ok && get_map(g.b, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.sbk, BK, &tb);
   if (!ok) return cudaErrorInvalidValue;
-#define GO(BN)                                                                                     \
-  if (form == 1) return g.out_f32 ? launch_inst<BN, false, false, true>(st, g, ta, tb)             \
-                                  : launch_inst<BN, false, false, false>(st, g, ta, tb);           \
-  if (form == 2) return g.out_f32 ? launch_inst<BN, false, true, true>(st, g, ta, tb)              \
-                                  : launch_inst<BN, false, true, false>(st, g, ta, tb);            \
-  return launch_inst<BN, true, true, true>(st, g, ta, tb);
-  if (bn == 256) { GO(256) } else if (bn == 128) { GO(128) } else { GO(64) }
-#undef GO
+  if (form == 1) return g.out_f32 ? launch_inst<false, false, true>(st, g, ta, tb, bn)
+                                  : launch_inst<false, false, false>(st, g, ta, tb, bn);
+  if (form == 2) return g.out_f32 ? launch_inst<false, true, true>(st, g, ta, tb, bn)
+                                  : launch_inst<false, true, false>(st, g, ta, tb, bn);
+  return launch_inst<true, true, true>(st, g, ta, tb, bn);
 }
 
 const int* gemm_tc_error_device_ptr() {
