@@ -78,7 +78,8 @@ typedef struct {
  * precision of Section "Mixing Precision" (only the active group's fp32 master
  * is on the GPU). */
 typedef struct {
-  int32_t kind;              /* 0 AdamW, 1 AdaGrad, 2 SGD with momentum            */
+  int32_t kind;              /* 0 AdamW, 1 AdaGrad, 2 SGD with momentum, 3 plain SGD
+                                (no optimizer state: only the fp32 master, if any, is paged) */
   int32_t sched;             /* 0 constant, 1 linear decay lr*(1 - cycle/total)    */
   int32_t total_cycles;      /* horizon of the linear schedule                     */
   int32_t offload_state;     /* 1: inactive groups' master+state in pinned host    */
@@ -170,7 +171,8 @@ hift_status hift_last_step_timeline(hift_ctx *ctx, double *ms6);
  * One streaming pass over n elements (the update Algorithm 1 applies to the
  * active group once "UpdateOptimizerParameter" has pointed P at theta_s).  All
  * pointers are device pointers, 16-byte aligned.  master/grad/s0/s1 are fp32;
- * s1 is used by AdamW only (may be NULL otherwise); param_bf16 may be NULL
+ * s1 is used by AdamW only (may be NULL otherwise), s0 by all but plain SGD
+ * (kind 3; may be NULL there); param_bf16 may be NULL
  * (fp32 configs).  tau >= 1 is the number of updates this group has had,
  * including this one (bias correction).  Launches on `cuda_stream`, does not
  * synchronise. */

@@ -584,6 +584,11 @@ def sgdm_update(theta, g, buf, lr, mu):
     return theta, buf
 
 
+def sgd_update(theta, g, lr):
+    """Plain stochastic gradient descent: theta -= lr g (no state; the paper's zero-traffic case)."""
+    return theta - lr * g
+
+
 # --------------------------------------------------------------------------
 # The training step (Algorithm 1)
 # --------------------------------------------------------------------------
@@ -637,9 +642,11 @@ class HiFTOracle:
             elif o.kind == 1:
                 self.master[name], self.s0[name] = adagrad_update(
                     self.master[name], gr, self.s0[name], lr, o.eps)
-            else:
+            elif o.kind == 2:
                 self.master[name], self.s0[name] = sgdm_update(
                     self.master[name], gr, self.s0[name], lr, o.momentum)
+            else:
+                self.master[name] = sgd_update(self.master[name], gr, lr)
         self.last_grads = grads
         self.t += 1
         return loss

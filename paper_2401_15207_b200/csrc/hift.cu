@@ -395,8 +395,8 @@ void attn_bwd(hift_ctx* c, const void* qkv, const void* o, const float* lse, con
   c->step_launches += attention_use_mma(c->mixed, c->dh) ? 2 : 1;   // dsum, dq, dkv or dq, dkv
 }
 void rope(hift_ctx* c, void* qkv, float sign) {
-  const size_t n = (size_t)c->T * c->H * (c->dh / 2);
-  LAUNCH(HIFT_K_ELEMWISE, 8.0 * n * c->es,
+  const size_t n = (size_t)c->T * c->H * (c->dh / 16);      // one thread per 8 pairs
+  LAUNCH(HIFT_K_ELEMWISE, 64.0 * n * c->es,
          if (c->mixed) rope_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>((bf16*)qkv, c->rope_cs, c->T, c->S, c->H, c->dh, sign);
          else rope_kernel<float><<<grid_for(n, 256), 256, 0, c->st>>>((float*)qkv, c->rope_cs, c->T, c->S, c->H, c->dh, sign));
 }
@@ -639,12 +639,12 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
   } else {
     if (c->mixed) { mst = c->master_all + gr.off; pbf = c->params + gr.off * c->es; }
     else mst = (float*)c->params + gr.off;
-    s0 = c->s0_all + gr.off;
+    s0 = c->s0_all ? c->s0_all + gr.off : nullptr;
     s1 = c->s1_all ? c->s1_all + gr.off : nullptr;
   }
   const OptScalars hs = make_opt_scalars(c->oc.kind, lr, c->oc.beta1, c->oc.beta2, c->oc.eps,
                                          c->oc.weight_decay, c->oc.momentum, gr.tau);
-  const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : 20.0) + (pbf ? 2.0 : 0.0));
+  const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
   LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs));
 
   // ---------------- state back to the host (step k)
@@ -703,7 +703,7 @@ float* plane_ptr(hift_ctx* c, int ti, int plane, bool* on_host) {
     return (float*)gr.blob + (size_t)pl * gr.numel + (r.off - gr.off);
   }
   if (plane == 0) return c->master_all + r.off;
-  if (plane == 1) return c->s0_all + r.off;
+  if (plane == 1) return c->s0_all ? c->s0_all + r.off : nullptr;
   return c->s1_all ? c->s1_all + r.off : nullptr;
 }
 
@@ -757,13 +757,14 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     return HIFT_ERR_CFG;
   if (m->d_model % 8 || m->d_ffn % 8 || m->d_model % m->n_heads) return HIFT_ERR_CFG;
   if (!attention_head_ok(m->d_model / m->n_heads)) return HIFT_ERR_CFG;
+  if (m->arch == 2 && (m->d_model / m->n_heads) % 16) return HIFT_ERR_CFG;   // RoPE rotates 8 pairs per thread
   if (m->dtype != 0 && m->dtype != 1) return HIFT_ERR_CFG;
   if (m->arch != 2 && m->max_pos < m->seq) return HIFT_ERR_CFG;
   if (m->arch == 1 && (m->n_classes < 2 || m->tie_head)) return HIFT_ERR_CFG;
   // the embedding-gradient kernel keeps one occurrence list of <= batch*seq ints in shared memory
   if ((int64_t)m->batch * m->seq > 8192) return HIFT_ERR_CFG;
   if (gc->layers_per_group < 1 || gc->order < 0 || gc->order > 2) return HIFT_ERR_CFG;
-  if (oc->kind < 0 || oc->kind > 2 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
+  if (oc->kind < 0 || oc->kind > 3 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
   if (oc->sched == 1 && oc->total_cycles < 1) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
@@ -775,8 +776,9 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   c->L = m->n_blocks; c->d = m->d_model; c->f = m->d_ffn; c->fa = m->arch == 2 ? 2 * m->d_ffn : m->d_ffn;
   c->H = m->n_heads; c->dh = m->d_model / m->n_heads; c->B = m->batch; c->S = m->seq; c->T = m->batch * m->seq;
   c->V = m->vocab; c->Vp = (int)align_up(m->vocab, 128);
-  c->n_state = oc->kind == 0 ? 2 : 1;
-  c->offload = oc->offload_state != 0;
+  c->n_state = oc->kind == 0 ? 2 : (oc->kind == 3 ? 0 : 1);
+  // plain SGD on fp32 parameters has nothing to page (the paper's "no state, zero traffic" case)
+  c->offload = oc->offload_state != 0 && ((m->dtype == 1 ? 1 : 0) + c->n_state) > 0;
   c->n_slots = (c->offload && oc->prefetch_groups) ? 2 : 1;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
@@ -825,8 +827,10 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
       if ((rc = dev_alloc(c, (void**)&c->master_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
       cudaMemsetAsync(c->master_all, 0, c->total * sizeof(float), c->st);
     }
-    if ((rc = dev_alloc(c, (void**)&c->s0_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
-    cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
+    if (c->n_state >= 1) {
+      if ((rc = dev_alloc(c, (void**)&c->s0_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
+    }
     if (c->n_state == 2) {
       if ((rc = dev_alloc(c, (void**)&c->s1_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
       cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
@@ -1020,7 +1024,7 @@ hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
     gr.tau = 0;
   }
   if (!c->offload) {
-    cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
+    if (c->s0_all) cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
     if (c->s1_all) cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
   }
   return cudaStreamSynchronize(c->st) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
@@ -1065,7 +1069,7 @@ hift_status hift_last_step_timeline(hift_ctx* c, double* ms6) {
 hift_status hift_opt_step(int32_t kind, size_t n, void* param_bf16, float* master, const float* grad,
                           float* s0, float* s1, double lr, double b1, double b2, double eps,
                           double wd, double mu, int64_t tau, void* stream) {
-  if (kind < 0 || kind > 2 || !master || !grad || !s0 || (kind == 0 && !s1) || tau < 1) return HIFT_ERR_CFG;
+  if (kind < 0 || kind > 3 || !master || !grad || (kind != 3 && !s0) || (kind == 0 && !s1) || tau < 1) return HIFT_ERR_CFG;
   const uintptr_t al = (uintptr_t)master | (uintptr_t)grad | (uintptr_t)s0 | (uintptr_t)s1 | (uintptr_t)param_bf16;
   if (al & 15) return HIFT_ERR_CFG;
   const OptScalars h = make_opt_scalars(kind, lr, b1, b2, eps, wd, mu, tau);

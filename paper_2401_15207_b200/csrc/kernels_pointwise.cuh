@@ -389,27 +389,37 @@ __global__ void swiglu_bwd_kernel(const T* __restrict__ ds, const T* __restrict_
 // ------------------------------------------------------------------ RoPE
 // In place on the q and k column blocks of qkv[T,3d]: pair (j, j+half) of every head rotated
 // by angle(pos, j) (sign = +1) or its inverse (sign = -1).  cs: [S, half] cos | [S, half] sin.
+// One thread rotates 8 consecutive pairs of q and of k (16-byte accesses); half % 8 == 0.
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ qkv, const float* __restrict__ cs, int64_t Ttot, int S,
                             int H, int dh, float sign) {
-  const int half = dh / 2;
-  const size_t n = (size_t)Ttot * H * half;
+  const int half = dh / 2, hc = half / 8;
+  const size_t n = (size_t)Ttot * H * hc;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   const int d = H * dh;
   for (; i < n; i += stride) {
-    const int j = i % half;
-    const int h = (i / half) % H;
-    const size_t t = i / ((size_t)half * H);
-    const int pos = t % S;
-    const float c = cs[(size_t)pos * half + j];
-    const float s = sign * cs[(size_t)S * half + (size_t)pos * half + j];
+    const int j = (int)(i % hc) * 8;
+    const int h = (int)((i / hc) % H);
+    const size_t t = i / ((size_t)hc * H);
+    const int pos = (int)(t % S);
+    float c[8], sn[8];
+    load8(cs + (size_t)pos * half + j, c);
+    load8(cs + (size_t)S * half + (size_t)pos * half + j, sn);
 #pragma unroll
     for (int part = 0; part < 2; ++part) {          // q then k
-      T* p = qkv + t * 3 * d + (size_t)part * d + (size_t)h * dh;
-      const float x1 = to_f(p[j]), x2 = to_f(p[j + half]);
-      p[j] = from_f<T>(x1 * c - x2 * s);
-      p[j + half] = from_f<T>(x1 * s + x2 * c);
+      T* p = qkv + t * 3 * d + (size_t)part * d + (size_t)h * dh + j;
+      float x1[8], x2[8], y1[8], y2[8];
+      load8(p, x1);
+      load8(p + half, x2);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float s = sign * sn[e];
+        y1[e] = x1[e] * c[e] - x2[e] * s;
+        y2[e] = x1[e] * s + x2[e] * c[e];
+      }
+      store8(p, y1);
+      store8(p + half, y2);
     }
   }
 }
@@ -485,7 +495,7 @@ __global__ void publish_scalars_kernel(const float* __restrict__ src, const int*
 
 // ------------------------------------------------------------------ fused group optimizer
 // One streaming pass over the group's flat buffers: 128-bit loads/stores, 4 elements per
-// thread per iteration.  KIND 0 AdamW, 1 AdaGrad, 2 SGD-momentum.  Scalars precomputed on the
+// thread per iteration.  KIND 0 AdamW, 1 AdaGrad, 2 SGD-momentum, 3 plain SGD (no state).  Scalars precomputed on the
 // host in double: decay = 1 - lr*wd, omb1 = 1-beta1, omb2 = 1-beta2, c1 = 1/(1-beta1^tau),
 // c2 = 1/(1-beta2^tau).  IEEE sqrt and division.
 struct OptScalars {
@@ -504,9 +514,11 @@ __device__ __forceinline__ void opt_update(float& th, float g, float& s0, float&
   } else if (KIND == 1) {
     s0 = s0 + g * g;
     th = th - __fdiv_rn(h.lr * g, __fsqrt_rn(s0) + h.eps);
-  } else {
+  } else if (KIND == 2) {
     s0 = h.mu * s0 + g;
     th = th - h.lr * s0;
+  } else {
+    th = th - h.lr * g;
   }
 }
 template <int KIND, bool HAS_BF16>
@@ -519,7 +531,8 @@ fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const flo
   for (; i < n4; i += stride) {
     float4 th = reinterpret_cast<const float4*>(master)[i];
     const float4 g = __ldcs(reinterpret_cast<const float4*>(grad) + i);
-    float4 a = reinterpret_cast<const float4*>(s0)[i];
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (KIND != 3) a = reinterpret_cast<const float4*>(s0)[i];
     float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
     if (KIND == 0) b = reinterpret_cast<const float4*>(s1)[i];
     opt_update<KIND>(th.x, g.x, a.x, b.x, h);
@@ -527,7 +540,7 @@ fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const flo
     opt_update<KIND>(th.z, g.z, a.z, b.z, h);
     opt_update<KIND>(th.w, g.w, a.w, b.w, h);
     reinterpret_cast<float4*>(master)[i] = th;
-    reinterpret_cast<float4*>(s0)[i] = a;
+    if (KIND != 3) reinterpret_cast<float4*>(s0)[i] = a;
     if (KIND == 0) reinterpret_cast<float4*>(s1)[i] = b;
     if (HAS_BF16) {
       uint2 pk;
@@ -540,10 +553,10 @@ fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const flo
   // ragged tail (n not a multiple of 4)
   const size_t t = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) {
-    float th = master[t], a = s0[t], b = (KIND == 0) ? s1[t] : 0.f;
+    float th = master[t], a = (KIND != 3) ? s0[t] : 0.f, b = (KIND == 0) ? s1[t] : 0.f;
     opt_update<KIND>(th, grad[t], a, b, h);
     master[t] = th;
-    s0[t] = a;
+    if (KIND != 3) s0[t] = a;
     if (KIND == 0) s1[t] = b;
     if (HAS_BF16) param[t] = __float2bfloat16_rn(th);
   }

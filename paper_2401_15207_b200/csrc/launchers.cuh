@@ -200,7 +200,7 @@ inline void launch_fused_opt(cudaStream_t st, int kind, size_t n, void* param_bf
 #define OPT(K)                                                                                         \
   if (param_bf16) fused_opt_kernel<K, true><<<grid, block, 0, st>>>((bf16*)param_bf16, master, grad, s0, s1, n, h); \
   else fused_opt_kernel<K, false><<<grid, block, 0, st>>>(nullptr, master, grad, s0, s1, n, h)
-  if (kind == 0) { OPT(0); } else if (kind == 1) { OPT(1); } else { OPT(2); }
+  if (kind == 0) { OPT(0); } else if (kind == 1) { OPT(1); } else if (kind == 2) { OPT(2); } else { OPT(3); }
 #undef OPT
 }
 

@@ -58,6 +58,19 @@ def test_fused_optimizer_matches_oracle_1e6(kind, n):
     assert np.array_equal(tp.float().cpu().numpy(), O.bf16_round(gm))
 
 
+def test_plain_sgd_kernel_needs_no_state():
+    import torch
+    from paper_2401_15207_b200 import opt_step
+    n = 100003
+    master, grad, _, _ = synth.flat_optimizer_inputs(n, seed=11)
+    tm, tg = _t(master), _t(grad)
+    tp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    opt_step(3, n, tp, tm, tg, None, None, lr=0.5, tau=1)
+    ref = O.sgd_update(master.astype(np.float64), grad.astype(np.float64), 0.5)
+    assert rel_l2(tm.cpu().numpy(), ref) <= 1e-6
+    assert np.array_equal(tp.float().cpu().numpy(), O.bf16_round(tm.cpu().numpy()))
+
+
 def test_fused_optimizer_fp32_params_and_argument_checks():
     import torch
     from paper_2401_15207_b200 import opt_step, HiftError

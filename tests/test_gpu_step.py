@@ -68,6 +68,23 @@ def test_mini_bf16_gpt2_style_groups(kind):
     lockstep(cfg, gc, oc, 5, "zipf", BF16_LOSS, BF16_GRAD, resync=True)
 
 
+@pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
+def test_plain_sgd_pages_only_the_master(dtype):
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(2, dtype)
+    oc = synth.OptCfg(kind=synth.OPT_SGD, lr=1e-2, offload_state=1, prefetch_groups=1)
+    tol = (FP32_LOSS, FP32_GRAD) if dtype == synth.DTYPE_FP32 else (BF16_LOSS, BF16_GRAD)
+    lockstep(cfg, synth.GroupCfg(1), oc, 6, "zipf", tol[0], tol[1], resync=True)
+    h = HiFT(cfg, synth.GroupCfg(1), oc)
+    # fp32 parameters + no state: nothing to page at all; bf16: 4 bytes per parameter (the master)
+    total = sum(synth.count_params(cfg))
+    if dtype == synth.DTYPE_FP32:
+        assert h.pinned_host_bytes() < 64
+    else:
+        assert 4 * total <= h.pinned_host_bytes() < 4 * total + 64 * 1024
+    h.close()
+
+
 def test_free_running_trajectories_stay_close():
     """No resynchronisation: the two trajectories only share the initial weights."""
     cfg = mini(0, synth.DTYPE_BF16, tie_head=1)

@@ -40,6 +40,16 @@ def test_adagrad_and_sgdm_closed_forms():
     assert float(s2) == pytest.approx(th - lr * g1 - lr * (mu * g1 + g2), rel=1e-14)
 
 
+def test_plain_sgd_closed_form_and_torch():
+    th, g = np.array([0.5, -2.0]), np.array([0.25, 4.0])
+    assert np.array_equal(O.sgd_update(th, g, 0.1), np.array([0.5 - 0.025, -2.0 - 0.4]))
+    p = torch.nn.Parameter(torch.tensor(th))
+    opt = torch.optim.SGD([p], lr=0.1)
+    p.grad = torch.tensor(g)
+    opt.step()
+    assert np.allclose(O.sgd_update(th, g, 0.1), p.detach().numpy(), rtol=1e-15)
+
+
 def test_optimizers_against_torch_optim_fp64():
     rng = np.random.default_rng(4)
     n, steps = 257, 5
