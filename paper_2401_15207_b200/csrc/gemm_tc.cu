@@ -21,6 +21,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include <mutex>
 #include <unordered_map>
@@ -327,6 +329,245 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   }
 }
 
+// ------------------------------------------------------------------ CTA-pair kernel
+// Two CTAs of a cluster share one 256 x 256 output tile: each stages its own 128 rows of A and
+// its own 128 columns of B, and one thread of the pair's first CTA issues tcgen05.mma with
+// cta_group::2 (M = 256), which reads both CTAs' shared memory and writes each CTA's half of
+// the accumulator into that CTA's tensor memory.  Per CTA the operand traffic from L2 drops by a
+// third (16 + 16 KB per stage instead of 16 + 32 KB) for the same flops.  No multicast load:
+// every CTA fetches what it stages; only mbarrier signals cross the pair.
+constexpr int kBN2 = 256;
+constexpr int kB2Bytes = (kBN2 / 2) * BK * 2;          // this CTA's half of B
+constexpr int kStage2Bytes = kABytes + kB2Bytes;       // 32 KB
+constexpr int kStages2 = kSmemBudget / kStage2Bytes;   // 6
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion is counted on a barrier that may live in the peer CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"((uint64_t)map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {      // arrives on `bar` in both CTAs of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_c, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_c), "l"(da), "l"(db), "r"(idesc), "r"(accum) : "memory");
+}
+
+template <bool A_MN, bool B_MN, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
+                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
+                int tiles_m, int num_tiles) {
+  constexpr int S = kStages2;
+  constexpr int BN = kBN2;
+  extern __shared__ uint8_t smem_raw[];
+  // both CTAs of a pair read the same flag value only by luck, so decide nothing on it before the
+  // pair has synchronised once; an early exit of one CTA alone would strand its peer
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = base + S * kStage2Bytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  auto acc_full = [&](int a) { return bar_base + 8u * (2 * S + a); };
+  auto acc_empty = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
+  const uint32_t tmem_slot = bar_base + 8u * (2 * S + 4);
+  uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + S * kStage2Bytes + 8 * (2 * S + 4));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (K + BK - 1) / BK;
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(acc_full(a), 1); mbar_init(acc_empty(a), 8); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(2 * kAccStride) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();                                  // barriers of both CTAs are initialised
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_gen;
+  const bool poisoned = *(volatile int*)&g_tc_error != 0;   // read after the pair sync; see the exit below
+
+  if (warp == 0) {
+    // ---------------- TMA producer (one thread per CTA): own rows of A, own columns of B;
+    //                  completion is counted on the first CTA's barrier
+    if (lane == 0 && !poisoned) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM;
+        const int n0 = (tile / tiles_m) * BN + (int)rank * (BN / 2);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); ok = false; break; }
+          const uint32_t sa = base + s * kStage2Bytes, sb = sa + kABytes;
+          const uint32_t fb = map_to_cta(full_bar(s), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStage2Bytes);
+          const int k0 = kb * BK;
+          if (A_MN) {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, fb, m0 + j * 64, k0);
+          } else {
+            tma_load_2d_pair(sa, &tmap_a, fb, k0, m0);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int j = 0; j < BN / 128; ++j) tma_load_2d_pair(sb + j * (BK * 128), &tmap_b, fb, n0 + j * 64, k0);
+          } else {
+            tma_load_2d_pair(sb, &tmap_b, fb, k0, n0);
+          }
+          if (++s == S) { s = 0; ph ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: one thread of the pair's first CTA
+    if (lane == 0 && rank == 0 && !poisoned) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                             ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      int s = 0, lt = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++lt) {
+        const int ab = lt & 1;
+        const uint32_t aph = (lt >> 1) & 1;
+        if (!mbar_wait(acc_empty(ab), aph ^ 1)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + (uint32_t)(ab * kAccStride);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(s), ph)) { atomicCAS(&g_tc_error, 0, 2); ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + s * kStage2Bytes, sb = sa + kABytes;
+          const uint64_t da = make_desc(sa, A_MN), db = make_desc(sb, B_MN);
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            const uint64_t adv_a = A_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
+            const uint64_t adv_b = B_MN ? (uint64_t)(kk * UMMA_K * 128 >> 4) : (uint64_t)(kk * UMMA_K * 2 >> 4);
+            tc_mma_pair(tacc, da + adv_a, db + adv_b, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit_pair(empty_bar(s));      // frees the stage in both CTAs
+          if (++s == S) { s = 0; ph ^= 1; }
+        }
+        tc_commit_pair(acc_full(ab));        // both CTAs' epilogues may drain their half
+      }
+    }
+  } else {
+    // ---------------- epilogue (both CTAs): tensor-memory lanes 32*(warp%4).. hold rows of this CTA's half
+    const int q = warp & 3;
+    int lt = 0;
+    for (int tile = pair; tile < num_tiles && !poisoned; tile += num_pairs, ++lt) {
+      const int ab = lt & 1;
+      const uint32_t aph = (lt >> 1) & 1;
+      const bool ready = mbar_wait(acc_full(ab), aph);
+      if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 3);
+      tc_fence_after();
+      if (!__all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0)) break;
+      const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM, n0 = (tile / tiles_m) * BN;
+      const int m = m0 + q * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (n0 + c0 >= N) break;
+        uint32_t v[32];
+        tmem_ld32(taddr + c0, v);
+        if (m < M) {
+          const int n = n0 + c0;
+          float f[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+          if (n + 32 <= N) {
+            if (bias) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                const uint4 b4 = *reinterpret_cast<const uint4*>(bias + n + j);
+                const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b4);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                  const float2 bf = __bfloat1622float2(hb[t]);
+                  f[j + 2 * t] += bf.x; f[j + 2 * t + 1] += bf.y;
+                }
+              }
+            }
+            if (OUT_F32) {
+              float* crow = reinterpret_cast<float*>(cptr) + (int64_t)m * ldc + n;
+              if (residual) {
+                const float* rrow = residual + (int64_t)m * ldr + n;
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                  const float4 r = *reinterpret_cast<const float4*>(rrow + j);
+                  f[j] += r.x; f[j + 1] += r.y; f[j + 2] += r.z; f[j + 3] += r.w;
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(crow + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+            } else {
+              __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * ldc + n;
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 o;
+                __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) ho[t] = __floats2bfloat162_rn(f[j + 2 * t], f[j + 2 * t + 1]);
+                *reinterpret_cast<uint4*>(crow + j) = o;
+              }
+            }
+          } else {
+            for (int j = 0; j < 32 && n + j < N; ++j) {
+              float x = f[j];
+              if (bias) x += __bfloat162float(bias[n + j]);
+              if (OUT_F32) {
+                if (residual) x += residual[(int64_t)m * ldr + n + j];
+                reinterpret_cast<float*>(cptr)[(int64_t)m * ldc + n + j] = x;
+              } else {
+                reinterpret_cast<__nv_bfloat16*>(cptr)[(int64_t)m * ldc + n + j] = __float2bfloat16_rn(x);
+              }
+            }
+          }
+        }
+      }
+      // hand this CTA's half of the accumulator back: the MMA thread counts 8 warps (4 per CTA)
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(map_to_cta(acc_empty(ab), 0));
+    }
+  }
+  // nobody leaves while the peer may still signal this CTA's barriers or read its shared memory
+  tc_fence_before();
+  cluster_sync_all();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kAccStride) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -388,6 +629,32 @@ cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   return cudaGetLastError();
 }
 
+template <bool A_MN, bool B_MN, bool OUT_F32>
+cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& ta, const CUtensorMap& tb) {
+  const int tiles_m = (g.M + 2 * BM - 1) / (2 * BM), tiles_n = (g.N + kBN2 - 1) / kBN2;
+  const int num_tiles = tiles_m * tiles_n;
+  int pairs = g_num_sms / 2;
+  if (num_tiles < pairs) pairs = num_tiles;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
+                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles);
+}
+template <bool A_MN, bool B_MN, bool OUT_F32>
+cudaError_t set_smem_attr2() {
+  return cudaFuncSetAttribute(gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+int g_pair_mode = 1;     // CTA-pair kernel for 256-wide tiles (HIFT_GEMM_PAIR=0 falls back to one CTA per tile)
+
 }  // namespace
 
 int gemm_tc_init() {
@@ -412,6 +679,12 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr<false, true, false>();
   if (e == cudaSuccess) e = set_smem_attr<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr<true, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr2<false, false, false>();
+  if (e == cudaSuccess) e = set_smem_attr2<false, false, true>();
+  if (e == cudaSuccess) e = set_smem_attr2<false, true, false>();
+  if (e == cudaSuccess) e = set_smem_attr2<false, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr2<true, true, true>();
+  if (const char* pm = getenv("HIFT_GEMM_PAIR")) g_pair_mode = atoi(pm);
   if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
   g_init_state = 0;
   return 0;
@@ -458,6 +731,17 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   }
   CUtensorMap ta, tb;
   bool ok;
+  if (g_pair_mode && bn == 256 && g.M >= 256) {
+    // CTA pair: each CTA stages 128 rows of A and 128 columns of B
+    if (form == 3) ok = get_map(g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.sak, BK, &ta);
+    else ok = get_map(g.a, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.sam, BM, &ta);
+    if (form == 1) ok = ok && get_map(g.b, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.sbn, (uint32_t)(kBN2 / 2), &tb);
+    else ok = ok && get_map(g.b, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.sbk, BK, &tb);
+    if (!ok) return cudaErrorInvalidValue;
+    if (form == 1) return g.out_f32 ? launch_pair<false, false, true>(st, g, ta, tb) : launch_pair<false, false, false>(st, g, ta, tb);
+    if (form == 2) return g.out_f32 ? launch_pair<false, true, true>(st, g, ta, tb) : launch_pair<false, true, false>(st, g, ta, tb);
+    return launch_pair<true, true, true>(st, g, ta, tb);
+  }
   // K-major operand: tensor [rows = M or N][inner = K]; MN-major operand: tensor [rows = K][inner = M or N]
   if (form == 3) ok = get_map(g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.sak, BK, &ta);
   else ok = get_map(g.a, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.sam, BM, &ta);
