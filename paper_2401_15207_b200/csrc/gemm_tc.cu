@@ -710,10 +710,12 @@ bool gemm_tc_eligible(const GemmArgs& g) { return classify(g) != 0; }
 cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   const int form = classify(g);
   if (!form) return cudaErrorInvalidValue;
-  // Tile width: wide tiles keep the tensor pipe busiest (less shared-memory traffic per flop), but a
-  // grid that leaves most SMs idle in its last round loses more.  Score every multiple of 32:
-  // fraction of SM-rounds doing work x a per-tile efficiency that falls with narrower tiles.
+  // Tile choice.  Wide tiles keep the tensor pipe busiest (less operand traffic per flop), the CTA-pair
+  // kernel (256 x 256 per pair) more so; but a grid that leaves most SMs idle in its last round loses
+  // more.  Score = fraction of SM-rounds doing work x columns that exist x a per-tile efficiency
+  // (measured: pair 1.0, one CTA at width w about 0.87 * (w / (w + 48)) / (256 / 304)).
   int bn = 256;
+  bool use_pair = false;
   {
     const int tm = (g.M + BM - 1) / BM;
     double best = -1.0;
@@ -723,15 +725,23 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
       const int tiles = tm * tn;
       const int rounds = (tiles + g_num_sms - 1) / g_num_sms;
       const double useful = (double)g.N / ((double)tn * cand);            // columns of the last tile that exist
-      double tile_eff = (double)cand / (cand + 48.0);                      // narrower tiles: more operand traffic per flop
+      double tile_eff = 0.87 * ((double)cand / (cand + 48.0)) / (256.0 / 304.0);
       if (b_mn) tile_eff *= (double)cand / (double)(((cand + 63) / 64) * 64);   // N-major B is staged in whole 64-wide boxes
       const double score = (double)tiles / ((double)rounds * g_num_sms) * useful * tile_eff;
       if (score > best * 1.08) { best = score; bn = cand; }               // leave a wider tile only for a clear gain
     }
+    if (g_pair_mode && g.M >= 256 && g.N >= 256) {
+      const int pm = (g.M + 2 * BM - 1) / (2 * BM), pn = (g.N + kBN2 - 1) / kBN2;
+      const int pairs = g_num_sms / 2, ptiles = pm * pn;
+      const int rounds = (ptiles + pairs - 1) / pairs;
+      const double useful = ((double)g.N / ((double)pn * kBN2)) * ((double)g.M / ((double)pm * 2 * BM));
+      const double score = (double)ptiles / ((double)rounds * pairs) * useful;
+      if (score >= best) use_pair = true;
+    }
   }
   CUtensorMap ta, tb;
   bool ok;
-  if (g_pair_mode && bn == 256 && g.M >= 256) {
+  if (use_pair) {
     // CTA pair: each CTA stages 128 rows of A and 128 columns of B
     if (form == 3) ok = get_map(g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.sak, BK, &ta);
     else ok = get_map(g.a, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.sam, BM, &ta);
