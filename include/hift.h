@@ -167,6 +167,14 @@ hift_status hift_last_step_paging(const hift_ctx *ctx, size_t *h2d_bytes, size_t
  * for the copies to finish. */
 hift_status hift_last_step_timeline(hift_ctx *ctx, double *ms6);
 
+/* The tensor-core GEMM bounds every device-side wait; a wait that gives up records a code in a
+ * device flag, after which every tensor-core GEMM launch returns at once and hift_step reports
+ * HIFT_ERR_TIMEOUT.  This call reads the flag (set_value < 0) or overwrites it first
+ * (set_value >= 0; 0 clears it, which is how a caller resumes after a time-out, and a non-zero
+ * value lets a test walk the time-out path without stalling anything).  Returns the flag, or -1
+ * if the tensor-core path is unavailable.  Synchronises the device. */
+int32_t hift_tc_error_flag(int32_t set_value);
+
 /* ---- the group-local fused optimizer on caller-owned flat buffers --------
  * One streaming pass over n elements (the update Algorithm 1 applies to the
  * active group once "UpdateOptimizerParameter" has pointed P at theta_s).  All

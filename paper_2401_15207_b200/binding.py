@@ -84,6 +84,7 @@ def _prototypes():
         "hift_last_step_launches": (i64, [vp]),
         "hift_last_step_paging": (C.c_int, [vp, C.POINTER(sz), C.POINTER(sz)]),
         "hift_last_step_timeline": (C.c_int, [vp, C.POINTER(f64)]),
+        "hift_tc_error_flag": (i32, [i32]),
         "hift_opt_step": (C.c_int, [i32, sz, vp, vp, vp, vp, vp, f64, f64, f64, f64, f64, f64, i64, vp]),
         "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
@@ -290,6 +291,10 @@ def opt_step(kind, n, param_bf16, master, grad, s0, s1, lr, beta1=0.9, beta2=0.9
              weight_decay=0.0, momentum=0.9, tau=1, stream=None):
     _check(lib().hift_opt_step(kind, n, _ptr(param_bf16), _ptr(master), _ptr(grad), _ptr(s0), _ptr(s1),
                                lr, beta1, beta2, eps, weight_decay, momentum, tau, _st(stream)), "hift_opt_step")
+
+
+def tc_error_flag(set_value: int = -1) -> int:
+    return lib().hift_tc_error_flag(set_value)
 
 
 def k_linear(form, dtype, M, N, K, a, b, out, bias=None, residual=None, path=0, stream=None):

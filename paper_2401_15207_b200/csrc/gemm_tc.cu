@@ -775,6 +775,10 @@ const int* gemm_tc_error_device_ptr() {
   return ptr;
 }
 
+int gemm_tc_set_error(int v) {
+  return cudaMemcpyToSymbol(g_tc_error, &v, sizeof(int)) == cudaSuccess ? 0 : -1;
+}
+
 int gemm_tc_poll_error() {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)) != cudaSuccess) return -1;

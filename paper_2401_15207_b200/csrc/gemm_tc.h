@@ -17,6 +17,9 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g);
 // 0 if no tensor-core kernel has given up on a bounded wait since the library was loaded, else the
 // code of the first one (1 producer, 2 MMA issuer, 3 epilogue); -1 if the flag cannot be read.
 int gemm_tc_poll_error();
+// Overwrites the flag (0 clears it).  While it is non-zero every tensor-core GEMM launch returns without
+// computing, which is what a launch after a real time-out does.  0 on success.
+int gemm_tc_set_error(int v);
 // Device address of that flag (an int), or nullptr if it cannot be resolved.
 const int* gemm_tc_error_device_ptr();
 

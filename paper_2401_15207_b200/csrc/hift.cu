@@ -1065,6 +1065,13 @@ hift_status hift_last_step_timeline(hift_ctx* c, double* ms6) {
   return HIFT_OK;
 }
 
+int32_t hift_tc_error_flag(int32_t set_value) {
+  if (gemm_tc_init() != 0) return -1;
+  cudaDeviceSynchronize();
+  if (set_value >= 0 && gemm_tc_set_error(set_value) != 0) return -1;
+  return gemm_tc_poll_error();
+}
+
 // ---------------------------------------------------------------- optimizer on flat buffers
 hift_status hift_opt_step(int32_t kind, size_t n, void* param_bf16, float* master, const float* grad,
                           float* s0, float* s1, double lr, double b1, double b2, double eps,

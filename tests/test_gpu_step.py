@@ -142,3 +142,37 @@ def test_step_host_matches_step_and_is_deterministic():
     for o in outs[1:]:
         assert o[0] == outs[0][0]                         # same bits, run to run and across entry points
         assert np.array_equal(o[1], outs[0][1]) and np.array_equal(o[2], outs[0][2])
+
+
+def test_timeout_flag_path_reports_and_recovers():
+    """Walk the time-out path without stalling anything: with the flag set, every tensor-core GEMM
+    returns at once (releasing its tensor memory), the step reports HIFT_ERR_TIMEOUT, and after the
+    flag is cleared the same context computes correct steps again."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError, tc_error_flag
+    cfg = synth.ModelCfg(arch=2, n_blocks=2, d_model=512, n_heads=4, d_ffn=1024, vocab=1000, norm_eps=1e-6,
+                         dtype=synth.DTYPE_BF16, batch=2, seq=256)
+    gc, oc = synth.GroupCfg(1), synth.OptCfg(kind=2, lr=1e-3)
+    p0 = synth.init_params(cfg, 3)
+    tok, lab = synth.lm_batch(cfg, 1, 0)
+    tt, ll = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
+    ref = HiFT(cfg, gc, oc)
+    ref.set_params(p0)
+    good = [ref.step(tt, ll) for _ in range(2)]
+    ref.close()
+    h = HiFT(cfg, gc, oc)
+    h.set_params(p0)
+    assert tc_error_flag() == 0
+    try:
+        assert tc_error_flag(2) == 2
+        with pytest.raises(HiftError) as e:
+            h.step(tt, ll)
+        assert e.value.status == 6                      # HIFT_ERR_TIMEOUT
+    finally:
+        assert tc_error_flag(0) == 0
+    h.set_params(p0)                                    # the aborted step updated group 0 from garbage
+    h2 = HiFT(cfg, gc, oc)                              # a fresh context and the recovered one agree with the reference
+    h2.set_params(p0)
+    assert h2.step(tt, ll) == good[0]
+    h2.close()
+    h.close()

@@ -1,0 +1,82 @@
+"""The pins must be able to fail: plant plausible mistakes in the oracle (on the CPU) and check
+that the finite-difference / closed-form / library pins catch each of them."""
+import numpy as np
+import pytest
+
+import synth
+from oracle import hift_oracle as O
+from test_oracle_math import _fd_check, mini
+
+
+def _expect_caught(fn):
+    with pytest.raises(AssertionError):
+        fn()
+
+
+def test_wrong_sign_in_rope_backward_is_caught(monkeypatch):
+    orig = O.rope_apply
+    monkeypatch.setattr(O, "rope_apply", lambda x, c, s, inverse=False: orig(x, c, s, inverse=False))
+    _expect_caught(lambda: _fd_check(mini(2), n_samples=3))
+
+
+def test_dropped_term_in_gelu_derivative_is_caught(monkeypatch):
+    import math
+    from scipy.special import erf
+    monkeypatch.setattr(O, "gelu_bwd", lambda d, a: d * 0.5 * (1.0 + erf(a / math.sqrt(2.0))))   # a*pdf term dropped
+    _expect_caught(lambda: _fd_check(mini(0), n_samples=3))
+
+
+def test_missing_attention_scale_in_dk_is_caught(monkeypatch):
+    orig = O.attention_bwd
+
+    def bad(do, q, k, v, p):
+        dq, dk, dv = orig(do, q, k, v, p)
+        return dq, dk * np.sqrt(q.shape[-1]), dv
+    monkeypatch.setattr(O, "attention_bwd", bad)
+    _expect_caught(lambda: _fd_check(mini(1), n_samples=3))
+
+
+def test_layernorm_backward_without_mean_subtraction_is_caught(monkeypatch):
+    def bad(dy, cache, g):
+        xhat, rstd = cache
+        dg = (dy * xhat).reshape(-1, xhat.shape[-1]).sum(axis=0)
+        db = dy.reshape(-1, xhat.shape[-1]).sum(axis=0)
+        dxh = dy * g
+        return rstd * (dxh - xhat * (dxh * xhat).mean(axis=-1, keepdims=True)), dg, db
+    monkeypatch.setattr(O, "layernorm_bwd", bad)
+    _expect_caught(lambda: _fd_check(mini(0), n_samples=3))
+
+
+def test_transposed_weight_gradient_is_caught():
+    # a transposed dW has the wrong shape unless the layer is square: w_o is square, so plant it there
+    cfg = mini(0)
+    P = {k: v.astype(np.float64) for k, v in synth.init_params(cfg, 3, perturb=0.1).items()}
+    tok, lab = synth.batch_for(cfg, 11, 0, dist="uniform")
+    loss, cache = O.forward(cfg, P, tok, lab)
+    G = O.backward(cfg, P, cache, None)
+    h = 1e-5
+    name, i, j = "b0.w_o", 3, 7
+    P[name][i, j] += h
+    lp, _ = O.forward(cfg, P, tok, lab)
+    P[name][i, j] -= 2 * h
+    lm, _ = O.forward(cfg, P, tok, lab)
+    fd = (lp - lm) / (2 * h)
+    assert abs(fd - G[name][i, j]) < 1e-6 * np.abs(G[name]).max()
+    assert abs(fd - G[name].T[i, j]) > 1e-3 * np.abs(G[name]).max()       # the transposed entry would not pass
+
+
+def test_bias_correction_with_global_step_is_caught():
+    # Adam with the global step count instead of the group's update count gives a different update
+    th, g = np.array([0.3]), np.array([0.02])
+    a, _, _ = O.adamw_update(th, g, np.zeros(1), np.zeros(1), 1e-3, 0.9, 0.999, 1e-8, 0.0, 1)
+    b, _, _ = O.adamw_update(th, g, np.zeros(1), np.zeros(1), 1e-3, 0.9, 0.999, 1e-8, 0.0, 7)
+    assert abs(a[0] - (0.3 - 1e-3 * 0.02 / (0.02 + 1e-8))) < 1e-15
+    assert abs(a[0] - b[0]) > 1e-5
+
+
+def test_eps_inside_the_square_root_is_caught():
+    th, g, eps = 0.5, 1e-6, 1e-8
+    t1, _, _ = O.adamw_update(np.array(th), np.array(g), np.array(0.0), np.array(0.0), 1e-2, 0.9, 0.999, eps, 0.0, 1)
+    outside = th - 1e-2 * g / (abs(g) + eps)
+    inside = th - 1e-2 * g / np.sqrt(g * g + eps)
+    assert abs(float(t1) - outside) < 1e-15 and abs(float(t1) - inside) > 1e-4
