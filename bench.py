@@ -208,6 +208,12 @@ def run_ours(args, cfg, gcfg, ocfg):
     dev = [(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for a, b in host[:W + K]]
     groups = [h.group_units(g) for g in range(k)]
 
+    step_host = h.step_host
+    if args.parallel == "dp":
+        h.step = lambda tok, lab: dist_util.data_parallel_step(h, tok, lab)
+        # end to end in this mode: pageable host batch -> device inside the timed call, then the same step
+        step_host = lambda tok, lab: h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
+
     # ---- device-resident leg, timed twice over the same K steps' worth of work: once plain (the
     #      reported value) and once with every kernel launch bracketed by CUDA events on the
     #      launching stream (the roofline figures; the brackets cost a few per cent)
@@ -253,11 +259,11 @@ def run_ours(args, cfg, gcfg, ocfg):
     ms_e2e = float("nan")
     if not args.skip_e2e:
         for t in range(W):
-            h.step_host(*host[W + K + t])
+            step_host(*host[W + K + t])
         barrier()
         e0.record()
         for t in range(K):
-            last_loss = h.step_host(*host[2 * W + K + t])
+            last_loss = step_host(*host[2 * W + K + t])
         e1.record()
         barrier()
         ms_e2e = e0.elapsed_time(e1)
@@ -311,7 +317,7 @@ def run_ours(args, cfg, gcfg, ocfg):
             "config": {"workload": args.workload, "global_batch": cfg.batch * world, "seq_len": cfg.seq,
                        "groups": k, "groups_trained": trained, "optimizer": ["adamw", "adagrad", "sgdm"][ocfg.kind],
                        "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups,
-                       "parallelism": "replicas" if world > 1 else "single",
+                       "parallelism": (("dp%d" % world) if args.parallel == "dp" else "replicas") if world > 1 else "single",
                        "l2_policy": "inputs larger than L2 (weights + activations of a step exceed 126 MB)"},
             "peak_hbm_gb": peak_hbm / 1e9, "pinned_host_gb": pinned / 1e9,
             "paging_bytes_per_step": {"h2d": paging[0], "d2h": paging[1]},
@@ -447,6 +453,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b", choices=sorted(WORKLOADS))
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "dp"],
+                    help="N > 1: independent replicas (default), or data parallel with an NCCL all-reduce of the "
+                         "active group's gradient between the backward pass and the update")
     ap.add_argument("--prefetch", type=int, default=1)
     ap.add_argument("--offload", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -111,6 +111,20 @@ hift_status hift_step(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *l
 hift_status hift_step_host(hift_ctx *ctx, const int32_t *tokens_host, const int32_t *labels_host,
                            float *loss_host);
 
+/* The same step in two halves, for data-parallel training (several contexts, one per GPU, each
+ * on its shard of the batch; the paper's method itself is single-device).  hift_step_begin runs
+ * the forward pass and the truncated backward pass and returns the loss; the active group's flat
+ * fp32 gradient (its tensors in layout order, zero in the alignment gaps) is then exposed by
+ * hift_grad_view as a device pointer the caller may reduce over ranks and scale (1/k of the
+ * volume a full-parameter step would exchange); hift_step_end applies the optimizer to the group,
+ * starts the state write-back and advances t.  Work the caller enqueued on the stream given to
+ * hift_create is ordered before the update.  begin/end must alternate; hift_step in between is
+ * refused with HIFT_ERR_CFG. */
+hift_status hift_step_begin(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *labels_dev,
+                            float *loss_host);
+hift_status hift_grad_view(hift_ctx *ctx, float **grad_dev, size_t *n);
+hift_status hift_step_end(hift_ctx *ctx);
+
 int32_t hift_active_group(const hift_ctx *ctx);   /* group the NEXT hift_step trains */
 int32_t hift_num_groups(const hift_ctx *ctx);     /* k                               */
 int64_t hift_step_count(const hift_ctx *ctx);     /* t, steps taken so far           */

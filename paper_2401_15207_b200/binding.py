@@ -63,6 +63,9 @@ def _prototypes():
         "hift_destroy": (None, [vp]),
         "hift_step": (C.c_int, [vp, vp, vp, pf]),
         "hift_step_host": (C.c_int, [vp, vp, vp, pf]),
+        "hift_step_begin": (C.c_int, [vp, vp, vp, pf]),
+        "hift_grad_view": (C.c_int, [vp, C.POINTER(vp), C.POINTER(sz)]),
+        "hift_step_end": (C.c_int, [vp]),
         "hift_active_group": (i32, [vp]),
         "hift_num_groups": (i32, [vp]),
         "hift_step_count": (i64, [vp]),
@@ -186,6 +189,25 @@ class HiFT:
         st = lib().hift_step_host(self._h, tokens.ctypes.data, labels.ctypes.data, C.byref(loss))
         _check(st, "hift_step_host")
         return loss.value
+
+    def step_begin(self, tokens, labels) -> float:
+        """Forward + truncated backward; the group's gradient stays on the device (see grad_view)."""
+        loss = C.c_float()
+        _check(lib().hift_step_begin(self._h, tokens.data_ptr(), labels.data_ptr(), C.byref(loss)), "hift_step_begin")
+        return loss.value
+
+    def grad_view(self):
+        """The active group's flat fp32 gradient as a torch CUDA tensor sharing the library's memory."""
+        import torch
+        ptr, n = C.c_void_p(), C.c_size_t()
+        _check(lib().hift_grad_view(self._h, C.byref(ptr), C.byref(n)), "hift_grad_view")
+
+        class _View:
+            __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<f4", "data": (ptr.value, False), "version": 3}
+        return torch.as_tensor(_View(), device="cuda")
+
+    def step_end(self):
+        _check(lib().hift_step_end(self._h), "hift_step_end")
 
     # -- getters
     def active_group(self) -> int:

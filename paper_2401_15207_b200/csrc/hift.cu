@@ -73,6 +73,8 @@ struct hift_ctx {
   size_t total = 0, max_group = 0;
   int64_t t = 0;
   int forced = -1, last_group = -1;
+  int cur_sl = 0; double cur_lr = 0.0;   // slot and learning rate of the step in flight
+  bool pending_update = false;           // between hift_step_begin and hift_step_end
 
   // device memory
   std::vector<void*> dev_allocs;
@@ -514,7 +516,9 @@ void issue_h2d(hift_ctx* c, int g, int sl, bool after_forward) {
   c->step_h2d = gr.blob_bytes;
 }
 
-hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
+// Forward and truncated backward of one step, enqueued on the context's stream; the active group's
+// gradient is left in c->grad.
+hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int32_t* lab) {
   const hift_model_cfg& m = c->m;
   const int L = c->L, T = c->T, d = c->d, V = c->V, Vp = c->Vp, B = c->B, S = c->S;
   const int k = (int)c->groups.size();
@@ -526,6 +530,7 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
   c->step_launches = 0; c->step_h2d = 0; c->step_d2h = 0;
   c->first_err = cudaSuccess;
   const int sl = c->n_slots == 2 ? (int)(c->t & 1) : 0;
+  c->cur_sl = sl; c->cur_lr = lr;
   auto active = [&](int u) { return u >= lo && u <= hi; };
 
   plan_slots(c, g, true);
@@ -625,6 +630,14 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
     }
   }
 
+  return HIFT_OK;
+}
+
+// Optimizer on the active group and write-back of its state, enqueued after the backward pass.
+void enqueue_update(hift_ctx* c) {
+  GroupRec& gr = c->groups[c->last_group];
+  const int sl = c->cur_sl;
+  const double lr = c->cur_lr;
   // ---------------- group-local optimizer (Algorithm 1: P now points at theta_s only)
   gr.tau += 1;
   float *mst, *s0, *s1;
@@ -659,13 +672,16 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
     c->d2h_pending[sl] = true;
     c->step_d2h = gr.blob_bytes;
   }
+}
 
+// Publishes the step's scalars, waits for the compute stream, and turns what it finds into a status.
+hift_status finish_step(hift_ctx* c, float* loss_host, bool advance) {
   // the loss goes to mapped host memory by a kernel store: a copy would queue behind the state transfers
   publish_scalars_kernel<<<1, 32, 0, c->st>>>(c->scal, c->mixed ? gemm_tc_error_device_ptr() : nullptr, c->scal_host_dev);
   c->note(cudaGetLastError());
   c->note(cudaStreamSynchronize(c->st));
   c->prof_collect();
-  c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
+  if (advance) c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
   if (c->first_err != cudaSuccess) return HIFT_ERR_CUDA;
   int tc_err;
   memcpy(&tc_err, &c->scal_host[3], sizeof(int));
@@ -677,6 +693,14 @@ hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* 
   if (bad_h) return HIFT_ERR_INPUT;
   if (!isfinite(loss)) return HIFT_ERR_NONFINITE;
   return HIFT_OK;
+}
+
+hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
+  if (c->pending_update) return HIFT_ERR_CFG;       // hift_step_begin without hift_step_end
+  const hift_status s = enqueue_forward_backward(c, tok, lab);
+  if (s != HIFT_OK) return s;
+  enqueue_update(c);
+  return finish_step(c, loss_host, true);
 }
 
 void sync_all(hift_ctx* c) {
@@ -903,6 +927,34 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
 hift_status hift_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
   if (!c || !tok || !lab) return HIFT_ERR_INPUT;
   return do_step(c, tok, lab, loss_host);
+}
+
+hift_status hift_step_begin(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
+  if (!c || !tok || !lab) return HIFT_ERR_INPUT;
+  if (c->pending_update) return HIFT_ERR_CFG;
+  hift_status s = enqueue_forward_backward(c, tok, lab);
+  if (s != HIFT_OK) return s;
+  s = finish_step(c, loss_host, false);
+  if (s == HIFT_OK || s == HIFT_ERR_NONFINITE) c->pending_update = true;
+  return s;
+}
+hift_status hift_grad_view(hift_ctx* c, float** grad_dev, size_t* n) {
+  if (!c || !grad_dev || !n || c->last_group < 0) return HIFT_ERR_CFG;
+  *grad_dev = c->grad;
+  *n = c->groups[c->last_group].numel;
+  return HIFT_OK;
+}
+hift_status hift_step_end(hift_ctx* c) {
+  if (!c || !c->pending_update) return HIFT_ERR_CFG;
+  // whatever the caller did to the gradient on its own stream is ordered before the update
+  c->note(cudaEventRecord(c->ev_in, c->caller));
+  c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
+  enqueue_update(c);
+  c->pending_update = false;
+  c->note(cudaStreamSynchronize(c->st));
+  c->prof_collect();
+  c->t += 1;
+  return c->first_err == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 
 hift_status hift_step_host(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {

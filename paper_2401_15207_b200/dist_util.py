@@ -39,3 +39,23 @@ def aggregate_throughput(units_per_rank: float, seconds_per_rank: float, device:
     _, n = world()
     (slowest,) = max_over_ranks([seconds_per_rank], device)
     return units_per_rank * n / slowest
+
+
+def allreduce_mean_(tensor):
+    """In-place mean over ranks of a gradient buffer (sum all-reduce, then 1/world): the one exchange
+    of data-parallel HiFT, over the active group's flat gradient only."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(tensor, op=dist.ReduceOp.SUM)
+        tensor.mul_(1.0 / dist.get_world_size())
+    return tensor
+
+
+def data_parallel_step(h, tokens, labels) -> float:
+    """One data-parallel step of context `h` on this rank's shard: forward + truncated backward,
+    mean of the group's gradient over ranks, update.  Every rank follows the same group schedule,
+    so no communication is needed to agree on the group."""
+    loss = h.step_begin(tokens, labels)
+    allreduce_mean_(h.grad_view())
+    h.step_end()
+    return loss

@@ -26,6 +26,9 @@ def _worker(rank, world, port, out):
         # rank r "measures" r+1 seconds and 10*(r+1) ms: the job is as slow as its slowest rank
         mx = dist_util.max_over_ranks([float(rank + 1), 10.0 * (rank + 1)])
         thr = dist_util.aggregate_throughput(2048.0, float(rank + 1))
+        gbuf = torch.full((5,), float(rank + 1))          # rank r holds gradient r+1 everywhere
+        dist_util.allreduce_mean_(gbuf)
+        assert torch.equal(gbuf, torch.full((5,), 1.5))   # mean of 1 and 2 on both ranks
         seeds = [None] * world
         dist.all_gather_object(seeds, dist_util.rank_seed(77, rank))
         dist.barrier()
