@@ -51,6 +51,26 @@ __device__ __forceinline__ void stage_tile(uint8_t* tile, const bf16* __restrict
     *reinterpret_cast<uint4*>(tile + swz<DH>(r, c * 8)) = v;
   }
 }
+// The same through cp.async (16 bytes per request, zero-filled past the end), so that the next
+// tile streams in while the tensor cores work on the current one.
+__device__ __forceinline__ void cp_async16(uint32_t saddr, const void* g, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(saddr), "l"(g), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+template <int ROWS, int DH>
+__device__ __forceinline__ void stage_tile_async(uint32_t tile, const bf16* __restrict__ g, int64_t pitch,
+                                                 int row0, int rows_total) {
+  constexpr int CH = DH / 8;
+  for (int idx = threadIdx.x; idx < ROWS * CH; idx += blockDim.x) {
+    const int r = idx / CH, c = idx % CH;
+    const bool ok = row0 + r < rows_total;
+    const bf16* src = g + (int64_t)(ok ? row0 + r : 0) * pitch + c * 8;
+    cp_async16(tile + swz<DH>(r, c * 8), src, ok);
+  }
+}
+
 // A fragment (16 rows x 16 k) of a row-major tile at (r0, c0)
 template <int DH>
 __device__ __forceinline__ void load_a(uint32_t (&a)[4], uint32_t tile, int r0, int c0, int lane) {
@@ -69,14 +89,18 @@ __device__ __forceinline__ void load_b_kn(uint32_t (&r)[4], uint32_t tile, int k
 }
 
 // ------------------------------------------------------------------ forward
+// dynamic shared memory: K[2], V[2] tiles of 64 x DH bf16
+template <int DH>
+constexpr int attn_fwd_smem_bytes() { return 4 * 64 * DH * 2; }
+
 template <int DH>
 __global__ void __launch_bounds__(128)
 attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* __restrict__ lse,
                     int S, int H, int causal, float scale) {
   constexpr int BQ = 64, BKV = 64, KS = DH / 16;
-  __shared__ __align__(128) uint8_t sQ[BQ * DH * 2];
-  __shared__ __align__(128) uint8_t sK[BKV * DH * 2];
-  __shared__ __align__(128) uint8_t sV[BKV * DH * 2];
+  constexpr int TB = BKV * DH * 2;                    // bytes of one K or V tile
+  extern __shared__ __align__(128) uint8_t smem_att[];   // K[2] | V[2]; Q is staged through V[1] first
+  uint8_t* sQ = smem_att + 3 * TB;
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * BQ;
   const int d = H * DH;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -84,14 +108,15 @@ attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* _
   const bf16* kb = qb + d;
   const bf16* vb = qb + 2 * d;
   const uint32_t tQ = (uint32_t)__cvta_generic_to_shared(sQ);
-  const uint32_t tK = (uint32_t)__cvta_generic_to_shared(sK);
-  const uint32_t tV = (uint32_t)__cvta_generic_to_shared(sV);
+  const uint32_t tKb = (uint32_t)__cvta_generic_to_shared(smem_att);
+  const uint32_t tVb = tKb + 2 * TB;
 
   stage_tile<BQ, DH>(sQ, qb, 3 * d, q0, S);
   __syncthreads();
   uint32_t qa[KS][4];
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) load_a<DH>(qa[ks], tQ, warp * 16, ks * 16, lane);
+  __syncthreads();                                      // Q fragments are in registers: V[1] may be overwritten
 
   float oacc[DH / 8][4];
 #pragma unroll
@@ -101,11 +126,21 @@ attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* _
   const int row_lo = q0 + warp * 16 + g;              // this thread's rows: row_lo, row_lo + 8
   const int k_end = causal ? min(S, q0 + BQ) : S;
 
-  for (int k0 = 0; k0 < k_end; k0 += BKV) {
+  stage_tile_async<BKV, DH>(tKb, kb, 3 * d, 0, S);
+  stage_tile_async<BKV, DH>(tVb, vb, 3 * d, 0, S);
+  cp_async_commit();
+  int buf = 0;
+  for (int k0 = 0; k0 < k_end; k0 += BKV, buf ^= 1) {
+    if (k0 + BKV < k_end) {                            // the next tile streams in behind this one
+      stage_tile_async<BKV, DH>(tKb + (buf ^ 1) * TB, kb, 3 * d, k0 + BKV, S);
+      stage_tile_async<BKV, DH>(tVb + (buf ^ 1) * TB, vb, 3 * d, k0 + BKV, S);
+      cp_async_commit();
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
     __syncthreads();
-    stage_tile<BKV, DH>(sK, kb, 3 * d, k0, S);
-    stage_tile<BKV, DH>(sV, vb, 3 * d, k0, S);
-    __syncthreads();
+    const uint32_t tK = tKb + buf * TB, tV = tVb + buf * TB;
     float sacc[BKV / 8][4];
 #pragma unroll
     for (int i = 0; i < BKV / 8; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
@@ -173,6 +208,7 @@ attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* _
         mma16816(oacc[2 * np + 1], pa, bfr[2], bfr[3]);
       }
     }
+    __syncthreads();                                   // this buffer is refilled two iterations from now
   }
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
@@ -221,9 +257,10 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
                        const bf16* __restrict__ dout, const float* __restrict__ dsum,
                        bf16* __restrict__ dqkv, int S, int H, int causal, float scale) {
   constexpr int BQ = 64, BKV = 32, KS = DH / 16;
+  constexpr int TB = BKV * DH * 2;
   __shared__ __align__(128) uint8_t sX[BQ * DH * 2];       // q tile, then do tile (fragments are kept in registers)
-  __shared__ __align__(128) uint8_t sK[BKV * DH * 2];
-  __shared__ __align__(128) uint8_t sV[BKV * DH * 2];
+  __shared__ __align__(128) uint8_t sK[2 * TB];            // double-buffered
+  __shared__ __align__(128) uint8_t sV[2 * TB];
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * BQ;
   const int d = H * DH;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -232,8 +269,13 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
   const bf16* vb = qb + 2 * d;
   const bf16* gb = dout + (int64_t)b * S * d + (int64_t)h * DH;
   const uint32_t tX = (uint32_t)__cvta_generic_to_shared(sX);
-  const uint32_t tK = (uint32_t)__cvta_generic_to_shared(sK);
-  const uint32_t tV = (uint32_t)__cvta_generic_to_shared(sV);
+  const uint32_t tKb = (uint32_t)__cvta_generic_to_shared(sK);
+  const uint32_t tVb = (uint32_t)__cvta_generic_to_shared(sV);
+
+  const int k_end = causal ? min(S, q0 + BQ) : S;
+  stage_tile_async<BKV, DH>(tKb, kb, 3 * d, 0, S);         // first K/V tile streams in behind the Q / dO staging
+  stage_tile_async<BKV, DH>(tVb, vb, 3 * d, 0, S);
+  cp_async_commit();
 
   uint32_t qa[KS][4], ga[KS][4];
   stage_tile<BQ, DH>(sX, qb, 3 * d, q0, S);
@@ -259,13 +301,19 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
 #pragma unroll
   for (int i = 0; i < DH / 8; ++i) { dq[i][0] = dq[i][1] = dq[i][2] = dq[i][3] = 0.f; }
   const float sl2 = scale * kLog2e;
-  const int k_end = causal ? min(S, q0 + BQ) : S;
 
-  for (int k0 = 0; k0 < k_end; k0 += BKV) {
+  int buf = 0;
+  for (int k0 = 0; k0 < k_end; k0 += BKV, buf ^= 1) {
+    if (k0 + BKV < k_end) {
+      stage_tile_async<BKV, DH>(tKb + (buf ^ 1) * TB, kb, 3 * d, k0 + BKV, S);
+      stage_tile_async<BKV, DH>(tVb + (buf ^ 1) * TB, vb, 3 * d, k0 + BKV, S);
+      cp_async_commit();
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
     __syncthreads();
-    stage_tile<BKV, DH>(sK, kb, 3 * d, k0, S);
-    stage_tile<BKV, DH>(sV, vb, 3 * d, k0, S);
-    __syncthreads();
+    const uint32_t tK = tKb + buf * TB, tV = tVb + buf * TB;
     float sacc[BKV / 8][4], pacc[BKV / 8][4];
 #pragma unroll
     for (int i = 0; i < BKV / 8; ++i) {
@@ -316,6 +364,7 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
         mma16816(dq[2 * np + 1], pa, bfr[2], bfr[3]);
       }
     }
+    __syncthreads();                                   // this buffer is refilled two iterations from now
   }
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
@@ -329,9 +378,9 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
 }
 
 // ------------------------------------------------------------------ backward: dk, dv (owner of key rows)
-// dynamic shared memory: K tile [64][DH], V tile [64][DH], Q tile [32][DH], dO tile [32][DH], L2[32], D[32]
+// dynamic shared memory: K tile [64][DH], V tile [64][DH], double-buffered Q and dO tiles [2][32][DH], L2[2][32], D[2][32]
 template <int DH>
-constexpr int attn_dkv_smem_bytes() { return (64 + 64 + 32 + 32) * DH * 2 + 2 * 32 * 4; }
+constexpr int attn_dkv_smem_bytes() { return (64 + 64 + 2 * 32 + 2 * 32) * DH * 2 + 4 * 32 * 4; }
 
 template <int DH>
 __global__ void __launch_bounds__(128)
@@ -342,10 +391,11 @@ attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ 
   extern __shared__ __align__(128) uint8_t smem_dkv[];
   uint8_t* sK = smem_dkv;
   uint8_t* sV = sK + BKV * DH * 2;
+  constexpr int TB = BQ * DH * 2;
   uint8_t* sQ = sV + BKV * DH * 2;
-  uint8_t* sG = sQ + BQ * DH * 2;
-  float* sL = reinterpret_cast<float*>(sG + BQ * DH * 2);
-  float* sD = sL + BQ;
+  uint8_t* sG = sQ + 2 * TB;
+  float* sLb = reinterpret_cast<float*>(sG + 2 * TB);
+  float* sDb = sLb + 2 * BQ;
   const int b = blockIdx.z, h = blockIdx.y, kr0 = blockIdx.x * BKV;
   const int d = H * DH;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -355,8 +405,8 @@ attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ 
   const bf16* gb = dout + (int64_t)b * S * d + (int64_t)h * DH;
   const uint32_t tK = (uint32_t)__cvta_generic_to_shared(sK);
   const uint32_t tV = (uint32_t)__cvta_generic_to_shared(sV);
-  const uint32_t tQ = (uint32_t)__cvta_generic_to_shared(sQ);
-  const uint32_t tG = (uint32_t)__cvta_generic_to_shared(sG);
+  const uint32_t tQb = (uint32_t)__cvta_generic_to_shared(sQ);
+  const uint32_t tGb = (uint32_t)__cvta_generic_to_shared(sG);
 
   stage_tile<BKV, DH>(sK, kb, 3 * d, kr0, S);
   stage_tile<BKV, DH>(sV, vb, 3 * d, kr0, S);
@@ -371,17 +421,31 @@ attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ 
   const int key_lo = kr0 + warp * 16 + g;             // this thread's key rows: key_lo, key_lo + 8
   const int q_begin = causal ? (kr0 / BQ) * BQ : 0;
 
-  for (int q0 = q_begin; q0 < S; q0 += BQ) {
-    __syncthreads();
-    stage_tile<BQ, DH>(sQ, qb, 3 * d, q0, S);
-    stage_tile<BQ, DH>(sG, gb, d, q0, S);
+  // per query tile: Q and dO rows through cp.async, LSE and dsum with plain loads, all double-buffered
+  auto prefetch = [&](int q0, int bf) {
+    stage_tile_async<BQ, DH>(tQb + bf * TB, qb, 3 * d, q0, S);
+    stage_tile_async<BQ, DH>(tGb + bf * TB, gb, d, q0, S);
+    cp_async_commit();
     if (threadIdx.x < BQ) {
       const int row = q0 + threadIdx.x;
       const bool ok = row < S;
-      sL[threadIdx.x] = ok ? lse[((int64_t)b * H + h) * S + row] * kLog2e : 0.f;
-      sD[threadIdx.x] = ok ? dsum[((int64_t)b * H + h) * S + row] : 0.f;
+      sLb[bf * BQ + threadIdx.x] = ok ? lse[((int64_t)b * H + h) * S + row] * kLog2e : 0.f;
+      sDb[bf * BQ + threadIdx.x] = ok ? dsum[((int64_t)b * H + h) * S + row] : 0.f;
+    }
+  };
+  if (q_begin < S) prefetch(q_begin, 0);
+  int buf = 0;
+  for (int q0 = q_begin; q0 < S; q0 += BQ, buf ^= 1) {
+    if (q0 + BQ < S) {
+      prefetch(q0 + BQ, buf ^ 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
     __syncthreads();
+    const uint32_t tQ = tQb + buf * TB, tG = tGb + buf * TB;
+    const float* sL = sLb + buf * BQ;
+    const float* sD = sDb + buf * BQ;
     // S^T = K Q^T and dP^T = V dO^T, 16 keys x 32 queries per warp
     float sacc[BQ / 8][4], pacc[BQ / 8][4];
 #pragma unroll
@@ -445,6 +509,7 @@ attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ 
         mma16816(dk[2 * np + 1], da, bfr[2], bfr[3]);
       }
     }
+    __syncthreads();                                   // this buffer is refilled two iterations from now
   }
 #pragma unroll
   for (int r = 0; r < 2; ++r) {

@@ -74,8 +74,14 @@ inline void attention_bwd_inst(cudaStream_t st, int B, int S, int H, int causal,
 inline bool attention_use_mma(int dtype, int dh) { return dtype == 1 && (dh == 64 || dh == 128); }
 template <int DH>
 inline void attention_mma_fwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, void* o, float* lse) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(attn_fwd_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_fwd_smem_bytes<DH>());
+    attr_set = true;
+  }
   dim3 grid((S + 63) / 64, H, B);
-  attn_fwd_mma_kernel<DH><<<grid, 128, 0, st>>>((const bf16*)qkv, (bf16*)o, lse, S, H, causal, 1.0f / sqrtf((float)DH));
+  attn_fwd_mma_kernel<DH><<<grid, 128, attn_fwd_smem_bytes<DH>(), st>>>((const bf16*)qkv, (bf16*)o, lse, S, H, causal,
+                                                                       1.0f / sqrtf((float)DH));
 }
 template <int DH>
 inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, const void* o,
