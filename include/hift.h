@@ -79,7 +79,10 @@ typedef struct {
  * is on the GPU). */
 typedef struct {
   int32_t kind;              /* 0 AdamW, 1 AdaGrad, 2 SGD with momentum, 3 plain SGD
-                                (no optimizer state: only the fp32 master, if any, is paged) */
+                                (no optimizer state: only the fp32 master, if any, is paged),
+                                4 Adafactor (factored second moment: rows + cols floats of state per
+                                matrix; `lr` caps the relative step, `eps` is its epsilon_1;
+                                epsilon_2 = 1e-3, clipping d = 1, decay exponent -0.8, no momentum) */
   int32_t sched;             /* 0 constant, 1 linear decay lr*(1 - cycle/total)    */
   int32_t total_cycles;      /* horizon of the linear schedule                     */
   int32_t offload_state;     /* 1: inactive groups' master+state in pinned host    */
@@ -152,6 +155,9 @@ hift_status hift_get_param(hift_ctx *ctx, int32_t tensor, float *dst_host, size_
 hift_status hift_get_model_param(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t n);
 /* Optimizer state `which` (0: first moment / accumulator / momentum, 1: second moment). */
 hift_status hift_get_state(hift_ctx *ctx, int32_t tensor, int32_t which, float *dst_host, size_t n);
+/* Adafactor only: which = 0 the row statistics R [rows] (for a vector, rows = 1: its second
+ * moment V [cols]), which = 1 the column statistics C [cols]. */
+hift_status hift_get_factored_state(hift_ctx *ctx, int32_t tensor, int32_t which, float *dst_host, size_t n);
 /* fp32 gradient of a tensor of the group trained by the LAST step. */
 hift_status hift_get_grad(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t n);
 /* Fill every parameter on the device: matrices N(0, std^2) from a counter-based
@@ -203,6 +209,15 @@ hift_status hift_opt_step(int32_t kind, size_t n, void *param_bf16_dev, float *m
                           double lr, double beta1, double beta2, double eps,
                           double weight_decay, double momentum, int64_t tau,
                           void *cuda_stream);
+
+/* Adafactor (one of the optimizers the paper profiles; its formulas are Shazeer & Stern 2018,
+ * Algorithms 4-5) on one caller-owned tensor [rows, cols] (rows = 1: a vector, unfactored).
+ * master/grad: fp32 [rows*cols]; state: fp32, R[rows] | C[cols] for a matrix, V[cols] for a
+ * vector; scratch: fp32, 2*rows + 64*cols + 8 floats; param_bf16 may be NULL.  tau >= 1 as in
+ * hift_opt_step.  Launches several small kernels on `cuda_stream`; does not synchronise. */
+hift_status hift_adafactor_step(int64_t rows, int64_t cols, void *param_bf16_dev, float *master_dev,
+                                const float *grad_dev, float *state_dev, float *scratch_dev,
+                                double lr, double eps1, double weight_decay, int64_t tau, void *cuda_stream);
 
 /* ---- single kernels on caller-owned device buffers (per-kernel parity) ----
  * These are the pieces of Algorithm 1's "ForwardPropagation"/"Backpropagation"

@@ -589,6 +589,26 @@ def sgd_update(theta, g, lr):
     return theta - lr * g
 
 
+def adafactor_update(theta, g, s0, s1, lr, eps1, wd, tau, eps2=1e-3, d=1.0, decay=-0.8):
+    """Adafactor (Shazeer & Stern 2018, Algorithms 4-5) with relative step size, parameter
+    scaling, update clipping and no momentum.  Matrices keep row statistics s0 = R [n] and column
+    statistics s1 = C [m]; vectors keep the unfactored second moment in s0.  Returns theta, s0, s1."""
+    w = float(tau) ** decay                                   # 1 - beta2_t
+    rho = min(lr, 1.0 / math.sqrt(tau))
+    alpha = max(eps2, math.sqrt(float((theta * theta).mean()))) * rho
+    theta = theta * (1.0 - lr * wd)
+    if g.ndim > 1:
+        s0 = s0 + w * ((g * g).mean(axis=-1) - s0)
+        s1 = s1 + w * ((g * g).mean(axis=-2) - s1)
+        vhat = np.outer(s0, s1) / max(float(s0.mean()), eps1)
+    else:
+        s0 = s0 + w * (g * g - s0)
+        vhat = s0
+    u = g / np.sqrt(np.maximum(vhat, eps1 * eps1))
+    u = u / max(1.0, math.sqrt(float((u * u).mean())) / d)
+    return theta - alpha * u, s0, s1
+
+
 # --------------------------------------------------------------------------
 # The training step (Algorithm 1)
 # --------------------------------------------------------------------------
@@ -645,8 +665,15 @@ class HiFTOracle:
             elif o.kind == 2:
                 self.master[name], self.s0[name] = sgdm_update(
                     self.master[name], gr, self.s0[name], lr, o.momentum)
-            else:
+            elif o.kind == 3:
                 self.master[name] = sgd_update(self.master[name], gr, lr)
+            else:
+                if self.tau[g] == 1:                          # factored state has its own shapes
+                    m = self.master[name]
+                    self.s0[name] = np.zeros(m.shape[0]) if m.ndim > 1 else np.zeros_like(m)
+                    self.s1[name] = np.zeros(m.shape[1]) if m.ndim > 1 else np.zeros(0)
+                self.master[name], self.s0[name], self.s1[name] = adafactor_update(
+                    self.master[name], gr, self.s0[name], self.s1[name], lr, o.eps, o.weight_decay, self.tau[g])
         self.last_grads = grads
         self.t += 1
         return loss

@@ -81,6 +81,8 @@ def _prototypes():
         "hift_get_model_param": (C.c_int, [vp, i32, vp, sz]),
         "hift_get_grad": (C.c_int, [vp, i32, vp, sz]),
         "hift_get_state": (C.c_int, [vp, i32, i32, vp, sz]),
+        "hift_get_factored_state": (C.c_int, [vp, i32, i32, vp, sz]),
+        "hift_adafactor_step": (C.c_int, [i64, i64, vp, vp, vp, vp, vp, f64, f64, f64, i64, vp]),
         "hift_init_synthetic": (C.c_int, [vp, C.c_uint64, f64]),
         "hift_profile_enable": (C.c_int, [vp, i32]),
         "hift_profile": (C.c_int, [vp, i32, C.POINTER(i64), C.POINTER(f64), C.POINTER(f64)]),
@@ -274,6 +276,14 @@ class HiFT:
     def get_state(self, name: str, which: int) -> np.ndarray:
         return self._get(lib().hift_get_state, "hift_get_state", name, which)
 
+    def get_factored_state(self, name: str, which: int) -> np.ndarray:
+        _, _, r, c = self._info[self._names[name]]
+        n = c if (r == 1 or which == 1) else r
+        out = np.empty(n, dtype=np.float32)
+        _check(lib().hift_get_factored_state(self._h, self._names[name], which, out.ctypes.data, n),
+               "hift_get_factored_state")
+        return out
+
     def init_synthetic(self, seed: int, std: float = 0.02):
         _check(lib().hift_init_synthetic(self._h, seed, std), "hift_init_synthetic")
 
@@ -313,6 +323,12 @@ def opt_step(kind, n, param_bf16, master, grad, s0, s1, lr, beta1=0.9, beta2=0.9
              weight_decay=0.0, momentum=0.9, tau=1, stream=None):
     _check(lib().hift_opt_step(kind, n, _ptr(param_bf16), _ptr(master), _ptr(grad), _ptr(s0), _ptr(s1),
                                lr, beta1, beta2, eps, weight_decay, momentum, tau, _st(stream)), "hift_opt_step")
+
+
+def adafactor_step(rows, cols, param_bf16, master, grad, state, scratch, lr, eps1=1e-30, weight_decay=0.0, tau=1,
+                   stream=None):
+    _check(lib().hift_adafactor_step(rows, cols, _ptr(param_bf16), _ptr(master), _ptr(grad), _ptr(state),
+                                     _ptr(scratch), lr, eps1, weight_decay, tau, _st(stream)), "hift_adafactor_step")
 
 
 def tc_error_flag(set_value: int = -1) -> int:

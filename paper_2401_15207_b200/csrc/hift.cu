@@ -16,6 +16,7 @@
 #include <vector>
 
 #include "gemm_tc.h"
+#include "kernels_adafactor.cuh"
 #include "launchers.cuh"
 
 using namespace hift;
@@ -38,13 +39,16 @@ struct TensorRec {
   int64_t rows, cols;
   size_t numel, off;
   int init_kind;   // 0 normal, 1 ones, 2 zeros
+  size_t af_off;   // Adafactor: offset of this tensor's factored state inside its group's compact state
 };
 struct GroupRec {
   int unit_lo, unit_hi;
   size_t off, numel;      // span in the flat parameter buffer (padded)
   int64_t tau;            // updates so far
-  char* blob;             // pinned host: [master][s0][s1]
+  char* blob;             // pinned host: [master][state]
   size_t blob_bytes;
+  size_t state_floats;    // floats of optimizer state (n_state * numel, or the compact Adafactor state)
+  size_t af_base;         // Adafactor, state resident: offset of the group's compact state in af_all
 };
 struct BlockIdx {          // tensor indices of one block, -1 if absent
   int n1_g, n1_b, w_qkv, b_qkv, w_o, b_o, n2_g, n2_b, w_fc1, b_fc1, w_fc2, b_fc2;
@@ -82,6 +86,9 @@ struct hift_ctx {
   char* params = nullptr;           // [total] of element type
   float* master_all = nullptr;      // non-offload mixed mode
   float* s0_all = nullptr; float* s1_all = nullptr;
+  float* af_all = nullptr;          // Adafactor, state resident: compact state of every group
+  float* af_scratch = nullptr;      // Adafactor work space, sized for the largest tensor
+  bool af = false;
   char* slot[2] = {nullptr, nullptr};   // offload staging: [master][s0][s1] per slot
   int n_slots = 1;
   float* grad = nullptr;            // [max_group]
@@ -640,6 +647,24 @@ void enqueue_update(hift_ctx* c) {
   const double lr = c->cur_lr;
   // ---------------- group-local optimizer (Algorithm 1: P now points at theta_s only)
   gr.tau += 1;
+  if (c->af) {
+    // Adafactor works tensor by tensor (its statistics are per row and column of each matrix)
+    float* base = c->offload ? (float*)c->slot[sl] : nullptr;
+    if (c->offload) c->note(cudaStreamWaitEvent(c->st, c->ev_h2d[sl], 0));
+    for (int u = gr.unit_lo; u <= gr.unit_hi; ++u)
+      for (int ti : c->unit_tens[u]) {
+        const TensorRec& r = c->tens[ti];
+        float* mst_t;
+        if (!c->mixed) mst_t = (float*)c->params + r.off;
+        else mst_t = c->offload ? base + (r.off - gr.off) : c->master_all + r.off;
+        float* st_t = c->offload ? base + (c->mixed ? gr.numel : 0) + r.af_off : c->af_all + gr.af_base + r.af_off;
+        c->pre(HIFT_K_OPT, (double)r.numel * (20.0 + (c->mixed ? 2.0 : 0.0)));
+        const int nk = launch_adafactor_tensor(c->st, r.rows, r.cols, c->mixed ? c->P(ti) : nullptr, mst_t, c->G(ti), st_t,
+                                               c->af_scratch, lr, c->oc.eps, c->oc.weight_decay, gr.tau);
+        c->post();
+        c->step_launches += nk - 1;
+      }
+  } else {
   float *mst, *s0, *s1;
   void* pbf = nullptr;
   if (c->offload) {
@@ -659,6 +684,7 @@ void enqueue_update(hift_ctx* c) {
                                          c->oc.weight_decay, c->oc.momentum, gr.tau);
   const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
   LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs));
+  }
 
   // ---------------- state back to the host (step k)
   if (c->offload) {
@@ -788,7 +814,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // the embedding-gradient kernel keeps one occurrence list of <= batch*seq ints in shared memory
   if ((int64_t)m->batch * m->seq > 8192) return HIFT_ERR_CFG;
   if (gc->layers_per_group < 1 || gc->order < 0 || gc->order > 2) return HIFT_ERR_CFG;
-  if (oc->kind < 0 || oc->kind > 3 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
+  if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
   if (oc->sched == 1 && oc->total_cycles < 1) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
@@ -800,14 +826,32 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   c->L = m->n_blocks; c->d = m->d_model; c->f = m->d_ffn; c->fa = m->arch == 2 ? 2 * m->d_ffn : m->d_ffn;
   c->H = m->n_heads; c->dh = m->d_model / m->n_heads; c->B = m->batch; c->S = m->seq; c->T = m->batch * m->seq;
   c->V = m->vocab; c->Vp = (int)align_up(m->vocab, 128);
-  c->n_state = oc->kind == 0 ? 2 : (oc->kind == 3 ? 0 : 1);
+  c->af = oc->kind == 4;
+  c->n_state = oc->kind == 0 ? 2 : (oc->kind >= 3 ? 0 : 1);
   // plain SGD on fp32 parameters has nothing to page (the paper's "no state, zero traffic" case)
-  c->offload = oc->offload_state != 0 && ((m->dtype == 1 ? 1 : 0) + c->n_state) > 0;
+  c->offload = oc->offload_state != 0 && ((m->dtype == 1 ? 1 : 0) + c->n_state + (c->af ? 1 : 0)) > 0;
   c->n_slots = (c->offload && oc->prefetch_groups) ? 2 : 1;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_work, 0, sizeof(c->prof_work));
   build_layout(c);
+  {
+    size_t base = 0;
+    for (auto& g : c->groups) {
+      g.state_floats = (size_t)c->n_state * g.numel;
+      if (c->af) {
+        size_t o = 0;
+        for (int u = g.unit_lo; u <= g.unit_hi; ++u)
+          for (int ti : c->unit_tens[u]) {
+            c->tens[ti].af_off = o;
+            o = align_up(o + af_state_floats(c->tens[ti].rows, c->tens[ti].cols), 4);
+          }
+        g.state_floats = o;
+        g.af_base = base;
+        base += o;
+      }
+    }
+  }
 
   hift_status rc = HIFT_OK;
   auto fail = [&](hift_status s) { hift_destroy(c); return s; };
@@ -827,17 +871,19 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (cudaStreamCreateWithFlags(&c->st_d2h, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
   // ---- parameters, gradients, optimizer state
-  const size_t planes = (size_t)(c->mixed ? 1 : 0) + c->n_state;
+  auto blob_floats = [&](const GroupRec& g) { return (c->mixed ? g.numel : 0) + g.state_floats; };
+  size_t slot_floats = 0, af_total = 0;
+  for (auto& g : c->groups) { slot_floats = std::max(slot_floats, blob_floats(g)); af_total += c->af ? g.state_floats : 0; }
   if ((rc = dev_alloc(c, (void**)&c->params, c->total * c->es)) != HIFT_OK) return fail(rc);
   cudaMemsetAsync(c->params, 0, c->total * c->es, c->st);
   if ((rc = dev_alloc(c, (void**)&c->grad, c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
   if (c->offload) {
     for (int s = 0; s < c->n_slots; ++s) {
-      if ((rc = dev_alloc(c, (void**)&c->slot[s], planes * c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
-      cudaMemsetAsync(c->slot[s], 0, planes * c->max_group * sizeof(float), c->st);
+      if ((rc = dev_alloc(c, (void**)&c->slot[s], slot_floats * sizeof(float))) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->slot[s], 0, slot_floats * sizeof(float), c->st);
     }
     for (auto& g : c->groups) {
-      g.blob_bytes = planes * g.numel * sizeof(float);
+      g.blob_bytes = blob_floats(g) * sizeof(float);
       if (cudaHostAlloc((void**)&g.blob, g.blob_bytes, cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         g.blob = nullptr;
@@ -859,6 +905,15 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
       if ((rc = dev_alloc(c, (void**)&c->s1_all, c->total * sizeof(float))) != HIFT_OK) return fail(rc);
       cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
     }
+    if (c->af) {
+      if ((rc = dev_alloc(c, (void**)&c->af_all, af_total * sizeof(float))) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->af_all, 0, af_total * sizeof(float), c->st);
+    }
+  }
+  if (c->af) {
+    size_t mx = 0;
+    for (auto& r : c->tens) mx = std::max(mx, af_scratch_floats(r.rows, r.cols));
+    if ((rc = dev_alloc(c, (void**)&c->af_scratch, mx * sizeof(float))) != HIFT_OK) return fail(rc);
   }
   if (cudaHostAlloc((void**)&c->scal_host, 4 * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
   if (cudaHostGetDevicePointer((void**)&c->scal_host_dev, c->scal_host, 0) != cudaSuccess) return fail(HIFT_ERR_CUDA);
@@ -1046,6 +1101,23 @@ hift_status hift_get_state(hift_ctx* c, int32_t ti, int32_t which, float* dst, s
   else if (cudaMemcpy(dst, sp, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
   return HIFT_OK;
 }
+hift_status hift_get_factored_state(hift_ctx* c, int32_t ti, int32_t which, float* dst, size_t n) {
+  if (!c || !c->af || ti < 0 || ti >= (int)c->tens.size() || !dst || which < 0 || which > 1) return HIFT_ERR_CFG;
+  const TensorRec& r = c->tens[ti];
+  const bool vec = r.rows == 1;
+  if (vec && which == 1) return HIFT_ERR_CFG;
+  const size_t want = vec ? (size_t)r.cols : (which == 0 ? (size_t)r.rows : (size_t)r.cols);
+  if (n != want) return HIFT_ERR_CFG;
+  sync_all(c);
+  const GroupRec& gr = c->groups[group_of_unit(c, r.unit)];
+  const size_t o = r.af_off + ((!vec && which == 1) ? (size_t)r.rows : 0);
+  if (c->offload) {
+    memcpy(dst, (float*)gr.blob + (c->mixed ? gr.numel : 0) + o, n * sizeof(float));
+    return HIFT_OK;
+  }
+  return cudaMemcpy(dst, c->af_all + gr.af_base + o, n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+
 hift_status hift_get_grad(hift_ctx* c, int32_t ti, float* dst, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   if (c->last_group < 0 || group_of_unit(c, c->tens[ti].unit) != c->last_group) return HIFT_ERR_CFG;
@@ -1055,10 +1127,9 @@ hift_status hift_get_grad(hift_ctx* c, int32_t ti, float* dst, size_t n) {
 
 hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
   sync_all(c);
-  const size_t planes = (size_t)(c->mixed ? 1 : 0) + c->n_state;
   for (size_t g = 0; g < c->groups.size(); ++g) {
     GroupRec& gr = c->groups[g];
-    if (c->offload) cudaMemsetAsync(c->slot[0], 0, planes * gr.numel * sizeof(float), c->st);
+    if (c->offload) cudaMemsetAsync(c->slot[0], 0, gr.blob_bytes, c->st);
     for (int u = gr.unit_lo; u <= gr.unit_hi; ++u) {
       for (int ti : c->unit_tens[u]) {
         const TensorRec& r = c->tens[ti];
@@ -1078,6 +1149,11 @@ hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
   if (!c->offload) {
     if (c->s0_all) cudaMemsetAsync(c->s0_all, 0, c->total * sizeof(float), c->st);
     if (c->s1_all) cudaMemsetAsync(c->s1_all, 0, c->total * sizeof(float), c->st);
+    if (c->af_all) {
+      size_t tot = 0;
+      for (auto& g : c->groups) tot += g.state_floats;
+      cudaMemsetAsync(c->af_all, 0, tot * sizeof(float), c->st);
+    }
   }
   return cudaStreamSynchronize(c->st) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
@@ -1133,6 +1209,14 @@ hift_status hift_opt_step(int32_t kind, size_t n, void* param_bf16, float* maste
   if (al & 15) return HIFT_ERR_CFG;
   const OptScalars h = make_opt_scalars(kind, lr, b1, b2, eps, wd, mu, tau);
   launch_fused_opt((cudaStream_t)stream, kind, n, param_bf16, master, grad, s0, s1, h);
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+
+hift_status hift_adafactor_step(int64_t rows, int64_t cols, void* param_bf16, float* master, const float* grad,
+                                float* state, float* scratch, double lr, double eps1, double wd, int64_t tau,
+                                void* stream) {
+  if (rows < 1 || cols < 1 || !master || !grad || !state || !scratch || tau < 1) return HIFT_ERR_CFG;
+  launch_adafactor_tensor((cudaStream_t)stream, rows, cols, param_bf16, master, grad, state, scratch, lr, eps1, wd, tau);
   return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 

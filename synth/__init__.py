@@ -29,7 +29,7 @@ ARCH_LLAMA = 2          # RMSNorm, RoPE, SwiGLU, no biases
 DTYPE_FP32 = 0          # fp32 parameters and activations
 DTYPE_BF16 = 1          # bf16 parameters/activations with fp32 master weights
 
-OPT_ADAMW, OPT_ADAGRAD, OPT_SGDM, OPT_SGD = 0, 1, 2, 3
+OPT_ADAMW, OPT_ADAGRAD, OPT_SGDM, OPT_SGD, OPT_ADAFACTOR = 0, 1, 2, 3, 4
 ORDER_BOTTOM2UP, ORDER_TOP2DOWN, ORDER_RANDOM = 0, 1, 2
 SCHED_CONST, SCHED_LINEAR = 0, 1
 

@@ -74,7 +74,11 @@ def lockstep(cfg, gcfg, ocfg, steps, dist, tol_loss, tol_grad, seed=1, data_seed
                         assert np.linalg.norm(err) <= check_update * np.linalg.norm(upd) + ulp + 1e-12, (t, n)
                     if resync:
                         orc.master[n] = after.astype(np.float64).reshape(orc.master[n].shape)
-                        if ocfg.kind != 3:
+                        if ocfg.kind == 4:
+                            orc.s0[n] = h.get_factored_state(n, 0).astype(np.float64)
+                            if orc.master[n].ndim > 1:
+                                orc.s1[n] = h.get_factored_state(n, 1).astype(np.float64)
+                        elif ocfg.kind != 3:
                             orc.s0[n] = h.get_state(n, 0).astype(np.float64).reshape(orc.master[n].shape)
                         if ocfg.kind == 0:
                             orc.s1[n] = h.get_state(n, 1).astype(np.float64).reshape(orc.master[n].shape)

@@ -71,6 +71,36 @@ def test_plain_sgd_kernel_needs_no_state():
     assert np.array_equal(tp.float().cpu().numpy(), O.bf16_round(tm.cpu().numpy()))
 
 
+@pytest.mark.parametrize("rows,cols", [(1, 777), (5, 8), (300, 1280), (2050, 96)])
+def test_adafactor_tensor_update_matches_oracle(rows, cols):
+    import torch
+    from paper_2401_15207_b200 import adafactor_step
+    rng = np.random.default_rng(rows * 3 + cols)
+    shape = (cols,) if rows == 1 else (rows, cols)
+    theta = (rng.standard_normal(shape) * 0.02).astype(np.float32)
+    n_state = cols if rows == 1 else rows + cols
+    tm = _t(theta.reshape(-1))
+    ts = torch.zeros(n_state, device="cuda")
+    tp = torch.zeros(rows * cols, dtype=torch.bfloat16, device="cuda")
+    scratch = torch.empty(2 * rows + 64 * cols + 8, device="cuda")
+    th64 = theta.astype(np.float64)
+    s0 = np.zeros(shape[0]) if rows > 1 else np.zeros(shape)
+    s1 = np.zeros(cols) if rows > 1 else np.zeros(0)
+    for tau in (1, 2, 3):
+        g = (rng.standard_normal(shape) * 1e-3).astype(np.float32)
+        adafactor_step(rows, cols, tp, tm, _t(g.reshape(-1)), ts, scratch, lr=1e-2, eps1=1e-30, weight_decay=0.01, tau=tau)
+        th64, s0, s1 = O.adafactor_update(th64, g.astype(np.float64), s0, s1, 1e-2, 1e-30, 0.01, tau)
+    torch.cuda.synchronize()
+    gm = tm.cpu().numpy().reshape(shape)
+    assert rel_l2(gm, th64) <= 1e-6
+    st = ts.cpu().numpy()
+    if rows > 1:
+        assert rel_l2(st[:rows], s0) <= 2e-6 and rel_l2(st[rows:], s1) <= 2e-6
+    else:
+        assert rel_l2(st, s0) <= 2e-6
+    assert np.array_equal(tp.float().cpu().numpy().reshape(shape), O.bf16_round(gm))
+
+
 def test_fused_optimizer_fp32_params_and_argument_checks():
     import torch
     from paper_2401_15207_b200 import opt_step, HiftError

@@ -85,6 +85,23 @@ def test_plain_sgd_pages_only_the_master(dtype):
     h.close()
 
 
+@pytest.mark.parametrize("arch,dtype,offload", [(0, synth.DTYPE_FP32, 1), (2, synth.DTYPE_BF16, 1), (1, synth.DTYPE_BF16, 0)])
+def test_adafactor_state_is_rows_plus_cols(arch, dtype, offload):
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(arch, dtype, tie_head=1 if arch == 0 else 0)
+    oc = synth.OptCfg(kind=synth.OPT_ADAFACTOR, lr=1e-2, eps=1e-30, weight_decay=0.01, offload_state=offload,
+                      prefetch_groups=1)
+    tol = (FP32_LOSS, FP32_GRAD) if dtype == synth.DTYPE_FP32 else (BF16_LOSS, BF16_GRAD)
+    lockstep(cfg, synth.GroupCfg(1), oc, 8, "zipf", tol[0], tol[1], resync=True,
+             check_update=2e-3 if dtype == synth.DTYPE_FP32 else None)
+    if offload and dtype == synth.DTYPE_FP32:
+        h = HiFT(cfg, synth.GroupCfg(1), oc)
+        # the whole optimizer state of the model: sum over tensors of rows + cols (vectors: their length)
+        want = sum((s[0] + s[1]) if len(s) == 2 else s[0] for u in synth.unit_tensors(cfg) for _, s, _ in u)
+        assert 4 * want <= h.pinned_host_bytes() <= 4 * want + 16 * 64
+        h.close()
+
+
 def test_free_running_trajectories_stay_close():
     """No resynchronisation: the two trajectories only share the initial weights."""
     cfg = mini(0, synth.DTYPE_BF16, tie_head=1)

@@ -50,6 +50,34 @@ def test_plain_sgd_closed_form_and_torch():
     assert np.allclose(O.sgd_update(th, g, 0.1), p.detach().numpy(), rtol=1e-15)
 
 
+def test_adafactor_first_step_by_hand_and_against_torch():
+    # 2 x 2 by hand at tau = 1: w = 1, so R, C are the row / column means of g^2
+    th = np.array([[1.0, -2.0], [0.5, 4.0]])
+    g = np.array([[0.1, -0.2], [0.3, 0.4]])
+    R, Cc = (g * g).mean(1), (g * g).mean(0)
+    V = np.outer(R, Cc) / R.mean()
+    U = g / np.sqrt(V)
+    U = U / max(1.0, math.sqrt((U * U).mean()))
+    alpha = max(1e-3, math.sqrt((th * th).mean())) * min(1e-2, 1.0)
+    got, s0, s1 = O.adafactor_update(th, g, np.zeros(2), np.zeros(2), 1e-2, 1e-30, 0.0, 1)
+    assert np.allclose(got, th - alpha * U, rtol=1e-14) and np.allclose(s0, R) and np.allclose(s1, Cc)
+    # several steps, a matrix and a vector, weight decay on, against the library routine
+    rng = np.random.default_rng(8)
+    for shape in ((7, 5), (11,)):
+        p0 = rng.standard_normal(shape)
+        grads = [rng.standard_normal(shape) * 1e-2 for _ in range(6)]
+        p = torch.nn.Parameter(torch.tensor(p0))
+        opt = torch.optim.Adafactor([p], lr=3e-3, eps=(1e-30, 1e-3), weight_decay=0.05, foreach=False)
+        th = p0.copy()
+        s0 = np.zeros(shape[0]) if len(shape) > 1 else np.zeros(shape)
+        s1 = np.zeros(shape[1]) if len(shape) > 1 else np.zeros(0)
+        for i, gr in enumerate(grads):
+            p.grad = torch.tensor(gr)
+            opt.step()
+            th, s0, s1 = O.adafactor_update(th, gr, s0, s1, 3e-3, 1e-30, 0.05, i + 1)
+            assert np.allclose(th, p.detach().numpy(), rtol=1e-11, atol=1e-14), (shape, i)
+
+
 def test_optimizers_against_torch_optim_fp64():
     rng = np.random.default_rng(4)
     n, steps = 257, 5
