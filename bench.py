@@ -302,6 +302,20 @@ def run_ours(args, cfg, gcfg, ocfg):
                                 "tflops": v["work"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0}
                             for c, v in g.items()}}
         kernel_share = {c: round(v["ms"], 3) for c, v in prof.items()}
+        # every kernel class against its own roofline (event-bracketed: the brackets add a few
+        # microseconds per launch, which shows on the short bandwidth-bound kernels)
+        per_kernel = {}
+        for cname, v in prof.items():
+            if v["launches"] == 0 or v["ms"] <= 0:
+                continue
+            tensor = cname.startswith("gemm") or cname.startswith("attn")
+            ach = v["work"] / (v["ms"] * 1e-3) / (1e12 if tensor else 1e9)
+            pk = (peaks["bf16_tflops_sustained"] if cfg.dtype == 1 else None) if tensor else peaks["hbm_gbs"]
+            per_kernel[cname] = {"launches": v["launches"], "ms": round(v["ms"], 3),
+                                 "avg_us": round(1e3 * v["ms"] / v["launches"], 2),
+                                 "achieved": round(ach, 1), "unit": "TFLOP/s" if tensor else "GB/s",
+                                 "bound": "tensor" if tensor else "hbm",
+                                 "frac": round(ach / pk, 3) if pk else None}
         opt = prof["optimizer"]
         opt_gbs = opt["work"] / (opt["ms"] * 1e-3) / 1e9 if opt["ms"] > 0 else 0.0
         cpu = None
@@ -330,6 +344,7 @@ def run_ours(args, cfg, gcfg, ocfg):
             "roofline": roof,
             "optimizer_gbs": opt_gbs, "optimizer_frac_of_hbm": opt_gbs / peaks["hbm_gbs"],
             "kernel_ms": kernel_share,
+            "kernels": per_kernel,
             "clocks": clocks,
             "full_param_reference": full_ref,
             "cpu_baseline": cpu,

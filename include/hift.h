@@ -164,6 +164,14 @@ hift_status hift_get_grad(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t
  * hash of (seed, element index), gains 1, biases 0; optimizer state zero. */
 hift_status hift_init_synthetic(hift_ctx *ctx, uint64_t seed, double std);
 
+/* Checkpoint: the whole training state is the fp32 master (or fp32 parameters), the optimizer
+ * state and update count of every group (which Algorithm 1 keeps on the host between a group's
+ * turns anyway), and the step counter t; the group order follows from the configuration.
+ * hift_load needs a context created with the same configuration (HIFT_ERR_CFG otherwise) and
+ * rebuilds the bf16 model copy.  A missing / short / foreign file gives HIFT_ERR_INPUT. */
+hift_status hift_save(hift_ctx *ctx, const char *path);
+hift_status hift_load(hift_ctx *ctx, const char *path);
+
 /* ---- instrumentation ------------------------------------------------------ */
 /* Kernel classes for hift_profile(). */
 enum { HIFT_K_GEMM_FWD = 0, HIFT_K_GEMM_DX = 1, HIFT_K_GEMM_DW = 2, HIFT_K_ATTN_FWD = 3,

@@ -84,6 +84,8 @@ def _prototypes():
         "hift_get_factored_state": (C.c_int, [vp, i32, i32, vp, sz]),
         "hift_adafactor_step": (C.c_int, [i64, i64, vp, vp, vp, vp, vp, f64, f64, f64, i64, vp]),
         "hift_init_synthetic": (C.c_int, [vp, C.c_uint64, f64]),
+        "hift_save": (C.c_int, [vp, C.c_char_p]),
+        "hift_load": (C.c_int, [vp, C.c_char_p]),
         "hift_profile_enable": (C.c_int, [vp, i32]),
         "hift_profile": (C.c_int, [vp, i32, C.POINTER(i64), C.POINTER(f64), C.POINTER(f64)]),
         "hift_last_step_launches": (i64, [vp]),
@@ -286,6 +288,12 @@ class HiFT:
 
     def init_synthetic(self, seed: int, std: float = 0.02):
         _check(lib().hift_init_synthetic(self._h, seed, std), "hift_init_synthetic")
+
+    def save(self, path: str):
+        _check(lib().hift_save(self._h, path.encode()), "hift_save")
+
+    def load(self, path: str):
+        _check(lib().hift_load(self._h, path.encode()), "hift_load")
 
     # -- instrumentation
     def profile_enable(self, on: bool):

@@ -1158,6 +1158,107 @@ hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
   return cudaStreamSynchronize(c->st) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------- checkpoint
+namespace {
+struct CkptHeader {
+  char magic[8];            // "HIFTCKPT"
+  uint32_t version;
+  uint32_t kind, dtype, n_groups;
+  uint64_t total, t;
+};
+// device or pinned location of the group's fp32 master (or fp32 parameters) and of its state
+void group_locations(hift_ctx* c, GroupRec& gr, float** master, bool* master_host, float** state, bool* state_host) {
+  *master_host = false; *state_host = false;
+  if (!c->mixed) *master = (float*)c->params + gr.off;
+  else if (c->offload) { *master = (float*)gr.blob; *master_host = true; }
+  else *master = c->master_all + gr.off;
+  if (c->offload) { *state = (float*)gr.blob + (c->mixed ? gr.numel : 0); *state_host = true; }
+  else if (c->af) *state = c->af_all + gr.af_base;
+  else *state = nullptr;      // two separate planes, handled by the caller
+}
+}  // namespace
+
+hift_status hift_save(hift_ctx* c, const char* path) {
+  if (!c || !path || c->pending_update) return HIFT_ERR_CFG;
+  sync_all(c);
+  FILE* f = fopen(path, "wb");
+  if (!f) return HIFT_ERR_INPUT;
+  CkptHeader h;
+  memset(&h, 0, sizeof(h));
+  memcpy(h.magic, "HIFTCKPT", 8);
+  h.version = 1; h.kind = (uint32_t)c->oc.kind; h.dtype = (uint32_t)c->m.dtype; h.n_groups = (uint32_t)c->groups.size();
+  h.total = c->total; h.t = (uint64_t)c->t;
+  bool ok = fwrite(&h, sizeof(h), 1, f) == 1;
+  std::vector<float> tmp;
+  for (auto& gr : c->groups) {
+    if (!ok) break;
+    ok = fwrite(&gr.tau, sizeof(gr.tau), 1, f) == 1;
+    float *mp, *sp; bool mh, sh;
+    group_locations(c, gr, &mp, &mh, &sp, &sh);
+    auto put = [&](const float* p, bool host, size_t n) {
+      if (!ok || n == 0) return;
+      if (host) { ok = fwrite(p, sizeof(float), n, f) == n; return; }
+      tmp.resize(n);
+      ok = cudaMemcpy(tmp.data(), p, n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess &&
+           fwrite(tmp.data(), sizeof(float), n, f) == n;
+    };
+    put(mp, mh, gr.numel);
+    if (sp) put(sp, sh, gr.state_floats);
+    else {
+      if (c->s0_all) put(c->s0_all + gr.off, false, gr.numel);
+      if (c->s1_all) put(c->s1_all + gr.off, false, gr.numel);
+    }
+  }
+  ok = (fclose(f) == 0) && ok;
+  return ok ? HIFT_OK : HIFT_ERR_INPUT;
+}
+
+hift_status hift_load(hift_ctx* c, const char* path) {
+  if (!c || !path || c->pending_update) return HIFT_ERR_CFG;
+  sync_all(c);
+  FILE* f = fopen(path, "rb");
+  if (!f) return HIFT_ERR_INPUT;
+  CkptHeader h;
+  bool ok = fread(&h, sizeof(h), 1, f) == 1 && memcmp(h.magic, "HIFTCKPT", 8) == 0 && h.version == 1;
+  if (ok && (h.kind != (uint32_t)c->oc.kind || h.dtype != (uint32_t)c->m.dtype || h.n_groups != c->groups.size() ||
+             h.total != c->total)) { fclose(f); return HIFT_ERR_CFG; }
+  std::vector<float> tmp;
+  for (auto& gr : c->groups) {
+    if (!ok) break;
+    ok = fread(&gr.tau, sizeof(gr.tau), 1, f) == 1;
+    float *mp, *sp; bool mh, sh;
+    group_locations(c, gr, &mp, &mh, &sp, &sh);
+    auto get = [&](float* p, bool host, size_t n) {
+      if (!ok || n == 0) return;
+      if (host) { ok = fread(p, sizeof(float), n, f) == n; return; }
+      tmp.resize(n);
+      ok = fread(tmp.data(), sizeof(float), n, f) == n &&
+           cudaMemcpy(p, tmp.data(), n * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess;
+    };
+    get(mp, mh, gr.numel);
+    if (sp) get(sp, sh, gr.state_floats);
+    else {
+      if (c->s0_all) get(c->s0_all + gr.off, false, gr.numel);
+      if (c->s1_all) get(c->s1_all + gr.off, false, gr.numel);
+    }
+    if (ok && c->mixed) {
+      // rebuild the bf16 model copy of this group from its master values
+      const float* src = mp;
+      if (mh) {
+        ok = cudaMemcpyAsync(c->grad, mp, gr.numel * sizeof(float), cudaMemcpyHostToDevice, c->st) == cudaSuccess;
+        src = c->grad;
+      }
+      cast_from_f32_kernel<bf16><<<grid_for(gr.numel, 256), 256, 0, c->st>>>(src, (bf16*)(c->params + gr.off * c->es), gr.numel);
+      ok = ok && cudaStreamSynchronize(c->st) == cudaSuccess;
+    }
+  }
+  fclose(f);
+  if (!ok) return HIFT_ERR_INPUT;
+  c->t = (int64_t)h.t;
+  c->d2h_pending[0] = c->d2h_pending[1] = false;
+  return HIFT_OK;
+}
+
 hift_status hift_profile_enable(hift_ctx* c, int32_t on) {
   sync_all(c);
   c->prof_on = on != 0;

@@ -193,3 +193,36 @@ def test_timeout_flag_path_reports_and_recovers():
     assert h2.step(tt, ll) == good[0]
     h2.close()
     h.close()
+
+
+@pytest.mark.parametrize("kind,offload,dtype", [(0, 1, synth.DTYPE_BF16), (0, 0, synth.DTYPE_BF16),
+                                                (4, 1, synth.DTYPE_BF16), (2, 1, synth.DTYPE_FP32)])
+def test_checkpoint_resume_is_bitwise(kind, offload, dtype, tmp_path):
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError
+    cfg = mini(2, dtype)
+    gc = synth.GroupCfg(layers_per_group=2, order=synth.ORDER_RANDOM, order_seed=4)
+    oc = synth.OptCfg(kind=kind, lr=1e-3, eps=1e-8 if kind != 4 else 1e-30, sched=1, total_cycles=5,
+                      offload_state=offload, prefetch_groups=1)
+    batches = [tuple(torch.from_numpy(a).cuda() for a in synth.lm_batch(cfg, 6, t)) for t in range(9)]
+    a = HiFT(cfg, gc, oc)
+    a.set_params(synth.init_params(cfg, 2))
+    for t in range(4):
+        a.step(*batches[t])
+    path = str(tmp_path / "ckpt.bin")
+    a.save(path)
+    b = HiFT(cfg, gc, oc)
+    b.load(path)
+    assert b.step_count() == 4 and b.active_group() == a.active_group() and b.current_lr() == a.current_lr()
+    for t in range(4, 9):
+        assert a.step(*batches[t]) == b.step(*batches[t])
+    for n in a.tensor_names():
+        assert np.array_equal(a.get_param(n), b.get_param(n)), n
+        assert np.array_equal(a.get_model_param(n), b.get_model_param(n)), n
+    other = HiFT(cfg, gc, synth.OptCfg(kind=(kind + 1) % 3, lr=1e-3))
+    with pytest.raises(HiftError):
+        other.load(path)                                   # different optimizer: refused
+    with pytest.raises(HiftError):
+        b.load(str(tmp_path / "missing.bin"))
+    for h in (a, b, other):
+        h.close()
