@@ -94,7 +94,7 @@ template <int DH>
 constexpr int attn_fwd_smem_bytes() { return 4 * 64 * DH * 2; }
 
 template <int DH>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 3)
 attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* __restrict__ lse,
                     int S, int H, int causal, float scale) {
   constexpr int BQ = 64, BKV = 64, KS = DH / 16;

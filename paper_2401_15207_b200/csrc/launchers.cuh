@@ -77,6 +77,7 @@ inline void attention_mma_fwd(cudaStream_t st, int B, int S, int H, int causal, 
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(attn_fwd_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_fwd_smem_bytes<DH>());
+    cudaFuncSetAttribute(attn_fwd_mma_kernel<DH>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);   // three CTAs per SM
     attr_set = true;
   }
   dim3 grid((S + 63) / 64, H, B);
@@ -89,6 +90,8 @@ inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, 
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(attn_bwd_dkv_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_dkv_smem_bytes<DH>());
+    cudaFuncSetAttribute(attn_bwd_dkv_mma_kernel<DH>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    cudaFuncSetAttribute(attn_bwd_dq_mma_kernel<DH>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     attr_set = true;
   }
   const float scale = 1.0f / sqrtf((float)DH);
