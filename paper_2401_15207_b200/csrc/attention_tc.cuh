@@ -1,0 +1,281 @@
+// Attention forward on tcgen05: scores and the output accumulator live in tensor memory.
+// Included into gemm_tc.cu (inside its unnamed namespace) so that it shares the PTX wrappers,
+// the bounded mbarrier waits, the time-out flag and the tensor-map cache.
+//
+// One CTA = one (batch, head) and 128 query rows; key blocks of 128.
+//   warp 0    : TMA producer (Q once; K and V blocks through two 2-deep rings)
+//   warp 1    : MMA issuer and tensor-memory owner
+//                 S_j = Q K_j^T        (M 128 x N 128, k = d_h)      -> TMEM columns [0,128) / [128,256)
+//                 O  += P_j V_j        (M 128 x N d_h, k = 128 keys) -> TMEM columns [256, 256 + d_h)
+//   warps 2-5 : softmax, one thread per query row (= one tensor-memory lane): read S_j, mask,
+//               running max / sum, write P_j as bf16 into a 128-byte-swizzled shared tile (the A
+//               operand of the second product), rescale O in tensor memory when the maximum moved,
+//               and at the end normalise and store O and the log-sum-exp.
+// Q and K are K-major operands (d_h contiguous), V is an N-major operand (B(k = key, n = e) =
+// V[key][e]): all three are read straight out of qkv[T, 3d] by one tensor map, nothing is copied
+// or transposed.  Rows of a tile that lie beyond this batch entry's sequence hold the next
+// entry's (finite) values or TMA zero fill; their scores are masked, their probabilities are 0.
+#pragma once
+
+constexpr int kAttThreads = 192;
+constexpr int kAttBQ = 128, kAttBK = 128;
+
+template <int DH> struct AttnTcCfg {
+  static constexpr int kSpans = DH / 64;                       // 64-column swizzle spans per row
+  static constexpr int kTileBytes = 128 * DH * 2;              // one Q / K / V tile
+  static constexpr int kPBytes = 128 * kAttBK * 2;             // P tile: 128 rows x 128 keys
+  static constexpr int kSmem = 5 * kTileBytes + kPBytes + 1024 + 256;
+};
+
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+        "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+        "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// descriptor of a K-major tile with rows of 64 elements (one span), 128-byte swizzle
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// descriptor of an N-major operand staged as [k rows][64] boxes that are `box_bytes` apart along N
+__device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr, uint32_t box_bytes) {
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(box_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(kAttThreads, 1)
+attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* __restrict__ o,
+                   float* __restrict__ lse, int S, int H, int causal, float scale) {
+  typedef AttnTcCfg<DH> Cfg;
+  constexpr int SP = Cfg::kSpans;
+  constexpr int SPAN_BYTES = 128 * 128;                 // 128 rows x 64 elements x 2 bytes
+  extern __shared__ uint8_t smem_raw[];
+  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kAttBQ;
+  const int d = H * DH;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = base;
+  const uint32_t sK = sQ + Cfg::kTileBytes;             // two stages
+  const uint32_t sV = sK + 2 * Cfg::kTileBytes;         // two stages
+  const uint32_t sP = sV + 2 * Cfg::kTileBytes;
+  const uint32_t bar = sP + Cfg::kPBytes;
+  const uint32_t q_full = bar, k_full0 = bar + 8, k_empty0 = bar + 24, v_full0 = bar + 40, v_empty0 = bar + 56,
+                 s_full0 = bar + 72, p_ready = bar + 88, o_done = bar + 96, tmem_slot = bar + 104;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
+  uint8_t* p_gen = gen + (sP - base);
+
+  const int kv_len = causal ? min(S, q0 + kAttBQ) : S;
+  const int nblk = (kv_len + kAttBK - 1) / kAttBK;
+  const bool poisoned = g_tc_error != 0;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(k_full0 + 8 * i, 1); mbar_init(k_empty0 + 8 * i, 1);
+      mbar_init(v_full0 + 8 * i, 1); mbar_init(v_empty0 + 8 * i, 1);
+      mbar_init(s_full0 + 8 * i, 1);
+    }
+    mbar_init(p_ready, 4);                              // one arrival per softmax warp
+    mbar_init(o_done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_gen;
+  const uint32_t tO = tmem_base + 256;
+
+  const int row_g0 = b * S;                             // first row of this batch entry in qkv
+  const int colQ = h * DH, colK = d + h * DH, colV = 2 * d + h * DH;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0 && !poisoned) {
+      mbar_expect_tx(q_full, Cfg::kTileBytes);
+#pragma unroll
+      for (int sp = 0; sp < SP; ++sp) tma_load_2d(sQ + sp * SPAN_BYTES, &tmap_qkv, q_full, colQ + sp * 64, row_g0 + q0);
+      bool ok = true;
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        const int krow = row_g0 + j * kAttBK;
+        if (!mbar_wait(k_empty0 + 8 * st, ph ^ 1)) { atomicCAS(&g_tc_error, 0, 4); ok = false; break; }
+        mbar_expect_tx(k_full0 + 8 * st, Cfg::kTileBytes);
+#pragma unroll
+        for (int sp = 0; sp < SP; ++sp)
+          tma_load_2d(sK + st * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, k_full0 + 8 * st, colK + sp * 64, krow);
+        if (!mbar_wait(v_empty0 + 8 * st, ph ^ 1)) { atomicCAS(&g_tc_error, 0, 4); ok = false; break; }
+        mbar_expect_tx(v_full0 + 8 * st, Cfg::kTileBytes);
+#pragma unroll
+        for (int sp = 0; sp < SP; ++sp)
+          tma_load_2d(sV + st * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, v_full0 + 8 * st, colV + sp * 64, krow);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0 && !poisoned) {
+      // S: A = Q (K-major), B = K (K-major), N = 128.  O: A = P (K-major), B = V (N-major), N = DH.
+      const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAttBK >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      bool ok = mbar_wait(q_full, 0);
+      if (!ok) atomicCAS(&g_tc_error, 0, 5);
+      auto issue_s = [&](int j) -> bool {
+        const int st = j & 1;
+        if (!mbar_wait(k_full0 + 8 * st, (j >> 1) & 1)) { atomicCAS(&g_tc_error, 0, 5); return false; }
+        tc_fence_after();
+        const uint32_t ts = tmem_base + (uint32_t)(st * 128);
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint32_t off = (uint32_t)((kk / 4) * SPAN_BYTES + (kk % 4) * 32);
+          tc_mma(ts, desc_kmajor(sQ + off), desc_kmajor(sK + st * Cfg::kTileBytes + off), idesc_s, kk > 0 ? 1u : 0u);
+        }
+        tc_commit(s_full0 + 8 * st);
+        tc_commit(k_empty0 + 8 * st);
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      if (ok && nblk > 1) ok = issue_s(1);
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int st = j & 1;
+        if (!mbar_wait(p_ready, j & 1)) { atomicCAS(&g_tc_error, 0, 5); ok = false; break; }
+        if (!mbar_wait(v_full0 + 8 * st, (j >> 1) & 1)) { atomicCAS(&g_tc_error, 0, 5); ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kAttBK / 16; ++kk) {
+          // P: 128 keys = two 64-key spans, 32 bytes per 16 keys inside a span; V: 16 key rows of 128 bytes
+          const uint64_t da = desc_kmajor(sP + (uint32_t)((kk / 4) * SPAN_BYTES + (kk % 4) * 32));
+          const uint64_t db = desc_nmajor(sV + st * Cfg::kTileBytes + (uint32_t)(kk * 16 * 128), SPAN_BYTES);
+          tc_mma(tO, da, db, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(o_done);
+        tc_commit(v_empty0 + 8 * st);
+        if (j + 2 < nblk) ok = issue_s(j + 2);
+      }
+    }
+  } else {
+    // ---------------- softmax and epilogue: thread = query row = tensor-memory lane
+    const int q = warp & 3;
+    const int r = q * 32 + lane;                        // row inside the tile
+    const int qrow = q0 + r;
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    const float sl2 = scale * 1.4426950408889634f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = !poisoned;
+    for (int j = 0; j < nblk; ++j) {
+      const int st = j & 1;
+      bool ready = ok && mbar_wait(s_full0 + 8 * st, (j >> 1) & 1);
+      if (ok && !ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
+      tc_fence_after();
+      ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
+      if (!ok) break;
+      // scores of this row: 128 columns
+      float sc[kAttBK];
+#pragma unroll
+      for (int c0 = 0; c0 < kAttBK; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + lane_off + (uint32_t)(st * 128 + c0), v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sc[c0 + i] = __uint_as_float(v[i]);
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < kAttBK; ++i) {
+        const int key = j * kAttBK + i;
+        float x = sc[i] * sl2;
+        if (key >= S || (causal && key > qrow)) x = -INFINITY;
+        sc[i] = x;
+        mx = fmaxf(mx, x);
+      }
+      const float mnew = fmaxf(m, mx);
+      const float muse = (mnew == -INFINITY) ? 0.f : mnew;
+      const float corr = exp2f(m - muse);
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < kAttBK; ++i) { sc[i] = exp2f(sc[i] - muse); sum += sc[i]; }
+      l = l * corr + sum;
+      m = mnew;
+      // the previous P V product must be finished before P is overwritten and O is rescaled
+      if (j > 0) {
+        ready = mbar_wait(o_done, (j - 1) & 1);
+        if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
+        tc_fence_after();
+        ok = __all_sync(0xffffffffu, ready);
+        if (!ok) break;
+      }
+      // P row -> shared memory, bf16, K-major with the 128-byte swizzle the MMA descriptor expects
+#pragma unroll
+      for (int ch = 0; ch < kAttBK / 8; ++ch) {
+        uint4 pk;
+        __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) hp[t] = __floats2bfloat162_rn(sc[ch * 8 + 2 * t], sc[ch * 8 + 2 * t + 1]);
+        const int span = ch >> 3, c = ch & 7;
+        *reinterpret_cast<uint4*>(p_gen + span * SPAN_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = pk;
+      }
+      if (j > 0) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < DH; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
+          tmem_st32(tO + lane_off + (uint32_t)c0, v);
+        }
+        tmem_st_wait();
+      }
+      fence_async_smem();                               // P is read by the tensor core (async proxy)
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_ready);
+    }
+    // last product done -> normalise and store
+    if (ok && nblk > 0) {
+      const bool ready = mbar_wait(o_done, (nblk - 1) & 1);
+      if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
+      tc_fence_after();
+      ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
+    }
+    if (ok) {
+      const float inv = 1.0f / l;
+      __nv_bfloat16* orow = o + ((int64_t)(row_g0 + qrow)) * d + (int64_t)h * DH;
+#pragma unroll 1
+      for (int c0 = 0; c0 < DH; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+        if (qrow < S) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 pk;
+            __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+              hp[t] = __floats2bfloat162_rn(__uint_as_float(v[i + 2 * t]) * inv, __uint_as_float(v[i + 2 * t + 1]) * inv);
+            *reinterpret_cast<uint4*>(orow + c0 + i) = pk;
+          }
+        }
+      }
+      if (qrow < S) lse[((int64_t)b * H + h) * S + qrow] = (m + log2f(l)) * 0.6931471805599453f;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}

@@ -20,6 +20,7 @@
 
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
@@ -568,6 +569,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   }
 }
 
+#include "attention_tc.cuh"
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -653,6 +656,7 @@ template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr2() {
   return cudaFuncSetAttribute(gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
+int g_attn_tc = 1;       // tcgen05 attention forward (HIFT_ATTN_TC=0 falls back to the mma.sync kernel)
 int g_pair_mode = 1;     // CTA-pair kernel for 256-wide tiles (HIFT_GEMM_PAIR=0 falls back to one CTA per tile)
 
 }  // namespace
@@ -685,6 +689,9 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr2<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr2<true, true, true>();
   if (const char* pm = getenv("HIFT_GEMM_PAIR")) g_pair_mode = atoi(pm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
+  if (const char* am = getenv("HIFT_ATTN_TC")) g_attn_tc = atoi(am);
   if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
   g_init_state = 0;
   return 0;
@@ -773,6 +780,25 @@ const int* gemm_tc_error_device_ptr() {
     else cudaGetLastError();
   }
   return ptr;
+}
+
+bool attn_tc_eligible(int dh, const void* qkv, int H) {
+  // head size 128 only: at 64 the softmax threads, not the tensor cores, set the pace and the
+  // warp-level kernel (more CTAs per SM) is faster; HIFT_ATTN_TC=2 forces this kernel for both sizes
+  return g_init_state == 0 && g_attn_tc && (dh == 128 || (dh == 64 && g_attn_tc == 2)) && (((uintptr_t)qkv) & 15) == 0 &&
+         ((3 * H * dh) % 8) == 0;
+}
+cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse) {
+  CUtensorMap tm;
+  const uint64_t d3 = 3ull * H * dh;
+  if (!get_map(qkv, d3, (uint64_t)B * S, d3, 128, &tm)) return cudaErrorInvalidValue;
+  dim3 grid((S + kAttBQ - 1) / kAttBQ, H, B);
+  const float scale = 1.0f / sqrtf((float)dh);
+  if (dh == 64)
+    attn_fwd_tc_kernel<64><<<grid, kAttThreads, AttnTcCfg<64>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, S, H, causal, scale);
+  else
+    attn_fwd_tc_kernel<128><<<grid, kAttThreads, AttnTcCfg<128>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, S, H, causal, scale);
+  return cudaGetLastError();
 }
 
 int gemm_tc_set_error(int v) {

@@ -14,6 +14,9 @@ int gemm_tc_init();
 // 16-byte aligned with 16-byte-multiple leading dimensions.
 bool gemm_tc_eligible(const GemmArgs& g);
 cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g);
+// Attention forward on tcgen05 (scores and output in tensor memory): bf16, head size 64 or 128.
+bool attn_tc_eligible(int dh, const void* qkv, int H);
+cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse);
 // 0 if no tensor-core kernel has given up on a bounded wait since the library was loaded, else the
 // code of the first one (1 producer, 2 MMA issuer, 3 epilogue); -1 if the flag cannot be read.
 int gemm_tc_poll_error();

@@ -2,6 +2,7 @@
 // grid.  Shared by the training-step engine and the single-kernel C entry points.
 #pragma once
 #include "gemm_args.h"
+#include "gemm_tc.h"
 #include "kernels_attention.cuh"
 #include "kernels_attention_mma.cuh"
 #include "kernels_gemm_simt.cuh"
@@ -105,6 +106,10 @@ inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, 
 inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
                                  const void* qkv, void* o, float* lse) {
   if (attention_use_mma(dtype, dh)) {
+    if (gemm_tc_init() == 0 && attn_tc_eligible(dh, qkv, H)) {        // tcgen05 kernel
+      attn_tc_fwd_launch(st, B, S, H, dh, causal, qkv, o, lse);
+      return;
+    }
     if (dh == 64) attention_mma_fwd<64>(st, B, S, H, causal, qkv, o, lse);
     else attention_mma_fwd<128>(st, B, S, H, causal, qkv, o, lse);
     return;
