@@ -570,6 +570,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 }
 
 #include "attention_tc.cuh"
+#include "attention_bwd_tc.cuh"
 
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -657,6 +658,12 @@ cudaError_t set_smem_attr2() {
   return cudaFuncSetAttribute(gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 int g_attn_tc = 1;       // tcgen05 attention forward (HIFT_ATTN_TC=0 falls back to the mma.sync kernel)
+int g_attn_bwd_tc = 1;   // tcgen05 attention backward (HIFT_ATTN_BWD_TC=0 falls back to the mma.sync kernels)
+template <int DH, int MODE>
+cudaError_t set_smem_attr_ab() {
+  return cudaFuncSetAttribute(attn_bwd_tc_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              AttnBwdCfg<DH, MODE>::kSmem);
+}
 int g_pair_mode = 1;     // CTA-pair kernel for 256-wide tiles (HIFT_GEMM_PAIR=0 falls back to one CTA per tile)
 
 }  // namespace
@@ -692,6 +699,11 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
   if (const char* am = getenv("HIFT_ATTN_TC")) g_attn_tc = atoi(am);
+  if (e == cudaSuccess) e = set_smem_attr_ab<64, 0>();
+  if (e == cudaSuccess) e = set_smem_attr_ab<64, 1>();
+  if (e == cudaSuccess) e = set_smem_attr_ab<128, 0>();
+  if (e == cudaSuccess) e = set_smem_attr_ab<128, 1>();
+  if (const char* am = getenv("HIFT_ATTN_BWD_TC")) g_attn_bwd_tc = atoi(am);
   if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
   g_init_state = 0;
   return 0;
@@ -799,6 +811,34 @@ cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int
   else
     attn_fwd_tc_kernel<128><<<grid, kAttThreads, AttnTcCfg<128>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, S, H, causal, scale);
   return cudaGetLastError();
+}
+
+bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, const void* dqkv) {
+  return g_init_state == 0 && g_attn_bwd_tc && (dh == 64 || dh == 128) && ((H * dh) % 8) == 0 &&
+         ((((uintptr_t)qkv) | ((uintptr_t)dout) | ((uintptr_t)dqkv)) & 15) == 0;
+}
+template <int DH>
+static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, const void* dout,
+                                    const float* lse, const float* dsum, void* dqkv) {
+  const uint64_t d = (uint64_t)H * DH, d3 = 3 * d, rows = (uint64_t)B * S;
+  CUtensorMap qkv_f, qkv_x, do_f, do_x;
+  if (!get_map(qkv, d3, rows, d3, kAbF, &qkv_f) || !get_map(qkv, d3, rows, d3, kAbX, &qkv_x) ||
+      !get_map(dout, d, rows, d, kAbF, &do_f) || !get_map(dout, d, rows, d, kAbX, &do_x))
+    return cudaErrorInvalidValue;
+  dim3 grid((S + kAbF - 1) / kAbF, H, B);
+  const float scale = 1.0f / sqrtf((float)DH);
+  // dK, dV: fixed K, V; streamed Q, dO
+  attn_bwd_tc_kernel<DH, 0><<<grid, kAbThreads, AttnBwdCfg<DH, 0>::kSmem, st>>>(
+      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, S, H, causal, scale);
+  // dQ: fixed Q, dO; streamed K, V
+  attn_bwd_tc_kernel<DH, 1><<<grid, kAbThreads, AttnBwdCfg<DH, 1>::kSmem, st>>>(
+      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, S, H, causal, scale);
+  return cudaGetLastError();
+}
+cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,
+                               const float* lse, const float* dsum, void* dqkv) {
+  if (dh == 64) return attn_tc_bwd_inst<64>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv);
+  return attn_tc_bwd_inst<128>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv);
 }
 
 int gemm_tc_set_error(int v) {

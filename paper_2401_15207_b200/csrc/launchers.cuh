@@ -124,6 +124,12 @@ inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H
                                  const void* qkv, const void* o, const float* lse, const void* dout,
                                  void* dqkv, float* dsum) {
   if (attention_use_mma(dtype, dh)) {
+    if (gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv)) {   // tcgen05 kernels
+      const int64_t warps = (int64_t)B * S * H;
+      attn_dsum_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
+      attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv);
+      return;
+    }
     if (dh == 64) attention_mma_bwd<64>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum);
     else attention_mma_bwd<128>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum);
     return;
