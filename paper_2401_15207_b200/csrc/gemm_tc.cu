@@ -825,14 +825,15 @@ static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int ca
   if (!get_map(qkv, d3, rows, d3, kAbF, &qkv_f) || !get_map(qkv, d3, rows, d3, kAbX, &qkv_x) ||
       !get_map(dout, d, rows, d, kAbF, &do_f) || !get_map(dout, d, rows, d, kAbX, &do_x))
     return cudaErrorInvalidValue;
-  dim3 grid((S + kAbF - 1) / kAbF, H, B);
+  const int nitems = ((S + kAbF - 1) / kAbF) * H * B;
+  const int grid = nitems < g_num_sms ? nitems : g_num_sms;       // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)DH);
   // dK, dV: fixed K, V; streamed Q, dO
   attn_bwd_tc_kernel<DH, 0><<<grid, kAbThreads, AttnBwdCfg<DH, 0>::kSmem, st>>>(
-      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, S, H, causal, scale);
+      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale);
   // dQ: fixed Q, dO; streamed K, V
   attn_bwd_tc_kernel<DH, 1><<<grid, kAbThreads, AttnBwdCfg<DH, 1>::kSmem, st>>>(
-      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, S, H, causal, scale);
+      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale);
   return cudaGetLastError();
 }
 cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,

@@ -229,25 +229,38 @@ attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* _
 }
 
 // ------------------------------------------------------------------ backward: dsum = rowsum(do * o)
-// one warp per (token, head)
+// DH/8 consecutive lanes per (token, head) row, 16 bytes of o and of do per lane; the row sum is
+// a shuffle reduction inside that lane group (fixed order).  dsum layout [B, H, S].
+template <int DH>
 __global__ void attn_dsum_kernel(const bf16* __restrict__ o, const bf16* __restrict__ dout,
-                                 float* __restrict__ dsum, int B, int S, int H, int DH) {
-  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (w >= (int64_t)B * S * H) return;
-  const int h = (int)(w % H);
-  const int64_t tok = w / H;
-  const int b = (int)(tok / S), s = (int)(tok % S);
-  const bf16* po = o + tok * (int64_t)H * DH + (int64_t)h * DH;
-  const bf16* pg = dout + tok * (int64_t)H * DH + (int64_t)h * DH;
+                                 float* __restrict__ dsum, int B, int S, int H) {
+  constexpr int LPR = DH / 8;                              // lanes per row: 8 or 16
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t row = i / LPR;                             // (token, head)
+  const int part = (int)(i % LPR);
+  const int64_t nrows = (int64_t)B * S * H;
   float acc = 0.f;
-  for (int e = lane * 2; e < DH; e += 64) {
-    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + e));
-    const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pg + e));
-    acc += a.x * c.x + a.y * c.y;
+  if (row < nrows) {
+    float a[8], c[8];
+    load8(o + row * DH + part * 8, a);
+    load8(dout + row * DH + part * 8, c);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc += a[e] * c[e];
   }
-  acc = warp_sum(acc);
-  if (lane == 0) dsum[((int64_t)b * H + h) * S + s] = acc;
+#pragma unroll
+  for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (row < nrows && part == 0) {
+    const int h = (int)(row % H);
+    const int64_t tok = row / H;
+    const int b = (int)(tok / S), sq = (int)(tok % S);
+    dsum[((int64_t)b * H + h) * S + sq] = acc;
+  }
+}
+inline void launch_attn_dsum(cudaStream_t st, const bf16* o, const bf16* dout, float* dsum, int B, int S, int H, int DH) {
+  const int64_t threads = (int64_t)B * S * H * (DH / 8);
+  const unsigned grid = (unsigned)((threads + 255) / 256);
+  if (DH == 64) attn_dsum_kernel<64><<<grid, 256, 0, st>>>(o, dout, dsum, B, S, H);
+  else attn_dsum_kernel<128><<<grid, 256, 0, st>>>(o, dout, dsum, B, S, H);
 }
 
 // ------------------------------------------------------------------ backward: dq (owner of query rows)

@@ -96,8 +96,7 @@ inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, 
     attr_set = true;
   }
   const float scale = 1.0f / sqrtf((float)DH);
-  const int64_t warps = (int64_t)B * S * H;
-  attn_dsum_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)dout, dsum, B, S, H, DH);
+  launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, DH);
   dim3 grid((S + 63) / 64, H, B);
   attn_bwd_dq_mma_kernel<DH><<<grid, 128, 0, st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum, (bf16*)dqkv, S, H, causal, scale);
   attn_bwd_dkv_mma_kernel<DH><<<grid, 128, attn_dkv_smem_bytes<DH>(), st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum,
@@ -124,9 +123,8 @@ inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H
                                  const void* qkv, const void* o, const float* lse, const void* dout,
                                  void* dqkv, float* dsum) {
   if (attention_use_mma(dtype, dh)) {
-    if (gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv)) {   // tcgen05 kernels
-      const int64_t warps = (int64_t)B * S * H;
-      attn_dsum_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
+    if (gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv) && (((uintptr_t)o) & 15) == 0) {   // tcgen05 kernels
+      launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
       attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv);
       return;
     }
