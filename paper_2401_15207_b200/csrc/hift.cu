@@ -45,7 +45,7 @@ struct GroupRec {
   int unit_lo, unit_hi;
   size_t off, numel;      // span in the flat parameter buffer (padded)
   int64_t tau;            // updates so far
-  char* blob;             // pinned host: [master][state]
+  char* blob;             // pinned host: [master][state]; compact master: [state][low halves u16][carry bits]
   size_t blob_bytes;
   size_t state_floats;    // floats of optimizer state (n_state * numel, or the compact Adafactor state)
   size_t af_base;         // Adafactor, state resident: offset of the group's compact state in af_all
@@ -68,6 +68,7 @@ struct hift_ctx {
   int L = 0, d = 0, f = 0, fa = 0, H = 0, dh = 0, T = 0, B = 0, S = 0, V = 0, Vp = 0;
   int n_state = 2;
   bool mixed = true, offload = false;
+  bool compact = false;             // paged master = low halves + carry bits beside the bf16 copy (see blob layout)
   std::vector<TensorRec> tens;
   std::vector<std::vector<int>> unit_tens;
   std::vector<GroupRec> groups;
@@ -89,7 +90,7 @@ struct hift_ctx {
   float* af_all = nullptr;          // Adafactor, state resident: compact state of every group
   float* af_scratch = nullptr;      // Adafactor work space, sized for the largest tensor
   bool af = false;
-  char* slot[2] = {nullptr, nullptr};   // offload staging: [master][s0][s1] per slot
+  char* slot[2] = {nullptr, nullptr};   // offload staging, laid out like the blob
   int n_slots = 1;
   float* grad = nullptr;            // [max_group]
   char* arena = nullptr; size_t arena_cap = 0, arena_off = 0, arena_fixed = 0;
@@ -669,7 +670,8 @@ void enqueue_update(hift_ctx* c) {
   void* pbf = nullptr;
   if (c->offload) {
     float* base = (float*)c->slot[sl];
-    if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
+    if (c->compact) { mst = nullptr; s0 = base; s1 = base + gr.numel; pbf = c->params + gr.off * c->es; }
+    else if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
     else { mst = (float*)c->params + gr.off; s0 = base; s1 = base + gr.numel; }
     c->note(cudaEventRecord(c->tl[3], c->st));
     c->note(cudaStreamWaitEvent(c->st, c->ev_h2d[sl], 0));
@@ -682,8 +684,16 @@ void enqueue_update(hift_ctx* c) {
   }
   const OptScalars hs = make_opt_scalars(c->oc.kind, lr, c->oc.beta1, c->oc.beta2, c->oc.eps,
                                          c->oc.weight_decay, c->oc.momentum, gr.tau);
+  if (c->compact) {
+    // read p, lo, carry, gradient, state; write p, lo, carry, state
+    const double opt_bytes = (double)gr.numel * (12.25 + 8.0 * c->n_state);
+    uint16_t* lo16 = (uint16_t*)((float*)c->slot[sl] + gr.state_floats);
+    uint8_t* carry8 = (uint8_t*)(lo16 + gr.numel);
+    LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, gr.numel, pbf, lo16, carry8, c->grad, s0, s1, hs));
+  } else {
   const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
   LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs));
+  }
   }
 
   // ---------------- state back to the host (step k)
@@ -749,12 +759,54 @@ float* plane_ptr(hift_ctx* c, int ti, int plane, bool* on_host) {
   if (plane == 0 && !c->mixed) return (float*)c->params + r.off;
   if (c->offload) {
     *on_host = true;
-    const int pl = c->mixed ? plane : plane - 1;
+    if (c->compact && plane == 0) return nullptr;        // not stored as floats: see master_read / master_write
+    const int pl = (c->mixed && !c->compact) ? plane : plane - 1;
     return (float*)gr.blob + (size_t)pl * gr.numel + (r.off - gr.off);
   }
   if (plane == 0) return c->master_all + r.off;
   if (plane == 1) return c->s0_all ? c->s0_all + r.off : nullptr;
   return c->s1_all ? c->s1_all + r.off : nullptr;
+}
+
+// ---- compact master on the host side (same arithmetic as master_pack / master_unpack on the device)
+inline void host_master_pack(uint32_t u, uint32_t& p, uint32_t& lo, uint32_t& carry) {
+  lo = u & 0xFFFFu;
+  if ((u & 0x7F800000u) == 0x7F800000u) {
+    p = u >> 16;
+    if (lo && !(p & 0x7Fu)) p |= 0x40u;
+    carry = 0;
+  } else {
+    p = (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+    carry = p - (u >> 16);
+  }
+}
+uint16_t* blob_lo16(const hift_ctx* c, const GroupRec& gr) { (void)c; return (uint16_t*)((float*)gr.blob + gr.state_floats); }
+uint8_t* blob_carry8(const hift_ctx* c, const GroupRec& gr) { return (uint8_t*)(blob_lo16(c, gr) + gr.numel); }
+// fp32 master values of elements [o, o + n) of a group, rebuilt from the device's bf16 copy and the blob
+bool master_read(hift_ctx* c, const GroupRec& gr, size_t o, size_t n, float* dst) {
+  std::vector<uint16_t> p(n);
+  if (cudaMemcpy(p.data(), c->params + (gr.off + o) * c->es, n * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return false;
+  const uint16_t* lo = blob_lo16(c, gr) + o;
+  const uint8_t* cr = blob_carry8(c, gr);
+  for (size_t i = 0; i < n; ++i) {
+    const uint32_t carry = (cr[(o + i) >> 3] >> ((o + i) & 7)) & 1u;
+    const uint32_t u = (((uint32_t)p[i] - carry) << 16) | lo[i];
+    memcpy(dst + i, &u, 4);
+  }
+  return true;
+}
+// the blob's share of new master values (the bf16 copy on the device is the caller's job)
+void master_write(hift_ctx* c, GroupRec& gr, size_t o, size_t n, const float* src) {
+  uint16_t* lo = blob_lo16(c, gr) + o;
+  uint8_t* cr = blob_carry8(c, gr);
+  for (size_t i = 0; i < n; ++i) {
+    uint32_t u, p, l, carry;
+    memcpy(&u, src + i, 4);
+    host_master_pack(u, p, l, carry);
+    lo[i] = (uint16_t)l;
+    uint8_t& byte = cr[(o + i) >> 3];
+    byte = (uint8_t)((byte & ~(1u << ((o + i) & 7))) | (carry << ((o + i) & 7)));
+  }
 }
 
 }  // namespace
@@ -831,6 +883,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // plain SGD on fp32 parameters has nothing to page (the paper's "no state, zero traffic" case)
   c->offload = oc->offload_state != 0 && ((m->dtype == 1 ? 1 : 0) + c->n_state + (c->af ? 1 : 0)) > 0;
   c->n_slots = (c->offload && oc->prefetch_groups) ? 2 : 1;
+  // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
+  c->compact = c->mixed && c->offload && !c->af;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_work, 0, sizeof(c->prof_work));
@@ -871,19 +925,22 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (cudaStreamCreateWithFlags(&c->st_d2h, cudaStreamNonBlocking) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
   // ---- parameters, gradients, optimizer state
-  auto blob_floats = [&](const GroupRec& g) { return (c->mixed ? g.numel : 0) + g.state_floats; };
-  size_t slot_floats = 0, af_total = 0;
-  for (auto& g : c->groups) { slot_floats = std::max(slot_floats, blob_floats(g)); af_total += c->af ? g.state_floats : 0; }
+  auto blob_bytes_of = [&](const GroupRec& g) {
+    if (c->compact) return g.state_floats * sizeof(float) + g.numel * 2 + g.numel / 8;     // numel is a multiple of 128
+    return ((c->mixed ? g.numel : 0) + g.state_floats) * sizeof(float);
+  };
+  size_t slot_bytes_max = 0, af_total = 0;
+  for (auto& g : c->groups) { slot_bytes_max = std::max(slot_bytes_max, blob_bytes_of(g)); af_total += c->af ? g.state_floats : 0; }
   if ((rc = dev_alloc(c, (void**)&c->params, c->total * c->es)) != HIFT_OK) return fail(rc);
   cudaMemsetAsync(c->params, 0, c->total * c->es, c->st);
   if ((rc = dev_alloc(c, (void**)&c->grad, c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
   if (c->offload) {
     for (int s = 0; s < c->n_slots; ++s) {
-      if ((rc = dev_alloc(c, (void**)&c->slot[s], slot_floats * sizeof(float))) != HIFT_OK) return fail(rc);
-      cudaMemsetAsync(c->slot[s], 0, slot_floats * sizeof(float), c->st);
+      if ((rc = dev_alloc(c, (void**)&c->slot[s], slot_bytes_max)) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->slot[s], 0, slot_bytes_max, c->st);
     }
     for (auto& g : c->groups) {
-      g.blob_bytes = blob_floats(g) * sizeof(float);
+      g.blob_bytes = blob_bytes_of(g);
       if (cudaHostAlloc((void**)&g.blob, g.blob_bytes, cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         g.blob = nullptr;
@@ -1060,7 +1117,10 @@ hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) 
   bool on_host;
   float* mp = plane_ptr(c, ti, 0, &on_host);
   // every copy goes through the context's stream, so the cast below is ordered after its input
-  if (on_host) memcpy(mp, src, n * sizeof(float));
+  if (c->compact) {
+    GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
+    master_write(c, gr, c->tens[ti].off - gr.off, n, src);
+  } else if (on_host) memcpy(mp, src, n * sizeof(float));
   else if (cudaMemcpyAsync(mp, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
   if (c->mixed) {
     // stage the fp32 values in the gradient buffer (any tensor fits in the largest group)
@@ -1074,6 +1134,10 @@ hift_status hift_get_param(hift_ctx* c, int32_t ti, float* dst, size_t n) {
   sync_all(c);
   bool on_host;
   float* mp = plane_ptr(c, ti, 0, &on_host);
+  if (c->compact) {
+    const GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
+    return master_read(c, gr, c->tens[ti].off - gr.off, n, dst) ? HIFT_OK : HIFT_ERR_CUDA;
+  }
   if (on_host) memcpy(dst, mp, n * sizeof(float));
   else if (cudaMemcpy(dst, mp, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
   return HIFT_OK;
@@ -1130,15 +1194,21 @@ hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
   for (size_t g = 0; g < c->groups.size(); ++g) {
     GroupRec& gr = c->groups[g];
     if (c->offload) cudaMemsetAsync(c->slot[0], 0, gr.blob_bytes, c->st);
+    if (c->compact) cudaMemsetAsync(c->grad, 0, gr.numel * sizeof(float), c->st);     // alignment gaps pack to zero
     for (int u = gr.unit_lo; u <= gr.unit_hi; ++u) {
       for (int ti : c->unit_tens[u]) {
         const TensorRec& r = c->tens[ti];
         float* mp = nullptr;
-        if (c->mixed) mp = c->offload ? (float*)c->slot[0] + (r.off - gr.off) : c->master_all + r.off;
+        if (c->compact) mp = c->grad + (r.off - gr.off);           // staged as floats, packed below
+        else if (c->mixed) mp = c->offload ? (float*)c->slot[0] + (r.off - gr.off) : c->master_all + r.off;
         const uint64_t sd = seed * 0x9E3779B97F4A7C15ull + (uint64_t)ti * 0xD1B54A32D192ED03ull;
         if (c->mixed) init_tensor_kernel<bf16><<<grid_for(r.numel, 256), 256, 0, c->st>>>((bf16*)c->P(ti), mp, r.numel, r.init_kind, (float)stdv, sd);
         else init_tensor_kernel<float><<<grid_for(r.numel, 256), 256, 0, c->st>>>((float*)c->P(ti), nullptr, r.numel, r.init_kind, (float)stdv, sd);
       }
+    }
+    if (c->compact) {
+      uint16_t* lo16 = (uint16_t*)((float*)c->slot[0] + gr.state_floats);
+      master_pack_kernel<<<grid_for(gr.numel / 8, 256), 256, 0, c->st>>>(c->grad, lo16, (uint8_t*)(lo16 + gr.numel), gr.numel / 8);
     }
     if (c->offload) {
       cudaMemcpyAsync(gr.blob, c->slot[0], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st);
@@ -1170,9 +1240,10 @@ struct CkptHeader {
 void group_locations(hift_ctx* c, GroupRec& gr, float** master, bool* master_host, float** state, bool* state_host) {
   *master_host = false; *state_host = false;
   if (!c->mixed) *master = (float*)c->params + gr.off;
+  else if (c->compact) { *master = nullptr; *master_host = true; }       // rebuilt / packed by the caller
   else if (c->offload) { *master = (float*)gr.blob; *master_host = true; }
   else *master = c->master_all + gr.off;
-  if (c->offload) { *state = (float*)gr.blob + (c->mixed ? gr.numel : 0); *state_host = true; }
+  if (c->offload) { *state = (float*)gr.blob + ((c->mixed && !c->compact) ? gr.numel : 0); *state_host = true; }
   else if (c->af) *state = c->af_all + gr.af_base;
   else *state = nullptr;      // two separate planes, handled by the caller
 }
@@ -1202,7 +1273,12 @@ hift_status hift_save(hift_ctx* c, const char* path) {
       ok = cudaMemcpy(tmp.data(), p, n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess &&
            fwrite(tmp.data(), sizeof(float), n, f) == n;
     };
-    put(mp, mh, gr.numel);
+    if (c->compact) {
+      // the file always holds fp32 master values, whatever the paged form
+      std::vector<float> mv(gr.numel);
+      ok = ok && master_read(c, gr, 0, gr.numel, mv.data());
+      put(mv.data(), true, gr.numel);
+    } else put(mp, mh, gr.numel);
     if (sp) put(sp, sh, gr.state_floats);
     else {
       if (c->s0_all) put(c->s0_all + gr.off, false, gr.numel);
@@ -1235,7 +1311,13 @@ hift_status hift_load(hift_ctx* c, const char* path) {
       ok = fread(tmp.data(), sizeof(float), n, f) == n &&
            cudaMemcpy(p, tmp.data(), n * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess;
     };
-    get(mp, mh, gr.numel);
+    std::vector<float> mv;
+    if (c->compact) {
+      mv.resize(gr.numel);
+      get(mv.data(), true, gr.numel);
+      if (ok) master_write(c, gr, 0, gr.numel, mv.data());
+      mp = mv.data();
+    } else get(mp, mh, gr.numel);
     if (sp) get(sp, sh, gr.state_floats);
     else {
       if (c->s0_all) get(c->s0_all + gr.off, false, gr.numel);

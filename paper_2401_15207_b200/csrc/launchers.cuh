@@ -222,4 +222,15 @@ inline void launch_fused_opt(cudaStream_t st, int kind, size_t n, void* param_bf
 #undef OPT
 }
 
+// compact master (bf16 copy + low halves + carry bits); n must be a multiple of 8
+inline void launch_fused_opt_compact(cudaStream_t st, int kind, size_t n, void* param_bf16, uint16_t* lo16, uint8_t* carry8,
+                                     const float* grad, float* s0, float* s1, const OptScalars& h) {
+  if (n == 0) return;
+  const size_t n8 = n / 8;
+  const int grid = grid_for(n8, 256, 148 * 8);
+#define OPTC(K) fused_opt_compact_kernel<K><<<grid, 256, 0, st>>>((uint16_t*)param_bf16, lo16, carry8, grad, s0, s1, n8, h)
+  if (kind == 0) { OPTC(0); } else if (kind == 1) { OPTC(1); } else if (kind == 2) { OPTC(2); } else { OPTC(3); }
+#undef OPTC
+}
+
 }  // namespace hift
