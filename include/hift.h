@@ -250,6 +250,16 @@ hift_status hift_k_attention_bwd(int32_t dtype, int32_t batch, int32_t seq, int3
                                  int32_t d_head, int32_t causal, const void *qkv_dev,
                                  const void *o_dev, const float *lse_dev, const void *do_dev,
                                  void *dqkv_dev, float *dsum_dev, void *cuda_stream);
+/* Rotary models (RoPE on q and k, as in the LLaMA-shaped configuration the paper profiles) on the
+ * tensor-core path: the rotation is fused into the epilogue of the qkv projection, and this hook
+ * exposes exactly that kernel: out[M,N] = rope(x[M,K] w[N,K]^T + bias) on columns [0, rope_cols),
+ * plain beyond.  cs_dev: fp32 [seq, d_head/2] cosines followed by [seq, d_head/2] sines of
+ * angle(pos, j) = pos * base^(-2j/d_head); pair (j, j + d_head/2); row r has position r mod seq.
+ * HIFT_ERR_CFG when the fused kernel does not apply (d_head != 128, operands not 16-byte aligned,
+ * N or rope_cols not a multiple of 128). */
+hift_status hift_k_linear_rope(int64_t M, int64_t N, int64_t K, const void *a_dev, const void *b_dev, void *out_dev,
+                               const void *bias_dev, const float *cs_dev, int32_t seq, int32_t d_head,
+                               int64_t rope_cols, void *cuda_stream);
 /* kind 0 LayerNorm (gain, bias), 1 RMSNorm (gain).  x is the fp32 residual stream in every
  * dtype; gain/bias/y have the operand type.  stats: fp32 [2*rows] (mean|rstd). */
 hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,

@@ -96,6 +96,7 @@ def _prototypes():
         "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
         "hift_k_attention_bwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+        "hift_k_linear_rope": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, i64, vp]),
         "hift_k_norm_fwd": (C.c_int, [i32, i32, i64, i64, f64, vp, vp, vp, vp, vp, vp]),
         "hift_k_norm_bwd": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "hift_k_norm_bwd_static": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
@@ -356,6 +357,11 @@ def k_attention_fwd(dtype, B, S, H, dh, causal, qkv, o, lse, stream=None):
 def k_attention_bwd(dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, stream=None):
     _check(lib().hift_k_attention_bwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout),
                                       _ptr(dqkv), _ptr(dsum), _st(stream)), "hift_k_attention_bwd")
+
+
+def k_linear_rope(M, N, K, a, b, out, bias, cs, seq, d_head, rope_cols, stream=None):
+    _check(lib().hift_k_linear_rope(M, N, K, _ptr(a), _ptr(b), _ptr(out), _ptr(bias), _ptr(cs), seq, d_head, rope_cols,
+                                    _st(stream)), "hift_k_linear_rope")
 
 
 def k_norm_fwd(dtype, kind, rows, cols, eps, x, gain, bias, y, stats, stream=None):

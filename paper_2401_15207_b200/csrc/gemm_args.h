@@ -14,6 +14,13 @@ struct GemmArgs {
   const void* bias;                    // operand type, [N]
   const float* residual; int64_t ldr;  // fp32 (the residual stream); only with out_f32
   bool out_f32;          // bf16 operands, fp32 output (weight gradients, residual stream)
+  // Optional rotary embedding applied to the output before it is stored (the q and k column
+  // blocks of a fused qkv projection): columns [0, rope_cols) are heads of rope_dh columns whose
+  // pair (j, j + rope_dh/2) is rotated by the angle of (row mod rope_seq, j).  rope_cs: fp32
+  // [rope_seq, rope_dh/2] cosines followed by [rope_seq, rope_dh/2] sines; nullptr = none.
+  const float* rope_cs = nullptr;
+  int rope_seq = 0, rope_dh = 0;
+  int64_t rope_cols = 0;
 };
 
 }  // namespace hift

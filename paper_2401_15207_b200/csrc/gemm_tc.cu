@@ -130,6 +130,120 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
   return (uint64_t)((saddr & 0x3FFFF) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// ------------------------------------------------------------------ epilogue pieces
+struct RopeArgs { const float* cs; int seq; int64_t cols; };   // head size 128; cs == nullptr: none
+
+// 32 consecutive outputs of row m starting at column n: bias, residual, conversion, store.
+// FULL: the caller knows that all 32 columns exist.
+template <bool OUT_F32, bool FULL>
+__device__ __forceinline__ void epi_store32(float (&f)[32], void* __restrict__ cptr, int64_t ldc, int m, int n, int N,
+                                            const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual,
+                                            int64_t ldr) {
+  if (FULL || n + 32 <= N) {
+    if (bias) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        const uint4 b4 = *reinterpret_cast<const uint4*>(bias + n + j);
+        const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b4);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const float2 bf = __bfloat1622float2(hb[t]);
+          f[j + 2 * t] += bf.x; f[j + 2 * t + 1] += bf.y;
+        }
+      }
+    }
+    if (OUT_F32) {
+      float* crow = reinterpret_cast<float*>(cptr) + (int64_t)m * ldc + n;
+      if (residual) {
+        const float* rrow = residual + (int64_t)m * ldr + n;
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 r = *reinterpret_cast<const float4*>(rrow + j);
+          f[j] += r.x; f[j + 1] += r.y; f[j + 2] += r.z; f[j + 3] += r.w;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 32; j += 4)
+        *reinterpret_cast<float4*>(crow + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+    } else {
+      __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * ldc + n;
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) {
+        uint4 o;
+        __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) ho[t] = __floats2bfloat162_rn(f[j + 2 * t], f[j + 2 * t + 1]);
+        *reinterpret_cast<uint4*>(crow + j) = o;
+      }
+    }
+  } else if (!FULL) {
+    for (int j = 0; j < 32 && n + j < N; ++j) {     // ragged right edge
+      float x = f[j];
+      if (bias) x += __bfloat162float(bias[n + j]);
+      if (OUT_F32) {
+        if (residual) x += residual[(int64_t)m * ldr + n + j];
+        reinterpret_cast<float*>(cptr)[(int64_t)m * ldc + n + j] = x;
+      } else {
+        reinterpret_cast<__nv_bfloat16*>(cptr)[(int64_t)m * ldc + n + j] = __float2bfloat16_rn(x);
+      }
+    }
+  }
+}
+
+// One row's share of an output tile: BN columns from tensor memory at taddr, starting at column n0.
+// With a rotary embedding (tiles are then whole heads of 128 columns) the chunk at head-local
+// column j < 64 is read together with its partner at j + 64, both get their bias, and the pair is
+// rotated in fp32 before the single rounding of the store.
+template <bool OUT_F32>
+__device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr, int64_t ldc,
+                                        const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
+                                        const RopeArgs& rope) {
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    if (n0 + c0 >= N) break;                       // uniform across the warp
+    const int n = n0 + c0;
+    if (!OUT_F32 && rope.cs != nullptr && n < rope.cols) {
+      if (c0 & 64) continue;                       // second halves go with their partners
+      uint32_t v1[32], v2[32];
+      tmem_ld32(taddr + c0, v1);
+      tmem_ld32(taddr + c0 + 64, v2);
+      if (m < M) {
+        float f1[32], f2[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { f1[j] = __uint_as_float(v1[j]); f2[j] = __uint_as_float(v2[j]); }
+        if (bias) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) { f1[j] += __bfloat162float(bias[n + j]); f2[j] += __bfloat162float(bias[n + 64 + j]); }
+        }
+        const float* cr = rope.cs + (int64_t)(m % rope.seq) * 64 + (c0 & 32);
+        const float* sr = cr + (int64_t)rope.seq * 64;
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 c4 = *reinterpret_cast<const float4*>(cr + j), s4 = *reinterpret_cast<const float4*>(sr + j);
+          const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const float x1 = f1[j + t], x2 = f2[j + t];
+            f1[j + t] = x1 * cc[t] - x2 * ss[t];
+            f2[j + t] = x1 * ss[t] + x2 * cc[t];
+          }
+        }
+        epi_store32<OUT_F32, true>(f1, cptr, ldc, m, n, N, nullptr, nullptr, 0);
+        epi_store32<OUT_F32, true>(f2, cptr, ldc, m, n + 64, N, nullptr, nullptr, 0);
+      }
+    } else {
+      uint32_t v[32];
+      tmem_ld32(taddr + c0, v);
+      if (m < M) {
+        float f[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+        epi_store32<OUT_F32, false>(f, cptr, ldc, m, n, N, bias, residual, ldr);
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ kernel
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -143,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-               int tiles_m, int num_tiles, TileRt tc) {
+               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope) {
   const int BN = tc.bn, S = tc.stages;
   const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
@@ -255,67 +369,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= N) break;                       // uniform across the warp
-        uint32_t v[32];
-        tmem_ld32(taddr + c0, v);
-        if (m < M) {
-          const int n = n0 + c0;
-          float f[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
-          if (n + 32 <= N) {
-            if (bias) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                const uint4 b4 = *reinterpret_cast<const uint4*>(bias + n + j);
-                const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b4);
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                  const float2 bf = __bfloat1622float2(hb[t]);
-                  f[j + 2 * t] += bf.x; f[j + 2 * t + 1] += bf.y;
-                }
-              }
-            }
-            if (OUT_F32) {
-              float* crow = reinterpret_cast<float*>(cptr) + (int64_t)m * ldc + n;
-              if (residual) {
-                const float* rrow = residual + (int64_t)m * ldr + n;
-#pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                  const float4 r = *reinterpret_cast<const float4*>(rrow + j);
-                  f[j] += r.x; f[j + 1] += r.y; f[j + 2] += r.z; f[j + 3] += r.w;
-                }
-              }
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(crow + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-            } else {
-              __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * ldc + n;
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 o;
-                __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-                for (int t = 0; t < 4; ++t) ho[t] = __floats2bfloat162_rn(f[j + 2 * t], f[j + 2 * t + 1]);
-                *reinterpret_cast<uint4*>(crow + j) = o;
-              }
-            }
-          } else {
-            for (int j = 0; j < 32 && n + j < N; ++j) {     // ragged right edge
-              float x = f[j];
-              if (bias) x += __bfloat162float(bias[n + j]);
-              if (OUT_F32) {
-                if (residual) x += residual[(int64_t)m * ldr + n + j];
-                reinterpret_cast<float*>(cptr)[(int64_t)m * ldc + n + j] = x;
-              } else {
-                reinterpret_cast<__nv_bfloat16*>(cptr)[(int64_t)m * ldc + n + j] = __float2bfloat16_rn(x);
-              }
-            }
-          }
-        }
-      }
+      epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand the accumulator back to the MMA thread
       tc_fence_before();
       __syncwarp();
@@ -381,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                 const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-                int tiles_m, int num_tiles) {
+                int tiles_m, int num_tiles, RopeArgs rope) {
   constexpr int S = kStages2;
   constexpr int BN = kBN2;
   extern __shared__ uint8_t smem_raw[];
@@ -494,67 +548,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= N) break;
-        uint32_t v[32];
-        tmem_ld32(taddr + c0, v);
-        if (m < M) {
-          const int n = n0 + c0;
-          float f[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
-          if (n + 32 <= N) {
-            if (bias) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                const uint4 b4 = *reinterpret_cast<const uint4*>(bias + n + j);
-                const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b4);
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                  const float2 bf = __bfloat1622float2(hb[t]);
-                  f[j + 2 * t] += bf.x; f[j + 2 * t + 1] += bf.y;
-                }
-              }
-            }
-            if (OUT_F32) {
-              float* crow = reinterpret_cast<float*>(cptr) + (int64_t)m * ldc + n;
-              if (residual) {
-                const float* rrow = residual + (int64_t)m * ldr + n;
-#pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                  const float4 r = *reinterpret_cast<const float4*>(rrow + j);
-                  f[j] += r.x; f[j + 1] += r.y; f[j + 2] += r.z; f[j + 3] += r.w;
-                }
-              }
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(crow + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-            } else {
-              __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * ldc + n;
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 o;
-                __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-                for (int t = 0; t < 4; ++t) ho[t] = __floats2bfloat162_rn(f[j + 2 * t], f[j + 2 * t + 1]);
-                *reinterpret_cast<uint4*>(crow + j) = o;
-              }
-            }
-          } else {
-            for (int j = 0; j < 32 && n + j < N; ++j) {
-              float x = f[j];
-              if (bias) x += __bfloat162float(bias[n + j]);
-              if (OUT_F32) {
-                if (residual) x += residual[(int64_t)m * ldr + n + j];
-                reinterpret_cast<float*>(cptr)[(int64_t)m * ldc + n + j] = x;
-              } else {
-                reinterpret_cast<__nv_bfloat16*>(cptr)[(int64_t)m * ldc + n + j] = __float2bfloat16_rn(x);
-              }
-            }
-          }
-        }
-      }
+      epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand this CTA's half of the accumulator back: the MMA thread counts 8 warps (4 per CTA)
       tc_fence_before();
       __syncwarp();
@@ -629,7 +623,8 @@ cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   const int num_tiles = tiles_m * tiles_n;
   const int grid = num_tiles < g_num_sms ? num_tiles : g_num_sms;
   gemm_tc_kernel<A_MN, B_MN, OUT_F32><<<grid, kThreads, kSmemBytes, st>>>(
-      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc);
+      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
+      RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols});
   return cudaGetLastError();
 }
 
@@ -651,7 +646,8 @@ cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
-                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles);
+                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles,
+                            RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols});
 }
 template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr2() {
@@ -722,6 +718,9 @@ static int classify(const GemmArgs& g) {
   if (g.bias && ((uintptr_t)g.bias & 15)) return 0;
   if (g.residual && (!g.out_f32 || ((uintptr_t)g.residual & 15) || g.ldr % 4)) return 0;
   if (form == 3 && (!g.out_f32 || g.bias || g.residual)) return 0;
+  // rotary embedding in the epilogue: forward form, bf16 output, whole heads of 128 columns per tile
+  if (g.rope_cs && (form != 1 || g.out_f32 || g.rope_dh != 128 || g.rope_seq < 1 || g.rope_cols % 128 || g.N % 128 ||
+                    g.rope_cols > g.N || (((uintptr_t)g.rope_cs) & 15))) return 0;
   return form;
 }
 bool gemm_tc_eligible(const GemmArgs& g) { return classify(g) != 0; }
@@ -740,6 +739,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
     double best = -1.0;
     const bool b_mn = form != 1;
     for (int cand = 256; cand >= 64; cand -= 32) {
+      if (g.rope_cs && cand % 128) continue;                               // tiles must hold whole heads
       const int tn = (g.N + cand - 1) / cand;
       const int tiles = tm * tn;
       const int rounds = (tiles + g_num_sms - 1) / g_num_sms;

@@ -404,6 +404,20 @@ void attn_bwd(hift_ctx* c, const void* qkv, const void* o, const float* lse, con
                               dout, dqkv, c->dsum));
   c->step_launches += attention_use_mma(c->mixed, c->dh) ? 2 : 1;   // dsum, dq, dkv or dq, dkv
 }
+// qkv projection of a rotary model: on the tensor-core path the rotation of the q and k column blocks
+// happens in the GEMM's epilogue (head size 128); otherwise the projection is followed by the
+// in-place kernel below.
+void rope(hift_ctx* c, void* qkv, float sign);
+void linear_fwd_qkv_rope(hift_ctx* c, int M, int d, const void* x, const void* w, void* qkv, const void* bias) {
+  GemmArgs g{M, 3 * d, d, x, d, 1, w, 1, d, qkv, 3 * d, bias, nullptr, 0, false};
+  g.rope_cs = c->rope_cs; g.rope_seq = c->S; g.rope_dh = c->dh; g.rope_cols = 2 * (int64_t)d;
+  if (c->mixed && gemm_tc_eligible(g)) {
+    LAUNCH(HIFT_K_GEMM_FWD, 2.0 * M * 3.0 * d * d, c->note(gemm_tc_launch(c->st, g)));
+    return;
+  }
+  linear_fwd(c, M, 3 * d, d, x, d, w, qkv, 3 * d, bias, nullptr, 0, false);
+  rope(c, qkv, 1.0f);
+}
 void rope(hift_ctx* c, void* qkv, float sign) {
   const size_t n = (size_t)c->T * c->H * (c->dh / 16);      // one thread per 8 pairs
   LAUNCH(HIFT_K_ELEMWISE, 64.0 * n * c->es,
@@ -458,8 +472,8 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     return;
   }
   norm_fwd(c, x_r, b.n1_g, b.n1_b, s[S_H1], nullptr, (float*)s[S_ST1]);
-  linear_fwd(c, T, 3 * d, d, s[S_H1], d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
-  if (c->m.arch == 2) rope(c, s[S_QKV], 1.0f);
+  if (c->m.arch == 2) linear_fwd_qkv_rope(c, T, d, s[S_H1], c->P(b.w_qkv), s[S_QKV], c->Pn(b.b_qkv));
+  else linear_fwd(c, T, 3 * d, d, s[S_H1], d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
   attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
   linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);
   norm_fwd(c, x2, b.n2_g, b.n2_b, s[S_H2], nullptr, (float*)s[S_ST2]);
@@ -1434,6 +1448,14 @@ hift_status hift_k_attention_bwd(int32_t dtype, int32_t B, int32_t S, int32_t H,
   if (!attention_head_ok(dh) || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
   launch_attention_bwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum);
   return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_linear_rope(int64_t M, int64_t N, int64_t K, const void* a, const void* b, void* out, const void* bias,
+                               const float* cs, int32_t seq, int32_t d_head, int64_t rope_cols, void* stream) {
+  if (M < 1 || N < 1 || K < 1 || !cs || seq < 1) return HIFT_ERR_CFG;
+  GemmArgs g{(int)M, (int)N, (int)K, a, K, 1, b, 1, K, out, N, bias, nullptr, 0, false};
+  g.rope_cs = cs; g.rope_seq = seq; g.rope_dh = d_head; g.rope_cols = rope_cols;
+  if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
+  return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,
                             const float* x, const void* gain, const void* bias, void* y, float* stats,

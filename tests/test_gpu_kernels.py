@@ -192,6 +192,38 @@ def test_attention_forward_backward(dtype, dh, causal):
         assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= tolb, i
 
 
+# ------------------------------------------------------------------ rotary embedding fused into the qkv projection
+def _rope_cs(S, dh, base=10000.0):
+    cos, sin = O.rope_tables(S, dh, base)
+    return np.concatenate([cos.reshape(-1), sin.reshape(-1)]).astype(np.float32), cos, sin
+
+
+@pytest.mark.parametrize("M,N,K,rope_cols,bias", [(300, 768, 256, 512, False), (256, 640, 192, 640, True)])
+def test_linear_with_rope_in_the_epilogue(M, N, K, rope_cols, bias):
+    """qkv projection whose q and k column blocks leave the GEMM already rotated (head size 128):
+    against linear -> RoPE of the oracle on the same bf16 operands.  Rows are positions r mod S with
+    S = 100, so the tile's 128 rows span a wrap of the position."""
+    import torch
+    from paper_2401_15207_b200 import k_linear_rope
+    dh, S = 128, 100
+    rng = np.random.default_rng(M + N)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) / np.sqrt(K)).astype(np.float32)
+    b = (0.5 * rng.standard_normal(N)).astype(np.float32)
+    cs, cos, sin = _rope_cs(S, dh)
+    out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    tb = _t(b, torch.bfloat16) if bias else None
+    k_linear_rope(M, N, K, _t(x, torch.bfloat16), _t(w, torch.bfloat16), out, tb, _t(cs), S, dh, rope_cols)
+    y = _bf(x) @ _bf(w).T + (_bf(b) if bias else 0.0)
+    pos = np.arange(M) % S
+    ref = y.copy()
+    heads = y[:, :rope_cols].reshape(1, M, rope_cols // dh, dh)      # rows play the sequence axis, each with its own angle
+    ref[:, :rope_cols] = O.rope_apply(heads, cos[pos], sin[pos]).reshape(M, rope_cols)
+    got = out.float().cpu().numpy()
+    assert rel_l2(got[:, :rope_cols], ref[:, :rope_cols]) <= 4e-3
+    assert rel_l2(got[:, rope_cols:], ref[:, rope_cols:]) <= 4e-3 or rope_cols == N
+
+
 # ------------------------------------------------------------------ norms
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("kind", [0, 1])
