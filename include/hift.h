@@ -260,6 +260,13 @@ hift_status hift_k_attention_bwd(int32_t dtype, int32_t batch, int32_t seq, int3
 hift_status hift_k_linear_rope(int64_t M, int64_t N, int64_t K, const void *a_dev, const void *b_dev, void *out_dev,
                                const void *bias_dev, const float *cs_dev, int32_t seq, int32_t d_head,
                                int64_t rope_cols, void *cuda_stream);
+/* SwiGLU blocks on the tensor-core path: the gate | up projection (w[2f, K]: f gate rows, then f up rows) and
+ * the activation are one kernel.  s_dev[M, f] = silu(gate) * up (bf16); gu_dev[M, 2f] receives the two
+ * pre-activations, or may be NULL when nothing will read them (blocks below the active group keep no
+ * activations).  HIFT_ERR_CFG when the fused kernel does not apply (f not a multiple of 128, M < 128,
+ * operands not 16-byte aligned). */
+hift_status hift_k_linear_swiglu(int64_t M, int64_t f, int64_t K, const void *a_dev, const void *b_dev, void *gu_dev,
+                                 void *s_dev, const void *bias_dev, void *cuda_stream);
 /* kind 0 LayerNorm (gain, bias), 1 RMSNorm (gain).  x is the fp32 residual stream in every
  * dtype; gain/bias/y have the operand type.  stats: fp32 [2*rows] (mean|rstd). */
 hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,

@@ -21,6 +21,10 @@ struct GemmArgs {
   const float* rope_cs = nullptr;
   int rope_seq = 0, rope_dh = 0;
   int64_t rope_cols = 0;
+  // Optional gated activation applied to the output (a fused gate | up projection, N = 2f): besides
+  // (or, with c == nullptr, instead of) c[m, 0..2f), the epilogue stores
+  //     swiglu_out[m, j] = silu(y[m, j]) * y[m, f + j],  j < f,   as bf16 with leading dimension f.
+  void* swiglu_out = nullptr;
 };
 
 }  // namespace hift

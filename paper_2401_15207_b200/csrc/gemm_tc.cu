@@ -244,6 +244,37 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
   }
 }
 
+// Gate | up tile: accumulator columns [0, 128) are gate columns nb .. nb+127, columns [128, 256) the
+// up columns of the same index.  Stores silu(gate) * up, and the two pre-activations themselves
+// when the backward pass will need them (cptr != nullptr).
+struct SwigluArgs { __nv_bfloat16* out; int half; };          // out == nullptr: none; half = f
+__device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int nb, void* __restrict__ cptr, int64_t ldc,
+                                               const __nv_bfloat16* __restrict__ bias, const SwigluArgs& sw) {
+#pragma unroll 1
+  for (int c0 = 0; c0 < 128; c0 += 32) {
+    uint32_t vg[32], vu[32];
+    tmem_ld32(taddr + c0, vg);
+    tmem_ld32(taddr + 128 + c0, vu);
+    if (m < M) {
+      float g[32], u[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) { g[j] = __uint_as_float(vg[j]); u[j] = __uint_as_float(vu[j]); }
+      if (bias) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { g[j] += __bfloat162float(bias[nb + c0 + j]); u[j] += __bfloat162float(bias[sw.half + nb + c0 + j]); }
+      }
+      float sgl[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) sgl[j] = g[j] / (1.0f + expf(-g[j])) * u[j];
+      if (cptr) {
+        epi_store32<false, true>(g, cptr, ldc, m, nb + c0, 0, nullptr, nullptr, 0);
+        epi_store32<false, true>(u, cptr, ldc, m, sw.half + nb + c0, 0, nullptr, nullptr, 0);
+      }
+      epi_store32<false, true>(sgl, sw.out, sw.half, m, nb + c0, 0, nullptr, nullptr, 0);
+    }
+  }
+}
+
 // ------------------------------------------------------------------ kernel
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -257,7 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope) {
+               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope, SwigluArgs swg) {
   const int BN = tc.bn, S = tc.stages;
   const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
@@ -311,6 +342,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
           if (B_MN) {
             for (int j = 0; j * 64 < BN; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
+          } else if (swg.out != nullptr) {
+            // gate | up: 128 rows of the gate block and the 128 rows of the same index in the up block
+            const int nb = (tile / tiles_m) * 128;
+            tma_load_2d(sb, &tmap_b, full_bar(s), k0, nb);
+            tma_load_2d(sb + 128 * 128, &tmap_b, full_bar(s), k0, swg.half + nb);
           } else {
             tma_load_2d(sb, &tmap_b, full_bar(s), k0, n0);
           }
@@ -369,7 +405,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-      epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
+      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
+      else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand the accumulator back to the MMA thread
       tc_fence_before();
       __syncwarp();
@@ -435,7 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                 const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-                int tiles_m, int num_tiles, RopeArgs rope) {
+                int tiles_m, int num_tiles, RopeArgs rope, SwigluArgs swg) {
   constexpr int S = kStages2;
   constexpr int BN = kBN2;
   extern __shared__ uint8_t smem_raw[];
@@ -480,7 +517,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
         const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM;
-        const int n0 = (tile / tiles_m) * BN + (int)rank * (BN / 2);
+        // this CTA's 128 columns of B; gate | up: the first CTA stages the gate rows, the second the up rows
+        const int n0 = (!B_MN && swg.out != nullptr) ? (tile / tiles_m) * 128 + (int)rank * swg.half
+                                                     : (tile / tiles_m) * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); ok = false; break; }
           const uint32_t sa = base + s * kStage2Bytes, sb = sa + kABytes;
@@ -548,7 +587,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-      epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
+      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
+      else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand this CTA's half of the accumulator back: the MMA thread counts 8 warps (4 per CTA)
       tc_fence_before();
       __syncwarp();
@@ -619,12 +659,12 @@ cudaError_t set_smem_attr() {
 template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& ta, const CUtensorMap& tb, int bn) {
   const TileRt tc = make_tile(bn, B_MN);
-  const int tiles_m = (g.M + BM - 1) / BM, tiles_n = (g.N + bn - 1) / bn;
+  const int tiles_m = (g.M + BM - 1) / BM, tiles_n = g.swiglu_out ? g.N / 256 : (g.N + bn - 1) / bn;
   const int num_tiles = tiles_m * tiles_n;
   const int grid = num_tiles < g_num_sms ? num_tiles : g_num_sms;
   gemm_tc_kernel<A_MN, B_MN, OUT_F32><<<grid, kThreads, kSmemBytes, st>>>(
       ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
-      RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols});
+      RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2});
   return cudaGetLastError();
 }
 
@@ -647,7 +687,7 @@ cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
                             (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles,
-                            RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols});
+                            RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2});
 }
 template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr2() {
@@ -719,6 +759,9 @@ static int classify(const GemmArgs& g) {
   if (g.residual && (!g.out_f32 || ((uintptr_t)g.residual & 15) || g.ldr % 4)) return 0;
   if (form == 3 && (!g.out_f32 || g.bias || g.residual)) return 0;
   // rotary embedding in the epilogue: forward form, bf16 output, whole heads of 128 columns per tile
+  // gated activation in the epilogue: forward form, bf16 output, f a multiple of 128 (a tile = 128 gate + 128 up columns)
+  if (g.swiglu_out && (form != 1 || g.out_f32 || g.residual || g.rope_cs || (g.N / 2) % 128 || g.N % 2 ||
+                       (((uintptr_t)g.swiglu_out) & 15))) return 0;
   if (g.rope_cs && (form != 1 || g.out_f32 || g.rope_dh != 128 || g.rope_seq < 1 || g.rope_cols % 128 || g.N % 128 ||
                     g.rope_cols > g.N || (((uintptr_t)g.rope_cs) & 15))) return 0;
   return form;
@@ -740,6 +783,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
     const bool b_mn = form != 1;
     for (int cand = 256; cand >= 64; cand -= 32) {
       if (g.rope_cs && cand % 128) continue;                               // tiles must hold whole heads
+      if (g.swiglu_out && cand != 256) continue;                           // 128 gate + 128 up columns
       const int tn = (g.N + cand - 1) / cand;
       const int tiles = tm * tn;
       const int rounds = (tiles + g_num_sms - 1) / g_num_sms;
@@ -774,7 +818,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
   // K-major operand: tensor [rows = M or N][inner = K]; MN-major operand: tensor [rows = K][inner = M or N]
   if (form == 3) ok = get_map(g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.sak, BK, &ta);
   else ok = get_map(g.a, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.sam, BM, &ta);
-  if (form == 1) ok = ok && get_map(g.b, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.sbn, (uint32_t)bn, &tb);
+  if (form == 1) ok = ok && get_map(g.b, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.sbn, (uint32_t)(g.swiglu_out ? 128 : bn), &tb);
   else ok = ok && get_map(g.b, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.sbk, BK, &tb);
   if (!ok) return cudaErrorInvalidValue;
   if (form == 1) return g.out_f32 ? launch_inst<false, false, true>(st, g, ta, tb, bn)

@@ -436,6 +436,20 @@ void act_fwd(hift_ctx* c, const void* a, void* u) {
            else gelu_fwd_kernel<float><<<grid_for(n / 8, 256), 256, 0, c->st>>>((const float*)a, (float*)u, n / 8));
   }
 }
+// Gate | up projection of a SwiGLU block followed by the activation: on the tensor-core path one GEMM
+// whose epilogue stores silu(gate) * up, and the pre-activations only if the backward pass will read
+// them (`keep`); otherwise the projection and the activation kernel.
+void linear_fwd_swiglu(hift_ctx* c, int M, int f, int K, const void* x, const void* w, void* gu, void* sact,
+                       const void* bias, bool keep) {
+  GemmArgs g{M, 2 * f, K, x, K, 1, w, 1, K, keep ? gu : nullptr, 2 * (int64_t)f, bias, nullptr, 0, false};
+  g.swiglu_out = sact;
+  if (c->mixed && gemm_tc_eligible(g)) {
+    LAUNCH(HIFT_K_GEMM_FWD, 2.0 * M * 2.0 * f * K, c->note(gemm_tc_launch(c->st, g)));
+    return;
+  }
+  linear_fwd(c, M, 2 * f, K, x, K, w, gu, 2 * f, bias, nullptr, 0, false);
+  act_fwd(c, gu, sact);
+}
 // GELU: du (in c->dbig, [T,f]) *= gelu'(a) in place.
 // SwiGLU: ds (in c->dsw, [T,f]) -> dgu in c->dbig [T,2f].
 void act_bwd(hift_ctx* c, const void* a) {
@@ -477,8 +491,13 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
   attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
   linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);
   norm_fwd(c, x2, b.n2_g, b.n2_b, s[S_H2], nullptr, (float*)s[S_ST2]);
-  linear_fwd(c, T, fa, d, s[S_H2], d, c->P(b.w_fc1), s[S_A], fa, c->Pn(b.b_fc1), nullptr, 0, false);
-  act_fwd(c, s[S_A], s[S_U]);
+  if (c->m.arch == 2) {
+    // blocks below the active group keep nothing: their pre-activations live in the scratch slot and are never read
+    linear_fwd_swiglu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
+  } else {
+    linear_fwd(c, T, fa, d, s[S_H2], d, c->P(b.w_fc1), s[S_A], fa, c->Pn(b.b_fc1), nullptr, 0, false);
+    act_fwd(c, s[S_A], s[S_U]);
+  }
   linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
 }
 
@@ -1435,6 +1454,14 @@ hift_status hift_k_linear(int32_t form, int32_t dtype, int32_t path, int64_t M, 
   }
   launch_gemm_simt((cudaStream_t)stream, dtype, g);
   return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_linear_swiglu(int64_t M, int64_t f, int64_t K, const void* a, const void* b, void* gu, void* sact,
+                                 const void* bias, void* stream) {
+  if (M < 1 || f < 1 || K < 1 || !sact) return HIFT_ERR_CFG;
+  GemmArgs g{(int)M, (int)(2 * f), (int)K, a, K, 1, b, 1, K, gu, 2 * f, bias, nullptr, 0, false};
+  g.swiglu_out = sact;
+  if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
+  return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_k_attention_fwd(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
                                  const void* qkv, void* o, float* lse, void* stream) {

@@ -224,6 +224,26 @@ def test_linear_with_rope_in_the_epilogue(M, N, K, rope_cols, bias):
     assert rel_l2(got[:, rope_cols:], ref[:, rope_cols:]) <= 4e-3 or rope_cols == N
 
 
+@pytest.mark.parametrize("M,f,K,keep,bias", [(300, 384, 256, True, False), (256, 128, 192, False, True), (520, 1152, 128, True, True)])
+def test_gate_up_projection_with_swiglu_in_the_epilogue(M, f, K, keep, bias):
+    """Gate | up GEMM whose epilogue stores silu(gate) * up (and the pre-activations when kept):
+    against linear -> swiglu of the oracle on the same bf16 operands."""
+    import torch
+    from paper_2401_15207_b200 import k_linear_swiglu
+    rng = np.random.default_rng(M + f)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((2 * f, K)) * (2.0 / np.sqrt(K))).astype(np.float32)
+    b = (0.5 * rng.standard_normal(2 * f)).astype(np.float32)
+    gu = torch.full((M, 2 * f), 7.0, dtype=torch.bfloat16, device="cuda") if keep else None
+    s = torch.empty((M, f), dtype=torch.bfloat16, device="cuda")
+    k_linear_swiglu(M, f, K, _t(x, torch.bfloat16), _t(w, torch.bfloat16), gu, s, _t(b, torch.bfloat16) if bias else None)
+    y = _bf(x) @ _bf(w).T + (_bf(b) if bias else 0.0)
+    s_ref = O.swiglu_fwd(y[:, :f], y[:, f:])
+    assert rel_l2(s.float().cpu().numpy(), s_ref) <= 4e-3
+    if keep:
+        assert rel_l2(gu.float().cpu().numpy(), y) <= 4e-3
+
+
 # ------------------------------------------------------------------ norms
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("kind", [0, 1])
