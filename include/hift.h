@@ -267,6 +267,12 @@ hift_status hift_k_linear_rope(int64_t M, int64_t N, int64_t K, const void *a_de
  * operands not 16-byte aligned). */
 hift_status hift_k_linear_swiglu(int64_t M, int64_t f, int64_t K, const void *a_dev, const void *b_dev, void *gu_dev,
                                  void *s_dev, const void *bias_dev, void *cuda_stream);
+/* ... and its backward: dgu_dev[M, 2f] = swiglu_bwd(dy[M,N] w[N,f]; gu_dev[M, 2f]), i.e. the dX product of the
+ * down projection (w is the down matrix [N = d_model, f]) with the activation's backward applied in
+ * its epilogue: d gate in columns [0, f), d up in [f, 2f).  HIFT_ERR_CFG when the fused kernel does not
+ * apply (f not a multiple of 32, M < 128, operands not 16-byte aligned). */
+hift_status hift_k_linear_dx_swiglu_bwd(int64_t M, int64_t N, int64_t f, const void *dy_dev, const void *w_dev,
+                                        const void *gu_dev, void *dgu_dev, void *cuda_stream);
 /* kind 0 LayerNorm (gain, bias), 1 RMSNorm (gain).  x is the fp32 residual stream in every
  * dtype; gain/bias/y have the operand type.  stats: fp32 [2*rows] (mean|rstd). */
 hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,

@@ -25,6 +25,12 @@ struct GemmArgs {
   // (or, with c == nullptr, instead of) c[m, 0..2f), the epilogue stores
   //     swiglu_out[m, j] = silu(y[m, j]) * y[m, f + j],  j < f,   as bf16 with leading dimension f.
   void* swiglu_out = nullptr;
+  // Optional backward of that activation applied to the output of the down projection's dX product
+  // (y = ds[M, f], N = f): instead of ds the epilogue stores, into c[M, 2f] (ldc = 2f),
+  //     c[m, j]     = ds * up * sig * (1 + gate * (1 - sig)),   sig = sigmoid(gate)
+  //     c[m, f + j] = ds * gate * sig
+  // with gate = swiglu_bwd_gu[m, j], up = swiglu_bwd_gu[m, f + j] (the saved pre-activations, bf16).
+  const void* swiglu_bwd_gu = nullptr;
 };
 
 }  // namespace hift

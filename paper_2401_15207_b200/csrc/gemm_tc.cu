@@ -198,6 +198,36 @@ template <bool OUT_F32>
 __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr, int64_t ldc,
                                         const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
                                         const RopeArgs& rope) {
+  // (the tensor-memory loads are warp-collective: take this path only if every row of the warp exists)
+  if (OUT_F32 && residual != nullptr && n0 + BN <= N && __all_sync(0xffffffffu, m < M)) {
+    // Output into the residual stream: the residual chunk of the next 32 columns is fetched while
+    // this chunk is read from tensor memory, added and stored, so that only the first load's latency
+    // is exposed per tile.
+    const float* rrow = residual + (int64_t)m * ldr + n0;
+    float4 rn[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) rn[j] = *reinterpret_cast<const float4*>(rrow + 4 * j);
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      float4 rc[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) rc[j] = rn[j];
+      if (c0 + 32 < BN) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) rn[j] = *reinterpret_cast<const float4*>(rrow + c0 + 32 + 4 * j);
+      }
+      uint32_t v[32];
+      tmem_ld32(taddr + c0, v);
+      float f[32];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        f[4 * j] = __uint_as_float(v[4 * j]) + rc[j].x; f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + rc[j].y;
+        f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + rc[j].z; f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + rc[j].w;
+      }
+      epi_store32<OUT_F32, true>(f, cptr, ldc, m, n0 + c0, N, bias, nullptr, 0);
+    }
+    return;
+  }
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 32) {
     if (n0 + c0 >= N) break;                       // uniform across the warp
@@ -275,6 +305,58 @@ __device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int
   }
 }
 
+// Backward of the gated activation on a tile of ds = dy W_down (columns n0 .. of f): reads the saved
+// gate / up pre-activations of the same columns (the next chunk's while this one is worked on) and
+// stores d gate and d up into the [M, 2f] gradient of the gate | up projection.
+struct SwigluBwdArgs { const __nv_bfloat16* gu; };            // gu == nullptr: none
+__device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
+                                                   const SwigluBwdArgs& sb) {
+  const bool rowok = m < M;
+  const __nv_bfloat16* grow = sb.gu + (int64_t)m * (2 * (int64_t)N) + n0;
+  __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * (2 * (int64_t)N) + n0;
+  uint4 gn[4], un[4];
+  if (rowok && n0 < N) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { gn[j] = *reinterpret_cast<const uint4*>(grow + 8 * j); un[j] = *reinterpret_cast<const uint4*>(grow + N + 8 * j); }
+  }
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    if (n0 + c0 >= N) break;                       // uniform across the warp; N is a multiple of 32
+    uint4 gc[4], uc[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { gc[j] = gn[j]; uc[j] = un[j]; }
+    if (rowok && c0 + 32 < BN && n0 + c0 + 32 < N) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        gn[j] = *reinterpret_cast<const uint4*>(grow + c0 + 32 + 8 * j);
+        un[j] = *reinterpret_cast<const uint4*>(grow + N + c0 + 32 + 8 * j);
+      }
+    }
+    uint32_t v[32];
+    tmem_ld32(taddr + c0, v);
+    if (rowok) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat162* hg = reinterpret_cast<const __nv_bfloat162*>(&gc[j]);
+        const __nv_bfloat162* hu = reinterpret_cast<const __nv_bfloat162*>(&uc[j]);
+        uint4 og, ou;
+        __nv_bfloat162* pg = reinterpret_cast<__nv_bfloat162*>(&og);
+        __nv_bfloat162* pu = reinterpret_cast<__nv_bfloat162*>(&ou);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const float2 g2 = __bfloat1622float2(hg[t]), u2 = __bfloat1622float2(hu[t]);
+          const float d0 = __uint_as_float(v[8 * j + 2 * t]), d1 = __uint_as_float(v[8 * j + 2 * t + 1]);
+          const float s0 = 1.0f / (1.0f + expf(-g2.x)), s1 = 1.0f / (1.0f + expf(-g2.y));
+          pg[t] = __floats2bfloat162_rn(d0 * u2.x * s0 * (1.0f + g2.x * (1.0f - s0)), d1 * u2.y * s1 * (1.0f + g2.y * (1.0f - s1)));
+          pu[t] = __floats2bfloat162_rn(d0 * g2.x * s0, d1 * g2.y * s1);
+        }
+        *reinterpret_cast<uint4*>(orow + c0 + 8 * j) = og;
+        *reinterpret_cast<uint4*>(orow + N + c0 + 8 * j) = ou;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ kernel
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -288,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope, SwigluArgs swg) {
+               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb) {
   const int BN = tc.bn, S = tc.stages;
   const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
@@ -406,6 +488,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
       if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
+      else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb);
       else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand the accumulator back to the MMA thread
       tc_fence_before();
@@ -472,7 +555,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                 const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-                int tiles_m, int num_tiles, RopeArgs rope, SwigluArgs swg) {
+                int tiles_m, int num_tiles, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb) {
   constexpr int S = kStages2;
   constexpr int BN = kBN2;
   extern __shared__ uint8_t smem_raw[];
@@ -588,6 +671,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
       if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
+      else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb);
       else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand this CTA's half of the accumulator back: the MMA thread counts 8 warps (4 per CTA)
       tc_fence_before();
@@ -664,7 +748,8 @@ cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   const int grid = num_tiles < g_num_sms ? num_tiles : g_num_sms;
   gemm_tc_kernel<A_MN, B_MN, OUT_F32><<<grid, kThreads, kSmemBytes, st>>>(
       ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
-      RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2});
+      RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
+      SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu});
   return cudaGetLastError();
 }
 
@@ -687,7 +772,8 @@ cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
                             (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles,
-                            RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2});
+                            RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
+                            SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu});
 }
 template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr2() {
@@ -762,6 +848,9 @@ static int classify(const GemmArgs& g) {
   // gated activation in the epilogue: forward form, bf16 output, f a multiple of 128 (a tile = 128 gate + 128 up columns)
   if (g.swiglu_out && (form != 1 || g.out_f32 || g.residual || g.rope_cs || (g.N / 2) % 128 || g.N % 2 ||
                        (((uintptr_t)g.swiglu_out) & 15))) return 0;
+  // backward of the gated activation in the epilogue: dX form, bf16 output of 2N columns
+  if (g.swiglu_bwd_gu && (form != 2 || g.out_f32 || g.bias || g.residual || g.N % 32 || g.ldc != 2 * (int64_t)g.N ||
+                          (((uintptr_t)g.swiglu_bwd_gu) & 15))) return 0;
   if (g.rope_cs && (form != 1 || g.out_f32 || g.rope_dh != 128 || g.rope_seq < 1 || g.rope_cols % 128 || g.N % 128 ||
                     g.rope_cols > g.N || (((uintptr_t)g.rope_cs) & 15))) return 0;
   return form;

@@ -528,9 +528,19 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
     if (need_dx) linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dxa, d, c->dxb, d, true);
     return;
   }
-  linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);                 // du / ds
+  // SwiGLU on the tensor-core path: the dX product of the down projection stores d gate | d up directly
+  bool act_done = false;
+  if (c->m.arch == 2 && c->mixed) {
+    GemmArgs g{T, f, d, c->dxa_a, d, 1, c->P(b.w_fc2), f, 1, c->dbig, 2 * (int64_t)f, nullptr, nullptr, 0, false};
+    g.swiglu_bwd_gu = s[S_A];
+    if (gemm_tc_eligible(g)) {
+      LAUNCH(HIFT_K_GEMM_DX, 2.0 * T * (double)f * d, c->note(gemm_tc_launch(c->st, g)));
+      act_done = true;
+    }
+  }
+  if (!act_done) linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);  // du / ds
   if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxa, true, T, d, d, b.b_fc2); }
-  act_bwd(c, s[S_A]);                                                                               // da in dbig [T,fa]
+  if (!act_done) act_bwd(c, s[S_A]);                                                                // da in dbig [T,fa]
   linear_dx(c, T, fa, d, c->dbig, fa, c->P(b.w_fc1), c->dt1, d, nullptr, 0, false);                 // dh2
   if (on) { linear_dw(c, T, fa, d, c->dbig, fa, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, fa, fa, b.b_fc1); }
   if (on) norm_bwd_params(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, b.n2_b);
@@ -1460,6 +1470,14 @@ hift_status hift_k_linear_swiglu(int64_t M, int64_t f, int64_t K, const void* a,
   if (M < 1 || f < 1 || K < 1 || !sact) return HIFT_ERR_CFG;
   GemmArgs g{(int)M, (int)(2 * f), (int)K, a, K, 1, b, 1, K, gu, 2 * f, bias, nullptr, 0, false};
   g.swiglu_out = sact;
+  if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
+  return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_linear_dx_swiglu_bwd(int64_t M, int64_t N, int64_t f, const void* dy, const void* w, const void* gu,
+                                        void* dgu, void* stream) {
+  if (M < 1 || N < 1 || f < 1 || !gu || !dgu) return HIFT_ERR_CFG;
+  GemmArgs g{(int)M, (int)f, (int)N, dy, N, 1, w, f, 1, dgu, 2 * f, nullptr, nullptr, 0, false};
+  g.swiglu_bwd_gu = gu;
   if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
   return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }

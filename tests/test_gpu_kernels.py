@@ -244,6 +244,25 @@ def test_gate_up_projection_with_swiglu_in_the_epilogue(M, f, K, keep, bias):
         assert rel_l2(gu.float().cpu().numpy(), y) <= 4e-3
 
 
+@pytest.mark.parametrize("M,N,f", [(300, 256, 416), (256, 128, 1024), (200, 192, 96)])
+def test_down_projection_dx_with_swiglu_backward_in_the_epilogue(M, N, f):
+    """ds = dy W_down and the activation's backward in one kernel: against linear dX -> swiglu_bwd of the
+    oracle on the same bf16 operands (f spans several tiles with a ragged last one)."""
+    import torch
+    from paper_2401_15207_b200 import k_linear_dx_swiglu_bwd
+    rng = np.random.default_rng(M + f)
+    dy = rng.standard_normal((M, N)).astype(np.float32)
+    w = (rng.standard_normal((N, f)) / np.sqrt(N)).astype(np.float32)
+    gu = (1.5 * rng.standard_normal((M, 2 * f))).astype(np.float32)
+    dgu = torch.empty((M, 2 * f), dtype=torch.bfloat16, device="cuda")
+    k_linear_dx_swiglu_bwd(M, N, f, _t(dy, torch.bfloat16), _t(w, torch.bfloat16), _t(gu, torch.bfloat16), dgu)
+    ds = _bf(dy) @ _bf(w)
+    dg_ref, du_ref = O.swiglu_bwd(ds, _bf(gu)[:, :f], _bf(gu)[:, f:])
+    got = dgu.float().cpu().numpy()
+    assert rel_l2(got[:, :f], dg_ref) <= 4e-3
+    assert rel_l2(got[:, f:], du_ref) <= 4e-3
+
+
 # ------------------------------------------------------------------ norms
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("kind", [0, 1])
