@@ -9,8 +9,9 @@ group-local optimizer, optimizer-state paging.  Default workload: the LLaMA-7B-s
 master, one block per group plus embedding and head groups, bottom2up, AdamW with inactive-group
 state in pinned host memory).  Prints ONE JSON line on rank 0.
 
-N > 1 runs N independent replicas (one process per GPU, no data-path collective): the step has
-no exchange inside it on one GPU, and the data-parallel variant is not built yet.
+N > 1 runs N independent replicas by default (one process per GPU, no data-path collective: the
+step has no exchange inside it on one GPU); --parallel dp trains one model data-parallel with an
+all-reduce of the active group's gradient between the backward pass and the update.
 """
 from __future__ import annotations
 
@@ -388,7 +389,7 @@ def run_sweep_optimizer(args):
     from paper_2401_15207_b200 import opt_step
     peaks = measured_peaks()
     rows = []
-    for kind, name, bpe in ((0, "adamw", 30), (1, "adagrad", 22), (2, "sgdm", 22)):
+    for kind, name, bpe in ((0, "adamw", 30), (1, "adagrad", 22), (2, "sgdm", 22)):      # fp32-master form of hift_opt_step
         for lg in range(20, 31):
             n = 1 << lg
             # rotate over enough buffer sets to exceed L2 (126 MB) between visits
