@@ -39,6 +39,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // descriptor of a K-major tile with rows of 64 elements (one span), 128-byte swizzle
@@ -181,34 +186,43 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       bool ready = ok && mbar_wait(s_full0 + 8 * st, (j >> 1) & 1);
       if (ok && !ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
       tc_fence_after();
-      ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
+      ok = __all_sync(0xffffffffu, ready);
       if (!ok) break;
-      // scores of this row: 128 columns
+      // scores of this row: 128 columns, in log2 units
       float sc[kAttBK];
 #pragma unroll
       for (int c0 = 0; c0 < kAttBK; c0 += 32) {
         uint32_t v[32];
         tmem_ld32(tmem_base + lane_off + (uint32_t)(st * 128 + c0), v);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sc[c0 + i] = __uint_as_float(v[i]);
+        for (int i = 0; i < 32; ++i) sc[c0 + i] = __uint_as_float(v[i]) * sl2;
+      }
+      // masking only where the block touches the diagonal or the end of the sequence (uniform per CTA)
+      if ((causal && j * kAttBK + kAttBK - 1 > q0) || (j + 1) * kAttBK > S) {
+#pragma unroll
+        for (int i = 0; i < kAttBK; ++i) {
+          const int key = j * kAttBK + i;
+          if (key >= S || (causal && key > qrow)) sc[i] = -INFINITY;
+        }
       }
       float mx = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < kAttBK; ++i) {
-        const int key = j * kAttBK + i;
-        float x = sc[i] * sl2;
-        if (key >= S || (causal && key > qrow)) x = -INFINITY;
-        sc[i] = x;
-        mx = fmaxf(mx, x);
+      for (int i = 0; i < kAttBK; ++i) mx = fmaxf(mx, sc[i]);
+      // Lazy reference maximum: m moves (and O is rescaled) only when some row of the warp has grown by
+      // more than 2^8 over it; until then probabilities up to 256 are summed against the old reference,
+      // which changes nothing in the final O / l and lse = m + log2(l).
+      const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
+      float corr = 1.0f;
+      if (grow) {
+        const float mnew = fmaxf(m, mx);
+        corr = (mnew == -INFINITY) ? 1.0f : ex2_approx(m - mnew);      // m = -inf: corr = 0, nothing accumulated yet
+        m = mnew;
       }
-      const float mnew = fmaxf(m, mx);
-      const float muse = (mnew == -INFINITY) ? 0.f : mnew;
-      const float corr = exp2f(m - muse);
+      const float muse = (m == -INFINITY) ? 0.f : m;
       float sum = 0.f;
 #pragma unroll
-      for (int i = 0; i < kAttBK; ++i) { sc[i] = exp2f(sc[i] - muse); sum += sc[i]; }
+      for (int i = 0; i < kAttBK; ++i) { sc[i] = ex2_approx(sc[i] - muse); sum += sc[i]; }
       l = l * corr + sum;
-      m = mnew;
       // the previous P V product must be finished before P is overwritten and O is rescaled
       if (j > 0) {
         ready = mbar_wait(o_done, (j - 1) & 1);
@@ -227,7 +241,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
         const int span = ch >> 3, c = ch & 7;
         *reinterpret_cast<uint4*>(p_gen + span * SPAN_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = pk;
       }
-      if (j > 0) {
+      if (j > 0 && grow) {                              // warp-uniform
 #pragma unroll 1
         for (int c0 = 0; c0 < DH; c0 += 32) {
           uint32_t v[32];
