@@ -2,29 +2,31 @@
 // Included into gemm_tc.cu (inside its unnamed namespace) so that it shares the PTX wrappers,
 // the bounded mbarrier waits, the time-out flag and the tensor-map cache.
 //
-// One CTA = one (batch, head) and 128 query rows; key blocks of 128.
-//   warp 0    : TMA producer (Q once; K and V blocks through two 2-deep rings)
-//   warp 1    : MMA issuer and tensor-memory owner
-//                 S_j = Q K_j^T        (M 128 x N 128, k = d_h)      -> TMEM columns [0,128) / [128,256)
-//                 O  += P_j V_j        (M 128 x N d_h, k = 128 keys) -> TMEM columns [256, 256 + d_h)
-//   warps 2-5 : softmax, one thread per query row (= one tensor-memory lane): read S_j, mask,
+// Work item = one (batch, head) and 128 query rows; key blocks of 128.  The kernel is persistent:
+// a CTA walks a list of items, those with the most key blocks first, and the next item's Q tile,
+// first scores and first P V products overlap the normalisation and store of the current item
+// (two Q buffers, two score buffers, two output accumulators).
+//   warp 0    : TMA producer (Q per item; K and V blocks through two 2-deep rings)
+//   warp 1    : issues S_j = Q K_j^T   (M 128 x N 128, k = d_h)      -> TMEM columns [0,128) / [128,256); owns the tensor memory
+//   warp 2    : issues O += P_j V_j    (M 128 x N d_h, k = 128 keys) -> TMEM columns [256,384) / [384,512) by item parity
+//   warps 3-6 : softmax, one thread per query row (= one tensor-memory lane): read S_j, mask,
 //               running max / sum, write P_j as bf16 into a 128-byte-swizzled shared tile (the A
-//               operand of the second product), rescale O in tensor memory when the maximum moved,
-//               and at the end normalise and store O and the log-sum-exp.
+//               operand of the second product), rescale O in tensor memory when the reference
+//               maximum moved, and at the end normalise and store O and the log-sum-exp.
 // Q and K are K-major operands (d_h contiguous), V is an N-major operand (B(k = key, n = e) =
 // V[key][e]): all three are read straight out of qkv[T, 3d] by one tensor map, nothing is copied
 // or transposed.  Rows of a tile that lie beyond this batch entry's sequence hold the next
 // entry's (finite) values or TMA zero fill; their scores are masked, their probabilities are 0.
 #pragma once
 
-constexpr int kAttThreads = 192;
+constexpr int kAttThreads = 224;
 constexpr int kAttBQ = 128, kAttBK = 128;
 
 template <int DH> struct AttnTcCfg {
   static constexpr int kSpans = DH / 64;                       // 64-column swizzle spans per row
   static constexpr int kTileBytes = 128 * DH * 2;              // one Q / K / V tile
   static constexpr int kPBytes = 128 * kAttBK * 2;             // P tile: 128 rows x 128 keys
-  static constexpr int kSmem = 5 * kTileBytes + kPBytes + 1024 + 256;
+  static constexpr int kSmem = 6 * kTileBytes + kPBytes + 1024 + 256;      // Q x 2, K x 2, V x 2, P
 };
 
 __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]) {
@@ -59,40 +61,60 @@ __device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr, uint32_t box_byt
 template <int DH>
 __global__ void __launch_bounds__(kAttThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* __restrict__ o,
-                   float* __restrict__ lse, int S, int H, int causal, float scale) {
+                   float* __restrict__ lse, int B, int S, int H, int causal, float scale) {
   typedef AttnTcCfg<DH> Cfg;
   constexpr int SP = Cfg::kSpans;
   constexpr int SPAN_BYTES = 128 * 128;                 // 128 rows x 64 elements x 2 bytes
   extern __shared__ uint8_t smem_raw[];
-  const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kAttBQ;
   const int d = H * DH;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = base;
-  const uint32_t sK = sQ + Cfg::kTileBytes;             // two stages
+  const uint32_t sQ = base;                             // two buffers (item parity)
+  const uint32_t sK = sQ + 2 * Cfg::kTileBytes;         // two stages
   const uint32_t sV = sK + 2 * Cfg::kTileBytes;         // two stages
   const uint32_t sP = sV + 2 * Cfg::kTileBytes;
   const uint32_t bar = sP + Cfg::kPBytes;
-  const uint32_t q_full = bar, k_full0 = bar + 8, k_empty0 = bar + 24, v_full0 = bar + 40, v_empty0 = bar + 56,
-                 s_full0 = bar + 72, p_ready = bar + 88, o_done = bar + 96, tmem_slot = bar + 104;
+  auto q_full = [&](int i) { return bar + 8u * i; };
+  auto q_empty = [&](int i) { return bar + 16u + 8u * i; };
+  auto k_full = [&](int i) { return bar + 32u + 8u * i; };
+  auto k_empty = [&](int i) { return bar + 48u + 8u * i; };
+  auto v_full = [&](int i) { return bar + 64u + 8u * i; };
+  auto v_empty = [&](int i) { return bar + 80u + 8u * i; };
+  auto s_full = [&](int i) { return bar + 96u + 8u * i; };
+  auto s_free = [&](int i) { return bar + 112u + 8u * i; };
+  auto o_done = [&](int i) { return bar + 128u + 8u * i; };
+  auto o_free = [&](int i) { return bar + 144u + 8u * i; };
+  const uint32_t p_ready = bar + 160u, p_free = bar + 168u, tmem_slot = bar + 176u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
   uint8_t* p_gen = gen + (sP - base);
 
-  const int kv_len = causal ? min(S, q0 + kAttBQ) : S;
-  const int nblk = (kv_len + kAttBK - 1) / kAttBK;
+  // work items, heaviest first; every role walks the same list and counts key blocks (g)
+  const int nqb = (S + kAttBQ - 1) / kAttBQ, nbh = B * H, nitems = nqb * nbh;
+  struct Item { int b, h, q0, nblk; };
+  auto item_of = [&](int idx) {
+    Item it;
+    const int rank = idx / nbh, bh = idx - rank * nbh;
+    it.b = bh / H;
+    it.h = bh - it.b * H;
+    it.q0 = (causal ? nqb - 1 - rank : rank) * kAttBQ;
+    const int kv_len = causal ? min(S, it.q0 + kAttBQ) : S;
+    it.nblk = (kv_len + kAttBK - 1) / kAttBK;
+    return it;
+  };
   const bool poisoned = g_tc_error != 0;
 
   if (threadIdx.x == 0) {
-    mbar_init(q_full, 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(k_full0 + 8 * i, 1); mbar_init(k_empty0 + 8 * i, 1);
-      mbar_init(v_full0 + 8 * i, 1); mbar_init(v_empty0 + 8 * i, 1);
-      mbar_init(s_full0 + 8 * i, 1);
+      mbar_init(q_full(i), 1); mbar_init(q_empty(i), 1);
+      mbar_init(k_full(i), 1); mbar_init(k_empty(i), 1);
+      mbar_init(v_full(i), 1); mbar_init(v_empty(i), 1);
+      mbar_init(s_full(i), 1); mbar_init(s_free(i), 4);
+      mbar_init(o_done(i), 1); mbar_init(o_free(i), 4);
     }
     mbar_init(p_ready, 4);                              // one arrival per softmax warp
-    mbar_init(o_done, 1);
+    mbar_init(p_free, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -103,174 +125,217 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
-  const uint32_t tO = tmem_base + 256;
-
-  const int row_g0 = b * S;                             // first row of this batch entry in qkv
-  const int colQ = h * DH, colK = d + h * DH, colV = 2 * d + h * DH;
 
   if (warp == 0) {
     // ---------------- TMA producer
     if (lane == 0 && !poisoned) {
-      mbar_expect_tx(q_full, Cfg::kTileBytes);
-#pragma unroll
-      for (int sp = 0; sp < SP; ++sp) tma_load_2d(sQ + sp * SPAN_BYTES, &tmap_qkv, q_full, colQ + sp * 64, row_g0 + q0);
+      int g = 0, n = 0;
       bool ok = true;
-      for (int j = 0; j < nblk && ok; ++j) {
-        const int st = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        const int krow = row_g0 + j * kAttBK;
-        if (!mbar_wait(k_empty0 + 8 * st, ph ^ 1)) { atomicCAS(&g_tc_error, 0, 4); ok = false; break; }
-        mbar_expect_tx(k_full0 + 8 * st, Cfg::kTileBytes);
+      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+        const Item it = item_of(idx);
+        const int row_g0 = it.b * S;                    // first row of this batch entry in qkv
+        const int colQ = it.h * DH, colK = d + it.h * DH, colV = 2 * d + it.h * DH;
+        const int qi = n & 1;
+        if (!mbar_wait(q_empty(qi), (uint32_t)(((n >> 1) & 1) ^ 1))) { atomicCAS(&g_tc_error, 0, 4); break; }
+        mbar_expect_tx(q_full(qi), Cfg::kTileBytes);
 #pragma unroll
-        for (int sp = 0; sp < SP; ++sp)
-          tma_load_2d(sK + st * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, k_full0 + 8 * st, colK + sp * 64, krow);
-        if (!mbar_wait(v_empty0 + 8 * st, ph ^ 1)) { atomicCAS(&g_tc_error, 0, 4); ok = false; break; }
-        mbar_expect_tx(v_full0 + 8 * st, Cfg::kTileBytes);
+        for (int sp = 0; sp < SP; ++sp) tma_load_2d(sQ + qi * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, q_full(qi), colQ + sp * 64, row_g0 + it.q0);
+        for (int j = 0; j < it.nblk; ++j, ++g) {
+          const int st = g & 1;
+          const uint32_t ph = (uint32_t)((g >> 1) & 1);
+          const int krow = row_g0 + j * kAttBK;
+          if (!mbar_wait(k_empty(st), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 4); ok = false; break; }
+          mbar_expect_tx(k_full(st), Cfg::kTileBytes);
 #pragma unroll
-        for (int sp = 0; sp < SP; ++sp)
-          tma_load_2d(sV + st * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, v_full0 + 8 * st, colV + sp * 64, krow);
+          for (int sp = 0; sp < SP; ++sp)
+            tma_load_2d(sK + st * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, k_full(st), colK + sp * 64, krow);
+          if (!mbar_wait(v_empty(st), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 4); ok = false; break; }
+          mbar_expect_tx(v_full(st), Cfg::kTileBytes);
+#pragma unroll
+          for (int sp = 0; sp < SP; ++sp)
+            tma_load_2d(sV + st * Cfg::kTileBytes + sp * SPAN_BYTES, &tmap_qkv, v_full(st), colV + sp * 64, krow);
+        }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer
+    // ---------------- MMA issuer 1: scores.  A = Q (K-major), B = K (K-major), N = 128; runs ahead of the
+    //                  softmax warps as far as the two score buffers allow, into the next item too
     if (lane == 0 && !poisoned) {
-      // S: A = Q (K-major), B = K (K-major), N = 128.  O: A = P (K-major), B = V (N-major), N = DH.
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAttBK >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      int g = 0, n = 0;
+      bool ok = true;
+      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+        const Item it = item_of(idx);
+        const int qi = n & 1;
+        if (!mbar_wait(q_full(qi), (uint32_t)((n >> 1) & 1))) { atomicCAS(&g_tc_error, 0, 5); break; }
+        const uint64_t dQ = desc_kmajor(sQ + qi * Cfg::kTileBytes);
+        for (int j = 0; j < it.nblk; ++j, ++g) {
+          const int st = g & 1;
+          const uint32_t ph = (uint32_t)((g >> 1) & 1);
+          if (!mbar_wait(k_full(st), ph) || !mbar_wait(s_free(st), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 5); ok = false; break; }
+          tc_fence_after();
+          const uint64_t dK = desc_kmajor(sK + st * Cfg::kTileBytes);
+          const uint32_t ts = tmem_base + (uint32_t)(st * 128);
+#pragma unroll
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint64_t off = (uint64_t)(((kk / 4) * SPAN_BYTES + (kk % 4) * 32) >> 4);
+            tc_mma(ts, dQ + off, dK + off, idesc_s, kk > 0 ? 1u : 0u);
+          }
+          tc_commit(s_full(st));
+          tc_commit(k_empty(st));
+        }
+        if (ok) tc_commit(q_empty(qi));
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------- MMA issuer 2: O += P V.  A = P (K-major), B = V (N-major), N = DH
+    if (lane == 0 && !poisoned) {
       const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-      bool ok = mbar_wait(q_full, 0);
-      if (!ok) atomicCAS(&g_tc_error, 0, 5);
-      auto issue_s = [&](int j) -> bool {
-        const int st = j & 1;
-        if (!mbar_wait(k_full0 + 8 * st, (j >> 1) & 1)) { atomicCAS(&g_tc_error, 0, 5); return false; }
-        tc_fence_after();
-        const uint32_t ts = tmem_base + (uint32_t)(st * 128);
+      int g = 0, n = 0;
+      bool ok = true;
+      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+        const Item it = item_of(idx);
+        const uint32_t tO = tmem_base + 256u + (uint32_t)((n & 1) * 128);
+        for (int j = 0; j < it.nblk; ++j, ++g) {
+          const int st = g & 1;
+          if (!mbar_wait(p_ready, (uint32_t)(g & 1)) || !mbar_wait(v_full(st), (uint32_t)((g >> 1) & 1))) {
+            atomicCAS(&g_tc_error, 0, 5); ok = false; break;
+          }
+          // the first product of an item overwrites its accumulator: the item two before must have been stored
+          if (j == 0 && n >= 2 && !mbar_wait(o_free(n & 1), (uint32_t)(((n >> 1) - 1) & 1))) { atomicCAS(&g_tc_error, 0, 5); ok = false; break; }
+          tc_fence_after();
+          const uint64_t dP = desc_kmajor(sP), dV = desc_nmajor(sV + st * Cfg::kTileBytes, SPAN_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (uint32_t)((kk / 4) * SPAN_BYTES + (kk % 4) * 32);
-          tc_mma(ts, desc_kmajor(sQ + off), desc_kmajor(sK + st * Cfg::kTileBytes + off), idesc_s, kk > 0 ? 1u : 0u);
+          for (int kk = 0; kk < kAttBK / 16; ++kk) {
+            // P: 128 keys = two 64-key spans, 32 bytes per 16 keys inside a span; V: 16 key rows of 128 bytes
+            tc_mma(tO, dP + (uint64_t)(((kk / 4) * SPAN_BYTES + (kk % 4) * 32) >> 4), dV + (uint64_t)((kk * 16 * 128) >> 4), idesc_o,
+                   (j > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit(p_free);
+          tc_commit(v_empty(st));
         }
-        tc_commit(s_full0 + 8 * st);
-        tc_commit(k_empty0 + 8 * st);
-        return true;
-      };
-      if (ok) ok = issue_s(0);
-      if (ok && nblk > 1) ok = issue_s(1);
-      for (int j = 0; j < nblk && ok; ++j) {
-        const int st = j & 1;
-        if (!mbar_wait(p_ready, j & 1)) { atomicCAS(&g_tc_error, 0, 5); ok = false; break; }
-        if (!mbar_wait(v_full0 + 8 * st, (j >> 1) & 1)) { atomicCAS(&g_tc_error, 0, 5); ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < kAttBK / 16; ++kk) {
-          // P: 128 keys = two 64-key spans, 32 bytes per 16 keys inside a span; V: 16 key rows of 128 bytes
-          const uint64_t da = desc_kmajor(sP + (uint32_t)((kk / 4) * SPAN_BYTES + (kk % 4) * 32));
-          const uint64_t db = desc_nmajor(sV + st * Cfg::kTileBytes + (uint32_t)(kk * 16 * 128), SPAN_BYTES);
-          tc_mma(tO, da, db, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
-        }
-        tc_commit(o_done);
-        tc_commit(v_empty0 + 8 * st);
-        if (j + 2 < nblk) ok = issue_s(j + 2);
+        if (ok) tc_commit(o_done(n & 1));
       }
     }
   } else {
     // ---------------- softmax and epilogue: thread = query row = tensor-memory lane
     const int q = warp & 3;
     const int r = q * 32 + lane;                        // row inside the tile
-    const int qrow = q0 + r;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const float sl2 = scale * 1.4426950408889634f;
-    float m = -INFINITY, l = 0.f;
     bool ok = !poisoned;
-    for (int j = 0; j < nblk; ++j) {
-      const int st = j & 1;
-      bool ready = ok && mbar_wait(s_full0 + 8 * st, (j >> 1) & 1);
-      if (ok && !ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
-      tc_fence_after();
-      ok = __all_sync(0xffffffffu, ready);
-      if (!ok) break;
-      // scores of this row: 128 columns, in log2 units
-      float sc[kAttBK];
-#pragma unroll
-      for (int c0 = 0; c0 < kAttBK; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + lane_off + (uint32_t)(st * 128 + c0), v);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) sc[c0 + i] = __uint_as_float(v[i]) * sl2;
-      }
-      // masking only where the block touches the diagonal or the end of the sequence (uniform per CTA)
-      if ((causal && j * kAttBK + kAttBK - 1 > q0) || (j + 1) * kAttBK > S) {
-#pragma unroll
-        for (int i = 0; i < kAttBK; ++i) {
-          const int key = j * kAttBK + i;
-          if (key >= S || (causal && key > qrow)) sc[i] = -INFINITY;
-        }
-      }
-      float mx = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < kAttBK; ++i) mx = fmaxf(mx, sc[i]);
-      // Lazy reference maximum: m moves (and O is rescaled) only when some row of the warp has grown by
-      // more than 2^8 over it; until then probabilities up to 256 are summed against the old reference,
-      // which changes nothing in the final O / l and lse = m + log2(l).
-      const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
-      float corr = 1.0f;
-      if (grow) {
-        const float mnew = fmaxf(m, mx);
-        corr = (mnew == -INFINITY) ? 1.0f : ex2_approx(m - mnew);      // m = -inf: corr = 0, nothing accumulated yet
-        m = mnew;
-      }
-      const float muse = (m == -INFINITY) ? 0.f : m;
-      float sum = 0.f;
-#pragma unroll
-      for (int i = 0; i < kAttBK; ++i) { sc[i] = ex2_approx(sc[i] - muse); sum += sc[i]; }
-      l = l * corr + sum;
-      // the previous P V product must be finished before P is overwritten and O is rescaled
-      if (j > 0) {
-        ready = mbar_wait(o_done, (j - 1) & 1);
+    int g = 0, n = 0;
+    for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      const Item it = item_of(idx);
+      const int q0 = it.q0, qrow = q0 + r, row_g0 = it.b * S;
+      const uint32_t tO = tmem_base + 256u + (uint32_t)((n & 1) * 128);
+      float m = -INFINITY, l = 0.f;
+      for (int j = 0; j < it.nblk; ++j, ++g) {
+        const int st = g & 1;
+        bool ready = mbar_wait(s_full(st), (uint32_t)((g >> 1) & 1));
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
         tc_fence_after();
         ok = __all_sync(0xffffffffu, ready);
         if (!ok) break;
-      }
-      // P row -> shared memory, bf16, K-major with the 128-byte swizzle the MMA descriptor expects
+        // scores of this row: 128 columns (raw; the scale is folded into the exponent below)
+        float sc[kAttBK];
 #pragma unroll
-      for (int ch = 0; ch < kAttBK / 8; ++ch) {
-        uint4 pk;
-        __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-        for (int t = 0; t < 4; ++t) hp[t] = __floats2bfloat162_rn(sc[ch * 8 + 2 * t], sc[ch * 8 + 2 * t + 1]);
-        const int span = ch >> 3, c = ch & 7;
-        *reinterpret_cast<uint4*>(p_gen + span * SPAN_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = pk;
-      }
-      if (j > 0 && grow) {                              // warp-uniform
-#pragma unroll 1
-        for (int c0 = 0; c0 < DH; c0 += 32) {
+        for (int c0 = 0; c0 < kAttBK; c0 += 32) {
           uint32_t v[32];
-          tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+          tmem_ld32(tmem_base + lane_off + (uint32_t)(st * 128 + c0), v);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
-          tmem_st32(tO + lane_off + (uint32_t)c0, v);
+          for (int i = 0; i < 32; ++i) sc[c0 + i] = __uint_as_float(v[i]);
         }
-        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_free(st));         // the tensor core may overwrite this score buffer
+        // masking only where the block touches the diagonal or the end of the sequence (uniform per CTA)
+        if ((causal && j * kAttBK + kAttBK - 1 > q0) || (j + 1) * kAttBK > S) {
+#pragma unroll
+          for (int i = 0; i < kAttBK; ++i) {
+            const int key = j * kAttBK + i;
+            if (key >= S || (causal && key > qrow)) sc[i] = -INFINITY;
+          }
+        }
+        // four independent chains each for the maximum and the sum: one warp per scheduler has nobody
+        // else to hide a serial chain's latency behind
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < kAttBK; i += 4) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], sc[i + e]);
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;     // in log2 units (scale > 0)
+        // Lazy reference maximum: m moves (and O is rescaled) only when some row of the warp has grown by
+        // more than 2^8 over it; until then probabilities up to 256 are summed against the old reference,
+        // which changes nothing in the final O / l and lse = m + log2(l).
+        const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
+        float corr = 1.0f;
+        if (grow) {
+          const float mnew = fmaxf(m, mx);
+          corr = (mnew == -INFINITY) ? 1.0f : ex2_approx(m - mnew);    // m = -inf: corr = 0, nothing accumulated yet
+          m = mnew;
+        }
+        const float nmuse = (m == -INFINITY) ? 0.f : -m;
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < kAttBK; i += 4) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { sc[i + e] = ex2_approx(fmaf(sc[i + e], sl2, nmuse)); sum4[e] += sc[i + e]; }
+        }
+        l = l * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+        // the previous P V product must be finished before P is overwritten and O is rescaled
+        ready = mbar_wait(p_free, (uint32_t)((g & 1) ^ 1));
+        if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
+        tc_fence_after();
+        ok = __all_sync(0xffffffffu, ready);
+        if (!ok) break;
+        // P row -> shared memory, bf16, K-major with the 128-byte swizzle the MMA descriptor expects
+#pragma unroll
+        for (int ch = 0; ch < kAttBK / 8; ++ch) {
+          uint4 pk;
+          __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+          for (int t = 0; t < 4; ++t) hp[t] = __floats2bfloat162_rn(sc[ch * 8 + 2 * t], sc[ch * 8 + 2 * t + 1]);
+          const int span = ch >> 3, c = ch & 7;
+          *reinterpret_cast<uint4*>(p_gen + span * SPAN_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = pk;
+        }
+        if (j > 0 && grow) {                            // warp-uniform
+#pragma unroll 1
+          for (int c0 = 0; c0 < DH; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
+            tmem_st32(tO + lane_off + (uint32_t)c0, v);
+          }
+          tmem_st_wait();
+        }
+        fence_async_smem();                             // P is read by the tensor core (async proxy)
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_ready);
       }
-      fence_async_smem();                               // P is read by the tensor core (async proxy)
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(p_ready);
-    }
-    // last product done -> normalise and store
-    if (ok && nblk > 0) {
-      const bool ready = mbar_wait(o_done, (nblk - 1) & 1);
-      if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
-      tc_fence_after();
-      ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
-    }
-    if (ok) {
+      if (!ok) break;
+      // last product of the item done -> normalise and store
+      {
+        const bool ready = mbar_wait(o_done(n & 1), (uint32_t)((n >> 1) & 1));
+        if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
+        tc_fence_after();
+        ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
+        if (!ok) break;
+      }
       const float inv = 1.0f / l;
-      __nv_bfloat16* orow = o + ((int64_t)(row_g0 + qrow)) * d + (int64_t)h * DH;
+      __nv_bfloat16* orow = o + ((int64_t)(row_g0 + qrow)) * d + (int64_t)it.h * DH;
 #pragma unroll 1
       for (int c0 = 0; c0 < DH; c0 += 32) {
         uint32_t v[32];
         tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+        if (c0 + 32 >= DH) {                            // everything read: the accumulator may be reused
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(o_free(n & 1));
+        }
         if (qrow < S) {
 #pragma unroll
           for (int i = 0; i < 32; i += 8) {
@@ -283,7 +348,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
           }
         }
       }
-      if (qrow < S) lse[((int64_t)b * H + h) * S + qrow] = (m + log2f(l)) * 0.6931471805599453f;
+      if (qrow < S) lse[((int64_t)it.b * H + it.h) * S + qrow] = (m + log2f(l)) * 0.6931471805599453f;
     }
   }
   tc_fence_before();

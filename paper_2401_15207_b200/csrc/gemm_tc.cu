@@ -937,12 +937,13 @@ cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int
   CUtensorMap tm;
   const uint64_t d3 = 3ull * H * dh;
   if (!get_map(qkv, d3, (uint64_t)B * S, d3, 128, &tm)) return cudaErrorInvalidValue;
-  dim3 grid((S + kAttBQ - 1) / kAttBQ, H, B);
+  const int nitems = ((S + kAttBQ - 1) / kAttBQ) * H * B;
+  const int grid = nitems < g_num_sms ? nitems : g_num_sms;          // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)dh);
   if (dh == 64)
-    attn_fwd_tc_kernel<64><<<grid, kAttThreads, AttnTcCfg<64>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, S, H, causal, scale);
+    attn_fwd_tc_kernel<64><<<grid, kAttThreads, AttnTcCfg<64>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
   else
-    attn_fwd_tc_kernel<128><<<grid, kAttThreads, AttnTcCfg<128>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, S, H, causal, scale);
+    attn_fwd_tc_kernel<128><<<grid, kAttThreads, AttnTcCfg<128>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
   return cudaGetLastError();
 }
 
