@@ -83,12 +83,15 @@ typedef struct {
                                 4 Adafactor (factored second moment: rows + cols floats of state per
                                 matrix; `lr` caps the relative step, `eps` is its epsilon_1;
                                 epsilon_2 = 1e-3, clipping d = 1, decay exponent -0.8, no momentum) */
-  int32_t sched;             /* 0 constant, 1 linear decay lr*(1 - cycle/total)    */
-  int32_t total_cycles;      /* horizon of the linear schedule                     */
+  int32_t sched;             /* 0 constant, 1 linear: warm-up, then decay to 0     */
+  int32_t total_cycles;      /* horizon C of the linear schedule, in cycles        */
   int32_t offload_state;     /* 1: inactive groups' master+state in pinned host    */
   int32_t prefetch_groups;   /* 0: one state slot, H2D issued after the forward
                                    (the paper's order); 1: two slots, H2D issued at
                                    step start and overlapped with the previous D2H  */
+  int32_t warmup_cycles;     /* W (sched 1; the warm-up the paper's hyper-parameter tables list, counted in
+                                cycles because the rate moves once per cycle): cycle c < W runs at
+                                lr*c/W, cycle c >= W at lr*max(0, (C-c)/(C-W)); 0 = none             */
   double lr, beta1, beta2, eps, weight_decay, momentum;
 } hift_opt_cfg;
 

@@ -128,12 +128,23 @@ def queue_walk(n_units: int, m: int, order: int, steps: int) -> List[List[int]]:
     return out
 
 
-def lr_for_cycle(lr0: float, sched: int, cycle: int, total_cycles: int) -> float:
+def lr_for_cycle(lr0: float, sched: int, cycle: int, total_cycles: int, warmup_cycles: int = 0) -> float:
     """Delayed learning rate: a function of the completed-cycle count only, so
-    it is constant inside a cycle.  const -> lr0; linear -> lr0*max(0, 1-c/C)."""
+    it is constant inside a cycle.  const -> lr0; linear -> lr0*max(0, 1-c/C).
+
+    The paper's hyper-parameter tables list a warm-up ratio next to the linear
+    schedule (Appendix, hyper-parameter tables: warmup in {0, 0.02, 0.06}).  Read
+    as the usual linear warm-up of that schedule, counted in cycles because the
+    schedule only moves once per cycle: with W = warmup_cycles,
+        c <  W : lr0 * c / W                     (the first cycle runs at 0)
+        c >= W : lr0 * max(0, (C - c) / (C - W))
+    which is the formula above when W = 0."""
     if sched == 0:
         return lr0
-    return lr0 * max(0.0, 1.0 - cycle / float(total_cycles))
+    W, C = int(warmup_cycles), int(total_cycles)
+    if cycle < W:
+        return lr0 * cycle / float(W)
+    return lr0 * max(0.0, (C - cycle) / float(max(1, C - W)))
 
 
 # --------------------------------------------------------------------------
@@ -633,7 +644,7 @@ class HiFTOracle:
 
     def current_lr(self) -> float:
         o = self.ocfg
-        return lr_for_cycle(o.lr, o.sched, self.t // self.k, o.total_cycles)
+        return lr_for_cycle(o.lr, o.sched, self.t // self.k, o.total_cycles, getattr(o, "warmup_cycles", 0))
 
     def model_params(self) -> Dict[str, np.ndarray]:
         """What the forward pass reads: the master itself (fp32 configs) or its

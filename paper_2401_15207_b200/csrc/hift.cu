@@ -181,7 +181,9 @@ std::vector<int> make_order(int k, int order, uint64_t seed) {
 }
 double lr_for_cycle(const hift_opt_cfg& oc, int64_t cycle) {
   if (oc.sched == 0) return oc.lr;
-  const double fct = 1.0 - (double)cycle / (double)oc.total_cycles;
+  const int64_t W = oc.warmup_cycles, C = oc.total_cycles;
+  if (cycle < W) return oc.lr * (double)cycle / (double)W;
+  const double fct = (double)(C - cycle) / (double)(C - W > 1 ? C - W : 1);
   return oc.lr * (fct > 0.0 ? fct : 0.0);
 }
 
@@ -910,7 +912,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if ((int64_t)m->batch * m->seq > 8192) return HIFT_ERR_CFG;
   if (gc->layers_per_group < 1 || gc->order < 0 || gc->order > 2) return HIFT_ERR_CFG;
   if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
-  if (oc->sched == 1 && oc->total_cycles < 1) return HIFT_ERR_CFG;
+  if (oc->sched == 1 && (oc->total_cycles < 1 || oc->warmup_cycles < 0 || oc->warmup_cycles >= oc->total_cycles)) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
   hift_ctx* c = new hift_ctx();

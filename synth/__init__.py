@@ -89,6 +89,7 @@ class OptCfg:
     total_cycles: int = 1
     offload_state: int = 1
     prefetch_groups: int = 0
+    warmup_cycles: int = 0
 
 
 # --------------------------------------------------------------------------

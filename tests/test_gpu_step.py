@@ -305,3 +305,30 @@ def test_paged_and_resident_state_give_identical_bits(kind):
     finally:
         for h in ctxs:
             h.close()
+
+
+def test_warmup_then_decay_moves_once_per_cycle():
+    """Linear schedule with a warm-up counted in cycles: the learning rate the library reports is
+    bit-identical to the oracle's in every step, and the first cycle, run at rate 0, leaves every
+    parameter untouched under SGD (so the reported rate is the one used)."""
+    from paper_2401_15207_b200 import HiFT
+    import torch
+    cfg = mini(2, synth.DTYPE_FP32)
+    oc = synth.OptCfg(kind=synth.OPT_SGD, lr=1e-2, sched=synth.SCHED_LINEAR, total_cycles=4, warmup_cycles=2, offload_state=0)
+    gc = synth.GroupCfg(layers_per_group=2)
+    h = HiFT(cfg, gc, oc)
+    p0 = synth.init_params(cfg, 3, perturb=0.05)
+    h.set_params(p0)
+    k = h.num_groups()
+    lrs = []
+    for t in range(4 * k):
+        lrs.append(h.current_lr())
+        tok, lab = synth.batch_for(cfg, 9, t, "zipf")
+        h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
+        if t == k - 1:
+            for name in h.tensor_names():
+                assert np.array_equal(np.asarray(h.get_param(name)).reshape(-1), np.asarray(p0[name], dtype=np.float32).reshape(-1)), name
+    h.close()
+    from oracle import hift_oracle as O
+    assert lrs == [O.lr_for_cycle(oc.lr, oc.sched, t // k, oc.total_cycles, oc.warmup_cycles) for t in range(4 * k)]
+    assert lrs == pytest.approx([0.0] * k + [0.5e-2] * k + [1e-2] * k + [0.5e-2] * k, rel=1e-15, abs=0.0)

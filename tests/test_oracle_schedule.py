@@ -109,6 +109,23 @@ def test_delayed_lr_constant_within_cycle():
     assert O.lr_for_cycle(lr0, 1, 7, 3) == 0.0
 
 
+def test_linear_schedule_with_warmup_in_cycles():
+    # warm-up of the paper's hyper-parameter tables, counted in cycles (the rate moves once per cycle):
+    # values by hand for C = 10, W = 2; W = 0 is the plain linear decay; the ramp meets the decay at lr0
+    lr0, C, W = 1e-3, 10, 2
+    got = [O.lr_for_cycle(lr0, 1, c, C, W) for c in range(12)]
+    want = [0.0, 0.5e-3, 1e-3, 0.875e-3, 0.75e-3, 0.625e-3, 0.5e-3, 0.375e-3, 0.25e-3, 0.125e-3, 0.0, 0.0]
+    assert got == pytest.approx(want, rel=1e-15, abs=0.0)
+    assert max(got) == lr0 and got.index(lr0) == W
+    for c in range(12):
+        assert O.lr_for_cycle(lr0, 1, c, C, 0) == O.lr_for_cycle(lr0, 1, c, C)
+        assert O.lr_for_cycle(lr0, 0, c, C, W) == lr0                      # the constant schedule ignores it
+    # still a function of the cycle only: constant inside a cycle of k steps
+    k = 6
+    orc_lrs = [O.lr_for_cycle(lr0, 1, t // k, C, W) for t in range(k * C)]
+    assert all(len(set(orc_lrs[c * k:(c + 1) * k])) == 1 for c in range(C))
+
+
 def test_memory_model_against_paper():
     g = _golden()
     z1 = g["zeta1_7b_fp32_G"]
