@@ -276,6 +276,15 @@ hift_status hift_k_linear_swiglu(int64_t M, int64_t f, int64_t K, const void *a_
  * apply (f not a multiple of 32, M < 128, operands not 16-byte aligned). */
 hift_status hift_k_linear_dx_swiglu_bwd(int64_t M, int64_t N, int64_t f, const void *dy_dev, const void *w_dev,
                                         const void *gu_dev, void *dgu_dev, void *cuda_stream);
+/* GELU blocks (the GPT-2- and RoBERTa-shaped configurations), same two fusions:
+ *   hift_k_linear_gelu       : pre_dev[M,N] = x[M,K] w[N,K]^T + bias (may be NULL when not needed), act_dev[M,N] = gelu(pre)
+ *   hift_k_linear_dx_gelu_bwd: da_dev[M,f] = (dy[M,N] w[N,f]) * gelu'(pre_dev[M,f])
+ * exact (erf) GELU; HIFT_ERR_CFG when the fused kernel does not apply (output width not a multiple of 32, M < 128,
+ * operands not 16-byte aligned). */
+hift_status hift_k_linear_gelu(int64_t M, int64_t N, int64_t K, const void *a_dev, const void *b_dev, void *pre_dev,
+                               void *act_dev, const void *bias_dev, void *cuda_stream);
+hift_status hift_k_linear_dx_gelu_bwd(int64_t M, int64_t N, int64_t f, const void *dy_dev, const void *w_dev,
+                                      const void *pre_dev, void *da_dev, void *cuda_stream);
 /* kind 0 LayerNorm (gain, bias), 1 RMSNorm (gain).  x is the fp32 residual stream in every
  * dtype; gain/bias/y have the operand type.  stats: fp32 [2*rows] (mean|rstd). */
 hift_status hift_k_norm_fwd(int32_t dtype, int32_t kind, int64_t rows, int64_t cols, double eps,

@@ -99,6 +99,8 @@ def _prototypes():
         "hift_k_linear_rope": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, i64, vp]),
         "hift_k_linear_swiglu": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_linear_dx_swiglu_bwd": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp]),
+        "hift_k_linear_gelu": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, vp]),
+        "hift_k_linear_dx_gelu_bwd": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp]),
         "hift_k_norm_fwd": (C.c_int, [i32, i32, i64, i64, f64, vp, vp, vp, vp, vp, vp]),
         "hift_k_norm_bwd": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "hift_k_norm_bwd_static": (C.c_int, [i32, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
@@ -374,6 +376,16 @@ def k_linear_swiglu(M, f, K, a, b, gu, s, bias=None, stream=None):
 def k_linear_dx_swiglu_bwd(M, N, f, dy, w, gu, dgu, stream=None):
     _check(lib().hift_k_linear_dx_swiglu_bwd(M, N, f, _ptr(dy), _ptr(w), _ptr(gu), _ptr(dgu), _st(stream)),
            "hift_k_linear_dx_swiglu_bwd")
+
+
+def k_linear_gelu(M, N, K, a, b, pre, act, bias=None, stream=None):
+    _check(lib().hift_k_linear_gelu(M, N, K, _ptr(a), _ptr(b), _ptr(pre), _ptr(act), _ptr(bias), _st(stream)),
+           "hift_k_linear_gelu")
+
+
+def k_linear_dx_gelu_bwd(M, N, f, dy, w, pre, da, stream=None):
+    _check(lib().hift_k_linear_dx_gelu_bwd(M, N, f, _ptr(dy), _ptr(w), _ptr(pre), _ptr(da), _st(stream)),
+           "hift_k_linear_dx_gelu_bwd")
 
 
 def k_norm_fwd(dtype, kind, rows, cols, eps, x, gain, bias, y, stats, stream=None):

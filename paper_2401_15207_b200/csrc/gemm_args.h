@@ -31,6 +31,12 @@ struct GemmArgs {
   //     c[m, f + j] = ds * gate * sig
   // with gate = swiglu_bwd_gu[m, j], up = swiglu_bwd_gu[m, f + j] (the saved pre-activations, bf16).
   const void* swiglu_bwd_gu = nullptr;
+  // GELU (exact, erf) blocks: the same two fusions for the plain feed-forward.
+  //   gelu_out (forward form): besides (or, with c == nullptr, instead of) the pre-activation y in c, the
+  //   epilogue stores gelu_out[m, n] = gelu(y[m, n]) as bf16 with leading dimension N.
+  //   gelu_bwd_a (dX form): the output is multiplied by gelu'(a[m, n]), a = the saved pre-activation (bf16, ld N).
+  void* gelu_out = nullptr;
+  const void* gelu_bwd_a = nullptr;
 };
 
 }  // namespace hift

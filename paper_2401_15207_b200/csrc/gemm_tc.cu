@@ -357,6 +357,75 @@ __device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m
   }
 }
 
+// GELU (exact) in the epilogue.  Forward: stores gelu(y) (and y itself when cptr != nullptr).  Backward: the
+// dX product's output times gelu'(a), a = saved pre-activation of the same element, prefetched a chunk ahead.
+struct GeluArgs { __nv_bfloat16* out; const __nv_bfloat16* bwd_a; };      // both nullptr: none
+__device__ __forceinline__ float gelu_tc(float a) { return 0.5f * a * (1.0f + erff(a * 0.70710678118654752440f)); }
+__device__ __forceinline__ float gelu_grad_tc(float a) {
+  const float cdf = 0.5f * (1.0f + erff(a * 0.70710678118654752440f));
+  return cdf + a * expf(-0.5f * a * a) * 0.39894228040143267794f;
+}
+__device__ __forceinline__ void epi_row_gelu_fwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
+                                                 int64_t ldc, const __nv_bfloat16* __restrict__ bias, const GeluArgs& ge) {
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    if (n0 + c0 >= N) break;                       // uniform across the warp; N is a multiple of 32
+    uint32_t v[32];
+    tmem_ld32(taddr + c0, v);
+    if (m < M) {
+      const int n = n0 + c0;
+      float f[32], u[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+      if (bias) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) f[j] += __bfloat162float(bias[n + j]);
+      }
+#pragma unroll
+      for (int j = 0; j < 32; ++j) u[j] = gelu_tc(f[j]);
+      if (cptr) epi_store32<false, true>(f, cptr, ldc, m, n, N, nullptr, nullptr, 0);
+      epi_store32<false, true>(u, ge.out, N, m, n, N, nullptr, nullptr, 0);
+    }
+  }
+}
+__device__ __forceinline__ void epi_row_gelu_bwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
+                                                 int64_t ldc, const GeluArgs& ge) {
+  const bool rowok = m < M;
+  const __nv_bfloat16* arow = ge.bwd_a + (int64_t)m * N + n0;
+  uint4 an[4];
+  if (rowok && n0 < N) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) an[j] = *reinterpret_cast<const uint4*>(arow + 8 * j);
+  }
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    if (n0 + c0 >= N) break;
+    uint4 ac[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) ac[j] = an[j];
+    if (rowok && c0 + 32 < BN && n0 + c0 + 32 < N) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) an[j] = *reinterpret_cast<const uint4*>(arow + c0 + 32 + 8 * j);
+    }
+    uint32_t v[32];
+    tmem_ld32(taddr + c0, v);
+    if (rowok) {
+      float f[32];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&ac[j]);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const float2 a2 = __bfloat1622float2(ha[t]);
+          f[8 * j + 2 * t] = __uint_as_float(v[8 * j + 2 * t]) * gelu_grad_tc(a2.x);
+          f[8 * j + 2 * t + 1] = __uint_as_float(v[8 * j + 2 * t + 1]) * gelu_grad_tc(a2.y);
+        }
+      }
+      epi_store32<false, true>(f, cptr, ldc, m, n0 + c0, N, nullptr, nullptr, 0);
+    }
+  }
+}
+
 // ------------------------------------------------------------------ kernel
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -370,7 +439,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb) {
+               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb, GeluArgs ge) {
   const int BN = tc.bn, S = tc.stages;
   const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
@@ -489,6 +558,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
       if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
       else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb);
+      else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge);
+      else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge);
       else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand the accumulator back to the MMA thread
       tc_fence_before();
@@ -555,7 +626,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                 const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-                int tiles_m, int num_tiles, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb) {
+                int tiles_m, int num_tiles, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb, GeluArgs ge) {
   constexpr int S = kStages2;
   constexpr int BN = kBN2;
   extern __shared__ uint8_t smem_raw[];
@@ -672,6 +743,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
       if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
       else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb);
+      else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge);
+      else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge);
       else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
       // hand this CTA's half of the accumulator back: the MMA thread counts 8 warps (4 per CTA)
       tc_fence_before();
@@ -749,7 +822,7 @@ cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   gemm_tc_kernel<A_MN, B_MN, OUT_F32><<<grid, kThreads, kSmemBytes, st>>>(
       ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
       RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
-      SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu});
+      SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu}, GeluArgs{(__nv_bfloat16*)g.gelu_out, (const __nv_bfloat16*)g.gelu_bwd_a});
   return cudaGetLastError();
 }
 
@@ -773,7 +846,8 @@ cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
                             (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles,
                             RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
-                            SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu});
+                            SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu},
+                            GeluArgs{(__nv_bfloat16*)g.gelu_out, (const __nv_bfloat16*)g.gelu_bwd_a});
 }
 template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr2() {
@@ -851,6 +925,9 @@ static int classify(const GemmArgs& g) {
   // backward of the gated activation in the epilogue: dX form, bf16 output of 2N columns
   if (g.swiglu_bwd_gu && (form != 2 || g.out_f32 || g.bias || g.residual || g.N % 32 || g.ldc != 2 * (int64_t)g.N ||
                           (((uintptr_t)g.swiglu_bwd_gu) & 15))) return 0;
+  // GELU in the epilogue: forward form (gelu_out) or dX form (gelu_bwd_a), bf16 output, N a multiple of 32
+  if (g.gelu_out && (form != 1 || g.out_f32 || g.residual || g.rope_cs || g.swiglu_out || g.N % 32 || (((uintptr_t)g.gelu_out) & 15))) return 0;
+  if (g.gelu_bwd_a && (form != 2 || g.out_f32 || g.bias || g.residual || g.swiglu_bwd_gu || g.N % 32 || (((uintptr_t)g.gelu_bwd_a) & 15))) return 0;
   if (g.rope_cs && (form != 1 || g.out_f32 || g.rope_dh != 128 || g.rope_seq < 1 || g.rope_cols % 128 || g.N % 128 ||
                     g.rope_cols > g.N || (((uintptr_t)g.rope_cs) & 15))) return 0;
   return form;

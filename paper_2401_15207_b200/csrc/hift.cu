@@ -452,6 +452,30 @@ void linear_fwd_swiglu(hift_ctx* c, int M, int f, int K, const void* x, const vo
   linear_fwd(c, M, 2 * f, K, x, K, w, gu, 2 * f, bias, nullptr, 0, false);
   act_fwd(c, gu, sact);
 }
+// Up projection of a GELU block followed by the activation, and the down projection's dX product followed by
+// the activation's backward: one GEMM each on the tensor-core path (the activation runs in the epilogue),
+// else the GEMM and the activation kernel.
+void linear_fwd_gelu(hift_ctx* c, int M, int f, int K, const void* x, const void* w, void* a, void* u, const void* bias, bool keep) {
+  GemmArgs g{M, f, K, x, K, 1, w, 1, K, keep ? a : nullptr, (int64_t)f, bias, nullptr, 0, false};
+  g.gelu_out = u;
+  if (c->mixed && gemm_tc_eligible(g)) {
+    LAUNCH(HIFT_K_GEMM_FWD, 2.0 * M * (double)f * K, c->note(gemm_tc_launch(c->st, g)));
+    return;
+  }
+  linear_fwd(c, M, f, K, x, K, w, a, f, bias, nullptr, 0, false);
+  act_fwd(c, a, u);
+}
+void act_bwd(hift_ctx* c, const void* a);
+void linear_dx_gelu_bwd(hift_ctx* c, int M, int N, int f, const void* dy, const void* w, const void* a) {
+  GemmArgs g{M, f, N, dy, N, 1, w, f, 1, c->dbig, (int64_t)f, nullptr, nullptr, 0, false};
+  g.gelu_bwd_a = a;
+  if (c->mixed && gemm_tc_eligible(g)) {
+    LAUNCH(HIFT_K_GEMM_DX, 2.0 * M * (double)f * N, c->note(gemm_tc_launch(c->st, g)));
+    return;
+  }
+  linear_dx(c, M, N, f, dy, N, w, c->dbig, f, nullptr, 0, false);
+  act_bwd(c, a);
+}
 // GELU: du (in c->dbig, [T,f]) *= gelu'(a) in place.
 // SwiGLU: ds (in c->dsw, [T,f]) -> dgu in c->dbig [T,2f].
 void act_bwd(hift_ctx* c, const void* a) {
@@ -481,8 +505,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
     linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);             // y
     norm_fwd(c, x2, b.n1_g, b.n1_b, s[S_H2], x1r, (float*)s[S_ST1]);                                 // x1
-    linear_fwd(c, T, f, d, s[S_H2], d, c->P(b.w_fc1), s[S_A], f, c->Pn(b.b_fc1), nullptr, 0, false);
-    act_fwd(c, s[S_A], s[S_U]);
+    linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
     linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), z, d, c->Pn(b.b_fc2), x1r, d, true);           // z
     norm_fwd(c, z, b.n2_g, b.n2_b, xo_a, xo_r, (float*)s[S_ST2]);
     return;
@@ -497,8 +520,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     // blocks below the active group keep nothing: their pre-activations live in the scratch slot and are never read
     linear_fwd_swiglu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
   } else {
-    linear_fwd(c, T, fa, d, s[S_H2], d, c->P(b.w_fc1), s[S_A], fa, c->Pn(b.b_fc1), nullptr, 0, false);
-    act_fwd(c, s[S_A], s[S_U]);
+    linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
   }
   linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
 }
@@ -516,9 +538,8 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
     float* z = (float*)s[S_Z];
     if (on) norm_bwd_params(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, b.n2_b);
     norm_bwd_dx(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, nullptr, c->dxb, c->dxb_a);          // dz
-    linear_dx(c, T, d, f, c->dxb_a, d, c->P(b.w_fc2), c->dbig, f, nullptr, 0, false);               // du
+    linear_dx_gelu_bwd(c, T, d, f, c->dxb_a, c->P(b.w_fc2), s[S_A]);                                // du -> da
     if (on) { linear_dw(c, T, d, f, c->dxb_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxb, true, T, d, d, b.b_fc2); }
-    act_bwd(c, s[S_A]);                                                                             // da
     linear_dx(c, T, f, d, c->dbig, f, c->P(b.w_fc1), c->dxa, d, c->dxb, d, true);                   // dx1
     if (on) { linear_dw(c, T, f, d, c->dbig, f, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, f, f, b.b_fc1); }
     if (on) norm_bwd_params(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, b.n1_b);
@@ -540,7 +561,8 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
       act_done = true;
     }
   }
-  if (!act_done) linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);  // du / ds
+  if (!act_done && c->m.arch != 2) { linear_dx_gelu_bwd(c, T, d, f, c->dxa_a, c->P(b.w_fc2), s[S_A]); act_done = true; }
+  if (!act_done) linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);  // ds
   if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxa, true, T, d, d, b.b_fc2); }
   if (!act_done) act_bwd(c, s[S_A]);                                                                // da in dbig [T,fa]
   linear_dx(c, T, fa, d, c->dbig, fa, c->P(b.w_fc1), c->dt1, d, nullptr, 0, false);                 // dh2
@@ -1480,6 +1502,22 @@ hift_status hift_k_linear_dx_swiglu_bwd(int64_t M, int64_t N, int64_t f, const v
   if (M < 1 || N < 1 || f < 1 || !gu || !dgu) return HIFT_ERR_CFG;
   GemmArgs g{(int)M, (int)f, (int)N, dy, N, 1, w, f, 1, dgu, 2 * f, nullptr, nullptr, 0, false};
   g.swiglu_bwd_gu = gu;
+  if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
+  return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_linear_gelu(int64_t M, int64_t N, int64_t K, const void* a, const void* b, void* pre, void* act,
+                               const void* bias, void* stream) {
+  if (M < 1 || N < 1 || K < 1 || !act) return HIFT_ERR_CFG;
+  GemmArgs g{(int)M, (int)N, (int)K, a, K, 1, b, 1, K, pre, N, bias, nullptr, 0, false};
+  g.gelu_out = act;
+  if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
+  return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_linear_dx_gelu_bwd(int64_t M, int64_t N, int64_t f, const void* dy, const void* w, const void* pre,
+                                      void* da, void* stream) {
+  if (M < 1 || N < 1 || f < 1 || !pre || !da) return HIFT_ERR_CFG;
+  GemmArgs g{(int)M, (int)f, (int)N, dy, N, 1, w, f, 1, da, f, nullptr, nullptr, 0, false};
+  g.gelu_bwd_a = pre;
   if (gemm_tc_init() != 0 || !gemm_tc_eligible(g)) return HIFT_ERR_CFG;
   return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }

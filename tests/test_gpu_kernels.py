@@ -263,6 +263,37 @@ def test_down_projection_dx_with_swiglu_backward_in_the_epilogue(M, N, f):
     assert rel_l2(got[:, f:], du_ref) <= 4e-3
 
 
+@pytest.mark.parametrize("M,N,K,keep,bias", [(300, 416, 256, True, True), (256, 1024, 192, False, False)])
+def test_up_projection_with_gelu_in_the_epilogue(M, N, K, keep, bias):
+    import torch
+    from paper_2401_15207_b200 import k_linear_gelu
+    rng = np.random.default_rng(M + N)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * (2.0 / np.sqrt(K))).astype(np.float32)
+    b = (0.5 * rng.standard_normal(N)).astype(np.float32)
+    pre = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda") if keep else None
+    act = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    k_linear_gelu(M, N, K, _t(x, torch.bfloat16), _t(w, torch.bfloat16), pre, act, _t(b, torch.bfloat16) if bias else None)
+    y = _bf(x) @ _bf(w).T + (_bf(b) if bias else 0.0)
+    assert rel_l2(act.float().cpu().numpy(), O.gelu_fwd(y)) <= 4e-3
+    if keep:
+        assert rel_l2(pre.float().cpu().numpy(), y) <= 4e-3
+
+
+@pytest.mark.parametrize("M,N,f", [(300, 256, 416), (200, 192, 96)])
+def test_down_projection_dx_with_gelu_backward_in_the_epilogue(M, N, f):
+    import torch
+    from paper_2401_15207_b200 import k_linear_dx_gelu_bwd
+    rng = np.random.default_rng(M + f)
+    dy = rng.standard_normal((M, N)).astype(np.float32)
+    w = (rng.standard_normal((N, f)) / np.sqrt(N)).astype(np.float32)
+    a = (1.5 * rng.standard_normal((M, f))).astype(np.float32)
+    da = torch.empty((M, f), dtype=torch.bfloat16, device="cuda")
+    k_linear_dx_gelu_bwd(M, N, f, _t(dy, torch.bfloat16), _t(w, torch.bfloat16), _t(a, torch.bfloat16), da)
+    ref = O.gelu_bwd(_bf(dy) @ _bf(w), _bf(a))
+    assert rel_l2(da.float().cpu().numpy(), ref) <= 4e-3
+
+
 # ------------------------------------------------------------------ norms
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("kind", [0, 1])
