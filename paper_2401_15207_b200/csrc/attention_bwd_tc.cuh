@@ -177,6 +177,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
+  pdl_trigger();
+  pdl_wait();                                          // the set-up above may run under the predecessor's tail
   // tensor-memory columns: tS[u] at 64u, tP[u] at 128 + 64u, accumulators from 256
   const uint32_t tAcc0 = tmem_base + 256;                // dS-fed accumulator: dK (MODE 0) / dQ (MODE 1)
   const uint32_t tAcc1 = tmem_base + 256 + DH;           // P-fed accumulator: dV (MODE 0 only)

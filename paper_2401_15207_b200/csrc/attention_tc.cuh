@@ -125,6 +125,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
+  pdl_trigger();
+  pdl_wait();                                          // the set-up above may run under the predecessor's tail
 
   if (warp == 0) {
     // ---------------- TMA producer

@@ -93,6 +93,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while
+// its predecessor in the stream is still draining; pdl_wait() returns once the predecessor has completed and
+// its writes are visible, and nothing before it may touch global data.  pdl_trigger() lets the successor of
+// this kernel be scheduled as soon as every CTA has passed it (or exited).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -471,6 +477,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
+  pdl_trigger();
+  pdl_wait();                                        // barriers and tensor memory were set up under the predecessor's tail
 
   if (warp == 0) {
     // ---------------- TMA producer (one thread)
@@ -660,6 +668,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   cluster_sync_all();                                  // barriers of both CTAs are initialised
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
+  pdl_trigger();
+  pdl_wait();                                          // set-up above overlaps the predecessor's tail
   const bool poisoned = *(volatile int*)&g_tc_error != 0;   // read after the pair sync; see the exit below
 
   if (warp == 0) {
@@ -771,6 +781,7 @@ EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 148;
 int g_init_state = -1;    // -1 not tried, 0 ok, 1 failed
 std::mutex g_mu;
+int g_pdl = 1;            // programmatic dependent launch of the GEMM kernels (HIFT_PDL=0: plain stream order)
 
 struct MapKey {
   const void* p; uint64_t inner, outer, stride; uint32_t box_outer;
@@ -808,6 +819,18 @@ bool get_map(const void* p, uint64_t inner, uint64_t outer, uint64_t stride_elem
   return true;
 }
 
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_tc(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = g_pdl;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr() {
   return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -819,11 +842,22 @@ cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   const int tiles_m = (g.M + BM - 1) / BM, tiles_n = g.swiglu_out ? g.N / 256 : (g.N + bn - 1) / bn;
   const int num_tiles = tiles_m * tiles_n;
   const int grid = num_tiles < g_num_sms ? num_tiles : g_num_sms;
-  gemm_tc_kernel<A_MN, B_MN, OUT_F32><<<grid, kThreads, kSmemBytes, st>>>(
-      ta, tb, g.M, g.N, g.K, g.c, g.ldc, (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
-      RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
-      SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu}, GeluArgs{(__nv_bfloat16*)g.gelu_out, (const __nv_bfloat16*)g.gelu_bwd_a});
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = g_pdl;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
+                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
+                            RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
+                            SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu},
+                            GeluArgs{(__nv_bfloat16*)g.gelu_out, (const __nv_bfloat16*)g.gelu_bwd_a});
 }
 
 template <bool A_MN, bool B_MN, bool OUT_F32>
@@ -838,11 +872,13 @@ cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = g_pdl;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
                             (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles,
                             RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
@@ -892,6 +928,7 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr2<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr2<true, true, true>();
   if (const char* pm = getenv("HIFT_GEMM_PAIR")) g_pair_mode = atoi(pm);
+  if (const char* pd = getenv("HIFT_PDL")) g_pdl = atoi(pd);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
   if (const char* am = getenv("HIFT_ATTN_TC")) g_attn_tc = atoi(am);
@@ -1018,10 +1055,8 @@ cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int
   const int grid = nitems < g_num_sms ? nitems : g_num_sms;          // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)dh);
   if (dh == 64)
-    attn_fwd_tc_kernel<64><<<grid, kAttThreads, AttnTcCfg<64>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
-  else
-    attn_fwd_tc_kernel<128><<<grid, kAttThreads, AttnTcCfg<128>::kSmem, st>>>(tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
-  return cudaGetLastError();
+    return launch_pdl_tc(attn_fwd_tc_kernel<64>, dim3(grid), dim3(kAttThreads), AttnTcCfg<64>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
+  return launch_pdl_tc(attn_fwd_tc_kernel<128>, dim3(grid), dim3(kAttThreads), AttnTcCfg<128>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
 }
 
 bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, const void* dqkv) {
@@ -1040,12 +1075,12 @@ static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int ca
   const int grid = nitems < g_num_sms ? nitems : g_num_sms;       // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)DH);
   // dK, dV: fixed K, V; streamed Q, dO
-  attn_bwd_tc_kernel<DH, 0><<<grid, kAbThreads, AttnBwdCfg<DH, 0>::kSmem, st>>>(
+  cudaError_t e = launch_pdl_tc(attn_bwd_tc_kernel<DH, 0>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 0>::kSmem, st,
       qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale);
+  if (e != cudaSuccess) return e;
   // dQ: fixed Q, dO; streamed K, V
-  attn_bwd_tc_kernel<DH, 1><<<grid, kAbThreads, AttnBwdCfg<DH, 1>::kSmem, st>>>(
+  return launch_pdl_tc(attn_bwd_tc_kernel<DH, 1>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 1>::kSmem, st,
       qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale);
-  return cudaGetLastError();
 }
 cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,
                                const float* lse, const float* dsum, void* dqkv) {

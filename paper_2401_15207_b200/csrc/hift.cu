@@ -423,8 +423,8 @@ void linear_fwd_qkv_rope(hift_ctx* c, int M, int d, const void* x, const void* w
 void rope(hift_ctx* c, void* qkv, float sign) {
   const size_t n = (size_t)c->T * c->H * (c->dh / 16);      // one thread per 8 pairs
   LAUNCH(HIFT_K_ELEMWISE, 64.0 * n * c->es,
-         if (c->mixed) rope_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>((bf16*)qkv, c->rope_cs, c->T, c->S, c->H, c->dh, sign);
-         else rope_kernel<float><<<grid_for(n, 256), 256, 0, c->st>>>((float*)qkv, c->rope_cs, c->T, c->S, c->H, c->dh, sign));
+         if (c->mixed) launch_pdl(rope_kernel<bf16>, dim3(grid_for(n, 256)), dim3(256), 0, c->st, (bf16*)qkv, c->rope_cs, (int64_t)c->T, c->S, c->H, c->dh, sign);
+         else launch_pdl(rope_kernel<float>, dim3(grid_for(n, 256)), dim3(256), 0, c->st, (float*)qkv, c->rope_cs, (int64_t)c->T, c->S, c->H, c->dh, sign));
 }
 void act_fwd(hift_ctx* c, const void* a, void* u) {
   const size_t n = (size_t)c->T * c->f;

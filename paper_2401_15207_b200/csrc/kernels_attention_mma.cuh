@@ -235,6 +235,8 @@ template <int DH>
 __global__ void attn_dsum_kernel(const bf16* __restrict__ o, const bf16* __restrict__ dout,
                                  float* __restrict__ dsum, int B, int S, int H) {
   constexpr int LPR = DH / 8;                              // lanes per row: 8 or 16
+  pdl_launch_next();
+  pdl_wait_prior();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t row = i / LPR;                             // (token, head)
   const int part = (int)(i % LPR);
@@ -259,8 +261,8 @@ __global__ void attn_dsum_kernel(const bf16* __restrict__ o, const bf16* __restr
 inline void launch_attn_dsum(cudaStream_t st, const bf16* o, const bf16* dout, float* dsum, int B, int S, int H, int DH) {
   const int64_t threads = (int64_t)B * S * H * (DH / 8);
   const unsigned grid = (unsigned)((threads + 255) / 256);
-  if (DH == 64) attn_dsum_kernel<64><<<grid, 256, 0, st>>>(o, dout, dsum, B, S, H);
-  else attn_dsum_kernel<128><<<grid, 256, 0, st>>>(o, dout, dsum, B, S, H);
+  if (DH == 64) launch_pdl(attn_dsum_kernel<64>, dim3(grid), dim3(256), 0, st, o, dout, dsum, B, S, H);
+  else launch_pdl(attn_dsum_kernel<128>, dim3(grid), dim3(256), 0, st, o, dout, dsum, B, S, H);
 }
 
 // ------------------------------------------------------------------ backward: dq (owner of query rows)

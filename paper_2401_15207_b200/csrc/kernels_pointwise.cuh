@@ -144,6 +144,8 @@ __global__ void norm_fwd_kernel(const float* __restrict__ x, const P* __restrict
                                 const P* __restrict__ bias, P* __restrict__ y_a,
                                 float* __restrict__ y_r, float* __restrict__ stats, int64_t rows,
                                 int cols, float eps) {
+  pdl_launch_next();
+  pdl_wait_prior();
   __shared__ float red[33];
   const int64_t row = blockIdx.x;
   const float* xr = x + row * cols;
@@ -197,6 +199,8 @@ __global__ void norm_bwd_dx_kernel(const DY* __restrict__ dy, const float* __res
                                    const float* __restrict__ stats, const P* __restrict__ gain,
                                    const float* __restrict__ add, float* __restrict__ dx_r,
                                    P* __restrict__ dx_a, int64_t rows, int cols) {
+  pdl_launch_next();
+  pdl_wait_prior();
   __shared__ float red[33];
   const int64_t row = blockIdx.x;
   const float mean = stats[row], rstd = stats[rows + row];
@@ -393,6 +397,8 @@ __global__ void swiglu_bwd_kernel(const T* __restrict__ ds, const T* __restrict_
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ qkv, const float* __restrict__ cs, int64_t Ttot, int S,
                             int H, int dh, float sign) {
+  pdl_launch_next();
+  pdl_wait_prior();
   const int half = dh / 2, hc = half / 8;
   const size_t n = (size_t)Ttot * H * hc;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;

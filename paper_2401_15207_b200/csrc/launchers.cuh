@@ -145,7 +145,7 @@ inline void launch_norm_fwd(cudaStream_t st, int dtype, int kind, int64_t rows, 
                             const float* x, const void* gain, const void* bias, void* y_a, float* y_r,
                             float* stats) {
   const int th = norm_threads(cols);
-#define NF(P, K) norm_fwd_kernel<P, K><<<(unsigned)rows, th, 0, st>>>(x, (const P*)gain, (const P*)bias, (P*)y_a, y_r, stats, rows, cols, eps)
+#define NF(P, K) launch_pdl(norm_fwd_kernel<P, K>, dim3((unsigned)rows), dim3(th), 0, st, x, (const P*)gain, (const P*)bias, (P*)y_a, y_r, stats, rows, cols, eps)
   if (dtype == 0) { if (kind == 0) NF(float, 0); else NF(float, 1); }
   else { if (kind == 0) NF(bf16, 0); else NF(bf16, 1); }
 #undef NF
@@ -155,7 +155,7 @@ inline void launch_norm_bwd_dx(cudaStream_t st, int dtype, int kind, bool dy_f32
                                const void* dy, const float* x, const float* stats, const void* gain,
                                const float* add, float* dx_r, void* dx_a) {
   const int th = norm_threads(cols);
-#define NB(DY, P, K) norm_bwd_dx_kernel<DY, P, K><<<(unsigned)rows, th, 0, st>>>((const DY*)dy, x, stats, (const P*)gain, add, dx_r, (P*)dx_a, rows, cols)
+#define NB(DY, P, K) launch_pdl(norm_bwd_dx_kernel<DY, P, K>, dim3((unsigned)rows), dim3(th), 0, st, (const DY*)dy, x, stats, (const P*)gain, add, dx_r, (P*)dx_a, rows, cols)
   if (dtype == 0) { if (kind == 0) NB(float, float, 0); else NB(float, float, 1); }
   else if (dy_f32) { if (kind == 0) NB(float, bf16, 0); else NB(float, bf16, 1); }
   else { if (kind == 0) NB(bf16, bf16, 0); else NB(bf16, bf16, 1); }
