@@ -332,3 +332,48 @@ def test_warmup_then_decay_moves_once_per_cycle():
     from oracle import hift_oracle as O
     assert lrs == [O.lr_for_cycle(oc.lr, oc.sched, t // k, oc.total_cycles, oc.warmup_cycles) for t in range(4 * k)]
     assert lrs == pytest.approx([0.0] * k + [0.5e-2] * k + [1e-2] * k + [0.5e-2] * k, rel=1e-15, abs=0.0)
+
+
+_PDL_SCRIPT = r"""
+import sys, hashlib, numpy as np, torch
+sys.path.insert(0, sys.argv[1])
+import synth
+from paper_2401_15207_b200 import HiFT
+arch = int(sys.argv[2])
+cfg = synth.ModelCfg(arch=arch, n_blocks=3, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=768 if arch == 2 else 1024, vocab=1000,
+                     max_pos=128, causal=1, tie_head=0, norm_eps=1e-6 if arch == 2 else 1e-5, dtype=synth.DTYPE_BF16,
+                     batch=2, seq=128, init_std=0.05)
+oc = synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
+h = HiFT(cfg, synth.GroupCfg(1), oc)
+h.set_params(synth.init_params(cfg, 4, perturb=0.05))
+losses = []
+for t in range(2 * h.num_groups()):
+    tok, lab = synth.batch_for(cfg, 21, t, "zipf")
+    losses.append(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
+m = hashlib.sha256()
+for n in h.tensor_names():
+    m.update(np.ascontiguousarray(h.get_param(n)).tobytes())
+print("RESULT", m.hexdigest(), " ".join(repr(x) for x in losses))
+"""
+
+
+@pytest.mark.parametrize("arch", [0, 2])
+def test_dependent_launch_changes_no_bits(arch, tmp_path):
+    """Programmatic dependent launch lets a kernel start under its predecessor's tail; it must wait before it
+    touches memory.  Two fresh processes, one with it (the default) and one in plain stream order, run the same
+    two cycles on a model large enough for the tensor-core kernels: every loss and every parameter bit agree."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "pdl_run.py"
+    script.write_text(_PDL_SCRIPT)
+    outs = []
+    for pdl in ("1", "0"):
+        env = dict(os.environ, HIFT_PDL=pdl)
+        r = subprocess.run([sys.executable, str(script), root, str(arch)], capture_output=True, text=True, env=env, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        line = [l for l in r.stdout.splitlines() if l.startswith("RESULT")]
+        assert line, r.stdout[-500:]
+        outs.append(line[0])
+    assert outs[0] == outs[1]
