@@ -192,6 +192,40 @@ def test_attention_forward_backward(dtype, dh, causal):
         assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= tolb, i
 
 
+@pytest.mark.parametrize("dh", [64, 128])
+@pytest.mark.parametrize("B,S,H", [(1, 1, 1), (1, 64, 2), (3, 129, 1), (2, 300, 2), (1, 640, 1)])
+@pytest.mark.parametrize("causal", [0, 1])
+def test_attention_tensor_core_edge_lengths(dh, B, S, H, causal):
+    """bf16 attention on the tensor-core kernels at the degenerate and ragged sequence lengths: a single
+    position, exactly one tile, one row past a tile, several tiles with a tail, more tiles than a CTA's
+    double buffers; batch entries that share a tile with their neighbour."""
+    import torch
+    from paper_2401_15207_b200 import k_attention_fwd, k_attention_bwd
+    d = H * dh
+    rng = np.random.default_rng(1000 * dh + 10 * S + causal)
+    qkv = rng.standard_normal((B * S, 3 * d)).astype(np.float32)
+    do = rng.standard_normal((B * S, d)).astype(np.float32)
+    q, k, v = (_bf(qkv)[:, i * d:(i + 1) * d].reshape(B, S, H, dh) for i in range(3))
+    o_ref, p = O.attention_fwd(q, k, v, bool(causal))
+    tq = _t(qkv, torch.bfloat16)
+    o = torch.full((B * S, d), 9.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((B, H, S), 9.0, dtype=torch.float32, device="cuda")
+    k_attention_fwd(1, B, S, H, dh, causal, tq, o, lse)
+    assert rel_l2(o.float().cpu().numpy(), o_ref.reshape(B * S, d)) <= 6e-3
+    dqkv = torch.full((B * S, 3 * d), 9.0, dtype=torch.bfloat16, device="cuda")
+    dsum = torch.empty(B * S * H, dtype=torch.float32, device="cuda")
+    k_attention_bwd(1, B, S, H, dh, causal, tq, o, lse, _t(do, torch.bfloat16), dqkv, dsum)
+    dq, dk, dv = O.attention_bwd(_bf(do).reshape(B, S, H, dh), q, k, v, p)
+    ref = np.concatenate([t.reshape(B * S, d) for t in (dq, dk, dv)], axis=1)
+    got = dqkv.float().cpu().numpy()
+    for i in range(3):
+        r = ref[:, i * d:(i + 1) * d]
+        if np.linalg.norm(r) == 0.0:                         # S = 1: dq and dk vanish identically
+            assert np.abs(got[:, i * d:(i + 1) * d]).max() <= 1e-3
+        else:
+            assert rel_l2(got[:, i * d:(i + 1) * d], r) <= 1.5e-2, i
+
+
 # ------------------------------------------------------------------ rotary embedding fused into the qkv projection
 def _rope_cs(S, dh, base=10000.0):
     cos, sin = O.rope_tables(S, dh, base)
