@@ -1042,10 +1042,8 @@ const int* gemm_tc_error_device_ptr() {
 }
 
 bool attn_tc_eligible(int dh, const void* qkv, int H) {
-  // head size 128 only: at 64 the softmax threads, not the tensor cores, set the pace and the
-  // warp-level kernel (more CTAs per SM) is faster; HIFT_ATTN_TC=2 forces this kernel for both sizes
-  return g_init_state == 0 && g_attn_tc && (dh == 128 || (dh == 64 && g_attn_tc == 2)) && (((uintptr_t)qkv) & 15) == 0 &&
-         ((3 * H * dh) % 8) == 0;
+  // head sizes 64 and 128 (HIFT_ATTN_TC=0 sends both to the warp-level kernel)
+  return g_init_state == 0 && g_attn_tc && (dh == 128 || dh == 64) && (((uintptr_t)qkv) & 15) == 0 && ((3 * H * dh) % 8) == 0;
 }
 cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse) {
   CUtensorMap tm;
