@@ -9,24 +9,27 @@
 //   warp 0    : TMA producer (Q per item; K and V blocks through two 2-deep rings)
 //   warp 1    : issues S_j = Q K_j^T   (M 128 x N 128, k = d_h)      -> TMEM columns [0,128) / [128,256); owns the tensor memory
 //   warp 2    : issues O += P_j V_j    (M 128 x N d_h, k = 128 keys) -> TMEM columns [256,384) / [384,512) by item parity
-//   warps 3-6 : softmax, one thread per query row (= one tensor-memory lane): read S_j, mask,
-//               running max / sum, write P_j as bf16 into a 128-byte-swizzled shared tile (the A
-//               operand of the second product), rescale O in tensor memory when the reference
-//               maximum moved, and at the end normalise and store O and the log-sum-exp.
+//   warps 3-10: softmax, two threads per query row (= one tensor-memory lane; warps w and w + 4 share
+//               a lane quarter and take 64 of the block's 128 columns each): read S_j, mask, running
+//               max / sum, write P_j as bf16 into a 128-byte-swizzled shared tile (the A operand of
+//               the second product), rescale their half of O's columns in tensor memory when the
+//               reference maximum moved, and at the end normalise and store O and the log-sum-exp.
+//               The two threads of a row agree on the block maximum (and at the end on the sum)
+//               through a 1 KB exchange in shared memory and a named barrier of their two warps.
 // Q and K are K-major operands (d_h contiguous), V is an N-major operand (B(k = key, n = e) =
 // V[key][e]): all three are read straight out of qkv[T, 3d] by one tensor map, nothing is copied
 // or transposed.  Rows of a tile that lie beyond this batch entry's sequence hold the next
 // entry's (finite) values or TMA zero fill; their scores are masked, their probabilities are 0.
 #pragma once
 
-constexpr int kAttThreads = 224;
+constexpr int kAttThreads = 352;
 constexpr int kAttBQ = 128, kAttBK = 128;
 
 template <int DH> struct AttnTcCfg {
   static constexpr int kSpans = DH / 64;                       // 64-column swizzle spans per row
   static constexpr int kTileBytes = 128 * DH * 2;              // one Q / K / V tile
   static constexpr int kPBytes = 128 * kAttBK * 2;             // P tile: 128 rows x 128 keys
-  static constexpr int kSmem = 6 * kTileBytes + kPBytes + 1024 + 256;      // Q x 2, K x 2, V x 2, P
+  static constexpr int kSmem = 6 * kTileBytes + kPBytes + 1024 + 256 + 1024;      // Q x 2, K x 2, V x 2, P, row exchange
 };
 
 __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&v)[32]) {
@@ -86,6 +89,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
   auto o_done = [&](int i) { return bar + 128u + 8u * i; };
   auto o_free = [&](int i) { return bar + 144u + 8u * i; };
   const uint32_t p_ready = bar + 160u, p_free = bar + 168u, tmem_slot = bar + 176u;
+  float* xch = reinterpret_cast<float*>(smem_raw + (bar + 256u - smem_u32(smem_raw)));       // [128 rows][2 halves]
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
   uint8_t* p_gen = gen + (sP - base);
@@ -103,17 +107,20 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
     it.nblk = (kv_len + kAttBK - 1) / kAttBK;
     return it;
   };
-  const bool poisoned = g_tc_error != 0;
+  // one thread reads the time-out flag and the CTA shares the answer: the softmax warps meet at named
+  // barriers in pairs, so they must all take the same way
+  volatile uint32_t* poison_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot + 8u - base));
 
   if (threadIdx.x == 0) {
+    *poison_gen = g_tc_error != 0 ? 1u : 0u;
     for (int i = 0; i < 2; ++i) {
       mbar_init(q_full(i), 1); mbar_init(q_empty(i), 1);
       mbar_init(k_full(i), 1); mbar_init(k_empty(i), 1);
       mbar_init(v_full(i), 1); mbar_init(v_empty(i), 1);
-      mbar_init(s_full(i), 1); mbar_init(s_free(i), 4);
-      mbar_init(o_done(i), 1); mbar_init(o_free(i), 4);
+      mbar_init(s_full(i), 1); mbar_init(s_free(i), 8);
+      mbar_init(o_done(i), 1); mbar_init(o_free(i), 8);
     }
-    mbar_init(p_ready, 4);                              // one arrival per softmax warp
+    mbar_init(p_ready, 8);                              // one arrival per softmax warp
     mbar_init(p_free, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -125,6 +132,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
+  const bool poisoned = *poison_gen != 0;
   pdl_trigger();
   pdl_wait();                                          // the set-up above may run under the predecessor's tail
 
@@ -220,31 +228,40 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       }
     }
   } else {
-    // ---------------- softmax and epilogue: thread = query row = tensor-memory lane
-    const int q = warp & 3;
+    // ---------------- softmax and epilogue: two threads per query row (= tensor-memory lane)
+    const int q = warp & 3;                             // lane quarter; warps w and w + 4 share it
+    const int half = (warp - 3) >> 2;                   // which 64 of the block's 128 columns, which half of O's columns
     const int r = q * 32 + lane;                        // row inside the tile
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const float sl2 = scale * 1.4426950408889634f;
+    constexpr int HB = kAttBK / 2, OC = DH / 2;
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory"); };
+    // a warp that gives up on a bounded wait must not leave its partner at the named barrier: it arrives (without
+    // waiting) for every meeting the partner can still reach before its own next bounded wait ends it
+    auto pair_release = [&]() {
+#pragma unroll 1
+      for (int i = 0; i < 4; ++i) asm volatile("bar.arrive %0, 64;" ::"r"(1 + q) : "memory");
+    };
     bool ok = !poisoned;
     int g = 0, n = 0;
     for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
       const Item it = item_of(idx);
       const int q0 = it.q0, qrow = q0 + r, row_g0 = it.b * S;
       const uint32_t tO = tmem_base + 256u + (uint32_t)((n & 1) * 128);
-      float m = -INFINITY, l = 0.f;
+      float m = -INFINITY, l = 0.f;                     // m: the row's reference maximum (same in both threads); l: this half's sum
       for (int j = 0; j < it.nblk; ++j, ++g) {
         const int st = g & 1;
         bool ready = mbar_wait(s_full(st), (uint32_t)((g >> 1) & 1));
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
         tc_fence_after();
         ok = __all_sync(0xffffffffu, ready);
-        if (!ok) break;
-        // scores of this row: 128 columns (raw; the scale is folded into the exponent below)
-        float sc[kAttBK];
+        if (!ok) { pair_release(); break; }
+        // this thread's 64 scores of the row (raw; the scale is folded into the exponent below)
+        float sc[HB];
 #pragma unroll
-        for (int c0 = 0; c0 < kAttBK; c0 += 32) {
+        for (int c0 = 0; c0 < HB; c0 += 32) {
           uint32_t v[32];
-          tmem_ld32(tmem_base + lane_off + (uint32_t)(st * 128 + c0), v);
+          tmem_ld32(tmem_base + lane_off + (uint32_t)(st * 128 + half * HB + c0), v);
 #pragma unroll
           for (int i = 0; i < 32; ++i) sc[c0 + i] = __uint_as_float(v[i]);
         }
@@ -254,23 +271,28 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
         // masking only where the block touches the diagonal or the end of the sequence (uniform per CTA)
         if ((causal && j * kAttBK + kAttBK - 1 > q0) || (j + 1) * kAttBK > S) {
 #pragma unroll
-          for (int i = 0; i < kAttBK; ++i) {
-            const int key = j * kAttBK + i;
+          for (int i = 0; i < HB; ++i) {
+            const int key = j * kAttBK + half * HB + i;
             if (key >= S || (causal && key > qrow)) sc[i] = -INFINITY;
           }
         }
-        // four independent chains each for the maximum and the sum: one warp per scheduler has nobody
-        // else to hide a serial chain's latency behind
+        // four independent chains each for the maximum and the sum
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < kAttBK; i += 4) {
+        for (int i = 0; i < HB; i += 4) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) mx4[e] = fmaxf(mx4[e], sc[i + e]);
         }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;     // in log2 units (scale > 0)
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;     // in log2 units (scale > 0)
+        // the row's block maximum = the larger of the two halves'
+        xch[r * 2 + half] = mx;
+        pair_sync();
+        mx = fmaxf(mx, xch[r * 2 + (half ^ 1)]);
+        pair_sync();
         // Lazy reference maximum: m moves (and O is rescaled) only when some row of the warp has grown by
         // more than 2^8 over it; until then probabilities up to 256 are summed against the old reference,
-        // which changes nothing in the final O / l and lse = m + log2(l).
+        // which changes nothing in the final O / l and lse = m + log2(l).  Both warps of a quarter see the
+        // same m and mx per row, so they take the same decision.
         const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
         float corr = 1.0f;
         if (grow) {
@@ -281,7 +303,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
         const float nmuse = (m == -INFINITY) ? 0.f : -m;
         float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < kAttBK; i += 4) {
+        for (int i = 0; i < HB; i += 4) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) { sc[i + e] = ex2_approx(fmaf(sc[i + e], sl2, nmuse)); sum4[e] += sc[i + e]; }
         }
@@ -291,25 +313,24 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
         tc_fence_after();
         ok = __all_sync(0xffffffffu, ready);
-        if (!ok) break;
-        // P row -> shared memory, bf16, K-major with the 128-byte swizzle the MMA descriptor expects
+        if (!ok) { pair_release(); break; }
+        // this half of the P row -> shared memory, bf16: one 64-key span of the K-major, 128-byte-swizzled tile
 #pragma unroll
-        for (int ch = 0; ch < kAttBK / 8; ++ch) {
+        for (int c = 0; c < HB / 8; ++c) {
           uint4 pk;
           __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
-          for (int t = 0; t < 4; ++t) hp[t] = __floats2bfloat162_rn(sc[ch * 8 + 2 * t], sc[ch * 8 + 2 * t + 1]);
-          const int span = ch >> 3, c = ch & 7;
-          *reinterpret_cast<uint4*>(p_gen + span * SPAN_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = pk;
+          for (int t = 0; t < 4; ++t) hp[t] = __floats2bfloat162_rn(sc[c * 8 + 2 * t], sc[c * 8 + 2 * t + 1]);
+          *reinterpret_cast<uint4*>(p_gen + half * SPAN_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = pk;
         }
-        if (j > 0 && grow) {                            // warp-uniform
+        if (j > 0 && grow) {                            // warp-uniform; this thread's half of O's columns
 #pragma unroll 1
-          for (int c0 = 0; c0 < DH; c0 += 32) {
+          for (int c0 = 0; c0 < OC; c0 += 32) {
             uint32_t v[32];
-            tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+            tmem_ld32(tO + lane_off + (uint32_t)(half * OC + c0), v);
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
-            tmem_st32(tO + lane_off + (uint32_t)c0, v);
+            tmem_st32(tO + lane_off + (uint32_t)(half * OC + c0), v);
           }
           tmem_st_wait();
         }
@@ -319,21 +340,26 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
         if (lane == 0) mbar_arrive(p_ready);
       }
       if (!ok) break;
+      // the row's sum = the two halves' (both relative to the same m)
+      xch[r * 2 + half] = l;
+      pair_sync();
+      const float ltot = l + xch[r * 2 + (half ^ 1)];
+      pair_sync();
       // last product of the item done -> normalise and store
       {
         const bool ready = mbar_wait(o_done(n & 1), (uint32_t)((n >> 1) & 1));
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
         tc_fence_after();
         ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
-        if (!ok) break;
+        if (!ok) { pair_release(); break; }
       }
-      const float inv = 1.0f / l;
-      __nv_bfloat16* orow = o + ((int64_t)(row_g0 + qrow)) * d + (int64_t)it.h * DH;
+      const float inv = 1.0f / ltot;
+      __nv_bfloat16* orow = o + ((int64_t)(row_g0 + qrow)) * d + (int64_t)it.h * DH + half * OC;
 #pragma unroll 1
-      for (int c0 = 0; c0 < DH; c0 += 32) {
+      for (int c0 = 0; c0 < OC; c0 += 32) {
         uint32_t v[32];
-        tmem_ld32(tO + lane_off + (uint32_t)c0, v);
-        if (c0 + 32 >= DH) {                            // everything read: the accumulator may be reused
+        tmem_ld32(tO + lane_off + (uint32_t)(half * OC + c0), v);
+        if (c0 + 32 >= OC) {                            // everything read: the accumulator may be reused
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(o_free(n & 1));
@@ -350,7 +376,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
           }
         }
       }
-      if (qrow < S) lse[((int64_t)it.b * H + it.h) * S + qrow] = (m + log2f(l)) * 0.6931471805599453f;
+      if (half == 0 && qrow < S) lse[((int64_t)it.b * H + it.h) * S + qrow] = (m + log2f(ltot)) * 0.6931471805599453f;
     }
   }
   tc_fence_before();
