@@ -19,13 +19,14 @@
 //   warp 2     : issues the accumulating products (one thread); two issuers, because these
 //                products are small and one thread cannot issue them as fast as they execute
 //   warps 3-18 : element-wise stage in two groups of eight that take alternate steps; thread = one
-//                tensor-memory lane (a key in MODE 0, a query in MODE 1) x 32 of the 64 streamed columns: read tS and tP, form P and dS, write
-//                them as bf16 into 128-byte-swizzled shared tiles (the A operands of the
-//                accumulating products); at the end convert and store the accumulators.
+//                tensor-memory lane (a key in MODE 0, a query in MODE 1) x 32 of the 64 streamed
+//                columns: read tS and tP, form P and dS, write them as bf16 into 128-byte-swizzled
+//                shared tiles (the A operands of the accumulating products); at the end all sixteen
+//                warps convert and store the accumulators.
 // tS / tP are double-buffered, so the tensor core works on step t+1's scores while the
-// element-wise warps are busy with step t.  The kernel is persistent: a CTA walks
-// a list of (batch, head, 128-row block) items, heaviest first; the next item's fixed tiles are
-// fetched and its first scores computed while the current item is still being worked on.
+// element-wise warps are busy with step t.  The kernel is persistent: a CTA walks a list of
+// (batch, head, 128-row block) items, heaviest first; with a second set of fixed tiles (d_h = 64) the
+// next item's tiles are fetched and its first scores computed while the current item finishes.
 #pragma once
 
 constexpr int kAbThreads = 608;
