@@ -199,7 +199,8 @@ def run_ours(args, cfg, gcfg, ocfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": args.prefetch, "offload_state": args.offload})
+    ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": args.prefetch, "offload_state": args.offload,
+                           "recompute": args.recompute})
     h = HiFT(cfg, gcfg, ocfg)
     h.init_synthetic(dist_util.rank_seed(1234, rank), cfg.init_std)
     k = h.num_groups()
@@ -331,7 +332,7 @@ def run_ours(args, cfg, gcfg, ocfg):
             "vs_baseline": None, "dtype": "bf16" if cfg.dtype == 1 else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "global_batch": cfg.batch * world, "seq_len": cfg.seq,
                        "groups": k, "groups_trained": trained, "optimizer": ["adamw", "adagrad", "sgdm"][ocfg.kind],
-                       "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups,
+                       "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups, "recompute": ocfg.recompute,
                        "parallelism": (("dp%d" % world) if args.parallel == "dp" else "replicas") if world > 1 else "single",
                        "l2_policy": "inputs larger than L2 (weights + activations of a step exceed 126 MB)"},
             "peak_hbm_gb": peak_hbm / 1e9, "pinned_host_gb": pinned / 1e9,
@@ -474,6 +475,9 @@ def main():
                          "active group's gradient between the backward pass and the update")
     ap.add_argument("--prefetch", type=int, default=1)
     ap.add_argument("--offload", type=int, default=1)
+    ap.add_argument("--recompute", type=int, default=0,
+                    help="1: frozen blocks above the group keep only their input and are recomputed in the backward pass "
+                         "(less HBM, one more forward of those blocks)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--full-param", action="store_true",
                     help="one group holding every unit, state resident: the ordinary full-parameter step")

@@ -89,6 +89,10 @@ typedef struct {
   int32_t prefetch_groups;   /* 0: one state slot, H2D issued after the forward
                                    (the paper's order); 1: two slots, H2D issued at
                                    step start and overlapped with the previous D2H  */
+  int32_t recompute;         /* 1: frozen blocks above the active group keep only their input during the
+                                forward pass; what their backward (dX) needs is recomputed block by block in
+                                the backward pass.  Same bits, less HBM (the paper's concern), one extra
+                                forward of those blocks per step.  0: keep (default)                */
   int32_t warmup_cycles;     /* W (sched 1; the warm-up the paper's hyper-parameter tables list, counted in
                                 cycles because the rate moves once per cycle): cycle c < W runs at
                                 lr*c/W, cycle c >= W at lr*max(0, (C-c)/(C-W)); 0 = none             */

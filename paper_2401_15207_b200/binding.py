@@ -48,7 +48,7 @@ class GroupCfgC(C.Structure):
 
 class OptCfgC(C.Structure):
     _fields_ = [("kind", C.c_int32), ("sched", C.c_int32), ("total_cycles", C.c_int32),
-                ("offload_state", C.c_int32), ("prefetch_groups", C.c_int32), ("warmup_cycles", C.c_int32),
+                ("offload_state", C.c_int32), ("prefetch_groups", C.c_int32), ("recompute", C.c_int32), ("warmup_cycles", C.c_int32),
                 ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
                 ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double)]
 
@@ -157,7 +157,7 @@ class HiFT:
                       model.dtype, model.batch, model.seq, model.norm_eps, model.rope_base)
         g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed)
         o = OptCfgC(opt.kind, opt.sched, opt.total_cycles, opt.offload_state, opt.prefetch_groups,
-                    getattr(opt, "warmup_cycles", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
+                    getattr(opt, "recompute", 0), getattr(opt, "warmup_cycles", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
         self._h = C.c_void_p()
         self._stream = _stream_ptr() if stream is None else stream
         _check(lib().hift_create(C.byref(m), C.byref(g), C.byref(o), self._stream, C.byref(self._h)), "hift_create")

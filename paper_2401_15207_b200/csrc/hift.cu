@@ -68,6 +68,8 @@ struct hift_ctx {
   int L = 0, d = 0, f = 0, fa = 0, H = 0, dh = 0, T = 0, B = 0, S = 0, V = 0, Vp = 0;
   int n_state = 2;
   bool mixed = true, offload = false;
+  bool recompute = false;           // frozen blocks above the group keep only their input; see plan_slots
+  bool keep_all = false;            // set while such a block is recomputed: its forward must store what the backward reads
   bool compact = false;             // paged master = low halves + carry bits beside the bf16 copy (see blob layout)
   std::vector<TensorRec> tens;
   std::vector<std::vector<int>> unit_tens;
@@ -328,7 +330,10 @@ size_t plan_slots(hift_ctx* c, int g, bool assign) {
     for (int s = 0; s < S_NUM; ++s) {
       const int need = slot_min_level(c->m.arch, s);
       if (need == 99) { if (assign) c->slots[i][s] = nullptr; continue; }
-      if (lvl >= need) {
+      // recompute: a frozen block above the group keeps its input only (stream, and operand copy where the
+      // architecture has one); everything else lives in the shared scratch copy until the backward pass redoes it
+      const bool keep = (c->recompute && lvl == 1) ? (s == S_XIN || s == S_XINA) : lvl >= need;
+      if (keep) {
         char* p = arena_take(c, slot_bytes(c, s));
         if (assign) c->slots[i][s] = p;
       } else if (assign) {
@@ -505,7 +510,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
     linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);             // y
     norm_fwd(c, x2, b.n1_g, b.n1_b, s[S_H2], x1r, (float*)s[S_ST1]);                                 // x1
-    linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
+    linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
     linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), z, d, c->Pn(b.b_fc2), x1r, d, true);           // z
     norm_fwd(c, z, b.n2_g, b.n2_b, xo_a, xo_r, (float*)s[S_ST2]);
     return;
@@ -518,9 +523,9 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
   norm_fwd(c, x2, b.n2_g, b.n2_b, s[S_H2], nullptr, (float*)s[S_ST2]);
   if (c->m.arch == 2) {
     // blocks below the active group keep nothing: their pre-activations live in the scratch slot and are never read
-    linear_fwd_swiglu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
+    linear_fwd_swiglu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
   } else {
-    linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), s[S_A] != c->slots[c->L][S_A]);
+    linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
   }
   linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
 }
@@ -686,6 +691,12 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
     for (int i = L - 1; i >= 0; --i) {
       const int u = i + 1;
       if (u < lo) break;
+      if (c->recompute && !active(u)) {
+        // redo this frozen block's forward from its kept input into the scratch slots (its output goes nowhere)
+        c->keep_all = true;
+        forward_block(c, i, chain_r[i], chain_a[i], c->pp[0], c->ppa[0]);
+        c->keep_all = false;
+      }
       backward_block(c, i, chain_r[i], chain_a[i], active(u), u > lo);
       if (u == lo) break;
     }
@@ -952,6 +963,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   c->n_slots = (c->offload && oc->prefetch_groups) ? 2 : 1;
   // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
   c->compact = c->mixed && c->offload && !c->af;
+  c->recompute = oc->recompute != 0;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_work, 0, sizeof(c->prof_work));

@@ -90,6 +90,7 @@ class OptCfg:
     offload_state: int = 1
     prefetch_groups: int = 0
     warmup_cycles: int = 0
+    recompute: int = 0
 
 
 # --------------------------------------------------------------------------

@@ -1,4 +1,5 @@
 """The C-ABI library loads and exports every symbol include/hift.h declares (no GPU needed)."""
+import pytest
 import os
 import re
 
@@ -32,8 +33,35 @@ def test_strerror_covers_all_codes():
     assert msgs[0] == "ok" and len(set(msgs)) == 9
 
 
-def test_structs_match_header_sizes():
+def test_structs_match_header_layout(tmp_path):
+    """The ctypes mirrors of the three configuration structs have the size and the field offsets a C compiler
+    gives the declarations in include/hift.h."""
     import ctypes as C
-    assert C.sizeof(binding.ModelCfgC) == 13 * 4 + 4 + 16      # 13 int32, pad, 2 doubles
-    assert C.sizeof(binding.GroupCfgC) == 3 * 4 + 4 + 8
-    assert C.sizeof(binding.OptCfgC) == 5 * 4 + 4 + 6 * 8
+    import os
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    mirrors = {"hift_model_cfg": binding.ModelCfgC, "hift_group_cfg": binding.GroupCfgC, "hift_opt_cfg": binding.OptCfgC}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "hift.h"', 'int main(void) {']
+    for cname, cls in mirrors.items():
+        lines.append(f'  printf("{cname} size %zu\\n", sizeof({cname}));')
+        for fname, _ in cls._fields_:
+            lines.append(f'  printf("{cname} {fname} %zu\\n", offsetof({cname}, {fname}));')
+    lines += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run([gcc, "-I", inc, "-o", str(exe), str(src)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    seen = 0
+    for line in out:
+        if not line:
+            continue
+        cname, what, val = line.split()
+        cls = mirrors[cname]
+        assert int(val) == (C.sizeof(cls) if what == "size" else getattr(cls, what).offset), line
+        seen += 1
+    assert seen == sum(1 + len(c._fields_) for c in mirrors.values())

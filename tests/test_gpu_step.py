@@ -377,3 +377,32 @@ def test_dependent_launch_changes_no_bits(arch, tmp_path):
         assert line, r.stdout[-500:]
         outs.append(line[0])
     assert outs[0] == outs[1]
+
+
+@pytest.mark.parametrize("arch", [0, 1, 2])
+def test_recomputing_frozen_blocks_changes_no_bits_and_saves_memory(arch):
+    """recompute = 1: the frozen blocks above the active group keep only their input in the forward pass and
+    are run again, one at a time, in the backward pass.  The kernels are deterministic, so the losses and every
+    parameter bit are those of the keeping mode; the activation arena is smaller."""
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(arch, synth.DTYPE_BF16, n_blocks=4, tie_head=1 if arch == 0 else 0)
+    gc = synth.GroupCfg(layers_per_group=1, order=0)
+    p0 = synth.init_params(cfg, 5, perturb=0.05)
+    ctxs = []
+    for rc in (0, 1):
+        h = HiFT(cfg, gc, synth.OptCfg(kind=0, lr=1e-3, weight_decay=0.01, offload_state=1, prefetch_groups=1, recompute=rc))
+        h.set_params(p0)
+        ctxs.append(h)
+    try:
+        assert ctxs[1].peak_hbm_bytes() < ctxs[0].peak_hbm_bytes()
+        for t in range(ctxs[0].num_groups()):
+            tok, lab = synth.batch_for(cfg, 13, t, "zipf")
+            dt, dl = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
+            assert ctxs[0].step(dt, dl) == ctxs[1].step(dt, dl), t
+        for name in ctxs[0].tensor_names():
+            assert np.array_equal(np.asarray(ctxs[0].get_param(name)).view(np.uint32),
+                                  np.asarray(ctxs[1].get_param(name)).view(np.uint32)), name
+    finally:
+        for h in ctxs:
+            h.close()
