@@ -527,7 +527,8 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
   } else {
     linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
   }
-  linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
+  // a block that is only being recomputed for its backward needs everything above, not its output
+  if (!c->keep_all) linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
 }
 
 // ------------------------------------------------------------------ backward
