@@ -207,6 +207,9 @@ def run_ours(args, cfg, gcfg, ocfg):
     K, W = args.steps, args.warmup
     n_batches = 2 * (W + K)
     host = [synth.batch_for(cfg, dist_util.rank_seed(77, rank), t) for t in range(n_batches)]
+    # the end-to-end leg copies its inputs from pinned host memory: numpy views of pinned tensors (kept alive here)
+    pinned_keep = [tuple(torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).pin_memory() for x in pair) for pair in host]
+    host = [tuple(t.numpy() for t in pair) for pair in pinned_keep]
     dev = [(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for a, b in host[:W + K]]
     groups = [h.group_units(g) for g in range(k)]
 
