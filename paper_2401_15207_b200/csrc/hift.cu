@@ -1149,14 +1149,33 @@ hift_status hift_step_end(hift_ctx* c) {
   return c->first_err == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 
+namespace {
+__global__ void copy_i32_kernel(const int32_t* __restrict__ src, int32_t* __restrict__ dst, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) dst[i] = src[i];
+}
+// A step's token ids and labels are a few kilobytes.  From pinned (or registered) host memory a copy would be a
+// DMA job and could queue on a copy engine behind the gigabytes of optimizer state in flight; a kernel reads such
+// memory directly instead.  From pageable memory the runtime stages the bytes itself and no engine queue is involved.
+void upload_i32(hift_ctx* c, int32_t* dst, const int32_t* src, size_t n) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, src) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer != nullptr) {
+    copy_i32_kernel<<<(unsigned)((n + 255) / 256 < 64 ? (n + 255) / 256 : 64), 256, 0, c->st>>>((const int32_t*)at.devicePointer, dst, n);
+    c->note(cudaGetLastError());
+    return;
+  }
+  cudaGetLastError();
+  c->note(cudaMemcpyAsync(dst, src, n * sizeof(int32_t), cudaMemcpyHostToDevice, c->st));
+}
+}  // namespace
+
 hift_status hift_step_host(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
   if (!c || !tok || !lab) return HIFT_ERR_INPUT;
   const size_t nlab = c->m.arch == 1 ? c->B : c->T;
   for (int i = 0; i < c->T; ++i) if (tok[i] < 0 || tok[i] >= c->V) return HIFT_ERR_INPUT;
   const int nl = c->m.arch == 1 ? c->m.n_classes : c->V;
   for (size_t i = 0; i < nlab; ++i) if (lab[i] >= nl) return HIFT_ERR_INPUT;
-  cudaMemcpyAsync(c->tok_dev, tok, c->T * sizeof(int32_t), cudaMemcpyHostToDevice, c->st);
-  cudaMemcpyAsync(c->lab_dev, lab, nlab * sizeof(int32_t), cudaMemcpyHostToDevice, c->st);
+  upload_i32(c, c->tok_dev, tok, (size_t)c->T);
+  upload_i32(c, c->lab_dev, lab, nlab);
   return do_step(c, c->tok_dev, c->lab_dev, loss_host);
 }
 

@@ -406,3 +406,26 @@ def test_recomputing_frozen_blocks_changes_no_bits_and_saves_memory(arch):
     finally:
         for h in ctxs:
             h.close()
+
+
+def test_host_batches_from_pinned_and_pageable_memory_agree():
+    """hift_step_host takes the batch from pageable memory (staged copy) or from pinned memory (read by a small
+    kernel, so that it cannot queue behind the state transfers on a copy engine): same step either way."""
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(2, synth.DTYPE_BF16)
+    gc, oc = synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
+    p0 = synth.init_params(cfg, 6, perturb=0.05)
+    a, b = HiFT(cfg, gc, oc), HiFT(cfg, gc, oc)
+    try:
+        a.set_params(p0)
+        b.set_params(p0)
+        for t in range(a.num_groups()):
+            tok, lab = synth.batch_for(cfg, 17, t, "zipf")
+            ptok, plab = torch.from_numpy(tok.astype(np.int32)).pin_memory(), torch.from_numpy(lab.astype(np.int32)).pin_memory()
+            assert a.step_host(tok, lab) == b.step_host(ptok.numpy(), plab.numpy())
+        for name in a.tensor_names():
+            assert np.array_equal(a.get_param(name), b.get_param(name)), name
+    finally:
+        a.close()
+        b.close()
