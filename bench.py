@@ -230,10 +230,13 @@ def run_ours(args, cfg, gcfg, ocfg):
     barrier()
     launches = 0
     trained = []
+    step_ms = []
     e0.record()
     for t in range(W, W + K):
         trained.append(h.active_group())
-        h.step(*dev[t])
+        t_host = time.perf_counter()
+        h.step(*dev[t])                      # returns when the step's loss is on the host
+        step_ms.append(round((time.perf_counter() - t_host) * 1e3, 2))
         launches += h.last_step_launches()
     e1.record()
     barrier()
@@ -334,7 +337,7 @@ def run_ours(args, cfg, gcfg, ocfg):
             "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if cfg.dtype == 1 else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "global_batch": cfg.batch * world, "seq_len": cfg.seq,
-                       "groups": k, "groups_trained": trained, "optimizer": ["adamw", "adagrad", "sgdm"][ocfg.kind],
+                       "groups": k, "groups_trained": trained, "ms_by_step": step_ms, "optimizer": ["adamw", "adagrad", "sgdm"][ocfg.kind],
                        "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups, "recompute": ocfg.recompute,
                        "parallelism": (("dp%d" % world) if args.parallel == "dp" else "replicas") if world > 1 else "single",
                        "l2_policy": "inputs larger than L2 (weights + activations of a step exceed 126 MB)"},
