@@ -71,6 +71,12 @@ typedef struct {
   int32_t split_emb_head;    /* 1: embedding | blocks in chunks of m | head        */
   int32_t order;             /* 0 bottom2up, 1 top2down, 2 random (shuffled once)  */
   uint64_t order_seed;       /* seed of the one-time shuffle                       */
+  const int32_t *group_sizes;/* host; NULL = the uniform rule above.  Otherwise n_group_sizes counts of
+                                consecutive units per group, bottom first, each >= 1, summing to
+                                n_blocks + 2 (groups of unequal size: the paper's grouping is uniform,
+                                this is the same fixed partition with the chunk lengths chosen by the
+                                caller); read during hift_create only, not kept            */
+  int32_t n_group_sizes;
 } hift_group_cfg;
 
 /* Optimizer P and schedule eta_t of Algorithm 1's "Require" list; state residency

@@ -67,11 +67,21 @@ def num_groups(n: int, m: int) -> int:
     return n // m if n % m == 0 else n // m + 1
 
 
-def build_groups(n_units: int, m: int, split_emb_head: int = 0) -> List[List[int]]:
+def build_groups(n_units: int, m: int, split_emb_head: int = 0, sizes: Sequence[int] = ()) -> List[List[int]]:
     """Fixed partition of unit ids 0..n-1 (0 = embedding, n-1 = head) into
     consecutive chunks of m, last chunk short.  With split_emb_head the
     embedding and the head are groups of their own and only the blocks are
-    chunked."""
+    chunked.  With `sizes` the chunk lengths are the caller's (the paper's
+    Notation paragraph groups uniformly; an uneven partition keeps every
+    other rule of Algorithm 1: fixed groups, each trained once per cycle)."""
+    if len(sizes) > 0:
+        if any(int(z) < 1 for z in sizes) or sum(int(z) for z in sizes) != n_units:
+            raise ValueError("group sizes must be >= 1 and sum to the number of units")
+        out, u = [], 0
+        for z in sizes:
+            out.append(list(range(u, u + int(z))))
+            u += int(z)
+        return out
     if m < 1:
         raise ValueError("m must be >= 1")
     if split_emb_head:
@@ -632,7 +642,8 @@ class HiFTOracle:
         self.master = {k: np.array(v, dtype=F64) for k, v in params_fp32.items()}
         self.s0 = {k: np.zeros_like(v) for k, v in self.master.items()}
         self.s1 = {k: np.zeros_like(v) for k, v in self.master.items()}
-        self.groups = build_groups(cfg.n_units, gcfg.layers_per_group, gcfg.split_emb_head)
+        self.groups = build_groups(cfg.n_units, gcfg.layers_per_group, gcfg.split_emb_head,
+                                   getattr(gcfg, "group_sizes", ()))
         self.k = len(self.groups)
         self.order = group_order(self.k, gcfg.order, gcfg.order_seed)
         self.t = 0

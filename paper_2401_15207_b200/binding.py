@@ -43,7 +43,8 @@ class ModelCfgC(C.Structure):
 
 class GroupCfgC(C.Structure):
     _fields_ = [("layers_per_group", C.c_int32), ("split_emb_head", C.c_int32),
-                ("order", C.c_int32), ("order_seed", C.c_uint64)]
+                ("order", C.c_int32), ("order_seed", C.c_uint64),
+                ("group_sizes", C.POINTER(C.c_int32)), ("n_group_sizes", C.c_int32)]
 
 
 class OptCfgC(C.Structure):
@@ -155,7 +156,10 @@ class HiFT:
         m = ModelCfgC(model.arch, model.n_blocks, model.d_model, model.n_heads, model.d_ffn,
                       model.vocab, model.max_pos, model.n_classes, model.causal, model.tie_head,
                       model.dtype, model.batch, model.seq, model.norm_eps, model.rope_base)
-        g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed)
+        sizes = tuple(getattr(groups, "group_sizes", None) or ())
+        arr = (C.c_int32 * len(sizes))(*sizes) if sizes else None
+        g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed,
+                      C.cast(arr, C.POINTER(C.c_int32)) if sizes else None, len(sizes))
         o = OptCfgC(opt.kind, opt.sched, opt.total_cycles, opt.offload_state, opt.prefetch_groups,
                     getattr(opt, "recompute", 0), getattr(opt, "warmup_cycles", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
         self._h = C.c_void_p()

@@ -74,6 +74,7 @@ struct hift_ctx {
   std::vector<TensorRec> tens;
   std::vector<std::vector<int>> unit_tens;
   std::vector<GroupRec> groups;
+  std::vector<int> group_sizes;     // caller-chosen chunk lengths (empty = the uniform rule)
   std::vector<int> order;
   std::vector<BlockIdx> bidx;
   int t_tok = -1, t_pos = -1, t_eg = -1, t_eb = -1, t_fg = -1, t_fb = -1, t_wh = -1, t_wc = -1, t_bc = -1;
@@ -246,7 +247,10 @@ void build_layout(hift_ctx* c) {
   // groups: consecutive chunks of m units (paper, Notation), or embedding | chunks | head
   const int n = L + 2, mm = c->gc.layers_per_group;
   std::vector<std::pair<int, int>> spans;
-  if (c->gc.split_emb_head) {
+  if (!c->group_sizes.empty()) {
+    int u = 0;
+    for (int sz : c->group_sizes) { spans.push_back({u, u + sz - 1}); u += sz; }
+  } else if (c->gc.split_emb_head) {
     spans.push_back({0, 0});
     for (int u = 1; u <= L; u += mm) spans.push_back({u, std::min(u + mm - 1, L)});
     spans.push_back({n - 1, n - 1});
@@ -945,12 +949,23 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // the embedding-gradient kernel keeps one occurrence list of <= batch*seq ints in shared memory
   if ((int64_t)m->batch * m->seq > 8192) return HIFT_ERR_CFG;
   if (gc->layers_per_group < 1 || gc->order < 0 || gc->order > 2) return HIFT_ERR_CFG;
+  if (gc->group_sizes != nullptr) {
+    if (gc->n_group_sizes < 1) return HIFT_ERR_CFG;
+    int64_t sum = 0;
+    for (int i = 0; i < gc->n_group_sizes; ++i) {
+      if (gc->group_sizes[i] < 1) return HIFT_ERR_CFG;
+      sum += gc->group_sizes[i];
+    }
+    if (sum != (int64_t)m->n_blocks + 2) return HIFT_ERR_CFG;
+  }
   if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
   if (oc->sched == 1 && (oc->total_cycles < 1 || oc->warmup_cycles < 0 || oc->warmup_cycles >= oc->total_cycles)) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
   hift_ctx* c = new hift_ctx();
   c->m = *m; c->gc = *gc; c->oc = *oc;
+  if (gc->group_sizes != nullptr) c->group_sizes.assign(gc->group_sizes, gc->group_sizes + gc->n_group_sizes);
+  c->gc.group_sizes = nullptr; c->gc.n_group_sizes = 0;   // the caller's array is not kept
   c->caller = (cudaStream_t)cuda_stream;
   c->mixed = m->dtype == 1;
   c->es = c->mixed ? 2 : 4;

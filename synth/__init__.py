@@ -74,6 +74,7 @@ class GroupCfg:
     split_emb_head: int = 0            # 1: embedding | blocks in chunks of m | head
     order: int = ORDER_BOTTOM2UP
     order_seed: int = 0
+    group_sizes: tuple = ()            # non-empty: consecutive units per group, bottom first (overrides m)
 
 
 @dataclass(frozen=True)

@@ -51,6 +51,24 @@ def test_mini_fp32_grouped_and_split(arch):
              FP32_LOSS, FP32_GRAD, resync=True)
 
 
+@pytest.mark.parametrize("arch", [0, 2])
+def test_uneven_caller_chosen_groups(arch):
+    """Groups of unequal size given as a list of chunk lengths: the same step, the partition is the caller's."""
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(arch, synth.DTYPE_FP32, n_blocks=5)                      # 7 units
+    gc = synth.GroupCfg(order=1, group_sizes=(2, 1, 3, 1))
+    rep = lockstep(cfg, gc, synth.OptCfg(kind=0, lr=1e-3, weight_decay=0.01), 6, "zipf", FP32_LOSS, FP32_GRAD,
+                   resync=True)
+    assert [g for _, g, _, _, _ in rep] == [3, 2, 1, 0, 3, 2]
+    cfgb = mini(arch, synth.DTYPE_BF16, n_blocks=5)
+    lockstep(cfgb, synth.GroupCfg(order=0, group_sizes=(1, 4, 2)),
+             synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1), 4, "zipf", BF16_LOSS, BF16_GRAD,
+             resync=True)
+    for bad in [(2, 1, 3), (7, 0), (3, 3, 3)]:
+        with pytest.raises(RuntimeError):
+            HiFT(cfg, synth.GroupCfg(group_sizes=bad), synth.OptCfg())
+
+
 @pytest.mark.parametrize("arch", [0, 1, 2])
 @pytest.mark.parametrize("offload,prefetch", [(0, 0), (1, 0), (1, 1)])
 def test_mini_bf16_paging_modes(arch, offload, prefetch):

@@ -51,6 +51,19 @@ def test_split_grouping_gpt2_large():
     assert groups[1] == [1, 2] and groups[18] == [35, 36]
 
 
+def test_caller_chosen_group_sizes():
+    # the uniform rule written out as sizes gives the uniform partition; an uneven list is a partition of
+    # 0..n-1 into consecutive runs of exactly those lengths; bad lists are refused
+    assert O.build_groups(10, 3, sizes=(3, 3, 3, 1)) == O.build_groups(10, 3)
+    assert O.build_groups(38, 2, 1, sizes=(1,) + (2,) * 18 + (1,)) == O.build_groups(38, 2, 1)
+    g = O.build_groups(7, 1, sizes=(2, 1, 4))
+    assert g == [[0, 1], [2], [3, 4, 5, 6]]
+    assert sorted(u for grp in g for u in grp) == list(range(7))
+    for bad in [(2, 1, 3), (2, 0, 5), (8,)]:
+        with pytest.raises(ValueError):
+            O.build_groups(7, 1, sizes=bad)
+
+
 def test_orders():
     k = 20
     assert O.group_order(k, 0) == list(range(k))
