@@ -127,6 +127,15 @@ hift_status hift_step(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *l
 hift_status hift_step_host(hift_ctx *ctx, const int32_t *tokens_host, const int32_t *labels_host,
                            float *loss_host);
 
+/* Batches of unequal length, padded on the right to `seq` (what fine-tuning on the paper's tasks feeds a
+ * model; the paper does not discuss it): lens_host[b] in [1, seq] is the number of real tokens of batch
+ * entry b.  From the next step on, attention lets every query of entry b see keys 0 .. lens_host[b]-1 only
+ * (on top of the causal mask, if any); NULL switches the table off again.  Padded positions still run
+ * through the model; the caller keeps them out of the loss with label -1 (arch 0, 2; arch 1 reads
+ * token 0 only), and then no gradient flows through them.  The table is copied during the call.
+ * HIFT_ERR_INPUT if a length is out of range. */
+hift_status hift_set_key_lengths(hift_ctx *ctx, const int32_t *lens_host);
+
 /* The same step in two halves, for data-parallel training (several contexts, one per GPU, each
  * on its shard of the batch; the paper's method itself is single-device).  hift_step_begin runs
  * the forward pass and the truncated backward pass and returns the loss; the active group's flat
@@ -254,15 +263,19 @@ hift_status hift_adafactor_step(int64_t rows, int64_t cols, void *param_bf16_dev
 hift_status hift_k_linear(int32_t form, int32_t dtype, int32_t path, int64_t M, int64_t N, int64_t K,
                           const void *a_dev, const void *b_dev, void *out_dev,
                           const void *bias_dev, const float *residual_dev, void *cuda_stream);
-/* qkv[T,3d] (q|k|v column blocks, head h at columns h*d_h) -> o[T,d], lse[B,H,S] fp32. */
+/* qkv[T,3d] (q|k|v column blocks, head h at columns h*d_h) -> o[T,d], lse[B,H,S] fp32.
+ * key_lens_dev: int32 [batch] or NULL; entry b attends to keys 0 .. key_lens[b]-1 only (values are
+ * clamped to [1, seq] on the device). */
 hift_status hift_k_attention_fwd(int32_t dtype, int32_t batch, int32_t seq, int32_t n_heads,
                                  int32_t d_head, int32_t causal, const void *qkv_dev, void *o_dev,
-                                 float *lse_dev, void *cuda_stream);
-/* -> dqkv[T,3d]; dsum_dev is fp32 scratch of batch*seq*n_heads elements. */
+                                 float *lse_dev, const int32_t *key_lens_dev, void *cuda_stream);
+/* -> dqkv[T,3d]; dsum_dev is fp32 scratch of batch*seq*n_heads elements.  Rows of dk, dv at padded
+ * keys are written as zeros. */
 hift_status hift_k_attention_bwd(int32_t dtype, int32_t batch, int32_t seq, int32_t n_heads,
                                  int32_t d_head, int32_t causal, const void *qkv_dev,
                                  const void *o_dev, const float *lse_dev, const void *do_dev,
-                                 void *dqkv_dev, float *dsum_dev, void *cuda_stream);
+                                 void *dqkv_dev, float *dsum_dev, const int32_t *key_lens_dev,
+                                 void *cuda_stream);
 /* Rotary models (RoPE on q and k, as in the LLaMA-shaped configuration the paper profiles) on the
  * tensor-core path: the rotation is fused into the epilogue of the qkv projection, and this hook
  * exposes exactly that kernel: out[M,N] = rope(x[M,K] w[N,K]^T + bias) on columns [0, rope_cols),

@@ -247,14 +247,21 @@ def rope_apply(x, cos, sin, inverse=False):
     return np.concatenate([x1 * c - x2 * s, x1 * s + x2 * c], axis=-1)
 
 
-def attention_fwd(q, k, v, causal: bool):
-    """q,k,v: [B, S, H, d_h] -> o [B, S, H, d_h]; softmax(q k^T / sqrt(d_h) + mask) v."""
+def attention_fwd(q, k, v, causal: bool, lens=None):
+    """q,k,v: [B, S, H, d_h] -> o [B, S, H, d_h]; softmax(q k^T / sqrt(d_h) + mask) v.
+    lens (optional, [B] ints in 1..S): batch entry b is a sequence of lens[b] real
+    tokens padded on the right; keys at positions >= lens[b] get probability 0
+    (the usual key-padding mask of the models the paper fine-tunes; the paper
+    itself does not describe batching)."""
     B, S, H, dh = q.shape
     qh, kh, vh = (t.transpose(0, 2, 1, 3) for t in (q, k, v))      # [B,H,S,dh]
     s = np.matmul(qh, kh.transpose(0, 1, 3, 2)) / math.sqrt(dh)
     if causal:
         mask = np.triu(np.ones((S, S), dtype=bool), k=1)
         s = np.where(mask, -np.inf, s)
+    if lens is not None:
+        pad = np.arange(S)[None, :] >= np.asarray(lens).reshape(B, 1)          # [B, S] True at padded keys
+        s = np.where(pad[:, None, None, :], -np.inf, s)
     s = s - s.max(axis=-1, keepdims=True)
     p = np.exp(s)
     p = p / p.sum(axis=-1, keepdims=True)
@@ -328,7 +335,7 @@ def _merge_heads(t):
     return t.reshape(B, S, H * dh)
 
 
-def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarray):
+def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarray, lens=None):
     """Whole-model forward in fp64.  Returns (loss, cache)."""
     B, S = tokens.shape
     d, H = cfg.d_model, cfg.n_heads
@@ -351,7 +358,7 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             h1, c["ln1"] = layernorm_fwd(x, P[p + "ln1_g"], P[p + "ln1_b"], eps)
             qkv = h1 @ P[p + "w_qkv"].T + P[p + "b_qkv"]
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
-            o, prob = attention_fwd(q, k, v, causal)
+            o, prob = attention_fwd(q, k, v, causal, lens)
             om = _merge_heads(o)
             x2 = x + om @ P[p + "w_o"].T + P[p + "b_o"]
             h2, c["ln2"] = layernorm_fwd(x2, P[p + "ln2_g"], P[p + "ln2_b"], eps)
@@ -363,7 +370,7 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
         elif cfg.arch == 1:        # post-LN: x = LN1(x + Attn x); x = LN2(x + FFN x)
             qkv = x @ P[p + "w_qkv"].T + P[p + "b_qkv"]
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
-            o, prob = attention_fwd(q, k, v, causal)
+            o, prob = attention_fwd(q, k, v, causal, lens)
             om = _merge_heads(o)
             y = x + om @ P[p + "w_o"].T + P[p + "b_o"]
             x1, c["ln1"] = layernorm_fwd(y, P[p + "ln1_g"], P[p + "ln1_b"], eps)
@@ -379,7 +386,7 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
             q = rope_apply(q, cos, sin)
             k = rope_apply(k, cos, sin)
-            o, prob = attention_fwd(q, k, v, causal)
+            o, prob = attention_fwd(q, k, v, causal, lens)
             om = _merge_heads(o)
             x2 = x + om @ P[p + "w_o"].T
             h2, c["rms2"] = rmsnorm_fwd(x2, P[p + "rms2_g"], eps)
@@ -667,11 +674,11 @@ class HiFTOracle:
     def group_tensor_names(self, g: int) -> List[str]:
         return [n for u in self.groups[g] for n in tensor_names_of_unit(self.cfg, u)]
 
-    def step(self, tokens: np.ndarray, labels: np.ndarray) -> float:
+    def step(self, tokens: np.ndarray, labels: np.ndarray, lens=None) -> float:
         g = self.active_group()
         lr = self.current_lr()
         P = self.model_params()
-        loss, cache = forward(self.cfg, P, tokens, labels)
+        loss, cache = forward(self.cfg, P, tokens, labels, lens)
         grads = backward(self.cfg, P, cache, active_units=self.groups[g])
         self.tau[g] += 1
         o = self.ocfg

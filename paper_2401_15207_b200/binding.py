@@ -64,6 +64,7 @@ def _prototypes():
         "hift_destroy": (None, [vp]),
         "hift_step": (C.c_int, [vp, vp, vp, pf]),
         "hift_step_host": (C.c_int, [vp, vp, vp, pf]),
+        "hift_set_key_lengths": (C.c_int, [vp, vp]),
         "hift_step_begin": (C.c_int, [vp, vp, vp, pf]),
         "hift_grad_view": (C.c_int, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "hift_step_end": (C.c_int, [vp]),
@@ -95,8 +96,8 @@ def _prototypes():
         "hift_tc_error_flag": (i32, [i32]),
         "hift_opt_step": (C.c_int, [i32, sz, vp, vp, vp, vp, vp, f64, f64, f64, f64, f64, f64, i64, vp]),
         "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
-        "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
-        "hift_k_attention_bwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+        "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
+        "hift_k_attention_bwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
         "hift_k_linear_rope": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, i64, vp]),
         "hift_k_linear_swiglu": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_linear_dx_swiglu_bwd": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp]),
@@ -194,6 +195,16 @@ class HiFT:
         st = lib().hift_step(self._h, tokens.data_ptr(), labels.data_ptr(), C.byref(loss))
         _check(st, "hift_step")
         return loss.value
+
+    def set_key_lengths(self, lens) -> None:
+        """lens: batch ints in [1, seq] (real tokens per right-padded batch entry), or None for no padding."""
+        if lens is None:
+            _check(lib().hift_set_key_lengths(self._h, None), "hift_set_key_lengths")
+            return
+        a = np.ascontiguousarray(lens, dtype=np.int32)
+        if a.shape != (self.model.batch,):
+            raise ValueError("one length per batch entry")
+        _check(lib().hift_set_key_lengths(self._h, a.ctypes.data), "hift_set_key_lengths")
 
     def step_host(self, tokens: np.ndarray, labels: np.ndarray) -> float:
         tokens = np.ascontiguousarray(tokens, dtype=np.int32)
@@ -357,14 +368,14 @@ def k_linear(form, dtype, M, N, K, a, b, out, bias=None, residual=None, path=0, 
                                _ptr(residual), _st(stream)), "hift_k_linear")
 
 
-def k_attention_fwd(dtype, B, S, H, dh, causal, qkv, o, lse, stream=None):
-    _check(lib().hift_k_attention_fwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _st(stream)),
-           "hift_k_attention_fwd")
+def k_attention_fwd(dtype, B, S, H, dh, causal, qkv, o, lse, stream=None, key_lens=None):
+    _check(lib().hift_k_attention_fwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(key_lens),
+                                      _st(stream)), "hift_k_attention_fwd")
 
 
-def k_attention_bwd(dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, stream=None):
+def k_attention_bwd(dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, stream=None, key_lens=None):
     _check(lib().hift_k_attention_bwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout),
-                                      _ptr(dqkv), _ptr(dsum), _st(stream)), "hift_k_attention_bwd")
+                                      _ptr(dqkv), _ptr(dsum), _ptr(key_lens), _st(stream)), "hift_k_attention_bwd")
 
 
 def k_linear_rope(M, N, K, a, b, out, bias, cs, seq, d_head, rope_cols, stream=None):

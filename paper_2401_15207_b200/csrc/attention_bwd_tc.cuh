@@ -79,7 +79,7 @@ __device__ __forceinline__ void tmem_ld_wait32(uint32_t (&v)[32]) {
 //              common case carries no comparisons)
 template <int MODE, bool MASKED>
 __device__ __forceinline__ void ab_p_ds16(const uint32_t (&sv)[16], const uint32_t (&pv)[16], float col_l2, float col_d,
-                                          int lane_base, float row_l2, float row_d, float sl2, int S, int causal,
+                                          int lane_base, float row_l2, float row_d, float sl2, int S, int klen, int causal,
                                           int frow, int x_first, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8]) {
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
@@ -92,7 +92,7 @@ __device__ __forceinline__ void ab_p_ds16(const uint32_t (&sv)[16], const uint32
       if (MASKED) {
         const int xi = x_first + i + e;
         const int key = MODE == 0 ? frow : xi, qry = MODE == 0 ? xi : frow;
-        if (key >= S || qry >= S || (causal && key > qry)) p = 0.f;
+        if (key >= klen || qry >= S || (causal && key > qry)) p = 0.f;
       }
       pp[e] = p;
       dd[e] = p * (__uint_as_float(pv[i + e]) - dv);
@@ -109,7 +109,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
                    const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1,
                    int col_f0, int col_f1, int col_x0, int col_x1,      // column of head 0 in each tensor
                    const float* __restrict__ lse, const float* __restrict__ dsum,
-                   __nv_bfloat16* __restrict__ dqkv, int B, int S, int H, int causal, float scale) {
+                   __nv_bfloat16* __restrict__ dqkv, int B, int S, int H, int causal, float scale,
+                   const int* __restrict__ lens) {
   typedef AttnBwdCfg<DH, MODE> Cfg;
   constexpr int SP = DH / 64;                            // 64-column swizzle spans per tile row
   constexpr int FSPAN = kAbF * 128, XSPAN = kAbX * 128;  // bytes of one span of a fixed / streamed tile
@@ -309,6 +310,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       const Item it = item_of(idx);
       const int f0 = it.f0, row_g0 = it.b * S;
       const int frow = f0 + r;                            // key (MODE 0) / query (MODE 1) index in the sequence
+      const int klen = tc_key_len(lens, it.b, S);         // keys at or after klen are padding: P = dS = 0 there
       const float* lse_bh = lse + ((int64_t)it.b * H + it.h) * S;
       const float* dsum_bh = dsum + ((int64_t)it.b * H + it.h) * S;
       float row_l2 = 0.f, row_d = 0.f;                    // MODE 1: this query's lse * log2(e) and D
@@ -332,7 +334,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
         // masking is needed only where the block touches the diagonal or the end of the sequence
         const int k_hi = MODE == 0 ? f0 + kAbF - 1 : xb0 + kAbX - 1;      // largest key of the block
         const int q_lo = MODE == 0 ? xb0 : f0;                            // smallest query of the block
-        const bool masked = (causal && k_hi > q_lo) || f0 + kAbF > S || xb0 + kAbX > S;
+        const bool masked = (causal && k_hi > q_lo) || f0 + kAbF > S || xb0 + kAbX > S || k_hi >= klen;
         bool ready = mbar_wait(s_full(u), par);
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 9);
         tc_fence_after();
@@ -360,8 +362,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
             if (lane == 0) mbar_arrive(s_free(u));        // the tensor core may overwrite tS / tP [u]
           }
           uint32_t pk_p[8], pk_ds[8];
-          if (masked) ab_p_ds16<MODE, true>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, causal, frow, xb0 + cb, pk_p, pk_ds);
-          else ab_p_ds16<MODE, false>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, causal, frow, xb0 + cb, pk_p, pk_ds);
+          if (masked) ab_p_ds16<MODE, true>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds);
+          else ab_p_ds16<MODE, false>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds);
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             const int chunk = hc * 4 + hf * 2 + c;

@@ -61,10 +61,16 @@ __device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr, uint32_t box_byt
          (1ull << 46) | (2ull << 61);
 }
 
+// Key padding: batch entry b attends to keys 0 .. lens[b]-1 only (clamped to [1, S]); null = all S keys.
+__device__ __forceinline__ int tc_key_len(const int* __restrict__ lens, int b, int S) {
+  return lens != nullptr ? max(1, min(lens[b], S)) : S;
+}
+
 template <int DH>
 __global__ void __launch_bounds__(kAttThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* __restrict__ o,
-                   float* __restrict__ lse, int B, int S, int H, int causal, float scale) {
+                   float* __restrict__ lse, int B, int S, int H, int causal, float scale,
+                   const int* __restrict__ lens) {
   typedef AttnTcCfg<DH> Cfg;
   constexpr int SP = Cfg::kSpans;
   constexpr int SPAN_BYTES = 128 * 128;                 // 128 rows x 64 elements x 2 bytes
@@ -96,14 +102,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
 
   // work items, heaviest first; every role walks the same list and counts key blocks (g)
   const int nqb = (S + kAttBQ - 1) / kAttBQ, nbh = B * H, nitems = nqb * nbh;
-  struct Item { int b, h, q0, nblk; };
+  struct Item { int b, h, q0, nblk, klen; };
   auto item_of = [&](int idx) {
     Item it;
     const int rank = idx / nbh, bh = idx - rank * nbh;
     it.b = bh / H;
     it.h = bh - it.b * H;
     it.q0 = (causal ? nqb - 1 - rank : rank) * kAttBQ;
-    const int kv_len = causal ? min(S, it.q0 + kAttBQ) : S;
+    it.klen = tc_key_len(lens, it.b, S);                // keys at or after klen are padding
+    const int kv_len = min(causal ? min(S, it.q0 + kAttBQ) : S, it.klen);
     it.nblk = (kv_len + kAttBK - 1) / kAttBK;
     return it;
   };
@@ -246,7 +253,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
     int g = 0, n = 0;
     for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
       const Item it = item_of(idx);
-      const int q0 = it.q0, qrow = q0 + r, row_g0 = it.b * S;
+      const int q0 = it.q0, qrow = q0 + r, row_g0 = it.b * S, klen = it.klen;
       const uint32_t tO = tmem_base + 256u + (uint32_t)((n & 1) * 128);
       float m = -INFINITY, l = 0.f;                     // m: the row's reference maximum (same in both threads); l: this half's sum
       for (int j = 0; j < it.nblk; ++j, ++g) {
@@ -269,11 +276,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
         __syncwarp();
         if (lane == 0) mbar_arrive(s_free(st));         // the tensor core may overwrite this score buffer
         // masking only where the block touches the diagonal or the end of the sequence (uniform per CTA)
-        if ((causal && j * kAttBK + kAttBK - 1 > q0) || (j + 1) * kAttBK > S) {
+        if ((causal && j * kAttBK + kAttBK - 1 > q0) || (j + 1) * kAttBK > klen) {
 #pragma unroll
           for (int i = 0; i < HB; ++i) {
             const int key = j * kAttBK + half * HB + i;
-            if (key >= S || (causal && key > qrow)) sc[i] = -INFINITY;
+            if (key >= klen || (causal && key > qrow)) sc[i] = -INFINITY;
           }
         }
         // four independent chains each for the maximum and the sum

@@ -109,4 +109,10 @@ __device__ __forceinline__ float block_max(float v, float* red) {
   return red[32];
 }
 
+// Key padding: attention of batch row b sees keys 0 .. lens[b]-1 only (clamped to [1, S]); a null
+// table means every row has all S keys.
+__device__ __forceinline__ int key_len_of(const int* __restrict__ lens, int b, int S) {
+  return lens != nullptr ? max(1, min(lens[b], S)) : S;
+}
+
 }  // namespace hift

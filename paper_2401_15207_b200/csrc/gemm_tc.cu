@@ -1045,7 +1045,8 @@ bool attn_tc_eligible(int dh, const void* qkv, int H) {
   // head sizes 64 and 128 (HIFT_ATTN_TC=0 sends both to the warp-level kernel)
   return g_init_state == 0 && g_attn_tc && (dh == 128 || dh == 64) && (((uintptr_t)qkv) & 15) == 0 && ((3 * H * dh) % 8) == 0;
 }
-cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse) {
+cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse,
+                               const int* lens) {
   CUtensorMap tm;
   const uint64_t d3 = 3ull * H * dh;
   if (!get_map(qkv, d3, (uint64_t)B * S, d3, 128, &tm)) return cudaErrorInvalidValue;
@@ -1053,8 +1054,8 @@ cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int
   const int grid = nitems < g_num_sms ? nitems : g_num_sms;          // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)dh);
   if (dh == 64)
-    return launch_pdl_tc(attn_fwd_tc_kernel<64>, dim3(grid), dim3(kAttThreads), AttnTcCfg<64>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
-  return launch_pdl_tc(attn_fwd_tc_kernel<128>, dim3(grid), dim3(kAttThreads), AttnTcCfg<128>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale);
+    return launch_pdl_tc(attn_fwd_tc_kernel<64>, dim3(grid), dim3(kAttThreads), AttnTcCfg<64>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale, lens);
+  return launch_pdl_tc(attn_fwd_tc_kernel<128>, dim3(grid), dim3(kAttThreads), AttnTcCfg<128>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale, lens);
 }
 
 bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, const void* dqkv) {
@@ -1063,7 +1064,7 @@ bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, cons
 }
 template <int DH>
 static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, const void* dout,
-                                    const float* lse, const float* dsum, void* dqkv) {
+                                    const float* lse, const float* dsum, void* dqkv, const int* lens) {
   const uint64_t d = (uint64_t)H * DH, d3 = 3 * d, rows = (uint64_t)B * S;
   CUtensorMap qkv_f, qkv_x, do_f, do_x;
   if (!get_map(qkv, d3, rows, d3, kAbF, &qkv_f) || !get_map(qkv, d3, rows, d3, kAbX, &qkv_x) ||
@@ -1074,16 +1075,16 @@ static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int ca
   const float scale = 1.0f / sqrtf((float)DH);
   // dK, dV: fixed K, V; streamed Q, dO
   cudaError_t e = launch_pdl_tc(attn_bwd_tc_kernel<DH, 0>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 0>::kSmem, st,
-      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale);
+      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale, lens);
   if (e != cudaSuccess) return e;
   // dQ: fixed Q, dO; streamed K, V
   return launch_pdl_tc(attn_bwd_tc_kernel<DH, 1>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 1>::kSmem, st,
-      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale);
+      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale, lens);
 }
 cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,
-                               const float* lse, const float* dsum, void* dqkv) {
-  if (dh == 64) return attn_tc_bwd_inst<64>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv);
-  return attn_tc_bwd_inst<128>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv);
+                               const float* lse, const float* dsum, void* dqkv, const int* lens) {
+  if (dh == 64) return attn_tc_bwd_inst<64>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv, lens);
+  return attn_tc_bwd_inst<128>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv, lens);
 }
 
 int gemm_tc_set_error(int v) {

@@ -15,13 +15,15 @@ int gemm_tc_init();
 bool gemm_tc_eligible(const GemmArgs& g);
 cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g);
 // Attention forward on tcgen05 (scores and output in tensor memory): bf16, head size 64 or 128.
+// `lens` (device, [B], may be null): batch entry b attends to its first lens[b] keys only.
 bool attn_tc_eligible(int dh, const void* qkv, int H);
-cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse);
+cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse,
+                               const int* lens);
 // Attention backward on tcgen05 (two launches: dK/dV, then dQ): bf16, head size 64 or 128.  `dsum` holds
 // rowsum(dO o O) per (batch, head, query); qkv, dout and dqkv must be 16-byte aligned.
 bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, const void* dqkv);
 cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,
-                               const float* lse, const float* dsum, void* dqkv);
+                               const float* lse, const float* dsum, void* dqkv, const int* lens);
 // 0 if no tensor-core kernel has given up on a bounded wait since the library was loaded, else the
 // code of the first one (1 producer, 2 MMA issuer, 3 epilogue); -1 if the flag cannot be read.
 int gemm_tc_poll_error();

@@ -104,6 +104,8 @@ struct hift_ctx {
   bool d2h_pending[2] = {false, false};
   // fixed work buffers
   int32_t *tok_dev = nullptr, *lab_dev = nullptr;
+  int32_t* lens_dev = nullptr;      // [B] valid keys per batch entry (key padding), used while use_lens
+  bool use_lens = false;
   float *dxa = nullptr, *dxb = nullptr;             // residual-stream gradients (fp32)
   char *dxa_a = nullptr, *dxb_a = nullptr;          // the same, rounded once to the operand type
   char *dt1 = nullptr, *dqkv = nullptr, *dbig = nullptr, *dsw = nullptr;
@@ -406,13 +408,14 @@ void bias_grad(hift_ctx* c, const void* dy, bool dy_f32, int64_t rows, int cols,
 void attn_fwd(hift_ctx* c, const void* qkv, void* o, float* lse) {
   const double work = 4.0 * c->B * c->H * (double)c->S * c->S * c->dh * (c->m.causal ? 0.5 : 1.0);
   LAUNCH(HIFT_K_ATTN_FWD, work,
-         launch_attention_fwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse));
+         launch_attention_fwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse,
+                              c->use_lens ? c->lens_dev : nullptr));
 }
 void attn_bwd(hift_ctx* c, const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv) {
   const double work = 10.0 * c->B * c->H * (double)c->S * c->S * c->dh * (c->m.causal ? 0.5 : 1.0);
   LAUNCH(HIFT_K_ATTN_BWD, work,
          launch_attention_bwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse,
-                              dout, dqkv, c->dsum));
+                              dout, dqkv, c->dsum, c->use_lens ? c->lens_dev : nullptr));
   c->step_launches += attention_use_mma(c->mixed, c->dh) ? 2 : 1;   // dsum, dq, dkv or dq, dkv
 }
 // qkv projection of a rotary model: on the tensor-core path the rotation of the q and k column blocks
@@ -1067,7 +1070,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     for (auto& r : c->tens) mx = std::max(mx, af_scratch_floats(r.rows, r.cols));
     if ((rc = dev_alloc(c, (void**)&c->af_scratch, mx * sizeof(float))) != HIFT_OK) return fail(rc);
   }
-  if (cudaHostAlloc((void**)&c->scal_host, 4 * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
+  // four scalars the step publishes, then a staging row for the key-length table
+  if (cudaHostAlloc((void**)&c->scal_host, (4 + (size_t)c->B) * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
   if (cudaHostGetDevicePointer((void**)&c->scal_host_dev, c->scal_host, 0) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
   // ---- activation arena: fixed work buffers, one scratch copy of every slot, then the
@@ -1078,6 +1082,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     c->arena_off = 0;
     c->tok_dev = (int32_t*)arena_take(c, T * sizeof(int32_t));
     c->lab_dev = (int32_t*)arena_take(c, T * sizeof(int32_t));
+    c->lens_dev = (int32_t*)arena_take(c, (size_t)c->B * sizeof(int32_t));
     c->dxa = (float*)arena_take(c, T * d * 4); c->dxb = (float*)arena_take(c, T * d * 4);
     c->dxa_a = arena_take(c, T * d * es); c->dxb_a = arena_take(c, T * d * es); c->dt1 = arena_take(c, T * d * es);
     c->dqkv = arena_take(c, T * 3 * d * es);
@@ -1182,6 +1187,20 @@ void upload_i32(hift_ctx* c, int32_t* dst, const int32_t* src, size_t n) {
   c->note(cudaMemcpyAsync(dst, src, n * sizeof(int32_t), cudaMemcpyHostToDevice, c->st));
 }
 }  // namespace
+
+hift_status hift_set_key_lengths(hift_ctx* c, const int32_t* lens_host) {
+  if (!c) return HIFT_ERR_INPUT;
+  if (c->pending_update) return HIFT_ERR_CFG;            // not between the two halves of a step
+  if (lens_host == nullptr) { c->use_lens = false; return HIFT_OK; }
+  for (int b = 0; b < c->B; ++b) if (lens_host[b] < 1 || lens_host[b] > c->S) return HIFT_ERR_INPUT;
+  c->note(cudaStreamSynchronize(c->st));                 // nothing enqueued earlier still reads the staging row
+  memcpy(c->scal_host + 4, lens_host, (size_t)c->B * sizeof(int32_t));
+  copy_i32_kernel<<<1, 256, 0, c->st>>>((const int32_t*)(c->scal_host_dev + 4), c->lens_dev, (size_t)c->B);
+  c->note(cudaGetLastError());
+  c->note(cudaStreamSynchronize(c->st));
+  c->use_lens = c->first_err == cudaSuccess;
+  return c->use_lens ? HIFT_OK : HIFT_ERR_CUDA;
+}
 
 hift_status hift_step_host(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
   if (!c || !tok || !lab) return HIFT_ERR_INPUT;
@@ -1569,16 +1588,16 @@ hift_status hift_k_linear_dx_gelu_bwd(int64_t M, int64_t N, int64_t f, const voi
   return gemm_tc_launch((cudaStream_t)stream, g) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_k_attention_fwd(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
-                                 const void* qkv, void* o, float* lse, void* stream) {
+                                 const void* qkv, void* o, float* lse, const int32_t* key_lens, void* stream) {
   if (!attention_head_ok(dh) || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
-  launch_attention_fwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse);
+  launch_attention_fwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, key_lens);
   return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_k_attention_bwd(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
                                  const void* qkv, const void* o, const float* lse, const void* dout,
-                                 void* dqkv, float* dsum, void* stream) {
+                                 void* dqkv, float* dsum, const int32_t* key_lens, void* stream) {
   if (!attention_head_ok(dh) || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
-  launch_attention_bwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum);
+  launch_attention_bwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, key_lens);
   return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_k_linear_rope(int64_t M, int64_t N, int64_t K, const void* a, const void* b, void* out, const void* bias,

@@ -38,11 +38,12 @@ __device__ __forceinline__ void stage_rows(float (*dst)[DH], const T* __restrict
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 attention_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o, float* __restrict__ lse,
-                     int S, int H, int causal, float scale) {
+                     int S, int H, int causal, float scale, const int* __restrict__ lens) {
   constexpr int E = DH / 4;
   __shared__ float Ks[kAttTile][DH];
   __shared__ float Vs[kAttTile][DH];
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kAttRows;
+  const int klen = key_len_of(lens, b, S);
   const int d = H * DH;
   const int p = threadIdx.x & 3, r = threadIdx.x >> 2;
   const int qrow = q0 + r;
@@ -58,7 +59,7 @@ attention_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o, float* __rest
   }
   float m = -INFINITY, l = 0.f;
   const int q_last = min(q0 + kAttRows, S) - 1;
-  const int k_end = causal ? q_last + 1 : S;
+  const int k_end = min(causal ? q_last + 1 : S, klen);
   for (int k0 = 0; k0 < k_end; k0 += kAttTile) {
     const int nk = min(kAttTile, S - k0);
     __syncthreads();
@@ -71,7 +72,7 @@ attention_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o, float* __rest
       for (int i = 0; i < E; ++i) s = fmaf(q[i], Ks[j][4 * i + p], s);
       s = quad_sum(s);
       const int key = k0 + j;
-      if (active && (!causal || key <= qrow)) {
+      if (active && key < klen && (!causal || key <= qrow)) {
         const float mn = fmaxf(m, s);
         const float corr = expf(m - mn);
         const float pj = expf(s - mn);
@@ -97,11 +98,12 @@ __global__ void __launch_bounds__(256)
 attention_bwd_dq_kernel(const T* __restrict__ qkv, const T* __restrict__ o,
                         const float* __restrict__ lse, const T* __restrict__ dout,
                         T* __restrict__ dqkv, float* __restrict__ dsum, int S, int H, int causal,
-                        float scale) {
+                        float scale, const int* __restrict__ lens) {
   constexpr int E = DH / 4;
   __shared__ float Ks[kAttTile][DH];
   __shared__ float Vs[kAttTile][DH];
   const int b = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * kAttRows;
+  const int klen = key_len_of(lens, b, S);
   const int d = H * DH;
   const int p = threadIdx.x & 3, r = threadIdx.x >> 2;
   const int qrow = q0 + r;
@@ -128,7 +130,7 @@ attention_bwd_dq_kernel(const T* __restrict__ qkv, const T* __restrict__ o,
   D = quad_sum(D);
   if (active && p == 0) dsum[((int64_t)b * H + h) * S + qrow] = D;
   const int q_last = min(q0 + kAttRows, S) - 1;
-  const int k_end = causal ? q_last + 1 : S;
+  const int k_end = min(causal ? q_last + 1 : S, klen);
   for (int k0 = 0; k0 < k_end; k0 += kAttTile) {
     const int nk = min(kAttTile, S - k0);
     __syncthreads();
@@ -145,7 +147,7 @@ attention_bwd_dq_kernel(const T* __restrict__ qkv, const T* __restrict__ o,
       s = quad_sum(s);
       dp = quad_sum(dp);
       const int key = k0 + j;
-      if (active && (!causal || key <= qrow)) {
+      if (active && key < klen && (!causal || key <= qrow)) {
         const float ds = expf(s - L) * (dp - D);
 #pragma unroll
         for (int i = 0; i < E; ++i) dq[i] = fmaf(ds, Ks[j][4 * i + p], dq[i]);
@@ -164,12 +166,14 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 attention_bwd_dkv_kernel(const T* __restrict__ qkv, const float* __restrict__ lse,
                          const T* __restrict__ dout, const float* __restrict__ dsum,
-                         T* __restrict__ dqkv, int S, int H, int causal, float scale) {
+                         T* __restrict__ dqkv, int S, int H, int causal, float scale,
+                         const int* __restrict__ lens) {
   constexpr int E = DH / 4;
   __shared__ float Qs[kAttTile][DH];
   __shared__ float Gs[kAttTile][DH];
   __shared__ float Ls[kAttTile], Ds[kAttTile];
   const int b = blockIdx.z, h = blockIdx.y, kr0 = blockIdx.x * kAttRows;
+  const int klen = key_len_of(lens, b, S);
   const int d = H * DH;
   const int p = threadIdx.x & 3, r = threadIdx.x >> 2;
   const int krow = kr0 + r;
@@ -207,7 +211,7 @@ attention_bwd_dkv_kernel(const T* __restrict__ qkv, const float* __restrict__ ls
       s = quad_sum(s);
       dp = quad_sum(dp);
       const int qrow = q0 + j;
-      if (active && (!causal || krow <= qrow)) {
+      if (active && krow < klen && (!causal || krow <= qrow)) {
         const float pr = expf(s * scale - Ls[j]);
         const float ds = pr * (dp - Ds[j]);
 #pragma unroll

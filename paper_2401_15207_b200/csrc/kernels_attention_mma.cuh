@@ -96,7 +96,7 @@ constexpr int attn_fwd_smem_bytes() { return 4 * 64 * DH * 2; }
 template <int DH>
 __global__ void __launch_bounds__(128, 3)
 attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* __restrict__ lse,
-                    int S, int H, int causal, float scale) {
+                    int S, int H, int causal, float scale, const int* __restrict__ lens) {
   constexpr int BQ = 64, BKV = 64, KS = DH / 16;
   constexpr int TB = BKV * DH * 2;                    // bytes of one K or V tile
   extern __shared__ __align__(128) uint8_t smem_att[];   // K[2] | V[2]; Q is staged through V[1] first
@@ -124,7 +124,8 @@ attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* _
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
   const float sl2 = scale * kLog2e;
   const int row_lo = q0 + warp * 16 + g;              // this thread's rows: row_lo, row_lo + 8
-  const int k_end = causal ? min(S, q0 + BQ) : S;
+  const int klen = key_len_of(lens, b, S);             // keys at or after klen are padding
+  const int k_end = min(causal ? min(S, q0 + BQ) : S, klen);
 
   stage_tile_async<BKV, DH>(tKb, kb, 3 * d, 0, S);
   stage_tile_async<BKV, DH>(tVb, vb, 3 * d, 0, S);
@@ -163,7 +164,7 @@ attn_fwd_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o, float* _
         const int col = k0 + i * 8 + 2 * t + (e & 1);
         const int row = row_lo + (e >> 1) * 8;
         float v = sacc[i][e] * sl2;
-        if (col >= S || (causal && col > row)) v = -INFINITY;
+        if (col >= klen || (causal && col > row)) v = -INFINITY;
         sacc[i][e] = v;
         mx[e >> 1] = fmaxf(mx[e >> 1], v);
       }
@@ -270,7 +271,8 @@ template <int DH>
 __global__ void __launch_bounds__(128)
 attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse,
                        const bf16* __restrict__ dout, const float* __restrict__ dsum,
-                       bf16* __restrict__ dqkv, int S, int H, int causal, float scale) {
+                       bf16* __restrict__ dqkv, int S, int H, int causal, float scale,
+                       const int* __restrict__ lens) {
   constexpr int BQ = 64, BKV = 32, KS = DH / 16;
   constexpr int TB = BKV * DH * 2;
   __shared__ __align__(128) uint8_t sX[BQ * DH * 2];       // q tile, then do tile (fragments are kept in registers)
@@ -287,7 +289,8 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
   const uint32_t tKb = (uint32_t)__cvta_generic_to_shared(sK);
   const uint32_t tVb = (uint32_t)__cvta_generic_to_shared(sV);
 
-  const int k_end = causal ? min(S, q0 + BQ) : S;
+  const int klen = key_len_of(lens, b, S);             // keys at or after klen are padding
+  const int k_end = min(causal ? min(S, q0 + BQ) : S, klen);
   stage_tile_async<BKV, DH>(tKb, kb, 3 * d, 0, S);         // first K/V tile streams in behind the Q / dO staging
   stage_tile_async<BKV, DH>(tVb, vb, 3 * d, 0, S);
   cp_async_commit();
@@ -356,7 +359,7 @@ attn_bwd_dq_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ l
         const int col = k0 + i * 8 + 2 * t + (e & 1);
         const int row = row_lo + (e >> 1) * 8;
         float ds = 0.f;
-        if (col < S && row < S && !(causal && col > row)) {
+        if (col < klen && row < S && !(causal && col > row)) {
           const float p = exp2f(sacc[i][e] * sl2 - L2[e >> 1]);
           ds = p * (pacc[i][e] - Dr[e >> 1]);
         }
@@ -401,7 +404,8 @@ template <int DH>
 __global__ void __launch_bounds__(128)
 attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse,
                         const bf16* __restrict__ dout, const float* __restrict__ dsum,
-                        bf16* __restrict__ dqkv, int S, int H, int causal, float scale) {
+                        bf16* __restrict__ dqkv, int S, int H, int causal, float scale,
+                        const int* __restrict__ lens) {
   constexpr int BKV = 64, BQ = 32, KS = DH / 16;
   extern __shared__ __align__(128) uint8_t smem_dkv[];
   uint8_t* sK = smem_dkv;
@@ -435,6 +439,7 @@ attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ 
   const float sl2 = scale * kLog2e;
   const int key_lo = kr0 + warp * 16 + g;             // this thread's key rows: key_lo, key_lo + 8
   const int q_begin = causal ? (kr0 / BQ) * BQ : 0;
+  const int klen = key_len_of(lens, b, S);             // keys at or after klen are padding: dk = dv = 0
 
   // per query tile: Q and dO rows through cp.async, LSE and dsum with plain loads, all double-buffered
   auto prefetch = [&](int q0, int bf) {
@@ -493,7 +498,7 @@ attn_bwd_dkv_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ 
         const int qrow = q0 + qc;
         const int key = key_lo + (e >> 1) * 8;
         float p = 0.f, ds = 0.f;
-        if (qrow < S && key < S && !(causal && key > qrow)) {
+        if (qrow < S && key < klen && !(causal && key > qrow)) {
           p = exp2f(sacc[i][e] * sl2 - sL[qc]);
           ds = p * (pacc[i][e] - sD[qc]);
         }

@@ -46,21 +46,21 @@ inline bool attention_head_ok(int dh) { return dh == 8 || dh == 16 || dh == 32 |
 
 template <typename T, int DH>
 inline void attention_fwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv,
-                               void* o, float* lse) {
+                               void* o, float* lse, const int* lens) {
   dim3 grid((S + kAttRows - 1) / kAttRows, H, B);
   attention_fwd_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, (T*)o, lse, S, H, causal,
-                                                    1.0f / sqrtf((float)DH));
+                                                    1.0f / sqrtf((float)DH), lens);
 }
 template <typename T, int DH>
 inline void attention_bwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv,
                                const void* o, const float* lse, const void* dout, void* dqkv,
-                               float* dsum) {
+                               float* dsum, const int* lens) {
   dim3 grid((S + kAttRows - 1) / kAttRows, H, B);
   const float scale = 1.0f / sqrtf((float)DH);
   attention_bwd_dq_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, (const T*)o, lse,
-                                                       (const T*)dout, (T*)dqkv, dsum, S, H, causal, scale);
+                                                       (const T*)dout, (T*)dqkv, dsum, S, H, causal, scale, lens);
   attention_bwd_dkv_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, lse, (const T*)dout, dsum,
-                                                        (T*)dqkv, S, H, causal, scale);
+                                                        (T*)dqkv, S, H, causal, scale, lens);
 }
 #define HIFT_DH_SWITCH(dh, CALL)            \
   switch (dh) {                             \
@@ -74,7 +74,8 @@ inline void attention_bwd_inst(cudaStream_t st, int B, int S, int H, int causal,
 // bf16 with head size 64 or 128 goes to the tensor-core kernels
 inline bool attention_use_mma(int dtype, int dh) { return dtype == 1 && (dh == 64 || dh == 128); }
 template <int DH>
-inline void attention_mma_fwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, void* o, float* lse) {
+inline void attention_mma_fwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, void* o, float* lse,
+                              const int* lens) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(attn_fwd_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_fwd_smem_bytes<DH>());
@@ -83,11 +84,11 @@ inline void attention_mma_fwd(cudaStream_t st, int B, int S, int H, int causal, 
   }
   dim3 grid((S + 63) / 64, H, B);
   attn_fwd_mma_kernel<DH><<<grid, 128, attn_fwd_smem_bytes<DH>(), st>>>((const bf16*)qkv, (bf16*)o, lse, S, H, causal,
-                                                                       1.0f / sqrtf((float)DH));
+                                                                       1.0f / sqrtf((float)DH), lens);
 }
 template <int DH>
 inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, const void* o,
-                              const float* lse, const void* dout, void* dqkv, float* dsum) {
+                              const float* lse, const void* dout, void* dqkv, float* dsum, const int* lens) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(attn_bwd_dkv_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_dkv_smem_bytes<DH>());
@@ -98,43 +99,43 @@ inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, 
   const float scale = 1.0f / sqrtf((float)DH);
   launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, DH);
   dim3 grid((S + 63) / 64, H, B);
-  attn_bwd_dq_mma_kernel<DH><<<grid, 128, 0, st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum, (bf16*)dqkv, S, H, causal, scale);
+  attn_bwd_dq_mma_kernel<DH><<<grid, 128, 0, st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum, (bf16*)dqkv, S, H, causal, scale, lens);
   attn_bwd_dkv_mma_kernel<DH><<<grid, 128, attn_dkv_smem_bytes<DH>(), st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum,
-                                                                           (bf16*)dqkv, S, H, causal, scale);
+                                                                           (bf16*)dqkv, S, H, causal, scale, lens);
 }
 inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
-                                 const void* qkv, void* o, float* lse) {
+                                 const void* qkv, void* o, float* lse, const int* lens = nullptr) {
   if (attention_use_mma(dtype, dh)) {
     if (gemm_tc_init() == 0 && attn_tc_eligible(dh, qkv, H)) {        // tcgen05 kernel
-      attn_tc_fwd_launch(st, B, S, H, dh, causal, qkv, o, lse);
+      attn_tc_fwd_launch(st, B, S, H, dh, causal, qkv, o, lse, lens);
       return;
     }
-    if (dh == 64) attention_mma_fwd<64>(st, B, S, H, causal, qkv, o, lse);
-    else attention_mma_fwd<128>(st, B, S, H, causal, qkv, o, lse);
+    if (dh == 64) attention_mma_fwd<64>(st, B, S, H, causal, qkv, o, lse, lens);
+    else attention_mma_fwd<128>(st, B, S, H, causal, qkv, o, lse, lens);
     return;
   }
 #define CALL_F(D)                                                              \
-  if (dtype == 0) attention_fwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse); \
-  else attention_fwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse)
+  if (dtype == 0) attention_fwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, lens); \
+  else attention_fwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, lens)
   HIFT_DH_SWITCH(dh, CALL_F)
 #undef CALL_F
 }
 inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
                                  const void* qkv, const void* o, const float* lse, const void* dout,
-                                 void* dqkv, float* dsum) {
+                                 void* dqkv, float* dsum, const int* lens = nullptr) {
   if (attention_use_mma(dtype, dh)) {
     if (gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv) && (((uintptr_t)o) & 15) == 0) {   // tcgen05 kernels
       launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
-      attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv);
+      attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv, lens);
       return;
     }
-    if (dh == 64) attention_mma_bwd<64>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum);
-    else attention_mma_bwd<128>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum);
+    if (dh == 64) attention_mma_bwd<64>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens);
+    else attention_mma_bwd<128>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens);
     return;
   }
 #define CALL_B(D)                                                                              \
-  if (dtype == 0) attention_bwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum); \
-  else attention_bwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum)
+  if (dtype == 0) attention_bwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens); \
+  else attention_bwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens)
   HIFT_DH_SWITCH(dh, CALL_B)
 #undef CALL_B
 }

@@ -24,7 +24,7 @@ def make_pair(cfg, gcfg, ocfg, seed=1, perturb=0.05):
 
 
 def lockstep(cfg, gcfg, ocfg, steps, dist, tol_loss, tol_grad, seed=1, data_seed=5, perturb=0.05,
-             check_update=None, resync=False):
+             check_update=None, resync=False, lens=None):
     """Run `steps` iterations on both sides with the same batches and compare
     group choice (exact), learning rate (exact), loss, every gradient tensor of
     the active group, and frozen parameters (bit-exact).
@@ -32,7 +32,11 @@ def lockstep(cfg, gcfg, ocfg, steps, dist, tol_loss, tol_grad, seed=1, data_seed
     resync=True copies the library's updated fp32 master values into the oracle
     after every step, so that each step is compared from identical parameters
     (the tolerances are per step; without it the two parameter trajectories
-    drift apart by the accumulated rounding of earlier updates)."""
+    drift apart by the accumulated rounding of earlier updates).
+
+    lens: optional function step -> list of real-token counts per batch entry
+    (right-padded batches): both sides get the table, padded positions of a
+    language-model batch carry label -1."""
     import torch
     import synth
     h, orc, p0 = make_pair(cfg, gcfg, ocfg, seed, perturb)
@@ -43,13 +47,21 @@ def lockstep(cfg, gcfg, ocfg, steps, dist, tol_loss, tol_grad, seed=1, data_seed
     try:
         for t in range(steps):
             tok, lab = synth.batch_for(cfg, data_seed, t, dist)
+            kl = None
+            if lens is not None:
+                kl = [int(v) for v in lens(t)]
+                h.set_key_lengths(kl)
+                if lab.ndim == 2:
+                    lab = lab.copy()
+                    for b, l in enumerate(kl):
+                        lab[b, l:] = -1
             g = h.active_group()
             assert g == orc.active_group(), (t, g, orc.active_group())
             assert h.current_lr() == orc.current_lr()
             active = set(orc.group_tensor_names(g))
             before = {n: h.get_param(n) for n in names}
             loss = h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
-            loss_ref = orc.step(tok, lab)
+            loss_ref = orc.step(tok, lab, kl)
             assert abs(loss - loss_ref) <= tol_loss * abs(loss_ref), (t, loss, loss_ref)
             worst = 0.0
             for n in sorted(active):

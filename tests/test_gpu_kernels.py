@@ -226,6 +226,63 @@ def test_attention_tensor_core_edge_lengths(dh, B, S, H, causal):
             assert rel_l2(got[:, i * d:(i + 1) * d], r) <= 1.5e-2, i
 
 
+@pytest.mark.parametrize("dtype,dh", [(0, 32), (1, 64), (1, 128)])
+@pytest.mark.parametrize("causal", [0, 1])
+def test_attention_key_lengths(dtype, dh, causal):
+    """Right-padded batch entries: keys at or after an entry's length get no weight and no gradient.  Lengths
+    of a full row, one past a tile, exactly a tile, a few keys and a single key."""
+    import torch
+    from paper_2401_15207_b200 import k_attention_fwd, k_attention_bwd
+    B, S, H = 5, 300, 2
+    lens = [300, 129, 128, 37, 1]
+    d = H * dh
+    rng = np.random.default_rng(77 + dh + causal)
+    qkv = rng.standard_normal((B * S, 3 * d)).astype(np.float32)
+    do = rng.standard_normal((B * S, d)).astype(np.float32)
+    td = torch.float32 if dtype == 0 else torch.bfloat16
+    cvt = (lambda a: a.astype(np.float64)) if dtype == 0 else _bf
+    q, k, v = (cvt(qkv)[:, i * d:(i + 1) * d].reshape(B, S, H, dh) for i in range(3))
+    o_ref, p = O.attention_fwd(q, k, v, bool(causal), lens)
+    tq = _t(qkv, td)
+    tl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    o = torch.full((B * S, d), 9.0, dtype=td, device="cuda")
+    lse = torch.full((B, H, S), 9.0, dtype=torch.float32, device="cuda")
+    k_attention_fwd(dtype, B, S, H, dh, causal, tq, o, lse, key_lens=tl)
+    assert rel_l2(o.float().cpu().numpy(), o_ref.reshape(B * S, d)) <= (3e-6 if dtype == 0 else 6e-3)
+    dqkv = torch.full((B * S, 3 * d), 9.0, dtype=td, device="cuda")
+    dsum = torch.empty(B * S * H, dtype=torch.float32, device="cuda")
+    k_attention_bwd(dtype, B, S, H, dh, causal, tq, o, lse, _t(do, td), dqkv, dsum, key_lens=tl)
+    dq, dk, dv = O.attention_bwd(cvt(do).reshape(B, S, H, dh), q, k, v, p)
+    ref = np.concatenate([t.reshape(B * S, d) for t in (dq, dk, dv)], axis=1)
+    got = dqkv.float().cpu().numpy()
+    tolb = 5e-6 if dtype == 0 else 1.5e-2
+    for i in range(3):
+        assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= tolb, i
+    g4 = got.reshape(B, S, 3, d)
+    for b, l in enumerate(lens):
+        assert np.all(g4[b, l:, 1:] == 0.0), b                # dk, dv of padded keys: exact zeros
+    # the full-length table is the same computation as no table
+    o2 = torch.empty_like(o)
+    lse2 = torch.empty_like(lse)
+    k_attention_fwd(dtype, B, S, H, dh, causal, tq, o2, lse2)
+    k_attention_fwd(dtype, B, S, H, dh, causal, tq, o, lse, key_lens=torch.full((B,), S, dtype=torch.int32, device="cuda"))
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)
+
+
+def test_attention_key_lengths_on_the_warp_level_kernels():
+    """The same cases with the tcgen05 attention switched off (the switch is read when the library loads)."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, HIFT_ATTN_TC="0", HIFT_ATTN_BWD_TC="0")
+    here = os.path.abspath(__file__)
+    r = subprocess.run([sys.executable, "-m", "pytest", here, "-q", "-x", "-m", "gpu", "-k",
+                        "test_attention_key_lengths and not warp_level", "-p", "no:cacheprovider"],
+                       env=env, capture_output=True, text=True, cwd=os.path.dirname(os.path.dirname(here)))
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert "6 passed" in r.stdout, r.stdout[-500:]
+
+
 # ------------------------------------------------------------------ rotary embedding fused into the qkv projection
 def _rope_cs(S, dh, base=10000.0):
     cos, sin = O.rope_tables(S, dh, base)

@@ -51,6 +51,29 @@ def test_mini_fp32_grouped_and_split(arch):
              FP32_LOSS, FP32_GRAD, resync=True)
 
 
+@pytest.mark.parametrize("arch", [0, 1, 2])
+@pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
+def test_right_padded_batches_with_key_lengths(arch, dtype):
+    """Batches of unequal length: the key-length table changes from step to step, padded language-model
+    positions carry no label; loss and gradients follow the oracle's masked attention."""
+    from paper_2401_15207_b200 import HiFT
+    bf = dtype == synth.DTYPE_BF16
+    cfg = mini(arch, dtype, **(dict(d_model=128, n_heads=2, d_ffn=256) if bf else {}))
+    tables = [[40, 17, 1], [5, 40, 33], [40, 40, 40], [2, 3, 9], [29, 1, 40]]
+    lockstep(cfg, synth.GroupCfg(layers_per_group=1, order=1), synth.OptCfg(kind=0, lr=1e-3), 5, "zipf",
+             BF16_LOSS if bf else FP32_LOSS, BF16_GRAD if bf else FP32_GRAD, resync=True,
+             lens=lambda t: tables[t])
+    h = HiFT(cfg, synth.GroupCfg(), synth.OptCfg())
+    try:
+        for bad in ([0, 1, 1], [41, 1, 1]):
+            with pytest.raises(RuntimeError):
+                h.set_key_lengths(bad)
+        h.set_key_lengths([1, 2, 3])
+        h.set_key_lengths(None)
+    finally:
+        h.close()
+
+
 @pytest.mark.parametrize("arch", [0, 2])
 def test_uneven_caller_chosen_groups(arch):
     """Groups of unequal size given as a list of chunk lengths: the same step, the partition is the caller's."""

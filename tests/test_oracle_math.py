@@ -37,10 +37,14 @@ def batch(cfg, seed=11, ignore=False):
 
 
 # ---------------------------------------------------------------- P1: finite differences
-def _fd_check(cfg, n_samples=5, h=1e-5, rel=2e-6, ignore=False):
+def _fd_check(cfg, n_samples=5, h=1e-5, rel=2e-6, ignore=False, lens=None):
     P = params64(cfg)
     tok, lab = batch(cfg, ignore=ignore)
-    loss, cache = O.forward(cfg, P, tok, lab)
+    if lens is not None and lab.ndim == 2:                      # padded positions carry no label
+        lab = lab.copy()
+        for b, l in enumerate(lens):
+            lab[b, l:] = -1
+    loss, cache = O.forward(cfg, P, tok, lab, lens)
     G = O.backward(cfg, P, cache, None)
     rng = np.random.default_rng(0)
     assert set(G.keys()) == set(P.keys())
@@ -55,9 +59,9 @@ def _fd_check(cfg, n_samples=5, h=1e-5, rel=2e-6, ignore=False):
         for i in idx:
             old = flat[i]
             flat[i] = old + h
-            lp, _ = O.forward(cfg, P, tok, lab)
+            lp, _ = O.forward(cfg, P, tok, lab, lens)
             flat[i] = old - h
-            lm, _ = O.forward(cfg, P, tok, lab)
+            lm, _ = O.forward(cfg, P, tok, lab, lens)
             flat[i] = old
             fd = (lp - lm) / (2 * h)
             assert abs(fd - g.reshape(-1)[i]) <= rel * scale + 1e-9, (name, i, fd, g.reshape(-1)[i])
@@ -79,6 +83,63 @@ def test_fd_postln_classifier():
 def test_fd_llama():
     _fd_check(mini(2))
     _fd_check(mini(2, tie_head=1), n_samples=2)
+
+
+def test_fd_with_key_padding():
+    _fd_check(mini(1), lens=[5, 8], n_samples=3)
+    _fd_check(mini(0), lens=[3, 6], n_samples=3)
+    _fd_check(mini(2), lens=[8, 1], n_samples=2)
+
+
+# ---------------------------------------------------------------- key padding reduces to shorter sequences
+def test_key_padding_equals_attention_on_the_unpadded_rows():
+    rng = np.random.default_rng(5)
+    B, S, H, dh = 3, 7, 2, 4
+    q, k, v = (rng.standard_normal((B, S, H, dh)) for _ in range(3))
+    lens = [7, 3, 1]
+    for causal in (False, True):
+        full, _ = O.attention_fwd(q, k, v, causal)
+        same, _ = O.attention_fwd(q, k, v, causal, lens=[S] * B)
+        assert np.array_equal(full, same)
+        o, p = O.attention_fwd(q, k, v, causal, lens=lens)
+        for b, l in enumerate(lens):
+            ref, _ = O.attention_fwd(q[b:b + 1, :l], k[b:b + 1, :l], v[b:b + 1, :l], causal)
+            np.testing.assert_allclose(o[b, :l], ref[0], rtol=1e-13, atol=1e-15)
+            assert np.all(p[b, :, :, l:] == 0.0)                       # no weight on padded keys
+            np.testing.assert_allclose(p[b].sum(-1), 1.0, rtol=1e-13)
+        # no gradient reaches padded keys or values
+        do = rng.standard_normal((B, S, H, dh))
+        _, dk, dv = O.attention_bwd(do, q, k, v, p)
+        for b, l in enumerate(lens):
+            assert np.all(dk[b, l:] == 0.0) and np.all(dv[b, l:] == 0.0)
+
+
+def test_padded_batch_equals_the_sequences_run_alone():
+    """Encoder + classifier: the loss of a right-padded batch with the length table is the mean of the losses of
+    the unpadded sequences run one by one, whatever the pad token is; and the pad token's embedding gets no gradient."""
+    cfg = mini(1, batch=3)
+    P = params64(cfg)
+    tok, lab = synth.batch_for(cfg, 11, 0, dist="uniform")
+    lens = [8, 4, 2]
+    pad_id = cfg.vocab - 1
+    tok = np.where(tok == pad_id, 0, tok)
+    for b, l in enumerate(lens):
+        tok[b, l:] = pad_id
+    loss, cache = O.forward(cfg, P, tok, lab, lens)
+    alone = []
+    for b, l in enumerate(lens):
+        c1 = cfg.scaled(batch=1, seq=l)
+        lb, _ = O.forward(c1, P, tok[b:b + 1, :l], lab[b:b + 1])
+        alone.append(lb)
+    assert loss == pytest.approx(np.mean(alone), rel=1e-12)
+    tok2 = tok.copy()
+    tok2[1, 4:] = 7                                                    # other pad content: same loss
+    loss2, _ = O.forward(cfg, P, tok2, lab, lens)
+    assert loss2 == pytest.approx(loss, rel=1e-13)
+    G = O.backward(cfg, P, cache, None)
+    assert np.all(G["tok_emb"][pad_id] == 0.0)
+    loss_nomask, _ = O.forward(cfg, P, tok, lab)
+    assert abs(loss_nomask - loss) > 1e-6                              # the table matters
 
 
 # ---------------------------------------------------------------- P7: truncated == full restricted
