@@ -292,6 +292,7 @@ def run_ours(args, cfg, gcfg, ocfg):
 
     if rank == 0:
         peaks = measured_peaks()
+        default_llama = args.workload == "llama7b" and not args.full_param and not args.recompute
         g = {c: prof[c] for c in ("gemm_fwd", "gemm_dx", "gemm_dw")}
         g_launch = sum(v["launches"] for v in g.values())
         g_ms = sum(v["ms"] for v in g.values())
@@ -300,9 +301,11 @@ def run_ours(args, cfg, gcfg, ocfg):
         peak = peaks["bf16_tflops_sustained"] if cfg.dtype == 1 else None
         roof = {"kernel": "linear-layer GEMMs (forward, dX, dW)", "bound": "tensor" if cfg.dtype == 1 else "alu",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": (achieved / peak) if peak else None, "traffic": None,
-                "traffic_note": "launches of many shapes are averaged here; per-shape DRAM counters are in "
-                                "profiles/gemm_tc_kernel_m2048_n12288_k4096.md (traffic / algorithmic bytes 0.88-1.32)",
+                "frac": (achieved / peak) if peak else None,
+                "traffic": NCU_GEMM_TRAFFIC["bytes_per_launch"] if default_llama else None,
+                "traffic_unit": "bytes per launch",
+                "traffic_note": NCU_GEMM_TRAFFIC["note"] if default_llama else
+                                "DRAM counters were taken on the llama7b workload only",
                 "peak_source": f"bf16 dense sustained, {peaks['source']}",
                 "launches": g_launch, "avg_launch_ms": g_ms / max(g_launch, 1),
                 "profiled_ms_per_step": ms_prof / K,
@@ -467,6 +470,16 @@ def run_sweep_depth(args):
     h.close()
     print(json.dumps({"sweep": "depth", "workload": "gpt2large", "peak_tflops": peaks["bf16_tflops_sustained"],
                       "rows": rows}))
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of the tensor-core GEMM launches of one llama7b step (the step that
+# trains block 4: 129 forward, 113 dX, 4 dW launches), from a one-pass ncu capture of this file's own command line;
+# the table with every kernel of the step is profiles/launch_list_llama7b_step.md.
+NCU_GEMM_TRAFFIC = {
+    "bytes_per_launch": 53.462e9 / 246,
+    "note": "ncu, one step (block 4 active): 53.46 GB over 246 GEMM launches = 217.3 MB per launch, against 205.1 MB of "
+            "operands and results per launch (1.06); profiles/launch_list_llama7b_step.md",
+}
 
 
 def main():
