@@ -36,6 +36,29 @@ def test_missing_attention_scale_in_dk_is_caught(monkeypatch):
     _expect_caught(lambda: _fd_check(mini(1), n_samples=3))
 
 
+def test_key_padding_off_by_one_or_on_the_wrong_axis_is_caught(monkeypatch):
+    from test_oracle_math import test_key_padding_equals_attention_on_the_unpadded_rows as pin_rows
+    from test_oracle_math import test_padded_batch_equals_the_sequences_run_alone as pin_batch
+    orig = O.attention_fwd
+    # the key at position len still visible
+    monkeypatch.setattr(O, "attention_fwd", lambda q, k, v, causal, lens=None:
+                        orig(q, k, v, causal, None if lens is None else [min(int(l) + 1, q.shape[1]) for l in lens]))
+    _expect_caught(pin_rows)
+    _expect_caught(pin_batch)
+
+    # the table applied to queries instead of keys: padded query rows zeroed, padded keys still seen
+    def on_queries(q, k, v, causal, lens=None):
+        o, p = orig(q, k, v, causal)
+        if lens is not None:
+            o = o.copy()
+            for b, l in enumerate(lens):
+                o[b, int(l):] = 0.0
+        return o, p
+    monkeypatch.setattr(O, "attention_fwd", on_queries)
+    _expect_caught(pin_rows)
+    _expect_caught(pin_batch)
+
+
 def test_layernorm_backward_without_mean_subtraction_is_caught(monkeypatch):
     def bad(dy, cache, g):
         xhat, rstd = cache
