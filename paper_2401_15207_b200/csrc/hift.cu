@@ -1390,13 +1390,14 @@ hift_status hift_save(hift_ctx* c, const char* path) {
   CkptHeader h;
   memset(&h, 0, sizeof(h));
   memcpy(h.magic, "HIFTCKPT", 8);
-  h.version = 1; h.kind = (uint32_t)c->oc.kind; h.dtype = (uint32_t)c->m.dtype; h.n_groups = (uint32_t)c->groups.size();
+  h.version = 2; h.kind = (uint32_t)c->oc.kind; h.dtype = (uint32_t)c->m.dtype; h.n_groups = (uint32_t)c->groups.size();
   h.total = c->total; h.t = (uint64_t)c->t;
   bool ok = fwrite(&h, sizeof(h), 1, f) == 1;
   std::vector<float> tmp;
   for (auto& gr : c->groups) {
     if (!ok) break;
-    ok = fwrite(&gr.tau, sizeof(gr.tau), 1, f) == 1;
+    const uint64_t span[2] = {(uint64_t)gr.off, (uint64_t)gr.numel};   // the partition is part of the format
+    ok = fwrite(span, sizeof(span), 1, f) == 1 && fwrite(&gr.tau, sizeof(gr.tau), 1, f) == 1;
     float *mp, *sp; bool mh, sh;
     group_locations(c, gr, &mp, &mh, &sp, &sh);
     auto put = [&](const float* p, bool host, size_t n) {
@@ -1428,13 +1429,16 @@ hift_status hift_load(hift_ctx* c, const char* path) {
   FILE* f = fopen(path, "rb");
   if (!f) return HIFT_ERR_INPUT;
   CkptHeader h;
-  bool ok = fread(&h, sizeof(h), 1, f) == 1 && memcmp(h.magic, "HIFTCKPT", 8) == 0 && h.version == 1;
+  bool ok = fread(&h, sizeof(h), 1, f) == 1 && memcmp(h.magic, "HIFTCKPT", 8) == 0 && h.version == 2;
   if (ok && (h.kind != (uint32_t)c->oc.kind || h.dtype != (uint32_t)c->m.dtype || h.n_groups != c->groups.size() ||
              h.total != c->total)) { fclose(f); return HIFT_ERR_CFG; }
   std::vector<float> tmp;
   for (auto& gr : c->groups) {
     if (!ok) break;
-    ok = fread(&gr.tau, sizeof(gr.tau), 1, f) == 1;
+    uint64_t span[2] = {0, 0};
+    ok = fread(span, sizeof(span), 1, f) == 1;
+    if (ok && (span[0] != (uint64_t)gr.off || span[1] != (uint64_t)gr.numel)) { fclose(f); return HIFT_ERR_CFG; }   // other grouping
+    ok = ok && fread(&gr.tau, sizeof(gr.tau), 1, f) == 1;
     float *mp, *sp; bool mh, sh;
     group_locations(c, gr, &mp, &mh, &sp, &sh);
     auto get = [&](float* p, bool host, size_t n) {

@@ -266,7 +266,11 @@ def test_checkpoint_resume_is_bitwise(kind, offload, dtype, tmp_path):
         other.load(path)                                   # different optimizer: refused
     with pytest.raises(HiftError):
         b.load(str(tmp_path / "missing.bin"))
-    for h in (a, b, other):
+    regrouped = HiFT(cfg, synth.GroupCfg(order=synth.ORDER_RANDOM, order_seed=4, group_sizes=(1, 2, 2)), oc)
+    assert regrouped.num_groups() == a.num_groups()
+    with pytest.raises(HiftError):
+        regrouped.load(path)                               # same number of groups, other partition: refused
+    for h in (a, b, other, regrouped):
         h.close()
 
 
