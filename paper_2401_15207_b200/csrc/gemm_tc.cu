@@ -280,6 +280,10 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
   }
 }
 
+// Logistic function for the epilogues whose result is rounded to bf16: hardware exp2 and reciprocal
+// (a few ulp of fp32, against the 2^-9 of the store); exp(-g) = inf gives 0, exp(-g) = 0 gives 1.
+__device__ __forceinline__ float sigmoid_tc(float g) { return __fdividef(1.0f, 1.0f + __expf(-g)); }
+
 // Gate | up tile: accumulator columns [0, 128) are gate columns nb .. nb+127, columns [128, 256) the
 // up columns of the same index.  Stores silu(gate) * up, and the two pre-activations themselves
 // when the backward pass will need them (cptr != nullptr).
@@ -301,7 +305,7 @@ __device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int
       }
       float sgl[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) sgl[j] = g[j] / (1.0f + expf(-g[j])) * u[j];
+      for (int j = 0; j < 32; ++j) sgl[j] = g[j] * sigmoid_tc(g[j]) * u[j];
       if (cptr) {
         epi_store32<false, true>(g, cptr, ldc, m, nb + c0, 0, nullptr, nullptr, 0);
         epi_store32<false, true>(u, cptr, ldc, m, sw.half + nb + c0, 0, nullptr, nullptr, 0);
@@ -352,7 +356,7 @@ __device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m
         for (int t = 0; t < 4; ++t) {
           const float2 g2 = __bfloat1622float2(hg[t]), u2 = __bfloat1622float2(hu[t]);
           const float d0 = __uint_as_float(v[8 * j + 2 * t]), d1 = __uint_as_float(v[8 * j + 2 * t + 1]);
-          const float s0 = 1.0f / (1.0f + expf(-g2.x)), s1 = 1.0f / (1.0f + expf(-g2.y));
+          const float s0 = sigmoid_tc(g2.x), s1 = sigmoid_tc(g2.y);
           pg[t] = __floats2bfloat162_rn(d0 * u2.x * s0 * (1.0f + g2.x * (1.0f - s0)), d1 * u2.y * s1 * (1.0f + g2.y * (1.0f - s1)));
           pu[t] = __floats2bfloat162_rn(d0 * g2.x * s0, d1 * g2.y * s1);
         }
