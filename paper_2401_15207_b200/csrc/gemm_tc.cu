@@ -111,7 +111,10 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem_c, uint64_t da, uint64_t db
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_c), "l"(da), "l"(db), "r"(idesc), "r"(accum) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+// 32 consecutive accumulator columns of this thread's lane.  The load is asynchronous: its registers
+// may be read only after tmem_ld_wait32, which names them as in/out operands so that no use can be
+// scheduled ahead of the wait.  (The wait covers every load this thread has issued so far.)
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t addr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -121,7 +124,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
         "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
         "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(addr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait32(uint32_t (&v)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                 "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                 "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                 "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+               :: "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+  tmem_ld32_nowait(addr, v);
+  tmem_ld_wait32(v);
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle.  Fields in 16-byte units: start address
@@ -213,8 +227,9 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
     float4 rn[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) rn[j] = *reinterpret_cast<const float4*>(rrow + 4 * j);
-#pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += 32) {
+    // the accumulator chunk after this one is requested from tensor memory before this one is worked on
+    uint32_t va[32], vb[32];
+    auto chunk = [&](uint32_t (&v)[32], int c0) {
       float4 rc[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) rc[j] = rn[j];
@@ -222,8 +237,6 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
 #pragma unroll
         for (int j = 0; j < 8; ++j) rn[j] = *reinterpret_cast<const float4*>(rrow + c0 + 32 + 4 * j);
       }
-      uint32_t v[32];
-      tmem_ld32(taddr + c0, v);
       float f[32];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -231,6 +244,47 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
         f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + rc[j].z; f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + rc[j].w;
       }
       epi_store32<OUT_F32, true>(f, cptr, ldc, m, n0 + c0, N, bias, nullptr, 0);
+    };
+    tmem_ld32_nowait(taddr, va);
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 64) {
+      tmem_ld_wait32(va);
+      const bool second = c0 + 32 < BN;              // uniform across the warp
+      if (second) tmem_ld32_nowait(taddr + c0 + 32, vb);
+      chunk(va, c0);
+      if (second) {
+        tmem_ld_wait32(vb);
+        if (c0 + 64 < BN) tmem_ld32_nowait(taddr + c0 + 64, va);
+        chunk(vb, c0 + 32);
+      }
+    }
+    return;
+  }
+  if (OUT_F32 || rope.cs == nullptr || n0 >= rope.cols) {
+    // no rotation in this tile: bias / residual / conversion per 32-column chunk, the next chunk's
+    // tensor-memory load in flight meanwhile
+    const int span = min(BN, ((N - n0 + 31) >> 5) << 5);      // columns to visit, a multiple of 32, uniform across the warp
+    uint32_t va[32], vb[32];
+    auto chunk = [&](uint32_t (&v)[32], int c0) {
+      if (m < M) {
+        float f[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+        epi_store32<OUT_F32, false>(f, cptr, ldc, m, n0 + c0, N, bias, residual, ldr);
+      }
+    };
+    if (span > 0) tmem_ld32_nowait(taddr, va);
+#pragma unroll 1
+    for (int c0 = 0; c0 < span; c0 += 64) {
+      tmem_ld_wait32(va);
+      const bool second = c0 + 32 < span;
+      if (second) tmem_ld32_nowait(taddr + c0 + 32, vb);
+      chunk(va, c0);
+      if (second) {
+        tmem_ld_wait32(vb);
+        if (c0 + 64 < span) tmem_ld32_nowait(taddr + c0 + 64, va);
+        chunk(vb, c0 + 32);
+      }
     }
     return;
   }
