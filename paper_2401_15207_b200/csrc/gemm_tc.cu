@@ -424,10 +424,29 @@ __device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m
 // GELU (exact) in the epilogue.  Forward: stores gelu(y) (and y itself when cptr != nullptr).  Backward: the
 // dX product's output times gelu'(a), a = saved pre-activation of the same element, prefetched a chunk ahead.
 struct GeluArgs { __nv_bfloat16* out; const __nv_bfloat16* bwd_a; };      // both nullptr: none
-__device__ __forceinline__ float gelu_tc(float a) { return 0.5f * a * (1.0f + erff(a * 0.70710678118654752440f)); }
+// Normal CDF and density for epilogues whose result is rounded to bf16: erfc(x) = P(t) exp(-x^2),
+// t = 1 / (1 + p x), x >= 0, the five-term rational approximation 7.1.26 of Abramowitz & Stegun
+// (absolute error 1.5e-7, evaluated here with the hardware exp2 and reciprocal); the negative side
+// uses erfc directly, so the small tail values carry no cancellation.  exp(-x^2) = exp(-a^2 / 2)
+// also gives the density.
+__device__ __forceinline__ void normal_cdf_pdf_tc(float a, float& cdf, float& pdf) {
+  const float x = fabsf(a) * 0.70710678118654752440f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, x, 1.0f));
+  const float poly = t * fmaf(t, fmaf(t, fmaf(t, fmaf(t, 1.061405429f, -1.453152027f), 1.421413741f), -0.284496736f), 0.254829592f);
+  const float e = __expf(-x * x);
+  const float half_erfc = 0.5f * poly * e;
+  cdf = a >= 0.0f ? 1.0f - half_erfc : half_erfc;
+  pdf = e * 0.39894228040143267794f;
+}
+__device__ __forceinline__ float gelu_tc(float a) {
+  float cdf, pdf;
+  normal_cdf_pdf_tc(a, cdf, pdf);
+  return a * cdf;
+}
 __device__ __forceinline__ float gelu_grad_tc(float a) {
-  const float cdf = 0.5f * (1.0f + erff(a * 0.70710678118654752440f));
-  return cdf + a * expf(-0.5f * a * a) * 0.39894228040143267794f;
+  float cdf, pdf;
+  normal_cdf_pdf_tc(a, cdf, pdf);
+  return fmaf(a, pdf, cdf);
 }
 __device__ __forceinline__ void epi_row_gelu_fwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
                                                  int64_t ldc, const __nv_bfloat16* __restrict__ bias, const GeluArgs& ge) {
