@@ -45,7 +45,8 @@ __device__ int g_tc_error = 0;   // 0 ok; 1 producer, 2 MMA issuer, 3 epilogue g
 // BN x 64 bf16 when K-major and ceil(BN/64) boxes of 64 x 64 when N-major.
 constexpr int kABytes = BM * BK * 2;
 constexpr int kSmemBudget = 196608;                 // operand ring
-constexpr int kSmemBytes = kSmemBudget + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kStoreStage = 4096;                   // per epilogue warp: one 32 x 32 fp32 chunk on its way to global memory
+constexpr int kSmemBytes = kSmemBudget + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * kStoreStage;
 constexpr int kMaxStages = 8;
 constexpr int kAccStride = 256;                     // tensor-memory columns between the two accumulators
 struct TileRt { int bn, b_bytes, stage_bytes, stages; };
@@ -210,6 +211,64 @@ __device__ __forceinline__ void epi_store32(float (&f)[32], void* __restrict__ c
   }
 }
 
+// The same 32 x 32 chunk of a warp (lane = row), written as whole lines.  A thread that stores its own row puts
+// 16 bytes into each of 32 different lines per instruction, and the store path charges per line touched, not per
+// byte: on short-K products that was what a tile waited for.  Here the warp parks the chunk in its 4 KB of shared
+// memory (16-byte segments XOR-swizzled so that neither side has bank conflicts) and writes it back with
+// consecutive lanes on consecutive segments of a row: 8 rows x 64 bytes (bf16) or 4 rows x 128 bytes (fp32) per
+// instruction.  Only for chunks whose 32 columns all exist; `m` is this lane's row, rows at or beyond M are skipped.
+template <bool OUT_F32>
+__device__ __forceinline__ void epi_store32_lines(float (&f)[32], uint8_t* __restrict__ stage, void* __restrict__ cptr, int64_t ldc,
+                                                  int m, int lane, int M, int n, const __nv_bfloat16* __restrict__ bias) {
+  if (bias) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 8) {
+      const uint4 b4 = *reinterpret_cast<const uint4*>(bias + n + j);
+      const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b4);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const float2 bf = __bfloat1622float2(hb[t]);
+        f[j + 2 * t] += bf.x; f[j + 2 * t + 1] += bf.y;
+      }
+    }
+  }
+  const int row_base = m - lane;
+  if (OUT_F32) {
+    uint8_t* mine = stage + lane * 128;
+#pragma unroll
+    for (int sg = 0; sg < 8; ++sg)
+      *reinterpret_cast<float4*>(mine + ((sg ^ (lane & 7)) << 4)) = make_float4(f[4 * sg], f[4 * sg + 1], f[4 * sg + 2], f[4 * sg + 3]);
+    __syncwarp();
+    const int sg = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = 4 * i + (lane >> 3);
+      const float4 v = *reinterpret_cast<const float4*>(stage + r * 128 + ((sg ^ (r & 7)) << 4));
+      if (row_base + r < M) *reinterpret_cast<float4*>(reinterpret_cast<float*>(cptr) + (int64_t)(row_base + r) * ldc + n + 4 * sg) = v;
+    }
+  } else {
+    uint8_t* mine = stage + lane * 64;
+#pragma unroll
+    for (int sg = 0; sg < 4; ++sg) {
+      uint4 o;
+      __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) ho[t] = __floats2bfloat162_rn(f[8 * sg + 2 * t], f[8 * sg + 2 * t + 1]);
+      *reinterpret_cast<uint4*>(mine + ((sg ^ ((lane >> 1) & 3)) << 4)) = o;
+    }
+    __syncwarp();
+    const int sg = lane & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = 8 * i + (lane >> 2);
+      const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 64 + ((sg ^ ((r >> 1) & 3)) << 4));
+      if (row_base + r < M)
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)(row_base + r) * ldc + n + 8 * sg) = v;
+    }
+  }
+  __syncwarp();                                        // the next chunk overwrites the staging rows
+}
+
 // One row's share of an output tile: BN columns from tensor memory at taddr, starting at column n0.
 // With a rotary embedding (tiles are then whole heads of 128 columns) the chunk at head-local
 // column j < 64 is read together with its partner at j + 64, both get their bias, and the pair is
@@ -217,7 +276,7 @@ __device__ __forceinline__ void epi_store32(float (&f)[32], void* __restrict__ c
 template <bool OUT_F32>
 __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr, int64_t ldc,
                                         const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-                                        const RopeArgs& rope) {
+                                        const RopeArgs& rope, uint8_t* __restrict__ stage, int lane) {
   // (the tensor-memory loads are warp-collective: take this path only if every row of the warp exists)
   if (OUT_F32 && residual != nullptr && n0 + BN <= N && __all_sync(0xffffffffu, m < M)) {
     // Output into the residual stream: the residual chunk of the next 32 columns is fetched while
@@ -243,7 +302,7 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
         f[4 * j] = __uint_as_float(v[4 * j]) + rc[j].x; f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + rc[j].y;
         f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + rc[j].z; f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + rc[j].w;
       }
-      epi_store32<OUT_F32, true>(f, cptr, ldc, m, n0 + c0, N, bias, nullptr, 0);
+      epi_store32_lines<OUT_F32>(f, stage, cptr, ldc, m, lane, M, n0 + c0, bias);
     };
     tmem_ld32_nowait(taddr, va);
 #pragma unroll 1
@@ -266,7 +325,12 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
     const int span = min(BN, ((N - n0 + 31) >> 5) << 5);      // columns to visit, a multiple of 32, uniform across the warp
     uint32_t va[32], vb[32];
     auto chunk = [&](uint32_t (&v)[32], int c0) {
-      if (m < M) {
+      if (residual == nullptr && n0 + c0 + 32 <= N) {    // uniform across the warp: every lane takes part
+        float f[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+        epi_store32_lines<OUT_F32>(f, stage, cptr, ldc, m, lane, M, n0 + c0, bias);
+      } else if (m < M) {
         float f[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
@@ -297,7 +361,7 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
       uint32_t v1[32], v2[32];
       tmem_ld32(taddr + c0, v1);
       tmem_ld32(taddr + c0 + 64, v2);
-      if (m < M) {
+      {                                             // every lane: the stores below are warp-wide (rows beyond M are not written)
         float f1[32], f2[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) { f1[j] = __uint_as_float(v1[j]); f2[j] = __uint_as_float(v2[j]); }
@@ -318,8 +382,8 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
             f2[j + t] = x1 * ss[t] + x2 * cc[t];
           }
         }
-        epi_store32<OUT_F32, true>(f1, cptr, ldc, m, n, N, nullptr, nullptr, 0);
-        epi_store32<OUT_F32, true>(f2, cptr, ldc, m, n + 64, N, nullptr, nullptr, 0);
+        epi_store32_lines<OUT_F32>(f1, stage, cptr, ldc, m, lane, M, n, nullptr);
+        epi_store32_lines<OUT_F32>(f2, stage, cptr, ldc, m, lane, M, n + 64, nullptr);
       }
     } else {
       uint32_t v[32];
@@ -343,13 +407,14 @@ __device__ __forceinline__ float sigmoid_tc(float g) { return __fdividef(1.0f, 1
 // when the backward pass will need them (cptr != nullptr).
 struct SwigluArgs { __nv_bfloat16* out; int half; };          // out == nullptr: none; half = f
 __device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int nb, void* __restrict__ cptr, int64_t ldc,
-                                               const __nv_bfloat16* __restrict__ bias, const SwigluArgs& sw) {
+                                               const __nv_bfloat16* __restrict__ bias, const SwigluArgs& sw,
+                                               uint8_t* __restrict__ stage, int lane) {
 #pragma unroll 1
   for (int c0 = 0; c0 < 128; c0 += 32) {
     uint32_t vg[32], vu[32];
     tmem_ld32(taddr + c0, vg);
     tmem_ld32(taddr + 128 + c0, vu);
-    if (m < M) {
+    {                                               // every lane: the stores are warp-wide (rows beyond M are not written)
       float g[32], u[32];
 #pragma unroll
       for (int j = 0; j < 32; ++j) { g[j] = __uint_as_float(vg[j]); u[j] = __uint_as_float(vu[j]); }
@@ -361,10 +426,10 @@ __device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int
 #pragma unroll
       for (int j = 0; j < 32; ++j) sgl[j] = g[j] * sigmoid_tc(g[j]) * u[j];
       if (cptr) {
-        epi_store32<false, true>(g, cptr, ldc, m, nb + c0, 0, nullptr, nullptr, 0);
-        epi_store32<false, true>(u, cptr, ldc, m, sw.half + nb + c0, 0, nullptr, nullptr, 0);
+        epi_store32_lines<false>(g, stage, cptr, ldc, m, lane, M, nb + c0, nullptr);
+        epi_store32_lines<false>(u, stage, cptr, ldc, m, lane, M, sw.half + nb + c0, nullptr);
       }
-      epi_store32<false, true>(sgl, sw.out, sw.half, m, nb + c0, 0, nullptr, nullptr, 0);
+      epi_store32_lines<false>(sgl, stage, sw.out, sw.half, m, lane, M, nb + c0, nullptr);
     }
   }
 }
@@ -374,11 +439,12 @@ __device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int
 // stores d gate and d up into the [M, 2f] gradient of the gate | up projection.
 struct SwigluBwdArgs { const __nv_bfloat16* gu; };            // gu == nullptr: none
 __device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
-                                                   const SwigluBwdArgs& sb) {
+                                                   const SwigluBwdArgs& sb, uint8_t* __restrict__ stage, int lane) {
   const bool rowok = m < M;
   const __nv_bfloat16* grow = sb.gu + (int64_t)m * (2 * (int64_t)N) + n0;
-  __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(cptr) + (int64_t)m * (2 * (int64_t)N) + n0;
   uint4 gn[4], un[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { gn[j] = make_uint4(0u, 0u, 0u, 0u); un[j] = gn[j]; }   // rows beyond M: computed on zeros, never stored
   if (rowok && n0 < N) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) { gn[j] = *reinterpret_cast<const uint4*>(grow + 8 * j); un[j] = *reinterpret_cast<const uint4*>(grow + N + 8 * j); }
@@ -398,26 +464,24 @@ __device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m
     }
     uint32_t v[32];
     tmem_ld32(taddr + c0, v);
-    if (rowok) {
+    float dg[32], du[32];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat162* hg = reinterpret_cast<const __nv_bfloat162*>(&gc[j]);
-        const __nv_bfloat162* hu = reinterpret_cast<const __nv_bfloat162*>(&uc[j]);
-        uint4 og, ou;
-        __nv_bfloat162* pg = reinterpret_cast<__nv_bfloat162*>(&og);
-        __nv_bfloat162* pu = reinterpret_cast<__nv_bfloat162*>(&ou);
+    for (int j = 0; j < 4; ++j) {
+      const __nv_bfloat162* hg = reinterpret_cast<const __nv_bfloat162*>(&gc[j]);
+      const __nv_bfloat162* hu = reinterpret_cast<const __nv_bfloat162*>(&uc[j]);
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const float2 g2 = __bfloat1622float2(hg[t]), u2 = __bfloat1622float2(hu[t]);
-          const float d0 = __uint_as_float(v[8 * j + 2 * t]), d1 = __uint_as_float(v[8 * j + 2 * t + 1]);
-          const float s0 = sigmoid_tc(g2.x), s1 = sigmoid_tc(g2.y);
-          pg[t] = __floats2bfloat162_rn(d0 * u2.x * s0 * (1.0f + g2.x * (1.0f - s0)), d1 * u2.y * s1 * (1.0f + g2.y * (1.0f - s1)));
-          pu[t] = __floats2bfloat162_rn(d0 * g2.x * s0, d1 * g2.y * s1);
-        }
-        *reinterpret_cast<uint4*>(orow + c0 + 8 * j) = og;
-        *reinterpret_cast<uint4*>(orow + N + c0 + 8 * j) = ou;
+      for (int t = 0; t < 4; ++t) {
+        const float2 g2 = __bfloat1622float2(hg[t]), u2 = __bfloat1622float2(hu[t]);
+        const float d0 = __uint_as_float(v[8 * j + 2 * t]), d1 = __uint_as_float(v[8 * j + 2 * t + 1]);
+        const float s0 = sigmoid_tc(g2.x), s1 = sigmoid_tc(g2.y);
+        dg[8 * j + 2 * t] = d0 * u2.x * s0 * (1.0f + g2.x * (1.0f - s0));
+        dg[8 * j + 2 * t + 1] = d1 * u2.y * s1 * (1.0f + g2.y * (1.0f - s1));
+        du[8 * j + 2 * t] = d0 * g2.x * s0;
+        du[8 * j + 2 * t + 1] = d1 * g2.y * s1;
       }
     }
+    epi_store32_lines<false>(dg, stage, cptr, 2 * (int64_t)N, m, lane, M, n0 + c0, nullptr);
+    epi_store32_lines<false>(du, stage, cptr, 2 * (int64_t)N, m, lane, M, N + n0 + c0, nullptr);
   }
 }
 
@@ -449,13 +513,14 @@ __device__ __forceinline__ float gelu_grad_tc(float a) {
   return fmaf(a, pdf, cdf);
 }
 __device__ __forceinline__ void epi_row_gelu_fwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
-                                                 int64_t ldc, const __nv_bfloat16* __restrict__ bias, const GeluArgs& ge) {
+                                                 int64_t ldc, const __nv_bfloat16* __restrict__ bias, const GeluArgs& ge,
+                                                 uint8_t* __restrict__ stage, int lane) {
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 32) {
     if (n0 + c0 >= N) break;                       // uniform across the warp; N is a multiple of 32
     uint32_t v[32];
     tmem_ld32(taddr + c0, v);
-    if (m < M) {
+    {                                               // every lane: the stores are warp-wide (rows beyond M are not written)
       const int n = n0 + c0;
       float f[32], u[32];
 #pragma unroll
@@ -466,16 +531,18 @@ __device__ __forceinline__ void epi_row_gelu_fwd(uint32_t taddr, int BN, int m, 
       }
 #pragma unroll
       for (int j = 0; j < 32; ++j) u[j] = gelu_tc(f[j]);
-      if (cptr) epi_store32<false, true>(f, cptr, ldc, m, n, N, nullptr, nullptr, 0);
-      epi_store32<false, true>(u, ge.out, N, m, n, N, nullptr, nullptr, 0);
+      if (cptr) epi_store32_lines<false>(f, stage, cptr, ldc, m, lane, M, n, nullptr);
+      epi_store32_lines<false>(u, stage, ge.out, N, m, lane, M, n, nullptr);
     }
   }
 }
 __device__ __forceinline__ void epi_row_gelu_bwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
-                                                 int64_t ldc, const GeluArgs& ge) {
+                                                 int64_t ldc, const GeluArgs& ge, uint8_t* __restrict__ stage, int lane) {
   const bool rowok = m < M;
   const __nv_bfloat16* arow = ge.bwd_a + (int64_t)m * N + n0;
   uint4 an[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) an[j] = make_uint4(0u, 0u, 0u, 0u);      // rows beyond M: computed on zeros, never stored
   if (rowok && n0 < N) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) an[j] = *reinterpret_cast<const uint4*>(arow + 8 * j);
@@ -492,7 +559,7 @@ __device__ __forceinline__ void epi_row_gelu_bwd(uint32_t taddr, int BN, int m, 
     }
     uint32_t v[32];
     tmem_ld32(taddr + c0, v);
-    if (rowok) {
+    {
       float f[32];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -504,7 +571,7 @@ __device__ __forceinline__ void epi_row_gelu_bwd(uint32_t taddr, int BN, int m, 
           f[8 * j + 2 * t + 1] = __uint_as_float(v[8 * j + 2 * t + 1]) * gelu_grad_tc(a2.y);
         }
       }
-      epi_store32<false, true>(f, cptr, ldc, m, n0 + c0, N, nullptr, nullptr, 0);
+      epi_store32_lines<false>(f, stage, cptr, ldc, m, lane, M, n0 + c0, nullptr);
     }
   }
 }
@@ -629,6 +696,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else {
     // ---------------- epilogue: warps 2..5 own tensor-memory lanes 32*(warp%4) .. +31
     const int q = warp & 3;
+    uint8_t* stage = smem_gen + S * kStageBytes + 256 + (warp - 2) * kStoreStage;   // behind the barriers
     int lt = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++lt) {
       const int ab = lt & 1;
@@ -641,11 +709,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
-      else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb);
-      else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge);
-      else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge);
-      else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
+      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg, stage, lane);
+      else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb, stage, lane);
+      else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge, stage, lane);
+      else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge, stage, lane);
+      else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope, stage, lane);
       // hand the accumulator back to the MMA thread
       tc_fence_before();
       __syncwarp();
@@ -817,6 +885,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   } else {
     // ---------------- epilogue (both CTAs): tensor-memory lanes 32*(warp%4).. hold rows of this CTA's half
     const int q = warp & 3;
+    uint8_t* stage = smem_gen + S * kStage2Bytes + 256 + (warp - 2) * kStoreStage;   // behind the barriers
     int lt = 0;
     for (int tile = pair; tile < num_tiles && !poisoned; tile += num_pairs, ++lt) {
       const int ab = lt & 1;
@@ -828,11 +897,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM, n0 = (tile / tiles_m) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg);
-      else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb);
-      else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge);
-      else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge);
-      else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope);
+      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg, stage, lane);
+      else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb, stage, lane);
+      else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge, stage, lane);
+      else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge, stage, lane);
+      else epi_row<OUT_F32>(taddr, BN, m, M, n0, N, cptr, ldc, bias, residual, ldr, rope, stage, lane);
       // hand this CTA's half of the accumulator back: the MMA thread counts 8 warps (4 per CTA)
       tc_fence_before();
       __syncwarp();
