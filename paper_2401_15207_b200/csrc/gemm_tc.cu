@@ -269,6 +269,50 @@ __device__ __forceinline__ void epi_store32_lines(float (&f)[32], uint8_t* __res
   __syncwarp();                                        // the next chunk overwrites the staging rows
 }
 
+// The reverse trip for what an epilogue reads per row (saved pre-activations, the fp32 residual): the warp fetches
+// the 32 x 32 chunk as whole lines (lane -> one 16-byte segment of a row; this can be issued a chunk ahead), and
+// when the chunk is due it goes through the warp's shared memory so that every lane ends up with its own row.
+// bf16: lane holds segment (lane & 3) of rows 8 i + (lane >> 2), i = 0..3; a chunk takes 2 KB of the staging area.
+__device__ __forceinline__ void lines_fetch_bf16(uint4 (&t)[4], const __nv_bfloat16* __restrict__ base, int64_t ld, int row_base,
+                                                 int lane, int M, int n) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = row_base + 8 * i + (lane >> 2);
+    t[i] = r < M ? *reinterpret_cast<const uint4*>(base + (int64_t)r * ld + n + 8 * (lane & 3)) : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+__device__ __forceinline__ void lines_park_bf16(const uint4 (&t)[4], uint8_t* __restrict__ stage, int lane) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = 8 * i + (lane >> 2);
+    *reinterpret_cast<uint4*>(stage + r * 64 + (((lane & 3) ^ ((r >> 1) & 3)) << 4)) = t[i];
+  }
+}
+__device__ __forceinline__ void lines_own_row_bf16(uint4 (&row)[4], const uint8_t* __restrict__ stage, int lane) {
+#pragma unroll
+  for (int sg = 0; sg < 4; ++sg) row[sg] = *reinterpret_cast<const uint4*>(stage + lane * 64 + ((sg ^ ((lane >> 1) & 3)) << 4));
+}
+// fp32: lane holds segment (lane & 7) of rows 4 i + (lane >> 3), i = 0..7; a chunk takes the whole 4 KB.
+__device__ __forceinline__ void lines_fetch_f32(float4 (&t)[8], const float* __restrict__ base, int64_t ld, int row_base, int lane,
+                                                int M, int n) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = row_base + 4 * i + (lane >> 3);
+    t[i] = r < M ? *reinterpret_cast<const float4*>(base + (int64_t)r * ld + n + 4 * (lane & 7)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
+__device__ __forceinline__ void lines_to_own_row_f32(const float4 (&t)[8], float4 (&row)[8], uint8_t* __restrict__ stage, int lane) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = 4 * i + (lane >> 3);
+    *reinterpret_cast<float4*>(stage + r * 128 + (((lane & 7) ^ (r & 7)) << 4)) = t[i];
+  }
+  __syncwarp();
+#pragma unroll
+  for (int sg = 0; sg < 8; ++sg) row[sg] = *reinterpret_cast<const float4*>(stage + lane * 128 + ((sg ^ (lane & 7)) << 4));
+  __syncwarp();
+}
+
 // One row's share of an output tile: BN columns from tensor memory at taddr, starting at column n0.
 // With a rotary embedding (tiles are then whole heads of 128 columns) the chunk at head-local
 // column j < 64 is read together with its partner at j + 64, both get their bias, and the pair is
@@ -282,20 +326,15 @@ __device__ __forceinline__ void epi_row(uint32_t taddr, int BN, int m, int M, in
     // Output into the residual stream: the residual chunk of the next 32 columns is fetched while
     // this chunk is read from tensor memory, added and stored, so that only the first load's latency
     // is exposed per tile.
-    const float* rrow = residual + (int64_t)m * ldr + n0;
-    float4 rn[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) rn[j] = *reinterpret_cast<const float4*>(rrow + 4 * j);
+    const int row_base = m - lane;
+    float4 rn[8];                                    // the next chunk of the residual, fetched as whole lines
+    lines_fetch_f32(rn, residual, ldr, row_base, lane, M, n0);
     // the accumulator chunk after this one is requested from tensor memory before this one is worked on
     uint32_t va[32], vb[32];
     auto chunk = [&](uint32_t (&v)[32], int c0) {
       float4 rc[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) rc[j] = rn[j];
-      if (c0 + 32 < BN) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) rn[j] = *reinterpret_cast<const float4*>(rrow + c0 + 32 + 4 * j);
-      }
+      lines_to_own_row_f32(rn, rc, stage, lane);
+      if (c0 + 32 < BN) lines_fetch_f32(rn, residual, ldr, row_base, lane, M, n0 + c0 + 32);
       float f[32];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -440,27 +479,26 @@ __device__ __forceinline__ void epi_row_swiglu(uint32_t taddr, int m, int M, int
 struct SwigluBwdArgs { const __nv_bfloat16* gu; };            // gu == nullptr: none
 __device__ __forceinline__ void epi_row_swiglu_bwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
                                                    const SwigluBwdArgs& sb, uint8_t* __restrict__ stage, int lane) {
-  const bool rowok = m < M;
-  const __nv_bfloat16* grow = sb.gu + (int64_t)m * (2 * (int64_t)N) + n0;
-  uint4 gn[4], un[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) { gn[j] = make_uint4(0u, 0u, 0u, 0u); un[j] = gn[j]; }   // rows beyond M: computed on zeros, never stored
-  if (rowok && n0 < N) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { gn[j] = *reinterpret_cast<const uint4*>(grow + 8 * j); un[j] = *reinterpret_cast<const uint4*>(grow + N + 8 * j); }
+  const int row_base = m - lane;
+  const int64_t ldg = 2 * (int64_t)N;
+  uint4 gn[4], un[4];                              // the next chunk of gate and up, fetched as whole lines (zeros beyond M)
+  if (n0 < N) {
+    lines_fetch_bf16(gn, sb.gu, ldg, row_base, lane, M, n0);
+    lines_fetch_bf16(un, sb.gu, ldg, row_base, lane, M, N + n0);
   }
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 32) {
     if (n0 + c0 >= N) break;                       // uniform across the warp; N is a multiple of 32
+    lines_park_bf16(gn, stage, lane);
+    lines_park_bf16(un, stage + 2048, lane);
+    __syncwarp();
     uint4 gc[4], uc[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { gc[j] = gn[j]; uc[j] = un[j]; }
-    if (rowok && c0 + 32 < BN && n0 + c0 + 32 < N) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        gn[j] = *reinterpret_cast<const uint4*>(grow + c0 + 32 + 8 * j);
-        un[j] = *reinterpret_cast<const uint4*>(grow + N + c0 + 32 + 8 * j);
-      }
+    lines_own_row_bf16(gc, stage, lane);
+    lines_own_row_bf16(uc, stage + 2048, lane);
+    __syncwarp();
+    if (c0 + 32 < BN && n0 + c0 + 32 < N) {
+      lines_fetch_bf16(gn, sb.gu, ldg, row_base, lane, M, n0 + c0 + 32);
+      lines_fetch_bf16(un, sb.gu, ldg, row_base, lane, M, N + n0 + c0 + 32);
     }
     uint32_t v[32];
     tmem_ld32(taddr + c0, v);
@@ -538,25 +576,18 @@ __device__ __forceinline__ void epi_row_gelu_fwd(uint32_t taddr, int BN, int m, 
 }
 __device__ __forceinline__ void epi_row_gelu_bwd(uint32_t taddr, int BN, int m, int M, int n0, int N, void* __restrict__ cptr,
                                                  int64_t ldc, const GeluArgs& ge, uint8_t* __restrict__ stage, int lane) {
-  const bool rowok = m < M;
-  const __nv_bfloat16* arow = ge.bwd_a + (int64_t)m * N + n0;
-  uint4 an[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) an[j] = make_uint4(0u, 0u, 0u, 0u);      // rows beyond M: computed on zeros, never stored
-  if (rowok && n0 < N) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) an[j] = *reinterpret_cast<const uint4*>(arow + 8 * j);
-  }
+  const int row_base = m - lane;
+  uint4 an[4];                                     // the next chunk of the saved pre-activation, fetched as whole lines
+  if (n0 < N) lines_fetch_bf16(an, ge.bwd_a, N, row_base, lane, M, n0);
 #pragma unroll 1
   for (int c0 = 0; c0 < BN; c0 += 32) {
     if (n0 + c0 >= N) break;
+    lines_park_bf16(an, stage, lane);
+    __syncwarp();
     uint4 ac[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) ac[j] = an[j];
-    if (rowok && c0 + 32 < BN && n0 + c0 + 32 < N) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) an[j] = *reinterpret_cast<const uint4*>(arow + c0 + 32 + 8 * j);
-    }
+    lines_own_row_bf16(ac, stage, lane);
+    __syncwarp();
+    if (c0 + 32 < BN && n0 + c0 + 32 < N) lines_fetch_bf16(an, ge.bwd_a, N, row_base, lane, M, n0 + c0 + 32);
     uint32_t v[32];
     tmem_ld32(taddr + c0, v);
     {
