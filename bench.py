@@ -476,9 +476,9 @@ def run_sweep_depth(args):
 # trains block 4: 129 forward, 113 dX, 4 dW launches), from a one-pass ncu capture of this file's own command line;
 # the table with every kernel of the step is profiles/launch_list_llama7b_step.md.
 NCU_GEMM_TRAFFIC = {
-    "bytes_per_launch": 53.462e9 / 246,
-    "note": "ncu, one step (block 4 active): 53.46 GB over 246 GEMM launches = 217.3 MB per launch, against 205.1 MB of "
-            "operands and results per launch (1.06); profiles/launch_list_llama7b_step.md",
+    "bytes_per_launch": 54.199e9 / 246,
+    "note": "ncu, one step (block 4 active): 54.20 GB over 246 GEMM launches = 220.3 MB per launch, against 205.1 MB of "
+            "operands and results per launch (1.07); profiles/launch_list_llama7b_step.md",
 }
 
 
