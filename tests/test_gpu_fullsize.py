@@ -206,6 +206,47 @@ def test_fused_epilogue_forms_at_7b_shapes_sampled():
     assert rel_l2(yo[ridx].cpu().numpy(), ref) <= 4e-5
 
 
+def test_gelu_epilogue_forms_at_gpt2_large_shapes_sampled():
+    """The two GEMMs of a GPT-2-large-shaped block whose epilogues carry the exact (erf) GELU, at the step's sizes
+    (T = 4096, d = 1280, f = 5120): up projection + bias + GELU with the pre-activation kept, and the down projection's
+    dX times GELU'.  Eight sampled rows, every column, against the oracle's gelu_fwd / gelu_bwd on the same bf16
+    operands; the far negative tail, where the epilogue's erfc approximation is least accurate in relative terms,
+    is checked on its own."""
+    import torch
+    from paper_2401_15207_b200 import k_linear_gelu, k_linear_dx_gelu_bwd
+    M, d, f = 4096, 1280, 5120
+    rng = np.random.default_rng(13)
+    rows = np.sort(rng.choice(M, 8, replace=False))
+    ridx = torch.from_numpy(rows).cuda()
+    x, x64 = _randn_bf16((M, d), 21)
+    w1, w164 = _randn_bf16((f, d), 22, 0.06)                # pre-activations of standard deviation ~2: both tails populated
+    b1, b164 = _randn_bf16((f,), 23, 0.5)
+    pre = torch.empty((M, f), dtype=torch.bfloat16, device="cuda")
+    act = torch.empty((M, f), dtype=torch.bfloat16, device="cuda")
+    k_linear_gelu(M, f, d, x, w1, pre, act, b1)
+    y = x64[rows] @ w164.T + b164
+    assert rel_l2(pre[ridx].float().cpu().numpy(), y) <= 6e-3
+    got = act[ridx].float().cpu().numpy()
+    ref = O.gelu_fwd(y)
+    assert rel_l2(got, ref) <= 6e-3
+    tail = y < -3.0
+    assert tail.sum() > 100
+    # in the tail gelu(y) is tiny: element by element within the bf16 rounding of the store (2^-9) plus the
+    # approximation's 0.4 %, wherever the value is not below what fp32 accumulation noise in y can move
+    big = tail & (np.abs(ref) > 1e-6)
+    assert big.sum() > 100
+    assert (np.abs(got[big] - ref[big]) / np.abs(ref[big])).max() <= 1.5e-2
+    y_kept = pre[ridx].float().cpu().numpy().astype(np.float64)
+    # dX of the down projection times GELU' at the kept pre-activations
+    dy, dy64 = _randn_bf16((M, d), 24)
+    w2, w264 = _randn_bf16((d, f), 25, 0.02)
+    da = torch.empty((M, f), dtype=torch.bfloat16, device="cuda")
+    k_linear_dx_gelu_bwd(M, d, f, dy, w2, pre, da)
+    du = dy64[rows] @ w264
+    ref = O.gelu_bwd(du, y_kept)
+    assert rel_l2(da[ridx].float().cpu().numpy(), ref) <= 8e-3
+
+
 # ------------------------------------------------------------------ (b) whole-step parity on big-enough miniatures
 def test_llama_miniature_takes_the_tensor_core_paths():
     cfg = synth.ModelCfg(arch=2, n_blocks=2, d_model=512, n_heads=4, d_ffn=1376, vocab=2000, norm_eps=1e-6,
