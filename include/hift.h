@@ -41,8 +41,8 @@ typedef enum {
   HIFT_ERR_OOM_DEVICE = 2,   /* cudaMalloc failed                                    */
   HIFT_ERR_OOM_PINNED = 3,   /* pinned host allocation failed                        */
   HIFT_ERR_INPUT = 4,        /* token id or label out of range, NULL pointer         */
-  HIFT_ERR_NONFINITE = 5,    /* the loss of the step was NaN/Inf (update was applied) */
-  HIFT_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up                   */
+  HIFT_ERR_NONFINITE = 5,    /* the loss of the step was NaN/Inf (no update was made)*/
+  HIFT_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up (no update made)  */
   HIFT_ERR_CUDA = 7,         /* any other CUDA runtime/driver error                  */
   HIFT_ERR_CAPACITY = 8      /* size exceeds the library's built-in scratch capacity */
 } hift_status;
@@ -92,9 +92,15 @@ typedef struct {
   int32_t sched;             /* 0 constant, 1 linear: warm-up, then decay to 0     */
   int32_t total_cycles;      /* horizon C of the linear schedule, in cycles        */
   int32_t offload_state;     /* 1: inactive groups' master+state in pinned host    */
-  int32_t prefetch_groups;   /* 0: one state slot, H2D issued after the forward
-                                   (the paper's order); 1: two slots, H2D issued at
-                                   step start and overlapped with the previous D2H  */
+  int32_t prefetch_groups;   /* state slots on the GPU beyond the first, 0..3 (each the size of the largest
+                                group's paged state).  0: one slot, upload issued after the forward pass
+                                (the paper's order).  1: two slots, upload at the start of the group's
+                                own step, overlapped with the previous write-back.  p >= 2: p + 1 slots,
+                                the uploads of the next p - 1 steps' groups are issued ahead (the order
+                                is known), so transfers stream across steps and a step no longer lasts
+                                at least one transfer.  Residency rule of Algorithm 1 steps i/k kept:
+                                only the active group and groups whose transfer is in flight are on
+                                the GPU.  Same bits in every mode.                                   */
   int32_t recompute;         /* 1: frozen blocks above the active group keep only their input during the
                                 forward pass; what their backward (dX) needs is recomputed block by block in
                                 the backward pass.  Same bits, less HBM (the paper's concern), one extra
@@ -118,8 +124,14 @@ void hift_destroy(hift_ctx *ctx);
  * -1 = position ignored) or int32 [batch] (arch 1).  The mean cross-entropy of
  * the batch, computed before the update, is written to *loss_host.  Returns
  * after the loss is on the host; state write-back may still be in flight.
- * An out-of-range token id is clamped on the device and reported as
- * HIFT_ERR_INPUT after the step has run. */
+ * A step that fails changes nothing: when a bounded device-side wait gave up
+ * (HIFT_ERR_TIMEOUT), a token id or label was out of range (HIFT_ERR_INPUT; the
+ * id is clamped on the device so that the pass itself stays in bounds) or the
+ * loss is not finite (HIFT_ERR_NONFINITE), the optimizer kernels see the
+ * failure on the device and store nothing, so every parameter, master value and
+ * optimizer-state value of every group keeps its bits, the group's update
+ * count and t do not advance, and the next call trains the same group again.
+ * (Gradients that overflow while the loss stays finite are not detected.) */
 hift_status hift_step(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *labels_dev,
                       float *loss_host);
 /* Same, with the batch in host memory (validated on the host, then copied to
@@ -144,11 +156,14 @@ hift_status hift_set_key_lengths(hift_ctx *ctx, const int32_t *lens_host);
  * volume a full-parameter step would exchange); hift_step_end applies the optimizer to the group,
  * starts the state write-back and advances t.  Work the caller enqueued on the stream given to
  * hift_create is ordered before the update.  begin/end must alternate; hift_step in between is
- * refused with HIFT_ERR_CFG. */
+ * refused with HIFT_ERR_CFG.  A hift_step_begin that fails leaves no update pending.
+ * hift_step_abort drops a pending update instead of applying it (t does not advance): what
+ * every rank calls when any rank's first half failed, so that replicas stay identical. */
 hift_status hift_step_begin(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *labels_dev,
                             float *loss_host);
 hift_status hift_grad_view(hift_ctx *ctx, float **grad_dev, size_t *n);
 hift_status hift_step_end(hift_ctx *ctx);
+hift_status hift_step_abort(hift_ctx *ctx);
 
 int32_t hift_active_group(const hift_ctx *ctx);   /* group the NEXT hift_step trains */
 int32_t hift_num_groups(const hift_ctx *ctx);     /* k                               */
@@ -212,9 +227,10 @@ int64_t hift_last_step_launches(const hift_ctx *ctx);
 hift_status hift_last_step_paging(const hift_ctx *ctx, size_t *h2d_bytes, size_t *d2h_bytes);
 
 /* Device timeline of the last step's state paging (Algorithm 1 steps i and k), in milliseconds
- * after the step's first kernel: [0] H2D begin, [1] H2D end, [2] optimizer reaches its wait
- * for the state, [3] wait over, [4] D2H begin, [5] D2H end.  -1 where offload is off.  Waits
- * for the copies to finish. */
+ * after the step's first kernel: [0] H2D begin, [1] H2D end (of the upload that made the group
+ * resident: negative when an earlier step issued it ahead), [2] optimizer reaches its wait
+ * for the state, [3] wait over, [4] D2H begin, [5] D2H end.  NaN where there is nothing to
+ * report (offload off).  Waits for the copies to finish. */
 hift_status hift_last_step_timeline(hift_ctx *ctx, double *ms6);
 
 /* The tensor-core GEMM bounds every device-side wait; a wait that gives up records a code in a

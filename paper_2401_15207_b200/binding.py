@@ -68,6 +68,7 @@ def _prototypes():
         "hift_step_begin": (C.c_int, [vp, vp, vp, pf]),
         "hift_grad_view": (C.c_int, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "hift_step_end": (C.c_int, [vp]),
+        "hift_step_abort": (C.c_int, [vp]),
         "hift_active_group": (i32, [vp]),
         "hift_num_groups": (i32, [vp]),
         "hift_step_count": (i64, [vp]),
@@ -232,6 +233,9 @@ class HiFT:
 
     def step_end(self):
         _check(lib().hift_step_end(self._h), "hift_step_end")
+
+    def step_abort(self):
+        _check(lib().hift_step_abort(self._h), "hift_step_abort")
 
     # -- getters
     def active_group(self) -> int:

@@ -24,6 +24,7 @@ using namespace hift;
 namespace {
 
 constexpr size_t kAlignElems = 128;   // every tensor starts on a multiple of 128 elements
+constexpr int kScalWords = 8;         // the step's scalar words: loss, valid count, bad input, (time-out flag), gate
 
 // Per-block activation slots.  Residual-stream tensors are fp32 in every configuration;
 // GEMM operands have the parameter type (bf16 or fp32).
@@ -54,6 +55,17 @@ struct BlockIdx {          // tensor indices of one block, -1 if absent
   int n1_g, n1_b, w_qkv, b_qkv, w_o, b_o, n2_g, n2_b, w_fc1, b_fc1, w_fc2, b_fc2;
 };
 struct ProfRec { int cls; cudaEvent_t e0, e1; double work; };
+// One device staging slot of the paged optimizer state, laid out like a group's blob.
+constexpr int kMaxSlots = 4;
+struct SlotRec {
+  char* mem = nullptr;
+  int group = -1;            // group whose latest master / state the slot holds (-1: nothing valid)
+  int64_t step = -1;         // step the slot is reserved for (< current step: free to evict)
+  bool d2h_pending = false;  // a write-back from this slot has been enqueued (ev_d2h recorded)
+  int64_t h2d_for_step = -1; // the step whose request started the upload that filled the slot
+  cudaEvent_t ev_h2d, ev_opt, ev_d2h;   // ordering only
+  cudaEvent_t tl_h2d0, tl_h2d1;         // timed: begin / end of the upload
+};
 
 }  // namespace
 
@@ -93,15 +105,16 @@ struct hift_ctx {
   float* af_all = nullptr;          // Adafactor, state resident: compact state of every group
   float* af_scratch = nullptr;      // Adafactor work space, sized for the largest tensor
   bool af = false;
-  char* slot[2] = {nullptr, nullptr};   // offload staging, laid out like the blob
+  SlotRec slot[kMaxSlots];          // offload staging ring
   int n_slots = 1;
+  int lookahead = 0;                // steps ahead of the current one whose state is uploaded early
+  int* gate = nullptr;              // device word: non-zero = the step failed, the optimizer must not write
   float* grad = nullptr;            // [max_group]
   char* arena = nullptr; size_t arena_cap = 0, arena_off = 0, arena_fixed = 0;
-  cudaEvent_t ev_h2d[2], ev_opt[2], ev_d2h[2], ev_fwd;
-  cudaEvent_t tl[7];                // timeline of the last step: start, h2d begin/end, optimizer wait begin/end, d2h begin/end
+  cudaEvent_t ev_fwd;
+  cudaEvent_t tl[7];                // timeline of the last step: start, (unused x2), optimizer wait begin/end, d2h begin/end
   bool tl_valid = false;
   bool events_made = false;
-  bool d2h_pending[2] = {false, false};
   // fixed work buffers
   int32_t *tok_dev = nullptr, *lab_dev = nullptr;
   int32_t* lens_dev = nullptr;      // [B] valid keys per batch entry (key padding), used while use_lens
@@ -592,16 +605,60 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
   if (need_dx) norm_bwd_dx(c, c->dt1, false, x_r, (float*)s[S_ST1], b.n1_g, c->dxb, c->dxa, c->dxa_a);
 }
 
-void issue_h2d(hift_ctx* c, int g, int sl, bool after_forward) {
+// ------------------------------------------------------------------ state paging (Algorithm 1, steps i and k)
+// The group order is known ahead, so the uploads need not wait for their own step: a ring of
+// slots holds the group being trained, the groups of the next `lookahead` steps (upload in flight
+// or landed) and groups whose write-back is still draining.  Only two orderings are enforced: an
+// upload into a slot waits for that slot's last write-back, and the optimizer waits for its own
+// slot's upload (and, when the group was still resident from an earlier step, for that slot's
+// write-back, which reads what the optimizer is about to overwrite).  A group is in at most one
+// slot, and a slot that holds a group holds its latest values: they change only by the optimizer
+// running in that slot, followed by the write-back from it.
+int group_at(const hift_ctx* c, int64_t step) {
+  return c->forced >= 0 ? c->forced : c->order[step % (int64_t)c->groups.size()];
+}
+void drop_reservations(hift_ctx* c) { for (int i = 0; i < c->n_slots; ++i) c->slot[i].step = -1; }
+// after the host has rewritten blobs (every stream idle): nothing on the device is current any more
+void invalidate_slots(hift_ctx* c) {
+  for (int i = 0; i < c->n_slots; ++i) { c->slot[i].group = -1; c->slot[i].step = -1; c->slot[i].d2h_pending = false; }
+}
+// Makes group g resident for step s (>= the current step c->t).  Returns its slot, or -1 when every
+// slot is reserved (only possible for look-ahead requests).
+int acquire_slot(hift_ctx* c, int g, int64_t s, bool after_forward) {
+  for (int i = 0; i < c->n_slots; ++i)
+    if (c->slot[i].group == g) {                      // still (or already) resident: no transfer
+      if (c->slot[i].step < s) c->slot[i].step = s;
+      return i;
+    }
+  int v = -1;
+  for (int i = 0; i < c->n_slots; ++i) {
+    if (c->slot[i].step >= c->t) continue;            // reserved for the current or a coming step
+    if (v < 0 || (c->slot[i].group < 0 && c->slot[v].group >= 0) ||
+        ((c->slot[i].group < 0) == (c->slot[v].group < 0) && c->slot[i].step < c->slot[v].step))
+      v = i;
+  }
+  if (v < 0) return -1;
+  SlotRec& sr = c->slot[v];
   GroupRec& gr = c->groups[g];
   if (after_forward) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_fwd, 0));
-  if (c->d2h_pending[sl]) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_d2h[sl], 0));
-  // slot layout follows the blob: consecutive planes of gr.numel floats
-  c->note(cudaEventRecord(c->tl[1], c->st_h2d));
-  c->note(cudaMemcpyAsync(c->slot[sl], gr.blob, gr.blob_bytes, cudaMemcpyHostToDevice, c->st_h2d));
-  c->note(cudaEventRecord(c->tl[2], c->st_h2d));
-  c->note(cudaEventRecord(c->ev_h2d[sl], c->st_h2d));
-  c->step_h2d = gr.blob_bytes;
+  if (sr.d2h_pending) c->note(cudaStreamWaitEvent(c->st_h2d, sr.ev_d2h, 0));
+  c->note(cudaEventRecord(sr.tl_h2d0, c->st_h2d));
+  c->note(cudaMemcpyAsync(sr.mem, gr.blob, gr.blob_bytes, cudaMemcpyHostToDevice, c->st_h2d));
+  c->note(cudaEventRecord(sr.tl_h2d1, c->st_h2d));
+  c->note(cudaEventRecord(sr.ev_h2d, c->st_h2d));
+  sr.group = g; sr.step = s; sr.d2h_pending = false; sr.h2d_for_step = s;
+  c->step_h2d += gr.blob_bytes;
+  return v;
+}
+// Step start (overlapped modes): the current group, then the groups of the next steps.
+void page_in_ahead(hift_ctx* c) {
+  c->cur_sl = acquire_slot(c, group_at(c, c->t), c->t, false);
+  for (int j = 1; j <= c->lookahead; ++j) {
+    const int gj = group_at(c, c->t + j);
+    bool earlier = false;                              // trained before step t + j: its blob is not final yet
+    for (int i = 0; i < j; ++i) earlier = earlier || group_at(c, c->t + i) == gj;
+    if (!earlier) acquire_slot(c, gj, c->t + j, false);
+  }
 }
 
 // Forward and truncated backward of one step, enqueued on the context's stream; the active group's
@@ -617,8 +674,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   c->last_group = g;
   c->step_launches = 0; c->step_h2d = 0; c->step_d2h = 0;
   c->first_err = cudaSuccess;
-  const int sl = c->n_slots == 2 ? (int)(c->t & 1) : 0;
-  c->cur_sl = sl; c->cur_lr = lr;
+  c->cur_sl = 0; c->cur_lr = lr;
   auto active = [&](int u) { return u >= lo && u <= hi; };
 
   plan_slots(c, g, true);
@@ -628,11 +684,11 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
   c->note(cudaEventRecord(c->tl[0], c->st));
 
-  if (c->offload && c->oc.prefetch_groups) issue_h2d(c, g, sl, false);
+  if (c->offload && c->oc.prefetch_groups) page_in_ahead(c);
 
   // "Clear gradients": the group's span of the gradient buffer starts at zero
   c->note(cudaMemsetAsync(c->grad, 0, gr.numel * sizeof(float), c->st));
-  c->note(cudaMemsetAsync(c->scal, 0, 4 * sizeof(float), c->st));
+  c->note(cudaMemsetAsync(c->scal, 0, kScalWords * sizeof(float), c->st));
   int* bad = (int*)(c->scal + 2);
   int* nvalid = (int*)(c->scal + 1);
 
@@ -667,7 +723,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   if (c->offload && !c->oc.prefetch_groups) {
     // the paper's order: optimizer state moves to the GPU after the forward pass (step i)
     c->note(cudaEventRecord(c->ev_fwd, c->st));
-    issue_h2d(c, g, sl, true);
+    c->cur_sl = acquire_slot(c, g, c->t, true);
   }
 
   // ---------------- backward, truncated at the group ("Backpropagation")
@@ -728,16 +784,27 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
 }
 
 // Optimizer on the active group and write-back of its state, enqueued after the backward pass.
+// The optimizer kernels read the step's gate word and leave every buffer as it is when the step
+// failed (a bounded wait gave up, a token or label was out of range, the loss is not finite).
 void enqueue_update(hift_ctx* c) {
   GroupRec& gr = c->groups[c->last_group];
   const int sl = c->cur_sl;
+  SlotRec* sr = c->offload ? &c->slot[sl] : nullptr;
   const double lr = c->cur_lr;
+  step_gate_kernel<<<1, 32, 0, c->st>>>(c->scal, c->mixed ? gemm_tc_error_device_ptr() : nullptr, c->gate);
+  c->note(cudaGetLastError());
+  if (c->offload) {
+    c->note(cudaEventRecord(c->tl[3], c->st));
+    c->note(cudaStreamWaitEvent(c->st, sr->ev_h2d, 0));
+    // a group still resident from an earlier step: its write-back reads what is about to change
+    if (sr->d2h_pending) c->note(cudaStreamWaitEvent(c->st, sr->ev_d2h, 0));
+    c->note(cudaEventRecord(c->tl[4], c->st));
+  }
   // ---------------- group-local optimizer (Algorithm 1: P now points at theta_s only)
   gr.tau += 1;
   if (c->af) {
     // Adafactor works tensor by tensor (its statistics are per row and column of each matrix)
-    float* base = c->offload ? (float*)c->slot[sl] : nullptr;
-    if (c->offload) c->note(cudaStreamWaitEvent(c->st, c->ev_h2d[sl], 0));
+    float* base = c->offload ? (float*)sr->mem : nullptr;
     for (int u = gr.unit_lo; u <= gr.unit_hi; ++u)
       for (int ti : c->unit_tens[u]) {
         const TensorRec& r = c->tens[ti];
@@ -747,82 +814,88 @@ void enqueue_update(hift_ctx* c) {
         float* st_t = c->offload ? base + (c->mixed ? gr.numel : 0) + r.af_off : c->af_all + gr.af_base + r.af_off;
         c->pre(HIFT_K_OPT, (double)r.numel * (20.0 + (c->mixed ? 2.0 : 0.0)));
         const int nk = launch_adafactor_tensor(c->st, r.rows, r.cols, c->mixed ? c->P(ti) : nullptr, mst_t, c->G(ti), st_t,
-                                               c->af_scratch, lr, c->oc.eps, c->oc.weight_decay, gr.tau);
+                                               c->af_scratch, lr, c->oc.eps, c->oc.weight_decay, gr.tau, c->gate);
         c->post();
         c->step_launches += nk - 1;
       }
   } else {
-  float *mst, *s0, *s1;
-  void* pbf = nullptr;
-  if (c->offload) {
-    float* base = (float*)c->slot[sl];
-    if (c->compact) { mst = nullptr; s0 = base; s1 = base + gr.numel; pbf = c->params + gr.off * c->es; }
-    else if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
-    else { mst = (float*)c->params + gr.off; s0 = base; s1 = base + gr.numel; }
-    c->note(cudaEventRecord(c->tl[3], c->st));
-    c->note(cudaStreamWaitEvent(c->st, c->ev_h2d[sl], 0));
-    c->note(cudaEventRecord(c->tl[4], c->st));
-  } else {
-    if (c->mixed) { mst = c->master_all + gr.off; pbf = c->params + gr.off * c->es; }
-    else mst = (float*)c->params + gr.off;
-    s0 = c->s0_all ? c->s0_all + gr.off : nullptr;
-    s1 = c->s1_all ? c->s1_all + gr.off : nullptr;
-  }
-  const OptScalars hs = make_opt_scalars(c->oc.kind, lr, c->oc.beta1, c->oc.beta2, c->oc.eps,
-                                         c->oc.weight_decay, c->oc.momentum, gr.tau);
-  if (c->compact) {
-    // read p, lo, carry, gradient, state; write p, lo, carry, state
-    const double opt_bytes = (double)gr.numel * (12.25 + 8.0 * c->n_state);
-    uint16_t* lo16 = (uint16_t*)((float*)c->slot[sl] + gr.state_floats);
-    uint8_t* carry8 = (uint8_t*)(lo16 + gr.numel);
-    LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, gr.numel, pbf, lo16, carry8, c->grad, s0, s1, hs));
-  } else {
-  const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
-  LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs));
-  }
+    float *mst, *s0, *s1;
+    void* pbf = nullptr;
+    if (c->offload) {
+      float* base = (float*)sr->mem;
+      if (c->compact) { mst = nullptr; s0 = base; s1 = base + gr.numel; pbf = c->params + gr.off * c->es; }
+      else if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
+      else { mst = (float*)c->params + gr.off; s0 = base; s1 = base + gr.numel; }
+    } else {
+      if (c->mixed) { mst = c->master_all + gr.off; pbf = c->params + gr.off * c->es; }
+      else mst = (float*)c->params + gr.off;
+      s0 = c->s0_all ? c->s0_all + gr.off : nullptr;
+      s1 = c->s1_all ? c->s1_all + gr.off : nullptr;
+    }
+    const OptScalars hs = make_opt_scalars(c->oc.kind, lr, c->oc.beta1, c->oc.beta2, c->oc.eps,
+                                           c->oc.weight_decay, c->oc.momentum, gr.tau);
+    if (c->compact) {
+      // read p, lo, carry, gradient, state; write p, lo, carry, state
+      const double opt_bytes = (double)gr.numel * (12.25 + 8.0 * c->n_state);
+      uint16_t* lo16 = (uint16_t*)((float*)sr->mem + gr.state_floats);
+      uint8_t* carry8 = (uint8_t*)(lo16 + gr.numel);
+      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, gr.numel, pbf, lo16, carry8, c->grad, s0, s1, hs, c->gate));
+    } else {
+      const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
+      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs, c->gate));
+    }
   }
 
   // ---------------- state back to the host (step k)
   if (c->offload) {
-    c->note(cudaEventRecord(c->ev_opt[sl], c->st));
-    c->note(cudaStreamWaitEvent(c->st_d2h, c->ev_opt[sl], 0));
+    c->note(cudaEventRecord(sr->ev_opt, c->st));
+    c->note(cudaStreamWaitEvent(c->st_d2h, sr->ev_opt, 0));
     c->note(cudaEventRecord(c->tl[5], c->st_d2h));
-    c->note(cudaMemcpyAsync(gr.blob, c->slot[sl], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st_d2h));
+    c->note(cudaMemcpyAsync(gr.blob, sr->mem, gr.blob_bytes, cudaMemcpyDeviceToHost, c->st_d2h));
     c->note(cudaEventRecord(c->tl[6], c->st_d2h));
-    c->note(cudaEventRecord(c->ev_d2h[sl], c->st_d2h));
+    c->note(cudaEventRecord(sr->ev_d2h, c->st_d2h));
     c->tl_valid = true;
-    c->d2h_pending[sl] = true;
+    sr->d2h_pending = true;
     c->step_d2h = gr.blob_bytes;
   }
 }
 
 // Publishes the step's scalars, waits for the compute stream, and turns what it finds into a status.
-hift_status finish_step(hift_ctx* c, float* loss_host, bool advance) {
+// `updated`: the optimizer was enqueued too, so the published gate word says whether it ran.
+hift_status finish_step(hift_ctx* c, float* loss_host, bool updated) {
   // the loss goes to mapped host memory by a kernel store: a copy would queue behind the state transfers
   publish_scalars_kernel<<<1, 32, 0, c->st>>>(c->scal, c->mixed ? gemm_tc_error_device_ptr() : nullptr, c->scal_host_dev);
   c->note(cudaGetLastError());
   c->note(cudaStreamSynchronize(c->st));
   c->prof_collect();
-  if (advance) c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
   if (c->first_err != cudaSuccess) return HIFT_ERR_CUDA;
-  int tc_err;
+  int tc_err, bad_h, gate_h;
   memcpy(&tc_err, &c->scal_host[3], sizeof(int));
-  if (tc_err > 0) return HIFT_ERR_TIMEOUT;
-  const float loss = c->scal_host[0];
-  int bad_h;
   memcpy(&bad_h, &c->scal_host[2], sizeof(int));
+  memcpy(&gate_h, &c->scal_host[4], sizeof(int));
+  const float loss = c->scal_host[0];
+  if (tc_err != 0) return HIFT_ERR_TIMEOUT;
   if (loss_host) *loss_host = loss;
   if (bad_h) return HIFT_ERR_INPUT;
   if (!isfinite(loss)) return HIFT_ERR_NONFINITE;
+  if (updated && gate_h != 0) return HIFT_ERR_TIMEOUT;     // the flag was raised between the two reads
   return HIFT_OK;
+}
+// A step that failed changed nothing on the device (the gate kept the optimizer out, the write-back
+// carried unchanged bytes): take back the update count; t stays, so the same group is next.
+void step_failed(hift_ctx* c) {
+  if (c->last_group >= 0 && c->groups[c->last_group].tau > 0) c->groups[c->last_group].tau -= 1;
 }
 
 hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
   if (c->pending_update) return HIFT_ERR_CFG;       // hift_step_begin without hift_step_end
-  const hift_status s = enqueue_forward_backward(c, tok, lab);
+  hift_status s = enqueue_forward_backward(c, tok, lab);
   if (s != HIFT_OK) return s;
   enqueue_update(c);
-  return finish_step(c, loss_host, true);
+  s = finish_step(c, loss_host, true);
+  if (s == HIFT_OK) c->t += 1;     // the learning rate is a function of t / k: it moves once per full cycle
+  else step_failed(c);
+  return s;
 }
 
 void sync_all(hift_ctx* c) {
@@ -923,7 +996,11 @@ void hift_destroy(hift_ctx* c) {
   if (c->scal_host) cudaFreeHost(c->scal_host);
   for (auto e : c->ev_pool) cudaEventDestroy(e);
   if (c->events_made) {
-    for (int i = 0; i < 2; ++i) { cudaEventDestroy(c->ev_h2d[i]); cudaEventDestroy(c->ev_opt[i]); cudaEventDestroy(c->ev_d2h[i]); }
+    for (int i = 0; i < kMaxSlots; ++i) {
+      SlotRec& sr = c->slot[i];
+      cudaEventDestroy(sr.ev_h2d); cudaEventDestroy(sr.ev_opt); cudaEventDestroy(sr.ev_d2h);
+      cudaEventDestroy(sr.tl_h2d0); cudaEventDestroy(sr.tl_h2d1);
+    }
     cudaEventDestroy(c->ev_fwd);
     cudaEventDestroy(c->ev_in);
     for (int i = 0; i < 7; ++i) cudaEventDestroy(c->tl[i]);
@@ -962,6 +1039,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     if (sum != (int64_t)m->n_blocks + 2) return HIFT_ERR_CFG;
   }
   if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
+  if (oc->prefetch_groups < 0 || oc->prefetch_groups > kMaxSlots - 1) return HIFT_ERR_CFG;
   if (oc->sched == 1 && (oc->total_cycles < 1 || oc->warmup_cycles < 0 || oc->warmup_cycles >= oc->total_cycles)) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
@@ -979,7 +1057,10 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   c->n_state = oc->kind == 0 ? 2 : (oc->kind >= 3 ? 0 : 1);
   // plain SGD on fp32 parameters has nothing to page (the paper's "no state, zero traffic" case)
   c->offload = oc->offload_state != 0 && ((m->dtype == 1 ? 1 : 0) + c->n_state + (c->af ? 1 : 0)) > 0;
-  c->n_slots = (c->offload && oc->prefetch_groups) ? 2 : 1;
+  // prefetch_groups p: 0 = one slot, upload after the forward pass; 1 = two slots, upload at the start of
+  // the group's own step; p >= 2 = p + 1 slots, uploads issued p - 1 steps ahead
+  c->n_slots = c->offload ? 1 + oc->prefetch_groups : 1;
+  c->lookahead = c->offload && oc->prefetch_groups >= 2 ? oc->prefetch_groups - 1 : 0;
   // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
   c->compact = c->mixed && c->offload && !c->af;
   c->recompute = oc->recompute != 0;
@@ -1007,10 +1088,13 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
 
   hift_status rc = HIFT_OK;
   auto fail = [&](hift_status s) { hift_destroy(c); return s; };
-  for (int i = 0; i < 2; ++i) {
-    cudaEventCreateWithFlags(&c->ev_h2d[i], cudaEventDisableTiming);
-    cudaEventCreateWithFlags(&c->ev_opt[i], cudaEventDisableTiming);
-    cudaEventCreateWithFlags(&c->ev_d2h[i], cudaEventDisableTiming);
+  for (int i = 0; i < kMaxSlots; ++i) {
+    SlotRec& sr = c->slot[i];
+    cudaEventCreateWithFlags(&sr.ev_h2d, cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&sr.ev_opt, cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&sr.ev_d2h, cudaEventDisableTiming);
+    cudaEventCreate(&sr.tl_h2d0);
+    cudaEventCreate(&sr.tl_h2d1);
   }
   cudaEventCreateWithFlags(&c->ev_fwd, cudaEventDisableTiming);
   for (int i = 0; i < 7; ++i) cudaEventCreate(&c->tl[i]);
@@ -1034,8 +1118,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if ((rc = dev_alloc(c, (void**)&c->grad, c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
   if (c->offload) {
     for (int s = 0; s < c->n_slots; ++s) {
-      if ((rc = dev_alloc(c, (void**)&c->slot[s], slot_bytes_max)) != HIFT_OK) return fail(rc);
-      cudaMemsetAsync(c->slot[s], 0, slot_bytes_max, c->st);
+      if ((rc = dev_alloc(c, (void**)&c->slot[s].mem, slot_bytes_max)) != HIFT_OK) return fail(rc);
+      cudaMemsetAsync(c->slot[s].mem, 0, slot_bytes_max, c->st);
     }
     for (auto& g : c->groups) {
       g.blob_bytes = blob_bytes_of(g);
@@ -1071,7 +1155,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     if ((rc = dev_alloc(c, (void**)&c->af_scratch, mx * sizeof(float))) != HIFT_OK) return fail(rc);
   }
   // four scalars the step publishes, then a staging row for the key-length table
-  if (cudaHostAlloc((void**)&c->scal_host, (4 + (size_t)c->B) * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
+  if (cudaHostAlloc((void**)&c->scal_host, (kScalWords + (size_t)c->B) * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
   if (cudaHostGetDevicePointer((void**)&c->scal_host_dev, c->scal_host, 0) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
   // ---- activation arena: fixed work buffers, one scratch copy of every slot, then the
@@ -1105,7 +1189,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     const size_t maxcols = std::max<size_t>(std::max<size_t>(3 * d, c->fa), 8);
     c->partial = (float*)arena_take(c, 2 * kColChunks * maxcols * sizeof(float));
     c->rowloss = (float*)arena_take(c, T * sizeof(float));
-    c->scal = (float*)arena_take(c, 4 * sizeof(float));
+    c->scal = (float*)arena_take(c, kScalWords * sizeof(float));
+    c->gate = (int*)(c->scal + 4);
     if (m->arch == 2) c->rope_cs = (float*)arena_take(c, 2 * (size_t)c->S * (c->dh / 2) * sizeof(float));
     for (int s = 0; s < S_NUM; ++s)
       c->slots[c->L][s] = (slot_min_level(m->arch, s) == 99 || s == S_XIN || s == S_XINA)
@@ -1147,7 +1232,7 @@ hift_status hift_step_begin(hift_ctx* c, const int32_t* tok, const int32_t* lab,
   hift_status s = enqueue_forward_backward(c, tok, lab);
   if (s != HIFT_OK) return s;
   s = finish_step(c, loss_host, false);
-  if (s == HIFT_OK || s == HIFT_ERR_NONFINITE) c->pending_update = true;
+  if (s == HIFT_OK) c->pending_update = true;
   return s;
 }
 hift_status hift_grad_view(hift_ctx* c, float** grad_dev, size_t* n) {
@@ -1163,10 +1248,15 @@ hift_status hift_step_end(hift_ctx* c) {
   c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
   enqueue_update(c);
   c->pending_update = false;
-  c->note(cudaStreamSynchronize(c->st));
-  c->prof_collect();
-  c->t += 1;
-  return c->first_err == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+  const hift_status s = finish_step(c, nullptr, true);
+  if (s == HIFT_OK) c->t += 1;
+  else step_failed(c);
+  return s;
+}
+hift_status hift_step_abort(hift_ctx* c) {
+  if (!c || !c->pending_update) return HIFT_ERR_CFG;
+  c->pending_update = false;       // the gradient is dropped; the state uploaded for the step stays resident
+  return HIFT_OK;
 }
 
 namespace {
@@ -1194,8 +1284,8 @@ hift_status hift_set_key_lengths(hift_ctx* c, const int32_t* lens_host) {
   if (lens_host == nullptr) { c->use_lens = false; return HIFT_OK; }
   for (int b = 0; b < c->B; ++b) if (lens_host[b] < 1 || lens_host[b] > c->S) return HIFT_ERR_INPUT;
   c->note(cudaStreamSynchronize(c->st));                 // nothing enqueued earlier still reads the staging row
-  memcpy(c->scal_host + 4, lens_host, (size_t)c->B * sizeof(int32_t));
-  copy_i32_kernel<<<1, 256, 0, c->st>>>((const int32_t*)(c->scal_host_dev + 4), c->lens_dev, (size_t)c->B);
+  memcpy(c->scal_host + kScalWords, lens_host, (size_t)c->B * sizeof(int32_t));
+  copy_i32_kernel<<<1, 256, 0, c->st>>>((const int32_t*)(c->scal_host_dev + kScalWords), c->lens_dev, (size_t)c->B);
   c->note(cudaGetLastError());
   c->note(cudaStreamSynchronize(c->st));
   c->use_lens = c->first_err == cudaSuccess;
@@ -1227,6 +1317,7 @@ hift_status hift_group_units(const hift_ctx* c, int32_t g, int32_t* lo, int32_t*
 }
 hift_status hift_force_group(hift_ctx* c, int32_t g) {
   if (g < -1 || g >= (int)c->groups.size()) return HIFT_ERR_CFG;
+  if (g != c->forced) drop_reservations(c);     // uploads made for the schedule's coming steps stay resident, unreserved
   c->forced = g;
   return HIFT_OK;
 }
@@ -1247,6 +1338,7 @@ hift_status hift_tensor_info(const hift_ctx* c, int32_t ti, char* name, int32_t*
 hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !src || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   sync_all(c);
+  invalidate_slots(c);
   bool on_host;
   float* mp = plane_ptr(c, ti, 0, &on_host);
   // every copy goes through the context's stream, so the cast below is ordered after its input
@@ -1324,27 +1416,28 @@ hift_status hift_get_grad(hift_ctx* c, int32_t ti, float* dst, size_t n) {
 
 hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
   sync_all(c);
+  invalidate_slots(c);
   for (size_t g = 0; g < c->groups.size(); ++g) {
     GroupRec& gr = c->groups[g];
-    if (c->offload) cudaMemsetAsync(c->slot[0], 0, gr.blob_bytes, c->st);
+    if (c->offload) cudaMemsetAsync(c->slot[0].mem, 0, gr.blob_bytes, c->st);
     if (c->compact) cudaMemsetAsync(c->grad, 0, gr.numel * sizeof(float), c->st);     // alignment gaps pack to zero
     for (int u = gr.unit_lo; u <= gr.unit_hi; ++u) {
       for (int ti : c->unit_tens[u]) {
         const TensorRec& r = c->tens[ti];
         float* mp = nullptr;
         if (c->compact) mp = c->grad + (r.off - gr.off);           // staged as floats, packed below
-        else if (c->mixed) mp = c->offload ? (float*)c->slot[0] + (r.off - gr.off) : c->master_all + r.off;
+        else if (c->mixed) mp = c->offload ? (float*)c->slot[0].mem + (r.off - gr.off) : c->master_all + r.off;
         const uint64_t sd = seed * 0x9E3779B97F4A7C15ull + (uint64_t)ti * 0xD1B54A32D192ED03ull;
         if (c->mixed) init_tensor_kernel<bf16><<<grid_for(r.numel, 256), 256, 0, c->st>>>((bf16*)c->P(ti), mp, r.numel, r.init_kind, (float)stdv, sd);
         else init_tensor_kernel<float><<<grid_for(r.numel, 256), 256, 0, c->st>>>((float*)c->P(ti), nullptr, r.numel, r.init_kind, (float)stdv, sd);
       }
     }
     if (c->compact) {
-      uint16_t* lo16 = (uint16_t*)((float*)c->slot[0] + gr.state_floats);
+      uint16_t* lo16 = (uint16_t*)((float*)c->slot[0].mem + gr.state_floats);
       master_pack_kernel<<<grid_for(gr.numel / 8, 256), 256, 0, c->st>>>(c->grad, lo16, (uint8_t*)(lo16 + gr.numel), gr.numel / 8);
     }
     if (c->offload) {
-      cudaMemcpyAsync(gr.blob, c->slot[0], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st);
+      cudaMemcpyAsync(gr.blob, c->slot[0].mem, gr.blob_bytes, cudaMemcpyDeviceToHost, c->st);
       if (cudaStreamSynchronize(c->st) != cudaSuccess) return HIFT_ERR_CUDA;
     }
     gr.tau = 0;
@@ -1474,7 +1567,7 @@ hift_status hift_load(hift_ctx* c, const char* path) {
   fclose(f);
   if (!ok) return HIFT_ERR_INPUT;
   c->t = (int64_t)h.t;
-  c->d2h_pending[0] = c->d2h_pending[1] = false;
+  invalidate_slots(c);
   return HIFT_OK;
 }
 
@@ -1502,12 +1595,15 @@ hift_status hift_last_step_paging(const hift_ctx* c, size_t* h2d, size_t* d2h) {
 
 hift_status hift_last_step_timeline(hift_ctx* c, double* ms6) {
   if (!c || !ms6) return HIFT_ERR_CFG;
-  for (int i = 0; i < 6; ++i) ms6[i] = -1.0;
+  for (int i = 0; i < 6; ++i) ms6[i] = nan("");
   if (!c->offload || !c->tl_valid) return HIFT_OK;
   sync_all(c);
+  const SlotRec& sr = c->slot[c->cur_sl];
+  const cudaEvent_t ev[6] = {sr.tl_h2d0, sr.tl_h2d1, c->tl[3], c->tl[4], c->tl[5], c->tl[6]};
   for (int i = 0; i < 6; ++i) {
+    if (i < 2 && sr.h2d_for_step < 0) continue;        // never uploaded
     float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, c->tl[0], c->tl[i + 1]) == cudaSuccess) ms6[i] = ms;
+    if (cudaEventElapsedTime(&ms, c->tl[0], ev[i]) == cudaSuccess) ms6[i] = ms;
     else cudaGetLastError();
   }
   return HIFT_OK;

@@ -8,6 +8,8 @@
 //   U = g / max(sqrt(V), eps1);  theta <- theta - alpha / max(1, RMS(U)/d) * U
 // State per matrix is n + m floats instead of n*m: this is why the paper lists Adafactor with
 // sub-megabyte optimizer-state traffic.  All reductions have a fixed order.
+// `gate` (device int, may be null): when non-zero, every kernel that would write state or
+// parameters returns at once (the training step failed; nothing may change).
 #pragma once
 #include "common.cuh"
 
@@ -17,7 +19,9 @@ struct AfScalars { float w, rho, eps1, eps2, d, decay; };
 
 // per row i: R_i <- lerp(R_i, mean_j g_ij^2, w);  row_tsq[i] = sum_j theta_ij^2
 __global__ void af_row_kernel(const float* __restrict__ g, const float* __restrict__ theta,
-                              float* __restrict__ R, float* __restrict__ row_tsq, int cols, float w) {
+                              float* __restrict__ R, float* __restrict__ row_tsq, int cols, float w,
+                              const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;
   __shared__ float red[33];
   const int64_t row = blockIdx.x;
   float a = 0.f, b = 0.f;
@@ -55,7 +59,8 @@ __global__ void af_col_stage1_kernel(const float* __restrict__ g, float* __restr
   }
 }
 __global__ void af_col_stage2_kernel(const float* __restrict__ partial, int nch, int cols, int64_t rows,
-                                     float* __restrict__ Cv, float w) {
+                                     float* __restrict__ Cv, float w, const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;
   const int col = blockIdx.x * blockDim.x + threadIdx.x;
   if (col >= cols) return;
   float t = 0.f;
@@ -101,7 +106,8 @@ __global__ void af_step_kernel(const float* __restrict__ row_usq, int rows, doub
 template <bool HAS_BF16>
 __global__ void af_apply_kernel(bf16* __restrict__ param, float* __restrict__ theta, const float* __restrict__ g,
                                 const float* __restrict__ R, const float* __restrict__ Cv, const float* __restrict__ scal,
-                                int64_t rows, int cols, float eps1, float decay) {
+                                int64_t rows, int cols, float eps1, float decay, const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;
   const size_t n = (size_t)rows * cols;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -116,7 +122,8 @@ __global__ void af_apply_kernel(bf16* __restrict__ param, float* __restrict__ th
 }
 // vectors (one block): V <- lerp(V, g^2, w); scal[1] = alpha; scal[2] = alpha / max(1, RMS(U)/d)
 __global__ void af_vector_kernel(const float* __restrict__ g, const float* __restrict__ theta, float* __restrict__ V,
-                                 int n, float* __restrict__ scal, AfScalars h) {
+                                 int n, float* __restrict__ scal, AfScalars h, const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;
   __shared__ float red[33];
   float a = 0.f, b = 0.f;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
@@ -138,7 +145,8 @@ __global__ void af_vector_kernel(const float* __restrict__ g, const float* __res
 template <bool HAS_BF16>
 __global__ void af_vector_apply_kernel(bf16* __restrict__ param, float* __restrict__ theta, const float* __restrict__ g,
                                        const float* __restrict__ V, const float* __restrict__ scal, int n,
-                                       float eps1, float decay) {
+                                       float eps1, float decay, const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const float u = g[i] * (1.0f / fmaxf(sqrtf(V[i]), eps1));
@@ -155,7 +163,7 @@ inline size_t af_scratch_floats(int64_t rows, int64_t cols) { return (size_t)(2 
 // scratch: at least af_scratch_floats(rows, cols) floats.  Returns the number of kernels launched.
 inline int launch_adafactor_tensor(cudaStream_t st, int64_t rows, int64_t cols, void* param_bf16, float* master,
                                    const float* grad, float* state, float* scratch, double lr, double eps1, double wd,
-                                   int64_t tau) {
+                                   int64_t tau, const int* gate = nullptr) {
   AfScalars h;
   h.w = (float)pow((double)tau, -0.8);
   h.rho = (float)fmin(lr, 1.0 / sqrt((double)tau));
@@ -164,10 +172,10 @@ inline int launch_adafactor_tensor(cudaStream_t st, int64_t rows, int64_t cols, 
   const float e1sq = (float)eps1;     // the clamp is applied after the square root: eps1^2 would underflow in fp32
   if (rows == 1) {
     float* scal = scratch;
-    af_vector_kernel<<<1, 256, 0, st>>>(grad, master, state, (int)cols, scal, h);
+    af_vector_kernel<<<1, 256, 0, st>>>(grad, master, state, (int)cols, scal, h, gate);
     const int grid = (int)((cols + 255) / 256);
-    if (param_bf16) af_vector_apply_kernel<true><<<grid, 256, 0, st>>>((bf16*)param_bf16, master, grad, state, scal, (int)cols, e1sq, h.decay);
-    else af_vector_apply_kernel<false><<<grid, 256, 0, st>>>(nullptr, master, grad, state, scal, (int)cols, e1sq, h.decay);
+    if (param_bf16) af_vector_apply_kernel<true><<<grid, 256, 0, st>>>((bf16*)param_bf16, master, grad, state, scal, (int)cols, e1sq, h.decay, gate);
+    else af_vector_apply_kernel<false><<<grid, 256, 0, st>>>(nullptr, master, grad, state, scal, (int)cols, e1sq, h.decay, gate);
     return 2;
   }
   float* R = state;
@@ -177,20 +185,20 @@ inline int launch_adafactor_tensor(cudaStream_t st, int64_t rows, int64_t cols, 
   float* partial = scratch + 2 * rows;
   float* scal = partial + 64 * (size_t)cols;
   const double numel = (double)rows * (double)cols;
-  af_row_kernel<<<(unsigned)rows, 256, 0, st>>>(grad, master, R, row_tsq, (int)cols, h.w);
+  af_row_kernel<<<(unsigned)rows, 256, 0, st>>>(grad, master, R, row_tsq, (int)cols, h.w, gate);
   int nch = (int)((rows + 31) / 32);
   if (nch > 64) nch = 64;
   if (nch < 1) nch = 1;
   af_col_stage1_kernel<<<dim3((unsigned)((cols + 31) / 32), nch), dim3(32, 8), 0, st>>>(grad, partial, rows, (int)cols);
-  af_col_stage2_kernel<<<(unsigned)((cols + 127) / 128), 128, 0, st>>>(partial, nch, (int)cols, rows, Cv, h.w);
+  af_col_stage2_kernel<<<(unsigned)((cols + 127) / 128), 128, 0, st>>>(partial, nch, (int)cols, rows, Cv, h.w, gate);
   af_scalars_kernel<<<1, 1024, 0, st>>>(R, row_tsq, (int)rows, numel, scal, h);
   af_usq_kernel<<<(unsigned)rows, 256, 0, st>>>(grad, R, Cv, scal, row_usq, (int)cols, e1sq);
   af_step_kernel<<<1, 1024, 0, st>>>(row_usq, (int)rows, numel, scal, h.d);
   size_t n = (size_t)rows * cols;
   size_t g = (n + 255) / 256;
   if (g > 148 * 16) g = 148 * 16;
-  if (param_bf16) af_apply_kernel<true><<<(unsigned)g, 256, 0, st>>>((bf16*)param_bf16, master, grad, R, Cv, scal, rows, (int)cols, e1sq, h.decay);
-  else af_apply_kernel<false><<<(unsigned)g, 256, 0, st>>>(nullptr, master, grad, R, Cv, scal, rows, (int)cols, e1sq, h.decay);
+  if (param_bf16) af_apply_kernel<true><<<(unsigned)g, 256, 0, st>>>((bf16*)param_bf16, master, grad, R, Cv, scal, rows, (int)cols, e1sq, h.decay, gate);
+  else af_apply_kernel<false><<<(unsigned)g, 256, 0, st>>>(nullptr, master, grad, R, Cv, scal, rows, (int)cols, e1sq, h.decay, gate);
   return 7;
 }
 

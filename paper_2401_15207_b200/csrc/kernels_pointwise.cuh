@@ -496,7 +496,23 @@ __global__ void publish_scalars_kernel(const float* __restrict__ src, const int*
                                        volatile float* dst_mapped_host) {
   if (threadIdx.x < 3) dst_mapped_host[threadIdx.x] = src[threadIdx.x];
   if (threadIdx.x == 3) dst_mapped_host[3] = tc_error ? __int_as_float(*tc_error) : 0.f;
+  if (threadIdx.x == 4) dst_mapped_host[4] = src[4];      // the gate word of the step's update
   __threadfence_system();
+}
+
+// The step's gate word, read by every optimizer kernel before its first store: non-zero when the
+// update must not happen.  src = the step's scalars ([0] loss, [2] bad-input flag); tc_error = the
+// tensor-core kernels' time-out flag (may be null).  Codes: the time-out code (> 0), -1 bad input,
+// -2 non-finite loss.
+__global__ void step_gate_kernel(const float* __restrict__ src, const int* __restrict__ tc_error, int* __restrict__ gate) {
+  if (threadIdx.x != 0) return;
+  int v = 0;
+  const int tc = tc_error ? *tc_error : 0;
+  const float loss = src[0];
+  if (tc != 0) v = tc;
+  else if (__float_as_int(src[2]) != 0) v = -1;
+  else if (!(fabsf(loss) <= 3.402823466e38f)) v = -2;
+  *gate = v;
 }
 
 // ------------------------------------------------------------------ fused group optimizer
@@ -533,7 +549,9 @@ __device__ __forceinline__ void opt_update(float& th, float g, float& s0, float&
 template <int KIND, bool HAS_BF16>
 __global__ void __launch_bounds__(256)
 fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const float* __restrict__ grad,
-                 float* __restrict__ s0, float* __restrict__ s1, size_t n, OptScalars h) {
+                 float* __restrict__ s0, float* __restrict__ s1, size_t n, OptScalars h,
+                 const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;        // the step failed: every buffer keeps its bits
   const size_t n4 = n / 4;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -599,7 +617,8 @@ template <int KIND>
 __global__ void __launch_bounds__(256)
 fused_opt_compact_kernel(uint16_t* __restrict__ param, uint16_t* __restrict__ lo16, uint8_t* __restrict__ carry8,
                          const float* __restrict__ grad, float* __restrict__ s0, float* __restrict__ s1,
-                         size_t n8, OptScalars h) {
+                         size_t n8, OptScalars h, const int* __restrict__ gate) {
+  if (gate != nullptr && *gate != 0) return;        // the step failed: every buffer keeps its bits
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (; i < n8; i += stride) {

@@ -212,24 +212,26 @@ inline OptScalars make_opt_scalars(int kind, double lr, double b1, double b2, do
   return h;
 }
 inline void launch_fused_opt(cudaStream_t st, int kind, size_t n, void* param_bf16, float* master,
-                             const float* grad, float* s0, float* s1, const OptScalars& h) {
+                             const float* grad, float* s0, float* s1, const OptScalars& h,
+                             const int* gate = nullptr) {
   if (n == 0) return;
   const int block = 256;
   int grid = grid_for((n + 3) / 4, block, 148 * 8);
 #define OPT(K)                                                                                         \
-  if (param_bf16) fused_opt_kernel<K, true><<<grid, block, 0, st>>>((bf16*)param_bf16, master, grad, s0, s1, n, h); \
-  else fused_opt_kernel<K, false><<<grid, block, 0, st>>>(nullptr, master, grad, s0, s1, n, h)
+  if (param_bf16) fused_opt_kernel<K, true><<<grid, block, 0, st>>>((bf16*)param_bf16, master, grad, s0, s1, n, h, gate); \
+  else fused_opt_kernel<K, false><<<grid, block, 0, st>>>(nullptr, master, grad, s0, s1, n, h, gate)
   if (kind == 0) { OPT(0); } else if (kind == 1) { OPT(1); } else if (kind == 2) { OPT(2); } else { OPT(3); }
 #undef OPT
 }
 
 // compact master (bf16 copy + low halves + carry bits); n must be a multiple of 8
 inline void launch_fused_opt_compact(cudaStream_t st, int kind, size_t n, void* param_bf16, uint16_t* lo16, uint8_t* carry8,
-                                     const float* grad, float* s0, float* s1, const OptScalars& h) {
+                                     const float* grad, float* s0, float* s1, const OptScalars& h,
+                                     const int* gate = nullptr) {
   if (n == 0) return;
   const size_t n8 = n / 8;
   const int grid = grid_for(n8, 256, 148 * 8);
-#define OPTC(K) fused_opt_compact_kernel<K><<<grid, 256, 0, st>>>((uint16_t*)param_bf16, lo16, carry8, grad, s0, s1, n8, h)
+#define OPTC(K) fused_opt_compact_kernel<K><<<grid, 256, 0, st>>>((uint16_t*)param_bf16, lo16, carry8, grad, s0, s1, n8, h, gate)
   if (kind == 0) { OPTC(0); } else if (kind == 1) { OPTC(1); } else if (kind == 2) { OPTC(2); } else { OPTC(3); }
 #undef OPTC
 }

@@ -229,11 +229,8 @@ def test_timeout_flag_path_reports_and_recovers():
         assert e.value.status == 6                      # HIFT_ERR_TIMEOUT
     finally:
         assert tc_error_flag(0) == 0
-    h.set_params(p0)                                    # the aborted step updated group 0 from garbage
-    h2 = HiFT(cfg, gc, oc)                              # a fresh context and the recovered one agree with the reference
-    h2.set_params(p0)
-    assert h2.step(tt, ll) == good[0]
-    h2.close()
+    assert h.step_count() == 0                          # the refused step did not count
+    assert [h.step(tt, ll) for _ in range(2)] == good   # and changed nothing: the context goes on like the reference
     h.close()
 
 
@@ -315,7 +312,8 @@ def test_paged_master_round_trip_is_exact(kind):
 
 @pytest.mark.parametrize("kind", [0, 1, 2, synth.OPT_SGD])
 def test_paged_and_resident_state_give_identical_bits(kind):
-    """Keeping the state on the GPU (fp32 master) and paging it (compact master) are two storage
+    """Keeping the state on the GPU (fp32 master) and paging it (compact master; one slot in the paper's
+    order, two slots, or a ring of three / four slots whose uploads run one / two steps ahead) are storage
     forms of the same numbers: after two cycles every master value and state value agrees bit for bit."""
     import torch
     from paper_2401_15207_b200 import HiFT
@@ -323,7 +321,7 @@ def test_paged_and_resident_state_give_identical_bits(kind):
     gc = synth.GroupCfg(layers_per_group=1, order=1)
     p0 = synth.init_params(cfg, 3, perturb=0.05)
     ctxs = []
-    for offload, prefetch in ((0, 0), (1, 1), (1, 0)):
+    for offload, prefetch in ((0, 0), (1, 1), (1, 0), (1, 2), (1, 3)):
         oc = synth.OptCfg(kind=kind, lr=1e-2, eps=1e-8, momentum=0.9, weight_decay=0.01, offload_state=offload,
                           prefetch_groups=prefetch)
         h = HiFT(cfg, gc, oc)
@@ -335,7 +333,7 @@ def test_paged_and_resident_state_give_identical_bits(kind):
             tok, lab = synth.batch_for(cfg, 11, t, "zipf")
             dt, dl = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
             losses = [h.step(dt, dl) for h in ctxs]
-            assert losses[0] == losses[1] == losses[2]
+            assert all(l == losses[0] for l in losses)
         n_state = {0: 2, 1: 1, 2: 1}.get(kind, 0)
         for name in ctxs[0].tensor_names():
             ref = np.asarray(ctxs[0].get_param(name)).view(np.uint32)
@@ -350,6 +348,132 @@ def test_paged_and_resident_state_give_identical_bits(kind):
     finally:
         for h in ctxs:
             h.close()
+
+
+def _state_bits(h, n_state):
+    out = {}
+    for name in h.tensor_names():
+        out[name] = [np.asarray(h.get_param(name)).view(np.uint32).copy(),
+                     np.asarray(h.get_model_param(name)).view(np.uint32).copy()]
+        for w in range(n_state):
+            out[name].append(np.asarray(h.get_state(name, w)).view(np.uint32).copy())
+        if h.opt.kind == 4:
+            rows = h.tensor_info(name)[1][0]
+            for w in range(1 if rows == 1 else 2):
+                out[name].append(np.asarray(h.get_factored_state(name, w)).view(np.uint32).copy())
+    return out
+
+
+def _same_bits(a, b):
+    for name in a:
+        for x, y in zip(a[name], b[name]):
+            assert np.array_equal(x, y), name
+
+
+@pytest.mark.parametrize("prefetch", [0, 1, 2, 3])
+@pytest.mark.parametrize("case", ["one_group", "forced", "two_groups", "forced_then_schedule"])
+def test_paging_when_a_group_trains_on_consecutive_steps(case, prefetch):
+    """A group that is trained again before (or while) its write-back lands must be updated from its
+    latest values: one group holding every unit (k = 1, the full-parameter identity of Eq. 2-3), a
+    forced group, fewer groups than state slots, and leaving a forced group with uploads of the
+    schedule's groups outstanding.  The paged run keeps the bits of the run with the state resident."""
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(0, synth.DTYPE_BF16, tie_head=1)
+    n = cfg.n_units
+    gc = {"one_group": synth.GroupCfg(layers_per_group=n), "forced": synth.GroupCfg(1),
+          "two_groups": synth.GroupCfg(layers_per_group=(n + 1) // 2),
+          "forced_then_schedule": synth.GroupCfg(1)}[case]
+    p0 = synth.init_params(cfg, 3, perturb=0.05)
+    ctxs = []
+    for offload in (0, 1):
+        h = HiFT(cfg, gc, synth.OptCfg(kind=0, lr=1e-2, weight_decay=0.01, offload_state=offload,
+                                       prefetch_groups=prefetch if offload else 0))
+        h.set_params(p0)
+        ctxs.append(h)
+    try:
+        for t in range(7):
+            if case == "forced":
+                for h in ctxs:
+                    h.force_group(2 if t < 4 else 1)
+            if case == "forced_then_schedule":
+                for h in ctxs:
+                    h.force_group(3 if 2 <= t < 5 else -1)
+            tok, lab = synth.batch_for(cfg, 11, t, "zipf")
+            dt, dl = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
+            assert ctxs[0].active_group() == ctxs[1].active_group()
+            a, b = ctxs[0].step(dt, dl), ctxs[1].step(dt, dl)
+            assert a == b, (t, a, b)
+        _same_bits(_state_bits(ctxs[0], 2), _state_bits(ctxs[1], 2))
+    finally:
+        for h in ctxs:
+            h.close()
+
+
+@pytest.mark.parametrize("kind,offload,prefetch,dtype", [(0, 1, 2, synth.DTYPE_BF16), (0, 0, 0, synth.DTYPE_BF16),
+                                                         (4, 1, 1, synth.DTYPE_BF16), (2, 1, 0, synth.DTYPE_FP32)])
+def test_a_failed_step_changes_nothing(kind, offload, prefetch, dtype):
+    """A step that reports a time-out (walked with the host-set flag: nothing stalls), a bad label or a
+    non-finite loss (a NaN planted in a parameter of a frozen group through hift_set_param) leaves every
+    parameter, master and state bit of every group as it was, does not advance t or the group's update
+    count, and the same context then continues exactly like one that never saw the failure."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError, tc_error_flag
+    cfg = synth.ModelCfg(arch=2, n_blocks=2, d_model=256, n_heads=2, d_ffn=512, vocab=1000, norm_eps=1e-6,
+                         dtype=dtype, batch=2, seq=128)
+    gc = synth.GroupCfg(1)
+    oc = synth.OptCfg(kind=kind, lr=1e-3, eps=1e-8 if kind != 4 else 1e-30, weight_decay=0.01,
+                      offload_state=offload, prefetch_groups=prefetch)
+    n_state = {0: 2, 1: 1, 2: 1}.get(kind, 0)
+    p0 = synth.init_params(cfg, 3)
+    batches = [tuple(torch.from_numpy(a).cuda() for a in synth.lm_batch(cfg, 1, t)) for t in range(6)]
+    ref, h = HiFT(cfg, gc, oc), HiFT(cfg, gc, oc)
+    try:
+        for c in (ref, h):
+            c.set_params(p0)
+            for t in range(2):
+                c.step(*batches[t])
+        before = _state_bits(h, n_state)
+        # (1) time-out flag (only the tensor-core path reads it)
+        if dtype == synth.DTYPE_BF16:
+            try:
+                assert tc_error_flag(2) == 2
+                with pytest.raises(HiftError) as e:
+                    h.step(*batches[2])
+                assert e.value.status == 6
+            finally:
+                assert tc_error_flag(0) == 0
+            assert h.step_count() == 2 and h.active_group() == ref.active_group()
+            _same_bits(before, _state_bits(h, n_state))
+        # (2) a label beyond the vocabulary
+        bad = batches[2][1].clone()
+        bad[0, 3] = cfg.vocab + 7
+        with pytest.raises(HiftError) as e:
+            h.step(batches[2][0], bad)
+        assert e.value.status == 4 and h.step_count() == 2
+        _same_bits(before, _state_bits(h, n_state))
+        # (3) non-finite loss: NaN in a tensor of a group that is not the active one
+        g = h.active_group()
+        lo, hi = h.group_units(g)
+        victim = [n for n in h.tensor_names() if not (lo <= h.tensor_info(n)[0] <= hi) and n.endswith("w_o")][0]
+        good = h.get_param(victim)
+        poisoned = good.copy()
+        poisoned[0, 0] = np.nan
+        h.set_param(victim, poisoned)
+        with_nan = _state_bits(h, n_state)
+        with pytest.raises(HiftError) as e:
+            h.step(*batches[2])
+        assert e.value.status == 5 and h.step_count() == 2
+        _same_bits(with_nan, _state_bits(h, n_state))
+        h.set_param(victim, good)
+        _same_bits(before, _state_bits(h, n_state))
+        # and on it goes, bit for bit like the context that never failed
+        for t in range(2, 6):
+            assert h.step(*batches[t]) == ref.step(*batches[t])
+        _same_bits(_state_bits(ref, n_state), _state_bits(h, n_state))
+    finally:
+        ref.close()
+        h.close()
 
 
 def test_warmup_then_decay_moves_once_per_cycle():
