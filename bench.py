@@ -182,6 +182,129 @@ def run_reference(args, cfg, gcfg, ocfg):
     print(json.dumps(line))
 
 
+def group_plan(k, K, W):
+    """Groups of the W warm-up steps and the K timed steps of one leg.  K a multiple of k: whole cycles of
+    the group ids 0 .. k-1 in ascending order; otherwise K group ids spread evenly over the cycle, both ends
+    (embedding group 0 and head group k-1) included.  The warm-up trains the tail of the same list, so the
+    paging ring is in its steady state when the clock starts.  Every leg uses this one list."""
+    if K % k == 0:
+        sel = [i % k for i in range(K)]
+        kind = f"{K // k} whole cycle(s), groups 0..{k - 1} in ascending order"
+    else:
+        sel = [int(round(i * (k - 1) / max(K - 1, 1))) for i in range(K)]
+        kind = f"{K} groups spread evenly over the cycle of {k} (both ends included)"
+    rot = [sel[(j - W) % K] for j in range(K)]        # step j of a leg trains rot[j % K]
+    return sel, rot, kind
+
+
+def pcie_ceiling(n_bytes=2 << 30, reps=3):
+    """Plain pinned-memory copies of n_bytes on two streams: host-to-device alone, device-to-host alone, both
+    at once (GB/s per direction), timed with CUDA events.  The ceiling of the optimizer-state paging."""
+    import torch
+    h_in = torch.empty(n_bytes, dtype=torch.uint8).pin_memory()
+    h_out = torch.empty(n_bytes, dtype=torch.uint8).pin_memory()
+    h_in.fill_(1)
+    d_in = torch.empty(n_bytes, dtype=torch.uint8, device="cuda")
+    d_out = torch.ones(n_bytes, dtype=torch.uint8, device="cuda")
+    s_up, s_dn = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def run(up, dn):
+        ev = []
+        for st, on, fn in ((s_up, up, lambda: d_in.copy_(h_in, non_blocking=True)),
+                           (s_dn, dn, lambda: h_out.copy_(d_out, non_blocking=True))):
+            if not on:
+                continue
+            with torch.cuda.stream(st):
+                fn()                                   # warm-up
+        torch.cuda.synchronize()
+        for st, on, fn in ((s_up, up, lambda: d_in.copy_(h_in, non_blocking=True)),
+                           (s_dn, dn, lambda: h_out.copy_(d_out, non_blocking=True))):
+            if not on:
+                continue
+            with torch.cuda.stream(st):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    fn()
+                e1.record()
+                ev.append((e0, e1))
+        torch.cuda.synchronize()
+        return [n_bytes * reps / (a.elapsed_time(b) * 1e-3) / 1e9 for a, b in ev]
+
+    up = run(True, False)[0]
+    dn = run(False, True)[0]
+    both = run(True, True)
+    del h_in, h_out, d_in, d_out
+    torch.cuda.empty_cache()
+    return {"h2d_alone_gbs": round(up, 1), "d2h_alone_gbs": round(dn, 1),
+            "both_h2d_gbs": round(both[0], 1), "both_d2h_gbs": round(both[1], 1),
+            "bytes_per_copy": n_bytes, "how": "pinned host memory, one copy stream per direction, CUDA events"}
+
+
+def standalone_kernels(cfg, peaks, launches=20):
+    """The short kernels of a step (tens of microseconds: norms, attention), each launched `launches` times
+    back to back on its own through the single-kernel entry points, at the workload's shapes, over buffer
+    sets that rotate so that consecutive launches do not find their inputs in L2.  An event bracket around a
+    single such launch inside the step would read several microseconds too long."""
+    import torch
+    from paper_2401_15207_b200 import binding as B
+    if cfg.dtype != 1:
+        return {}
+    T, d, H, S, Bt = cfg.tokens_per_step, cfg.d_model, cfg.n_heads, cfg.seq, cfg.batch
+    dh = d // H
+    kind = 1 if cfg.arch == synth.ARCH_LLAMA else 0
+    bf = torch.bfloat16
+    out = {}
+
+    def timed(fn, nsets):
+        for i in range(3):
+            fn(i % nsets)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(launches):
+            fn(i % nsets)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / launches          # microseconds per launch
+
+    def entry(name, us, work, tensor, note):
+        ach = work / (us * 1e-6) / (1e12 if tensor else 1e9)
+        pk = peaks["bf16_tflops_sustained"] if tensor else peaks["hbm_gbs"]
+        out[name] = {"avg_us": round(us, 2), "achieved": round(ach, 1), "unit": "TFLOP/s" if tensor else "GB/s",
+                     "bound": "tensor" if tensor else "hbm", "frac": round(ach / pk, 3), "what": note,
+                     "method": f"standalone loop, {launches} launches, CUDA events, rotating buffers"}
+
+    # norms: fp32 stream in, bf16 operand out (forward); bf16 dy + fp32 x + fp32 add in, fp32 + bf16 dx out (backward)
+    nsets = max(2, int(200e6 // (T * d * 6)) + 1)
+    xs = [torch.randn(T, d, device="cuda") for _ in range(nsets)]
+    ys = [torch.empty(T, d, device="cuda", dtype=bf) for _ in range(nsets)]
+    stats = [torch.empty(2 * T, device="cuda") for _ in range(nsets)]
+    gain = torch.ones(d, device="cuda", dtype=bf)
+    bias = torch.zeros(d, device="cuda", dtype=bf) if kind == 0 else None
+    us = timed(lambda i: B.k_norm_fwd(1, kind, T, d, cfg.norm_eps, xs[i], gain, bias, ys[i], stats[i]), nsets)
+    entry("norm_fwd", us, T * d * 6.0, False, f"[{T}, {d}] fp32 in, bf16 out")
+    dxs = [torch.empty(T, d, device="cuda") for _ in range(nsets)]
+    us = timed(lambda i: B.k_norm_bwd(1, kind, T, d, ys[i], xs[i], stats[i], gain, xs[(i + 1) % nsets], dxs[i], None, None, None), nsets)
+    entry("norm_bwd_dx", us, T * d * 14.0, False, f"[{T}, {d}] bf16 dy, fp32 x and residual gradient in, fp32 out")
+    del xs, ys, dxs
+    if dh in (64, 128):
+        nsets = max(2, int(200e6 // (T * d * 8)) + 1)
+        qkv = [torch.randn(T, 3 * d, device="cuda").to(bf) for _ in range(nsets)]
+        o = [torch.empty(T, d, device="cuda", dtype=bf) for _ in range(nsets)]
+        lse = [torch.empty(Bt * H * S, device="cuda") for _ in range(nsets)]
+        fl = 4.0 * Bt * H * S * S * dh * (0.5 if cfg.causal else 1.0)
+        us = timed(lambda i: B.k_attention_fwd(1, Bt, S, H, dh, cfg.causal, qkv[i], o[i], lse[i]), nsets)
+        entry("attn_fwd", us, fl, True, f"batch {Bt} x seq {S} x {H} heads x {dh}, causal={cfg.causal}")
+        do = [torch.randn(T, d, device="cuda").to(bf) for _ in range(nsets)]
+        dqkv = [torch.empty(T, 3 * d, device="cuda", dtype=bf) for _ in range(nsets)]
+        dsum = torch.empty(T * H, device="cuda")
+        us = timed(lambda i: B.k_attention_bwd(1, Bt, S, H, dh, cfg.causal, qkv[i], o[i], lse[i], do[i], dqkv[i], dsum), nsets)
+        entry("attn_bwd", us, 2.5 * fl, True, "same shape; dsum + dK/dV + dQ launches together")
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, cfg, gcfg, ocfg):
     import torch
     import torch.distributed as dist
@@ -201,80 +324,77 @@ def run_ours(args, cfg, gcfg, ocfg):
 
     ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": args.prefetch, "offload_state": args.offload,
                            "recompute": args.recompute})
+    peaks = measured_peaks()
+    pcie = None
+    if rank == 0 and world == 1 and ocfg.offload_state and not args.no_pcie:
+        pcie = pcie_ceiling()
     h = HiFT(cfg, gcfg, ocfg)
     h.init_synthetic(dist_util.rank_seed(1234, rank), cfg.init_std)
     k = h.num_groups()
     K, W = args.steps, args.warmup
-    n_batches = 2 * (W + K)
-    host = [synth.batch_for(cfg, dist_util.rank_seed(77, rank), t) for t in range(n_batches)]
+    sel, rot, plan_kind = group_plan(k, K, W)
+    host = [synth.batch_for(cfg, dist_util.rank_seed(77, rank), t) for t in range(W + K)]
     # the end-to-end leg copies its inputs from pinned host memory: numpy views of pinned tensors (kept alive here)
     pinned_keep = [tuple(torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).pin_memory() for x in pair) for pair in host]
     host = [tuple(t.numpy() for t in pair) for pair in pinned_keep]
-    dev = [(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for a, b in host[:W + K]]
+    dev = [(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()) for a, b in host]
     groups = [h.group_units(g) for g in range(k)]
 
-    step_host = h.step_host
+    step_dev, step_host = h.step, h.step_host
     if args.parallel == "dp":
-        h.step = lambda tok, lab: dist_util.data_parallel_step(h, tok, lab)
+        step_dev = lambda tok, lab: dist_util.data_parallel_step(h, tok, lab)
         # end to end in this mode: pageable host batch -> device inside the timed call, then the same step
-        step_host = lambda tok, lab: h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
+        step_host = lambda tok, lab: step_dev(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
 
-    # ---- device-resident leg, timed twice over the same K steps' worth of work: once plain (the
-    #      reported value) and once with every kernel launch bracketed by CUDA events on the
-    #      launching stream (the roofline figures; the brackets cost a few per cent)
-    for t in range(W):
-        h.step(*dev[t])
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local)
-    sampler.start()
-    barrier()
-    launches = 0
-    trained = []
-    step_ms = []
-    e0.record()
-    for t in range(W, W + K):
-        trained.append(h.active_group())
-        t_host = time.perf_counter()
-        h.step(*dev[t])                      # returns when the step's loss is on the host
-        step_ms.append(round((time.perf_counter() - t_host) * 1e3, 2))
-        launches += h.last_step_launches()
-    e1.record()
-    barrier()
-    ms = e0.elapsed_time(e1)
-    ms_prof = 0.0
-    if not args.skip_profiled:
-        for _ in range((k - K % k) % k):      # realign so that the profiled pass trains the same groups
-            h.step(*dev[0])
-        h.profile_enable(True)
+
+    paged = []
+
+    def leg(step_fn, batches):
+        """W warm-up steps, then K timed steps, on the groups of group_plan: the same ones in every leg."""
+        h.force_sequence(rot)
+        for t in range(W):
+            step_fn(*batches[t])
+        trained, step_ms, launches, last = [], [], 0, 0.0
+        paged.clear()
         barrier()
         e0.record()
         for t in range(W, W + K):
-            h.step(*dev[t])
+            trained.append(h.active_group())
+            t_host = time.perf_counter()
+            last = step_fn(*batches[t])              # returns when the step's loss is on the host
+            step_ms.append(round((time.perf_counter() - t_host) * 1e3, 2))
+            launches += h.last_step_launches()
+            paged.append(h.last_step_paging()[1])    # bytes written back = this group's paged state
         e1.record()
         barrier()
-        ms_prof = e0.elapsed_time(e1)
+        return e0.elapsed_time(e1), trained, step_ms, launches, last
+
+    # ---- device-resident leg, timed twice over the same K steps: once plain (the reported value) and once
+    #      with every kernel launch bracketed by CUDA events on the launching stream (time shares per class,
+    #      and the roofline figures of the long kernels; the brackets cost a few per cent)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, trained, step_ms, launches, _ = leg(step_dev, dev)
+    assert trained == sel
+    ms_prof = 0.0
+    if not args.skip_profiled:
+        h.profile_enable(True)
+        ms_prof, trained_prof, _, _, _ = leg(step_dev, dev)
+        assert trained_prof == sel
     prof = h.profile()
     h.profile_enable(False)
     clocks = sampler.stop()
     paging = h.last_step_paging()
     timeline = h.last_step_timeline()
-    if not args.skip_profiled and not args.skip_e2e:
-        for _ in range((k - K % k) % k):
-            h.step(*dev[0])
 
     # ---- end-to-end leg: host buffers, copies inside the call
     last_loss = 0.0
     ms_e2e = float("nan")
     if not args.skip_e2e:
-        for t in range(W):
-            step_host(*host[W + K + t])
-        barrier()
-        e0.record()
-        for t in range(K):
-            last_loss = step_host(*host[2 * W + K + t])
-        e1.record()
-        barrier()
-        ms_e2e = e0.elapsed_time(e1)
+        ms_e2e, trained_e2e, _, _, last_loss = leg(step_host, host)
+        assert trained_e2e == sel
+    h.force_sequence([])
 
     ms, ms_e2e = dist_util.max_over_ranks([ms, ms_e2e], device="cuda")
     tokens = cfg.tokens_per_step * K * world
@@ -283,6 +403,9 @@ def run_ours(args, cfg, gcfg, ocfg):
     peak_hbm = h.peak_hbm_bytes()
     pinned = h.pinned_host_bytes()
     h.close()
+    alone = {}
+    if rank == 0 and world == 1 and not args.skip_profiled:
+        alone = standalone_kernels(cfg, peaks)
     full_ref = None
     if world == 1 and not args.no_full_param_reference and not args.full_param and not args.skip_e2e:
         try:
@@ -291,7 +414,6 @@ def run_ours(args, cfg, gcfg, ocfg):
             full_ref = {"unavailable": str(e)[:200]}
 
     if rank == 0:
-        peaks = measured_peaks()
         default_llama = args.workload == "llama7b" and not args.full_param and not args.recompute
         g = {c: prof[c] for c in ("gemm_fwd", "gemm_dx", "gemm_dw")}
         g_launch = sum(v["launches"] for v in g.values())
@@ -313,8 +435,10 @@ def run_ours(args, cfg, gcfg, ocfg):
                                 "tflops": v["work"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0}
                             for c, v in g.items()}}
         kernel_share = {c: round(v["ms"], 3) for c, v in prof.items()}
-        # every kernel class against its own roofline (event-bracketed: the brackets add a few
-        # microseconds per launch, which shows on the short bandwidth-bound kernels)
+        # Every kernel class against its own roofline.  Classes whose launches last hundreds of microseconds
+        # are measured inside the step (one event bracket per launch); for the short ones (norms, attention)
+        # a bracket adds several microseconds per launch, so their roofline figure comes from the standalone
+        # loop and the in-step bracketed time is kept as `in_step_bracketed_us` (an upper bound).
         per_kernel = {}
         for cname, v in prof.items():
             if v["launches"] == 0 or v["ms"] <= 0:
@@ -322,11 +446,15 @@ def run_ours(args, cfg, gcfg, ocfg):
             tensor = cname.startswith("gemm") or cname.startswith("attn")
             ach = v["work"] / (v["ms"] * 1e-3) / (1e12 if tensor else 1e9)
             pk = (peaks["bf16_tflops_sustained"] if cfg.dtype == 1 else None) if tensor else peaks["hbm_gbs"]
-            per_kernel[cname] = {"launches": v["launches"], "ms": round(v["ms"], 3),
-                                 "avg_us": round(1e3 * v["ms"] / v["launches"], 2),
+            avg_us = 1e3 * v["ms"] / v["launches"]
+            per_kernel[cname] = {"launches": v["launches"], "ms": round(v["ms"], 3), "avg_us": round(avg_us, 2),
                                  "achieved": round(ach, 1), "unit": "TFLOP/s" if tensor else "GB/s",
                                  "bound": "tensor" if tensor else "hbm",
-                                 "frac": round(ach / pk, 3) if pk else None}
+                                 "frac": round(ach / pk, 3) if pk else None,
+                                 "method": "in-step event bracket per launch" +
+                                           (" (short launches: time is an upper bound, frac a lower bound)" if avg_us < 50 else "")}
+        for name, v in alone.items():
+            per_kernel[name + "_alone"] = v
         opt = prof["optimizer"]
         opt_gbs = opt["work"] / (opt["ms"] * 1e-3) / 1e9 if opt["ms"] > 0 else 0.0
         cpu = None
@@ -335,22 +463,36 @@ def run_ours(args, cfg, gcfg, ocfg):
             full = mean_step_flops(cfg, groups)
             cpu = {"value": cfg.tokens_per_step / (dt * full / flops), "unit": "tokens/s", "cores": threads,
                    "kind": "oracle", "sample": desc, "sample_seconds": dt}
+        if pcie is not None:
+            tl = timeline
+            if tl[1] == tl[1] and tl[0] == tl[0] and tl[1] > tl[0]:
+                pcie["in_step_h2d_gbs"] = round(paging[1] / ((tl[1] - tl[0]) * 1e-3) / 1e9, 1)
+            if tl[5] == tl[5] and tl[5] > tl[4]:
+                pcie["in_step_d2h_gbs"] = round(paging[1] / ((tl[5] - tl[4]) * 1e-3) / 1e9, 1)
+            pcie["paged_bytes_per_step_each_way"] = int(np.mean(paged)) if paged else 0
+            pcie["floor_ms_per_step"] = round(pcie["paged_bytes_per_step_each_way"] /
+                                              (min(pcie["both_h2d_gbs"], pcie["both_d2h_gbs"]) * 1e9) * 1e3, 2)
         line = {
             "metric": "HiFT step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if cfg.dtype == 1 else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "global_batch": cfg.batch * world, "seq_len": cfg.seq,
-                       "groups": k, "groups_trained": trained, "ms_by_step": step_ms, "optimizer": ["adamw", "adagrad", "sgdm"][ocfg.kind],
+                       "groups": k, "groups_timed": plan_kind + "; the warm-up trains the tail of the same list; "
+                       "the plain, the event-bracketed and the end-to-end leg train the same groups",
+                       "groups_trained": trained, "ms_by_step": step_ms,
+                       "optimizer": ["adamw", "adagrad", "sgdm", "sgd", "adafactor"][ocfg.kind],
                        "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups, "recompute": ocfg.recompute,
                        "parallelism": (("dp%d" % world) if args.parallel == "dp" else "replicas") if world > 1 else "single",
                        "l2_policy": "inputs larger than L2 (weights + activations of a step exceed 126 MB)"},
+            "cycle_mean_ms": round(float(np.mean(step_ms)), 3),
             "peak_hbm_gb": peak_hbm / 1e9, "pinned_host_gb": pinned / 1e9,
-            "paging_bytes_per_step": {"h2d": paging[0], "d2h": paging[1]},
+            "paging_bytes_last_step": {"h2d_issued": paging[0], "d2h": paging[1]},
             "paging_timeline_ms": dict(zip(["h2d_begin", "h2d_end", "opt_wait_begin", "opt_wait_end", "d2h_begin",
-                                            "d2h_end"], [round(x, 2) for x in timeline])),
+                                            "d2h_end"], [None if x != x else round(x, 2) for x in timeline])),
+            "pcie": pcie,
             "e2e": {"value": e2e_value, "unit": "tokens/s",
-                    "h2d_bytes_per_step": int(host[0][0].nbytes + host[0][1].nbytes) + paging[0],
-                    "d2h_bytes_per_step": 4 + paging[1], "ms_per_step": ms_e2e / K, "last_loss": last_loss},
+                    "h2d_bytes_per_step": int(host[0][0].nbytes + host[0][1].nbytes) + (int(np.mean(paged)) if paged else 0),
+                    "d2h_bytes_per_step": 4 + (int(np.mean(paged)) if paged else 0), "ms_per_step": ms_e2e / K, "last_loss": last_loss},
             "gpu_launches": int(launches),
             "roofline": roof,
             "optimizer_gbs": opt_gbs, "optimizer_frac_of_hbm": opt_gbs / peaks["hbm_gbs"],
@@ -473,12 +615,13 @@ def run_sweep_depth(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the tensor-core GEMM launches of one llama7b step (the step that
-# trains block 4: 129 forward, 113 dX, 4 dW launches), from a one-pass ncu capture of this file's own command line;
-# the table with every kernel of the step is profiles/launch_list_llama7b_step.md.
+# trains block 4: 129 forward, 113 dX, 4 dW launches), recorded once from an ncu capture.  A recorded figure, not one
+# to take again on the whole step: after a kernel change, capture one launch per GEMM shape on its own (a few GB on
+# the device) and weight by the launch counts the profile hook reports; time the whole step with CUDA events only.
 NCU_GEMM_TRAFFIC = {
     "bytes_per_launch": 54.199e9 / 246,
-    "note": "ncu, one step (block 4 active): 54.20 GB over 246 GEMM launches = 220.3 MB per launch, against 205.1 MB of "
-            "operands and results per launch (1.07); profiles/launch_list_llama7b_step.md",
+    "note": "ncu, recorded once: 54.20 GB over the 246 GEMM launches of one step (block 4 active) = 220.3 MB per "
+            "launch, against 205.1 MB of operands and results per launch (1.07)",
 }
 
 
@@ -492,7 +635,9 @@ def main():
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "dp"],
                     help="N > 1: independent replicas (default), or data parallel with an NCCL all-reduce of the "
                          "active group's gradient between the backward pass and the update")
-    ap.add_argument("--prefetch", type=int, default=1)
+    ap.add_argument("--prefetch", type=int, default=3,
+                    help="state slots beyond the first (0 paper order, 1 upload at step start, 2-3 uploads one or two steps ahead)")
+    ap.add_argument("--no-pcie", action="store_true", help="leave out the pinned-memcpy ceiling measurement")
     ap.add_argument("--offload", type=int, default=1)
     ap.add_argument("--recompute", type=int, default=0,
                     help="1: frozen blocks above the group keep only their input and are recomputed in the backward pass "

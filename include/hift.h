@@ -173,6 +173,12 @@ double  hift_current_lr(const hift_ctx *ctx);     /* lr the NEXT step will use  
 hift_status hift_group_units(const hift_ctx *ctx, int32_t g, int32_t *unit_lo, int32_t *unit_hi);
 /* Force the group trained by the next steps (depth sweeps); -1 restores the schedule. */
 hift_status hift_force_group(hift_ctx *ctx, int32_t g);
+/* The same for a list: the next steps train groups[0], groups[1], ..., groups[n-1], groups[0], ...
+ * (host array, copied; n = 0 restores the schedule; a forced single group takes precedence).  Unlike
+ * a group forced step by step, the list is known ahead, so look-ahead paging works on it: what a
+ * benchmark uses to time an even sample of the cycle.  t, the learning rate and the update counts
+ * advance as always. */
+hift_status hift_force_sequence(hift_ctx *ctx, const int32_t *groups, int32_t n);
 
 /* High-water mark, in bytes, of all device memory the context holds. */
 size_t hift_peak_hbm_bytes(const hift_ctx *ctx);

@@ -75,6 +75,7 @@ def _prototypes():
         "hift_current_lr": (f64, [vp]),
         "hift_group_units": (C.c_int, [vp, i32, C.POINTER(i32), C.POINTER(i32)]),
         "hift_force_group": (C.c_int, [vp, i32]),
+        "hift_force_sequence": (C.c_int, [vp, vp, i32]),
         "hift_peak_hbm_bytes": (sz, [vp]),
         "hift_pinned_host_bytes": (sz, [vp]),
         "hift_num_tensors": (i32, [vp]),
@@ -257,6 +258,11 @@ class HiFT:
 
     def force_group(self, g: int):
         _check(lib().hift_force_group(self._h, g), "hift_force_group")
+
+    def force_sequence(self, groups):
+        """The next steps train groups[0], groups[1], ... cyclically; an empty list restores the schedule."""
+        a = np.ascontiguousarray(list(groups), dtype=np.int32)
+        _check(lib().hift_force_sequence(self._h, a.ctypes.data if a.size else None, int(a.size)), "hift_force_sequence")
 
     def peak_hbm_bytes(self) -> int:
         return lib().hift_peak_hbm_bytes(self._h)

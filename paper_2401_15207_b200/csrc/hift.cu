@@ -93,6 +93,8 @@ struct hift_ctx {
   size_t total = 0, max_group = 0;
   int64_t t = 0;
   int forced = -1, last_group = -1;
+  std::vector<int> forced_seq;      // hift_force_sequence: groups of the coming steps, cyclic from step forced_seq_t0
+  int64_t forced_seq_t0 = 0;
   int cur_sl = 0; double cur_lr = 0.0;   // slot and learning rate of the step in flight
   bool pending_update = false;           // between hift_step_begin and hift_step_end
 
@@ -615,7 +617,12 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
 // slot, and a slot that holds a group holds its latest values: they change only by the optimizer
 // running in that slot, followed by the write-back from it.
 int group_at(const hift_ctx* c, int64_t step) {
-  return c->forced >= 0 ? c->forced : c->order[step % (int64_t)c->groups.size()];
+  if (c->forced >= 0) return c->forced;
+  if (!c->forced_seq.empty()) {
+    const int64_t n = (int64_t)c->forced_seq.size();
+    return c->forced_seq[(size_t)((((step - c->forced_seq_t0) % n) + n) % n)];
+  }
+  return c->order[step % (int64_t)c->groups.size()];
 }
 void drop_reservations(hift_ctx* c) { for (int i = 0; i < c->n_slots; ++i) c->slot[i].step = -1; }
 // after the host has rewritten blobs (every stream idle): nothing on the device is current any more
@@ -667,7 +674,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   const hift_model_cfg& m = c->m;
   const int L = c->L, T = c->T, d = c->d, V = c->V, Vp = c->Vp, B = c->B, S = c->S;
   const int k = (int)c->groups.size();
-  const int g = c->forced >= 0 ? c->forced : c->order[c->t % k];
+  const int g = group_at(c, c->t);
   GroupRec& gr = c->groups[g];
   const int lo = gr.unit_lo, hi = gr.unit_hi;
   const double lr = lr_for_cycle(c->oc, c->t / k);
@@ -1303,10 +1310,7 @@ hift_status hift_step_host(hift_ctx* c, const int32_t* tok, const int32_t* lab, 
   return do_step(c, c->tok_dev, c->lab_dev, loss_host);
 }
 
-int32_t hift_active_group(const hift_ctx* c) {
-  if (c->forced >= 0) return c->forced;
-  return c->order[c->t % (int64_t)c->groups.size()];
-}
+int32_t hift_active_group(const hift_ctx* c) { return group_at(c, c->t); }
 int32_t hift_num_groups(const hift_ctx* c) { return (int32_t)c->groups.size(); }
 int64_t hift_step_count(const hift_ctx* c) { return c->t; }
 double hift_current_lr(const hift_ctx* c) { return lr_for_cycle(c->oc, c->t / (int64_t)c->groups.size()); }
@@ -1319,6 +1323,14 @@ hift_status hift_force_group(hift_ctx* c, int32_t g) {
   if (g < -1 || g >= (int)c->groups.size()) return HIFT_ERR_CFG;
   if (g != c->forced) drop_reservations(c);     // uploads made for the schedule's coming steps stay resident, unreserved
   c->forced = g;
+  return HIFT_OK;
+}
+hift_status hift_force_sequence(hift_ctx* c, const int32_t* groups, int32_t n) {
+  if (!c || n < 0 || (n > 0 && !groups)) return HIFT_ERR_CFG;
+  for (int i = 0; i < n; ++i) if (groups[i] < 0 || groups[i] >= (int)c->groups.size()) return HIFT_ERR_CFG;
+  drop_reservations(c);
+  c->forced_seq.assign(groups, groups + n);
+  c->forced_seq_t0 = c->t;
   return HIFT_OK;
 }
 size_t hift_peak_hbm_bytes(const hift_ctx* c) { return c->dev_bytes; }

@@ -371,19 +371,19 @@ def _same_bits(a, b):
 
 
 @pytest.mark.parametrize("prefetch", [0, 1, 2, 3])
-@pytest.mark.parametrize("case", ["one_group", "forced", "two_groups", "forced_then_schedule"])
+@pytest.mark.parametrize("case", ["one_group", "forced", "two_groups", "forced_then_schedule", "sequence"])
 def test_paging_when_a_group_trains_on_consecutive_steps(case, prefetch):
     """A group that is trained again before (or while) its write-back lands must be updated from its
     latest values: one group holding every unit (k = 1, the full-parameter identity of Eq. 2-3), a
-    forced group, fewer groups than state slots, and leaving a forced group with uploads of the
-    schedule's groups outstanding.  The paged run keeps the bits of the run with the state resident."""
+    forced group, fewer groups than state slots, leaving a forced group with uploads of the
+    schedule's groups outstanding, and a forced list of groups with repeats.  The paged run keeps the bits of the run with the state resident."""
     import torch
     from paper_2401_15207_b200 import HiFT
     cfg = mini(0, synth.DTYPE_BF16, tie_head=1)
     n = cfg.n_units
     gc = {"one_group": synth.GroupCfg(layers_per_group=n), "forced": synth.GroupCfg(1),
           "two_groups": synth.GroupCfg(layers_per_group=(n + 1) // 2),
-          "forced_then_schedule": synth.GroupCfg(1)}[case]
+          "forced_then_schedule": synth.GroupCfg(1), "sequence": synth.GroupCfg(1)}[case]
     p0 = synth.init_params(cfg, 3, perturb=0.05)
     ctxs = []
     for offload in (0, 1):
@@ -392,7 +392,12 @@ def test_paging_when_a_group_trains_on_consecutive_steps(case, prefetch):
         h.set_params(p0)
         ctxs.append(h)
     try:
+        if case == "sequence":
+            for h in ctxs:
+                h.force_sequence([2, 0, 2, 3, 3, 1])
         for t in range(7):
+            if case == "sequence":
+                assert ctxs[1].active_group() == [2, 0, 2, 3, 3, 1][t % 6]
             if case == "forced":
                 for h in ctxs:
                     h.force_group(2 if t < 4 else 1)
