@@ -356,7 +356,10 @@ hift_status hift_k_norm_bwd(int32_t dtype, int32_t kind, int64_t rows, int64_t c
  * and has no allocator of its own for this device.
  *   - cols must be <= HIFT_STATIC_SCRATCH_MAX_COLS, else HIFT_ERR_CAPACITY (nothing is launched).
  *   - The first call on each device looks up the device address of the array (with that
- *     device current).  Make that first call before starting any stream capture.
+ *     device current).  Make that first call before starting any stream capture.  The address is
+ *     kept for the life of the process: it does not survive a cudaDeviceReset of that device.
+ *   - dy, x, stats and gain must not be NULL when dx or dgain is requested (HIFT_ERR_INPUT;
+ *     hift_k_norm_bwd checks the same).
  *   - All calls on one GPU share the one array, which keeps whatever the previous call left.
  *     Every word a call reads it has written earlier in the same call, so stale contents
  *     are harmless and nothing needs clearing; but two calls that overlap on the GPU (different

@@ -12,6 +12,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <atomic>
 #include <string>
 #include <vector>
 
@@ -1732,6 +1733,7 @@ hift_status hift_k_norm_bwd(int32_t dtype, int32_t kind, int64_t rows, int64_t c
                             float* dx, float* dgain, float* dbias, float* partial, void* stream) {
   if (cols % 8 || kind < 0 || kind > 1 || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
   if (dgain && !partial) return HIFT_ERR_CFG;
+  if ((dx || dgain) && (!dy || !x || !stats || !gain)) return HIFT_ERR_INPUT;
   cudaStream_t st = (cudaStream_t)stream;
   if (dx) launch_norm_bwd_dx(st, dtype, kind, false, rows, (int)cols, dy, x, stats, gain, add, dx, nullptr);
   if (dgain) launch_colreduce(st, dtype == 1, kind == 0 ? 1 : 2, rows, (int)cols, dy, cols, x, stats, partial, dgain, dbias);
@@ -1756,7 +1758,7 @@ hift_status hift_k_cross_entropy(int32_t dtype, int64_t rows, int64_t vocab, int
 namespace {
 constexpr int kStaticMaxDevices = 64;
 static __device__ __align__(256) float g_static_partial[2 * kColChunks * HIFT_STATIC_SCRATCH_MAX_COLS];
-float* g_static_partial_addr[kStaticMaxDevices] = {nullptr};
+std::atomic<float*> g_static_partial_addr[kStaticMaxDevices];     // zero-initialised; one slot per device ordinal
 }  // namespace
 
 extern "C" hift_status hift_k_norm_bwd_static(int32_t dtype, int32_t kind, int64_t rows, int64_t cols,
@@ -1765,14 +1767,17 @@ extern "C" hift_status hift_k_norm_bwd_static(int32_t dtype, int32_t kind, int64
                                               float* dgain, float* dbias, void* stream) {
   if (cols % 8 || cols < 8 || rows < 1 || kind < 0 || kind > 1 || dtype < 0 || dtype > 1) return HIFT_ERR_CFG;
   if (cols > HIFT_STATIC_SCRATCH_MAX_COLS) return HIFT_ERR_CAPACITY;
+  if ((dx || dgain) && (!dy || !x || !stats || !gain)) return HIFT_ERR_INPUT;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return HIFT_ERR_CUDA;
-  float* partial = g_static_partial_addr[dev];
+  float* partial = g_static_partial_addr[dev].load(std::memory_order_relaxed);
   if (!partial) {
-    // first call on this device (which is current): resolve the array's device address
+    // first call on this device (which is current): resolve the array's device address.  Two host threads
+    // racing here both get the same answer from the runtime, so a relaxed store is enough.
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_partial) != cudaSuccess || !p) { cudaGetLastError(); return HIFT_ERR_CUDA; }
-    partial = g_static_partial_addr[dev] = (float*)p;
+    partial = (float*)p;
+    g_static_partial_addr[dev].store(partial, std::memory_order_relaxed);
   }
   cudaStream_t st = (cudaStream_t)stream;
   if (dx) launch_norm_bwd_dx(st, dtype, kind, false, rows, (int)cols, dy, x, stats, gain, add, dx, nullptr);

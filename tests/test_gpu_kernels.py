@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 import synth
-from gpu_util import rel_l2
+from gpu_util import U_BF16, U_F32, assert_elem, attention_slack, gemm_slack, rel_l2
 from oracle import hift_oracle as O
 
 pytestmark = pytest.mark.gpu
@@ -134,23 +134,30 @@ def test_linear_three_forms(dtype, M, N, K):
     res = rng.standard_normal((M, N)).astype(np.float32)
     td = torch.float32 if dtype == 0 else torch.bfloat16
     tol = 2e-6 if dtype == 0 else 6e-3
+    u_out = 2 * U_F32 if dtype == 0 else U_BF16
     cvt = (lambda a: a.astype(np.float64)) if dtype == 0 else _bf
+    X, W, DY, Bv = cvt(x), cvt(w), cvt(dy), cvt(bias)
     # forward with bias
     y = torch.empty((M, N), dtype=td, device="cuda")
     k_linear(0, dtype, M, N, K, _t(x, td), _t(w, td), y, bias=_t(bias, td))
-    assert rel_l2(y.float().cpu().numpy(), cvt(x) @ cvt(w).T + cvt(bias)) <= tol
+    ref, slack = X @ W.T + Bv, gemm_slack(X, W.T) + 2 * U_F32 * np.abs(Bv)
+    assert rel_l2(y.float().cpu().numpy(), ref) <= tol
+    assert_elem(y.float().cpu().numpy(), ref, u_out, slack, "forward")
     # forward into the fp32 residual stream
     y32 = torch.empty((M, N), dtype=torch.float32, device="cuda")
     k_linear(0, dtype, M, N, K, _t(x, td), _t(w, td), y32, bias=_t(bias, td), residual=_t(res))
-    assert rel_l2(y32.cpu().numpy(), cvt(x) @ cvt(w).T + cvt(bias) + res) <= 2e-6 if dtype == 0 else 2e-3
+    assert rel_l2(y32.cpu().numpy(), ref + res) <= 2e-6
+    assert_elem(y32.cpu().numpy(), ref + res, 2 * U_F32, slack + 2 * U_F32 * np.abs(res), "forward into the stream")
     # activation gradient
     dx = torch.empty((M, K), dtype=td, device="cuda")
     k_linear(1, dtype, M, N, K, _t(dy, td), _t(w, td), dx)
-    assert rel_l2(dx.float().cpu().numpy(), cvt(dy) @ cvt(w)) <= tol
+    assert rel_l2(dx.float().cpu().numpy(), DY @ W) <= tol
+    assert_elem(dx.float().cpu().numpy(), DY @ W, u_out, gemm_slack(DY, W), "dX")
     # weight gradient (fp32 out)
     dw = torch.empty((N, K), dtype=torch.float32, device="cuda")
     k_linear(2, dtype, M, N, K, _t(dy, td), _t(x, td), dw)
-    assert rel_l2(dw.cpu().numpy(), cvt(dy).T @ cvt(x)) <= 2e-6
+    assert rel_l2(dw.cpu().numpy(), DY.T @ X) <= 2e-6
+    assert_elem(dw.cpu().numpy(), DY.T @ X, 2 * U_F32, gemm_slack(DY.T, X), "dW")
 
 
 # ------------------------------------------------------------------ attention
@@ -174,6 +181,9 @@ def test_attention_forward_backward(dtype, dh, causal):
     k_attention_fwd(dtype, B, S, H, dh, causal, tq, o, lse)
     tol = 3e-6 if dtype == 0 else 6e-3
     assert rel_l2(o.float().cpu().numpy(), o_ref.reshape(B * S, d)) <= tol
+    u = 16 * U_F32 if dtype == 0 else U_BF16
+    sl = attention_slack(q, k, v, p, cvt(do).reshape(B, S, H, dh), u=u)
+    assert_elem(o.float().cpu().numpy(), o_ref.reshape(B * S, d), u, sl[0].reshape(B * S, d), "o")
     # log-sum-exp against its definition
     s = np.einsum("bshe,bthe->bhst", q, k) / np.sqrt(dh)
     if causal:
@@ -190,6 +200,7 @@ def test_attention_forward_backward(dtype, dh, causal):
     got = dqkv.float().cpu().numpy()
     for i in range(3):
         assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= tolb, i
+        assert_elem(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d], u, sl[1 + i].reshape(B * S, d), "dq dk dv"[3 * i:3 * i + 2])
 
 
 @pytest.mark.parametrize("dh", [64, 128])
@@ -212,6 +223,8 @@ def test_attention_tensor_core_edge_lengths(dh, B, S, H, causal):
     lse = torch.full((B, H, S), 9.0, dtype=torch.float32, device="cuda")
     k_attention_fwd(1, B, S, H, dh, causal, tq, o, lse)
     assert rel_l2(o.float().cpu().numpy(), o_ref.reshape(B * S, d)) <= 6e-3
+    sl = attention_slack(q, k, v, p, _bf(do).reshape(B, S, H, dh))
+    assert_elem(o.float().cpu().numpy(), o_ref.reshape(B * S, d), U_BF16, sl[0].reshape(B * S, d), "o")
     dqkv = torch.full((B * S, 3 * d), 9.0, dtype=torch.bfloat16, device="cuda")
     dsum = torch.empty(B * S * H, dtype=torch.float32, device="cuda")
     k_attention_bwd(1, B, S, H, dh, causal, tq, o, lse, _t(do, torch.bfloat16), dqkv, dsum)
@@ -224,6 +237,7 @@ def test_attention_tensor_core_edge_lengths(dh, B, S, H, causal):
             assert np.abs(got[:, i * d:(i + 1) * d]).max() <= 1e-3
         else:
             assert rel_l2(got[:, i * d:(i + 1) * d], r) <= 1.5e-2, i
+        assert_elem(got[:, i * d:(i + 1) * d], r, U_BF16, sl[1 + i].reshape(B * S, d) + 1e-12, "dq dk dv"[3 * i:3 * i + 2])
 
 
 @pytest.mark.parametrize("dtype,dh", [(0, 32), (1, 64), (1, 128)])
@@ -249,6 +263,9 @@ def test_attention_key_lengths(dtype, dh, causal):
     lse = torch.full((B, H, S), 9.0, dtype=torch.float32, device="cuda")
     k_attention_fwd(dtype, B, S, H, dh, causal, tq, o, lse, key_lens=tl)
     assert rel_l2(o.float().cpu().numpy(), o_ref.reshape(B * S, d)) <= (3e-6 if dtype == 0 else 6e-3)
+    u = 16 * U_F32 if dtype == 0 else U_BF16
+    sl = attention_slack(q, k, v, p, cvt(do).reshape(B, S, H, dh), u=u)
+    assert_elem(o.float().cpu().numpy(), o_ref.reshape(B * S, d), u, sl[0].reshape(B * S, d), "o")
     dqkv = torch.full((B * S, 3 * d), 9.0, dtype=td, device="cuda")
     dsum = torch.empty(B * S * H, dtype=torch.float32, device="cuda")
     k_attention_bwd(dtype, B, S, H, dh, causal, tq, o, lse, _t(do, td), dqkv, dsum, key_lens=tl)
@@ -258,6 +275,7 @@ def test_attention_key_lengths(dtype, dh, causal):
     tolb = 5e-6 if dtype == 0 else 1.5e-2
     for i in range(3):
         assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= tolb, i
+        assert_elem(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d], u, sl[1 + i].reshape(B * S, d), "dq dk dv"[3 * i:3 * i + 2])
     g4 = got.reshape(B, S, 3, d)
     for b, l in enumerate(lens):
         assert np.all(g4[b, l:, 1:] == 0.0), b                # dk, dv of padded keys: exact zeros
@@ -313,6 +331,15 @@ def test_linear_with_rope_in_the_epilogue(M, N, K, rope_cols, bias):
     got = out.float().cpu().numpy()
     assert rel_l2(got[:, :rope_cols], ref[:, :rope_cols]) <= 4e-3
     assert rel_l2(got[:, rope_cols:], ref[:, rope_cols:]) <= 4e-3 or rope_cols == N
+    # a rotated element mixes two accumulators with |cos|, |sin| <= 1 (fp32 tables: 2^-24 each)
+    acc = gemm_slack(_bf(x), _bf(w).T) + 4 * U_F32 * np.abs(y)
+    part = acc[:, :rope_cols].reshape(M, rope_cols // dh, 2, dh // 2)
+    mixed = (part + part[:, :, ::-1, :]).reshape(M, rope_cols)
+    ymix = np.abs(y[:, :rope_cols]).reshape(M, rope_cols // dh, 2, dh // 2)
+    mixed = mixed + 4 * U_F32 * (ymix + ymix[:, :, ::-1, :]).reshape(M, rope_cols)
+    assert_elem(got[:, :rope_cols], ref[:, :rope_cols], U_BF16, mixed, "rotated columns")
+    if rope_cols < N:
+        assert_elem(got[:, rope_cols:], ref[:, rope_cols:], U_BF16, acc[:, rope_cols:], "plain columns")
 
 
 @pytest.mark.parametrize("M,f,K,keep,bias", [(300, 384, 256, True, False), (256, 128, 192, False, True), (520, 1152, 128, True, True)])
@@ -331,8 +358,15 @@ def test_gate_up_projection_with_swiglu_in_the_epilogue(M, f, K, keep, bias):
     y = _bf(x) @ _bf(w).T + (_bf(b) if bias else 0.0)
     s_ref = O.swiglu_fwd(y[:, :f], y[:, f:])
     assert rel_l2(s.float().cpu().numpy(), s_ref) <= 4e-3
+    acc = gemm_slack(_bf(x), _bf(w).T) + (2 * U_F32 * np.abs(_bf(b)) if bias else 0.0)
+    # d(silu(g) u)/dg and /du from the oracle's own backward with a unit upstream gradient; the logistic function
+    # comes from the hardware exp2 and reciprocal (a few fp32 units, relative to the value)
+    dg1, du1 = O.swiglu_bwd(np.ones_like(s_ref), y[:, :f], y[:, f:])
+    assert_elem(s.float().cpu().numpy(), s_ref, U_BF16 + 8 * U_F32,
+                np.abs(dg1) * acc[:, :f] + np.abs(du1) * acc[:, f:], "silu(gate) * up")
     if keep:
         assert rel_l2(gu.float().cpu().numpy(), y) <= 4e-3
+        assert_elem(gu.float().cpu().numpy(), y, U_BF16, acc, "kept pre-activations")
 
 
 @pytest.mark.parametrize("M,N,f", [(300, 256, 416), (256, 128, 1024), (200, 192, 96)])
@@ -352,6 +386,11 @@ def test_down_projection_dx_with_swiglu_backward_in_the_epilogue(M, N, f):
     got = dgu.float().cpu().numpy()
     assert rel_l2(got[:, :f], dg_ref) <= 4e-3
     assert rel_l2(got[:, f:], du_ref) <= 4e-3
+    # both outputs are ds times a factor that depends on the saved pre-activations only
+    acc = gemm_slack(_bf(dy), _bf(w))
+    fg, fu = O.swiglu_bwd(np.ones_like(ds), _bf(gu)[:, :f], _bf(gu)[:, f:])
+    assert_elem(got[:, :f], dg_ref, U_BF16 + 16 * U_F32, np.abs(fg) * acc, "d gate")
+    assert_elem(got[:, f:], du_ref, U_BF16 + 16 * U_F32, np.abs(fu) * acc, "d up")
 
 
 @pytest.mark.parametrize("M,N,K,keep,bias", [(300, 416, 256, True, True), (256, 1024, 192, False, False)])
@@ -367,8 +406,13 @@ def test_up_projection_with_gelu_in_the_epilogue(M, N, K, keep, bias):
     k_linear_gelu(M, N, K, _t(x, torch.bfloat16), _t(w, torch.bfloat16), pre, act, _t(b, torch.bfloat16) if bias else None)
     y = _bf(x) @ _bf(w).T + (_bf(b) if bias else 0.0)
     assert rel_l2(act.float().cpu().numpy(), O.gelu_fwd(y)) <= 4e-3
+    acc = gemm_slack(_bf(x), _bf(w).T) + (2 * U_F32 * np.abs(_bf(b)) if bias else 0.0)
+    # the epilogue's normal CDF: 3e-7 absolute (times |y|), at most 0.4 % relative in the far tail
+    assert_elem(act.float().cpu().numpy(), O.gelu_fwd(y), U_BF16 + 4e-3,
+                np.abs(O.gelu_bwd(np.ones_like(y), y)) * acc + 3e-7 * np.abs(y), "gelu")
     if keep:
         assert rel_l2(pre.float().cpu().numpy(), y) <= 4e-3
+        assert_elem(pre.float().cpu().numpy(), y, U_BF16, acc, "kept pre-activation")
 
 
 @pytest.mark.parametrize("M,N,f", [(300, 256, 416), (200, 192, 96)])
@@ -383,6 +427,10 @@ def test_down_projection_dx_with_gelu_backward_in_the_epilogue(M, N, f):
     k_linear_dx_gelu_bwd(M, N, f, _t(dy, torch.bfloat16), _t(w, torch.bfloat16), _t(a, torch.bfloat16), da)
     ref = O.gelu_bwd(_bf(dy) @ _bf(w), _bf(a))
     assert rel_l2(da.float().cpu().numpy(), ref) <= 4e-3
+    du = _bf(dy) @ _bf(w)
+    fac = np.abs(O.gelu_bwd(np.ones_like(du), _bf(a)))
+    # gelu'(a) = Phi(a) + a phi(a): the approximated CDF (3e-7 absolute) plus the density through exp2
+    assert_elem(da.float().cpu().numpy(), ref, U_BF16 + 16 * U_F32, fac * gemm_slack(_bf(dy), _bf(w)) + 1e-6 * np.abs(du), "gelu backward")
 
 
 # ------------------------------------------------------------------ norms
@@ -411,6 +459,10 @@ def test_norm_forward_backward(dtype, kind, rows, cols):
     else:
         y_ref, cache = O.rmsnorm_fwd(x64, cvt(gain), eps)
     assert rel_l2(y.float().cpu().numpy(), y_ref) <= (2e-6 if dtype == 0 else 4e-3)
+    # statistics in fp32 over `cols` elements: a few units of the row's scale
+    xs = np.abs(x64).max(axis=1, keepdims=True) * np.asarray(cache[1]).reshape(-1, 1)
+    assert_elem(y.float().cpu().numpy(), y_ref, (U_BF16 if dtype else 0.0) + 8 * U_F32,
+                8 * U_F32 * (xs * np.abs(cvt(gain)) + (np.abs(cvt(bias)) if kind == 0 else 0.0)), "norm forward")
     dx = torch.empty((rows, cols), dtype=torch.float32, device="cuda")
     dgain = torch.empty(cols, dtype=torch.float32, device="cuda")
     dbias = torch.empty(cols, dtype=torch.float32, device="cuda")
@@ -424,6 +476,16 @@ def test_norm_forward_backward(dtype, kind, rows, cols):
         dx_ref, dg_ref = O.rmsnorm_bwd(cvt(dy), cache, cvt(gain))
     assert rel_l2(dx.cpu().numpy(), dx_ref + add) <= 3e-6
     assert rel_l2(dgain.cpu().numpy(), dg_ref) <= 5e-6
+    # every term of dx is rstd * (gain dy) times a factor of at most 1 + |xhat|^2: bound per row
+    gdy = np.abs(cvt(dy) * cvt(gain))
+    rstd = np.asarray(cache[1]).reshape(-1, 1)                 # both norms keep (xhat or x, 1 / sigma)
+    xhat = np.abs(cache[0]) if kind == 0 else np.abs(cache[0] * cache[1])
+    rowscale = rstd * (gdy + gdy.mean(axis=1, keepdims=True) * (1.0 + xhat) + (gdy * xhat).mean(axis=1, keepdims=True) * xhat)
+    assert_elem(dx.cpu().numpy(), dx_ref + add, 2 * U_F32, 32 * U_F32 * rowscale + 2 * U_F32 * np.abs(add), "norm dx")
+    colscale = (np.abs(cvt(dy)) * xhat).sum(axis=0)
+    assert_elem(dgain.cpu().numpy(), dg_ref, 2 * U_F32, 64 * U_F32 * colscale, "d gain")
+    if kind == 0:
+        assert_elem(dbias.cpu().numpy(), db_ref, 2 * U_F32, 64 * U_F32 * np.abs(cvt(dy)).sum(axis=0), "d bias")
 
 
 # ------------------------------------------------------------------ cross-entropy
@@ -449,6 +511,10 @@ def test_cross_entropy(dtype, rows, vocab, ld):
     assert o[1:3].view(np.int32).tolist() == [int((labels >= 0).sum()), 0]
     got = tl.float().cpu().numpy()
     assert rel_l2(got[:, :vocab], d_ref) <= (3e-6 if dtype == 0 else 4e-3)
+    # softmax in fp32: the exponent's argument (|logit| up to ~15) and the row sum carry a few units each
+    nv = max(int((labels >= 0).sum()), 1)
+    p_ref = np.abs(d_ref) + (np.abs(d_ref) > 0.5 / nv) * (1.0 / nv)      # the probability itself, also at the label
+    assert_elem(got[:, :vocab], d_ref, (U_BF16 if dtype else 0.0) + 4 * U_F32, 64 * U_F32 * p_ref, "d logits")
     assert not got[:, vocab:].any()                          # padding columns carry no gradient
     if rows > 8:
         assert not got[3].any()
@@ -481,22 +547,27 @@ def test_linear_tensor_core_three_forms(M, N, K):
     y = torch.zeros((M, N), dtype=bf, device="cuda")
     k_linear(0, 1, M, N, K, tx, tw, y, bias=tb, path=2)
     ref = _bf(x) @ _bf(w).T + _bf(bias)
+    slack = gemm_slack(_bf(x), _bf(w).T) + 2 * U_F32 * np.abs(_bf(bias))
     assert rel_l2(y.float().cpu().numpy(), ref) <= 6e-3
+    assert_elem(y.float().cpu().numpy(), ref, U_BF16, slack, "forward")
     # forward into the fp32 residual stream
     res = rng.standard_normal((M, N)).astype(np.float32)
     y32 = torch.zeros((M, N), dtype=torch.float32, device="cuda")
     k_linear(0, 1, M, N, K, tx, tw, y32, bias=tb, residual=_t(res), path=2)
     assert rel_l2(y32.cpu().numpy(), ref + res) <= 1e-5
+    assert_elem(y32.cpu().numpy(), ref + res, 2 * U_F32, slack + 2 * U_F32 * np.abs(res), "forward into the stream")
     # activation gradient: dx[M,K] = dy[M,N] w[N,K]   (B operand N-major)
     if K >= 64 and N >= 64:
         dx = torch.zeros((M, K), dtype=torch.float32, device="cuda")
         k_linear(1, 1, M, N, K, tdy, tw, dx, residual=torch.zeros((M, K), dtype=torch.float32, device="cuda"), path=2)
         assert rel_l2(dx.cpu().numpy(), _bf(dy) @ _bf(w)) <= 1e-5
+        assert_elem(dx.cpu().numpy(), _bf(dy) @ _bf(w), 2 * U_F32, gemm_slack(_bf(dy), _bf(w)), "dX")
     # weight gradient: dw[N,K] = dy^T x   (both operands MN-major); needs N >= 128 rows of output
     if N >= 128:
         dw = torch.zeros((N, K), dtype=torch.float32, device="cuda")
         k_linear(2, 1, M, N, K, tdy, tx, dw, path=2)
         assert rel_l2(dw.cpu().numpy(), _bf(dy).T @ _bf(x)) <= 1e-5
+        assert_elem(dw.cpu().numpy(), _bf(dy).T @ _bf(x), 2 * U_F32, gemm_slack(_bf(dy).T, _bf(x)), "dW")
 
 
 def test_tensor_core_path_refuses_ineligible_shapes():
