@@ -114,7 +114,13 @@ typedef struct {
 /* Build a context.  `cuda_stream` is a cudaStream_t (NULL = default stream).
  * Parameters start as zeros; fill them with hift_set_param() or
  * hift_init_synthetic().  Fails with HIFT_ERR_OOM_* and leaves *out NULL if the
- * device or pinned memory cannot be had. */
+ * device or pinned memory cannot be had (everything allocated so far is released).
+ * One process drives one GPU: the tensor-core kernels' time-out flag, the SM count and the
+ * driver entry point for tensor maps are looked up once per process, for the device that
+ * was current at the first call; contexts on two different GPUs in one process are not
+ * supported (several contexts on the same GPU are).
+ * batch * seq <= 8192: the embedding-gradient kernel keeps the step's token positions in
+ * shared memory (HIFT_ERR_CFG beyond it). */
 hift_status hift_create(const hift_model_cfg *model, const hift_group_cfg *groups,
                         const hift_opt_cfg *opt, void *cuda_stream, hift_ctx **out);
 void hift_destroy(hift_ctx *ctx);
@@ -246,6 +252,23 @@ hift_status hift_last_step_timeline(hift_ctx *ctx, double *ms6);
  * value lets a test walk the time-out path without stalling anything).  Returns the flag, or -1
  * if the tensor-core path is unavailable.  Synchronises the device. */
 int32_t hift_tc_error_flag(int32_t set_value);
+
+/* Code-path switches for tests and A/B timing; every one defaults to 1, the fast path.  which = 0: CTA-pair
+ * tiles in the tensor-core GEMM (0 = one CTA per tile); 1: programmatic dependent launch (0 = plain stream
+ * order); 2: tcgen05 attention forward, 3: tcgen05 attention backward (0 = the warp-level mma.sync kernels).
+ * value >= 0 sets the switch, value < 0 only reads it; returns the previous value, or -1 for an unknown
+ * switch.  Process-wide, consulted at every launch, not thread-safe.  Results do not depend on switches 0
+ * and 1 (same bits); 2 and 3 select kernels with a different summation order.
+ * Two more, for fault-path tests that need no faulting GPU: which = 4: the value-th pinned host allocation
+ * from now on (0 = the next one) fails as if the host were out of pinned memory, once (value -1 = off),
+ * so that hift_create's HIFT_ERR_OOM_PINNED path and its clean-up run; which = 5: contexts created while it
+ * is 1 run in checked mode: every slice of the activation arena is followed by a 256-byte guard region that
+ * each step paints before its first kernel, and hift_check_arena() counts the regions a step wrote into. */
+int32_t hift_test_switch(int32_t which, int32_t value);
+/* Checked mode only (-1 otherwise): guard regions of the last step's arena plan that no longer hold their
+ * pattern (0 = no kernel wrote past the end of its buffer), and how many regions there are. */
+int64_t hift_check_arena(hift_ctx *ctx);
+int64_t hift_arena_guard_count(const hift_ctx *ctx);
 
 /* ---- the group-local fused optimizer on caller-owned flat buffers --------
  * One streaming pass over n elements (the update Algorithm 1 applies to the

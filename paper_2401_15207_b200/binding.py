@@ -96,6 +96,9 @@ def _prototypes():
         "hift_last_step_paging": (C.c_int, [vp, C.POINTER(sz), C.POINTER(sz)]),
         "hift_last_step_timeline": (C.c_int, [vp, C.POINTER(f64)]),
         "hift_tc_error_flag": (i32, [i32]),
+        "hift_test_switch": (i32, [i32, i32]),
+        "hift_check_arena": (i64, [vp]),
+        "hift_arena_guard_count": (i64, [vp]),
         "hift_opt_step": (C.c_int, [i32, sz, vp, vp, vp, vp, vp, f64, f64, f64, f64, f64, f64, i64, vp]),
         "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
@@ -337,6 +340,13 @@ class HiFT:
             out[name] = {"launches": n.value, "ms": ms.value, "work": w.value}
         return out
 
+    def check_arena(self) -> int:
+        """Checked mode: number of arena guard regions the last step overwrote (-1: not in checked mode)."""
+        return lib().hift_check_arena(self._h)
+
+    def arena_guard_count(self) -> int:
+        return lib().hift_arena_guard_count(self._h)
+
     def last_step_launches(self) -> int:
         return lib().hift_last_step_launches(self._h)
 
@@ -371,6 +381,14 @@ def adafactor_step(rows, cols, param_bf16, master, grad, state, scratch, lr, eps
 
 def tc_error_flag(set_value: int = -1) -> int:
     return lib().hift_tc_error_flag(set_value)
+
+
+SWITCH_GEMM_PAIR, SWITCH_PDL, SWITCH_ATTN_FWD_TC, SWITCH_ATTN_BWD_TC, SWITCH_FAIL_PINNED, SWITCH_CHECKED_ARENA = 0, 1, 2, 3, 4, 5
+
+
+def code_path_switch(which: int, value: int = -1) -> int:
+    """Sets (value >= 0) or reads a code-path switch of the library; returns the previous value."""
+    return lib().hift_test_switch(which, value)
 
 
 def k_linear(form, dtype, M, N, K, a, b, out, bias=None, residual=None, path=0, stream=None):

@@ -60,11 +60,8 @@ __device__ __forceinline__ float warp_max(float v) {
 // its writes are visible).  pdl_launch_next() lets the successor be scheduled early in turn.
 __device__ __forceinline__ void pdl_wait_prior() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_next() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-inline int pdl_enabled() {
-  static int v = -1;
-  if (v < 0) { const char* e = getenv("HIFT_PDL"); v = e ? atoi(e) : 1; }
-  return v;
-}
+int pdl_switch_value();      // 1 unless switched off through gemm_tc_switch (defined beside the other switches)
+inline int pdl_enabled() { return pdl_switch_value(); }
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
   cudaLaunchConfig_t cfg;

@@ -624,7 +624,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const int BN = tc.bn, S = tc.stages;
   const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
-  if (g_tc_error != 0) return;                       // an earlier launch timed out: do nothing
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned tiles
   const uint32_t bar_base = base + S * kStageBytes;
@@ -654,10 +653,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const uint32_t tmem_base = *tmem_slot_gen;
   pdl_trigger();
   pdl_wait();                                        // barriers and tensor memory were set up under the predecessor's tail
+  // An earlier launch timed out: do nothing but release the tensor memory.  The flag is global memory, so
+  // it is read after the wait above; every role takes its own reading, and if two of them ever disagreed
+  // the bounded waits below would end the launch the same way.
+  const bool poisoned = *(volatile int*)&g_tc_error != 0;
 
   if (warp == 0) {
     // ---------------- TMA producer (one thread)
-    if (lane == 0) {
+    if (lane == 0 && !poisoned) {
       int s = 0;
       uint32_t ph = 0;                   // ring position and its phase, advanced without divisions
       bool ok = true;
@@ -690,7 +693,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer (one thread)
-    if (lane == 0) {
+    if (lane == 0 && !poisoned) {
       // instruction descriptor: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
       // A / B major-ness (bits 15, 16: 1 = MN-major), N/8 at bits 17-22, M/16 at bits 24-28
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
@@ -729,7 +732,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int q = warp & 3;
     uint8_t* stage = smem_gen + S * kStageBytes + 256 + (warp - 2) * kStoreStage;   // behind the barriers
     int lt = 0;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++lt) {
+    for (int tile = blockIdx.x; tile < num_tiles && !poisoned; tile += gridDim.x, ++lt) {
       const int ab = lt & 1;
       const uint32_t aph = (lt >> 1) & 1;
       const bool ready = mbar_wait(acc_full(ab), aph);
@@ -958,7 +961,7 @@ EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 148;
 int g_init_state = -1;    // -1 not tried, 0 ok, 1 failed
 std::mutex g_mu;
-int g_pdl = 1;            // programmatic dependent launch of the GEMM kernels (HIFT_PDL=0: plain stream order)
+int g_pdl = 1;            // programmatic dependent launch of the GEMM kernels (switch 1 of gemm_tc_switch; 0: plain stream order)
 
 struct MapKey {
   const void* p; uint64_t inner, outer, stride; uint32_t box_outer;
@@ -1066,16 +1069,25 @@ template <bool A_MN, bool B_MN, bool OUT_F32>
 cudaError_t set_smem_attr2() {
   return cudaFuncSetAttribute(gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
-int g_attn_tc = 1;       // tcgen05 attention forward (HIFT_ATTN_TC=0 falls back to the mma.sync kernel)
-int g_attn_bwd_tc = 1;   // tcgen05 attention backward (HIFT_ATTN_BWD_TC=0 falls back to the mma.sync kernels)
+int g_attn_tc = 1;       // tcgen05 attention forward (switch 2; 0 falls back to the mma.sync kernel)
+int g_attn_bwd_tc = 1;   // tcgen05 attention backward (switch 3; 0 falls back to the mma.sync kernels)
 template <int DH, int MODE>
 cudaError_t set_smem_attr_ab() {
   return cudaFuncSetAttribute(attn_bwd_tc_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               AttnBwdCfg<DH, MODE>::kSmem);
 }
-int g_pair_mode = 1;     // CTA-pair kernel for 256-wide tiles (HIFT_GEMM_PAIR=0 falls back to one CTA per tile)
+int g_pair_mode = 1;     // CTA-pair kernel for 256-wide tiles (switch 0; 0 falls back to one CTA per tile)
 
 }  // namespace
+
+int gemm_tc_switch(int which, int value) {
+  int* sw[4] = {&g_pair_mode, &g_pdl, &g_attn_tc, &g_attn_bwd_tc};
+  if (which < 0 || which > 3) return -1;
+  const int old = *sw[which];
+  if (value >= 0) *sw[which] = value;
+  return old;
+}
+int pdl_switch_value() { return g_pdl; }
 
 int gemm_tc_init() {
   std::lock_guard<std::mutex> lk(g_mu);
@@ -1104,16 +1116,12 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr2<false, true, false>();
   if (e == cudaSuccess) e = set_smem_attr2<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr2<true, true, true>();
-  if (const char* pm = getenv("HIFT_GEMM_PAIR")) g_pair_mode = atoi(pm);
-  if (const char* pd = getenv("HIFT_PDL")) g_pdl = atoi(pd);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
-  if (const char* am = getenv("HIFT_ATTN_TC")) g_attn_tc = atoi(am);
   if (e == cudaSuccess) e = set_smem_attr_ab<64, 0>();
   if (e == cudaSuccess) e = set_smem_attr_ab<64, 1>();
   if (e == cudaSuccess) e = set_smem_attr_ab<128, 0>();
   if (e == cudaSuccess) e = set_smem_attr_ab<128, 1>();
-  if (const char* am = getenv("HIFT_ATTN_BWD_TC")) g_attn_bwd_tc = atoi(am);
   if (e != cudaSuccess) { cudaGetLastError(); return g_init_state; }
   g_init_state = 0;
   return 0;
@@ -1219,7 +1227,7 @@ const int* gemm_tc_error_device_ptr() {
 }
 
 bool attn_tc_eligible(int dh, const void* qkv, int H) {
-  // head sizes 64 and 128 (HIFT_ATTN_TC=0 sends both to the warp-level kernel)
+  // head sizes 64 and 128 (switch 2 off sends both to the warp-level kernel)
   return g_init_state == 0 && g_attn_tc && (dh == 128 || dh == 64) && (((uintptr_t)qkv) & 15) == 0 && ((3 * H * dh) % 8) == 0;
 }
 cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse,

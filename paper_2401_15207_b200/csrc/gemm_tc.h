@@ -24,6 +24,11 @@ cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int
 bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, const void* dqkv);
 cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,
                                const float* lse, const float* dsum, void* dqkv, const int* lens);
+// Code-path switches for A/B timing and for tests (all 1 by default = the fast path): which = 0 CTA-pair
+// GEMM tiles, 1 programmatic dependent launch, 2 tcgen05 attention forward, 3 tcgen05 attention backward.
+// value >= 0 sets the switch; returns its previous value (-1: no such switch).  Process-wide; read at
+// each launch.
+int gemm_tc_switch(int which, int value);
 // 0 if no tensor-core kernel has given up on a bounded wait since the library was loaded, else the
 // code of the first one (1 producer, 2 MMA issuer, 3 epilogue); -1 if the flag cannot be read.
 int gemm_tc_poll_error();

@@ -25,6 +25,10 @@ using namespace hift;
 namespace {
 
 constexpr size_t kAlignElems = 128;   // every tensor starts on a multiple of 128 elements
+constexpr size_t kGuardBytes = 256;   // checked mode: guard region behind every arena slice
+constexpr unsigned char kGuardByte = 0xC5;
+int g_checked_arena = 0;              // hift_test_switch 5: contexts created while set carry guard regions
+int g_fail_pinned_in = -1;            // hift_test_switch 4: the n-th pinned allocation from now fails (-1: off)
 constexpr int kScalWords = 8;         // the step's scalar words: loss, valid count, bad input, (time-out flag), gate
 
 // Per-block activation slots.  Residual-stream tensors are fp32 in every configuration;
@@ -114,6 +118,10 @@ struct hift_ctx {
   int* gate = nullptr;              // device word: non-zero = the step failed, the optimizer must not write
   float* grad = nullptr;            // [max_group]
   char* arena = nullptr; size_t arena_cap = 0, arena_off = 0, arena_fixed = 0;
+  bool checked = false;             // guard regions behind every arena slice, verified by hift_check_arena
+  bool record_guards = false;
+  std::vector<size_t> guards;       // offsets of the guard regions of the current plan
+  size_t n_fixed_guards = 0;        // the first of them belong to the fixed work buffers
   cudaEvent_t ev_fwd;
   cudaEvent_t tl[7];                // timeline of the last step: start, (unused x2), optimizer wait begin/end, d2h begin/end
   bool tl_valid = false;
@@ -302,7 +310,16 @@ hift_status dev_alloc(hift_ctx* c, void** p, size_t bytes) {
 char* arena_take(hift_ctx* c, size_t bytes) {
   const size_t o = c->arena_off;
   c->arena_off = align_up(o + bytes, 256);
+  if (c->checked) {
+    if (c->record_guards) c->guards.push_back(c->arena_off);
+    c->arena_off += kGuardBytes;
+  }
   return c->arena ? c->arena + o : (char*)(uintptr_t)o;
+}
+// pinned host memory through one door, so that a test can make the n-th request fail
+cudaError_t pinned_alloc(void** p, size_t bytes, unsigned flags) {
+  if (g_fail_pinned_in >= 0 && g_fail_pinned_in-- == 0) { *p = nullptr; return cudaErrorMemoryAllocation; }
+  return cudaHostAlloc(p, bytes, flags);
 }
 
 // Lowest level at which a slot must outlive the forward pass: 1 = activation gradients need
@@ -347,6 +364,7 @@ int level_of_block(const hift_ctx* c, int g, int i) {
 // bytes used.  With assign == false only sizes are computed.
 size_t plan_slots(hift_ctx* c, int g, bool assign) {
   c->arena_off = c->arena_fixed;
+  if (c->checked && assign) { c->guards.resize(c->n_fixed_guards); c->record_guards = true; }
   for (int i = 0; i < c->L; ++i) {
     const int lvl = level_of_block(c, g, i);
     for (int s = 0; s < S_NUM; ++s) {
@@ -363,6 +381,7 @@ size_t plan_slots(hift_ctx* c, int g, bool assign) {
       }
     }
   }
+  c->record_guards = false;
   return c->arena_off;
 }
 
@@ -687,6 +706,8 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
 
   plan_slots(c, g, true);
   if (c->arena_off > c->arena_cap) return HIFT_ERR_CFG;
+  if (c->checked)      // the plan moves with the group: paint this step's guard regions before anything runs
+    for (size_t o : c->guards) c->note(cudaMemsetAsync(c->arena + o, kGuardByte, kGuardBytes, c->st));
   // inputs produced on the caller's stream are visible to the step
   c->note(cudaEventRecord(c->ev_in, c->caller));
   c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
@@ -1072,6 +1093,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
   c->compact = c->mixed && c->offload && !c->af;
   c->recompute = oc->recompute != 0;
+  c->checked = g_checked_arena != 0;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_work, 0, sizeof(c->prof_work));
@@ -1131,7 +1153,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     }
     for (auto& g : c->groups) {
       g.blob_bytes = blob_bytes_of(g);
-      if (cudaHostAlloc((void**)&g.blob, g.blob_bytes, cudaHostAllocDefault) != cudaSuccess) {
+      if (pinned_alloc((void**)&g.blob, g.blob_bytes, cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         g.blob = nullptr;
         return fail(HIFT_ERR_OOM_PINNED);
@@ -1163,7 +1185,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     if ((rc = dev_alloc(c, (void**)&c->af_scratch, mx * sizeof(float))) != HIFT_OK) return fail(rc);
   }
   // four scalars the step publishes, then a staging row for the key-length table
-  if (cudaHostAlloc((void**)&c->scal_host, (kScalWords + (size_t)c->B) * sizeof(float), cudaHostAllocMapped) != cudaSuccess) return fail(HIFT_ERR_OOM_PINNED);
+  if (pinned_alloc((void**)&c->scal_host, (kScalWords + (size_t)c->B) * sizeof(float), cudaHostAllocMapped) != cudaSuccess) { cudaGetLastError(); c->scal_host = nullptr; return fail(HIFT_ERR_OOM_PINNED); }
   if (cudaHostGetDevicePointer((void**)&c->scal_host_dev, c->scal_host, 0) != cudaSuccess) return fail(HIFT_ERR_CUDA);
 
   // ---- activation arena: fixed work buffers, one scratch copy of every slot, then the
@@ -1172,6 +1194,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   c->slots.assign(c->L + 1, std::vector<char*>(S_NUM, nullptr));
   for (int pass = 0; pass < 2; ++pass) {
     c->arena_off = 0;
+    c->guards.clear();
+    c->record_guards = c->checked && pass == 1;
     c->tok_dev = (int32_t*)arena_take(c, T * sizeof(int32_t));
     c->lab_dev = (int32_t*)arena_take(c, T * sizeof(int32_t));
     c->lens_dev = (int32_t*)arena_take(c, (size_t)c->B * sizeof(int32_t));
@@ -1204,6 +1228,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
       c->slots[c->L][s] = (slot_min_level(m->arch, s) == 99 || s == S_XIN || s == S_XINA)
                               ? nullptr : arena_take(c, slot_bytes(c, s));
     c->arena_fixed = c->arena_off;
+    c->record_guards = false;
+    c->n_fixed_guards = c->guards.size();
     if (pass == 0) {
       size_t worst = c->arena_fixed;
       for (size_t g = 0; g < c->groups.size(); ++g) worst = std::max(worst, plan_slots(c, (int)g, false));
@@ -1621,6 +1647,25 @@ hift_status hift_last_step_timeline(hift_ctx* c, double* ms6) {
   }
   return HIFT_OK;
 }
+
+int32_t hift_test_switch(int32_t which, int32_t value) {
+  if (which == 4) { const int old = g_fail_pinned_in; g_fail_pinned_in = value; return old; }
+  if (which == 5) { const int old = g_checked_arena; if (value >= 0) g_checked_arena = value; return old; }
+  return gemm_tc_switch(which, value);
+}
+
+int64_t hift_check_arena(hift_ctx* c) {
+  if (!c || !c->checked) return -1;
+  sync_all(c);
+  std::vector<unsigned char> buf(kGuardBytes);
+  int64_t bad = 0;
+  for (size_t o : c->guards) {
+    if (cudaMemcpy(buf.data(), c->arena + o, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    for (unsigned char b : buf) if (b != kGuardByte) { ++bad; break; }
+  }
+  return bad;
+}
+int64_t hift_arena_guard_count(const hift_ctx* c) { return c && c->checked ? (int64_t)c->guards.size() : -1; }
 
 int32_t hift_tc_error_flag(int32_t set_value) {
   if (gemm_tc_init() != 0) return -1;

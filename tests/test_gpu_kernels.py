@@ -287,18 +287,17 @@ def test_attention_key_lengths(dtype, dh, causal):
     assert torch.equal(o, o2) and torch.equal(lse, lse2)
 
 
-def test_attention_key_lengths_on_the_warp_level_kernels():
-    """The same cases with the tcgen05 attention switched off (the switch is read when the library loads)."""
-    import os
-    import subprocess
-    import sys
-    env = dict(os.environ, HIFT_ATTN_TC="0", HIFT_ATTN_BWD_TC="0")
-    here = os.path.abspath(__file__)
-    r = subprocess.run([sys.executable, "-m", "pytest", here, "-q", "-x", "-m", "gpu", "-k",
-                        "test_attention_key_lengths and not warp_level", "-p", "no:cacheprovider"],
-                       env=env, capture_output=True, text=True, cwd=os.path.dirname(os.path.dirname(here)))
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
-    assert "6 passed" in r.stdout, r.stdout[-500:]
+@pytest.mark.parametrize("dh", [64, 128])
+@pytest.mark.parametrize("causal", [0, 1])
+def test_attention_key_lengths_on_the_warp_level_kernels(dh, causal):
+    """The same cases with the tcgen05 attention switched off: the mma.sync kernels behind it."""
+    from paper_2401_15207_b200 import code_path_switch
+    old = code_path_switch(2, 0), code_path_switch(3, 0)
+    try:
+        test_attention_key_lengths(1, dh, causal)
+    finally:
+        code_path_switch(2, old[0])
+        code_path_switch(3, old[1])
 
 
 # ------------------------------------------------------------------ rotary embedding fused into the qkv projection

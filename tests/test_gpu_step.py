@@ -508,48 +508,40 @@ def test_warmup_then_decay_moves_once_per_cycle():
     assert lrs == pytest.approx([0.0] * k + [0.5e-2] * k + [1e-2] * k + [0.5e-2] * k, rel=1e-15, abs=0.0)
 
 
-_PDL_SCRIPT = r"""
-import sys, hashlib, numpy as np, torch
-sys.path.insert(0, sys.argv[1])
-import synth
-from paper_2401_15207_b200 import HiFT
-arch = int(sys.argv[2])
-cfg = synth.ModelCfg(arch=arch, n_blocks=3, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=768 if arch == 2 else 1024, vocab=1000,
-                     max_pos=128, causal=1, tie_head=0, norm_eps=1e-6 if arch == 2 else 1e-5, dtype=synth.DTYPE_BF16,
-                     batch=2, seq=128, init_std=0.05)
-oc = synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
-h = HiFT(cfg, synth.GroupCfg(1), oc)
-h.set_params(synth.init_params(cfg, 4, perturb=0.05))
-losses = []
-for t in range(2 * h.num_groups()):
-    tok, lab = synth.batch_for(cfg, 21, t, "zipf")
-    losses.append(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
-m = hashlib.sha256()
-for n in h.tensor_names():
-    m.update(np.ascontiguousarray(h.get_param(n)).tobytes())
-print("RESULT", m.hexdigest(), " ".join(repr(x) for x in losses))
-"""
-
-
+@pytest.mark.parametrize("switch", [0, 1])
 @pytest.mark.parametrize("arch", [0, 2])
-def test_dependent_launch_changes_no_bits(arch, tmp_path):
-    """Programmatic dependent launch lets a kernel start under its predecessor's tail; it must wait before it
-    touches memory.  Two fresh processes, one with it (the default) and one in plain stream order, run the same
-    two cycles on a model large enough for the tensor-core kernels: every loss and every parameter bit agree."""
-    import os
-    import subprocess
-    import sys
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    script = tmp_path / "pdl_run.py"
-    script.write_text(_PDL_SCRIPT)
+def test_dependent_launch_and_cta_pairs_change_no_bits(arch, switch):
+    """Programmatic dependent launch lets a kernel start under its predecessor's tail (it must wait before it
+    touches memory), and CTA-pair tiles split one output tile over two SMs: neither may change a bit.  The same
+    two cycles with the switch on (the default) and off, on a model large enough for the tensor-core kernels:
+    every loss and every parameter bit agree."""
+    import hashlib
+    import torch
+    from paper_2401_15207_b200 import HiFT, code_path_switch
+    cfg = synth.ModelCfg(arch=arch, n_blocks=3, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=768 if arch == 2 else 1024,
+                         vocab=1000, max_pos=128, causal=1, tie_head=0, norm_eps=1e-6 if arch == 2 else 1e-5,
+                         dtype=synth.DTYPE_BF16, batch=2, seq=128, init_std=0.05)
+    oc = synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
     outs = []
-    for pdl in ("1", "0"):
-        env = dict(os.environ, HIFT_PDL=pdl)
-        r = subprocess.run([sys.executable, str(script), root, str(arch)], capture_output=True, text=True, env=env, timeout=600)
-        assert r.returncode == 0, r.stderr[-2000:]
-        line = [l for l in r.stdout.splitlines() if l.startswith("RESULT")]
-        assert line, r.stdout[-500:]
-        outs.append(line[0])
+    old = code_path_switch(switch, -1)
+    try:
+        for value in (1, 0):
+            code_path_switch(switch, value)
+            h = HiFT(cfg, synth.GroupCfg(1), oc)
+            try:
+                h.set_params(synth.init_params(cfg, 4, perturb=0.05))
+                losses = []
+                for t in range(2 * h.num_groups()):
+                    tok, lab = synth.batch_for(cfg, 21, t, "zipf")
+                    losses.append(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
+                m = hashlib.sha256()
+                for n in h.tensor_names():
+                    m.update(np.ascontiguousarray(h.get_param(n)).tobytes())
+                outs.append((m.hexdigest(), losses))
+            finally:
+                h.close()
+    finally:
+        code_path_switch(switch, old)
     assert outs[0] == outs[1]
 
 
@@ -603,3 +595,73 @@ def test_host_batches_from_pinned_and_pageable_memory_agree():
     finally:
         a.close()
         b.close()
+
+
+def test_pinned_allocation_failure_is_reported_and_leaves_nothing_behind():
+    """hift_create when the host runs out of pinned memory, without exhausting anything: the library's test
+    switch makes the n-th pinned allocation fail.  Whichever one it is (the first group's blob, a later one, the
+    mapped scalar words after all blobs), the call reports HIFT_ERR_OOM_PINNED, releases what it had allocated
+    (device memory returns to its level), and the next hift_create succeeds."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError, code_path_switch
+    cfg = mini(0, synth.DTYPE_BF16)
+    gc, oc = synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=2)
+    warm = HiFT(cfg, gc, oc)                                  # loads the kernels, so that later memory readings are steady
+    k = warm.num_groups()
+    warm.close()
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for n in (0, 2, k):                                       # blobs are allocated first, one per group, then the scalar words
+        try:
+            code_path_switch(4, n)
+            with pytest.raises(HiftError) as e:
+                HiFT(cfg, gc, oc)
+            assert e.value.status == 3 and "pinned" in str(e.value)
+            assert code_path_switch(4, -1) == -1              # the injected failure was consumed
+        finally:
+            code_path_switch(4, -1)
+        torch.cuda.synchronize()
+        assert abs(torch.cuda.mem_get_info()[0] - free0) <= (4 << 20)
+    h = HiFT(cfg, gc, oc)
+    # what the context says it holds is what the driver handed out (allocation granularity aside)
+    used = free0 - torch.cuda.mem_get_info()[0]
+    assert h.peak_hbm_bytes() <= used <= h.peak_hbm_bytes() + (64 << 20)
+    h.set_params(synth.init_params(cfg, 1))
+    tok, lab = synth.batch_for(cfg, 2, 0, "zipf")
+    assert np.isfinite(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
+    h.close()
+
+
+@pytest.mark.parametrize("arch,dtype,big", [(0, synth.DTYPE_FP32, False), (1, synth.DTYPE_BF16, False), (2, synth.DTYPE_BF16, False),
+                                            (0, synth.DTYPE_BF16, True), (1, synth.DTYPE_BF16, True), (2, synth.DTYPE_BF16, True)])
+def test_checked_mode_no_kernel_writes_past_its_buffer(arch, dtype, big):
+    """Checked mode puts a painted guard region behind every slice of the activation arena (work buffers,
+    scratch slots, kept activations) and looks at them after the step: with ragged sizes on the CUDA-core
+    kernels and with tile-sized ones on the tensor-core kernels, over a full cycle (every retention plan),
+    not one region is touched.  Stands in for a memory checker on the arena, which holds every buffer the
+    step's kernels write except parameters, gradients and state."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, code_path_switch
+    if big:
+        cfg = synth.ModelCfg(arch=arch, n_blocks=2, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=640, vocab=1001,
+                             max_pos=160, n_classes=2 if arch == 1 else 0, causal=0 if arch == 1 else 1,
+                             norm_eps=1e-6 if arch == 2 else 1e-5, dtype=dtype, batch=2, seq=160, init_std=0.05)
+    else:
+        cfg = mini(arch, dtype)
+    old = code_path_switch(5, 1)
+    try:
+        h = HiFT(cfg, synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1, recompute=1 if big else 0))
+    finally:
+        code_path_switch(5, old)
+    try:
+        assert h.arena_guard_count() > 20
+        h.set_params(synth.init_params(cfg, 2))
+        for t in range(h.num_groups()):
+            tok, lab = synth.batch_for(cfg, 4, t, "zipf")
+            h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
+            assert h.check_arena() == 0, (t, h.check_arena())
+    finally:
+        h.close()
+    plain = HiFT(cfg, synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3))
+    assert plain.check_arena() == -1 and plain.arena_guard_count() == -1
+    plain.close()
