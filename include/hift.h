@@ -285,8 +285,10 @@ hift_status hift_opt_step(int32_t kind, size_t n, void *param_bf16_dev, float *m
                           double weight_decay, double momentum, int64_t tau,
                           void *cuda_stream);
 
-/* Adafactor (one of the optimizers the paper profiles; its formulas are Shazeer & Stern 2018,
- * Algorithms 4-5) on one caller-owned tensor [rows, cols] (rows = 1: a vector, unfactored).
+/* Adafactor (one of the optimizers the paper profiles, without formulas; built in the form
+ * torch.optim.Adafactor uses for Shazeer & Stern 2018, Algorithms 4-5: epsilon_1 is a lower clamp on the
+ * factored second-moment estimate and on the root of it, not a term added to the squared gradient)
+ * on one caller-owned tensor [rows, cols] (rows = 1: a vector, unfactored).
  * master/grad: fp32 [rows*cols]; state: fp32, R[rows] | C[cols] for a matrix, V[cols] for a
  * vector; scratch: fp32, 2*rows + 64*cols + 8 floats; param_bf16 may be NULL.  tau >= 1 as in
  * hift_opt_step.  Launches several small kernels on `cuda_stream`; does not synchronise. */

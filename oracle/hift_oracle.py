@@ -619,7 +619,9 @@ def sgd_update(theta, g, lr):
 
 def adafactor_update(theta, g, s0, s1, lr, eps1, wd, tau, eps2=1e-3, d=1.0, decay=-0.8):
     """Adafactor (Shazeer & Stern 2018, Algorithms 4-5) with relative step size, parameter
-    scaling, update clipping and no momentum.  Matrices keep row statistics s0 = R [n] and column
+    scaling, update clipping and no momentum, in the form torch.optim.Adafactor gives it: eps1
+    clamps the factored estimate from below (max(mean(R), eps1), max(V, eps1^2)) instead of being
+    added to the squared gradient.  Matrices keep row statistics s0 = R [n] and column
     statistics s1 = C [m]; vectors keep the unfactored second moment in s0.  Returns theta, s0, s1."""
     w = float(tau) ** decay                                   # 1 - beta2_t
     rho = min(lr, 1.0 / math.sqrt(tau))

@@ -1,5 +1,6 @@
 // Adafactor (Shazeer & Stern 2018, Algorithms 4-5: factored second moment, update clipping,
-// relative step size and parameter scaling, no momentum) for one parameter tensor.
+// relative step size and parameter scaling, no momentum) for one parameter tensor, in the variant
+// where eps1 is a lower clamp on the estimate (as torch.optim.Adafactor has it), not an addend to g^2.
 //   w     = tau^-0.8                 (1 - beta2_t)
 //   rho   = min(lr, 1/sqrt(tau)),  alpha = max(eps2, RMS(theta)) * rho
 //   theta <- theta * (1 - lr * wd)

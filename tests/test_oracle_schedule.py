@@ -165,6 +165,11 @@ def test_peak_trainable_fraction():
     frac = O.peak_trainable_fraction(up, groups)
     assert frac == pytest.approx(202_383_360 / 6_738_415_616)
     assert 0.029 < frac < 0.031
+    # the paper's own figure for this quantity: 2.44 % at the 13B size (40 blocks, d 5120, SwiGLU 13824,
+    # vocabulary 32000, m = 1: the largest group is one block)
+    c13 = cfg.scaled(n_blocks=40, d_model=5120, n_heads=40, d_ffn=13824)
+    frac13 = O.peak_trainable_fraction(synth.count_params(c13), O.build_groups(c13.n_units, 1))
+    assert round(100 * frac13, 2) == _golden()["peak_trainable_fraction_13b_pct"]
     # names listed by the oracle agree with the synthetic tensor catalogue
     for cfgf in (synth.config_tiny_fp32, synth.config_roberta_base, synth.config_gpt2_large, synth.config_llama_7b):
         c = cfgf()[0]
