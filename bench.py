@@ -571,8 +571,35 @@ def run_sweep_optimizer(args):
                          "l2_resident": bool(n * bpe * sets < 126e6)})
             del bufs
             torch.cuda.empty_cache()
+    # the CPU side of the same table: the oracle's update functions (numpy, fp64), as they stand, on 2^20 .. 2^26
+    # elements; bytes counted as for the GPU (the arrays the update reads and writes, at the oracle's 8 bytes each)
+    from oracle import hift_oracle as O
+    cpu_rows = []
+    for kind, name, arrays in ((0, "adamw", 7), (1, "adagrad", 5), (2, "sgdm", 5)):
+        for lg in range(20, 27, 2):
+            n = 1 << lg
+            master, grad, s0, s1 = (x.astype(np.float64) for x in synth.flat_optimizer_inputs(n, seed=lg, warm=True))
+            s0 = np.abs(s0)
+            reps = max(1, min(5, (1 << 24) // n))
+            t0 = time.perf_counter()
+            for r in range(reps):
+                if kind == 0:
+                    master, s0, s1 = O.adamw_update(master, grad, s0, s1, 1e-3, 0.9, 0.999, 1e-8, 0.01, 2 + r)
+                elif kind == 1:
+                    master, s0 = O.adagrad_update(master, grad, s0, 1e-2, 1e-10)
+                else:
+                    master, s0 = O.sgdm_update(master, grad, s0, 1e-3, 0.9)
+            dt = (time.perf_counter() - t0) / reps
+            cpu_rows.append({"optimizer": name, "log2_n": lg, "ms": round(dt * 1e3, 2), "elements_per_s": round(n / dt / 1e6, 1),
+                             "gbs": round(n * 8 * arrays / dt / 1e9, 2)})
+    try:
+        threads = len(os.sched_getaffinity(0))
+    except Exception:
+        threads = os.cpu_count() or 1
     print(json.dumps({"sweep": "optimizer", "unit": "GB/s", "hbm_peak_gbs": peaks["hbm_gbs"],
-                      "peak_source": peaks["source"], "rows": rows}))
+                      "peak_source": peaks["source"], "rows": rows,
+                      "cpu_oracle": {"kind": "oracle (numpy fp64 update functions as they stand)", "cores": threads,
+                                     "elements_per_s_unit": "M elements/s", "rows": cpu_rows}}))
 
 
 def run_sweep_depth(args):

@@ -171,6 +171,40 @@ hift_status hift_grad_view(hift_ctx *ctx, float **grad_dev, size_t *n);
 hift_status hift_step_end(hift_ctx *ctx);
 hift_status hift_step_abort(hift_ctx *ctx);
 
+/* The exchange overlapped with the backward pass.  The truncated backward pass finishes the group's
+ * gradient from the top of its flat span downwards (the last block's down projection first, the lowest
+ * unit's first norm last), so the tail of the buffer can be reduced over the ranks while the head is
+ * still being computed: with one all-reduce per chunk this hides all but the last chunk's exchange
+ * behind the remaining dX / dW GEMMs.
+ *   hift_step_begin_async  enqueues forward + truncated backward and returns without waiting;
+ *   hift_grad_num_chunks / hift_grad_chunk  list the chunks of hift_grad_view's buffer in the order
+ *       they become final (offset and length in elements; together they tile the span exactly once;
+ *       each at least the size set by hift_set_grad_chunk_bytes, default 32 MiB, except the last);
+ *   hift_grad_chunk_wait   makes `cuda_stream` (the caller's communication stream) wait until chunk
+ *       i is final; waiting for the last chunk also covers the step's gate word;
+ *   hift_gate_view         device address of the step's gate word (int32): 0 = the update goes ahead,
+ *       otherwise a positive code of what failed.  Ranks reduce it with MAX next to the last chunk,
+ *       so that all of them call the update off when one of them failed;
+ *   hift_step_finish       = hift_step_end that also returns the loss: orders itself after the work
+ *       enqueued on the stream given to hift_create (make that stream wait for the communication
+ *       stream first), applies the optimizer, starts the write-back, waits for the step and returns
+ *       its status.  A rank whose own pass was fine but whose gate word a peer raised returns the
+ *       peer's failure.
+ * The chunk plan itself is host logic; hift_plan_grad_chunks runs it on a caller-given tensor list
+ * (ascending offsets) and completion order without touching a GPU: chunk_off / chunk_n receive the
+ * chunks, chunk_after[i] the index into completion_order after which chunk i is final.  Returns the
+ * number of chunks, or -1 (bad arguments, max_chunks too small). */
+hift_status hift_step_begin_async(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *labels_dev);
+int32_t     hift_grad_num_chunks(const hift_ctx *ctx);
+hift_status hift_grad_chunk(const hift_ctx *ctx, int32_t i, size_t *offset, size_t *n);
+hift_status hift_grad_chunk_wait(hift_ctx *ctx, int32_t i, void *cuda_stream);
+hift_status hift_gate_view(hift_ctx *ctx, int32_t **gate_dev);
+hift_status hift_set_grad_chunk_bytes(hift_ctx *ctx, size_t bytes);
+hift_status hift_step_finish(hift_ctx *ctx, float *loss_host);
+int32_t     hift_plan_grad_chunks(const size_t *offsets, const size_t *sizes, int32_t n_tensors, size_t span_elems,
+                                  const int32_t *completion_order, int32_t n_completed, size_t min_chunk_elems,
+                                  size_t *chunk_off, size_t *chunk_n, int32_t *chunk_after, int32_t max_chunks);
+
 int32_t hift_active_group(const hift_ctx *ctx);   /* group the NEXT hift_step trains */
 int32_t hift_num_groups(const hift_ctx *ctx);     /* k                               */
 int64_t hift_step_count(const hift_ctx *ctx);     /* t, steps taken so far           */

@@ -69,6 +69,14 @@ def _prototypes():
         "hift_grad_view": (C.c_int, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "hift_step_end": (C.c_int, [vp]),
         "hift_step_abort": (C.c_int, [vp]),
+        "hift_step_begin_async": (C.c_int, [vp, vp, vp]),
+        "hift_grad_num_chunks": (i32, [vp]),
+        "hift_grad_chunk": (C.c_int, [vp, i32, C.POINTER(sz), C.POINTER(sz)]),
+        "hift_grad_chunk_wait": (C.c_int, [vp, i32, vp]),
+        "hift_gate_view": (C.c_int, [vp, C.POINTER(vp)]),
+        "hift_set_grad_chunk_bytes": (C.c_int, [vp, sz]),
+        "hift_step_finish": (C.c_int, [vp, pf]),
+        "hift_plan_grad_chunks": (i32, [vp, vp, i32, sz, vp, i32, sz, vp, vp, vp, i32]),
         "hift_active_group": (i32, [vp]),
         "hift_num_groups": (i32, [vp]),
         "hift_step_count": (i64, [vp]),
@@ -241,6 +249,40 @@ class HiFT:
     def step_abort(self):
         _check(lib().hift_step_abort(self._h), "hift_step_abort")
 
+    def step_begin_async(self, tokens, labels) -> None:
+        """Enqueues forward + truncated backward and returns; see grad_chunks / step_finish."""
+        _check(lib().hift_step_begin_async(self._h, tokens.data_ptr(), labels.data_ptr()), "hift_step_begin_async")
+
+    def grad_chunks(self) -> List[Tuple[int, int]]:
+        """(offset, length) of the chunks of grad_view() in the order the backward pass completes them."""
+        out = []
+        for i in range(lib().hift_grad_num_chunks(self._h)):
+            o, n = C.c_size_t(), C.c_size_t()
+            _check(lib().hift_grad_chunk(self._h, i, C.byref(o), C.byref(n)), "hift_grad_chunk")
+            out.append((o.value, n.value))
+        return out
+
+    def grad_chunk_wait(self, i: int, stream: int) -> None:
+        _check(lib().hift_grad_chunk_wait(self._h, i, stream), "hift_grad_chunk_wait")
+
+    def gate_view(self):
+        """The step's gate word as a one-element int32 CUDA tensor sharing the library's memory."""
+        import torch
+        ptr = C.c_void_p()
+        _check(lib().hift_gate_view(self._h, C.byref(ptr)), "hift_gate_view")
+
+        class _View:
+            __cuda_array_interface__ = {"shape": (1,), "typestr": "<i4", "data": (ptr.value, False), "version": 3}
+        return torch.as_tensor(_View(), device="cuda")
+
+    def set_grad_chunk_bytes(self, nbytes: int) -> None:
+        _check(lib().hift_set_grad_chunk_bytes(self._h, nbytes), "hift_set_grad_chunk_bytes")
+
+    def step_finish(self) -> float:
+        loss = C.c_float()
+        _check(lib().hift_step_finish(self._h, C.byref(loss)), "hift_step_finish")
+        return loss.value
+
     # -- getters
     def active_group(self) -> int:
         return lib().hift_active_group(self._h)
@@ -377,6 +419,20 @@ def adafactor_step(rows, cols, param_bf16, master, grad, state, scratch, lr, eps
                    stream=None):
     _check(lib().hift_adafactor_step(rows, cols, _ptr(param_bf16), _ptr(master), _ptr(grad), _ptr(state),
                                      _ptr(scratch), lr, eps1, weight_decay, tau, _st(stream)), "hift_adafactor_step")
+
+
+def plan_grad_chunks(offsets, sizes, span_elems, completion_order, min_chunk_elems):
+    """Host-only chunk plan (hift_plan_grad_chunks): returns [(offset, length, after)]."""
+    off = np.ascontiguousarray(offsets, dtype=np.uint64)
+    siz = np.ascontiguousarray(sizes, dtype=np.uint64)
+    order = np.ascontiguousarray(completion_order, dtype=np.int32)
+    cap = len(off) + 1
+    co, cn, ca = np.zeros(cap, np.uint64), np.zeros(cap, np.uint64), np.zeros(cap, np.int32)
+    n = lib().hift_plan_grad_chunks(off.ctypes.data, siz.ctypes.data, len(off), int(span_elems), order.ctypes.data,
+                                    len(order), int(min_chunk_elems), co.ctypes.data, cn.ctypes.data, ca.ctypes.data, cap)
+    if n < 0:
+        raise ValueError("hift_plan_grad_chunks: bad arguments")
+    return [(int(co[i]), int(cn[i]), int(ca[i])) for i in range(n)]
 
 
 def tc_error_flag(set_value: int = -1) -> int:

@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "gemm_tc.h"
+#include "grad_chunks.h"
 #include "kernels_adafactor.cuh"
 #include "launchers.cuh"
 
@@ -102,6 +103,14 @@ struct hift_ctx {
   int64_t forced_seq_t0 = 0;
   int cur_sl = 0; double cur_lr = 0.0;   // slot and learning rate of the step in flight
   bool pending_update = false;           // between hift_step_begin and hift_step_end
+  // chunks of the active group's gradient in completion order (data-parallel overlap)
+  struct ChunkRec { size_t off, n; cudaEvent_t ev; };
+  GradChunkPlanner planner;
+  std::vector<int> planner_idx;          // tensor -> index in the planner (-1: not in the active group)
+  std::vector<ChunkRec> chunks;
+  std::vector<cudaEvent_t> chunk_events; // pool, grown on demand
+  size_t chunk_min_elems = (size_t)8 << 20;   // 32 MB of fp32 gradient
+  cudaEvent_t ev_bwd;                    // forward + backward (and the gate word) complete
 
   // device memory
   std::vector<void*> dev_allocs;
@@ -183,6 +192,25 @@ struct hift_ctx {
 };
 
 #define LAUNCH(cls, work, ...) do { c->pre(cls, work); __VA_ARGS__; c->post(); } while (0)
+
+namespace {
+void emit_chunk(hift_ctx* c, size_t off, size_t n) {
+  if (c->chunks.size() == c->chunk_events.size()) {
+    cudaEvent_t e;
+    c->note(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    c->chunk_events.push_back(e);
+  }
+  cudaEvent_t ev = c->chunk_events[c->chunks.size()];
+  c->note(cudaEventRecord(ev, c->st));
+  c->chunks.push_back(hift_ctx::ChunkRec{off, n, ev});
+}
+// The gradient of tensor ti has had its last contribution enqueued.
+void grad_done(hift_ctx* c, int ti) {
+  if (ti < 0 || c->planner_idx[ti] < 0) return;
+  size_t off, n;
+  if (c->planner.complete(c->planner_idx[ti], &off, &n)) emit_chunk(c, off, n);
+}
+}  // namespace
 
 namespace {
 
@@ -584,18 +612,18 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
   float* x2 = (float*)s[S_X2];
   if (c->m.arch == 1) {
     float* z = (float*)s[S_Z];
-    if (on) norm_bwd_params(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, b.n2_b);
+    if (on) { norm_bwd_params(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, b.n2_b); grad_done(c, b.n2_b); grad_done(c, b.n2_g); }
     norm_bwd_dx(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, nullptr, c->dxb, c->dxb_a);          // dz
     linear_dx_gelu_bwd(c, T, d, f, c->dxb_a, c->P(b.w_fc2), s[S_A]);                                // du -> da
-    if (on) { linear_dw(c, T, d, f, c->dxb_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxb, true, T, d, d, b.b_fc2); }
+    if (on) { linear_dw(c, T, d, f, c->dxb_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxb, true, T, d, d, b.b_fc2); grad_done(c, b.b_fc2); grad_done(c, b.w_fc2); }
     linear_dx(c, T, f, d, c->dbig, f, c->P(b.w_fc1), c->dxa, d, c->dxb, d, true);                   // dx1
-    if (on) { linear_dw(c, T, f, d, c->dbig, f, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, f, f, b.b_fc1); }
-    if (on) norm_bwd_params(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, b.n1_b);
+    if (on) { linear_dw(c, T, f, d, c->dbig, f, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, f, f, b.b_fc1); grad_done(c, b.b_fc1); grad_done(c, b.w_fc1); }
+    if (on) { norm_bwd_params(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, b.n1_b); grad_done(c, b.n1_b); grad_done(c, b.n1_g); }
     norm_bwd_dx(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, nullptr, c->dxb, c->dxb_a);         // dy
     linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                  // do
-    if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); }
+    if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
     attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
-    if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, x_a, d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); }
+    if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, x_a, d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); grad_done(c, b.b_qkv); grad_done(c, b.w_qkv); }
     if (need_dx) linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dxa, d, c->dxb, d, true);
     return;
   }
@@ -611,19 +639,19 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
   }
   if (!act_done && c->m.arch != 2) { linear_dx_gelu_bwd(c, T, d, f, c->dxa_a, c->P(b.w_fc2), s[S_A]); act_done = true; }
   if (!act_done) linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);  // ds
-  if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxa, true, T, d, d, b.b_fc2); }
+  if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxa, true, T, d, d, b.b_fc2); grad_done(c, b.b_fc2); grad_done(c, b.w_fc2); }
   if (!act_done) act_bwd(c, s[S_A]);                                                                // da in dbig [T,fa]
   linear_dx(c, T, fa, d, c->dbig, fa, c->P(b.w_fc1), c->dt1, d, nullptr, 0, false);                 // dh2
-  if (on) { linear_dw(c, T, fa, d, c->dbig, fa, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, fa, fa, b.b_fc1); }
-  if (on) norm_bwd_params(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, b.n2_b);
+  if (on) { linear_dw(c, T, fa, d, c->dbig, fa, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, fa, fa, b.b_fc1); grad_done(c, b.b_fc1); grad_done(c, b.w_fc1); }
+  if (on) { norm_bwd_params(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, b.n2_b); grad_done(c, b.n2_b); grad_done(c, b.n2_g); }
   norm_bwd_dx(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, c->dxa, c->dxb, c->dxb_a);            // dx2
   linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                    // do
-  if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); }
+  if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
   attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
   if (c->m.arch == 2) rope(c, c->dqkv, -1.0f);
   linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dt1, d, nullptr, 0, false);           // dh1
-  if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, s[S_H1], d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); }
-  if (on) norm_bwd_params(c, c->dt1, false, x_r, (float*)s[S_ST1], b.n1_g, b.n1_b);
+  if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, s[S_H1], d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); grad_done(c, b.b_qkv); grad_done(c, b.w_qkv); }
+  if (on) { norm_bwd_params(c, c->dt1, false, x_r, (float*)s[S_ST1], b.n1_g, b.n1_b); grad_done(c, b.n1_b); grad_done(c, b.n1_g); }
   if (need_dx) norm_bwd_dx(c, c->dt1, false, x_r, (float*)s[S_ST1], b.n1_g, c->dxb, c->dxa, c->dxa_a);
 }
 
@@ -708,6 +736,12 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   if (c->arena_off > c->arena_cap) return HIFT_ERR_CFG;
   if (c->checked)      // the plan moves with the group: paint this step's guard regions before anything runs
     for (size_t o : c->guards) c->note(cudaMemsetAsync(c->arena + o, kGuardByte, kGuardBytes, c->st));
+  // the group's tensors, for the completion-ordered chunks of its gradient
+  c->planner.reset(gr.numel, c->chunk_min_elems);
+  c->planner_idx.assign(c->tens.size(), -1);
+  c->chunks.clear();
+  for (int u = lo; u <= hi; ++u)
+    for (int ti : c->unit_tens[u]) c->planner_idx[ti] = c->planner.add(c->tens[ti].off - gr.off, c->tens[ti].numel);
   // inputs produced on the caller's stream are visible to the step
   c->note(cudaEventRecord(c->ev_in, c->caller));
   c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
@@ -764,6 +798,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
       // dWc[C,d] = dlogits^T pooled ; pooled rows have stride S*d
       gemm(c, HIFT_K_GEMM_DW, C, d, B, c->logits, 1, C, c->x_final_a, (int64_t)S * d, 1, c->G(c->t_wc), d, nullptr, nullptr, 0, true);
       bias_grad(c, c->logits, false, B, C, C, c->t_bc);
+      grad_done(c, c->t_bc); grad_done(c, c->t_wc);
     }
     if (lo == L + 1) done = true;
     else {
@@ -775,8 +810,9 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
     const int tw = m.tie_head ? c->t_tok : c->t_wh;
     const bool w_on = m.tie_head ? active(0) : head_on;
     if (w_on) linear_dw(c, T, V, d, c->logits, Vp, c->xf, d, c->G(tw));
+    if (w_on && !m.tie_head) grad_done(c, tw);          // a tied matrix still gets the embedding's share
     linear_dx(c, T, V, d, c->logits, Vp, c->P(tw), c->dt1, d, nullptr, 0, false);
-    if (head_on) norm_bwd_params(c, c->dt1, false, c->x_final, c->stf, c->t_fg, c->t_fb);
+    if (head_on) { norm_bwd_params(c, c->dt1, false, c->x_final, c->stf, c->t_fg, c->t_fb); grad_done(c, c->t_fb); grad_done(c, c->t_fg); }
     if (lo == L + 1) done = true;
     else norm_bwd_dx(c, c->dt1, false, c->x_final, c->stf, c->t_fg, nullptr, c->dxa, c->dxa_a);
   }
@@ -798,6 +834,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
     const float* src = c->dxa;
     if (m.arch == 1) {
       norm_bwd_params(c, c->dxa, true, c->emb_e, c->st_e, c->t_eg, c->t_eb);
+      grad_done(c, c->t_eb); grad_done(c, c->t_eg);
       norm_bwd_dx(c, c->dxa, true, c->emb_e, c->st_e, c->t_eg, nullptr, c->dxb, nullptr);
       src = c->dxb;
     }
@@ -806,9 +843,18 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
     if (c->t_pos >= 0) {
       LAUNCH(HIFT_K_EMBED, (double)T * d * 4 + (double)S * d * 4,
              embed_bwd_pos_kernel<<<S, 128, 0, c->st>>>(src, c->G(c->t_pos), B, S, d));
+      grad_done(c, c->t_pos);
     }
+    grad_done(c, c->t_tok);
   }
-
+  {
+    size_t off, n;
+    if (c->planner.flush(&off, &n)) emit_chunk(c, off, n);
+  }
+  // the gate word of this step's update: set once the whole pass is behind it, before the last chunk is released
+  step_gate_kernel<<<1, 32, 0, c->st>>>(c->scal, c->mixed ? gemm_tc_error_device_ptr() : nullptr, c->gate);
+  c->note(cudaGetLastError());
+  c->note(cudaEventRecord(c->ev_bwd, c->st));
   return HIFT_OK;
 }
 
@@ -820,8 +866,6 @@ void enqueue_update(hift_ctx* c) {
   const int sl = c->cur_sl;
   SlotRec* sr = c->offload ? &c->slot[sl] : nullptr;
   const double lr = c->cur_lr;
-  step_gate_kernel<<<1, 32, 0, c->st>>>(c->scal, c->mixed ? gemm_tc_error_device_ptr() : nullptr, c->gate);
-  c->note(cudaGetLastError());
   if (c->offload) {
     c->note(cudaEventRecord(c->tl[3], c->st));
     c->note(cudaStreamWaitEvent(c->st, sr->ev_h2d, 0));
@@ -907,7 +951,8 @@ hift_status finish_step(hift_ctx* c, float* loss_host, bool updated) {
   if (loss_host) *loss_host = loss;
   if (bad_h) return HIFT_ERR_INPUT;
   if (!isfinite(loss)) return HIFT_ERR_NONFINITE;
-  if (updated && gate_h != 0) return HIFT_ERR_TIMEOUT;     // the flag was raised between the two reads
+  if (updated && gate_h != 0)      // nothing wrong here, yet the update was called off: a peer's step failed
+    return gate_h == 100 ? HIFT_ERR_INPUT : (gate_h == 101 ? HIFT_ERR_NONFINITE : HIFT_ERR_TIMEOUT);
   return HIFT_OK;
 }
 // A step that failed changed nothing on the device (the gate kept the optimizer out, the write-back
@@ -1024,6 +1069,7 @@ void hift_destroy(hift_ctx* c) {
   for (auto& g : c->groups) if (g.blob) cudaFreeHost(g.blob);
   if (c->scal_host) cudaFreeHost(c->scal_host);
   for (auto e : c->ev_pool) cudaEventDestroy(e);
+  for (auto e : c->chunk_events) cudaEventDestroy(e);
   if (c->events_made) {
     for (int i = 0; i < kMaxSlots; ++i) {
       SlotRec& sr = c->slot[i];
@@ -1031,6 +1077,7 @@ void hift_destroy(hift_ctx* c) {
       cudaEventDestroy(sr.tl_h2d0); cudaEventDestroy(sr.tl_h2d1);
     }
     cudaEventDestroy(c->ev_fwd);
+    cudaEventDestroy(c->ev_bwd);
     cudaEventDestroy(c->ev_in);
     for (int i = 0; i < 7; ++i) cudaEventDestroy(c->tl[i]);
   }
@@ -1127,6 +1174,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     cudaEventCreate(&sr.tl_h2d1);
   }
   cudaEventCreateWithFlags(&c->ev_fwd, cudaEventDisableTiming);
+  cudaEventCreateWithFlags(&c->ev_bwd, cudaEventDisableTiming);
   for (int i = 0; i < 7; ++i) cudaEventCreate(&c->tl[i]);
   c->events_made = true;
   cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming);
@@ -1275,18 +1323,69 @@ hift_status hift_grad_view(hift_ctx* c, float** grad_dev, size_t* n) {
   *n = c->groups[c->last_group].numel;
   return HIFT_OK;
 }
-hift_status hift_step_end(hift_ctx* c) {
+hift_status hift_step_begin_async(hift_ctx* c, const int32_t* tok, const int32_t* lab) {
+  if (!c || !tok || !lab) return HIFT_ERR_INPUT;
+  if (c->pending_update) return HIFT_ERR_CFG;
+  const hift_status s = enqueue_forward_backward(c, tok, lab);
+  if (s != HIFT_OK) return s;
+  c->pending_update = true;
+  return c->first_err == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+int32_t hift_grad_num_chunks(const hift_ctx* c) { return c && c->pending_update ? (int32_t)c->chunks.size() : 0; }
+hift_status hift_grad_chunk(const hift_ctx* c, int32_t i, size_t* offset, size_t* n) {
+  if (!c || !c->pending_update || i < 0 || i >= (int)c->chunks.size() || !offset || !n) return HIFT_ERR_CFG;
+  *offset = c->chunks[i].off; *n = c->chunks[i].n;
+  return HIFT_OK;
+}
+hift_status hift_grad_chunk_wait(hift_ctx* c, int32_t i, void* stream) {
+  if (!c || !c->pending_update || i < 0 || i >= (int)c->chunks.size()) return HIFT_ERR_CFG;
+  cudaError_t e = cudaStreamWaitEvent((cudaStream_t)stream, c->chunks[i].ev, 0);
+  if (e == cudaSuccess && i + 1 == (int)c->chunks.size()) e = cudaStreamWaitEvent((cudaStream_t)stream, c->ev_bwd, 0);
+  return e == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_gate_view(hift_ctx* c, int32_t** gate_dev) {
+  if (!c || !gate_dev) return HIFT_ERR_CFG;
+  *gate_dev = c->gate;
+  return HIFT_OK;
+}
+hift_status hift_set_grad_chunk_bytes(hift_ctx* c, size_t bytes) {
+  if (!c || c->pending_update) return HIFT_ERR_CFG;
+  c->chunk_min_elems = bytes / sizeof(float) ? bytes / sizeof(float) : 1;
+  return HIFT_OK;
+}
+hift_status hift_step_finish(hift_ctx* c, float* loss_host) {
   if (!c || !c->pending_update) return HIFT_ERR_CFG;
-  // whatever the caller did to the gradient on its own stream is ordered before the update
   c->note(cudaEventRecord(c->ev_in, c->caller));
   c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
   enqueue_update(c);
   c->pending_update = false;
-  const hift_status s = finish_step(c, nullptr, true);
+  const hift_status s = finish_step(c, loss_host, true);
   if (s == HIFT_OK) c->t += 1;
   else step_failed(c);
   return s;
 }
+// Host-only: the chunk plan for a span of tensors and a completion order (no GPU involved).
+int32_t hift_plan_grad_chunks(const size_t* offsets, const size_t* sizes, int32_t n_tensors, size_t span_elems,
+                              const int32_t* completion_order, int32_t n_completed, size_t min_chunk_elems,
+                              size_t* chunk_off, size_t* chunk_n, int32_t* chunk_after, int32_t max_chunks) {
+  if (!offsets || !sizes || n_tensors < 1 || (n_completed > 0 && !completion_order) || !chunk_off || !chunk_n || max_chunks < 1) return -1;
+  GradChunkPlanner p;
+  p.reset(span_elems, min_chunk_elems);
+  for (int i = 0; i < n_tensors; ++i) p.add(offsets[i], sizes[i]);
+  int32_t nc = 0;
+  size_t off, n;
+  for (int i = 0; i < n_completed; ++i)
+    if (p.complete(completion_order[i], &off, &n)) {
+      if (nc == max_chunks) return -1;
+      chunk_off[nc] = off; chunk_n[nc] = n; if (chunk_after) chunk_after[nc] = i; ++nc;
+    }
+  if (p.flush(&off, &n)) {
+    if (nc == max_chunks) return -1;
+    chunk_off[nc] = off; chunk_n[nc] = n; if (chunk_after) chunk_after[nc] = n_completed; ++nc;
+  }
+  return nc;
+}
+hift_status hift_step_end(hift_ctx* c) { return hift_step_finish(c, nullptr); }
 hift_status hift_step_abort(hift_ctx* c) {
   if (!c || !c->pending_update) return HIFT_ERR_CFG;
   c->pending_update = false;       // the gradient is dropped; the state uploaded for the step stays resident

@@ -502,16 +502,17 @@ __global__ void publish_scalars_kernel(const float* __restrict__ src, const int*
 
 // The step's gate word, read by every optimizer kernel before its first store: non-zero when the
 // update must not happen.  src = the step's scalars ([0] loss, [2] bad-input flag); tc_error = the
-// tensor-core kernels' time-out flag (may be null).  Codes: the time-out code (> 0), -1 bad input,
-// -2 non-finite loss.
+// tensor-core kernels' time-out flag (may be null).  Codes: the time-out code (1 .. 9), 100 bad input,
+// 101 non-finite loss; all positive, so that data-parallel ranks can share the word with a MAX reduction and
+// every rank calls the update off when any rank's step failed.
 __global__ void step_gate_kernel(const float* __restrict__ src, const int* __restrict__ tc_error, int* __restrict__ gate) {
   if (threadIdx.x != 0) return;
   int v = 0;
   const int tc = tc_error ? *tc_error : 0;
   const float loss = src[0];
   if (tc != 0) v = tc;
-  else if (__float_as_int(src[2]) != 0) v = -1;
-  else if (!(fabsf(loss) <= 3.402823466e38f)) v = -2;
+  else if (__float_as_int(src[2]) != 0) v = 100;
+  else if (!(fabsf(loss) <= 3.402823466e38f)) v = 101;
   *gate = v;
 }
 

@@ -51,11 +51,60 @@ def allreduce_mean_(tensor):
     return tensor
 
 
-def data_parallel_step(h, tokens, labels) -> float:
+def allreduce_chunks_mean_(tensor, chunks, wait_for_chunk=None, flag=None):
+    """Mean over ranks of `tensor`, exchanged chunk by chunk in the given order (each (offset, length, ...)),
+    every chunk as its own asynchronous all-reduce so that later chunks can still be produced while earlier
+    ones travel.  wait_for_chunk(i) is called before chunk i is handed to the collective (on GPUs: makes
+    the communication stream wait for the event that says the chunk is final).  `flag` (one integer
+    element, optional) is reduced with MAX after the last chunk: non-zero on any rank means non-zero on
+    all.  Returns when every collective has been waited for (on GPUs: enqueued on the current stream)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        if wait_for_chunk is not None:
+            for i in range(len(chunks)):
+                wait_for_chunk(i)
+        return tensor
+    n = dist.get_world_size()
+    works = []
+    for i, ch in enumerate(chunks):
+        if wait_for_chunk is not None:
+            wait_for_chunk(i)
+        works.append(dist.all_reduce(tensor[ch[0]:ch[0] + ch[1]], op=dist.ReduceOp.SUM, async_op=True))
+    if flag is not None:
+        works.append(dist.all_reduce(flag, op=dist.ReduceOp.MAX, async_op=True))
+    for w in works:
+        w.wait()
+    tensor.mul_(1.0 / n)
+    return tensor
+
+
+_comm_streams = {}
+
+
+def data_parallel_step(h, tokens, labels, overlap: bool = True) -> float:
     """One data-parallel step of context `h` on this rank's shard: forward + truncated backward,
     mean of the group's gradient over ranks, update.  Every rank follows the same group schedule,
-    so no communication is needed to agree on the group."""
-    loss = h.step_begin(tokens, labels)
-    allreduce_mean_(h.grad_view())
-    h.step_end()
-    return loss
+    so no communication is needed to agree on the group.
+
+    overlap=True: the backward pass is enqueued without waiting, and the gradient is reduced chunk by
+    chunk on a communication stream in the order the backward pass completes the chunks (top of the
+    group's span first), so that all but the last exchange run under the remaining GEMMs; the ranks
+    also share the step's gate word, and all of them skip the update when one of them failed.
+    overlap=False: one all-reduce between the two synchronous halves of the step."""
+    import torch
+    if not overlap:
+        loss = h.step_begin(tokens, labels)
+        allreduce_mean_(h.grad_view())
+        h.step_end()
+        return loss
+    dev = torch.cuda.current_device()
+    comm = _comm_streams.get(dev)
+    if comm is None:
+        comm = _comm_streams[dev] = torch.cuda.Stream()
+    h.step_begin_async(tokens, labels)
+    grad, gate = h.grad_view(), h.gate_view()
+    chunks = h.grad_chunks()
+    with torch.cuda.stream(comm):
+        allreduce_chunks_mean_(grad, chunks, wait_for_chunk=lambda i: h.grad_chunk_wait(i, comm.cuda_stream), flag=gate)
+    torch.cuda.current_stream().wait_stream(comm)       # hift_step_finish orders itself after the current stream
+    return h.step_finish()

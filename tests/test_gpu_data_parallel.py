@@ -75,3 +75,115 @@ def test_two_emulated_ranks_average_gradients_and_stay_in_sync():
                 assert rel_l2(a0, ref.get_param(n)) <= 1e-4, (t, n)
     for h in (ref, r0, r1):
         h.close()
+
+
+def test_overlapped_exchange_chunks_tile_the_gradient_and_change_no_bits():
+    """The asynchronous first half + chunk list + hift_step_finish (what dist_util.data_parallel_step drives)
+    on one rank: the chunks come in the order the backward pass finishes them (from the top of the span
+    down), tile the flat gradient exactly once, respect the minimum size except for the last, and the step
+    leaves the same bits as hift_step."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, dist_util
+    cfg = _cfg(2)
+    gc, oc = synth.GroupCfg(layers_per_group=2), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=2)
+    p0 = synth.init_params(cfg, 2)
+    a, b = HiFT(cfg, gc, oc), HiFT(cfg, gc, oc)
+    a.set_params(p0)
+    b.set_params(p0)
+    b.set_grad_chunk_bytes(256 << 10)
+    seen = []
+    for t in range(2 * a.num_groups()):
+        tok, lab = synth.lm_batch(cfg, 4, t)
+        tt, ll = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
+        la = a.step(tt, ll)
+        if t % 2 == 0:
+            lb = dist_util.data_parallel_step(b, tt, ll)          # no process group: a world of one
+        else:
+            b.step_begin_async(tt, ll)
+            chunks = b.grad_chunks()
+            n = b.grad_view().numel()
+            assert sum(c[1] for c in chunks) == n
+            ends = [c[0] + c[1] for c in chunks]
+            assert ends[0] == n and chunks[-1][0] == 0
+            assert all(chunks[i + 1][0] + chunks[i + 1][1] == chunks[i][0] for i in range(len(chunks) - 1))   # descending, gap-free
+            assert all(c[1] >= (256 << 10) // 4 for c in chunks[:-1])
+            seen.append(len(chunks))
+            for i in range(len(chunks)):
+                b.grad_chunk_wait(i, torch.cuda.current_stream().cuda_stream)
+            assert int(b.gate_view().item()) == 0
+            lb = b.step_finish()
+        assert la == lb
+    assert max(seen) > 3                                          # the block groups really were cut into several chunks
+    for n in a.tensor_names():
+        assert np.array_equal(a.get_param(n), b.get_param(n)), n
+    a.close()
+    b.close()
+
+
+def test_two_emulated_ranks_exchange_chunk_by_chunk_and_share_the_gate():
+    """Two contexts as two ranks (run one after the other on one GPU): gradients averaged chunk by chunk in
+    the order the chunks complete keep the replicas bit-identical; and when one rank's step fails (a NaN
+    planted in one of its frozen parameters), the MAX of the gate words calls the update off on both, both
+    report the failure, and neither changes a bit."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError
+    half = _cfg(2)
+    gc, oc = synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
+    p0 = synth.init_params(half, 5)
+    r0, r1 = HiFT(half, gc, oc), HiFT(half, gc, oc)
+    for h in (r0, r1):
+        h.set_params(p0)
+        h.set_grad_chunk_bytes(128 << 10)
+    full = _cfg(4)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def exchange(poison=False):
+        g0, g1 = r0.grad_view(), r1.grad_view()
+        c0, c1 = r0.grad_chunks(), r1.grad_chunks()
+        assert c0 == c1                                            # same schedule on every rank, nothing to agree on
+        for i, (off, n) in enumerate(c0):
+            r0.grad_chunk_wait(i, st)
+            r1.grad_chunk_wait(i, st)
+            avg = (g0[off:off + n] + g1[off:off + n]) * 0.5
+            g0[off:off + n].copy_(avg)
+            g1[off:off + n].copy_(avg)
+        f0, f1 = r0.gate_view(), r1.gate_view()
+        m = torch.maximum(f0, f1)
+        f0.copy_(m)
+        f1.copy_(m)
+        return int(m.item())
+
+    for t in range(3):
+        tok, lab = synth.lm_batch(full, 8, t)
+        r0.step_begin_async(torch.from_numpy(tok[:2].copy()).cuda(), torch.from_numpy(lab[:2].copy()).cuda())
+        r1.step_begin_async(torch.from_numpy(tok[2:].copy()).cuda(), torch.from_numpy(lab[2:].copy()).cuda())
+        assert exchange() == 0
+        r0.step_finish()
+        r1.step_finish()
+        for n in r0.tensor_names():
+            assert np.array_equal(r0.get_param(n), r1.get_param(n)), (t, n)
+    # a failing rank
+    g = r1.active_group()
+    lo, hi = r1.group_units(g)
+    victim = [n for n in r1.tensor_names() if not (lo <= r1.tensor_info(n)[0] <= hi) and n.endswith("w_o")][0]
+    good = r1.get_param(victim)
+    bad = good.copy()
+    bad[0, 0] = np.nan
+    r1.set_param(victim, bad)
+    before0 = {n: r0.get_param(n) for n in r0.tensor_names()}
+    tok, lab = synth.lm_batch(full, 8, 7)
+    r0.step_begin_async(torch.from_numpy(tok[:2].copy()).cuda(), torch.from_numpy(lab[:2].copy()).cuda())
+    r1.step_begin_async(torch.from_numpy(tok[2:].copy()).cuda(), torch.from_numpy(lab[2:].copy()).cuda())
+    assert exchange() == 101                                       # non-finite loss on rank 1, now known to both
+    for h in (r0, r1):
+        with pytest.raises(HiftError) as e:
+            h.step_finish()
+        assert e.value.status == 5
+        assert h.step_count() == 3
+    for n in r0.tensor_names():
+        assert np.array_equal(r0.get_param(n), before0[n]), n      # rank 0 averaged a NaN gradient in, and still changed nothing
+    r1.set_param(victim, good)
+    for n in r0.tensor_names():
+        assert np.array_equal(r0.get_param(n), r1.get_param(n)), n
+    r0.close()
+    r1.close()
