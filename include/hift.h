@@ -247,6 +247,16 @@ hift_status hift_get_grad(hift_ctx *ctx, int32_t tensor, float *dst_host, size_t
  * hash of (seed, element index), gains 1, biases 0; optimizer state zero. */
 hift_status hift_init_synthetic(hift_ctx *ctx, uint64_t seed, double std);
 
+/* Weights from a file in the library's container format ("HIFTWTS1": magic[8], uint32 n, then n records of
+ * { char name[64]; uint32 dtype (0 fp32, 1 bf16); uint64 rows, cols; rows*cols elements }, names and shapes
+ * as hift_tensor_info reports them).  Each record goes through hift_set_param (fp32 master and bf16 model
+ * copy; optimizer state is left alone).  strict != 0: every tensor of the model must be in the file.
+ * *n_loaded (may be NULL) receives the number of tensors set.  HIFT_ERR_INPUT for a missing / short /
+ * foreign file, an unknown or repeated tensor, a wrong shape; tensors set before the error stay set.
+ * The package's weights.py writes this format and converts safetensors checkpoints with the public
+ * LLaMA / GPT-2 / RoBERTa tensor names into it. */
+hift_status hift_load_weights(hift_ctx *ctx, const char *path, int32_t strict, int32_t *n_loaded);
+
 /* Checkpoint: the whole training state is the fp32 master (or fp32 parameters), the optimizer
  * state and update count of every group (which Algorithm 1 keeps on the host between a group's
  * turns anyway), and the step counter t; the group order follows from the configuration.

@@ -297,6 +297,47 @@ def cross_entropy(logits, labels):
 
 
 # --------------------------------------------------------------------------
+# Dropout masks from a counter-based generator
+# --------------------------------------------------------------------------
+# The paper's hyper-parameter tables fine-tune with the models' usual dropout; a deterministic parity
+# check needs both sides to draw the same mask, so the mask is a pure function of (seed, step, site,
+# element): Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+# SC'11), key = the 64-bit seed, counter = (element // 4 as two words, site, step), word element % 4
+# of the output.  An element is kept iff its word >= floor(p * 2^32), and kept values are scaled by
+# 1 / (1 - p).  Sites: 0 = embedding output; 1 + 2 i = output of block i's attention projection and
+# 2 + 2 i = output of its feed-forward network, each before the residual addition.  Attention
+# probabilities are not dropped.
+_PHILOX_M0, _PHILOX_M1, _PHILOX_W0, _PHILOX_W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(c0, c1, c2, c3, k0: int, k1: int):
+    """Ten rounds of Philox-4x32 on arrays of 32-bit counter words; returns four arrays of 32-bit words."""
+    m32 = np.uint64(0xFFFFFFFF)
+    c = [np.asarray(x, dtype=np.uint64) & m32 for x in (c0, c1, c2, c3)]
+    k0, k1 = np.uint64(k0 & 0xFFFFFFFF), np.uint64(k1 & 0xFFFFFFFF)
+    for _ in range(10):
+        p0 = np.uint64(_PHILOX_M0) * c[0]
+        p1 = np.uint64(_PHILOX_M1) * c[2]
+        c = [(p1 >> np.uint64(32)) ^ c[1] ^ k0, p1 & m32, (p0 >> np.uint64(32)) ^ c[3] ^ k1, p0 & m32]
+        k0 = (k0 + np.uint64(_PHILOX_W0)) & m32
+        k1 = (k1 + np.uint64(_PHILOX_W1)) & m32
+    return c
+
+
+def dropout_mask(numel: int, p: float, seed: int, site: int, step: int) -> np.ndarray:
+    """Multiplier of each of `numel` elements (row-major order): 0 where dropped, 1 / (1 - p) where kept."""
+    if p <= 0.0:
+        return np.ones(numel, dtype=F64)
+    idx = np.arange(numel, dtype=np.uint64)
+    blk = idx >> np.uint64(2)
+    w = philox4x32_10(blk & np.uint64(0xFFFFFFFF), blk >> np.uint64(32), np.full(numel, site, dtype=np.uint64),
+                      np.full(numel, step & 0xFFFFFFFF, dtype=np.uint64), seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    word = np.choose((idx & np.uint64(3)).astype(np.int64), w)
+    thr = np.uint64(int(math.floor(p * 4294967296.0)))
+    return np.where(word >= thr, 1.0 / (1.0 - p), 0.0)
+
+
+# --------------------------------------------------------------------------
 # Model: forward, full backward, truncated backward
 # --------------------------------------------------------------------------
 def tensor_names_of_unit(cfg, unit: int) -> List[str]:
@@ -335,19 +376,28 @@ def _merge_heads(t):
     return t.reshape(B, S, H * dh)
 
 
-def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarray, lens=None):
-    """Whole-model forward in fp64.  Returns (loss, cache)."""
+def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarray, lens=None, drop=None):
+    """Whole-model forward in fp64.  Returns (loss, cache).
+    drop = (p, seed, step): dropout with the counter-based masks of dropout_mask; None: no dropout."""
     B, S = tokens.shape
     d, H = cfg.d_model, cfg.n_heads
     dh = d // H
     causal = bool(cfg.causal)
     eps = cfg.norm_eps
     cache = {"tokens": tokens, "labels": labels, "blocks": []}
+
+    def mask(site):
+        if drop is None or drop[0] <= 0.0:
+            return 1.0
+        return dropout_mask(B * S * d, drop[0], drop[1], site, drop[2]).reshape(B, S, d)
+
     x = P["tok_emb"][tokens]                                   # [B,S,d]
     if cfg.arch in (0, 1):
         x = x + P["pos_emb"][:S][None, :, :]
     if cfg.arch == 1:
         x, cache["emb_ln"] = layernorm_fwd(x, P["emb_ln_g"], P["emb_ln_b"], eps)
+    cache["mask_emb"] = mask(0)
+    x = x * cache["mask_emb"]
     if cfg.arch == 2:
         cos, sin = rope_tables(S, dh, cfg.rope_base)
         cache["rope"] = (cos, sin)
@@ -360,11 +410,12 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
             o, prob = attention_fwd(q, k, v, causal, lens)
             om = _merge_heads(o)
-            x2 = x + om @ P[p + "w_o"].T + P[p + "b_o"]
+            c["mask_a"], c["mask_f"] = mask(1 + 2 * i), mask(2 + 2 * i)
+            x2 = x + (om @ P[p + "w_o"].T + P[p + "b_o"]) * c["mask_a"]
             h2, c["ln2"] = layernorm_fwd(x2, P[p + "ln2_g"], P[p + "ln2_b"], eps)
             a = h2 @ P[p + "w_fc1"].T + P[p + "b_fc1"]
             u = gelu_fwd(a)
-            x3 = x2 + u @ P[p + "w_fc2"].T + P[p + "b_fc2"]
+            x3 = x2 + (u @ P[p + "w_fc2"].T + P[p + "b_fc2"]) * c["mask_f"]
             c.update(h1=h1, q=q, k=k, v=v, p=prob, om=om, h2=h2, a=a, u=u)
             x = x3
         elif cfg.arch == 1:        # post-LN: x = LN1(x + Attn x); x = LN2(x + FFN x)
@@ -372,11 +423,12 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
             o, prob = attention_fwd(q, k, v, causal, lens)
             om = _merge_heads(o)
-            y = x + om @ P[p + "w_o"].T + P[p + "b_o"]
+            c["mask_a"], c["mask_f"] = mask(1 + 2 * i), mask(2 + 2 * i)
+            y = x + (om @ P[p + "w_o"].T + P[p + "b_o"]) * c["mask_a"]
             x1, c["ln1"] = layernorm_fwd(y, P[p + "ln1_g"], P[p + "ln1_b"], eps)
             a = x1 @ P[p + "w_fc1"].T + P[p + "b_fc1"]
             u = gelu_fwd(a)
-            z = x1 + u @ P[p + "w_fc2"].T + P[p + "b_fc2"]
+            z = x1 + (u @ P[p + "w_fc2"].T + P[p + "b_fc2"]) * c["mask_f"]
             xo, c["ln2"] = layernorm_fwd(z, P[p + "ln2_g"], P[p + "ln2_b"], eps)
             c.update(xin=x, q=q, k=k, v=v, p=prob, om=om, x1=x1, a=a, u=u)
             x = xo
@@ -388,12 +440,13 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             k = rope_apply(k, cos, sin)
             o, prob = attention_fwd(q, k, v, causal, lens)
             om = _merge_heads(o)
-            x2 = x + om @ P[p + "w_o"].T
+            c["mask_a"], c["mask_f"] = mask(1 + 2 * i), mask(2 + 2 * i)
+            x2 = x + (om @ P[p + "w_o"].T) * c["mask_a"]
             h2, c["rms2"] = rmsnorm_fwd(x2, P[p + "rms2_g"], eps)
             gu = h2 @ P[p + "w_gu"].T
             gate, up = np.split(gu, 2, axis=-1)
             s = swiglu_fwd(gate, up)
-            x3 = x2 + s @ P[p + "w_down"].T
+            x3 = x2 + (s @ P[p + "w_down"].T) * c["mask_f"]
             c.update(h1=h1, q=q, k=k, v=v, p=prob, om=om, h2=h2, gate=gate, up=up, s=s)
             x = x3
         cache["blocks"].append(c)
@@ -482,10 +535,11 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
         c = cache["blocks"][i]
         p = f"b{i}."
         if cfg.arch == 0:
-            du = dx @ P[p + "w_fc2"]
+            dfo = dx * c["mask_f"]                               # through the dropout of the feed-forward output
+            du = dfo @ P[p + "w_fc2"]
             if on:
-                G[p + "w_fc2"] = _rows(dx).T @ _rows(c["u"])
-                G[p + "b_fc2"] = _rows(dx).sum(axis=0)
+                G[p + "w_fc2"] = _rows(dfo).T @ _rows(c["u"])
+                G[p + "b_fc2"] = _rows(dfo).sum(axis=0)
             da = gelu_bwd(du, c["a"])
             dh2 = da @ P[p + "w_fc1"]
             if on:
@@ -495,10 +549,11 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             if on:
                 G[p + "ln2_g"], G[p + "ln2_b"] = dg, db
             dx2 = dx + dn
-            dom = dx2 @ P[p + "w_o"]
+            dao = dx2 * c["mask_a"]                              # through the dropout of the attention output
+            dom = dao @ P[p + "w_o"]
             if on:
-                G[p + "w_o"] = _rows(dx2).T @ _rows(c["om"])
-                G[p + "b_o"] = _rows(dx2).sum(axis=0)
+                G[p + "w_o"] = _rows(dao).T @ _rows(c["om"])
+                G[p + "b_o"] = _rows(dao).sum(axis=0)
             dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"])
             dqkv = np.concatenate([_merge_heads(t) for t in (dq, dk, dv)], axis=-1)
             dh1 = dqkv @ P[p + "w_qkv"]
@@ -515,10 +570,11 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             dz, dg, db = layernorm_bwd(dx, c["ln2"], P[p + "ln2_g"])
             if on:
                 G[p + "ln2_g"], G[p + "ln2_b"] = dg, db
-            du = dz @ P[p + "w_fc2"]
+            dfo = dz * c["mask_f"]
+            du = dfo @ P[p + "w_fc2"]
             if on:
-                G[p + "w_fc2"] = _rows(dz).T @ _rows(c["u"])
-                G[p + "b_fc2"] = _rows(dz).sum(axis=0)
+                G[p + "w_fc2"] = _rows(dfo).T @ _rows(c["u"])
+                G[p + "b_fc2"] = _rows(dfo).sum(axis=0)
             da = gelu_bwd(du, c["a"])
             dx1 = dz + da @ P[p + "w_fc1"]
             if on:
@@ -527,10 +583,11 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             dy, dg, db = layernorm_bwd(dx1, c["ln1"], P[p + "ln1_g"])
             if on:
                 G[p + "ln1_g"], G[p + "ln1_b"] = dg, db
-            dom = dy @ P[p + "w_o"]
+            dao = dy * c["mask_a"]
+            dom = dao @ P[p + "w_o"]
             if on:
-                G[p + "w_o"] = _rows(dy).T @ _rows(c["om"])
-                G[p + "b_o"] = _rows(dy).sum(axis=0)
+                G[p + "w_o"] = _rows(dao).T @ _rows(c["om"])
+                G[p + "b_o"] = _rows(dao).sum(axis=0)
             dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"])
             dqkv = np.concatenate([_merge_heads(t) for t in (dq, dk, dv)], axis=-1)
             if on:
@@ -541,9 +598,10 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             dx = dy + dqkv @ P[p + "w_qkv"]
         else:
             cos, sin = cache["rope"]
-            ds = dx @ P[p + "w_down"]
+            dfo = dx * c["mask_f"]
+            ds = dfo @ P[p + "w_down"]
             if on:
-                G[p + "w_down"] = _rows(dx).T @ _rows(c["s"])
+                G[p + "w_down"] = _rows(dfo).T @ _rows(c["s"])
             dgate, dup = swiglu_bwd(ds, c["gate"], c["up"])
             dgu = np.concatenate([dgate, dup], axis=-1)
             dh2 = dgu @ P[p + "w_gu"]
@@ -553,9 +611,10 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             if on:
                 G[p + "rms2_g"] = dg
             dx2 = dx + dn
-            dom = dx2 @ P[p + "w_o"]
+            dao = dx2 * c["mask_a"]
+            dom = dao @ P[p + "w_o"]
             if on:
-                G[p + "w_o"] = _rows(dx2).T @ _rows(c["om"])
+                G[p + "w_o"] = _rows(dao).T @ _rows(c["om"])
             dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"])
             dq = rope_apply(dq, cos, sin, inverse=True)
             dk = rope_apply(dk, cos, sin, inverse=True)
@@ -571,6 +630,7 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             dx = dx2 + dn
     # ---- embedding ----
     if 0 in act:
+        dx = dx * cache["mask_emb"]
         if cfg.arch == 1:
             dx, dg, db = layernorm_bwd(dx, cache["emb_ln"], P["emb_ln_g"])
             G["emb_ln_g"], G["emb_ln_b"] = dg, db
@@ -680,7 +740,9 @@ class HiFTOracle:
         g = self.active_group()
         lr = self.current_lr()
         P = self.model_params()
-        loss, cache = forward(self.cfg, P, tokens, labels, lens)
+        pdrop = float(getattr(self.cfg, "dropout", 0.0))
+        drop = (pdrop, int(getattr(self.cfg, "dropout_seed", 0)), self.t) if pdrop > 0.0 else None
+        loss, cache = forward(self.cfg, P, tokens, labels, lens, drop)
         grads = backward(self.cfg, P, cache, active_units=self.groups[g])
         self.tau[g] += 1
         o = self.ocfg

@@ -96,6 +96,7 @@ def _prototypes():
         "hift_get_factored_state": (C.c_int, [vp, i32, i32, vp, sz]),
         "hift_adafactor_step": (C.c_int, [i64, i64, vp, vp, vp, vp, vp, f64, f64, f64, i64, vp]),
         "hift_init_synthetic": (C.c_int, [vp, C.c_uint64, f64]),
+        "hift_load_weights": (C.c_int, [vp, C.c_char_p, i32, C.POINTER(i32)]),
         "hift_save": (C.c_int, [vp, C.c_char_p]),
         "hift_load": (C.c_int, [vp, C.c_char_p]),
         "hift_profile_enable": (C.c_int, [vp, i32]),
@@ -363,6 +364,12 @@ class HiFT:
 
     def init_synthetic(self, seed: int, std: float = 0.02):
         _check(lib().hift_init_synthetic(self._h, seed, std), "hift_init_synthetic")
+
+    def load_weights(self, path: str, strict: bool = True) -> int:
+        """Sets parameters from a HIFTWTS1 file (see weights.py); returns the number of tensors set."""
+        n = C.c_int32()
+        _check(lib().hift_load_weights(self._h, path.encode(), 1 if strict else 0, C.byref(n)), "hift_load_weights")
+        return n.value
 
     def save(self, path: str):
         _check(lib().hift_save(self._h, path.encode()), "hift_save")

@@ -1473,6 +1473,50 @@ hift_status hift_tensor_info(const hift_ctx* c, int32_t ti, char* name, int32_t*
   return HIFT_OK;
 }
 
+hift_status hift_load_weights(hift_ctx* c, const char* path, int32_t strict, int32_t* n_loaded) {
+  if (!c || !path || c->pending_update) return HIFT_ERR_CFG;
+  FILE* f = fopen(path, "rb");
+  if (!f) return HIFT_ERR_INPUT;
+  char magic[8];
+  uint32_t n = 0;
+  bool ok = fread(magic, 8, 1, f) == 1 && memcmp(magic, "HIFTWTS1", 8) == 0 && fread(&n, 4, 1, f) == 1;
+  std::vector<char> seen(c->tens.size(), 0);
+  std::vector<float> vals;
+  std::vector<uint16_t> half;
+  int loaded = 0;
+  hift_status rc = HIFT_OK;
+  for (uint32_t r = 0; ok && r < n; ++r) {
+    char name[64];
+    uint32_t dtype = 0;
+    uint64_t rows = 0, cols = 0;
+    ok = fread(name, 64, 1, f) == 1 && fread(&dtype, 4, 1, f) == 1 && fread(&rows, 8, 1, f) == 1 && fread(&cols, 8, 1, f) == 1;
+    if (!ok) break;
+    name[63] = 0;
+    int ti = -1;
+    for (size_t i = 0; i < c->tens.size(); ++i) if (strcmp(c->tens[i].name, name) == 0) { ti = (int)i; break; }
+    // unknown tensor, a second record for the same tensor, a wrong shape or element type: refuse the file
+    if (ti < 0 || seen[ti] || dtype > 1 || rows != (uint64_t)c->tens[ti].rows || cols != (uint64_t)c->tens[ti].cols) { rc = HIFT_ERR_INPUT; break; }
+    const size_t cnt = c->tens[ti].numel;
+    vals.resize(cnt);
+    if (dtype == 1) {
+      half.resize(cnt);
+      ok = fread(half.data(), 2, cnt, f) == cnt;
+      for (size_t i = 0; ok && i < cnt; ++i) { const uint32_t u = (uint32_t)half[i] << 16; memcpy(&vals[i], &u, 4); }
+    } else ok = fread(vals.data(), 4, cnt, f) == cnt;
+    if (!ok) break;
+    rc = hift_set_param(c, ti, vals.data(), cnt);
+    if (rc != HIFT_OK) break;
+    seen[ti] = 1;
+    ++loaded;
+  }
+  fclose(f);
+  if (n_loaded) *n_loaded = loaded;
+  if (rc != HIFT_OK) return rc;
+  if (!ok) return HIFT_ERR_INPUT;
+  if (strict && loaded != (int)c->tens.size()) return HIFT_ERR_INPUT;
+  return HIFT_OK;
+}
+
 hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !src || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   sync_all(c);

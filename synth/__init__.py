@@ -52,6 +52,8 @@ class ModelCfg:
     dtype: int = DTYPE_BF16
     batch: int = 1
     seq: int = 1
+    dropout: float = 0.0               # probability of dropping an element at the residual-branch outputs and the embedding output
+    dropout_seed: int = 0
 
     @property
     def n_units(self) -> int:

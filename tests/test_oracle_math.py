@@ -37,14 +37,14 @@ def batch(cfg, seed=11, ignore=False):
 
 
 # ---------------------------------------------------------------- P1: finite differences
-def _fd_check(cfg, n_samples=5, h=1e-5, rel=2e-6, ignore=False, lens=None):
+def _fd_check(cfg, n_samples=5, h=1e-5, rel=2e-6, ignore=False, lens=None, drop=None):
     P = params64(cfg)
     tok, lab = batch(cfg, ignore=ignore)
     if lens is not None and lab.ndim == 2:                      # padded positions carry no label
         lab = lab.copy()
         for b, l in enumerate(lens):
             lab[b, l:] = -1
-    loss, cache = O.forward(cfg, P, tok, lab, lens)
+    loss, cache = O.forward(cfg, P, tok, lab, lens, drop)
     G = O.backward(cfg, P, cache, None)
     rng = np.random.default_rng(0)
     assert set(G.keys()) == set(P.keys())
@@ -59,9 +59,9 @@ def _fd_check(cfg, n_samples=5, h=1e-5, rel=2e-6, ignore=False, lens=None):
         for i in idx:
             old = flat[i]
             flat[i] = old + h
-            lp, _ = O.forward(cfg, P, tok, lab, lens)
+            lp, _ = O.forward(cfg, P, tok, lab, lens, drop)
             flat[i] = old - h
-            lm, _ = O.forward(cfg, P, tok, lab, lens)
+            lm, _ = O.forward(cfg, P, tok, lab, lens, drop)
             flat[i] = old
             fd = (lp - lm) / (2 * h)
             assert abs(fd - g.reshape(-1)[i]) <= rel * scale + 1e-9, (name, i, fd, g.reshape(-1)[i])
@@ -89,6 +89,63 @@ def test_fd_with_key_padding():
     _fd_check(mini(1), lens=[5, 8], n_samples=3)
     _fd_check(mini(0), lens=[3, 6], n_samples=3)
     _fd_check(mini(2), lens=[8, 1], n_samples=2)
+
+
+# ---------------------------------------------------------------- dropout from a counter-based generator
+def test_philox_known_answers():
+    """Philox4x32-10 against the known-answer vectors published with the generator (zero, all-ones and
+    digits-of-pi counters and keys)."""
+    kat = [((0, 0, 0, 0), (0, 0), (0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8)),
+           ((0xFFFFFFFF,) * 4, (0xFFFFFFFF,) * 2, (0x408F276D, 0x41C83B0E, 0xA20BC7C6, 0x6D5451FD)),
+           ((0x243F6A88, 0x85A308D3, 0x13198A2E, 0x03707344), (0xA4093822, 0x299F31D0), (0xD16CFE09, 0x94FDCCEB, 0x5001E420, 0x24126EA1))]
+    for ctr, key, want in kat:
+        got = O.philox4x32_10(*[np.array([c]) for c in ctr], key[0], key[1])
+        assert tuple(int(g[0]) for g in got) == want
+    # vectorised over counters = one call per counter
+    c0 = np.arange(5)
+    many = O.philox4x32_10(c0, np.zeros(5), np.full(5, 7), np.full(5, 9), 123, 456)
+    for i in range(5):
+        one = O.philox4x32_10(np.array([i]), np.array([0]), np.array([7]), np.array([9]), 123, 456)
+        assert [int(w[i]) for w in many] == [int(w[0]) for w in one]
+
+
+def test_dropout_mask_is_a_function_of_seed_step_site_element():
+    n, p = 200_000, 0.1
+    m = O.dropout_mask(n, p, seed=5, site=3, step=11)
+    assert set(np.unique(m).tolist()) == {0.0, 1.0 / (1.0 - p)}
+    dropped = float((m == 0.0).mean())
+    assert abs(dropped - p) < 4 * np.sqrt(p * (1 - p) / n)                # binomial, four sigma
+    assert abs(m.mean() - 1.0) < 0.01                                     # inverted dropout keeps the expectation
+    assert np.array_equal(m, O.dropout_mask(n, p, 5, 3, 11))
+    for other in (O.dropout_mask(n, p, 6, 3, 11), O.dropout_mask(n, p, 5, 4, 11), O.dropout_mask(n, p, 5, 3, 12)):
+        assert 0.15 < float((other != m).mean()) < 0.21                   # 2 p (1 - p) = 0.18 for independent masks
+    assert np.array_equal(O.dropout_mask(1000, p, 5, 3, 11), m[:1000])    # element i does not depend on the tensor's size
+    assert np.all(O.dropout_mask(64, 0.0, 5, 3, 11) == 1.0)
+    # the threshold is floor(p 2^32) on the element's word: word 0 of the first counter decides element 0
+    w = O.philox4x32_10(np.array([0]), np.array([0]), np.array([3]), np.array([11]), 5, 0)
+    assert (m[0] == 0.0) == (int(w[0][0]) < int(np.floor(p * 2 ** 32)))
+
+
+@pytest.mark.parametrize("arch", [0, 1, 2])
+def test_fd_with_dropout(arch):
+    """With the mask fixed by (seed, step), the loss is a smooth function of the parameters: finite differences
+    check the masked backward pass at all three sites (embedding, attention output, feed-forward output)."""
+    _fd_check(mini(arch), n_samples=3, drop=(0.25, 77, 3))
+
+
+def test_dropout_zero_is_the_plain_model_and_the_mask_reaches_every_site():
+    cfg = mini(0)
+    P = params64(cfg)
+    tok, lab = batch(cfg)
+    l0, _ = O.forward(cfg, P, tok, lab)
+    l1, _ = O.forward(cfg, P, tok, lab, None, (0.0, 1, 0))
+    assert l0 == l1
+    l2, c2 = O.forward(cfg, P, tok, lab, None, (0.2, 1, 0))
+    l3, _ = O.forward(cfg, P, tok, lab, None, (0.2, 1, 1))
+    assert l2 != l0 and l3 != l2                                          # another step, another mask
+    masks = [c2["mask_emb"]] + [c2["blocks"][i][k] for i in range(cfg.n_blocks) for k in ("mask_a", "mask_f")]
+    assert all(np.ndim(m) == 3 and 0.1 < float((m == 0).mean()) < 0.3 for m in masks)
+    assert len({m.tobytes() for m in masks}) == len(masks)                # every site draws its own
 
 
 # ---------------------------------------------------------------- key padding reduces to shorter sequences
