@@ -63,6 +63,15 @@ typedef struct {
   int32_t dtype;       /* 0: fp32 params+activations; 1: bf16 with fp32 master     */
   int32_t batch, seq;  /* fixed per context                                        */
   double  norm_eps, rope_base;
+  double  dropout;     /* probability p in [0, 1) of dropping an element at the outputs of each block's
+                          attention projection and feed-forward network (before the residual addition)
+                          and at the embedding output; kept values are scaled by 1/(1-p); 0 = none.
+                          The paper fine-tunes with the models' usual dropout without describing it;
+                          attention probabilities are not dropped here.                              */
+  uint64_t dropout_seed; /* the mask is Philox4x32-10(key = seed, counter = (element / 4, site, step)),
+                          word element % 4, kept iff word >= floor(p 2^32); site 0 = embedding,
+                          1 + 2 i = block i attention output, 2 + 2 i = its feed-forward output;
+                          step = t.  Reproducible from (seed, t) alone, also across checkpoints.     */
 } hift_model_cfg;
 
 /* Grouping and order (paper: Notation paragraph; Algorithm 1 "UpdateStrategy"). */

@@ -86,6 +86,8 @@ struct hift_ctx {
   int L = 0, d = 0, f = 0, fa = 0, H = 0, dh = 0, T = 0, B = 0, S = 0, V = 0, Vp = 0;
   int n_state = 2;
   bool mixed = true, offload = false;
+  bool drop_on = false;             // dropout at the residual-branch outputs and the embedding output
+  uint32_t drop_thr = 0; float drop_scale = 1.f;
   bool recompute = false;           // frozen blocks above the group keep only their input; see plan_slots
   bool keep_all = false;            // set while such a block is recomputed: its forward must store what the backward reads
   bool compact = false;             // paged master = low halves + carry bits beside the bf16 copy (see blob layout)
@@ -566,6 +568,42 @@ void act_bwd(hift_ctx* c, const void* a) {
   }
 }
 
+// ------------------------------------------------------------------ dropout sites
+DropArgs drop_args(const hift_ctx* c, int site) {
+  DropArgs a;
+  a.k0 = (uint32_t)c->m.dropout_seed; a.k1 = (uint32_t)(c->m.dropout_seed >> 32);
+  a.site = (uint32_t)site; a.step = (uint32_t)c->t; a.thr = c->drop_thr; a.scale = c->drop_scale;
+  return a;
+}
+// out = res + mask * t over the [T, d] stream
+void drop_add(hift_ctx* c, int site, const float* t, const float* res, float* out) {
+  const size_t n4 = (size_t)c->T * c->d / 4;
+  LAUNCH(HIFT_K_ELEMWISE, 48.0 * n4, dropout_add_kernel<<<grid_for(n4, 256), 256, 0, c->st>>>(t, res, out, n4, drop_args(c, site)));
+}
+void drop_inplace(hift_ctx* c, int site, float* x, void* x_a) {
+  const size_t n4 = (size_t)c->T * c->d / 4;
+  LAUNCH(HIFT_K_ELEMWISE, (32.0 + (x_a ? 4.0 * c->es : 0.0)) * n4,
+         if (c->mixed) dropout_inplace_kernel<bf16><<<grid_for(n4, 256), 256, 0, c->st>>>(x, (bf16*)x_a, n4, drop_args(c, site));
+         else dropout_inplace_kernel<float><<<grid_for(n4, 256), 256, 0, c->st>>>(x, (float*)x_a, n4, drop_args(c, site)));
+}
+// masked copies of the stream gradient dx: fp32 into the (idle in the backward pass) ping-pong buffer, operand into mop
+const float* drop_bwd(hift_ctx* c, int site, const float* dx, void* mop) {
+  const size_t n4 = (size_t)c->T * c->d / 4;
+  float* mf = c->pp[1];
+  LAUNCH(HIFT_K_ELEMWISE, (32.0 + 4.0 * c->es) * n4,
+         if (c->mixed) dropout_bwd_kernel<bf16><<<grid_for(n4, 256), 256, 0, c->st>>>(dx, mf, (bf16*)mop, n4, drop_args(c, site));
+         else dropout_bwd_kernel<float><<<grid_for(n4, 256), 256, 0, c->st>>>(dx, mf, (float*)mop, n4, drop_args(c, site)));
+  return mf;
+}
+// y = (x w^T + bias) [dropped] + res into the residual stream
+void linear_fwd_to_stream(hift_ctx* c, int site, int M, int N, int K, const void* x, const void* w, float* y, const void* bias,
+                          const float* res) {
+  if (!c->drop_on) { linear_fwd(c, M, N, K, x, K, w, y, N, bias, res, N, true); return; }
+  // the branch output in fp32 (dxb is idle in the forward pass), then the masked addition
+  linear_fwd(c, M, N, K, x, K, w, c->dxb, N, bias, nullptr, 0, true);
+  drop_add(c, site, c->dxb, res, y);
+}
+
 // ------------------------------------------------------------------ forward
 // x_r / x_a: the block input on the residual stream and (post-LN only) its operand copy.
 void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float* xo_r, char* xo_a) {
@@ -578,10 +616,10 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     float* z = (float*)s[S_Z];
     linear_fwd(c, T, 3 * d, d, x_a, d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
     attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
-    linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);             // y
+    linear_fwd_to_stream(c, 1 + 2 * i, T, d, d, s[S_O], c->P(b.w_o), x2, c->Pn(b.b_o), x_r);       // y
     norm_fwd(c, x2, b.n1_g, b.n1_b, s[S_H2], x1r, (float*)s[S_ST1]);                                 // x1
     linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
-    linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), z, d, c->Pn(b.b_fc2), x1r, d, true);           // z
+    linear_fwd_to_stream(c, 2 + 2 * i, T, d, f, s[S_U], c->P(b.w_fc2), z, c->Pn(b.b_fc2), x1r);     // z
     norm_fwd(c, z, b.n2_g, b.n2_b, xo_a, xo_r, (float*)s[S_ST2]);
     return;
   }
@@ -589,7 +627,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
   if (c->m.arch == 2) linear_fwd_qkv_rope(c, T, d, s[S_H1], c->P(b.w_qkv), s[S_QKV], c->Pn(b.b_qkv));
   else linear_fwd(c, T, 3 * d, d, s[S_H1], d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
   attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
-  linear_fwd(c, T, d, d, s[S_O], d, c->P(b.w_o), x2, d, c->Pn(b.b_o), x_r, d, true);
+  linear_fwd_to_stream(c, 1 + 2 * i, T, d, d, s[S_O], c->P(b.w_o), x2, c->Pn(b.b_o), x_r);
   norm_fwd(c, x2, b.n2_g, b.n2_b, s[S_H2], nullptr, (float*)s[S_ST2]);
   if (c->m.arch == 2) {
     // blocks below the active group keep nothing: their pre-activations live in the scratch slot and are never read
@@ -598,7 +636,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
   }
   // a block that is only being recomputed for its backward needs everything above, not its output
-  if (!c->keep_all) linear_fwd(c, T, d, f, s[S_U], f, c->P(b.w_fc2), xo_r, d, c->Pn(b.b_fc2), x2, d, true);
+  if (!c->keep_all) linear_fwd_to_stream(c, 2 + 2 * i, T, d, f, s[S_U], c->P(b.w_fc2), xo_r, c->Pn(b.b_fc2), x2);
 }
 
 // ------------------------------------------------------------------ backward
@@ -614,19 +652,25 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
     float* z = (float*)s[S_Z];
     if (on) { norm_bwd_params(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, b.n2_b); grad_done(c, b.n2_b); grad_done(c, b.n2_g); }
     norm_bwd_dx(c, c->dxa, true, z, (float*)s[S_ST2], b.n2_g, nullptr, c->dxb, c->dxb_a);          // dz
+    // through the dropout of the feed-forward output: the branch sees the masked gradient, the residual path dz itself
+    const float* gf = c->drop_on ? drop_bwd(c, 2 + 2 * i, c->dxb, c->dxb_a) : c->dxb;
     linear_dx_gelu_bwd(c, T, d, f, c->dxb_a, c->P(b.w_fc2), s[S_A]);                                // du -> da
-    if (on) { linear_dw(c, T, d, f, c->dxb_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxb, true, T, d, d, b.b_fc2); grad_done(c, b.b_fc2); grad_done(c, b.w_fc2); }
+    if (on) { linear_dw(c, T, d, f, c->dxb_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, gf, true, T, d, d, b.b_fc2); grad_done(c, b.b_fc2); grad_done(c, b.w_fc2); }
     linear_dx(c, T, f, d, c->dbig, f, c->P(b.w_fc1), c->dxa, d, c->dxb, d, true);                   // dx1
     if (on) { linear_dw(c, T, f, d, c->dbig, f, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, f, f, b.b_fc1); grad_done(c, b.b_fc1); grad_done(c, b.w_fc1); }
     if (on) { norm_bwd_params(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, b.n1_b); grad_done(c, b.n1_b); grad_done(c, b.n1_g); }
     norm_bwd_dx(c, c->dxa, true, x2, (float*)s[S_ST1], b.n1_g, nullptr, c->dxb, c->dxb_a);         // dy
+    const float* ga = c->drop_on ? drop_bwd(c, 1 + 2 * i, c->dxb, c->dxb_a) : c->dxb;
     linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                  // do
-    if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
+    if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, ga, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
     attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
     if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, x_a, d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); grad_done(c, b.b_qkv); grad_done(c, b.w_qkv); }
     if (need_dx) linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dxa, d, c->dxb, d, true);
     return;
   }
+  // through the dropout of the feed-forward output: the branch's GEMMs read the masked operand copy (dxa_a is not
+  // needed unmasked again: the residual path goes on in fp32), the bias gradient the masked fp32 copy
+  const float* gf = c->drop_on ? drop_bwd(c, 2 + 2 * i, c->dxa, c->dxa_a) : c->dxa;
   // SwiGLU on the tensor-core path: the dX product of the down projection stores d gate | d up directly
   bool act_done = false;
   if (c->m.arch == 2 && c->mixed) {
@@ -639,14 +683,15 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
   }
   if (!act_done && c->m.arch != 2) { linear_dx_gelu_bwd(c, T, d, f, c->dxa_a, c->P(b.w_fc2), s[S_A]); act_done = true; }
   if (!act_done) linear_dx(c, T, d, f, c->dxa_a, d, c->P(b.w_fc2), dact_in, f, nullptr, 0, false);  // ds
-  if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, c->dxa, true, T, d, d, b.b_fc2); grad_done(c, b.b_fc2); grad_done(c, b.w_fc2); }
+  if (on) { linear_dw(c, T, d, f, c->dxa_a, d, s[S_U], f, c->G(b.w_fc2)); bias_grad(c, gf, true, T, d, d, b.b_fc2); grad_done(c, b.b_fc2); grad_done(c, b.w_fc2); }
   if (!act_done) act_bwd(c, s[S_A]);                                                                // da in dbig [T,fa]
   linear_dx(c, T, fa, d, c->dbig, fa, c->P(b.w_fc1), c->dt1, d, nullptr, 0, false);                 // dh2
   if (on) { linear_dw(c, T, fa, d, c->dbig, fa, s[S_H2], d, c->G(b.w_fc1)); bias_grad(c, c->dbig, false, T, fa, fa, b.b_fc1); grad_done(c, b.b_fc1); grad_done(c, b.w_fc1); }
   if (on) { norm_bwd_params(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, b.n2_b); grad_done(c, b.n2_b); grad_done(c, b.n2_g); }
   norm_bwd_dx(c, c->dt1, false, x2, (float*)s[S_ST2], b.n2_g, c->dxa, c->dxb, c->dxb_a);            // dx2
+  const float* ga = c->drop_on ? drop_bwd(c, 1 + 2 * i, c->dxb, c->dxb_a) : c->dxb;
   linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                    // do
-  if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, c->dxb, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
+  if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, ga, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
   attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
   if (c->m.arch == 2) rope(c, c->dqkv, -1.0f);
   linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dt1, d, nullptr, 0, false);           // dh1
@@ -766,6 +811,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
            if (c->mixed) embed_fwd_kernel<bf16><<<T, norm_threads(d), 0, c->st>>>(tok, (const bf16*)c->P(c->t_tok), (const bf16*)c->Pn(c->t_pos), x0, S, d, V, bad);
            else embed_fwd_kernel<float><<<T, norm_threads(d), 0, c->st>>>(tok, (const float*)c->P(c->t_tok), (const float*)c->Pn(c->t_pos), x0, S, d, V, bad));
     if (m.arch == 1) norm_fwd(c, c->emb_e, c->t_eg, c->t_eb, chain_a[0], chain_r[0], c->st_e);
+    if (c->drop_on) drop_inplace(c, 0, chain_r[0], m.arch == 1 ? chain_a[0] : nullptr);
   }
   for (int i = 0; i < L; ++i) forward_block(c, i, chain_r[i], chain_a[i], chain_r[i + 1], chain_a[i + 1]);
   if (m.arch == 1) {
@@ -832,6 +878,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   }
   if (active(0)) {
     const float* src = c->dxa;
+    if (c->drop_on) drop_inplace(c, 0, c->dxa, nullptr);      // back through the dropout of the embedding output
     if (m.arch == 1) {
       norm_bwd_params(c, c->dxa, true, c->emb_e, c->st_e, c->t_eg, c->t_eb);
       grad_done(c, c->t_eb); grad_done(c, c->t_eg);
@@ -1100,6 +1147,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (!attention_head_ok(m->d_model / m->n_heads)) return HIFT_ERR_CFG;
   if (m->arch == 2 && (m->d_model / m->n_heads) % 16) return HIFT_ERR_CFG;   // RoPE rotates 8 pairs per thread
   if (m->dtype != 0 && m->dtype != 1) return HIFT_ERR_CFG;
+  if (!(m->dropout >= 0.0 && m->dropout < 1.0)) return HIFT_ERR_CFG;
   if (m->arch != 2 && m->max_pos < m->seq) return HIFT_ERR_CFG;
   if (m->arch == 1 && (m->n_classes < 2 || m->tie_head)) return HIFT_ERR_CFG;
   // the embedding-gradient kernel keeps one occurrence list of <= batch*seq ints in shared memory
@@ -1140,6 +1188,9 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
   c->compact = c->mixed && c->offload && !c->af;
   c->recompute = oc->recompute != 0;
+  c->drop_on = m->dropout > 0.0;
+  c->drop_thr = (uint32_t)floor(m->dropout * 4294967296.0);
+  c->drop_scale = (float)(1.0 / (1.0 - m->dropout));
   c->checked = g_checked_arena != 0;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));

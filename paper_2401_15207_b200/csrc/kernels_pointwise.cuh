@@ -500,6 +500,71 @@ __global__ void publish_scalars_kernel(const float* __restrict__ src, const int*
   __threadfence_system();
 }
 
+// ------------------------------------------------------------------ dropout
+// The mask is a pure function of (seed, step, site, element): Philox4x32-10 (Salmon et al., SC'11) with the
+// 64-bit seed as key and (element / 4 as two words, site, step) as counter gives four 32-bit words, one per
+// element of an aligned group of four; an element is kept iff its word >= floor(p 2^32), kept values are
+// scaled by 1 / (1 - p).  One thread draws one group of four.
+struct DropArgs { uint32_t k0, k1, site, step, thr; float scale; };
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+__device__ __forceinline__ float4 drop_mult4(size_t i4, const DropArgs& a) {
+  const uint4 w = philox4x32_10(make_uint4((uint32_t)i4, (uint32_t)(i4 >> 32), a.site, a.step), a.k0, a.k1);
+  return make_float4(w.x >= a.thr ? a.scale : 0.f, w.y >= a.thr ? a.scale : 0.f, w.z >= a.thr ? a.scale : 0.f,
+                     w.w >= a.thr ? a.scale : 0.f);
+}
+template <typename T>
+__device__ __forceinline__ void store4_op(T* p, float4 v);
+template <> __device__ __forceinline__ void store4_op<float>(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+template <> __device__ __forceinline__ void store4_op<bf16>(bf16* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 pk;
+  pk.x = *reinterpret_cast<uint32_t*>(&lo);
+  pk.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = pk;
+}
+// out = res + mask * t   (t: the branch output in fp32; out, res: the residual stream)
+__global__ void dropout_add_kernel(const float* __restrict__ t, const float* __restrict__ res, float* __restrict__ out,
+                                   size_t n4, DropArgs a) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 m = drop_mult4(i, a);
+    const float4 x = reinterpret_cast<const float4*>(t)[i], r = reinterpret_cast<const float4*>(res)[i];
+    reinterpret_cast<float4*>(out)[i] = make_float4(r.x + m.x * x.x, r.y + m.y * x.y, r.z + m.z * x.z, r.w + m.w * x.w);
+  }
+}
+// x *= mask in place on an fp32 tensor; the operand copy x_a (may be null) is rewritten from the masked value
+template <typename T>
+__global__ void dropout_inplace_kernel(float* __restrict__ x, T* __restrict__ x_a, size_t n4, DropArgs a) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 m = drop_mult4(i, a);
+    float4 v = reinterpret_cast<float4*>(x)[i];
+    v = make_float4(m.x * v.x, m.y * v.y, m.z * v.z, m.w * v.w);
+    reinterpret_cast<float4*>(x)[i] = v;
+    if (x_a != nullptr) store4_op<T>(x_a + 4 * i, v);
+  }
+}
+// backward through a dropout site: masked copies of the stream gradient dx, in fp32 (mf, may be null) and as the
+// GEMM operand (mop); dx itself is left alone (the residual path carries it on unmasked)
+template <typename T>
+__global__ void dropout_bwd_kernel(const float* __restrict__ dx, float* __restrict__ mf, T* __restrict__ mop, size_t n4, DropArgs a) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 m = drop_mult4(i, a);
+    float4 v = reinterpret_cast<const float4*>(dx)[i];
+    v = make_float4(m.x * v.x, m.y * v.y, m.z * v.z, m.w * v.w);
+    if (mf != nullptr) reinterpret_cast<float4*>(mf)[i] = v;
+    store4_op<T>(mop + 4 * i, v);
+  }
+}
+
 // The step's gate word, read by every optimizer kernel before its first store: non-zero when the
 // update must not happen.  src = the step's scalars ([0] loss, [2] bad-input flag); tc_error = the
 // tensor-core kernels' time-out flag (may be null).  Codes: the time-out code (1 .. 9), 100 bad input,

@@ -665,3 +665,53 @@ def test_checked_mode_no_kernel_writes_past_its_buffer(arch, dtype, big):
     plain = HiFT(cfg, synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3))
     assert plain.check_arena() == -1 and plain.arena_guard_count() == -1
     plain.close()
+
+
+@pytest.mark.parametrize("arch,dtype", [(0, synth.DTYPE_FP32), (1, synth.DTYPE_FP32), (2, synth.DTYPE_FP32),
+                                        (0, synth.DTYPE_BF16), (1, synth.DTYPE_BF16), (2, synth.DTYPE_BF16)])
+def test_dropout_masks_match_the_oracle(arch, dtype):
+    """Dropout at the three kinds of site (embedding output, attention output, feed-forward output) with masks
+    both sides draw from Philox4x32-10 keyed by (seed, step, site, element): a full cycle in lockstep, fp32 at
+    1e-5 (a single differing mask bit would move the loss far more) and bf16 at the bf16 tolerances."""
+    fp32 = dtype == synth.DTYPE_FP32
+    if fp32:
+        cfg = mini(arch, dtype, dropout=0.15, dropout_seed=0x1234_5678_9ABC)
+    else:
+        cfg = synth.ModelCfg(arch=arch, n_blocks=2, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=512, vocab=1001, max_pos=128,
+                             n_classes=2 if arch == 1 else 0, causal=0 if arch == 1 else 1, norm_eps=1e-6 if arch == 2 else 1e-5,
+                             dtype=dtype, batch=2, seq=128, init_std=0.05, dropout=0.1, dropout_seed=77)
+    oc = synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
+    lockstep(cfg, synth.GroupCfg(1), oc, cfg.n_units + 1, "zipf", FP32_LOSS if fp32 else BF16_LOSS, FP32_GRAD if fp32 else BF16_GRAD,
+             resync=True)
+
+
+def test_dropout_is_reproducible_and_recompute_redraws_the_same_masks():
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    base = dict(arch=2, n_blocks=3, d_model=256, n_heads=2, d_ffn=512, vocab=1001, norm_eps=1e-6, dtype=synth.DTYPE_BF16,
+                batch=2, seq=128, init_std=0.05)
+    p0 = synth.init_params(synth.ModelCfg(**base), 4)
+
+    def run(recompute=0, **kw):
+        cfg = synth.ModelCfg(**base, **kw)
+        h = HiFT(cfg, synth.GroupCfg(1), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=2, recompute=recompute))
+        try:
+            h.set_params(p0)
+            out = []
+            for t in range(h.num_groups()):
+                tok, lab = synth.lm_batch(cfg, 9, t)
+                out.append(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
+            return out, [h.get_param(n).copy() for n in h.tensor_names()]
+        finally:
+            h.close()
+
+    plain, _ = run()
+    zero, _ = run(dropout=0.0, dropout_seed=5)
+    a, pa = run(dropout=0.2, dropout_seed=5)
+    b, pb = run(dropout=0.2, dropout_seed=5)
+    c, _ = run(dropout=0.2, dropout_seed=6)
+    r, pr = run(recompute=1, dropout=0.2, dropout_seed=5)
+    assert plain == zero                      # p = 0 is the plain model, whatever the seed
+    assert a == b and all(np.array_equal(x, y) for x, y in zip(pa, pb))
+    assert a != plain and a != c              # the masks act, and follow the seed
+    assert a == r and all(np.array_equal(x, y) for x, y in zip(pa, pr))   # a recomputed block draws its masks again
