@@ -11,7 +11,8 @@ state in pinned host memory).  Prints ONE JSON line on rank 0.
 
 N > 1 runs N independent replicas by default (one process per GPU, no data-path collective: the
 step has no exchange inside it on one GPU); --parallel dp trains one model data-parallel with an
-all-reduce of the active group's gradient between the backward pass and the update.
+all-reduce of the active group's gradient, chunk by chunk behind the backward pass; --parallel zero1 also splits the
+optimizer state over the ranks.
 """
 from __future__ import annotations
 
@@ -323,7 +324,9 @@ def run_ours(args, cfg, gcfg, ocfg):
         torch.cuda.synchronize()
 
     ocfg = synth.OptCfg(**{**ocfg.__dict__, "prefetch_groups": args.prefetch, "offload_state": args.offload,
-                           "recompute": args.recompute})
+                           "recompute": args.recompute,
+                           "shard_rank": rank if args.parallel == "zero1" else 0,
+                           "shard_world": world if args.parallel == "zero1" else 0})
     peaks = measured_peaks()
     pcie = None
     if rank == 0 and world == 1 and ocfg.offload_state and not args.no_pcie:
@@ -341,8 +344,9 @@ def run_ours(args, cfg, gcfg, ocfg):
     groups = [h.group_units(g) for g in range(k)]
 
     step_dev, step_host = h.step, h.step_host
-    if args.parallel == "dp":
-        step_dev = lambda tok, lab: dist_util.data_parallel_step(h, tok, lab)
+    if args.parallel in ("dp", "zero1"):
+        dp_step = dist_util.data_parallel_step if args.parallel == "dp" else dist_util.data_parallel_step_sharded
+        step_dev = lambda tok, lab: dp_step(h, tok, lab)
         # end to end in this mode: pageable host batch -> device inside the timed call, then the same step
         step_host = lambda tok, lab: step_dev(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda())
 
@@ -482,7 +486,7 @@ def run_ours(args, cfg, gcfg, ocfg):
                        "groups_trained": trained, "ms_by_step": step_ms,
                        "optimizer": ["adamw", "adagrad", "sgdm", "sgd", "adafactor"][ocfg.kind],
                        "offload_state": ocfg.offload_state, "prefetch_groups": ocfg.prefetch_groups, "recompute": ocfg.recompute,
-                       "parallelism": (("dp%d" % world) if args.parallel == "dp" else "replicas") if world > 1 else "single",
+                       "parallelism": (("%s%d" % (args.parallel, world)) if args.parallel != "replicas" else "replicas") if world > 1 else "single",
                        "l2_policy": "inputs larger than L2 (weights + activations of a step exceed 126 MB)"},
             "cycle_mean_ms": round(float(np.mean(step_ms)), 3),
             "peak_hbm_gb": peak_hbm / 1e9, "pinned_host_gb": pinned / 1e9,
@@ -659,9 +663,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b", choices=sorted(WORKLOADS))
-    ap.add_argument("--parallel", default="replicas", choices=["replicas", "dp"],
-                    help="N > 1: independent replicas (default), or data parallel with an NCCL all-reduce of the "
-                         "active group's gradient between the backward pass and the update")
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "dp", "zero1"],
+                    help="N > 1: independent replicas (default); dp: one model, data parallel, the active group's gradient "
+                         "all-reduced chunk by chunk behind the backward pass; zero1: the same with the optimizer state (and its "
+                         "paging) split over the ranks: gradient pieces reduced to their owners, updated parameter pieces broadcast")
     ap.add_argument("--prefetch", type=int, default=3,
                     help="state slots beyond the first (0 paper order, 1 upload at step start, 2-3 uploads one or two steps ahead)")
     ap.add_argument("--no-pcie", action="store_true", help="leave out the pinned-memcpy ceiling measurement")

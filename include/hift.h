@@ -117,6 +117,17 @@ typedef struct {
   int32_t warmup_cycles;     /* W (sched 1; the warm-up the paper's hyper-parameter tables list, counted in
                                 cycles because the rate moves once per cycle): cycle c < W runs at
                                 lr*c/W, cycle c >= W at lr*max(0, (C-c)/(C-W)); 0 = none             */
+  int32_t shard_rank;        /* data-parallel ranks may split the optimizer state (ZeRO stage 1): with   */
+  int32_t shard_world;       /* shard_world = W > 1 this context holds fp32 master and state (device     */
+                             /* slots, pinned blobs, paging) only for piece shard_rank of every group's  */
+                             /* span (W contiguous pieces of whole 128-element lines, hift_shard_range), */
+                             /* and hift_step_end / hift_step_finish update only that piece; the caller  */
+                             /* reduces each piece of the gradient to its owner before, and broadcasts   */
+                             /* each piece of the updated parameters (hift_param_view) from its owner    */
+                             /* after.  The update is element-wise, so the pieces together are exactly   */
+                             /* the unsharded update.  0 or 1 = off.  Not with Adafactor (its statistics */
+                             /* span rows and columns); checkpoints are refused while sharded; outside   */
+                             /* its piece hift_get_param returns the model value, hift_get_state zeros.  */
   double lr, beta1, beta2, eps, weight_decay, momentum;
 } hift_opt_cfg;
 
@@ -209,6 +220,12 @@ hift_status hift_grad_chunk(const hift_ctx *ctx, int32_t i, size_t *offset, size
 hift_status hift_grad_chunk_wait(hift_ctx *ctx, int32_t i, void *cuda_stream);
 hift_status hift_gate_view(hift_ctx *ctx, int32_t **gate_dev);
 hift_status hift_set_grad_chunk_bytes(hift_ctx *ctx, size_t bytes);
+/* Sharded optimizer state (hift_opt_cfg.shard_world): the piece of group g's flat span that `rank` holds, as
+ * offset and length in elements of hift_grad_view / hift_param_view; and the parameters of the group trained
+ * by the step in flight (or the last one) as the forward pass reads them (bf16: elem_bytes 2, or fp32: 4),
+ * a device pointer to the group's whole span, for the exchange of the updated pieces. */
+hift_status hift_shard_range(const hift_ctx *ctx, int32_t g, int32_t rank, size_t *offset, size_t *n);
+hift_status hift_param_view(hift_ctx *ctx, void **param_dev, size_t *n, int32_t *elem_bytes);
 hift_status hift_step_finish(hift_ctx *ctx, float *loss_host);
 int32_t     hift_plan_grad_chunks(const size_t *offsets, const size_t *sizes, int32_t n_tensors, size_t span_elems,
                                   const int32_t *completion_order, int32_t n_completed, size_t min_chunk_elems,

@@ -51,6 +51,7 @@ class GroupCfgC(C.Structure):
 class OptCfgC(C.Structure):
     _fields_ = [("kind", C.c_int32), ("sched", C.c_int32), ("total_cycles", C.c_int32),
                 ("offload_state", C.c_int32), ("prefetch_groups", C.c_int32), ("recompute", C.c_int32), ("warmup_cycles", C.c_int32),
+                ("shard_rank", C.c_int32), ("shard_world", C.c_int32),
                 ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
                 ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double)]
 
@@ -76,6 +77,8 @@ def _prototypes():
         "hift_grad_chunk_wait": (C.c_int, [vp, i32, vp]),
         "hift_gate_view": (C.c_int, [vp, C.POINTER(vp)]),
         "hift_set_grad_chunk_bytes": (C.c_int, [vp, sz]),
+        "hift_shard_range": (C.c_int, [vp, i32, i32, C.POINTER(sz), C.POINTER(sz)]),
+        "hift_param_view": (C.c_int, [vp, C.POINTER(vp), C.POINTER(sz), C.POINTER(i32)]),
         "hift_step_finish": (C.c_int, [vp, pf]),
         "hift_plan_grad_chunks": (i32, [vp, vp, i32, sz, vp, i32, sz, vp, vp, vp, i32]),
         "hift_active_group": (i32, [vp]),
@@ -178,7 +181,8 @@ class HiFT:
         g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed,
                       C.cast(arr, C.POINTER(C.c_int32)) if sizes else None, len(sizes))
         o = OptCfgC(opt.kind, opt.sched, opt.total_cycles, opt.offload_state, opt.prefetch_groups,
-                    getattr(opt, "recompute", 0), getattr(opt, "warmup_cycles", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
+                    getattr(opt, "recompute", 0), getattr(opt, "warmup_cycles", 0),
+                    getattr(opt, "shard_rank", 0), getattr(opt, "shard_world", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
         self._h = C.c_void_p()
         self._stream = _stream_ptr() if stream is None else stream
         _check(lib().hift_create(C.byref(m), C.byref(g), C.byref(o), self._stream, C.byref(self._h)), "hift_create")
@@ -277,6 +281,26 @@ class HiFT:
         class _View:
             __cuda_array_interface__ = {"shape": (1,), "typestr": "<i4", "data": (ptr.value, False), "version": 3}
         return torch.as_tensor(_View(), device="cuda")
+
+    def shard_range(self, g: int, rank: int) -> Tuple[int, int]:
+        lo, n = C.c_size_t(), C.c_size_t()
+        _check(lib().hift_shard_range(self._h, g, rank, C.byref(lo), C.byref(n)), "hift_shard_range")
+        return lo.value, n.value
+
+    def param_view(self):
+        """Parameters of the group in flight (bf16 or fp32, as the forward pass reads them) as a torch CUDA tensor
+        sharing the library's memory."""
+        import torch
+        ptr, n, eb = C.c_void_p(), C.c_size_t(), C.c_int32()
+        _check(lib().hift_param_view(self._h, C.byref(ptr), C.byref(n), C.byref(eb)), "hift_param_view")
+        if eb.value == 4:
+            class _View:
+                __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<f4", "data": (ptr.value, False), "version": 3}
+            return torch.as_tensor(_View(), device="cuda")
+
+        class _View16:                                       # bf16 has no array-interface code: view the bits, reinterpret
+            __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<i2", "data": (ptr.value, False), "version": 3}
+        return torch.as_tensor(_View16(), device="cuda").view(torch.bfloat16)
 
     def set_grad_chunk_bytes(self, nbytes: int) -> None:
         _check(lib().hift_set_grad_chunk_bytes(self._h, nbytes), "hift_set_grad_chunk_bytes")

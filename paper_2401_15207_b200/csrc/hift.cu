@@ -51,6 +51,7 @@ struct TensorRec {
 struct GroupRec {
   int unit_lo, unit_hi;
   size_t off, numel;      // span in the flat parameter buffer (padded)
+  size_t own_lo, own_n;   // the part of the span whose master / state this rank holds (all of it unless sharded)
   int64_t tau;            // updates so far
   char* blob;             // pinned host: [master][state]; compact master: [state][low halves u16][carry bits]
   size_t blob_bytes;
@@ -86,6 +87,7 @@ struct hift_ctx {
   int L = 0, d = 0, f = 0, fa = 0, H = 0, dh = 0, T = 0, B = 0, S = 0, V = 0, Vp = 0;
   int n_state = 2;
   bool mixed = true, offload = false;
+  int shard_rank = 0, shard_world = 1;   // optimizer state sharded over data-parallel ranks (ZeRO stage 1)
   bool drop_on = false;             // dropout at the residual-branch outputs and the embedding output
   uint32_t drop_thr = 0; float drop_scale = 1.f;
   bool recompute = false;           // frozen blocks above the group keep only their input; see plan_slots
@@ -941,28 +943,31 @@ void enqueue_update(hift_ctx* c) {
   } else {
     float *mst, *s0, *s1;
     void* pbf = nullptr;
+    // the range of the group whose master / state this rank holds and updates (all of it unless sharded)
+    const size_t o0 = gr.off + gr.own_lo, on = gr.own_n;
+    const float* gsrc = c->grad + gr.own_lo;
     if (c->offload) {
       float* base = (float*)sr->mem;
-      if (c->compact) { mst = nullptr; s0 = base; s1 = base + gr.numel; pbf = c->params + gr.off * c->es; }
-      else if (c->mixed) { mst = base; s0 = base + gr.numel; s1 = base + 2 * gr.numel; pbf = c->params + gr.off * c->es; }
-      else { mst = (float*)c->params + gr.off; s0 = base; s1 = base + gr.numel; }
+      if (c->compact) { mst = nullptr; s0 = base; s1 = base + on; pbf = c->params + o0 * c->es; }
+      else if (c->mixed) { mst = base; s0 = base + on; s1 = base + 2 * on; pbf = c->params + o0 * c->es; }
+      else { mst = (float*)c->params + o0; s0 = base; s1 = base + on; }
     } else {
-      if (c->mixed) { mst = c->master_all + gr.off; pbf = c->params + gr.off * c->es; }
-      else mst = (float*)c->params + gr.off;
-      s0 = c->s0_all ? c->s0_all + gr.off : nullptr;
-      s1 = c->s1_all ? c->s1_all + gr.off : nullptr;
+      if (c->mixed) { mst = c->master_all + o0; pbf = c->params + o0 * c->es; }
+      else mst = (float*)c->params + o0;
+      s0 = c->s0_all ? c->s0_all + o0 : nullptr;
+      s1 = c->s1_all ? c->s1_all + o0 : nullptr;
     }
     const OptScalars hs = make_opt_scalars(c->oc.kind, lr, c->oc.beta1, c->oc.beta2, c->oc.eps,
                                            c->oc.weight_decay, c->oc.momentum, gr.tau);
     if (c->compact) {
       // read p, lo, carry, gradient, state; write p, lo, carry, state
-      const double opt_bytes = (double)gr.numel * (12.25 + 8.0 * c->n_state);
+      const double opt_bytes = (double)on * (12.25 + 8.0 * c->n_state);
       uint16_t* lo16 = (uint16_t*)((float*)sr->mem + gr.state_floats);
-      uint8_t* carry8 = (uint8_t*)(lo16 + gr.numel);
-      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, gr.numel, pbf, lo16, carry8, c->grad, s0, s1, hs, c->gate));
+      uint8_t* carry8 = (uint8_t*)(lo16 + on);
+      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, on, pbf, lo16, carry8, gsrc, s0, s1, hs, c->gate));
     } else {
-      const double opt_bytes = (double)gr.numel * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
-      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, gr.numel, pbf, mst, c->grad, s0, s1, hs, c->gate));
+      const double opt_bytes = (double)on * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
+      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, on, pbf, mst, gsrc, s0, s1, hs, c->gate));
     }
   }
 
@@ -1030,22 +1035,29 @@ int group_of_unit(const hift_ctx* c, int u) {
     if (u >= c->groups[g].unit_lo && u <= c->groups[g].unit_hi) return (int)g;
   return -1;
 }
-// where the fp32 master / state plane `plane` (0 master, 1 s0, 2 s1) of tensor ti lives
-float* plane_ptr(hift_ctx* c, int ti, int plane, bool* on_host) {
+// The part of tensor ti whose master / state this rank holds: tensor elements [t_lo, t_lo + n), found at
+// index p of the group's planes (everything unless the optimizer state is sharded over ranks).
+struct OwnPart { size_t t_lo, n, p; };
+OwnPart own_part(const hift_ctx* c, int ti) {
   const TensorRec& r = c->tens[ti];
-  const int g = group_of_unit(c, r.unit);
-  const GroupRec& gr = c->groups[g];
+  const GroupRec& gr = c->groups[group_of_unit(c, r.unit)];
+  const size_t a = r.off - gr.off, b = a + r.numel;
+  const size_t lo = std::max(a, gr.own_lo), hi = std::min(b, gr.own_lo + gr.own_n);
+  if (hi <= lo) return OwnPart{0, 0, 0};
+  return OwnPart{lo - a, hi - lo, lo - gr.own_lo};
+}
+// start of the fp32 master / state plane `plane` (0 master, 1 s0, 2 s1) of the group's held range
+float* plane_base(hift_ctx* c, const GroupRec& gr, int plane, bool* on_host) {
   *on_host = false;
-  if (plane == 0 && !c->mixed) return (float*)c->params + r.off;
+  if (plane == 0 && !c->mixed) return (float*)c->params + gr.off + gr.own_lo;
   if (c->offload) {
     *on_host = true;
     if (c->compact && plane == 0) return nullptr;        // not stored as floats: see master_read / master_write
     const int pl = (c->mixed && !c->compact) ? plane : plane - 1;
-    return (float*)gr.blob + (size_t)pl * gr.numel + (r.off - gr.off);
+    return (float*)gr.blob + (size_t)pl * gr.own_n;
   }
-  if (plane == 0) return c->master_all + r.off;
-  if (plane == 1) return c->s0_all ? c->s0_all + r.off : nullptr;
-  return c->s1_all ? c->s1_all + r.off : nullptr;
+  float* all = plane == 0 ? c->master_all : (plane == 1 ? c->s0_all : c->s1_all);
+  return all ? all + gr.off + gr.own_lo : nullptr;
 }
 
 // ---- compact master on the host side (same arithmetic as master_pack / master_unpack on the device)
@@ -1061,15 +1073,17 @@ inline void host_master_pack(uint32_t u, uint32_t& p, uint32_t& lo, uint32_t& ca
   }
 }
 uint16_t* blob_lo16(const hift_ctx* c, const GroupRec& gr) { (void)c; return (uint16_t*)((float*)gr.blob + gr.state_floats); }
-uint8_t* blob_carry8(const hift_ctx* c, const GroupRec& gr) { return (uint8_t*)(blob_lo16(c, gr) + gr.numel); }
-// fp32 master values of elements [o, o + n) of a group, rebuilt from the device's bf16 copy and the blob
+uint8_t* blob_carry8(const hift_ctx* c, const GroupRec& gr) { return (uint8_t*)(blob_lo16(c, gr) + gr.own_n); }
+// fp32 master values of elements [o, o + n) of a group (inside the range this rank holds), rebuilt from the
+// device's bf16 copy and the blob
 bool master_read(hift_ctx* c, const GroupRec& gr, size_t o, size_t n, float* dst) {
   std::vector<uint16_t> p(n);
   if (cudaMemcpy(p.data(), c->params + (gr.off + o) * c->es, n * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return false;
-  const uint16_t* lo = blob_lo16(c, gr) + o;
+  const size_t q = o - gr.own_lo;                      // index in the blob's planes
+  const uint16_t* lo = blob_lo16(c, gr) + q;
   const uint8_t* cr = blob_carry8(c, gr);
   for (size_t i = 0; i < n; ++i) {
-    const uint32_t carry = (cr[(o + i) >> 3] >> ((o + i) & 7)) & 1u;
+    const uint32_t carry = (cr[(q + i) >> 3] >> ((q + i) & 7)) & 1u;
     const uint32_t u = (((uint32_t)p[i] - carry) << 16) | lo[i];
     memcpy(dst + i, &u, 4);
   }
@@ -1077,15 +1091,16 @@ bool master_read(hift_ctx* c, const GroupRec& gr, size_t o, size_t n, float* dst
 }
 // the blob's share of new master values (the bf16 copy on the device is the caller's job)
 void master_write(hift_ctx* c, GroupRec& gr, size_t o, size_t n, const float* src) {
-  uint16_t* lo = blob_lo16(c, gr) + o;
+  const size_t q = o - gr.own_lo;
+  uint16_t* lo = blob_lo16(c, gr) + q;
   uint8_t* cr = blob_carry8(c, gr);
   for (size_t i = 0; i < n; ++i) {
     uint32_t u, p, l, carry;
     memcpy(&u, src + i, 4);
     host_master_pack(u, p, l, carry);
     lo[i] = (uint16_t)l;
-    uint8_t& byte = cr[(o + i) >> 3];
-    byte = (uint8_t)((byte & ~(1u << ((o + i) & 7))) | (carry << ((o + i) & 7)));
+    uint8_t& byte = cr[(q + i) >> 3];
+    byte = (uint8_t)((byte & ~(1u << ((q + i) & 7))) | (carry << ((q + i) & 7)));
   }
 }
 
@@ -1164,6 +1179,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   }
   if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
   if (oc->prefetch_groups < 0 || oc->prefetch_groups > kMaxSlots - 1) return HIFT_ERR_CFG;
+  if (oc->shard_world > 1 && (oc->shard_rank < 0 || oc->shard_rank >= oc->shard_world || oc->kind == 4)) return HIFT_ERR_CFG;
   if (oc->sched == 1 && (oc->total_cycles < 1 || oc->warmup_cycles < 0 || oc->warmup_cycles >= oc->total_cycles)) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
@@ -1196,10 +1212,16 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_work, 0, sizeof(c->prof_work));
   build_layout(c);
+  c->shard_world = oc->shard_world > 1 ? oc->shard_world : 1;
+  c->shard_rank = c->shard_world > 1 ? oc->shard_rank : 0;
   {
     size_t base = 0;
     for (auto& g : c->groups) {
-      g.state_floats = (size_t)c->n_state * g.numel;
+      // the contiguous piece of the group whose master and state this rank holds: pieces of whole 128-element lines
+      const size_t piece = align_up((g.numel + c->shard_world - 1) / c->shard_world, kAlignElems);
+      g.own_lo = std::min((size_t)c->shard_rank * piece, g.numel);
+      g.own_n = std::min(piece, g.numel - g.own_lo);
+      g.state_floats = (size_t)c->n_state * g.own_n;
       if (c->af) {
         size_t o = 0;
         for (int u = g.unit_lo; u <= g.unit_hi; ++u)
@@ -1237,8 +1259,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
 
   // ---- parameters, gradients, optimizer state
   auto blob_bytes_of = [&](const GroupRec& g) {
-    if (c->compact) return g.state_floats * sizeof(float) + g.numel * 2 + g.numel / 8;     // numel is a multiple of 128
-    return ((c->mixed ? g.numel : 0) + g.state_floats) * sizeof(float);
+    if (c->compact) return g.state_floats * sizeof(float) + g.own_n * 2 + g.own_n / 8;     // own_n is a multiple of 128
+    return ((c->mixed ? g.own_n : 0) + g.state_floats) * sizeof(float);
   };
   size_t slot_bytes_max = 0, af_total = 0;
   for (auto& g : c->groups) { slot_bytes_max = std::max(slot_bytes_max, blob_bytes_of(g)); af_total += c->af ? g.state_floats : 0; }
@@ -1252,7 +1274,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     }
     for (auto& g : c->groups) {
       g.blob_bytes = blob_bytes_of(g);
-      if (pinned_alloc((void**)&g.blob, g.blob_bytes, cudaHostAllocDefault) != cudaSuccess) {
+      if (pinned_alloc((void**)&g.blob, g.blob_bytes ? g.blob_bytes : 256, cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         g.blob = nullptr;
         return fail(HIFT_ERR_OOM_PINNED);
@@ -1397,6 +1419,22 @@ hift_status hift_grad_chunk_wait(hift_ctx* c, int32_t i, void* stream) {
 hift_status hift_gate_view(hift_ctx* c, int32_t** gate_dev) {
   if (!c || !gate_dev) return HIFT_ERR_CFG;
   *gate_dev = c->gate;
+  return HIFT_OK;
+}
+hift_status hift_shard_range(const hift_ctx* c, int32_t g, int32_t rank, size_t* lo, size_t* n) {
+  if (!c || g < 0 || g >= (int)c->groups.size() || rank < 0 || rank >= c->shard_world || !lo || !n) return HIFT_ERR_CFG;
+  const GroupRec& gr = c->groups[g];
+  const size_t piece = align_up((gr.numel + c->shard_world - 1) / c->shard_world, kAlignElems);
+  *lo = std::min((size_t)rank * piece, gr.numel);
+  *n = std::min(piece, gr.numel - *lo);
+  return HIFT_OK;
+}
+hift_status hift_param_view(hift_ctx* c, void** param_dev, size_t* n, int32_t* elem_bytes) {
+  if (!c || !param_dev || !n || c->last_group < 0) return HIFT_ERR_CFG;
+  const GroupRec& gr = c->groups[c->last_group];
+  *param_dev = c->params + gr.off * c->es;
+  *n = gr.numel;
+  if (elem_bytes) *elem_bytes = c->es;
   return HIFT_OK;
 }
 hift_status hift_set_grad_chunk_bytes(hift_ctx* c, size_t bytes) {
@@ -1572,32 +1610,42 @@ hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) 
   if (ti < 0 || ti >= (int)c->tens.size() || !src || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   sync_all(c);
   invalidate_slots(c);
-  bool on_host;
-  float* mp = plane_ptr(c, ti, 0, &on_host);
+  GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
+  const OwnPart op = own_part(c, ti);
   // every copy goes through the context's stream, so the cast below is ordered after its input
-  if (c->compact) {
-    GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
-    master_write(c, gr, c->tens[ti].off - gr.off, n, src);
-  } else if (on_host) memcpy(mp, src, n * sizeof(float));
-  else if (cudaMemcpyAsync(mp, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
+  if (op.n) {
+    bool on_host;
+    float* base = plane_base(c, gr, 0, &on_host);
+    if (c->compact) master_write(c, gr, (c->tens[ti].off - gr.off) + op.t_lo, op.n, src + op.t_lo);
+    else if (on_host) memcpy(base + op.p, src + op.t_lo, op.n * sizeof(float));
+    else if (cudaMemcpyAsync(base + op.p, src + op.t_lo, op.n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
+  }
   if (c->mixed) {
     // stage the fp32 values in the gradient buffer (any tensor fits in the largest group)
     if (cudaMemcpyAsync(c->grad, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
     cast_from_f32_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>(c->grad, (bf16*)c->P(ti), n);
+  } else if (op.n != n) {
+    // fp32 parameters are their own master: the part another rank updates is still this rank's model value
+    if (cudaMemcpyAsync(c->P(ti), src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
   }
   return cudaStreamSynchronize(c->st) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
 hift_status hift_get_param(hift_ctx* c, int32_t ti, float* dst, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   sync_all(c);
-  bool on_host;
-  float* mp = plane_ptr(c, ti, 0, &on_host);
-  if (c->compact) {
-    const GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
-    return master_read(c, gr, c->tens[ti].off - gr.off, n, dst) ? HIFT_OK : HIFT_ERR_CUDA;
+  if (!c->mixed) return cudaMemcpy(dst, c->P(ti), n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+  const GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
+  const OwnPart op = own_part(c, ti);
+  if (op.n != n) {                  // sharded state: outside this rank's part only the model value is known
+    const hift_status s = hift_get_model_param(c, ti, dst, n);
+    if (s != HIFT_OK) return s;
   }
-  if (on_host) memcpy(dst, mp, n * sizeof(float));
-  else if (cudaMemcpy(dst, mp, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
+  if (!op.n) return HIFT_OK;
+  if (c->compact) return master_read(c, gr, (c->tens[ti].off - gr.off) + op.t_lo, op.n, dst + op.t_lo) ? HIFT_OK : HIFT_ERR_CUDA;
+  bool on_host;
+  float* base = plane_base(c, const_cast<GroupRec&>(gr), 0, &on_host);
+  if (on_host) memcpy(dst + op.t_lo, base + op.p, op.n * sizeof(float));
+  else if (cudaMemcpy(dst + op.t_lo, base + op.p, op.n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
   return HIFT_OK;
 }
 hift_status hift_get_model_param(hift_ctx* c, int32_t ti, float* dst, size_t n) {
@@ -1616,11 +1664,15 @@ hift_status hift_get_state(hift_ctx* c, int32_t ti, int32_t which, float* dst, s
   if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   if (which < 0 || which >= c->n_state) return HIFT_ERR_CFG;
   sync_all(c);
+  const GroupRec& gr = c->groups[group_of_unit(c, c->tens[ti].unit)];
+  const OwnPart op = own_part(c, ti);
+  if (op.n != n) memset(dst, 0, n * sizeof(float));      // sharded state: zeros outside this rank's part
+  if (!op.n) return HIFT_OK;
   bool on_host;
-  float* sp = plane_ptr(c, ti, 1 + which, &on_host);
-  if (!sp) return HIFT_ERR_CFG;
-  if (on_host) memcpy(dst, sp, n * sizeof(float));
-  else if (cudaMemcpy(dst, sp, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
+  float* base = plane_base(c, gr, 1 + which, &on_host);
+  if (!base) return HIFT_ERR_CFG;
+  if (on_host) memcpy(dst + op.t_lo, base + op.p, op.n * sizeof(float));
+  else if (cudaMemcpy(dst + op.t_lo, base + op.p, op.n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
   return HIFT_OK;
 }
 hift_status hift_get_factored_state(hift_ctx* c, int32_t ti, int32_t which, float* dst, size_t n) {
@@ -1667,7 +1719,8 @@ hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
     }
     if (c->compact) {
       uint16_t* lo16 = (uint16_t*)((float*)c->slot[0].mem + gr.state_floats);
-      master_pack_kernel<<<grid_for(gr.numel / 8, 256), 256, 0, c->st>>>(c->grad, lo16, (uint8_t*)(lo16 + gr.numel), gr.numel / 8);
+      if (gr.own_n)
+        master_pack_kernel<<<grid_for(gr.own_n / 8, 256), 256, 0, c->st>>>(c->grad + gr.own_lo, lo16, (uint8_t*)(lo16 + gr.own_n), gr.own_n / 8);
     }
     if (c->offload) {
       cudaMemcpyAsync(gr.blob, c->slot[0].mem, gr.blob_bytes, cudaMemcpyDeviceToHost, c->st);
@@ -1709,7 +1762,7 @@ void group_locations(hift_ctx* c, GroupRec& gr, float** master, bool* master_hos
 }  // namespace
 
 hift_status hift_save(hift_ctx* c, const char* path) {
-  if (!c || !path || c->pending_update) return HIFT_ERR_CFG;
+  if (!c || !path || c->pending_update || c->shard_world > 1) return HIFT_ERR_CFG;
   sync_all(c);
   FILE* f = fopen(path, "wb");
   if (!f) return HIFT_ERR_INPUT;
@@ -1750,7 +1803,7 @@ hift_status hift_save(hift_ctx* c, const char* path) {
 }
 
 hift_status hift_load(hift_ctx* c, const char* path) {
-  if (!c || !path || c->pending_update) return HIFT_ERR_CFG;
+  if (!c || !path || c->pending_update || c->shard_world > 1) return HIFT_ERR_CFG;
   sync_all(c);
   FILE* f = fopen(path, "rb");
   if (!f) return HIFT_ERR_INPUT;

@@ -78,6 +78,56 @@ def allreduce_chunks_mean_(tensor, chunks, wait_for_chunk=None, flag=None):
     return tensor
 
 
+def reduce_pieces_mean_(grad, pieces, rank):
+    """Sharded optimizer state: piece r of the gradient (pieces[r] = (offset, length)) is summed over the ranks
+    onto rank r, which alone will use it; this rank's piece is then scaled to the mean.  The volume of a
+    reduce-scatter, with pieces that need not have equal lengths."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return grad
+    works = [dist.reduce(grad[lo:lo + n], dst=r, op=dist.ReduceOp.SUM, async_op=True) for r, (lo, n) in enumerate(pieces) if n]
+    for w in works:
+        w.wait()
+    lo, n = pieces[rank]
+    grad[lo:lo + n].mul_(1.0 / dist.get_world_size())
+    return grad
+
+
+def broadcast_pieces_(params, pieces):
+    """After the sharded update: every rank's piece of the group's parameters goes to all the others
+    (an all-gather with pieces of unequal length)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return params
+    works = [dist.broadcast(params[lo:lo + n], src=r, async_op=True) for r, (lo, n) in enumerate(pieces) if n]
+    for w in works:
+        w.wait()
+    return params
+
+
+def data_parallel_step_sharded(h, tokens, labels) -> float:
+    """The data-parallel step with the optimizer state split over the ranks (contexts created with
+    shard_rank / shard_world): forward + truncated backward, each piece of the group's gradient reduced to the
+    rank that holds its master and state, the update of that piece, and the updated pieces of the parameters
+    sent to everyone.  State memory and state paging per rank shrink by the number of ranks; the parameters
+    every rank ends up with are bit for bit those of the unsharded step, because the update is element-wise."""
+    import torch
+    import torch.distributed as dist
+    rank, world_size = world()
+    g = h.active_group()
+    pieces = [h.shard_range(g, r) for r in range(world_size)]
+    h.step_begin_async(tokens, labels)
+    grad, gate = h.grad_view(), h.gate_view()
+    for i in range(len(h.grad_chunks())):
+        h.grad_chunk_wait(i, torch.cuda.current_stream().cuda_stream)
+    reduce_pieces_mean_(grad, pieces, rank)
+    if world_size > 1:
+        dist.all_reduce(gate, op=dist.ReduceOp.MAX)
+    loss = h.step_finish()
+    broadcast_pieces_(h.param_view(), pieces)
+    return loss
+
+
 _comm_streams = {}
 
 

@@ -94,6 +94,8 @@ class OptCfg:
     prefetch_groups: int = 0
     warmup_cycles: int = 0
     recompute: int = 0
+    shard_rank: int = 0                # optimizer state sharded over data-parallel ranks (0 / 1 = off)
+    shard_world: int = 0
 
 
 # --------------------------------------------------------------------------

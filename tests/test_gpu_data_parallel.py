@@ -187,3 +187,72 @@ def test_two_emulated_ranks_exchange_chunk_by_chunk_and_share_the_gate():
         assert np.array_equal(r0.get_param(n), r1.get_param(n)), n
     r0.close()
     r1.close()
+
+
+@pytest.mark.parametrize("kind,dtype,offload", [(0, synth.DTYPE_BF16, 1), (0, synth.DTYPE_BF16, 0), (2, synth.DTYPE_FP32, 1)])
+def test_sharded_optimizer_state_gives_the_unsharded_parameters(kind, dtype, offload):
+    """Two emulated ranks that split every group's master and state in two pieces (one after the other on one
+    GPU; the reduce to the owner and the broadcast of the updated pieces done by hand) against two ranks that
+    each hold everything: identical model parameters after every step, master and state equal on the piece a
+    rank holds, and about half the pinned state per rank."""
+    import torch
+    from paper_2401_15207_b200 import HiFT, HiftError
+    half = synth.ModelCfg(arch=2, n_blocks=2, d_model=256, n_heads=2, d_ffn=512, vocab=1000, norm_eps=1e-6,
+                          dtype=dtype, batch=2, seq=128, init_std=0.05)
+    full = half.scaled(batch=4)
+    gc = synth.GroupCfg(1)
+    mk = lambda r, w: synth.OptCfg(kind=kind, lr=1e-3, momentum=0.9, weight_decay=0.01, offload_state=offload,
+                                   prefetch_groups=2 if offload else 0, shard_rank=r, shard_world=w)
+    p0 = synth.init_params(half, 5)
+    whole = [HiFT(half, gc, mk(0, 0)) for _ in range(2)]
+    shard = [HiFT(half, gc, mk(r, 2)) for r in range(2)]
+    try:
+        for h in whole + shard:
+            h.set_params(p0)
+        if offload:
+            assert shard[0].pinned_host_bytes() + shard[1].pinned_host_bytes() <= 1.02 * whole[0].pinned_host_bytes()
+        n_state = {0: 2, 2: 1}[kind]
+        for t in range(2 * whole[0].num_groups()):
+            tok, lab = synth.lm_batch(full, 8, t)
+            parts = [(torch.from_numpy(tok[:2].copy()).cuda(), torch.from_numpy(lab[:2].copy()).cuda()),
+                     (torch.from_numpy(tok[2:].copy()).cuda(), torch.from_numpy(lab[2:].copy()).cuda())]
+            g = whole[0].active_group()
+            for grp in (whole, shard):
+                for h, (tt, ll) in zip(grp, parts):
+                    h.step_begin(tt, ll)
+                g0, g1 = grp[0].grad_view(), grp[1].grad_view()
+                avg = (g0 + g1) * 0.5
+                g0.copy_(avg)
+                g1.copy_(avg)
+                torch.cuda.synchronize()
+                for h in grp:
+                    h.step_end()
+            # the broadcast of the updated pieces: rank r's piece of the group's parameters goes to the other rank
+            v0, v1 = shard[0].param_view(), shard[1].param_view()
+            for r, (src, dst) in enumerate(((v0, v1), (v1, v0))):
+                lo, n = shard[r].shard_range(g, r)
+                assert (lo, n) == shard[1 - r].shard_range(g, r)
+                dst[lo:lo + n].copy_(src[lo:lo + n])
+            torch.cuda.synchronize()
+            for name in whole[0].tensor_names():
+                ref = whole[0].get_model_param(name)
+                for h in shard:
+                    assert np.array_equal(h.get_model_param(name), ref), (t, name)
+        # master and state on the piece a rank holds; the two pieces tile every tensor
+        for name in whole[0].tensor_names():
+            ref_m = whole[0].get_param(name).reshape(-1)
+            model = whole[0].get_model_param(name).reshape(-1)
+            ms = [h.get_param(name).reshape(-1) for h in shard]
+            mine = [m != model for m in ms]                  # where a rank returned something other than the model value
+            assert np.array_equal(np.where(mine[0], ms[0], ms[1]), np.where(mine[0] | mine[1], ref_m, model)), name
+            for w in range(n_state):
+                ref_s = whole[0].get_state(name, w).reshape(-1)
+                got = sum(h.get_state(name, w).reshape(-1) for h in shard)      # zeros outside a rank's piece
+                assert np.array_equal(got, ref_s), (name, w)
+        with pytest.raises(HiftError):
+            shard[0].save("/tmp/never_written.ckpt")                           # checkpoints are refused while sharded
+    finally:
+        for h in whole + shard:
+            h.close()
+    with pytest.raises(HiftError):
+        HiFT(half, gc, synth.OptCfg(kind=4, lr=1e-2, eps=1e-30, shard_rank=0, shard_world=2))    # not with Adafactor

@@ -116,3 +116,35 @@ def test_two_ranks_chunked_exchange_equals_one_all_reduce(tmp_path):
     mp.spawn(_chunk_worker, args=(2, _free_port(), out), nprocs=2, join=True)
     r = torch.load(out)
     assert r["ok"] and r["chunks"] >= 3
+
+
+def _pieces_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        n = 1000
+        pieces = [(0, 640), (640, 360)]                          # whole 128-element lines first, the rest last
+        g = torch.Generator().manual_seed(7 + rank)
+        grad = torch.randn(n, generator=g)
+        mean = grad.clone()
+        dist_util.allreduce_mean_(mean)
+        dist_util.reduce_pieces_mean_(grad, pieces, rank)
+        lo, cnt = pieces[rank]
+        assert torch.allclose(grad[lo:lo + cnt], mean[lo:lo + cnt], rtol=0, atol=1e-7)   # the owner holds the mean of its piece
+        # each rank "updates" its own piece of the parameters, then the pieces travel
+        params = torch.zeros(n)
+        params[lo:lo + cnt] = float(rank + 1)
+        dist_util.broadcast_pieces_(params, pieces)
+        assert torch.equal(params[:640], torch.full((640,), 1.0)) and torch.equal(params[640:], torch.full((360,), 2.0))
+        dist.barrier()
+        if rank == 0:
+            torch.save({"ok": True}, out)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_piecewise_reduce_and_broadcast(tmp_path):
+    out = str(tmp_path / "p0.pt")
+    mp.spawn(_pieces_worker, args=(2, _free_port(), out), nprocs=2, join=True)
+    assert torch.load(out)["ok"]
