@@ -262,7 +262,8 @@ def standalone_kernels(cfg, peaks, launches=20):
             fn(i % nsets)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
-        e0.record()
+        torch.cuda._sleep(2_000_000)                 # about a millisecond: the launches below queue up behind it, so the
+        e0.record()                                  # host's per-call cost stays out of the measurement
         for i in range(launches):
             fn(i % nsets)
         e1.record()
@@ -274,7 +275,7 @@ def standalone_kernels(cfg, peaks, launches=20):
         pk = peaks["bf16_tflops_sustained"] if tensor else peaks["hbm_gbs"]
         out[name] = {"avg_us": round(us, 2), "achieved": round(ach, 1), "unit": "TFLOP/s" if tensor else "GB/s",
                      "bound": "tensor" if tensor else "hbm", "frac": round(ach / pk, 3), "what": note,
-                     "method": f"standalone loop, {launches} launches, CUDA events, rotating buffers"}
+                     "method": f"standalone loop, {launches} queued launches, CUDA events, rotating buffers"}
 
     # norms: fp32 stream in, bf16 operand out (forward); bf16 dy + fp32 x + fp32 add in, fp32 + bf16 dx out (backward)
     nsets = max(2, int(200e6 // (T * d * 6)) + 1)
@@ -511,6 +512,73 @@ def run_ours(args, cfg, gcfg, ocfg):
         dist.destroy_process_group()
 
 
+def linear_shapes(cfg):
+    """(name, form, M, N, K, launches per step in which one block group is active) of the plain linear-layer products of
+    one transformer block at the workload's sizes, in hift_k_linear's convention (form 0 forward y[M,N], 1 dX [M,K] from
+    dy[M,N], 2 dW [N,K])."""
+    T, d, f = cfg.tokens_per_step, cfg.d_model, cfg.d_ffn
+    fa = 2 * f if cfg.arch == synth.ARCH_LLAMA else f
+    layers = [("qkv", 3 * d, d), ("attn_out", d, d), ("ffn_up", fa, d), ("ffn_down", d, f)]
+    out = []
+    for name, n, k in layers:
+        for form, tag in ((0, "fwd"), (1, "dx"), (2, "dw")):
+            out.append((f"{name}_{tag}", form, T, n, k))
+    return out
+
+
+def run_micro(args, cfg):
+    """A few launches of single kernels at the workload's shapes through the single-kernel entry points: what an
+    `ncu` capture of one kernel is taken on (a few GB on the device, a handful of launches), and a quick timing of
+    each shape on its own (CUDA events over `--launches` back-to-back launches behind a queue-filling spin)."""
+    import torch
+    from paper_2401_15207_b200 import binding as B
+    peaks = measured_peaks()
+    bf = torch.bfloat16
+    rows = []
+    n_l = args.launches
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(2_000_000)                    # launches queue up behind it: the host is out of the timing
+        e0.record()
+        for _ in range(n_l):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / n_l
+
+    if args.micro == "gemm":
+        for name, form, M, N, K in linear_shapes(cfg):
+            if args.only and args.only not in name:
+                continue
+            x = torch.randn(M, K, device="cuda").to(bf)
+            w = (torch.randn(N, K, device="cuda") * 0.02).to(bf)
+            dy = torch.randn(M, N, device="cuda").to(bf)
+            if form == 0:
+                out = torch.empty(M, N, device="cuda", dtype=bf)
+                fn = lambda: B.k_linear(0, 1, M, N, K, x, w, out, path=2)
+            elif form == 1:
+                out = torch.empty(M, K, device="cuda", dtype=bf)
+                fn = lambda: B.k_linear(1, 1, M, N, K, dy, w, out, path=2)
+            else:
+                out = torch.empty(N, K, device="cuda", dtype=torch.float32)
+                fn = lambda: B.k_linear(2, 1, M, N, K, dy, x, out, path=2)
+            us = timed(fn)
+            fl = 2.0 * M * N * K
+            algo = 2.0 * (M * K + N * K + M * N) if form != 2 else 2.0 * (M * N + M * K) + 4.0 * N * K
+            rows.append({"shape": name, "form": form, "M": M, "N": N, "K": K, "us": round(us, 2),
+                         "tflops": round(fl / (us * 1e-6) / 1e12, 1),
+                         "frac_of_burst_peak": round(fl / (us * 1e-6) / 1e12 / peaks["bf16_tflops"], 3),
+                         "algorithmic_bytes": int(algo)})
+            del x, w, dy, out
+    else:
+        rows = [dict(kernel=k, **v) for k, v in standalone_kernels(cfg, peaks, launches=n_l).items()]
+    print(json.dumps({"micro": args.micro, "workload": args.workload, "launches": n_l,
+                      "peak_tflops_burst": peaks["bf16_tflops"], "rows": rows}))
+
+
 def run_full_param_reference(cfg, ocfg, steps=4, warmup=3):
     """The same model trained the ordinary way: one group holding every unit (k = 1), all master
     weights and optimizer state resident on the GPU, full backward.  Returns tokens/s and peak HBM."""
@@ -683,6 +751,10 @@ def main():
                     help="leave out the k = 1 full-parameter step of the same model (needs ~132 GB at the 7B shape)")
     ap.add_argument("--sweep", default=None, choices=["optimizer", "depth"],
                     help="kernel sweeps instead of the step benchmark")
+    ap.add_argument("--micro", default=None, choices=["gemm", "kernels"],
+                    help="single kernels at the workload's shapes, a few launches each (small enough for an ncu capture)")
+    ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--only", default=None, help="--micro gemm: only shapes whose name contains this")
     ap.add_argument("--steps-ref", type=int, default=2)
     ap.add_argument("--warmup-ref", type=int, default=0)
     args = ap.parse_args()
@@ -693,6 +765,8 @@ def main():
     if args.sweep == "depth":
         return run_sweep_depth(args)
     cfg, gcfg, ocfg = WORKLOADS[args.workload]()
+    if args.micro:
+        return run_micro(args, cfg)
     if args.full_param:
         gcfg = synth.GroupCfg(layers_per_group=cfg.n_units, split_emb_head=0, order=synth.ORDER_BOTTOM2UP)
         args.offload, args.prefetch = 0, 0
