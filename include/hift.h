@@ -86,6 +86,16 @@ typedef struct {
                                 this is the same fixed partition with the chunk lengths chosen by the
                                 caller); read during hift_create only, not kept            */
   int32_t n_group_sizes;
+  int32_t literal_queue;     /* 1: Algorithm 1, steps c-d, taken literally: a queue of the n units in the strategy's
+                                order (random: shuffled once); every step pops m units from its head and appends
+                                them to its tail.  When m divides n this is the fixed partition above.  When it does
+                                not, the sets drift: a set can wrap around (top and bottom units together) and a unit
+                                is trained ceil- or floor-many times per pass; every unit then keeps its own master,
+                                state and update count, a step trains a SET of units (hift_num_sets() distinct sets,
+                                set id = step mod that; hift_active_group() returns the set id and hift_set_units()
+                                its units), and the learning rate still moves every k = floor(n/m) + 1 steps
+                                (hift_num_groups()).  State paging uses one slot in this mode (sets share units).
+                                Not with group_sizes, split_emb_head or sharded state.                            */
 } hift_group_cfg;
 
 /* Optimizer P and schedule eta_t of Algorithm 1's "Require" list; state residency
@@ -232,10 +242,14 @@ int32_t     hift_plan_grad_chunks(const size_t *offsets, const size_t *sizes, in
                                   size_t *chunk_off, size_t *chunk_n, int32_t *chunk_after, int32_t max_chunks);
 
 int32_t hift_active_group(const hift_ctx *ctx);   /* group the NEXT hift_step trains */
-int32_t hift_num_groups(const hift_ctx *ctx);     /* k                               */
+int32_t hift_num_groups(const hift_ctx *ctx);     /* k: steps per learning-rate cycle */
+int32_t hift_num_sets(const hift_ctx *ctx);       /* distinct sets of units the schedule trains (= k unless the queue drifts) */
+/* Units of set `set_id` (ascending) into units_out[0 .. cap); *n_units receives their number. */
+hift_status hift_set_units(const hift_ctx *ctx, int32_t set_id, int32_t *units_out, int32_t cap, int32_t *n_units);
 int64_t hift_step_count(const hift_ctx *ctx);     /* t, steps taken so far           */
 double  hift_current_lr(const hift_ctx *ctx);     /* lr the NEXT step will use       */
-/* Units of group g: writes the first and last unit id (inclusive). */
+/* Units of group (set) g: writes the first and last unit id (inclusive); HIFT_ERR_CFG for a set of the drifting
+ * queue that is not an interval of units (use hift_set_units). */
 hift_status hift_group_units(const hift_ctx *ctx, int32_t g, int32_t *unit_lo, int32_t *unit_hi);
 /* Force the group trained by the next steps (depth sweeps); -1 restores the schedule. */
 hift_status hift_force_group(hift_ctx *ctx, int32_t g);

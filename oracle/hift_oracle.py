@@ -125,11 +125,11 @@ def group_order(k: int, order: int, seed: int = 0) -> List[int]:
     raise ValueError("order")
 
 
-def queue_walk(n_units: int, m: int, order: int, steps: int) -> List[List[int]]:
+def queue_walk(n_units: int, m: int, order: int, steps: int, seed: int = 0) -> List[List[int]]:
     """Literal queue of Algorithm 1 (steps c, d): Q holds unit ids in strategy
-    order; each step removes m ids from the head and appends them to the tail.
-    Only bottom2up/top2down (the deterministic strategies) are meaningful here."""
-    q = list(range(n_units)) if order == 0 else list(range(n_units))[::-1]
+    order (random: the one-time shuffle of the unit ids); each step removes m ids
+    from the head and appends them to the tail."""
+    q = group_order(n_units, order, seed)
     out = []
     for _ in range(steps):
         e, q = q[:m], q[m:]
@@ -718,8 +718,21 @@ class HiFTOracle:
         self.t = 0
         self.tau = [0] * self.k
         self.last_grads: Dict[str, np.ndarray] = {}
+        # Algorithm 1 c-d taken literally: when m does not divide n the sets popped from the queue drift, so the
+        # update count (Adam's bias correction) belongs to the unit, and a "group" id is the position in the
+        # period of the walk.  k (learning-rate cycle) stays floor(n / m) + 1.
+        n, m = cfg.n_units, gcfg.layers_per_group
+        self.drifting = bool(getattr(gcfg, "literal_queue", 0)) and not getattr(gcfg, "group_sizes", ()) \
+            and not gcfg.split_emb_head and n % m != 0 and m < n
+        if self.drifting:
+            self.n_sets = n // math.gcd(n, m)
+            self.groups = [sorted(e) for e in queue_walk(n, m, gcfg.order, self.n_sets, gcfg.order_seed)]
+            self.order = list(range(self.n_sets))
+            self.tau = [0] * n                                  # per unit
 
     def active_group(self) -> int:
+        if self.drifting:
+            return self.t % self.n_sets
         return self.order[self.t % self.k]
 
     def current_lr(self) -> float:
@@ -733,6 +746,16 @@ class HiFTOracle:
             return {k: bf16_round(v.astype(np.float32)).astype(F64) for k, v in self.master.items()}
         return self.master
 
+    def unit_of(self, name: str) -> int:
+        for u in range(self.cfg.n_units):
+            if name in tensor_names_of_unit(self.cfg, u):
+                return u
+        raise KeyError(name)
+
+    def tau_of(self, name: str, g: int) -> int:
+        """Updates the tensor has had (its unit's count under the drifting queue, else its group's)."""
+        return self.tau[self.unit_of(name)] if self.drifting else self.tau[g]
+
     def group_tensor_names(self, g: int) -> List[str]:
         return [n for u in self.groups[g] for n in tensor_names_of_unit(self.cfg, u)]
 
@@ -744,14 +767,19 @@ class HiFTOracle:
         drop = (pdrop, int(getattr(self.cfg, "dropout_seed", 0)), self.t) if pdrop > 0.0 else None
         loss, cache = forward(self.cfg, P, tokens, labels, lens, drop)
         grads = backward(self.cfg, P, cache, active_units=self.groups[g])
-        self.tau[g] += 1
         o = self.ocfg
+        if self.drifting:
+            for u in self.groups[g]:
+                self.tau[u] += 1
+        else:
+            self.tau[g] += 1
         for name in self.group_tensor_names(g):
             gr = grads[name]
+            tau = self.tau[self.unit_of(name)] if self.drifting else self.tau[g]
             if o.kind == 0:
                 self.master[name], self.s0[name], self.s1[name] = adamw_update(
                     self.master[name], gr, self.s0[name], self.s1[name],
-                    lr, o.beta1, o.beta2, o.eps, o.weight_decay, self.tau[g])
+                    lr, o.beta1, o.beta2, o.eps, o.weight_decay, tau)
             elif o.kind == 1:
                 self.master[name], self.s0[name] = adagrad_update(
                     self.master[name], gr, self.s0[name], lr, o.eps)
@@ -761,12 +789,12 @@ class HiFTOracle:
             elif o.kind == 3:
                 self.master[name] = sgd_update(self.master[name], gr, lr)
             else:
-                if self.tau[g] == 1:                          # factored state has its own shapes
+                if tau == 1:                                  # factored state has its own shapes
                     m = self.master[name]
                     self.s0[name] = np.zeros(m.shape[0]) if m.ndim > 1 else np.zeros_like(m)
                     self.s1[name] = np.zeros(m.shape[1]) if m.ndim > 1 else np.zeros(0)
                 self.master[name], self.s0[name], self.s1[name] = adafactor_update(
-                    self.master[name], gr, self.s0[name], self.s1[name], lr, o.eps, o.weight_decay, self.tau[g])
+                    self.master[name], gr, self.s0[name], self.s1[name], lr, o.eps, o.weight_decay, tau)
         self.last_grads = grads
         self.t += 1
         return loss

@@ -45,7 +45,8 @@ class ModelCfgC(C.Structure):
 class GroupCfgC(C.Structure):
     _fields_ = [("layers_per_group", C.c_int32), ("split_emb_head", C.c_int32),
                 ("order", C.c_int32), ("order_seed", C.c_uint64),
-                ("group_sizes", C.POINTER(C.c_int32)), ("n_group_sizes", C.c_int32)]
+                ("group_sizes", C.POINTER(C.c_int32)), ("n_group_sizes", C.c_int32),
+                ("literal_queue", C.c_int32)]
 
 
 class OptCfgC(C.Structure):
@@ -83,6 +84,8 @@ def _prototypes():
         "hift_plan_grad_chunks": (i32, [vp, vp, i32, sz, vp, i32, sz, vp, vp, vp, i32]),
         "hift_active_group": (i32, [vp]),
         "hift_num_groups": (i32, [vp]),
+        "hift_num_sets": (i32, [vp]),
+        "hift_set_units": (C.c_int, [vp, i32, C.POINTER(i32), i32, C.POINTER(i32)]),
         "hift_step_count": (i64, [vp]),
         "hift_current_lr": (f64, [vp]),
         "hift_group_units": (C.c_int, [vp, i32, C.POINTER(i32), C.POINTER(i32)]),
@@ -179,7 +182,7 @@ class HiFT:
         sizes = tuple(getattr(groups, "group_sizes", None) or ())
         arr = (C.c_int32 * len(sizes))(*sizes) if sizes else None
         g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed,
-                      C.cast(arr, C.POINTER(C.c_int32)) if sizes else None, len(sizes))
+                      C.cast(arr, C.POINTER(C.c_int32)) if sizes else None, len(sizes), int(getattr(groups, "literal_queue", 0)))
         o = OptCfgC(opt.kind, opt.sched, opt.total_cycles, opt.offload_state, opt.prefetch_groups,
                     getattr(opt, "recompute", 0), getattr(opt, "warmup_cycles", 0),
                     getattr(opt, "shard_rank", 0), getattr(opt, "shard_world", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
@@ -316,6 +319,15 @@ class HiFT:
 
     def num_groups(self) -> int:
         return lib().hift_num_groups(self._h)
+
+    def num_sets(self) -> int:
+        return lib().hift_num_sets(self._h)
+
+    def set_units(self, set_id: int) -> List[int]:
+        cap = self.model.n_blocks + 2
+        arr, n = (C.c_int32 * cap)(), C.c_int32()
+        _check(lib().hift_set_units(self._h, set_id, arr, cap, C.byref(n)), "hift_set_units")
+        return list(arr[:n.value])
 
     def step_count(self) -> int:
         return lib().hift_step_count(self._h)

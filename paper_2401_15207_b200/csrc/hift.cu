@@ -62,6 +62,17 @@ struct BlockIdx {          // tensor indices of one block, -1 if absent
   int n1_g, n1_b, w_qkv, b_qkv, w_o, b_o, n2_g, n2_b, w_fc1, b_fc1, w_fc2, b_fc2;
 };
 struct ProfRec { int cls; cudaEvent_t e0, e1; double work; };
+// What one step trains: one state group (the fixed partition), or, with the literal queue of Algorithm 1
+// when m does not divide n, the m units popped from the queue's head, whose membership drifts from cycle to
+// cycle; then every unit is a state group of its own and a set is a list of them.
+struct ActiveSet {
+  int id = -1;                         // set id: group index, or position in the queue walk's period
+  std::vector<int> groups;             // state groups trained, ascending units
+  std::vector<size_t> grad_base;       // element offset of each group's span in the gradient buffer
+  std::vector<size_t> slot_base;       // byte offset of each group's planes in a state slot
+  size_t grad_numel = 0, slot_bytes = 0;
+  int lo_unit = 0;
+};
 // One device staging slot of the paged optimizer state, laid out like a group's blob.
 constexpr int kMaxSlots = 4;
 struct SlotRec {
@@ -102,7 +113,14 @@ struct hift_ctx {
   int t_tok = -1, t_pos = -1, t_eg = -1, t_eb = -1, t_fg = -1, t_fb = -1, t_wh = -1, t_wc = -1, t_bc = -1;
   size_t total = 0, max_group = 0;
   int64_t t = 0;
-  int forced = -1, last_group = -1;
+  int forced = -1, last_group = -1;     // last_group: id of the set trained by the step in flight / the last one
+  bool queue = false;                   // literal queue (group membership drifts); see ActiveSet
+  std::vector<int> queue_units;         // the queue's initial order of unit ids
+  int n_sets = 0;                       // distinct sets in one period of the schedule
+  int k_cycle = 1;                      // steps per learning-rate cycle: the paper's k
+  ActiveSet act;
+  std::vector<size_t> grad_off;         // per tensor: element offset in the gradient buffer, SIZE_MAX if not trained now
+  std::vector<char> unit_on;            // per unit: trained by the step in flight
   std::vector<int> forced_seq;      // hift_force_sequence: groups of the coming steps, cyclic from step forced_seq_t0
   int64_t forced_seq_t0 = 0;
   int cur_sl = 0; double cur_lr = 0.0;   // slot and learning rate of the step in flight
@@ -167,7 +185,7 @@ struct hift_ctx {
   void note(cudaError_t e) { if (e != cudaSuccess && first_err == cudaSuccess) first_err = e; }
   void* P(int ti) const { return params + tens[ti].off * es; }
   void* Pn(int ti) const { return ti < 0 ? nullptr : P(ti); }
-  float* G(int ti) const { return grad + (tens[ti].off - groups[last_group].off); }
+  float* G(int ti) const { return grad + grad_off[ti]; }
   void pre(int cls, double work) {
     ++step_launches;
     if (!prof_on) return;
@@ -305,7 +323,9 @@ void build_layout(hift_ctx* c) {
   // groups: consecutive chunks of m units (paper, Notation), or embedding | chunks | head
   const int n = L + 2, mm = c->gc.layers_per_group;
   std::vector<std::pair<int, int>> spans;
-  if (!c->group_sizes.empty()) {
+  if (c->queue) {
+    for (int u = 0; u < n; ++u) spans.push_back({u, u});       // every unit keeps its own state
+  } else if (!c->group_sizes.empty()) {
     int u = 0;
     for (int sz : c->group_sizes) { spans.push_back({u, u + sz - 1}); u += sz; }
   } else if (c->gc.split_emb_head) {
@@ -326,7 +346,44 @@ void build_layout(hift_ctx* c) {
     c->max_group = std::max(c->max_group, g.numel);
     c->groups.push_back(g);
   }
-  c->order = make_order((int)c->groups.size(), c->gc.order, c->gc.order_seed);
+  if (c->queue) {
+    // Algorithm 1, c-d: the queue holds the units in the strategy's order; each step pops m from the head and
+    // appends them to the tail, so step t trains queue positions t m .. t m + m - 1 (mod n)
+    c->queue_units = make_order(n, c->gc.order, c->gc.order_seed);
+    int a = n, b = mm;
+    while (b) { const int r = a % b; a = b; b = r; }
+    c->n_sets = n / a;
+    c->k_cycle = (n + mm - 1) / mm;
+    c->order.clear();
+  } else {
+    c->order = make_order((int)c->groups.size(), c->gc.order, c->gc.order_seed);
+    c->n_sets = c->k_cycle = (int)c->groups.size();
+  }
+}
+
+// The state groups of set `id`, with their places in the gradient buffer and in a state slot.
+void fill_set(const hift_ctx* c, int id, ActiveSet* a) {
+  a->id = id;
+  a->groups.clear(); a->grad_base.clear(); a->slot_base.clear();
+  if (c->queue) {
+    const int n = (int)c->groups.size(), mm = c->gc.layers_per_group;
+    for (int j = 0; j < mm && j < n; ++j) a->groups.push_back(c->queue_units[(size_t)(((int64_t)id * mm + j) % n)]);
+    std::sort(a->groups.begin(), a->groups.end());
+  } else {
+    a->groups.push_back(id);
+  }
+  size_t go = 0, so = 0;
+  for (int g : a->groups) {
+    a->grad_base.push_back(go); a->slot_base.push_back(so);
+    go += c->groups[g].numel;
+    so += align_up(c->groups[g].blob_bytes, 256);
+  }
+  a->grad_numel = go; a->slot_bytes = so;
+  a->lo_unit = c->groups[a->groups.front()].unit_lo;
+}
+bool unit_in_set(const hift_ctx* c, const ActiveSet& a, int u) {
+  for (int g : a.groups) if (u >= c->groups[g].unit_lo && u <= c->groups[g].unit_hi) return true;
+  return false;
 }
 
 hift_status dev_alloc(hift_ctx* c, void** p, size_t bytes) {
@@ -387,14 +444,14 @@ size_t slot_bytes(const hift_ctx* c, int s) {
   }
   return 0;
 }
-int level_of_block(const hift_ctx* c, int g, int i) {
+int level_of_block(const hift_ctx* c, const ActiveSet& a, int i) {
   const int u = i + 1;
-  if (u < c->groups[g].unit_lo) return 0;
-  return u <= c->groups[g].unit_hi ? 2 : 1;
+  if (u < a.lo_unit) return 0;
+  return unit_in_set(c, a, u) ? 2 : 1;
 }
 // Assign the per-block activation slots for a step that trains group g.  Returns the arena
 // bytes used.  With assign == false only sizes are computed.
-size_t plan_slots(hift_ctx* c, int g, bool assign) {
+size_t plan_slots(hift_ctx* c, const ActiveSet& g, bool assign) {
   c->arena_off = c->arena_fixed;
   if (c->checked && assign) { c->guards.resize(c->n_fixed_guards); c->record_guards = true; }
   for (int i = 0; i < c->L; ++i) {
@@ -717,6 +774,7 @@ int group_at(const hift_ctx* c, int64_t step) {
     const int64_t n = (int64_t)c->forced_seq.size();
     return c->forced_seq[(size_t)((((step - c->forced_seq_t0) % n) + n) % n)];
   }
+  if (c->queue) return (int)(step % (int64_t)c->n_sets);
   return c->order[step % (int64_t)c->groups.size()];
 }
 void drop_reservations(hift_ctx* c) { for (int i = 0; i < c->n_slots; ++i) c->slot[i].step = -1; }
@@ -741,15 +799,19 @@ int acquire_slot(hift_ctx* c, int g, int64_t s, bool after_forward) {
   }
   if (v < 0) return -1;
   SlotRec& sr = c->slot[v];
-  GroupRec& gr = c->groups[g];
+  ActiveSet a;
+  fill_set(c, g, &a);
   if (after_forward) c->note(cudaStreamWaitEvent(c->st_h2d, c->ev_fwd, 0));
   if (sr.d2h_pending) c->note(cudaStreamWaitEvent(c->st_h2d, sr.ev_d2h, 0));
   c->note(cudaEventRecord(sr.tl_h2d0, c->st_h2d));
-  c->note(cudaMemcpyAsync(sr.mem, gr.blob, gr.blob_bytes, cudaMemcpyHostToDevice, c->st_h2d));
+  for (size_t i = 0; i < a.groups.size(); ++i) {
+    const GroupRec& gr = c->groups[a.groups[i]];
+    if (gr.blob_bytes) c->note(cudaMemcpyAsync(sr.mem + a.slot_base[i], gr.blob, gr.blob_bytes, cudaMemcpyHostToDevice, c->st_h2d));
+    c->step_h2d += gr.blob_bytes;
+  }
   c->note(cudaEventRecord(sr.tl_h2d1, c->st_h2d));
   c->note(cudaEventRecord(sr.ev_h2d, c->st_h2d));
   sr.group = g; sr.step = s; sr.d2h_pending = false; sr.h2d_for_step = s;
-  c->step_h2d += gr.blob_bytes;
   return v;
 }
 // Step start (overlapped modes): the current group, then the groups of the next steps.
@@ -768,27 +830,38 @@ void page_in_ahead(hift_ctx* c) {
 hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int32_t* lab) {
   const hift_model_cfg& m = c->m;
   const int L = c->L, T = c->T, d = c->d, V = c->V, Vp = c->Vp, B = c->B, S = c->S;
-  const int k = (int)c->groups.size();
   const int g = group_at(c, c->t);
-  GroupRec& gr = c->groups[g];
-  const int lo = gr.unit_lo, hi = gr.unit_hi;
-  const double lr = lr_for_cycle(c->oc, c->t / k);
+  fill_set(c, g, &c->act);
+  const ActiveSet& act = c->act;
+  const int lo = act.lo_unit;                                  // the backward pass stops below this unit
+  const double lr = lr_for_cycle(c->oc, c->t / c->k_cycle);
   c->last_group = g;
   c->step_launches = 0; c->step_h2d = 0; c->step_d2h = 0;
   c->first_err = cudaSuccess;
   c->cur_sl = 0; c->cur_lr = lr;
-  auto active = [&](int u) { return u >= lo && u <= hi; };
+  // where each trained tensor's gradient lives: the set's groups side by side, ascending units
+  c->unit_on.assign(L + 2, 0);
+  c->grad_off.assign(c->tens.size(), SIZE_MAX);
+  for (size_t i = 0; i < act.groups.size(); ++i) {
+    const GroupRec& gi = c->groups[act.groups[i]];
+    for (int u = gi.unit_lo; u <= gi.unit_hi; ++u) {
+      c->unit_on[u] = 1;
+      for (int ti : c->unit_tens[u]) c->grad_off[ti] = act.grad_base[i] + (c->tens[ti].off - gi.off);
+    }
+  }
+  auto active = [&](int u) { return c->unit_on[u] != 0; };
 
-  plan_slots(c, g, true);
+  plan_slots(c, act, true);
   if (c->arena_off > c->arena_cap) return HIFT_ERR_CFG;
   if (c->checked)      // the plan moves with the group: paint this step's guard regions before anything runs
     for (size_t o : c->guards) c->note(cudaMemsetAsync(c->arena + o, kGuardByte, kGuardBytes, c->st));
   // the group's tensors, for the completion-ordered chunks of its gradient
-  c->planner.reset(gr.numel, c->chunk_min_elems);
+  c->planner.reset(act.grad_numel, c->chunk_min_elems);
   c->planner_idx.assign(c->tens.size(), -1);
   c->chunks.clear();
-  for (int u = lo; u <= hi; ++u)
-    for (int ti : c->unit_tens[u]) c->planner_idx[ti] = c->planner.add(c->tens[ti].off - gr.off, c->tens[ti].numel);
+  for (int gi : act.groups)
+    for (int u = c->groups[gi].unit_lo; u <= c->groups[gi].unit_hi; ++u)
+      for (int ti : c->unit_tens[u]) c->planner_idx[ti] = c->planner.add(c->grad_off[ti], c->tens[ti].numel);
   // inputs produced on the caller's stream are visible to the step
   c->note(cudaEventRecord(c->ev_in, c->caller));
   c->note(cudaStreamWaitEvent(c->st, c->ev_in, 0));
@@ -797,7 +870,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   if (c->offload && c->oc.prefetch_groups) page_in_ahead(c);
 
   // "Clear gradients": the group's span of the gradient buffer starts at zero
-  c->note(cudaMemsetAsync(c->grad, 0, gr.numel * sizeof(float), c->st));
+  c->note(cudaMemsetAsync(c->grad, 0, act.grad_numel * sizeof(float), c->st));
   c->note(cudaMemsetAsync(c->scal, 0, kScalWords * sizeof(float), c->st));
   int* bad = (int*)(c->scal + 2);
   int* nvalid = (int*)(c->scal + 1);
@@ -911,7 +984,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
 // The optimizer kernels read the step's gate word and leave every buffer as it is when the step
 // failed (a bounded wait gave up, a token or label was out of range, the loss is not finite).
 void enqueue_update(hift_ctx* c) {
-  GroupRec& gr = c->groups[c->last_group];
+  const ActiveSet& act = c->act;
   const int sl = c->cur_sl;
   SlotRec* sr = c->offload ? &c->slot[sl] : nullptr;
   const double lr = c->cur_lr;
@@ -922,32 +995,37 @@ void enqueue_update(hift_ctx* c) {
     if (sr->d2h_pending) c->note(cudaStreamWaitEvent(c->st, sr->ev_d2h, 0));
     c->note(cudaEventRecord(c->tl[4], c->st));
   }
-  // ---------------- group-local optimizer (Algorithm 1: P now points at theta_s only)
-  gr.tau += 1;
-  if (c->af) {
-    // Adafactor works tensor by tensor (its statistics are per row and column of each matrix)
-    float* base = c->offload ? (float*)sr->mem : nullptr;
-    for (int u = gr.unit_lo; u <= gr.unit_hi; ++u)
-      for (int ti : c->unit_tens[u]) {
-        const TensorRec& r = c->tens[ti];
-        float* mst_t;
-        if (!c->mixed) mst_t = (float*)c->params + r.off;
-        else mst_t = c->offload ? base + (r.off - gr.off) : c->master_all + r.off;
-        float* st_t = c->offload ? base + (c->mixed ? gr.numel : 0) + r.af_off : c->af_all + gr.af_base + r.af_off;
-        c->pre(HIFT_K_OPT, (double)r.numel * (20.0 + (c->mixed ? 2.0 : 0.0)));
-        const int nk = launch_adafactor_tensor(c->st, r.rows, r.cols, c->mixed ? c->P(ti) : nullptr, mst_t, c->G(ti), st_t,
-                                               c->af_scratch, lr, c->oc.eps, c->oc.weight_decay, gr.tau, c->gate);
-        c->post();
-        c->step_launches += nk - 1;
-      }
-  } else {
+  // ---------------- group-local optimizer (Algorithm 1: P now points at theta_s only); one pass per state group
+  for (size_t gi = 0; gi < act.groups.size(); ++gi) {
+    GroupRec& gr = c->groups[act.groups[gi]];
+    char* slot_mem = c->offload ? sr->mem + act.slot_base[gi] : nullptr;      // this group's planes in the slot
+    float* grad_g = c->grad + act.grad_base[gi];                              // and its span of the gradient buffer
+    gr.tau += 1;
+    if (c->af) {
+      // Adafactor works tensor by tensor (its statistics are per row and column of each matrix)
+      float* base = (float*)slot_mem;
+      for (int u = gr.unit_lo; u <= gr.unit_hi; ++u)
+        for (int ti : c->unit_tens[u]) {
+          const TensorRec& r = c->tens[ti];
+          float* mst_t;
+          if (!c->mixed) mst_t = (float*)c->params + r.off;
+          else mst_t = c->offload ? base + (r.off - gr.off) : c->master_all + r.off;
+          float* st_t = c->offload ? base + (c->mixed ? gr.numel : 0) + r.af_off : c->af_all + gr.af_base + r.af_off;
+          c->pre(HIFT_K_OPT, (double)r.numel * (20.0 + (c->mixed ? 2.0 : 0.0)));
+          const int nk = launch_adafactor_tensor(c->st, r.rows, r.cols, c->mixed ? c->P(ti) : nullptr, mst_t, c->G(ti), st_t,
+                                                 c->af_scratch, lr, c->oc.eps, c->oc.weight_decay, gr.tau, c->gate);
+          c->post();
+          c->step_launches += nk - 1;
+        }
+      continue;
+    }
     float *mst, *s0, *s1;
     void* pbf = nullptr;
     // the range of the group whose master / state this rank holds and updates (all of it unless sharded)
     const size_t o0 = gr.off + gr.own_lo, on = gr.own_n;
-    const float* gsrc = c->grad + gr.own_lo;
+    const float* gsrc = grad_g + gr.own_lo;
     if (c->offload) {
-      float* base = (float*)sr->mem;
+      float* base = (float*)slot_mem;
       if (c->compact) { mst = nullptr; s0 = base; s1 = base + on; pbf = c->params + o0 * c->es; }
       else if (c->mixed) { mst = base; s0 = base + on; s1 = base + 2 * on; pbf = c->params + o0 * c->es; }
       else { mst = (float*)c->params + o0; s0 = base; s1 = base + on; }
@@ -962,7 +1040,7 @@ void enqueue_update(hift_ctx* c) {
     if (c->compact) {
       // read p, lo, carry, gradient, state; write p, lo, carry, state
       const double opt_bytes = (double)on * (12.25 + 8.0 * c->n_state);
-      uint16_t* lo16 = (uint16_t*)((float*)sr->mem + gr.state_floats);
+      uint16_t* lo16 = (uint16_t*)((float*)slot_mem + gr.state_floats);
       uint8_t* carry8 = (uint8_t*)(lo16 + on);
       LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, on, pbf, lo16, carry8, gsrc, s0, s1, hs, c->gate));
     } else {
@@ -976,12 +1054,16 @@ void enqueue_update(hift_ctx* c) {
     c->note(cudaEventRecord(sr->ev_opt, c->st));
     c->note(cudaStreamWaitEvent(c->st_d2h, sr->ev_opt, 0));
     c->note(cudaEventRecord(c->tl[5], c->st_d2h));
-    c->note(cudaMemcpyAsync(gr.blob, sr->mem, gr.blob_bytes, cudaMemcpyDeviceToHost, c->st_d2h));
+    c->step_d2h = 0;
+    for (size_t gi = 0; gi < act.groups.size(); ++gi) {
+      GroupRec& gr = c->groups[act.groups[gi]];
+      if (gr.blob_bytes) c->note(cudaMemcpyAsync(gr.blob, sr->mem + act.slot_base[gi], gr.blob_bytes, cudaMemcpyDeviceToHost, c->st_d2h));
+      c->step_d2h += gr.blob_bytes;
+    }
     c->note(cudaEventRecord(c->tl[6], c->st_d2h));
     c->note(cudaEventRecord(sr->ev_d2h, c->st_d2h));
     c->tl_valid = true;
     sr->d2h_pending = true;
-    c->step_d2h = gr.blob_bytes;
   }
 }
 
@@ -1010,7 +1092,7 @@ hift_status finish_step(hift_ctx* c, float* loss_host, bool updated) {
 // A step that failed changed nothing on the device (the gate kept the optimizer out, the write-back
 // carried unchanged bytes): take back the update count; t stays, so the same group is next.
 void step_failed(hift_ctx* c) {
-  if (c->last_group >= 0 && c->groups[c->last_group].tau > 0) c->groups[c->last_group].tau -= 1;
+  for (int g : c->act.groups) if (c->groups[g].tau > 0) c->groups[g].tau -= 1;
 }
 
 hift_status do_step(hift_ctx* c, const int32_t* tok, const int32_t* lab, float* loss_host) {
@@ -1180,6 +1262,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
   if (oc->prefetch_groups < 0 || oc->prefetch_groups > kMaxSlots - 1) return HIFT_ERR_CFG;
   if (oc->shard_world > 1 && (oc->shard_rank < 0 || oc->shard_rank >= oc->shard_world || oc->kind == 4)) return HIFT_ERR_CFG;
+  if (gc->literal_queue != 0 && (gc->group_sizes != nullptr || gc->split_emb_head || oc->shard_world > 1)) return HIFT_ERR_CFG;
   if (oc->sched == 1 && (oc->total_cycles < 1 || oc->warmup_cycles < 0 || oc->warmup_cycles >= oc->total_cycles)) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
 
@@ -1201,6 +1284,9 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // the group's own step; p >= 2 = p + 1 slots, uploads issued p - 1 steps ahead
   c->n_slots = c->offload ? 1 + oc->prefetch_groups : 1;
   c->lookahead = c->offload && oc->prefetch_groups >= 2 ? oc->prefetch_groups - 1 : 0;
+  const bool drifting = gc->literal_queue != 0 && (m->n_blocks + 2) % gc->layers_per_group != 0 && gc->layers_per_group < m->n_blocks + 2;
+  // drifting sets share units with one another: one slot, so that an upload always follows the last write-back
+  if (drifting) { c->n_slots = 1; c->lookahead = 0; }
   // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
   c->compact = c->mixed && c->offload && !c->af;
   c->recompute = oc->recompute != 0;
@@ -1211,6 +1297,9 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_work, 0, sizeof(c->prof_work));
+  // the literal queue only differs from the fixed partition when m does not divide n
+  c->queue = gc->literal_queue != 0 && gc->group_sizes == nullptr && !gc->split_emb_head &&
+             (m->n_blocks + 2) % gc->layers_per_group != 0 && gc->layers_per_group < m->n_blocks + 2;
   build_layout(c);
   c->shard_world = oc->shard_world > 1 ? oc->shard_world : 1;
   c->shard_rank = c->shard_world > 1 ? oc->shard_rank : 0;
@@ -1262,18 +1351,23 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     if (c->compact) return g.state_floats * sizeof(float) + g.own_n * 2 + g.own_n / 8;     // own_n is a multiple of 128
     return ((c->mixed ? g.own_n : 0) + g.state_floats) * sizeof(float);
   };
-  size_t slot_bytes_max = 0, af_total = 0;
-  for (auto& g : c->groups) { slot_bytes_max = std::max(slot_bytes_max, blob_bytes_of(g)); af_total += c->af ? g.state_floats : 0; }
+  size_t slot_bytes_max = 0, af_total = 0, grad_max = c->max_group;
+  for (auto& g : c->groups) { g.blob_bytes = c->offload ? blob_bytes_of(g) : 0; af_total += c->af ? g.state_floats : 0; }
+  for (int sid = 0; sid < c->n_sets; ++sid) {       // the largest set decides the gradient buffer and the state slots
+    ActiveSet a;
+    fill_set(c, sid, &a);
+    slot_bytes_max = std::max(slot_bytes_max, a.slot_bytes);
+    grad_max = std::max(grad_max, a.grad_numel);
+  }
   if ((rc = dev_alloc(c, (void**)&c->params, c->total * c->es)) != HIFT_OK) return fail(rc);
   cudaMemsetAsync(c->params, 0, c->total * c->es, c->st);
-  if ((rc = dev_alloc(c, (void**)&c->grad, c->max_group * sizeof(float))) != HIFT_OK) return fail(rc);
+  if ((rc = dev_alloc(c, (void**)&c->grad, grad_max * sizeof(float))) != HIFT_OK) return fail(rc);
   if (c->offload) {
     for (int s = 0; s < c->n_slots; ++s) {
       if ((rc = dev_alloc(c, (void**)&c->slot[s].mem, slot_bytes_max)) != HIFT_OK) return fail(rc);
       cudaMemsetAsync(c->slot[s].mem, 0, slot_bytes_max, c->st);
     }
     for (auto& g : c->groups) {
-      g.blob_bytes = blob_bytes_of(g);
       if (pinned_alloc((void**)&g.blob, g.blob_bytes ? g.blob_bytes : 256, cudaHostAllocDefault) != cudaSuccess) {
         cudaGetLastError();
         g.blob = nullptr;
@@ -1353,7 +1447,11 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
     c->n_fixed_guards = c->guards.size();
     if (pass == 0) {
       size_t worst = c->arena_fixed;
-      for (size_t g = 0; g < c->groups.size(); ++g) worst = std::max(worst, plan_slots(c, (int)g, false));
+      for (int sid = 0; sid < c->n_sets; ++sid) {
+        ActiveSet a;
+        fill_set(c, sid, &a);
+        worst = std::max(worst, plan_slots(c, a, false));
+      }
       c->arena_cap = worst;
       if ((rc = dev_alloc(c, (void**)&c->arena, c->arena_cap)) != HIFT_OK) return fail(rc);
     }
@@ -1393,7 +1491,7 @@ hift_status hift_step_begin(hift_ctx* c, const int32_t* tok, const int32_t* lab,
 hift_status hift_grad_view(hift_ctx* c, float** grad_dev, size_t* n) {
   if (!c || !grad_dev || !n || c->last_group < 0) return HIFT_ERR_CFG;
   *grad_dev = c->grad;
-  *n = c->groups[c->last_group].numel;
+  *n = c->act.grad_numel;
   return HIFT_OK;
 }
 hift_status hift_step_begin_async(hift_ctx* c, const int32_t* tok, const int32_t* lab) {
@@ -1422,7 +1520,7 @@ hift_status hift_gate_view(hift_ctx* c, int32_t** gate_dev) {
   return HIFT_OK;
 }
 hift_status hift_shard_range(const hift_ctx* c, int32_t g, int32_t rank, size_t* lo, size_t* n) {
-  if (!c || g < 0 || g >= (int)c->groups.size() || rank < 0 || rank >= c->shard_world || !lo || !n) return HIFT_ERR_CFG;
+  if (!c || c->queue || g < 0 || g >= (int)c->groups.size() || rank < 0 || rank >= c->shard_world || !lo || !n) return HIFT_ERR_CFG;
   const GroupRec& gr = c->groups[g];
   const size_t piece = align_up((gr.numel + c->shard_world - 1) / c->shard_world, kAlignElems);
   *lo = std::min((size_t)rank * piece, gr.numel);
@@ -1430,8 +1528,8 @@ hift_status hift_shard_range(const hift_ctx* c, int32_t g, int32_t rank, size_t*
   return HIFT_OK;
 }
 hift_status hift_param_view(hift_ctx* c, void** param_dev, size_t* n, int32_t* elem_bytes) {
-  if (!c || !param_dev || !n || c->last_group < 0) return HIFT_ERR_CFG;
-  const GroupRec& gr = c->groups[c->last_group];
+  if (!c || !param_dev || !n || c->last_group < 0 || c->act.groups.size() != 1) return HIFT_ERR_CFG;
+  const GroupRec& gr = c->groups[c->act.groups[0]];
   *param_dev = c->params + gr.off * c->es;
   *n = gr.numel;
   if (elem_bytes) *elem_bytes = c->es;
@@ -1526,23 +1624,42 @@ hift_status hift_step_host(hift_ctx* c, const int32_t* tok, const int32_t* lab, 
 }
 
 int32_t hift_active_group(const hift_ctx* c) { return group_at(c, c->t); }
-int32_t hift_num_groups(const hift_ctx* c) { return (int32_t)c->groups.size(); }
+int32_t hift_num_groups(const hift_ctx* c) { return (int32_t)c->k_cycle; }
+int32_t hift_num_sets(const hift_ctx* c) { return (int32_t)c->n_sets; }
+hift_status hift_set_units(const hift_ctx* c, int32_t set_id, int32_t* units, int32_t cap, int32_t* n_units) {
+  if (!c || set_id < 0 || set_id >= c->n_sets || !units || !n_units) return HIFT_ERR_CFG;
+  ActiveSet a;
+  fill_set(c, set_id, &a);
+  int n = 0;
+  for (int g : a.groups)
+    for (int u = c->groups[g].unit_lo; u <= c->groups[g].unit_hi; ++u) {
+      if (n == cap) return HIFT_ERR_CFG;
+      units[n++] = u;
+    }
+  *n_units = n;
+  return HIFT_OK;
+}
 int64_t hift_step_count(const hift_ctx* c) { return c->t; }
-double hift_current_lr(const hift_ctx* c) { return lr_for_cycle(c->oc, c->t / (int64_t)c->groups.size()); }
+double hift_current_lr(const hift_ctx* c) { return lr_for_cycle(c->oc, c->t / (int64_t)c->k_cycle); }
 hift_status hift_group_units(const hift_ctx* c, int32_t g, int32_t* lo, int32_t* hi) {
-  if (g < 0 || g >= (int)c->groups.size()) return HIFT_ERR_CFG;
-  *lo = c->groups[g].unit_lo; *hi = c->groups[g].unit_hi;
+  if (g < 0 || g >= c->n_sets) return HIFT_ERR_CFG;
+  ActiveSet a;
+  fill_set(c, g, &a);
+  *lo = c->groups[a.groups.front()].unit_lo; *hi = c->groups[a.groups.back()].unit_hi;
+  // a set of the drifting queue may wrap around (the top unit together with the bottom one): not an interval
+  for (size_t i = 1; i < a.groups.size(); ++i)
+    if (c->groups[a.groups[i]].unit_lo != c->groups[a.groups[i - 1]].unit_hi + 1) return HIFT_ERR_CFG;
   return HIFT_OK;
 }
 hift_status hift_force_group(hift_ctx* c, int32_t g) {
-  if (g < -1 || g >= (int)c->groups.size()) return HIFT_ERR_CFG;
+  if (g < -1 || g >= c->n_sets) return HIFT_ERR_CFG;
   if (g != c->forced) drop_reservations(c);     // uploads made for the schedule's coming steps stay resident, unreserved
   c->forced = g;
   return HIFT_OK;
 }
 hift_status hift_force_sequence(hift_ctx* c, const int32_t* groups, int32_t n) {
   if (!c || n < 0 || (n > 0 && !groups)) return HIFT_ERR_CFG;
-  for (int i = 0; i < n; ++i) if (groups[i] < 0 || groups[i] >= (int)c->groups.size()) return HIFT_ERR_CFG;
+  for (int i = 0; i < n; ++i) if (groups[i] < 0 || groups[i] >= c->n_sets) return HIFT_ERR_CFG;
   drop_reservations(c);
   c->forced_seq.assign(groups, groups + n);
   c->forced_seq_t0 = c->t;
@@ -1694,7 +1811,7 @@ hift_status hift_get_factored_state(hift_ctx* c, int32_t ti, int32_t which, floa
 
 hift_status hift_get_grad(hift_ctx* c, int32_t ti, float* dst, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
-  if (c->last_group < 0 || group_of_unit(c, c->tens[ti].unit) != c->last_group) return HIFT_ERR_CFG;
+  if (c->last_group < 0 || c->grad_off.size() != c->tens.size() || c->grad_off[ti] == SIZE_MAX) return HIFT_ERR_CFG;
   sync_all(c);
   return cudaMemcpy(dst, c->G(ti), n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }

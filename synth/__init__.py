@@ -77,6 +77,7 @@ class GroupCfg:
     order: int = ORDER_BOTTOM2UP
     order_seed: int = 0
     group_sizes: tuple = ()            # non-empty: consecutive units per group, bottom first (overrides m)
+    literal_queue: int = 0             # 1: pop m units from a queue per step (sets drift when m does not divide n)
 
 
 @dataclass(frozen=True)

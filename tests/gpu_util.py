@@ -115,7 +115,7 @@ def check_update_given_gradient(h, orc, ocfg, n, g, lr, master0, state0, tol=1e-
     shape = orc.master[n].shape
     grad = h.get_grad(n).astype(np.float64).reshape(shape)
     m0 = master0.astype(np.float64).reshape(shape)
-    tau = orc.tau[g]
+    tau = orc.tau_of(n, g)
     k = ocfg.kind
     if k == 0:
         ref = O.adamw_update(m0, grad, state0[0].astype(np.float64).reshape(shape), state0[1].astype(np.float64).reshape(shape),

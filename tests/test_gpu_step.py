@@ -715,3 +715,49 @@ def test_dropout_is_reproducible_and_recompute_redraws_the_same_masks():
     assert a == b and all(np.array_equal(x, y) for x, y in zip(pa, pb))
     assert a != plain and a != c              # the masks act, and follow the seed
     assert a == r and all(np.array_equal(x, y) for x, y in zip(pa, pr))   # a recomputed block draws its masks again
+
+
+@pytest.mark.parametrize("arch,dtype,m,order", [(0, synth.DTYPE_FP32, 2, 0), (1, synth.DTYPE_FP32, 2, 1), (2, synth.DTYPE_FP32, 3, 2),
+                                                (2, synth.DTYPE_FP32, 4, 0), (0, synth.DTYPE_BF16, 2, 0), (2, synth.DTYPE_BF16, 3, 1)])
+def test_literal_queue_with_drifting_sets(arch, dtype, m, order):
+    """Algorithm 1 c-d taken literally with m not dividing n (5 units): sets drift and wrap around (the top and
+    the bottom unit trained together, which makes the backward pass run the whole depth with weight gradients at
+    both ends only), every unit keeps its own state and update count.  A full period and more in lockstep with
+    the oracle: set ids, learning rate (moves every k = floor(n/m) + 1 steps), loss, gradients, frozen bits, and
+    the in-step update from the library's own gradient."""
+    from paper_2401_15207_b200 import HiFT
+    fp32 = dtype == synth.DTYPE_FP32
+    cfg = mini(arch, dtype, tie_head=1 if arch == 0 else 0)
+    gc = synth.GroupCfg(layers_per_group=m, order=order, order_seed=5, literal_queue=1)
+    oc = synth.OptCfg(kind=0, lr=1e-3, weight_decay=0.01, sched=1, total_cycles=6, offload_state=1, prefetch_groups=2)
+    h = HiFT(cfg, gc, oc)
+    try:
+        import math
+        n = cfg.n_units
+        assert h.num_groups() == n // m + 1 and h.num_sets() == n // math.gcd(n, m)
+        from oracle import hift_oracle as O
+        walk = O.queue_walk(n, m, order, h.num_sets(), 5)
+        assert [h.set_units(s) for s in range(h.num_sets())] == [sorted(e) for e in walk]
+    finally:
+        h.close()
+    lockstep(cfg, gc, oc, n // math.gcd(n, m) + 2, "zipf", FP32_LOSS if fp32 else BF16_LOSS, FP32_GRAD if fp32 else BF16_GRAD,
+             resync=True)
+
+
+def test_literal_queue_equals_the_fixed_partition_when_m_divides_n():
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    cfg = mini(2, synth.DTYPE_BF16, n_blocks=4)                 # 6 units, m = 2
+    p0 = synth.init_params(cfg, 2)
+    outs = []
+    for lq in (0, 1):
+        h = HiFT(cfg, synth.GroupCfg(layers_per_group=2, order=1, literal_queue=lq), synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=2))
+        h.set_params(p0)
+        assert h.num_sets() == h.num_groups() == 3
+        losses = []
+        for t in range(6):
+            tok, lab = synth.lm_batch(cfg, 3, t)
+            losses.append(h.step(torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()))
+        outs.append((losses, [h.get_param(n).copy() for n in h.tensor_names()]))
+        h.close()
+    assert outs[0][0] == outs[1][0] and all(np.array_equal(a, b) for a, b in zip(outs[0][1], outs[1][1]))

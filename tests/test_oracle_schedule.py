@@ -176,3 +176,57 @@ def test_peak_trainable_fraction():
         cat = synth.unit_tensors(c)
         for u in range(c.n_units):
             assert [n for n, _, _ in cat[u]] == O.tensor_names_of_unit(c, u)
+
+
+# ---------------------------------------------------------------- the literal queue when m does not divide n
+def test_drifting_queue_sets_follow_algorithm_1_and_cover_units_evenly():
+    """Algorithm 1 c-d with m not dividing n: the sets are what a literal pop-m / append-to-tail walk gives, they
+    repeat with period n / gcd(n, m), every unit is trained m / gcd(n, m) times per period, a set may wrap around
+    (top and bottom unit together), and the learning-rate cycle stays k = floor(n / m) + 1 steps."""
+    import math
+    from collections import Counter, deque
+    cfg = synth.ModelCfg(arch=0, n_blocks=3, d_model=16, n_heads=2, d_ffn=32, vocab=31, max_pos=8, batch=1, seq=4)
+    n = cfg.n_units                                                # 5 units
+    p0 = synth.init_params(cfg, 0)
+    for m in (2, 3, 4):
+        for order in (0, 1, 2):
+            gc = synth.GroupCfg(layers_per_group=m, order=order, order_seed=9, literal_queue=1)
+            orc = O.HiFTOracle(cfg, gc, synth.OptCfg(kind=2, lr=1e-2, sched=1, total_cycles=4), p0)
+            assert orc.drifting and orc.k == n // m + 1 and orc.n_sets == n // math.gcd(n, m)
+            # an independent walk with a deque
+            q = deque(O.group_order(n, order, 9))
+            seen = Counter()
+            for t in range(2 * orc.n_sets):
+                e = [q.popleft() for _ in range(m)]
+                q.extend(e)
+                assert orc.groups[t % orc.n_sets] == sorted(e)
+                if t < orc.n_sets:
+                    seen.update(e)
+            assert set(seen.values()) == {m // math.gcd(n, m)} and len(seen) == n
+            if order == 0 and m == 2:
+                assert orc.groups[2] == [0, 4]                      # the wrap-around set
+    # m dividing n: the flag changes nothing
+    gc0, gc1 = synth.GroupCfg(layers_per_group=5), synth.GroupCfg(layers_per_group=5, literal_queue=1)
+    assert not O.HiFTOracle(cfg, gc1, synth.OptCfg(), p0).drifting
+    assert O.HiFTOracle(cfg, gc1, synth.OptCfg(), p0).groups == O.HiFTOracle(cfg, gc0, synth.OptCfg(), p0).groups
+
+
+def test_drifting_queue_step_moves_only_the_popped_units_and_counts_updates_per_unit():
+    cfg = synth.ModelCfg(arch=0, n_blocks=3, d_model=16, n_heads=2, d_ffn=32, vocab=31, max_pos=8, batch=2, seq=6, init_std=0.1)
+    gc = synth.GroupCfg(layers_per_group=2, literal_queue=1)
+    oc = synth.OptCfg(kind=0, lr=1e-2, sched=1, total_cycles=5)
+    orc = O.HiFTOracle(cfg, gc, oc, synth.init_params(cfg, 1, perturb=0.1))
+    lrs = []
+    for t in range(7):
+        units = orc.groups[orc.active_group()]
+        before = {k: v.copy() for k, v in orc.master.items()}
+        tok, lab = synth.batch_for(cfg, 3, t, "uniform")
+        lrs.append(orc.current_lr())
+        orc.step(tok, lab)
+        for name in orc.master:
+            moved = not np.array_equal(orc.master[name], before[name])
+            assert moved == (orc.unit_of(name) in units), (t, name)
+    # sets: [0,1] [2,3] [0,4] [1,2] [3,4] [0,1] [2,3]: after 7 steps units 0..3 have 3 updates, unit 4 has 2
+    assert orc.tau == [3, 3, 3, 3, 2]
+    # k = 3: the rate moves after steps 3 and 6
+    assert lrs[0] == lrs[1] == lrs[2] and lrs[3] == lrs[4] == lrs[5] and lrs[2] > lrs[3] > lrs[6]
