@@ -138,6 +138,13 @@ typedef struct {
                              /* the unsharded update.  0 or 1 = off.  Not with Adafactor (its statistics */
                              /* span rows and columns); checkpoints are refused while sharded; outside   */
                              /* its piece hift_get_param returns the model value, hift_get_state zeros.  */
+  int32_t grad_bf16;         /* 1: the active group's gradient is kept in bf16: the weight-gradient GEMMs store  */
+                             /* bf16 from their fp32 accumulators, the other gradient producers round once, the   */
+                             /* optimizer reads bf16; half the gradient buffer, half the exchange volume of a     */
+                             /* data-parallel step, 2 bytes per element less optimizer traffic.  One rounding of  */
+                             /* 2^-9 relative per gradient element (within the 2e-2 gradient tolerance; the       */
+                             /* update given that gradient is exact as before).  bf16 models with AdamW, AdaGrad, */
+                             /* SGD-momentum or SGD only.  0: fp32 gradients.                                     */
   double lr, beta1, beta2, eps, weight_decay, momentum;
 } hift_opt_cfg;
 
@@ -197,7 +204,8 @@ hift_status hift_set_key_lengths(hift_ctx *ctx, const int32_t *lens_host);
  * every rank calls when any rank's first half failed, so that replicas stay identical. */
 hift_status hift_step_begin(hift_ctx *ctx, const int32_t *tokens_dev, const int32_t *labels_dev,
                             float *loss_host);
-hift_status hift_grad_view(hift_ctx *ctx, float **grad_dev, size_t *n);
+hift_status hift_grad_view(hift_ctx *ctx, void **grad_dev, size_t *n);   /* n elements of hift_grad_elem_bytes() each */
+int32_t     hift_grad_elem_bytes(const hift_ctx *ctx);                    /* 4: fp32 gradients, 2: bf16 (grad_bf16) */
 hift_status hift_step_end(hift_ctx *ctx);
 hift_status hift_step_abort(hift_ctx *ctx);
 

@@ -52,7 +52,7 @@ class GroupCfgC(C.Structure):
 class OptCfgC(C.Structure):
     _fields_ = [("kind", C.c_int32), ("sched", C.c_int32), ("total_cycles", C.c_int32),
                 ("offload_state", C.c_int32), ("prefetch_groups", C.c_int32), ("recompute", C.c_int32), ("warmup_cycles", C.c_int32),
-                ("shard_rank", C.c_int32), ("shard_world", C.c_int32),
+                ("shard_rank", C.c_int32), ("shard_world", C.c_int32), ("grad_bf16", C.c_int32),
                 ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
                 ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double)]
 
@@ -70,6 +70,7 @@ def _prototypes():
         "hift_set_key_lengths": (C.c_int, [vp, vp]),
         "hift_step_begin": (C.c_int, [vp, vp, vp, pf]),
         "hift_grad_view": (C.c_int, [vp, C.POINTER(vp), C.POINTER(sz)]),
+        "hift_grad_elem_bytes": (i32, [vp]),
         "hift_step_end": (C.c_int, [vp]),
         "hift_step_abort": (C.c_int, [vp]),
         "hift_step_begin_async": (C.c_int, [vp, vp, vp]),
@@ -185,7 +186,7 @@ class HiFT:
                       C.cast(arr, C.POINTER(C.c_int32)) if sizes else None, len(sizes), int(getattr(groups, "literal_queue", 0)))
         o = OptCfgC(opt.kind, opt.sched, opt.total_cycles, opt.offload_state, opt.prefetch_groups,
                     getattr(opt, "recompute", 0), getattr(opt, "warmup_cycles", 0),
-                    getattr(opt, "shard_rank", 0), getattr(opt, "shard_world", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
+                    getattr(opt, "shard_rank", 0), getattr(opt, "shard_world", 0), getattr(opt, "grad_bf16", 0), opt.lr, opt.beta1, opt.beta2, opt.eps, opt.weight_decay, opt.momentum)
         self._h = C.c_void_p()
         self._stream = _stream_ptr() if stream is None else stream
         _check(lib().hift_create(C.byref(m), C.byref(g), C.byref(o), self._stream, C.byref(self._h)), "hift_create")
@@ -244,14 +245,17 @@ class HiFT:
         return loss.value
 
     def grad_view(self):
-        """The active group's flat fp32 gradient as a torch CUDA tensor sharing the library's memory."""
+        """The active group's flat gradient (fp32, or bf16 with grad_bf16) as a torch CUDA tensor sharing the
+        library's memory."""
         import torch
         ptr, n = C.c_void_p(), C.c_size_t()
         _check(lib().hift_grad_view(self._h, C.byref(ptr), C.byref(n)), "hift_grad_view")
+        half = lib().hift_grad_elem_bytes(self._h) == 2
 
         class _View:
-            __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<f4", "data": (ptr.value, False), "version": 3}
-        return torch.as_tensor(_View(), device="cuda")
+            __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<i2" if half else "<f4", "data": (ptr.value, False), "version": 3}
+        t = torch.as_tensor(_View(), device="cuda")
+        return t.view(torch.bfloat16) if half else t
 
     def step_end(self):
         _check(lib().hift_step_end(self._h), "hift_step_end")

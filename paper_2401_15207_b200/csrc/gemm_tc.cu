@@ -1111,11 +1111,13 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr<false, true, false>();
   if (e == cudaSuccess) e = set_smem_attr<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr<true, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr<true, true, false>();
   if (e == cudaSuccess) e = set_smem_attr2<false, false, false>();
   if (e == cudaSuccess) e = set_smem_attr2<false, false, true>();
   if (e == cudaSuccess) e = set_smem_attr2<false, true, false>();
   if (e == cudaSuccess) e = set_smem_attr2<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr2<true, true, true>();
+  if (e == cudaSuccess) e = set_smem_attr2<true, true, false>();
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
   if (e == cudaSuccess) e = set_smem_attr_ab<64, 0>();
@@ -1139,7 +1141,7 @@ static int classify(const GemmArgs& g) {
   if (((uintptr_t)g.a | (uintptr_t)g.b | (uintptr_t)g.c) & 15) return 0;
   if (g.bias && ((uintptr_t)g.bias & 15)) return 0;
   if (g.residual && (!g.out_f32 || ((uintptr_t)g.residual & 15) || g.ldr % 4)) return 0;
-  if (form == 3 && (!g.out_f32 || g.bias || g.residual)) return 0;
+  if (form == 3 && (g.bias || g.residual)) return 0;        // weight gradients: fp32 out, or bf16 out when gradients are kept in bf16
   // rotary embedding in the epilogue: forward form, bf16 output, whole heads of 128 columns per tile
   // gated activation in the epilogue: forward form, bf16 output, f a multiple of 128 (a tile = 128 gate + 128 up columns)
   if (g.swiglu_out && (form != 1 || g.out_f32 || g.residual || g.rope_cs || (g.N / 2) % 128 || g.N % 2 ||
@@ -1201,7 +1203,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
     if (!ok) return cudaErrorInvalidValue;
     if (form == 1) return g.out_f32 ? launch_pair<false, false, true>(st, g, ta, tb) : launch_pair<false, false, false>(st, g, ta, tb);
     if (form == 2) return g.out_f32 ? launch_pair<false, true, true>(st, g, ta, tb) : launch_pair<false, true, false>(st, g, ta, tb);
-    return launch_pair<true, true, true>(st, g, ta, tb);
+    return g.out_f32 ? launch_pair<true, true, true>(st, g, ta, tb) : launch_pair<true, true, false>(st, g, ta, tb);
   }
   // K-major operand: tensor [rows = M or N][inner = K]; MN-major operand: tensor [rows = K][inner = M or N]
   if (form == 3) ok = get_map(g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.sak, BK, &ta);
@@ -1213,7 +1215,7 @@ cudaError_t gemm_tc_launch(cudaStream_t st, const GemmArgs& g) {
                                   : launch_inst<false, false, false>(st, g, ta, tb, bn);
   if (form == 2) return g.out_f32 ? launch_inst<false, true, true>(st, g, ta, tb, bn)
                                   : launch_inst<false, true, false>(st, g, ta, tb, bn);
-  return launch_inst<true, true, true>(st, g, ta, tb, bn);
+  return g.out_f32 ? launch_inst<true, true, true>(st, g, ta, tb, bn) : launch_inst<true, true, false>(st, g, ta, tb, bn);
 }
 
 const int* gemm_tc_error_device_ptr() {

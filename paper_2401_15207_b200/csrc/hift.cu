@@ -147,7 +147,9 @@ struct hift_ctx {
   int n_slots = 1;
   int lookahead = 0;                // steps ahead of the current one whose state is uploaded early
   int* gate = nullptr;              // device word: non-zero = the step failed, the optimizer must not write
-  float* grad = nullptr;            // [max_group]
+  float* grad = nullptr;            // gradient buffer of the largest set: fp32 elements, or bf16 ones (gbf)
+  bool gbf = false; int ges = 4;    // gradients kept in bf16; bytes per gradient element
+  float* stage = nullptr;           // set-up only, with bf16 gradients: fp32 staging that the gradient buffer is too small for
   char* arena = nullptr; size_t arena_cap = 0, arena_off = 0, arena_fixed = 0;
   bool checked = false;             // guard regions behind every arena slice, verified by hift_check_arena
   bool record_guards = false;
@@ -185,7 +187,7 @@ struct hift_ctx {
   void note(cudaError_t e) { if (e != cudaSuccess && first_err == cudaSuccess) first_err = e; }
   void* P(int ti) const { return params + tens[ti].off * es; }
   void* Pn(int ti) const { return ti < 0 ? nullptr : P(ti); }
-  float* G(int ti) const { return grad + grad_off[ti]; }
+  void* G(int ti) const { return (char*)grad + grad_off[ti] * ges; }
   void pre(int cls, double work) {
     ++step_launches;
     if (!prof_on) return;
@@ -499,8 +501,8 @@ void linear_dx(hift_ctx* c, int M, int N, int K, const void* dy, int64_t ldy, co
 }
 // dw[N,K] = dy[M,N]^T x[M,K]   (fp32 out)
 void linear_dw(hift_ctx* c, int M, int N, int K, const void* dy, int64_t ldy, const void* x,
-               int64_t ldx, float* dw) {
-  gemm(c, HIFT_K_GEMM_DW, N, K, M, dy, 1, ldy, x, ldx, 1, dw, K, nullptr, nullptr, 0, true);
+               int64_t ldx, void* dw) {
+  gemm(c, HIFT_K_GEMM_DW, N, K, M, dy, 1, ldy, x, ldx, 1, dw, K, nullptr, nullptr, 0, !c->gbf);
 }
 void norm_fwd(hift_ctx* c, const float* x, int tg, int tb, void* y_a, float* y_r, float* stats) {
   const int kind = c->m.arch == 2 ? 1 : 0;
@@ -519,14 +521,14 @@ void norm_bwd_params(hift_ctx* c, const void* dy, bool dy_f32, const float* x, c
   const int mode = c->m.arch == 2 ? 2 : 1;
   LAUNCH(HIFT_K_REDUCE, (double)c->T * c->d * ((dy_f32 ? 4 : c->es) + 4),
          launch_colreduce(c->st, c->mixed && !dy_f32, mode, c->T, c->d, dy, c->d, x, stats, c->partial,
-                          c->G(tg), tb >= 0 ? c->G(tb) : nullptr));
+                          c->G(tg), tb >= 0 ? c->G(tb) : nullptr, c->gbf));
   ++c->step_launches;   // two kernels per call
 }
 void bias_grad(hift_ctx* c, const void* dy, bool dy_f32, int64_t rows, int cols, int64_t ld, int tb) {
   if (tb < 0) return;
   LAUNCH(HIFT_K_REDUCE, (double)rows * cols * (dy_f32 ? 4 : c->es),
          launch_colreduce(c->st, c->mixed && !dy_f32, 0, rows, cols, dy, ld, nullptr, nullptr, c->partial,
-                          c->G(tb), nullptr));
+                          c->G(tb), nullptr, c->gbf));
   ++c->step_launches;
 }
 void attn_fwd(hift_ctx* c, const void* qkv, void* o, float* lse) {
@@ -830,6 +832,7 @@ void page_in_ahead(hift_ctx* c) {
 hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int32_t* lab) {
   const hift_model_cfg& m = c->m;
   const int L = c->L, T = c->T, d = c->d, V = c->V, Vp = c->Vp, B = c->B, S = c->S;
+  if (c->stage) { cudaStreamSynchronize(c->st); cudaFree(c->stage); c->stage = nullptr; }     // set-up is over
   const int g = group_at(c, c->t);
   fill_set(c, g, &c->act);
   const ActiveSet& act = c->act;
@@ -870,7 +873,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
   if (c->offload && c->oc.prefetch_groups) page_in_ahead(c);
 
   // "Clear gradients": the group's span of the gradient buffer starts at zero
-  c->note(cudaMemsetAsync(c->grad, 0, act.grad_numel * sizeof(float), c->st));
+  c->note(cudaMemsetAsync(c->grad, 0, act.grad_numel * c->ges, c->st));
   c->note(cudaMemsetAsync(c->scal, 0, kScalWords * sizeof(float), c->st));
   int* bad = (int*)(c->scal + 2);
   int* nvalid = (int*)(c->scal + 1);
@@ -917,7 +920,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
     const int C = m.n_classes;
     if (head_on) {
       // dWc[C,d] = dlogits^T pooled ; pooled rows have stride S*d
-      gemm(c, HIFT_K_GEMM_DW, C, d, B, c->logits, 1, C, c->x_final_a, (int64_t)S * d, 1, c->G(c->t_wc), d, nullptr, nullptr, 0, true);
+      gemm(c, HIFT_K_GEMM_DW, C, d, B, c->logits, 1, C, c->x_final_a, (int64_t)S * d, 1, c->G(c->t_wc), d, nullptr, nullptr, 0, !c->gbf);
       bias_grad(c, c->logits, false, B, C, C, c->t_bc);
       grad_done(c, c->t_bc); grad_done(c, c->t_wc);
     }
@@ -961,10 +964,10 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
       src = c->dxb;
     }
     LAUNCH(HIFT_K_EMBED, (double)T * d * 12,
-           embed_bwd_tok_kernel<<<T, 128, T * sizeof(int), c->st>>>(tok, src, c->G(c->t_tok), T, d, V));
+           embed_bwd_tok_kernel<<<T, 128, T * sizeof(int), c->st>>>(tok, src, c->G(c->t_tok), c->gbf, T, d, V));
     if (c->t_pos >= 0) {
       LAUNCH(HIFT_K_EMBED, (double)T * d * 4 + (double)S * d * 4,
-             embed_bwd_pos_kernel<<<S, 128, 0, c->st>>>(src, c->G(c->t_pos), B, S, d));
+             embed_bwd_pos_kernel<<<S, 128, 0, c->st>>>(src, c->G(c->t_pos), c->gbf, B, S, d));
       grad_done(c, c->t_pos);
     }
     grad_done(c, c->t_tok);
@@ -999,7 +1002,7 @@ void enqueue_update(hift_ctx* c) {
   for (size_t gi = 0; gi < act.groups.size(); ++gi) {
     GroupRec& gr = c->groups[act.groups[gi]];
     char* slot_mem = c->offload ? sr->mem + act.slot_base[gi] : nullptr;      // this group's planes in the slot
-    float* grad_g = c->grad + act.grad_base[gi];                              // and its span of the gradient buffer
+    const char* grad_g = (const char*)c->grad + act.grad_base[gi] * c->ges;  // and its span of the gradient buffer
     gr.tau += 1;
     if (c->af) {
       // Adafactor works tensor by tensor (its statistics are per row and column of each matrix)
@@ -1012,7 +1015,7 @@ void enqueue_update(hift_ctx* c) {
           else mst_t = c->offload ? base + (r.off - gr.off) : c->master_all + r.off;
           float* st_t = c->offload ? base + (c->mixed ? gr.numel : 0) + r.af_off : c->af_all + gr.af_base + r.af_off;
           c->pre(HIFT_K_OPT, (double)r.numel * (20.0 + (c->mixed ? 2.0 : 0.0)));
-          const int nk = launch_adafactor_tensor(c->st, r.rows, r.cols, c->mixed ? c->P(ti) : nullptr, mst_t, c->G(ti), st_t,
+          const int nk = launch_adafactor_tensor(c->st, r.rows, r.cols, c->mixed ? c->P(ti) : nullptr, mst_t, (const float*)c->G(ti), st_t,
                                                  c->af_scratch, lr, c->oc.eps, c->oc.weight_decay, gr.tau, c->gate);
           c->post();
           c->step_launches += nk - 1;
@@ -1023,7 +1026,7 @@ void enqueue_update(hift_ctx* c) {
     void* pbf = nullptr;
     // the range of the group whose master / state this rank holds and updates (all of it unless sharded)
     const size_t o0 = gr.off + gr.own_lo, on = gr.own_n;
-    const float* gsrc = grad_g + gr.own_lo;
+    const void* gsrc = grad_g + gr.own_lo * c->ges;
     if (c->offload) {
       float* base = (float*)slot_mem;
       if (c->compact) { mst = nullptr; s0 = base; s1 = base + on; pbf = c->params + o0 * c->es; }
@@ -1039,13 +1042,13 @@ void enqueue_update(hift_ctx* c) {
                                            c->oc.weight_decay, c->oc.momentum, gr.tau);
     if (c->compact) {
       // read p, lo, carry, gradient, state; write p, lo, carry, state
-      const double opt_bytes = (double)on * (12.25 + 8.0 * c->n_state);
+      const double opt_bytes = (double)on * (8.25 + c->ges + 8.0 * c->n_state);
       uint16_t* lo16 = (uint16_t*)((float*)slot_mem + gr.state_floats);
       uint8_t* carry8 = (uint8_t*)(lo16 + on);
-      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, on, pbf, lo16, carry8, gsrc, s0, s1, hs, c->gate));
+      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt_compact(c->st, c->oc.kind, on, pbf, lo16, carry8, gsrc, s0, s1, hs, c->gate, c->gbf));
     } else {
-      const double opt_bytes = (double)on * ((c->oc.kind == 0 ? 28.0 : (c->oc.kind == 3 ? 12.0 : 20.0)) + (pbf ? 2.0 : 0.0));
-      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, on, pbf, mst, gsrc, s0, s1, hs, c->gate));
+      const double opt_bytes = (double)on * ((c->oc.kind == 0 ? 24.0 : (c->oc.kind == 3 ? 8.0 : 16.0)) + c->ges + (pbf ? 2.0 : 0.0));
+      LAUNCH(HIFT_K_OPT, opt_bytes, launch_fused_opt(c->st, c->oc.kind, on, pbf, mst, gsrc, s0, s1, hs, c->gate, c->gbf));
     }
   }
 
@@ -1186,6 +1189,14 @@ void master_write(hift_ctx* c, GroupRec& gr, size_t o, size_t n, const float* sr
   }
 }
 
+// fp32 staging of up to max_group elements for the set-up calls: the gradient buffer itself, unless gradients are
+// kept in bf16 (then it is half the size and a buffer of its own is allocated, and released when training starts)
+float* staging(hift_ctx* c) {
+  if (!c->gbf) return c->grad;
+  if (!c->stage && cudaMalloc((void**)&c->stage, c->max_group * sizeof(float)) != cudaSuccess) { cudaGetLastError(); c->stage = nullptr; }
+  return c->stage;
+}
+
 }  // namespace
 
 // ====================================================================== C entry points
@@ -1210,6 +1221,7 @@ void hift_destroy(hift_ctx* c) {
   if (!c) return;
   sync_all(c);
   for (void* p : c->dev_allocs) cudaFree(p);
+  if (c->stage) cudaFree(c->stage);
   for (auto& g : c->groups) if (g.blob) cudaFreeHost(g.blob);
   if (c->scal_host) cudaFreeHost(c->scal_host);
   for (auto e : c->ev_pool) cudaEventDestroy(e);
@@ -1262,6 +1274,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (oc->kind < 0 || oc->kind > 4 || oc->sched < 0 || oc->sched > 1) return HIFT_ERR_CFG;
   if (oc->prefetch_groups < 0 || oc->prefetch_groups > kMaxSlots - 1) return HIFT_ERR_CFG;
   if (oc->shard_world > 1 && (oc->shard_rank < 0 || oc->shard_rank >= oc->shard_world || oc->kind == 4)) return HIFT_ERR_CFG;
+  if (oc->grad_bf16 != 0 && (m->dtype != 1 || oc->kind == 4)) return HIFT_ERR_CFG;      // bf16 gradients: bf16 model, fused optimizers
   if (gc->literal_queue != 0 && (gc->group_sizes != nullptr || gc->split_emb_head || oc->shard_world > 1)) return HIFT_ERR_CFG;
   if (oc->sched == 1 && (oc->total_cycles < 1 || oc->warmup_cycles < 0 || oc->warmup_cycles >= oc->total_cycles)) return HIFT_ERR_CFG;
   if (!(oc->lr >= 0.0)) return HIFT_ERR_CFG;
@@ -1290,6 +1303,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   // bf16 parameters + a fused optimizer: page 17 bits of master per element instead of 32
   c->compact = c->mixed && c->offload && !c->af;
   c->recompute = oc->recompute != 0;
+  c->gbf = oc->grad_bf16 != 0;
+  c->ges = c->gbf ? 2 : 4;
   c->drop_on = m->dropout > 0.0;
   c->drop_thr = (uint32_t)floor(m->dropout * 4294967296.0);
   c->drop_scale = (float)(1.0 / (1.0 - m->dropout));
@@ -1361,7 +1376,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   }
   if ((rc = dev_alloc(c, (void**)&c->params, c->total * c->es)) != HIFT_OK) return fail(rc);
   cudaMemsetAsync(c->params, 0, c->total * c->es, c->st);
-  if ((rc = dev_alloc(c, (void**)&c->grad, grad_max * sizeof(float))) != HIFT_OK) return fail(rc);
+  if ((rc = dev_alloc(c, (void**)&c->grad, grad_max * c->ges)) != HIFT_OK) return fail(rc);
   if (c->offload) {
     for (int s = 0; s < c->n_slots; ++s) {
       if ((rc = dev_alloc(c, (void**)&c->slot[s].mem, slot_bytes_max)) != HIFT_OK) return fail(rc);
@@ -1488,7 +1503,7 @@ hift_status hift_step_begin(hift_ctx* c, const int32_t* tok, const int32_t* lab,
   if (s == HIFT_OK) c->pending_update = true;
   return s;
 }
-hift_status hift_grad_view(hift_ctx* c, float** grad_dev, size_t* n) {
+hift_status hift_grad_view(hift_ctx* c, void** grad_dev, size_t* n) {
   if (!c || !grad_dev || !n || c->last_group < 0) return HIFT_ERR_CFG;
   *grad_dev = c->grad;
   *n = c->act.grad_numel;
@@ -1572,6 +1587,7 @@ int32_t hift_plan_grad_chunks(const size_t* offsets, const size_t* sizes, int32_
   }
   return nc;
 }
+int32_t hift_grad_elem_bytes(const hift_ctx* c) { return c ? c->ges : 0; }
 hift_status hift_step_end(hift_ctx* c) { return hift_step_finish(c, nullptr); }
 hift_status hift_step_abort(hift_ctx* c) {
   if (!c || !c->pending_update) return HIFT_ERR_CFG;
@@ -1739,8 +1755,10 @@ hift_status hift_set_param(hift_ctx* c, int32_t ti, const float* src, size_t n) 
   }
   if (c->mixed) {
     // stage the fp32 values in the gradient buffer (any tensor fits in the largest group)
-    if (cudaMemcpyAsync(c->grad, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
-    cast_from_f32_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>(c->grad, (bf16*)c->P(ti), n);
+    float* stg = staging(c);
+    if (!stg) return HIFT_ERR_OOM_DEVICE;
+    if (cudaMemcpyAsync(stg, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
+    cast_from_f32_kernel<bf16><<<grid_for(n, 256), 256, 0, c->st>>>(stg, (bf16*)c->P(ti), n);
   } else if (op.n != n) {
     // fp32 parameters are their own master: the part another rank updates is still this rank's model value
     if (cudaMemcpyAsync(c->P(ti), src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) return HIFT_ERR_CUDA;
@@ -1813,21 +1831,27 @@ hift_status hift_get_grad(hift_ctx* c, int32_t ti, float* dst, size_t n) {
   if (ti < 0 || ti >= (int)c->tens.size() || !dst || n != c->tens[ti].numel) return HIFT_ERR_CFG;
   if (c->last_group < 0 || c->grad_off.size() != c->tens.size() || c->grad_off[ti] == SIZE_MAX) return HIFT_ERR_CFG;
   sync_all(c);
-  return cudaMemcpy(dst, c->G(ti), n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+  if (!c->gbf) return cudaMemcpy(dst, c->G(ti), n * sizeof(float), cudaMemcpyDeviceToHost) == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+  std::vector<uint16_t> h(n);
+  if (cudaMemcpy(h.data(), c->G(ti), n * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return HIFT_ERR_CUDA;
+  for (size_t i = 0; i < n; ++i) { const uint32_t u = (uint32_t)h[i] << 16; memcpy(dst + i, &u, 4); }
+  return HIFT_OK;
 }
 
 hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
   sync_all(c);
   invalidate_slots(c);
+  float* stg = c->compact ? staging(c) : nullptr;
+  if (c->compact && !stg) return HIFT_ERR_OOM_DEVICE;
   for (size_t g = 0; g < c->groups.size(); ++g) {
     GroupRec& gr = c->groups[g];
     if (c->offload) cudaMemsetAsync(c->slot[0].mem, 0, gr.blob_bytes, c->st);
-    if (c->compact) cudaMemsetAsync(c->grad, 0, gr.numel * sizeof(float), c->st);     // alignment gaps pack to zero
+    if (c->compact) cudaMemsetAsync(stg, 0, gr.numel * sizeof(float), c->st);     // alignment gaps pack to zero
     for (int u = gr.unit_lo; u <= gr.unit_hi; ++u) {
       for (int ti : c->unit_tens[u]) {
         const TensorRec& r = c->tens[ti];
         float* mp = nullptr;
-        if (c->compact) mp = c->grad + (r.off - gr.off);           // staged as floats, packed below
+        if (c->compact) mp = stg + (r.off - gr.off);           // staged as floats, packed below
         else if (c->mixed) mp = c->offload ? (float*)c->slot[0].mem + (r.off - gr.off) : c->master_all + r.off;
         const uint64_t sd = seed * 0x9E3779B97F4A7C15ull + (uint64_t)ti * 0xD1B54A32D192ED03ull;
         if (c->mixed) init_tensor_kernel<bf16><<<grid_for(r.numel, 256), 256, 0, c->st>>>((bf16*)c->P(ti), mp, r.numel, r.init_kind, (float)stdv, sd);
@@ -1837,7 +1861,7 @@ hift_status hift_init_synthetic(hift_ctx* c, uint64_t seed, double stdv) {
     if (c->compact) {
       uint16_t* lo16 = (uint16_t*)((float*)c->slot[0].mem + gr.state_floats);
       if (gr.own_n)
-        master_pack_kernel<<<grid_for(gr.own_n / 8, 256), 256, 0, c->st>>>(c->grad + gr.own_lo, lo16, (uint8_t*)(lo16 + gr.own_n), gr.own_n / 8);
+        master_pack_kernel<<<grid_for(gr.own_n / 8, 256), 256, 0, c->st>>>(stg + gr.own_lo, lo16, (uint8_t*)(lo16 + gr.own_n), gr.own_n / 8);
     }
     if (c->offload) {
       cudaMemcpyAsync(gr.blob, c->slot[0].mem, gr.blob_bytes, cudaMemcpyDeviceToHost, c->st);
@@ -1960,8 +1984,9 @@ hift_status hift_load(hift_ctx* c, const char* path) {
       // rebuild the bf16 model copy of this group from its master values
       const float* src = mp;
       if (mh) {
-        ok = cudaMemcpyAsync(c->grad, mp, gr.numel * sizeof(float), cudaMemcpyHostToDevice, c->st) == cudaSuccess;
-        src = c->grad;
+        float* stg = staging(c);
+        ok = stg != nullptr && cudaMemcpyAsync(stg, mp, gr.numel * sizeof(float), cudaMemcpyHostToDevice, c->st) == cudaSuccess;
+        src = stg;
       }
       cast_from_f32_kernel<bf16><<<grid_for(gr.numel, 256), 256, 0, c->st>>>(src, (bf16*)(c->params + gr.off * c->es), gr.numel);
       ok = ok && cudaStreamSynchronize(c->st) == cudaSuccess;

@@ -80,11 +80,20 @@ __global__ void embed_fwd_kernel(const int32_t* __restrict__ ids, const T* __res
   }
 }
 
+// Gradients live in one flat buffer of fp32 or (hift_opt_cfg.grad_bf16) bf16 elements; the small producers
+// take the buffer as void* plus the element type.
+__device__ __forceinline__ float grad_load(const void* g, size_t i, int bf) {
+  return bf ? __bfloat162float(reinterpret_cast<const bf16*>(g)[i]) : reinterpret_cast<const float*>(g)[i];
+}
+__device__ __forceinline__ void grad_store(void* g, size_t i, float v, int bf) {
+  if (bf) reinterpret_cast<bf16*>(g)[i] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(g)[i] = v;
+}
 // grad_tok[id,:] += sum over positions t with ids[t] == id of dx[t,:], occurrences added in
 // increasing t.  Block t does the work for id = ids[t] only if t is the first occurrence, so
 // every gradient row has one writer and a fixed summation order (no atomics).
 __global__ void embed_bwd_tok_kernel(const int32_t* __restrict__ ids, const float* __restrict__ dx,
-                                     float* __restrict__ grad_tok, int Ttot, int d, int vocab) {
+                                     void* __restrict__ grad_tok, int gbf, int Ttot, int d, int vocab) {
   extern __shared__ int occ[];                       // positions of this id, in order
   __shared__ int n_occ;
   __shared__ int warp_cnt[32];
@@ -116,22 +125,22 @@ __global__ void embed_bwd_tok_kernel(const int32_t* __restrict__ ids, const floa
     __syncthreads();
   }
   const int n = n_occ;
-  float* gr = grad_tok + (size_t)id * d;
+  const size_t row = (size_t)id * d;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     float acc = 0.f;
     for (int i = 0; i < n; ++i) acc += dx[(size_t)occ[i] * d + c];
-    gr[c] += acc;
+    grad_store(grad_tok, row + c, grad_load(grad_tok, row + c, gbf) + acc, gbf);     // on top of a tied head's share
   }
 }
 
 // grad_pos[s,:] = sum over batch rows b of dx[b*S+s,:]
-__global__ void embed_bwd_pos_kernel(const float* __restrict__ dx, float* __restrict__ grad_pos,
+__global__ void embed_bwd_pos_kernel(const float* __restrict__ dx, void* __restrict__ grad_pos, int gbf,
                                      int B, int S, int d) {
   const int s = blockIdx.x;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     float acc = 0.f;
     for (int b = 0; b < B; ++b) acc += dx[((size_t)b * S + s) * d + c];
-    grad_pos[(size_t)s * d + c] = acc;
+    grad_store(grad_pos, (size_t)s * d + c, acc, gbf);
   }
 }
 
@@ -303,7 +312,7 @@ __global__ void colreduce_stage1_kernel(const DY* __restrict__ dy, int64_t ld,
 }
 // Stage 2: out0[col] = sum_chunk partial[0][chunk][col] (and out1 likewise from plane 1).
 __global__ void colreduce_stage2_kernel(const float* __restrict__ partial, int nch, int cols,
-                                        float* __restrict__ out0, float* __restrict__ out1) {
+                                        void* __restrict__ out0, void* __restrict__ out1, int gbf) {
   const int col = blockIdx.x * blockDim.x + threadIdx.x;
   if (col >= cols) return;
   double t0 = 0.0, t1 = 0.0;
@@ -311,8 +320,8 @@ __global__ void colreduce_stage2_kernel(const float* __restrict__ partial, int n
     t0 += partial[((size_t)c) * cols + col];
     if (out1) t1 += partial[((size_t)nch + c) * cols + col];
   }
-  out0[col] = (float)t0;
-  if (out1) out1[col] = (float)t1;
+  grad_store(out0, col, (float)t0, gbf);
+  if (out1) grad_store(out1, col, (float)t1, gbf);
 }
 
 // ------------------------------------------------------------------ activations
@@ -612,9 +621,18 @@ __device__ __forceinline__ void opt_update(float& th, float g, float& s0, float&
     th = __fmaf_rn(-h.lr, g, th);
   }
 }
-template <int KIND, bool HAS_BF16>
+// four consecutive gradient elements (16-byte or 8-byte load, streaming)
+template <typename GT> __device__ __forceinline__ float4 grad4(const GT* g, size_t i4);
+template <> __device__ __forceinline__ float4 grad4<float>(const float* g, size_t i4) { return __ldcs(reinterpret_cast<const float4*>(g) + i4); }
+template <> __device__ __forceinline__ float4 grad4<bf16>(const bf16* g, size_t i4) {
+  const uint2 r = __ldcs(reinterpret_cast<const uint2*>(g) + i4);
+  const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r.x));
+  const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&r.y));
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+template <int KIND, bool HAS_BF16, typename GT>
 __global__ void __launch_bounds__(256)
-fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const float* __restrict__ grad,
+fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const GT* __restrict__ grad,
                  float* __restrict__ s0, float* __restrict__ s1, size_t n, OptScalars h,
                  const int* __restrict__ gate) {
   if (gate != nullptr && *gate != 0) return;        // the step failed: every buffer keeps its bits
@@ -623,7 +641,7 @@ fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const flo
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (; i < n4; i += stride) {
     float4 th = reinterpret_cast<const float4*>(master)[i];
-    const float4 g = __ldcs(reinterpret_cast<const float4*>(grad) + i);
+    const float4 g = grad4<GT>(grad, i);
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
     if (KIND != 3) a = reinterpret_cast<const float4*>(s0)[i];
     float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -647,7 +665,7 @@ fused_opt_kernel(bf16* __restrict__ param, float* __restrict__ master, const flo
   const size_t t = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) {
     float th = master[t], a = (KIND != 3) ? s0[t] : 0.f, b = (KIND == 0) ? s1[t] : 0.f;
-    opt_update<KIND>(th, grad[t], a, b, h);
+    opt_update<KIND>(th, to_f(grad[t]), a, b, h);
     master[t] = th;
     if (KIND != 3) s0[t] = a;
     if (KIND == 0) s1[t] = b;
@@ -679,10 +697,10 @@ __device__ __forceinline__ void master_pack(uint32_t u, uint32_t& p, uint32_t& l
 __device__ __forceinline__ uint32_t master_unpack(uint32_t p, uint32_t lo, uint32_t carry) {
   return ((p - carry) << 16) | lo;
 }
-template <int KIND>
+template <int KIND, typename GT>
 __global__ void __launch_bounds__(256)
 fused_opt_compact_kernel(uint16_t* __restrict__ param, uint16_t* __restrict__ lo16, uint8_t* __restrict__ carry8,
-                         const float* __restrict__ grad, float* __restrict__ s0, float* __restrict__ s1,
+                         const GT* __restrict__ grad, float* __restrict__ s0, float* __restrict__ s1,
                          size_t n8, OptScalars h, const int* __restrict__ gate) {
   if (gate != nullptr && *gate != 0) return;        // the step failed: every buffer keeps its bits
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -694,7 +712,7 @@ fused_opt_compact_kernel(uint16_t* __restrict__ param, uint16_t* __restrict__ lo
     const uint32_t pws[4] = {pw.x, pw.y, pw.z, pw.w}, lws[4] = {lw.x, lw.y, lw.z, lw.w};
     float g[8], a[8], b[8], th[8];
     {
-      const float4 g0 = __ldcs(reinterpret_cast<const float4*>(grad) + 2 * i), g1 = __ldcs(reinterpret_cast<const float4*>(grad) + 2 * i + 1);
+      const float4 g0 = grad4<GT>(grad, 2 * i), g1 = grad4<GT>(grad, 2 * i + 1);
       g[0] = g0.x; g[1] = g0.y; g[2] = g0.z; g[3] = g0.w; g[4] = g1.x; g[5] = g1.y; g[6] = g1.z; g[7] = g1.w;
     }
     if (KIND != 3) load8(s0 + 8 * i, a);

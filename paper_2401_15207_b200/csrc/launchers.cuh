@@ -172,7 +172,7 @@ inline int colreduce_chunks(int64_t rows) {
 }
 inline void launch_colreduce(cudaStream_t st, bool dy_bf16, int mode, int64_t rows, int cols,
                              const void* dy, int64_t ld, const float* x, const float* stats,
-                             float* partial, float* out0, float* out1) {
+                             float* partial, void* out0, void* out1, int out_bf16 = 0) {
   const int nch = colreduce_chunks(rows);
   dim3 grid((cols + 31) / 32, nch), block(32, 8);
 #define CR(T, M) colreduce_stage1_kernel<T, M><<<grid, block, 0, st>>>((const T*)dy, ld, x, stats, partial, rows, cols)
@@ -180,7 +180,7 @@ inline void launch_colreduce(cudaStream_t st, bool dy_bf16, int mode, int64_t ro
   else { if (mode == 0) CR(bf16, 0); else if (mode == 1) CR(bf16, 1); else CR(bf16, 2); }
 #undef CR
   colreduce_stage2_kernel<<<(cols + 127) / 128, 128, 0, st>>>(partial, nch, cols, out0,
-                                                             mode == 1 ? out1 : nullptr);
+                                                             mode == 1 ? out1 : nullptr, out_bf16);
 }
 
 // ---- cross-entropy --------------------------------------------------------------
@@ -211,27 +211,32 @@ inline OptScalars make_opt_scalars(int kind, double lr, double b1, double b2, do
   h.mu = (float)mu;
   return h;
 }
+// grad_bf16: the gradient buffer holds bf16 elements (else fp32)
 inline void launch_fused_opt(cudaStream_t st, int kind, size_t n, void* param_bf16, float* master,
-                             const float* grad, float* s0, float* s1, const OptScalars& h,
-                             const int* gate = nullptr) {
+                             const void* grad, float* s0, float* s1, const OptScalars& h,
+                             const int* gate = nullptr, bool grad_bf16 = false) {
   if (n == 0) return;
   const int block = 256;
   int grid = grid_for((n + 3) / 4, block, 148 * 8);
-#define OPT(K)                                                                                         \
-  if (param_bf16) fused_opt_kernel<K, true><<<grid, block, 0, st>>>((bf16*)param_bf16, master, grad, s0, s1, n, h, gate); \
-  else fused_opt_kernel<K, false><<<grid, block, 0, st>>>(nullptr, master, grad, s0, s1, n, h, gate)
-  if (kind == 0) { OPT(0); } else if (kind == 1) { OPT(1); } else if (kind == 2) { OPT(2); } else { OPT(3); }
+#define OPTG(K, GT)                                                                                    \
+  if (param_bf16) fused_opt_kernel<K, true, GT><<<grid, block, 0, st>>>((bf16*)param_bf16, master, (const GT*)grad, s0, s1, n, h, gate); \
+  else fused_opt_kernel<K, false, GT><<<grid, block, 0, st>>>(nullptr, master, (const GT*)grad, s0, s1, n, h, gate)
+#define OPT(K) if (grad_bf16) { OPTG(K, bf16); } else { OPTG(K, float); }
+  if (kind == 0) { OPT(0) } else if (kind == 1) { OPT(1) } else if (kind == 2) { OPT(2) } else { OPT(3) }
 #undef OPT
+#undef OPTG
 }
 
 // compact master (bf16 copy + low halves + carry bits); n must be a multiple of 8
 inline void launch_fused_opt_compact(cudaStream_t st, int kind, size_t n, void* param_bf16, uint16_t* lo16, uint8_t* carry8,
-                                     const float* grad, float* s0, float* s1, const OptScalars& h,
-                                     const int* gate = nullptr) {
+                                     const void* grad, float* s0, float* s1, const OptScalars& h,
+                                     const int* gate = nullptr, bool grad_bf16 = false) {
   if (n == 0) return;
   const size_t n8 = n / 8;
   const int grid = grid_for(n8, 256, 148 * 8);
-#define OPTC(K) fused_opt_compact_kernel<K><<<grid, 256, 0, st>>>((uint16_t*)param_bf16, lo16, carry8, grad, s0, s1, n8, h, gate)
+#define OPTC(K)                                                                                                                              \
+  if (grad_bf16) fused_opt_compact_kernel<K, bf16><<<grid, 256, 0, st>>>((uint16_t*)param_bf16, lo16, carry8, (const bf16*)grad, s0, s1, n8, h, gate); \
+  else fused_opt_compact_kernel<K, float><<<grid, 256, 0, st>>>((uint16_t*)param_bf16, lo16, carry8, (const float*)grad, s0, s1, n8, h, gate)
   if (kind == 0) { OPTC(0); } else if (kind == 1) { OPTC(1); } else if (kind == 2) { OPTC(2); } else { OPTC(3); }
 #undef OPTC
 }

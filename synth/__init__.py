@@ -97,6 +97,7 @@ class OptCfg:
     recompute: int = 0
     shard_rank: int = 0                # optimizer state sharded over data-parallel ranks (0 / 1 = off)
     shard_world: int = 0
+    grad_bf16: int = 0                 # 1: the active group's gradient is kept in bf16
 
 
 # --------------------------------------------------------------------------

@@ -761,3 +761,44 @@ def test_literal_queue_equals_the_fixed_partition_when_m_divides_n():
         outs.append((losses, [h.get_param(n).copy() for n in h.tensor_names()]))
         h.close()
     assert outs[0][0] == outs[1][0] and all(np.array_equal(a, b) for a, b in zip(outs[0][1], outs[1][1]))
+
+
+@pytest.mark.parametrize("arch,big", [(0, True), (1, True), (2, True), (0, False), (2, False)])
+def test_gradients_kept_in_bf16(arch, big):
+    """grad_bf16: the weight-gradient GEMMs store bf16 from their fp32 accumulators (tensor-core and CUDA-core
+    kernels), the reductions and the embedding scatter round once (a tied head's share and the embedding's share
+    meet in bf16), the optimizer reads bf16.  In lockstep with the oracle at the bf16 tolerances; the update given
+    the library's own (bf16) gradient still agrees to 1e-6; every stored gradient is a bf16 value; the gradient
+    buffer is half the size."""
+    import torch
+    from paper_2401_15207_b200 import HiFT
+    if big:
+        cfg = synth.ModelCfg(arch=arch, n_blocks=2, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=512, vocab=1001, max_pos=128,
+                             n_classes=2 if arch == 1 else 0, causal=0 if arch == 1 else 1, tie_head=1 if arch == 0 else 0,
+                             norm_eps=1e-6 if arch == 2 else 1e-5, dtype=synth.DTYPE_BF16, batch=2, seq=128, init_std=0.05)
+    else:
+        cfg = mini(arch, synth.DTYPE_BF16, tie_head=1 if arch == 0 else 0)
+    gc = synth.GroupCfg(1)
+    oc = synth.OptCfg(kind=0, lr=1e-3, weight_decay=0.01, offload_state=1, prefetch_groups=2, grad_bf16=1)
+    lockstep(cfg, gc, oc, cfg.n_units + 1, "zipf", BF16_LOSS, BF16_GRAD, resync=True)
+    a, b = HiFT(cfg, gc, oc), HiFT(cfg, gc, synth.OptCfg(**{**oc.__dict__, "grad_bf16": 0}))
+    try:
+        biggest = max(sum(int(np.prod(a.tensor_info(n)[1])) for n in a.tensor_names() if a.tensor_info(n)[0] == u) for u in range(cfg.n_units))
+        assert b.peak_hbm_bytes() - a.peak_hbm_bytes() >= 2 * biggest - 4096          # 4 -> 2 bytes per gradient element
+        for h in (a, b):
+            h.set_params(synth.init_params(cfg, 2))
+        tok, lab = synth.batch_for(cfg, 3, 0, "zipf")
+        tt, ll = torch.from_numpy(tok).cuda(), torch.from_numpy(lab).cuda()
+        la, lb = a.step(tt, ll), b.step(tt, ll)
+        assert la == lb                                                                  # the forward pass is the same
+        for n in a.tensor_names():
+            if a.tensor_info(n)[0] == 0:
+                ga, gb = a.get_grad(n), b.get_grad(n)
+                assert not (ga.view(np.uint32) & 0xFFFF).any()                           # bf16 values
+                assert np.abs(ga - gb).max() <= 2.0 ** -8 * np.abs(gb).max() + 1e-30
+        assert a.grad_view().dtype == torch.bfloat16 and b.grad_view().dtype == torch.float32
+    finally:
+        a.close()
+        b.close()
+    with pytest.raises(Exception):
+        HiFT(cfg.scaled(dtype=synth.DTYPE_FP32), gc, oc)                                 # bf16 gradients need a bf16 model
