@@ -573,6 +573,31 @@ def run_micro(args, cfg):
                          "frac_of_burst_peak": round(fl / (us * 1e-6) / 1e12 / peaks["bf16_tflops"], 3),
                          "algorithmic_bytes": int(algo)})
             del x, w, dy, out
+    elif args.micro == "step":
+        # A three-block model of the workload's width: with the middle block as the active group, one step holds every
+        # kind of launch of the full-depth step (a frozen block below the group: forward only; the active block; a
+        # block above it: forward and dX; the head) on a few GB, so its GEMM launches can be captured one by one and
+        # scaled to the full depth by the number of blocks of each kind.
+        import dataclasses
+        from paper_2401_15207_b200 import HiFT
+        small = dataclasses.replace(cfg, n_blocks=3)
+        _, gcfg, ocfg = WORKLOADS[args.workload]()
+        h = HiFT(small, gcfg, ocfg)
+        try:
+            h.init_synthetic(1234, small.init_std)
+            mid = [g for g in range(h.num_groups()) if h.group_units(g)[0] == 2][0]    # units: embedding 0, blocks 1..3
+            h.force_sequence([mid])
+            tok, lab = (torch.from_numpy(a).cuda() for a in synth.batch_for(small, 77, 0))
+            h.profile_enable(True)
+            for _ in range(n_l):
+                loss = h.step(tok, lab)
+            prof = h.profile()
+            rows = [dict(kernel=k, launches=v["launches"] // n_l, ms_per_step=round(v["ms"] / n_l, 4))
+                    for k, v in prof.items() if v["launches"]]
+            rows.append({"active_group": mid, "units": list(h.group_units(mid)), "loss": loss,
+                         "peak_hbm_gb": round(h.peak_hbm_bytes() / 1e9, 2)})
+        finally:
+            h.close()
     else:
         rows = [dict(kernel=k, **v) for k, v in standalone_kernels(cfg, peaks, launches=n_l).items()]
     print(json.dumps({"micro": args.micro, "workload": args.workload, "launches": n_l,
@@ -714,13 +739,14 @@ def run_sweep_depth(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the tensor-core GEMM launches of one llama7b step (the step that
-# trains block 4: 129 forward, 113 dX, 4 dW launches), recorded once from an ncu capture.  A recorded figure, not one
-# to take again on the whole step: after a kernel change, capture one launch per GEMM shape on its own (a few GB on
-# the device) and weight by the launch counts the profile hook reports; time the whole step with CUDA events only.
+# trains block 4: 129 forward, 113 dX, 4 dW launches).  Taken with ncu on `--micro step` (the same model with three
+# blocks, a few GB: one frozen block, the active block, one block above it and the head) and scaled to 32 blocks by the
+# number of blocks of each kind; the whole step is timed with CUDA events only.  Retake it after a change to the GEMM.
 NCU_GEMM_TRAFFIC = {
-    "bytes_per_launch": 54.199e9 / 246,
-    "note": "ncu, recorded once: 54.20 GB over the 246 GEMM launches of one step (block 4 active) = 220.3 MB per "
-            "launch, against 205.1 MB of operands and results per launch (1.07)",
+    "bytes_per_launch": 53.214e9 / 246,
+    "note": "ncu on a three-block model of the same width, every GEMM launch of one step, scaled to 32 blocks by block "
+            "kind: 53.21 GB over the 246 GEMM launches of the step that trains block 4 = 216.3 MB per launch, against "
+            "205.1 MB of operands and results per launch (1.05)",
 }
 
 
@@ -751,7 +777,7 @@ def main():
                     help="leave out the k = 1 full-parameter step of the same model (needs ~132 GB at the 7B shape)")
     ap.add_argument("--sweep", default=None, choices=["optimizer", "depth"],
                     help="kernel sweeps instead of the step benchmark")
-    ap.add_argument("--micro", default=None, choices=["gemm", "kernels"],
+    ap.add_argument("--micro", default=None, choices=["gemm", "kernels", "step"],
                     help="single kernels at the workload's shapes, a few launches each (small enough for an ncu capture)")
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--only", default=None, help="--micro gemm: only shapes whose name contains this")

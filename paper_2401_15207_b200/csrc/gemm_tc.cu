@@ -620,7 +620,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-               int tiles_m, int num_tiles, TileRt tc, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb, GeluArgs ge) {
+               int tiles_m, int num_tiles, int n_fast, TileRt tc, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb, GeluArgs ge) {
+  // Tile walk.  CTAs that run together should share the LARGER operand's slab and leave the smaller operand to L2:
+  // row tiles fastest (n_fast = 0) when A is the smaller operand, column tiles fastest (n_fast = tiles along N) when B is.
+  auto tm_of = [&](int tile) { return n_fast ? tile / n_fast : tile % tiles_m; };
+  auto tn_of = [&](int tile) { return n_fast ? tile % n_fast : tile / tiles_m; };
   const int BN = tc.bn, S = tc.stages;
   const uint32_t kStageBytes = (uint32_t)tc.stage_bytes;
   extern __shared__ uint8_t smem_raw[];
@@ -665,7 +669,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       uint32_t ph = 0;                   // ring position and its phase, advanced without divisions
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        const int m0 = tm_of(tile) * BM, n0 = tn_of(tile) * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); ok = false; break; }
           const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
@@ -681,7 +685,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (int j = 0; j * 64 < BN; ++j) tma_load_2d(sb + j * (BK * 128), &tmap_b, full_bar(s), n0 + j * 64, k0);
           } else if (swg.out != nullptr) {
             // gate | up: 128 rows of the gate block and the 128 rows of the same index in the up block
-            const int nb = (tile / tiles_m) * 128;
+            const int nb = tn_of(tile) * 128;
             tma_load_2d(sb, &tmap_b, full_bar(s), k0, nb);
             tma_load_2d(sb + 128 * 128, &tmap_b, full_bar(s), k0, swg.half + nb);
           } else {
@@ -740,10 +744,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tc_fence_after();
       // one decision for the whole warp: the tensor-memory loads below are warp-collective
       if (!__all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0)) break;
-      const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+      const int m0 = tm_of(tile) * BM, n0 = tn_of(tile) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg, stage, lane);
+      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, tn_of(tile) * 128, cptr, ldc, bias, swg, stage, lane);
       else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb, stage, lane);
       else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge, stage, lane);
       else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge, stage, lane);
@@ -813,7 +817,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 int M, int N, int K, void* __restrict__ cptr, int64_t ldc,
                 const __nv_bfloat16* __restrict__ bias, const float* __restrict__ residual, int64_t ldr,
-                int tiles_m, int num_tiles, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb, GeluArgs ge) {
+                int tiles_m, int num_tiles, int n_fast, RopeArgs rope, SwigluArgs swg, SwigluBwdArgs swb, GeluArgs ge) {
+  auto tm_of = [&](int tile) { return n_fast ? tile / n_fast : tile % tiles_m; };      // see gemm_tc_kernel
+  auto tn_of = [&](int tile) { return n_fast ? tile % n_fast : tile / tiles_m; };
   constexpr int S = kStages2;
   constexpr int BN = kBN2;
   extern __shared__ uint8_t smem_raw[];
@@ -859,10 +865,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       uint32_t ph = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-        const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM;
+        const int m0 = tm_of(tile) * (2 * BM) + (int)rank * BM;
         // this CTA's 128 columns of B; gate | up: the first CTA stages the gate rows, the second the up rows
-        const int n0 = (!B_MN && swg.out != nullptr) ? (tile / tiles_m) * 128 + (int)rank * swg.half
-                                                     : (tile / tiles_m) * BN + (int)rank * (BN / 2);
+        const int n0 = (!B_MN && swg.out != nullptr) ? tn_of(tile) * 128 + (int)rank * swg.half
+                                                     : tn_of(tile) * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicCAS(&g_tc_error, 0, 1); ok = false; break; }
           const uint32_t sa = base + s * kStage2Bytes, sb = sa + kABytes;
@@ -928,10 +934,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 3);
       tc_fence_after();
       if (!__all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0)) break;
-      const int m0 = (tile % tiles_m) * (2 * BM) + (int)rank * BM, n0 = (tile / tiles_m) * BN;
+      const int m0 = tm_of(tile) * (2 * BM) + (int)rank * BM, n0 = tn_of(tile) * BN;
       const int m = m0 + q * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kAccStride);
-      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, (tile / tiles_m) * 128, cptr, ldc, bias, swg, stage, lane);
+      if (!OUT_F32 && swg.out != nullptr) epi_row_swiglu(taddr, m, M, tn_of(tile) * 128, cptr, ldc, bias, swg, stage, lane);
       else if (!OUT_F32 && swb.gu != nullptr) epi_row_swiglu_bwd(taddr, BN, m, M, n0, N, cptr, swb, stage, lane);
       else if (!OUT_F32 && ge.out != nullptr) epi_row_gelu_fwd(taddr, BN, m, M, n0, N, cptr, ldc, bias, ge, stage, lane);
       else if (!OUT_F32 && ge.bwd_a != nullptr) epi_row_gelu_bwd(taddr, BN, m, M, n0, N, cptr, ldc, ge, stage, lane);
@@ -1034,7 +1040,7 @@ cudaError_t launch_inst(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
-                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, tc,
+                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, g.M > g.N ? tiles_n : 0, tc,
                             RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
                             SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu},
                             GeluArgs{(__nv_bfloat16*)g.gelu_out, (const __nv_bfloat16*)g.gelu_bwd_a});
@@ -1060,7 +1066,7 @@ cudaError_t launch_pair(cudaStream_t st, const GemmArgs& g, const CUtensorMap& t
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<A_MN, B_MN, OUT_F32>, ta, tb, g.M, g.N, g.K, g.c, g.ldc,
-                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles,
+                            (const __nv_bfloat16*)g.bias, g.residual, g.ldr, tiles_m, num_tiles, g.M > g.N ? tiles_n : 0,
                             RopeArgs{g.rope_cs, g.rope_seq, g.rope_cols}, SwigluArgs{(__nv_bfloat16*)g.swiglu_out, g.N / 2},
                             SwigluBwdArgs{(const __nv_bfloat16*)g.swiglu_bwd_gu},
                             GeluArgs{(__nv_bfloat16*)g.gelu_out, (const __nv_bfloat16*)g.gelu_bwd_a});
