@@ -156,8 +156,7 @@ typedef struct {
  * driver entry point for tensor maps are looked up once per process, for the device that
  * was current at the first call; contexts on two different GPUs in one process are not
  * supported (several contexts on the same GPU are).
- * batch * seq <= 8192: the embedding-gradient kernel keeps the step's token positions in
- * shared memory (HIFT_ERR_CFG beyond it). */
+ * batch * seq <= 65536 tokens a step (HIFT_ERR_CFG beyond it). */
 hift_status hift_create(const hift_model_cfg *model, const hift_group_cfg *groups,
                         const hift_opt_cfg *opt, void *cuda_stream, hift_ctx **out);
 void hift_destroy(hift_ctx *ctx);

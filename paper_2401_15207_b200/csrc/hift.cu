@@ -964,7 +964,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
       src = c->dxb;
     }
     LAUNCH(HIFT_K_EMBED, (double)T * d * 12,
-           embed_bwd_tok_kernel<<<T, 128, T * sizeof(int), c->st>>>(tok, src, c->G(c->t_tok), c->gbf, T, d, V));
+           embed_bwd_tok_kernel<<<T, 128, 0, c->st>>>(tok, src, c->G(c->t_tok), c->gbf, T, d, V));
     if (c->t_pos >= 0) {
       LAUNCH(HIFT_K_EMBED, (double)T * d * 4 + (double)S * d * 4,
              embed_bwd_pos_kernel<<<S, 128, 0, c->st>>>(src, c->G(c->t_pos), c->gbf, B, S, d));
@@ -1259,8 +1259,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (!(m->dropout >= 0.0 && m->dropout < 1.0)) return HIFT_ERR_CFG;
   if (m->arch != 2 && m->max_pos < m->seq) return HIFT_ERR_CFG;
   if (m->arch == 1 && (m->n_classes < 2 || m->tie_head)) return HIFT_ERR_CFG;
-  // the embedding-gradient kernel keeps one occurrence list of <= batch*seq ints in shared memory
-  if ((int64_t)m->batch * m->seq > 8192) return HIFT_ERR_CFG;
+  // several kernels launch one block per token, and the attention grids put the batch on z
+  if ((int64_t)m->batch * m->seq > 65536 || m->batch > 65535) return HIFT_ERR_CFG;
   if (gc->layers_per_group < 1 || gc->order < 0 || gc->order > 2) return HIFT_ERR_CFG;
   if (gc->group_sizes != nullptr) {
     if (gc->n_group_sizes < 1) return HIFT_ERR_CFG;

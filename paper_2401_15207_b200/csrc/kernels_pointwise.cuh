@@ -91,10 +91,13 @@ __device__ __forceinline__ void grad_store(void* g, size_t i, float v, int bf) {
 }
 // grad_tok[id,:] += sum over positions t with ids[t] == id of dx[t,:], occurrences added in
 // increasing t.  Block t does the work for id = ids[t] only if t is the first occurrence, so
-// every gradient row has one writer and a fixed summation order (no atomics).
+// every gradient row has one writer and a fixed summation order (no atomics).  The positions of
+// the id are collected in order into a list of kEmbedOccCap entries; a full list is summed into
+// the gradient row and emptied, so the number of positions is not bounded by shared memory.
+constexpr int kEmbedOccCap = 2048;
 __global__ void embed_bwd_tok_kernel(const int32_t* __restrict__ ids, const float* __restrict__ dx,
                                      void* __restrict__ grad_tok, int gbf, int Ttot, int d, int vocab) {
-  extern __shared__ int occ[];                       // positions of this id, in order
+  __shared__ int occ[kEmbedOccCap];                  // positions of this id, in order
   __shared__ int n_occ;
   __shared__ int warp_cnt[32];
   const int t0 = blockIdx.x;
@@ -106,8 +109,22 @@ __global__ void embed_bwd_tok_kernel(const int32_t* __restrict__ ids, const floa
   if (threadIdx.x == 0) n_occ = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const size_t row = (size_t)id * d;
+  auto drain = [&](int n) {                          // gradient row += the listed positions, in order
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+      float acc = 0.f;
+      for (int i = 0; i < n; ++i) acc += dx[(size_t)occ[i] * d + c];
+      grad_store(grad_tok, row + c, grad_load(grad_tok, row + c, gbf) + acc, gbf);   // on top of a tied head's share
+    }
+  };
   // ordered compaction, one blockDim-sized chunk at a time
   for (int base = t0; base < Ttot; base += blockDim.x) {
+    if (n_occ + (int)blockDim.x > kEmbedOccCap) {    // uniform: n_occ is read after a barrier
+      drain(n_occ);
+      __syncthreads();
+      if (threadIdx.x == 0) n_occ = 0;
+      __syncthreads();
+    }
     const int t = base + threadIdx.x;
     const int hit = (t < Ttot) && (ids[t] == id);
     const unsigned bal = __ballot_sync(0xffffffffu, hit);
@@ -124,13 +141,7 @@ __global__ void embed_bwd_tok_kernel(const int32_t* __restrict__ ids, const floa
     }
     __syncthreads();
   }
-  const int n = n_occ;
-  const size_t row = (size_t)id * d;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    float acc = 0.f;
-    for (int i = 0; i < n; ++i) acc += dx[(size_t)occ[i] * d + c];
-    grad_store(grad_tok, row + c, grad_load(grad_tok, row + c, gbf) + acc, gbf);     // on top of a tied head's share
-  }
+  drain(n_occ);
 }
 
 // grad_pos[s,:] = sum over batch rows b of dx[b*S+s,:]

@@ -802,3 +802,16 @@ def test_gradients_kept_in_bf16(arch, big):
         b.close()
     with pytest.raises(Exception):
         HiFT(cfg.scaled(dtype=synth.DTYPE_FP32), gc, oc)                                 # bf16 gradients need a bf16 model
+
+
+@pytest.mark.parametrize("arch,dtype", [(0, synth.DTYPE_FP32), (2, synth.DTYPE_BF16)])
+def test_embedding_gradient_with_more_tokens_than_one_occurrence_list(arch, dtype):
+    """12288 tokens a step over a vocabulary of 31 ids: the commonest id sits at some thousands of positions,
+    more than the embedding-gradient kernel lists at once, so its row is summed in several passes; the first
+    step of the cycle trains the embedding group."""
+    bf = dtype == synth.DTYPE_BF16
+    cfg = mini(arch, dtype, n_blocks=1, vocab=31, batch=24, seq=512, max_pos=512, tie_head=1 if arch == 0 else 0)
+    tok, _ = synth.batch_for(cfg, 5, 0, "zipf")
+    assert np.bincount(tok.reshape(-1)).max() > 2048
+    lockstep(cfg, synth.GroupCfg(layers_per_group=1, order=0), synth.OptCfg(kind=0, lr=1e-3), 1, "zipf",
+             BF16_LOSS if bf else FP32_LOSS, BF16_GRAD if bf else FP32_GRAD, resync=True)
