@@ -3,9 +3,10 @@
 // the bounded mbarrier waits, the time-out flag and the tensor-map cache.
 //
 // Work item = one (batch, head) and 128 query rows; key blocks of 128.  The kernel is persistent:
-// a CTA walks a list of items, those with the most key blocks first, and the next item's Q tile,
-// first scores and first P V products overlap the normalisation and store of the current item
-// (two Q buffers, two score buffers, two output accumulators).
+// a CTA walks a list of items, those with the most key blocks first; the next item's Q tile and
+// first scores are ready when an item ends (two Q buffers, two score buffers, two output
+// accumulators), and an item's normalisation and store are put off until the softmax warps hold
+// the next item's first exponentials, so that they never wait for the item's last P V product.
 //   warp 0    : TMA producer (Q per item; K and V blocks through two 2-deep rings)
 //   warp 1    : issues S_j = Q K_j^T   (M 128 x N 128, k = d_h)      -> TMEM columns [0,128) / [128,256); owns the tensor memory
 //   warp 2    : issues O += P_j V_j    (M 128 x N d_h, k = 128 keys) -> TMEM columns [256,384) / [384,512) by item parity
@@ -61,6 +62,35 @@ __device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr, uint32_t box_byt
          (1ull << 46) | (2ull << 61);
 }
 
+// A warp's 32 rows x 64 bf16 columns (lane = row) written as whole 128-byte lines: parked in 4 KB of shared memory
+// (16-byte segments XOR-swizzled by row, conflict-free both ways) and written back with eight consecutive lanes on the
+// eight segments of a row, four rows per instruction.  att_stage32 parks 32 of the lane's fp32 values (times `mul`) as
+// segments seg0 .. seg0 + 3 of its row; att_flush64 writes the rows out, skipping rows at or beyond row_end.
+__device__ __forceinline__ void att_stage32(const uint32_t (&v)[32], float mul, uint8_t* __restrict__ stage, int lane, int seg0) {
+  uint8_t* mine = stage + lane * 128;
+#pragma unroll
+  for (int sg = 0; sg < 4; ++sg) {
+    uint4 pk;
+    __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+    for (int t = 0; t < 4; ++t)
+      hp[t] = __floats2bfloat162_rn(__uint_as_float(v[8 * sg + 2 * t]) * mul, __uint_as_float(v[8 * sg + 2 * t + 1]) * mul);
+    *reinterpret_cast<uint4*>(mine + (((seg0 + sg) ^ (lane & 7)) << 4)) = pk;
+  }
+}
+__device__ __forceinline__ void att_flush64(const uint8_t* __restrict__ stage, __nv_bfloat16* __restrict__ dst, int64_t ld, int row,
+                                            int lane, int row_end, int col) {
+  __syncwarp();
+  const int row_base = row - lane, sg = lane & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = 4 * i + (lane >> 3);
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 128 + ((sg ^ (r & 7)) << 4));
+    if (row_base + r < row_end) *reinterpret_cast<uint4*>(dst + (int64_t)(row_base + r) * ld + col + 8 * sg) = v;
+  }
+  __syncwarp();
+}
+
 // Key padding: batch entry b attends to keys 0 .. lens[b]-1 only (clamped to [1, S]); null = all S keys.
 __device__ __forceinline__ int tc_key_len(const int* __restrict__ lens, int b, int S) {
   return lens != nullptr ? max(1, min(lens[b], S)) : S;
@@ -103,10 +133,18 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
   // work items, heaviest first; every role walks the same list and counts key blocks (g)
   const int nqb = (S + kAttBQ - 1) / kAttBQ, nbh = B * H, nitems = nqb * nbh;
   struct Item { int b, h, q0, nblk, klen; };
+  // item indices stay far below 2^24, so a float reciprocal and one correction step divide exactly (an integer
+  // division by a run-time value costs a few hundred cycles of the softmax warps at every item boundary)
+  auto div_small = [](int x, int dv) {
+    int qt = (int)((float)x * __frcp_rn((float)dv));
+    if (qt * dv > x) --qt;
+    else if ((qt + 1) * dv <= x) ++qt;
+    return qt;
+  };
   auto item_of = [&](int idx) {
     Item it;
-    const int rank = idx / nbh, bh = idx - rank * nbh;
-    it.b = bh / H;
+    const int rank = div_small(idx, nbh), bh = idx - rank * nbh;
+    it.b = div_small(bh, H);
     it.h = bh - it.b * H;
     it.q0 = (causal ? nqb - 1 - rank : rank) * kAttBQ;
     it.klen = tc_key_len(lens, it.b, S);                // keys at or after klen are padding
@@ -251,6 +289,45 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
     };
     bool ok = !poisoned;
     int g = 0, n = 0;
+    // The normalisation and store of an item wait for its last P V product, so they are put off until this thread
+    // has the exponentials of the next item's first block in registers: by then the product is long finished, and the
+    // P tile (this warp's rows of it are the staging area of the stores) has not been written for the new item yet.
+    int pend_n = -1, pend_row = 0, pend_end = 0, pend_col = 0;      // pend_n < 0: nothing put off
+    float pend_inv = 0.f;
+    // Whole-line stores: the warp parks each 32 x 32 chunk in shared memory and writes it back with consecutive
+    // lanes on consecutive 16-byte segments of a row (its own 32 rows of its 64-key span of the P tile: 4 KB).
+    auto finish_item = [&]() -> bool {
+      const bool ready = mbar_wait(o_done(pend_n & 1), (uint32_t)((pend_n >> 1) & 1));
+      if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
+      tc_fence_after();
+      if (!__all_sync(0xffffffffu, ready)) return false;
+      const uint32_t tOp = tmem_base + 256u + (uint32_t)((pend_n & 1) * 128);
+      uint8_t* stage = p_gen + half * SPAN_BYTES + (q * 32) * 128;
+      if constexpr (OC == 64) {
+        uint32_t v[32];
+        tmem_ld32(tOp + lane_off + (uint32_t)(half * OC), v);
+        att_stage32(v, pend_inv, stage, lane, 0);
+        tmem_ld32(tOp + lane_off + (uint32_t)(half * OC + 32), v);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(o_free(pend_n & 1));   // everything read: the accumulator may be reused
+        att_stage32(v, pend_inv, stage, lane, 4);
+        att_flush64(stage, o, (int64_t)d, pend_row, lane, pend_end, pend_col);
+      } else {
+        uint32_t v[32];
+        tmem_ld32(tOp + lane_off + (uint32_t)(half * OC), v);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(o_free(pend_n & 1));
+        float f[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) * pend_inv;
+        // rows at or beyond the batch entry's sequence end are skipped
+        epi_store32_lines<false>(f, stage, o, (int64_t)d, pend_row, lane, pend_end, pend_col, nullptr);
+      }
+      pend_n = -1;
+      return true;
+    };
     for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
       const Item it = item_of(idx);
       const int q0 = it.q0, qrow = q0 + r, row_g0 = it.b * S, klen = it.klen;
@@ -315,6 +392,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
           for (int e = 0; e < 4; ++e) { sc[i + e] = ex2_approx(fmaf(sc[i + e], sl2, nmuse)); sum4[e] += sc[i + e]; }
         }
         l = l * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+        if (pend_n >= 0) {                              // the previous item's output (uniform across the CTA)
+          ok = finish_item();
+          if (!ok) { pair_release(); break; }
+        }
         // the previous P V product must be finished before P is overwritten and O is rescaled
         ready = mbar_wait(p_free, (uint32_t)((g & 1) ^ 1));
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
@@ -352,39 +433,14 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       pair_sync();
       const float ltot = l + xch[r * 2 + (half ^ 1)];
       pair_sync();
-      // last product of the item done -> normalise and store
-      {
-        const bool ready = mbar_wait(o_done(n & 1), (uint32_t)((n >> 1) & 1));
-        if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 6);
-        tc_fence_after();
-        ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
-        if (!ok) { pair_release(); break; }
-      }
-      const float inv = 1.0f / ltot;
-      __nv_bfloat16* orow = o + ((int64_t)(row_g0 + qrow)) * d + (int64_t)it.h * DH + half * OC;
-#pragma unroll 1
-      for (int c0 = 0; c0 < OC; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(tO + lane_off + (uint32_t)(half * OC + c0), v);
-        if (c0 + 32 >= OC) {                            // everything read: the accumulator may be reused
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(o_free(n & 1));
-        }
-        if (qrow < S) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 pk;
-            __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-            for (int t = 0; t < 4; ++t)
-              hp[t] = __floats2bfloat162_rn(__uint_as_float(v[i + 2 * t]) * inv, __uint_as_float(v[i + 2 * t + 1]) * inv);
-            *reinterpret_cast<uint4*>(orow + c0 + i) = pk;
-          }
-        }
-      }
       if (half == 0 && qrow < S) lse[((int64_t)it.b * H + it.h) * S + qrow] = (m + log2f(ltot)) * 0.6931471805599453f;
+      pend_n = n;
+      pend_inv = 1.0f / ltot;
+      pend_row = row_g0 + qrow;
+      pend_end = row_g0 + S;
+      pend_col = it.h * DH + half * OC;
     }
+    if (ok && pend_n >= 0) finish_item();                      // the last item of this CTA
   }
   tc_fence_before();
   __syncthreads();
