@@ -373,7 +373,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
         const bool ready = mbar_wait(acc_done, (uint32_t)(n & 1));
         if (!ready && lane == 0) atomicCAS(&g_tc_error, 0, 9);
         tc_fence_after();
-        ok = __all_sync(0xffffffffu, ready && *(volatile int*)&g_tc_error == 0);
+        ok = __all_sync(0xffffffffu, ready);              // a role that gave up leaves acc_done unset
         if (!ok) break;
       }
       constexpr int CW = DH / 4;                          // 16 or 32
@@ -392,31 +392,49 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_free);               // the next item may overwrite the accumulators
-      if (frow < S) {
-        // dS-fed accumulator, scaled: dK -> column block d (MODE 0) or dQ -> column block 0 (MODE 1); dV -> block 2d
-        __nv_bfloat16* orow = dqkv + ((int64_t)(row_g0 + frow)) * (3 * d) + (int64_t)it.h * DH + part * CW;
-        __nv_bfloat16* dst0 = orow + (MODE == 0 ? d : 0);
+      // dS-fed accumulator, scaled: dK -> column block d (MODE 0) or dQ -> column block 0 (MODE 1); dV -> block 2d.
+      // A thread that stored its own row would put 16 bytes into each of 32 lines per instruction, and the store path
+      // charges per line.  So the warp parks its 32 rows x CW columns in shared memory, in the 16-byte chunks of the
+      // dS (and P) tile of its group that only this warp ever writes (rows r, chunks 4 hc ..): every product that read
+      // them is finished (acc_done), and their next writer is this warp, after this block.  It then writes them back
+      // with NSEG consecutive lanes on the NSEG segments of a row, 32 / NSEG rows per instruction.
+      {
+        constexpr int NSEG = CW / 8;                      // 16-byte segments per row: 4 (d_h 128) or 2 (d_h 64)
+        constexpr int RPI = 32 / NSEG;                    // rows per store instruction
+        uint8_t* tile0 = p_gen + pb * NP * Cfg::kPBytes;  // dS tile of this group; the P tile follows it (MODE 0)
+        uint8_t* mine = tile0 + r * 128;
 #pragma unroll
-        for (int i = 0; i < CW; i += 8) {
+        for (int sgm = 0; sgm < NSEG; ++sgm) {
           uint4 pk;
           __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
           for (int e = 0; e < 4; ++e)
-            hp[e] = __floats2bfloat162_rn(__uint_as_float(v0[i + 2 * e]) * scale, __uint_as_float(v0[i + 2 * e + 1]) * scale);
-          *reinterpret_cast<uint4*>(dst0 + i) = pk;
-        }
-        if (MODE == 0) {
-          __nv_bfloat16* dst1 = orow + 2 * d;
-#pragma unroll
-          for (int i = 0; i < CW; i += 8) {
-            uint4 pk;
-            __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&pk);
+            hp[e] = __floats2bfloat162_rn(__uint_as_float(v0[8 * sgm + 2 * e]) * scale, __uint_as_float(v0[8 * sgm + 2 * e + 1]) * scale);
+          *reinterpret_cast<uint4*>(mine + (((hc * 4 + sgm) ^ (r & 7)) << 4)) = pk;
+          if (MODE == 0) {
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-              hp[e] = __floats2bfloat162_rn(__uint_as_float(v1[i + 2 * e]), __uint_as_float(v1[i + 2 * e + 1]));
-            *reinterpret_cast<uint4*>(dst1 + i) = pk;
+              hp[e] = __floats2bfloat162_rn(__uint_as_float(v1[8 * sgm + 2 * e]), __uint_as_float(v1[8 * sgm + 2 * e + 1]));
+            *reinterpret_cast<uint4*>(mine + Cfg::kPBytes + (((hc * 4 + sgm) ^ (r & 7)) << 4)) = pk;
           }
         }
+        __syncwarp();
+        const int sgm = lane % NSEG;
+        __nv_bfloat16* obase = dqkv + (int64_t)it.h * DH + part * CW + 8 * sgm;
+#pragma unroll
+        for (int i = 0; i < NSEG; ++i) {
+          const int rr = q * 32 + i * RPI + lane / NSEG;  // row of the fixed tile
+          const uint8_t* src = tile0 + rr * 128 + (((hc * 4 + sgm) ^ (rr & 7)) << 4);
+          const uint4 a0 = *reinterpret_cast<const uint4*>(src);
+          uint4 a1 = a0;
+          if (MODE == 0) a1 = *reinterpret_cast<const uint4*>(src + Cfg::kPBytes);
+          if (f0 + rr < S) {
+            __nv_bfloat16* orow = obase + ((int64_t)(row_g0 + f0 + rr)) * (3 * d);
+            *reinterpret_cast<uint4*>(orow + (MODE == 0 ? d : 0)) = a0;
+            if (MODE == 0) *reinterpret_cast<uint4*>(orow + 2 * d) = a1;
+          }
+        }
+        __syncwarp();
       }
     }
   }
