@@ -598,6 +598,41 @@ def run_micro(args, cfg):
                          "peak_hbm_gb": round(h.peak_hbm_bytes() / 1e9, 2)})
         finally:
             h.close()
+    elif args.micro == "sdpa":
+        # Context for the attention numbers: the vendor kernels behind torch's scaled_dot_product_attention (cuDNN and
+        # flash back ends) at the workload's attention shape, timed like this library's kernels beside them.  Nothing
+        # else in this repository calls them.
+        import torch.nn.functional as F
+        from torch.nn.attention import sdpa_kernel, SDPBackend
+        Bt, S, H, dh, causal = cfg.batch, cfg.seq, cfg.n_heads, cfg.d_model // cfg.n_heads, bool(cfg.causal)
+        d = H * dh
+        T = Bt * S
+        qkv = torch.randn(T, 3 * d, device="cuda").to(bf)
+        o = torch.empty(T, d, device="cuda", dtype=bf)
+        lse = torch.empty(Bt * H * S, device="cuda")
+        do = torch.randn(T, d, device="cuda").to(bf)
+        dqkv = torch.empty(T, 3 * d, device="cuda", dtype=bf)
+        dsum = torch.empty(T * H, device="cuda")
+        fl = 4.0 * Bt * H * S * S * dh * (0.5 if causal else 1.0)
+        us_f = timed(lambda: B.k_attention_fwd(1, Bt, S, H, dh, int(causal), qkv, o, lse))
+        us_b = timed(lambda: B.k_attention_bwd(1, Bt, S, H, dh, int(causal), qkv, o, lse, do, dqkv, dsum))
+        rows.append({"impl": "this library", "fwd_us": round(us_f, 2), "bwd_us": round(us_b, 2),
+                     "fwd_tflops": round(fl / us_f / 1e6, 1), "bwd_tflops": round(2.5 * fl / us_b / 1e6, 1)})
+        q, k, v = (torch.randn(Bt, H, S, dh, device="cuda", dtype=bf, requires_grad=True) for _ in range(3))
+        for name, be in (("torch sdpa, cuDNN back end", SDPBackend.CUDNN_ATTENTION), ("torch sdpa, flash back end", SDPBackend.FLASH_ATTENTION)):
+            try:
+                with sdpa_kernel(be):
+                    with torch.no_grad():
+                        us_f = timed(lambda: F.scaled_dot_product_attention(q, k, v, is_causal=causal))
+                    out = F.scaled_dot_product_attention(q, k, v, is_causal=causal)
+                    g = torch.randn_like(out)
+                    # autograd.grad: no accumulation kernels into .grad beside the backward kernel itself
+                    us_b = timed(lambda: torch.autograd.grad(out, (q, k, v), g, retain_graph=True))
+                rows.append({"impl": name, "fwd_us": round(us_f, 2), "bwd_us": round(us_b, 2),
+                             "fwd_tflops": round(fl / us_f / 1e6, 1), "bwd_tflops": round(2.5 * fl / us_b / 1e6, 1)})
+            except Exception as e:
+                rows.append({"impl": name, "unavailable": str(e)[:160]})
+        rows.append({"shape": f"batch {Bt} x seq {S} x {H} heads x {dh}, causal={int(causal)}", "flops_fwd": fl})
     else:
         rows = [dict(kernel=k, **v) for k, v in standalone_kernels(cfg, peaks, launches=n_l).items()]
     print(json.dumps({"micro": args.micro, "workload": args.workload, "launches": n_l,
@@ -777,7 +812,7 @@ def main():
                     help="leave out the k = 1 full-parameter step of the same model (needs ~132 GB at the 7B shape)")
     ap.add_argument("--sweep", default=None, choices=["optimizer", "depth"],
                     help="kernel sweeps instead of the step benchmark")
-    ap.add_argument("--micro", default=None, choices=["gemm", "kernels", "step"],
+    ap.add_argument("--micro", default=None, choices=["gemm", "kernels", "step", "sdpa"],
                     help="single kernels at the workload's shapes, a few launches each (small enough for an ncu capture)")
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--only", default=None, help="--micro gemm: only shapes whose name contains this")

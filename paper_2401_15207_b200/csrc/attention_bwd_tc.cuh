@@ -152,7 +152,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
   const bool poisoned = g_tc_error != 0;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < NF; ++i) { mbar_init(f_full(i), 1); mbar_init(f_empty(i), 2); }      // freed by both issuers
+    for (int i = 0; i < NF; ++i) { mbar_init(f_full(i), 1); mbar_init(f_empty(i), 1); }      // freed by the score issuer: only its products read them
     for (int i = 0; i < XS; ++i) { mbar_init(x_full(i), 1); mbar_init(x_empty(i), 2); }
     for (int i = 0; i < 2; ++i) { mbar_init(s_full(i), 1); mbar_init(s_free(i), kAbEwWarps / 2); }   // one group of warps each
     for (int i = 0; i < NPB; ++i) { mbar_init(p_ready(i), kAbEwWarps / 2); mbar_init(p_free(i), 1); }
@@ -184,7 +184,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
         const Item it = item_of(idx);
         const int row_g0 = it.b * S;
-        // this set of fixed tiles is free once every product of the item that used it has completed
+        // this set of fixed tiles is free once the last score product of the item that used it has completed (the
+        // accumulating products read the streamed tiles and P / dS only), a step or two before that item ends
         const int fi = n % NF;
         if (!mbar_wait(f_empty(fi), (uint32_t)(((n / NF) & 1) ^ 1))) { atomicCAS(&g_tc_error, 0, 7); break; }
         const uint32_t sF0 = sF + fi * 2 * Cfg::kFBytes, sF1 = sF0 + Cfg::kFBytes;
@@ -276,10 +277,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
           tc_commit(p_free(pb));
           tc_commit(x_empty(st));
         }
-        if (ok) {
-          tc_commit(acc_done);
-          tc_commit(f_empty(n % NF));
-        }
+        if (ok) tc_commit(acc_done);
       }
     }
   } else {
