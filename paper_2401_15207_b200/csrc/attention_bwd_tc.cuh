@@ -149,6 +149,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
     it.nsteps = x_hi - x_lo;
     return it;
   };
+  // The n-th item of this CTA.  The list is sorted by weight, so handing it out forwards on even rounds and backwards
+  // on odd ones pairs a CTA's heavy items with light ones (plain round-robin gave the first CTAs the heaviest item of
+  // every round: 10 key blocks against a mean of 8.65 at batch 4 x 512 x 32 heads, causal).
+  auto item_at = [&](int n) {
+    const int first = n * (int)gridDim.x;
+    return (n & 1) ? first + (int)gridDim.x - 1 - (int)blockIdx.x : first + (int)blockIdx.x;
+  };
   const bool poisoned = g_tc_error != 0;
 
   if (threadIdx.x == 0) {
@@ -181,7 +188,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       uint32_t ph = 0;
       bool ok = true;
       int n = 0;
-      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
         const Item it = item_of(idx);
         const int row_g0 = it.b * S;
         // this set of fixed tiles is free once the last score product of the item that used it has completed (the
@@ -217,7 +224,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAbX >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       int n = 0, g = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
         const Item it = item_of(idx);
         const int fi = n % NF;
         if (!mbar_wait(f_full(fi), (uint32_t)((n / NF) & 1))) { atomicCAS(&g_tc_error, 0, 8); break; }
@@ -253,7 +260,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       const uint32_t idesc_a = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       int n = 0, g = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
         const Item it = item_of(idx);
         for (int t = 0; t < it.nsteps; ++t, ++g) {
           const int st = g % XS, pb = g % NPB;
@@ -293,7 +300,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
     const int u = grp, pb = grp;                          // this group's tS / tP buffer and P / dS buffer
     bool ok = !poisoned;
     int g0 = 0, n = 0;
-    for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+    for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
       const Item it = item_of(idx);
       const int f0 = it.f0, row_g0 = it.b * S;
       const int frow = f0 + r;                            // key (MODE 0) / query (MODE 1) index in the sequence

@@ -152,6 +152,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
     it.nblk = (kv_len + kAttBK - 1) / kAttBK;
     return it;
   };
+  // The n-th item of this CTA.  The list is sorted by weight, so handing it out forwards on even rounds and backwards
+  // on odd ones pairs a CTA's heavy items with light ones (plain round-robin gave the first CTAs the heaviest item of
+  // every round: 10 key blocks against a mean of 8.65 at batch 4 x 512 x 32 heads, causal).
+  auto item_at = [&](int n) {
+    const int first = n * (int)gridDim.x;
+    return (n & 1) ? first + (int)gridDim.x - 1 - (int)blockIdx.x : first + (int)blockIdx.x;
+  };
   // one thread reads the time-out flag and the CTA shares the answer: the softmax warps meet at named
   // barriers in pairs, so they must all take the same way
   volatile uint32_t* poison_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot + 8u - base));
@@ -186,7 +193,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
     if (lane == 0 && !poisoned) {
       int g = 0, n = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
         const Item it = item_of(idx);
         const int row_g0 = it.b * S;                    // first row of this batch entry in qkv
         const int colQ = it.h * DH, colK = d + it.h * DH, colV = 2 * d + it.h * DH;
@@ -219,7 +226,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAttBK >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       int g = 0, n = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
         const Item it = item_of(idx);
         const int qi = n & 1;
         if (!mbar_wait(q_full(qi), (uint32_t)((n >> 1) & 1))) { atomicCAS(&g_tc_error, 0, 5); break; }
@@ -248,7 +255,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       int g = 0, n = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+      for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
         const Item it = item_of(idx);
         const uint32_t tO = tmem_base + 256u + (uint32_t)((n & 1) * 128);
         for (int j = 0; j < it.nblk; ++j, ++g) {
@@ -328,7 +335,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       pend_n = -1;
       return true;
     };
-    for (int idx = blockIdx.x; idx < nitems && ok; idx += gridDim.x, ++n) {
+    for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
       const Item it = item_of(idx);
       const int q0 = it.q0, qrow = q0 + r, row_g0 = it.b * S, klen = it.klen;
       const uint32_t tO = tmem_base + 256u + (uint32_t)((n & 1) * 128);
