@@ -300,25 +300,46 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
     const int u = grp, pb = grp;                          // this group's tS / tP buffer and P / dS buffer
     bool ok = !poisoned;
     int g0 = 0, n = 0;
+    // What an item needs before its first step (its description, the key length of its batch entry, and the first lse /
+    // D values: MODE 1 this query's, MODE 0 those of the first step's columns) is fetched while the previous item's last
+    // products finish, so that no global load stands between two items.
+    struct Pre { Item it; int klen; float a, b; };
+    auto prepare = [&](int idx, int g0v) {
+      Pre p;
+      p.a = 0.f; p.b = 0.f;
+      p.it = item_of(idx);
+      p.klen = tc_key_len(lens, p.it.b, S);
+      const float* lse_p = lse + ((int64_t)p.it.b * H + p.it.h) * S;
+      const float* dsum_p = dsum + ((int64_t)p.it.b * H + p.it.h) * S;
+      if (MODE == 1) {
+        const int qi = min(p.it.f0 + r, S - 1);
+        p.a = lse_p[qi] * 1.4426950408889634f;
+        p.b = dsum_p[qi];
+      } else {
+        const int t1 = (g0v ^ grp) & 1;
+        if (t1 < p.it.nsteps) {
+          const int c = min((p.it.x_lo + t1) * kAbX + hc * 32 + lane, S - 1);
+          p.a = lse_p[c];
+          p.b = dsum_p[c];
+        }
+      }
+      return p;
+    };
+    Pre cur;
+    if (item_at(0) < nitems && ok) cur = prepare(item_at(0), 0);
     for (int idx = item_at(n); idx < nitems && ok; idx = item_at(++n)) {
-      const Item it = item_of(idx);
+      const Item it = cur.it;
       const int f0 = it.f0, row_g0 = it.b * S;
       const int frow = f0 + r;                            // key (MODE 0) / query (MODE 1) index in the sequence
-      const int klen = tc_key_len(lens, it.b, S);         // keys at or after klen are padding: P = dS = 0 there
+      const int klen = cur.klen;                          // keys at or after klen are padding: P = dS = 0 there
       const float* lse_bh = lse + ((int64_t)it.b * H + it.h) * S;
       const float* dsum_bh = dsum + ((int64_t)it.b * H + it.h) * S;
-      float row_l2 = 0.f, row_d = 0.f;                    // MODE 1: this query's lse * log2(e) and D
-      if (MODE == 1) {
-        const int qi = min(frow, S - 1);
-        row_l2 = lse_bh[qi] * 1.4426950408889634f;
-        row_d = dsum_bh[qi];
-      }
+      const float row_l2 = cur.a, row_d = cur.b;          // MODE 1: this query's lse * log2(e) and D
       // MODE 0: lane i holds lse and D of column x0 + i of this thread's 32 columns; the values of
       // the group's next step are fetched while this step is worked on
       const int t_first = (g0 ^ grp) & 1;                 // first step of this item with (g & 1) == grp
       auto col_index = [&](int t) { return min((it.x_lo + t) * kAbX + hc * 32 + lane, S - 1); };
-      float lse_next = 0.f, d_next = 0.f;
-      if (MODE == 0 && t_first < it.nsteps) { lse_next = lse_bh[col_index(t_first)]; d_next = dsum_bh[col_index(t_first)]; }
+      float lse_next = cur.a, d_next = cur.b;
       for (int t = t_first; t < it.nsteps; t += 2) {
         const int g = g0 + t;
         const uint32_t par = (uint32_t)((g >> 1) & 1);
@@ -373,6 +394,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
       }
       if (!ok) break;
       g0 += it.nsteps;
+      if (item_at(n + 1) < nitems) cur = prepare(item_at(n + 1), g0);     // `it` and its values above are copies
       // ---------------- accumulators -> global: this thread stores DH/4 columns of its row
       {
         const bool ready = mbar_wait(acc_done, (uint32_t)(n & 1));
