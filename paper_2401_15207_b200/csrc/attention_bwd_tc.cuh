@@ -156,7 +156,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
     const int first = n * (int)gridDim.x;
     return (n & 1) ? first + (int)gridDim.x - 1 - (int)blockIdx.x : first + (int)blockIdx.x;
   };
-  const bool poisoned = g_tc_error != 0;
+  // one thread reads the time-out flag, after griddepcontrol.wait, and the CTA shares the answer: every role must take the same way
+  volatile uint32_t* poison_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot + 8u - base));
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NF; ++i) { mbar_init(f_full(i), 1); mbar_init(f_empty(i), 1); }      // freed by the score issuer: only its products read them
@@ -166,6 +167,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
     mbar_init(acc_done, 1);
     mbar_init(acc_free, kAbEwWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pdl_wait();                                          // no global access before it, the flag included
+    *poison_gen = g_tc_error != 0 ? 1u : 0u;
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
@@ -175,6 +178,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_gen;
+  const bool poisoned = *poison_gen != 0;
   pdl_trigger();
   pdl_wait();                                          // the set-up above may run under the predecessor's tail
   // tensor-memory columns: tS[u] at 64u, tP[u] at 128 + 64u, accumulators from 256

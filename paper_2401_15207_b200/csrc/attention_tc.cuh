@@ -164,7 +164,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
   volatile uint32_t* poison_gen = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot + 8u - base));
 
   if (threadIdx.x == 0) {
-    *poison_gen = g_tc_error != 0 ? 1u : 0u;
     for (int i = 0; i < 2; ++i) {
       mbar_init(q_full(i), 1); mbar_init(q_empty(i), 1);
       mbar_init(k_full(i), 1); mbar_init(k_empty(i), 1);
@@ -175,6 +174,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
     mbar_init(p_ready, 8);                              // one arrival per softmax warp
     mbar_init(p_free, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pdl_wait();                                         // no global access before it, the flag included
+    *poison_gen = g_tc_error != 0 ? 1u : 0u;
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
