@@ -355,7 +355,7 @@ def test_gpt2_large_full_size_invariants():
 
 # ------------------------------------------------------------------ config 2 at full size, against the oracle
 def test_roberta_base_full_size_one_cycle_top2down():
-    """The RoBERTa-base-shaped configuration as BASELINE states it (12 post-LN blocks, d 768, 12 heads, GELU 3072,
+    """The RoBERTa-base-shaped benchmark configuration (12 post-LN blocks, d 768, 12 heads, GELU 3072,
     vocabulary 50265, batch 16 x 128, one unit per group, top2down, AdamW 2e-5 with the linear schedule): one full
     cycle of 14 steps in lockstep with the fp64 oracle - group choice and learning rate exact, loss within 1e-2,
     every gradient tensor of the active group within 2e-2, frozen bits untouched, and the in-step update from the
