@@ -204,12 +204,14 @@ def test_attention_forward_backward(dtype, dh, causal):
 
 
 @pytest.mark.parametrize("dh", [64, 128])
-@pytest.mark.parametrize("B,S,H", [(1, 1, 1), (1, 64, 2), (3, 129, 1), (2, 300, 2), (1, 640, 1)])
+@pytest.mark.parametrize("B,S,H", [(1, 1, 1), (1, 64, 2), (3, 129, 1), (2, 300, 2), (1, 640, 1), (6, 300, 26)])
 @pytest.mark.parametrize("causal", [0, 1])
 def test_attention_tensor_core_edge_lengths(dh, B, S, H, causal):
     """bf16 attention on the tensor-core kernels at the degenerate and ragged sequence lengths: a single
     position, exactly one tile, one row past a tile, several tiles with a tail, more tiles than a CTA's
-    double buffers; batch entries that share a tile with their neighbour."""
+    double buffers; batch entries that share a tile with their neighbour; and more work items than SMs with a
+    ragged tail (468 items: every CTA takes several, so an item's output is stored while the next one runs, and
+    the last tile of every entry skips rows that belong to its neighbour)."""
     import torch
     from paper_2401_15207_b200 import k_attention_fwd, k_attention_bwd
     d = H * dh
