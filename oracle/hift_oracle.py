@@ -247,8 +247,10 @@ def rope_apply(x, cos, sin, inverse=False):
     return np.concatenate([x1 * c - x2 * s, x1 * s + x2 * c], axis=-1)
 
 
-def attention_fwd(q, k, v, causal: bool, lens=None):
+def attention_fwd(q, k, v, causal: bool, lens=None, pmask=None):
     """q,k,v: [B, S, H, d_h] -> o [B, S, H, d_h]; softmax(q k^T / sqrt(d_h) + mask) v.
+    pmask (optional, [B, H, S, S]): dropout multipliers of the probabilities (0 or 1 / (1 - p)),
+    applied after the softmax: o = (softmax o pmask) v; the returned p is the softmax itself.
     lens (optional, [B] ints in 1..S): batch entry b is a sequence of lens[b] real
     tokens padded on the right; keys at positions >= lens[b] get probability 0
     (the usual key-padding mask of the models the paper fine-tunes; the paper
@@ -265,15 +267,21 @@ def attention_fwd(q, k, v, causal: bool, lens=None):
     s = s - s.max(axis=-1, keepdims=True)
     p = np.exp(s)
     p = p / p.sum(axis=-1, keepdims=True)
-    o = np.matmul(p, vh).transpose(0, 2, 1, 3)
+    pd = p if pmask is None else p * pmask
+    o = np.matmul(pd, vh).transpose(0, 2, 1, 3)
     return o, p
 
 
-def attention_bwd(do, q, k, v, p):
+def attention_bwd(do, q, k, v, p, pmask=None):
+    """Backward of attention_fwd; with pmask, o = (p o pmask) v: dv takes the dropped probabilities and the
+    gradient of the softmax output is (do v^T) o pmask."""
     B, S, H, dh = q.shape
     qh, kh, vh, doh = (t.transpose(0, 2, 1, 3) for t in (q, k, v, do))
-    dv = np.matmul(p.transpose(0, 1, 3, 2), doh)
+    pd = p if pmask is None else p * pmask
+    dv = np.matmul(pd.transpose(0, 1, 3, 2), doh)
     dp = np.matmul(doh, vh.transpose(0, 1, 3, 2))
+    if pmask is not None:
+        dp = dp * pmask
     ds = p * (dp - (dp * p).sum(axis=-1, keepdims=True))
     dq = np.matmul(ds, kh) / math.sqrt(dh)
     dk = np.matmul(ds.transpose(0, 1, 3, 2), qh) / math.sqrt(dh)
@@ -305,8 +313,11 @@ def cross_entropy(logits, labels):
 # SC'11), key = the 64-bit seed, counter = (element // 4 as two words, site, step), word element % 4
 # of the output.  An element is kept iff its word >= floor(p * 2^32), and kept values are scaled by
 # 1 / (1 - p).  Sites: 0 = embedding output; 1 + 2 i = output of block i's attention projection and
-# 2 + 2 i = output of its feed-forward network, each before the residual addition.  Attention
-# probabilities are not dropped.
+# 2 + 2 i = output of its feed-forward network, each before the residual addition; 1000 + i = the
+# attention probabilities of block i (after the softmax, before the product with V, as the models'
+# usual implementations do it), with their own rate.  The probabilities' elements are numbered
+# ((b H + h) S + q) S' + k with S' = S rounded up to a multiple of 4, so that the four words of one
+# generator block always belong to one query row.
 _PHILOX_M0, _PHILOX_M1, _PHILOX_W0, _PHILOX_W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
 
 
@@ -378,7 +389,9 @@ def _merge_heads(t):
 
 def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarray, lens=None, drop=None):
     """Whole-model forward in fp64.  Returns (loss, cache).
-    drop = (p, seed, step): dropout with the counter-based masks of dropout_mask; None: no dropout."""
+    drop = (p, seed, step) or (p, seed, step, p_attn): dropout with the counter-based masks of dropout_mask
+    (p at the residual-branch outputs and the embedding output, p_attn on the attention probabilities);
+    None: no dropout."""
     B, S = tokens.shape
     d, H = cfg.d_model, cfg.n_heads
     dh = d // H
@@ -390,6 +403,12 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
         if drop is None or drop[0] <= 0.0:
             return 1.0
         return dropout_mask(B * S * d, drop[0], drop[1], site, drop[2]).reshape(B, S, d)
+
+    def pmask(i):
+        if drop is None or len(drop) < 4 or drop[3] <= 0.0:
+            return None
+        Sp = (S + 3) // 4 * 4
+        return dropout_mask(B * H * S * Sp, drop[3], drop[1], 1000 + i, drop[2]).reshape(B, H, S, Sp)[..., :S]
 
     x = P["tok_emb"][tokens]                                   # [B,S,d]
     if cfg.arch in (0, 1):
@@ -408,7 +427,8 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             h1, c["ln1"] = layernorm_fwd(x, P[p + "ln1_g"], P[p + "ln1_b"], eps)
             qkv = h1 @ P[p + "w_qkv"].T + P[p + "b_qkv"]
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
-            o, prob = attention_fwd(q, k, v, causal, lens)
+            c["pmask"] = pmask(i)
+            o, prob = attention_fwd(q, k, v, causal, lens, c["pmask"])
             om = _merge_heads(o)
             c["mask_a"], c["mask_f"] = mask(1 + 2 * i), mask(2 + 2 * i)
             x2 = x + (om @ P[p + "w_o"].T + P[p + "b_o"]) * c["mask_a"]
@@ -421,7 +441,8 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
         elif cfg.arch == 1:        # post-LN: x = LN1(x + Attn x); x = LN2(x + FFN x)
             qkv = x @ P[p + "w_qkv"].T + P[p + "b_qkv"]
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
-            o, prob = attention_fwd(q, k, v, causal, lens)
+            c["pmask"] = pmask(i)
+            o, prob = attention_fwd(q, k, v, causal, lens, c["pmask"])
             om = _merge_heads(o)
             c["mask_a"], c["mask_f"] = mask(1 + 2 * i), mask(2 + 2 * i)
             y = x + (om @ P[p + "w_o"].T + P[p + "b_o"]) * c["mask_a"]
@@ -438,7 +459,8 @@ def forward(cfg, P: Dict[str, np.ndarray], tokens: np.ndarray, labels: np.ndarra
             q, k, v = (_split_heads(t, H) for t in np.split(qkv, 3, axis=-1))
             q = rope_apply(q, cos, sin)
             k = rope_apply(k, cos, sin)
-            o, prob = attention_fwd(q, k, v, causal, lens)
+            c["pmask"] = pmask(i)
+            o, prob = attention_fwd(q, k, v, causal, lens, c["pmask"])
             om = _merge_heads(o)
             c["mask_a"], c["mask_f"] = mask(1 + 2 * i), mask(2 + 2 * i)
             x2 = x + (om @ P[p + "w_o"].T) * c["mask_a"]
@@ -554,7 +576,7 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             if on:
                 G[p + "w_o"] = _rows(dao).T @ _rows(c["om"])
                 G[p + "b_o"] = _rows(dao).sum(axis=0)
-            dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"])
+            dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"], c.get("pmask"))
             dqkv = np.concatenate([_merge_heads(t) for t in (dq, dk, dv)], axis=-1)
             dh1 = dqkv @ P[p + "w_qkv"]
             if on:
@@ -588,7 +610,7 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             if on:
                 G[p + "w_o"] = _rows(dao).T @ _rows(c["om"])
                 G[p + "b_o"] = _rows(dao).sum(axis=0)
-            dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"])
+            dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"], c.get("pmask"))
             dqkv = np.concatenate([_merge_heads(t) for t in (dq, dk, dv)], axis=-1)
             if on:
                 G[p + "w_qkv"] = _rows(dqkv).T @ _rows(c["xin"])
@@ -615,7 +637,7 @@ def backward(cfg, P, cache, active_units: Optional[Sequence[int]] = None) -> Dic
             dom = dao @ P[p + "w_o"]
             if on:
                 G[p + "w_o"] = _rows(dao).T @ _rows(c["om"])
-            dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"])
+            dq, dk, dv = attention_bwd(_split_heads(dom, H), c["q"], c["k"], c["v"], c["p"], c.get("pmask"))
             dq = rope_apply(dq, cos, sin, inverse=True)
             dk = rope_apply(dk, cos, sin, inverse=True)
             dqkv = np.concatenate([_merge_heads(t) for t in (dq, dk, dv)], axis=-1)
@@ -763,8 +785,8 @@ class HiFTOracle:
         g = self.active_group()
         lr = self.current_lr()
         P = self.model_params()
-        pdrop = float(getattr(self.cfg, "dropout", 0.0))
-        drop = (pdrop, int(getattr(self.cfg, "dropout_seed", 0)), self.t) if pdrop > 0.0 else None
+        pdrop, padrop = float(getattr(self.cfg, "dropout", 0.0)), float(getattr(self.cfg, "attn_dropout", 0.0))
+        drop = (pdrop, int(getattr(self.cfg, "dropout_seed", 0)), self.t, padrop) if max(pdrop, padrop) > 0.0 else None
         loss, cache = forward(self.cfg, P, tokens, labels, lens, drop)
         grads = backward(self.cfg, P, cache, active_units=self.groups[g])
         o = self.ocfg

@@ -54,6 +54,7 @@ class ModelCfg:
     seq: int = 1
     dropout: float = 0.0               # probability of dropping an element at the residual-branch outputs and the embedding output
     dropout_seed: int = 0
+    attn_dropout: float = 0.0          # probability of dropping an attention probability (after the softmax)
 
     @property
     def n_units(self) -> int:

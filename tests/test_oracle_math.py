@@ -133,6 +133,59 @@ def test_fd_with_dropout(arch):
     _fd_check(mini(arch), n_samples=3, drop=(0.25, 77, 3))
 
 
+@pytest.mark.parametrize("arch", [0, 1, 2])
+def test_fd_with_attention_probability_dropout(arch):
+    """The same with the attention probabilities dropped as well (their own rate, sites 1000 + block): finite
+    differences through o = (softmax o mask) v and its backward pass."""
+    _fd_check(mini(arch), n_samples=3, drop=(0.1, 77, 3, 0.3))
+    _fd_check(mini(arch), n_samples=2, drop=(0.0, 78, 1, 0.25))
+
+
+def test_attention_probability_dropout_by_loops_and_its_element_numbering():
+    """Attention with a probability mask against plain loops over (batch, head, query, key), forward and backward;
+    and the mask the model draws: element ((b H + h) S + q) S' + k of site 1000 + block, S' = S rounded up to 4."""
+    rng = np.random.default_rng(9)
+    B, S, H, dh = 2, 5, 3, 4
+    q, k, v, do = (rng.standard_normal((B, S, H, dh)) for _ in range(4))
+    pm = np.where(rng.random((B, H, S, S)) < 0.3, 0.0, 1.0 / 0.7)
+    for causal in (False, True):
+        o, p = O.attention_fwd(q, k, v, causal, None, pm)
+        dq, dk, dv = O.attention_bwd(do, q, k, v, p, pm)
+        o_ref, dq_ref, dk_ref, dv_ref = (np.zeros((B, S, H, dh)) for _ in range(4))
+        for b in range(B):
+            for h in range(H):
+                for i in range(S):
+                    keys = range(i + 1) if causal else range(S)
+                    sc = np.array([q[b, i, h] @ k[b, j, h] / np.sqrt(dh) for j in keys])
+                    pr = np.exp(sc - sc.max()); pr /= pr.sum()
+                    dp = np.array([(do[b, i, h] @ v[b, j, h]) * pm[b, h, i, j] for j in keys])
+                    ds = pr * (dp - (dp * pr).sum())
+                    for n, j in enumerate(keys):
+                        o_ref[b, i, h] += pr[n] * pm[b, h, i, j] * v[b, j, h]
+                        dv_ref[b, j, h] += pr[n] * pm[b, h, i, j] * do[b, i, h]
+                        dq_ref[b, i, h] += ds[n] * k[b, j, h] / np.sqrt(dh)
+                        dk_ref[b, j, h] += ds[n] * q[b, i, h] / np.sqrt(dh)
+        for got, ref in ((o, o_ref), (dq, dq_ref), (dk, dk_ref), (dv, dv_ref)):
+            np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-14)
+    cfg = mini(0)
+    P = params64(cfg)
+    tok, lab = batch(cfg)
+    _, c = O.forward(cfg, P, tok, lab, None, (0.0, 5, 2, 0.4))
+    Bc, Sc = tok.shape
+    Hc = cfg.n_heads
+    Sp = (Sc + 3) // 4 * 4
+    for i in range(cfg.n_blocks):
+        m = c["blocks"][i]["pmask"]
+        assert m.shape == (Bc, Hc, Sc, Sc) and 0.3 < float((m == 0).mean()) < 0.5
+        flat = O.dropout_mask(Bc * Hc * Sc * Sp, 0.4, 5, 1000 + i, 2)
+        b, h, qi, kj = 1, Hc - 1, Sc - 1, 2
+        assert m[b, h, qi, kj] == flat[((b * Hc + h) * Sc + qi) * Sp + kj]
+    assert np.all(c["mask_emb"] == 1.0)                                    # the other rate is its own
+    l_plain, _ = O.forward(cfg, P, tok, lab)
+    l_none, c0 = O.forward(cfg, P, tok, lab, None, (0.2, 5, 2))            # three-element form: no attention dropout
+    assert c0["blocks"][0]["pmask"] is None and l_none != l_plain
+
+
 def test_dropout_zero_is_the_plain_model_and_the_mask_reaches_every_site():
     cfg = mini(0)
     P = params64(cfg)
