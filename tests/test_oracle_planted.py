@@ -29,11 +29,37 @@ def test_dropped_term_in_gelu_derivative_is_caught(monkeypatch):
 def test_missing_attention_scale_in_dk_is_caught(monkeypatch):
     orig = O.attention_bwd
 
-    def bad(do, q, k, v, p):
-        dq, dk, dv = orig(do, q, k, v, p)
+    def bad(do, q, k, v, p, pmask=None):
+        dq, dk, dv = orig(do, q, k, v, p, pmask)
         return dq, dk * np.sqrt(q.shape[-1]), dv
     monkeypatch.setattr(O, "attention_bwd", bad)
     _expect_caught(lambda: _fd_check(mini(1), n_samples=3))
+
+
+def test_attention_probability_mask_left_out_of_a_gradient_is_caught(monkeypatch):
+    from test_oracle_math import test_attention_probability_dropout_by_loops_and_its_element_numbering as pin_loops
+    orig = O.attention_bwd
+    # the mask forgotten on the way back to the softmax (dv still right)
+    def no_mask_on_dp(do, q, k, v, p, pmask=None):
+        dq, dk, _ = orig(do, q, k, v, p, None)
+        _, _, dv = orig(do, q, k, v, p, pmask)
+        return dq, dk, dv
+    monkeypatch.setattr(O, "attention_bwd", no_mask_on_dp)
+    _expect_caught(pin_loops)
+    _expect_caught(lambda: _fd_check(mini(0), n_samples=3, drop=(0.0, 78, 1, 0.25)))
+    # the mask applied before the normalisation instead of after it
+    monkeypatch.setattr(O, "attention_bwd", orig)
+    fwd = O.attention_fwd
+
+    def renormalised(q, k, v, causal, lens=None, pmask=None):
+        o, p = fwd(q, k, v, causal, lens, pmask)
+        if pmask is not None:
+            pd = p * pmask
+            pd = pd / np.maximum(pd.sum(-1, keepdims=True), 1e-30)
+            o = np.matmul(pd, v.transpose(0, 2, 1, 3)).transpose(0, 2, 1, 3)
+        return o, p
+    monkeypatch.setattr(O, "attention_fwd", renormalised)
+    _expect_caught(pin_loops)
 
 
 def test_key_padding_off_by_one_or_on_the_wrong_axis_is_caught(monkeypatch):
@@ -41,14 +67,14 @@ def test_key_padding_off_by_one_or_on_the_wrong_axis_is_caught(monkeypatch):
     from test_oracle_math import test_padded_batch_equals_the_sequences_run_alone as pin_batch
     orig = O.attention_fwd
     # the key at position len still visible
-    monkeypatch.setattr(O, "attention_fwd", lambda q, k, v, causal, lens=None:
-                        orig(q, k, v, causal, None if lens is None else [min(int(l) + 1, q.shape[1]) for l in lens]))
+    monkeypatch.setattr(O, "attention_fwd", lambda q, k, v, causal, lens=None, pmask=None:
+                        orig(q, k, v, causal, None if lens is None else [min(int(l) + 1, q.shape[1]) for l in lens], pmask))
     _expect_caught(pin_rows)
     _expect_caught(pin_batch)
 
     # the table applied to queries instead of keys: padded query rows zeroed, padded keys still seen
-    def on_queries(q, k, v, causal, lens=None):
-        o, p = orig(q, k, v, causal)
+    def on_queries(q, k, v, causal, lens=None, pmask=None):
+        o, p = orig(q, k, v, causal, None, pmask)
         if lens is not None:
             o = o.copy()
             for b, l in enumerate(lens):
