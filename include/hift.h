@@ -66,12 +66,17 @@ typedef struct {
   double  dropout;     /* probability p in [0, 1) of dropping an element at the outputs of each block's
                           attention projection and feed-forward network (before the residual addition)
                           and at the embedding output; kept values are scaled by 1/(1-p); 0 = none.
-                          The paper fine-tunes with the models' usual dropout without describing it;
-                          attention probabilities are not dropped here.                              */
+                          The paper fine-tunes with the models' usual dropout without describing it.   */
   uint64_t dropout_seed; /* the mask is Philox4x32-10(key = seed, counter = (element / 4, site, step)),
                           word element % 4, kept iff word >= floor(p 2^32); site 0 = embedding,
                           1 + 2 i = block i attention output, 2 + 2 i = its feed-forward output;
                           step = t.  Reproducible from (seed, t) alone, also across checkpoints.     */
+  double  attn_dropout; /* probability in [0, 1) of dropping an attention probability, after the softmax and
+                          before the product with V (kept ones scaled by 1/(1-p)); 0 = none.  Same seed;
+                          site 1000 + i for block i; the probabilities are numbered ((b H + h) S + q) S' + k
+                          with S' = seq rounded up to a multiple of 4.  The CUDA-core attention kernels
+                          apply it for every type and head size, so a bf16 configuration with this rate
+                          above 0 does not run its attention on the tensor cores.                    */
 } hift_model_cfg;
 
 /* Grouping and order (paper: Notation paragraph; Algorithm 1 "UpdateStrategy"). */

@@ -39,7 +39,7 @@ class ModelCfgC(C.Structure):
                 ("max_pos", C.c_int32), ("n_classes", C.c_int32), ("causal", C.c_int32),
                 ("tie_head", C.c_int32), ("dtype", C.c_int32), ("batch", C.c_int32),
                 ("seq", C.c_int32), ("norm_eps", C.c_double), ("rope_base", C.c_double),
-                ("dropout", C.c_double), ("dropout_seed", C.c_uint64)]
+                ("dropout", C.c_double), ("dropout_seed", C.c_uint64), ("attn_dropout", C.c_double)]
 
 
 class GroupCfgC(C.Structure):
@@ -179,7 +179,8 @@ class HiFT:
         m = ModelCfgC(model.arch, model.n_blocks, model.d_model, model.n_heads, model.d_ffn,
                       model.vocab, model.max_pos, model.n_classes, model.causal, model.tie_head,
                       model.dtype, model.batch, model.seq, model.norm_eps, model.rope_base,
-                      float(getattr(model, "dropout", 0.0)), int(getattr(model, "dropout_seed", 0)))
+                      float(getattr(model, "dropout", 0.0)), int(getattr(model, "dropout_seed", 0)),
+                      float(getattr(model, "attn_dropout", 0.0)))
         sizes = tuple(getattr(groups, "group_sizes", None) or ())
         arr = (C.c_int32 * len(sizes))(*sizes) if sizes else None
         g = GroupCfgC(groups.layers_per_group, groups.split_emb_head, groups.order, groups.order_seed,

@@ -101,6 +101,7 @@ struct hift_ctx {
   int shard_rank = 0, shard_world = 1;   // optimizer state sharded over data-parallel ranks (ZeRO stage 1)
   bool drop_on = false;             // dropout at the residual-branch outputs and the embedding output
   uint32_t drop_thr = 0; float drop_scale = 1.f;
+  uint32_t adrop_thr = 0; float adrop_scale = 1.f;   // dropout on attention probabilities (site 1000 + block)
   bool recompute = false;           // frozen blocks above the group keep only their input; see plan_slots
   bool keep_all = false;            // set while such a block is recomputed: its forward must store what the backward reads
   bool compact = false;             // paged master = low halves + carry bits beside the bf16 copy (see blob layout)
@@ -531,18 +532,25 @@ void bias_grad(hift_ctx* c, const void* dy, bool dy_f32, int64_t rows, int cols,
                           c->G(tb), nullptr, c->gbf));
   ++c->step_launches;
 }
-void attn_fwd(hift_ctx* c, const void* qkv, void* o, float* lse) {
+// dropout on the attention probabilities of block `blk`: thr = 0 when the rate is 0
+DropArgs attn_drop_args(const hift_ctx* c, int blk) {
+  DropArgs a;
+  a.k0 = (uint32_t)c->m.dropout_seed; a.k1 = (uint32_t)(c->m.dropout_seed >> 32);
+  a.site = (uint32_t)(1000 + blk); a.step = (uint32_t)c->t; a.thr = c->adrop_thr; a.scale = c->adrop_scale;
+  return a;
+}
+void attn_fwd(hift_ctx* c, int blk, const void* qkv, void* o, float* lse) {
   const double work = 4.0 * c->B * c->H * (double)c->S * c->S * c->dh * (c->m.causal ? 0.5 : 1.0);
   LAUNCH(HIFT_K_ATTN_FWD, work,
          launch_attention_fwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse,
-                              c->use_lens ? c->lens_dev : nullptr));
+                              c->use_lens ? c->lens_dev : nullptr, attn_drop_args(c, blk)));
 }
-void attn_bwd(hift_ctx* c, const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv) {
+void attn_bwd(hift_ctx* c, int blk, const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv) {
   const double work = 10.0 * c->B * c->H * (double)c->S * c->S * c->dh * (c->m.causal ? 0.5 : 1.0);
   LAUNCH(HIFT_K_ATTN_BWD, work,
          launch_attention_bwd(c->st, c->mixed, c->B, c->S, c->H, c->dh, c->m.causal, qkv, o, lse,
-                              dout, dqkv, c->dsum, c->use_lens ? c->lens_dev : nullptr));
-  c->step_launches += attention_use_mma(c->mixed, c->dh) ? 2 : 1;   // dsum, dq, dkv or dq, dkv
+                              dout, dqkv, c->dsum, c->use_lens ? c->lens_dev : nullptr, attn_drop_args(c, blk)));
+  c->step_launches += (attention_use_mma(c->mixed, c->dh) && !c->adrop_thr) ? 2 : 1;   // dsum, dq, dkv or dq, dkv
 }
 // qkv projection of a rotary model: on the tensor-core path the rotation of the q and k column blocks
 // happens in the GEMM's epilogue (head size 128); otherwise the projection is followed by the
@@ -676,7 +684,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
     float* x1r = (float*)s[S_H2R];
     float* z = (float*)s[S_Z];
     linear_fwd(c, T, 3 * d, d, x_a, d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
-    attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
+    attn_fwd(c, i, s[S_QKV], s[S_O], (float*)s[S_LSE]);
     linear_fwd_to_stream(c, 1 + 2 * i, T, d, d, s[S_O], c->P(b.w_o), x2, c->Pn(b.b_o), x_r);       // y
     norm_fwd(c, x2, b.n1_g, b.n1_b, s[S_H2], x1r, (float*)s[S_ST1]);                                 // x1
     linear_fwd_gelu(c, T, f, d, s[S_H2], c->P(b.w_fc1), s[S_A], s[S_U], c->Pn(b.b_fc1), c->keep_all || s[S_A] != c->slots[c->L][S_A]);
@@ -687,7 +695,7 @@ void forward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, float*
   norm_fwd(c, x_r, b.n1_g, b.n1_b, s[S_H1], nullptr, (float*)s[S_ST1]);
   if (c->m.arch == 2) linear_fwd_qkv_rope(c, T, d, s[S_H1], c->P(b.w_qkv), s[S_QKV], c->Pn(b.b_qkv));
   else linear_fwd(c, T, 3 * d, d, s[S_H1], d, c->P(b.w_qkv), s[S_QKV], 3 * d, c->Pn(b.b_qkv), nullptr, 0, false);
-  attn_fwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE]);
+  attn_fwd(c, i, s[S_QKV], s[S_O], (float*)s[S_LSE]);
   linear_fwd_to_stream(c, 1 + 2 * i, T, d, d, s[S_O], c->P(b.w_o), x2, c->Pn(b.b_o), x_r);
   norm_fwd(c, x2, b.n2_g, b.n2_b, s[S_H2], nullptr, (float*)s[S_ST2]);
   if (c->m.arch == 2) {
@@ -724,7 +732,7 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
     const float* ga = c->drop_on ? drop_bwd(c, 1 + 2 * i, c->dxb, c->dxb_a) : c->dxb;
     linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                  // do
     if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, ga, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
-    attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
+    attn_bwd(c, i, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
     if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, x_a, d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); grad_done(c, b.b_qkv); grad_done(c, b.w_qkv); }
     if (need_dx) linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dxa, d, c->dxb, d, true);
     return;
@@ -753,7 +761,7 @@ void backward_block(hift_ctx* c, int i, const float* x_r, const char* x_a, bool 
   const float* ga = c->drop_on ? drop_bwd(c, 1 + 2 * i, c->dxb, c->dxb_a) : c->dxb;
   linear_dx(c, T, d, d, c->dxb_a, d, c->P(b.w_o), c->dt1, d, nullptr, 0, false);                    // do
   if (on) { linear_dw(c, T, d, d, c->dxb_a, d, s[S_O], d, c->G(b.w_o)); bias_grad(c, ga, true, T, d, d, b.b_o); grad_done(c, b.b_o); grad_done(c, b.w_o); }
-  attn_bwd(c, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
+  attn_bwd(c, i, s[S_QKV], s[S_O], (float*)s[S_LSE], c->dt1, c->dqkv);
   if (c->m.arch == 2) rope(c, c->dqkv, -1.0f);
   linear_dx(c, T, 3 * d, d, c->dqkv, 3 * d, c->P(b.w_qkv), c->dt1, d, nullptr, 0, false);           // dh1
   if (on) { linear_dw(c, T, 3 * d, d, c->dqkv, 3 * d, s[S_H1], d, c->G(b.w_qkv)); bias_grad(c, c->dqkv, false, T, 3 * d, 3 * d, b.b_qkv); grad_done(c, b.b_qkv); grad_done(c, b.w_qkv); }
@@ -1257,6 +1265,7 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   if (m->arch == 2 && (m->d_model / m->n_heads) % 16) return HIFT_ERR_CFG;   // RoPE rotates 8 pairs per thread
   if (m->dtype != 0 && m->dtype != 1) return HIFT_ERR_CFG;
   if (!(m->dropout >= 0.0 && m->dropout < 1.0)) return HIFT_ERR_CFG;
+  if (!(m->attn_dropout >= 0.0 && m->attn_dropout < 1.0)) return HIFT_ERR_CFG;
   if (m->arch != 2 && m->max_pos < m->seq) return HIFT_ERR_CFG;
   if (m->arch == 1 && (m->n_classes < 2 || m->tie_head)) return HIFT_ERR_CFG;
   // several kernels launch one block per token, and the attention grids put the batch on z
@@ -1308,6 +1317,8 @@ hift_status hift_create(const hift_model_cfg* m, const hift_group_cfg* gc, const
   c->drop_on = m->dropout > 0.0;
   c->drop_thr = (uint32_t)floor(m->dropout * 4294967296.0);
   c->drop_scale = (float)(1.0 / (1.0 - m->dropout));
+  c->adrop_thr = (uint32_t)floor(m->attn_dropout * 4294967296.0);
+  c->adrop_scale = (float)(1.0 / (1.0 - m->attn_dropout));
   c->checked = g_checked_arena != 0;
   memset(c->prof_launches, 0, sizeof(c->prof_launches));
   memset(c->prof_ms, 0, sizeof(c->prof_ms));

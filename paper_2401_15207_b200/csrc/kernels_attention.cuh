@@ -13,6 +13,7 @@
 // quad shuffles.
 #pragma once
 #include "common.cuh"
+#include "dropout_rng.cuh"
 
 namespace hift {
 
@@ -38,7 +39,7 @@ __device__ __forceinline__ void stage_rows(float (*dst)[DH], const T* __restrict
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 attention_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o, float* __restrict__ lse,
-                     int S, int H, int causal, float scale, const int* __restrict__ lens) {
+                     int S, int H, int causal, float scale, const int* __restrict__ lens, DropArgs da) {
   constexpr int E = DH / 4;
   __shared__ float Ks[kAttTile][DH];
   __shared__ float Vs[kAttTile][DH];
@@ -60,6 +61,11 @@ attention_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o, float* __rest
   float m = -INFINITY, l = 0.f;
   const int q_last = min(q0 + kAttRows, S) - 1;
   const int k_end = min(causal ? q_last + 1 : S, klen);
+  // dropout on the probabilities (da.thr != 0): the sum l runs over all of them, the product with V over the kept
+  // ones; 1 / (1 - p) goes into the final scaling.  Tiles start at multiples of 32, so a generator block (four keys)
+  // never straddles two tiles.
+  const bool drop = da.thr != 0u;
+  uint4 dw = make_uint4(0u, 0u, 0u, 0u);
   for (int k0 = 0; k0 < k_end; k0 += kAttTile) {
     const int nk = min(kAttTile, S - k0);
     __syncthreads();
@@ -72,19 +78,21 @@ attention_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o, float* __rest
       for (int i = 0; i < E; ++i) s = fmaf(q[i], Ks[j][4 * i + p], s);
       s = quad_sum(s);
       const int key = k0 + j;
+      if (drop && (key & 3) == 0 && active) dw = attn_drop_words(da, b * H + h, S, qrow, key);
       if (active && key < klen && (!causal || key <= qrow)) {
         const float mn = fmaxf(m, s);
         const float corr = expf(m - mn);
         const float pj = expf(s - mn);
         l = l * corr + pj;
+        const float pv = (drop && word_of(dw, key & 3) < da.thr) ? 0.f : pj;
 #pragma unroll
-        for (int i = 0; i < E; ++i) acc[i] = fmaf(pj, Vs[j][4 * i + p], acc[i] * corr);
+        for (int i = 0; i < E; ++i) acc[i] = fmaf(pv, Vs[j][4 * i + p], acc[i] * corr);
         m = mn;
       }
     }
   }
   if (active) {
-    const float inv = 1.0f / l;
+    const float inv = (drop ? da.scale : 1.0f) / l;
     T* orow = o + ((int64_t)b * S + qrow) * d + (int64_t)h * DH;
 #pragma unroll
     for (int i = 0; i < E; ++i) orow[4 * i + p] = from_f<T>(acc[i] * inv);
@@ -98,7 +106,7 @@ __global__ void __launch_bounds__(256)
 attention_bwd_dq_kernel(const T* __restrict__ qkv, const T* __restrict__ o,
                         const float* __restrict__ lse, const T* __restrict__ dout,
                         T* __restrict__ dqkv, float* __restrict__ dsum, int S, int H, int causal,
-                        float scale, const int* __restrict__ lens) {
+                        float scale, const int* __restrict__ lens, DropArgs da) {
   constexpr int E = DH / 4;
   __shared__ float Ks[kAttTile][DH];
   __shared__ float Vs[kAttTile][DH];
@@ -129,6 +137,8 @@ attention_bwd_dq_kernel(const T* __restrict__ qkv, const T* __restrict__ o,
   }
   D = quad_sum(D);
   if (active && p == 0) dsum[((int64_t)b * H + h) * S + qrow] = D;
+  const bool drop = da.thr != 0u;
+  uint4 dw = make_uint4(0u, 0u, 0u, 0u);
   const int q_last = min(q0 + kAttRows, S) - 1;
   const int k_end = min(causal ? q_last + 1 : S, klen);
   for (int k0 = 0; k0 < k_end; k0 += kAttTile) {
@@ -147,7 +157,10 @@ attention_bwd_dq_kernel(const T* __restrict__ qkv, const T* __restrict__ o,
       s = quad_sum(s);
       dp = quad_sum(dp);
       const int key = k0 + j;
+      if (drop && (key & 3) == 0 && active) dw = attn_drop_words(da, b * H + h, S, qrow, key);
       if (active && key < klen && (!causal || key <= qrow)) {
+        // with dropout the gradient reaches the probability through its mask: dp -> dp o mask / (1 - p)
+        if (drop) dp = word_of(dw, key & 3) < da.thr ? 0.f : dp * da.scale;
         const float ds = expf(s - L) * (dp - D);
 #pragma unroll
         for (int i = 0; i < E; ++i) dq[i] = fmaf(ds, Ks[j][4 * i + p], dq[i]);
@@ -167,7 +180,7 @@ __global__ void __launch_bounds__(256)
 attention_bwd_dkv_kernel(const T* __restrict__ qkv, const float* __restrict__ lse,
                          const T* __restrict__ dout, const float* __restrict__ dsum,
                          T* __restrict__ dqkv, int S, int H, int causal, float scale,
-                         const int* __restrict__ lens) {
+                         const int* __restrict__ lens, DropArgs da) {
   constexpr int E = DH / 4;
   __shared__ float Qs[kAttTile][DH];
   __shared__ float Gs[kAttTile][DH];
@@ -213,10 +226,14 @@ attention_bwd_dkv_kernel(const T* __restrict__ qkv, const float* __restrict__ ls
       const int qrow = q0 + j;
       if (active && krow < klen && (!causal || krow <= qrow)) {
         const float pr = expf(s * scale - Ls[j]);
-        const float ds = pr * (dp - Ds[j]);
+        // with dropout: dv takes the dropped probability, and dp comes back through the same mask
+        float keep = 1.0f;
+        if (da.thr != 0u) keep = word_of(attn_drop_words(da, b * H + h, S, qrow, krow & ~3), krow & 3) < da.thr ? 0.f : da.scale;
+        const float ds = pr * (dp * keep - Ds[j]);
+        const float pd = pr * keep;
 #pragma unroll
         for (int i = 0; i < E; ++i) {
-          dv[i] = fmaf(pr, Gs[j][4 * i + p], dv[i]);
+          dv[i] = fmaf(pd, Gs[j][4 * i + p], dv[i]);
           dk[i] = fmaf(ds, Qs[j][4 * i + p], dk[i]);
         }
       }

@@ -6,6 +6,7 @@
 // parameter and GEMM-operand type (bf16 or fp32).
 #pragma once
 #include "common.cuh"
+#include "dropout_rng.cuh"
 
 namespace hift {
 
@@ -525,18 +526,6 @@ __global__ void publish_scalars_kernel(const float* __restrict__ src, const int*
 // 64-bit seed as key and (element / 4 as two words, site, step) as counter gives four 32-bit words, one per
 // element of an aligned group of four; an element is kept iff its word >= floor(p 2^32), kept values are
 // scaled by 1 / (1 - p).  One thread draws one group of four.
-struct DropArgs { uint32_t k0, k1, site, step, thr; float scale; };
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
-    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-  return c;
-}
 __device__ __forceinline__ float4 drop_mult4(size_t i4, const DropArgs& a) {
   const uint4 w = philox4x32_10(make_uint4((uint32_t)i4, (uint32_t)(i4 >> 32), a.site, a.step), a.k0, a.k1);
   return make_float4(w.x >= a.thr ? a.scale : 0.f, w.y >= a.thr ? a.scale : 0.f, w.z >= a.thr ? a.scale : 0.f,

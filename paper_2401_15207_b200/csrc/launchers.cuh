@@ -46,21 +46,21 @@ inline bool attention_head_ok(int dh) { return dh == 8 || dh == 16 || dh == 32 |
 
 template <typename T, int DH>
 inline void attention_fwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv,
-                               void* o, float* lse, const int* lens) {
+                               void* o, float* lse, const int* lens, const DropArgs& da) {
   dim3 grid((S + kAttRows - 1) / kAttRows, H, B);
   attention_fwd_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, (T*)o, lse, S, H, causal,
-                                                    1.0f / sqrtf((float)DH), lens);
+                                                    1.0f / sqrtf((float)DH), lens, da);
 }
 template <typename T, int DH>
 inline void attention_bwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv,
                                const void* o, const float* lse, const void* dout, void* dqkv,
-                               float* dsum, const int* lens) {
+                               float* dsum, const int* lens, const DropArgs& da) {
   dim3 grid((S + kAttRows - 1) / kAttRows, H, B);
   const float scale = 1.0f / sqrtf((float)DH);
   attention_bwd_dq_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, (const T*)o, lse,
-                                                       (const T*)dout, (T*)dqkv, dsum, S, H, causal, scale, lens);
+                                                       (const T*)dout, (T*)dqkv, dsum, S, H, causal, scale, lens, da);
   attention_bwd_dkv_kernel<T, DH><<<grid, 256, 0, st>>>((const T*)qkv, lse, (const T*)dout, dsum,
-                                                        (T*)dqkv, S, H, causal, scale, lens);
+                                                        (T*)dqkv, S, H, causal, scale, lens, da);
 }
 #define HIFT_DH_SWITCH(dh, CALL)            \
   switch (dh) {                             \
@@ -103,9 +103,12 @@ inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, 
   attn_bwd_dkv_mma_kernel<DH><<<grid, 128, attn_dkv_smem_bytes<DH>(), st>>>((const bf16*)qkv, lse, (const bf16*)dout, dsum,
                                                                            (bf16*)dqkv, S, H, causal, scale, lens);
 }
+// `da` (thr != 0): dropout on the probabilities (dropout_rng.cuh).  The CUDA-core kernels take it for every type and
+// head size; the warp-level kernels do not, so a dropped bf16 launch they would have got goes to the CUDA-core kernels.
 inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
-                                 const void* qkv, void* o, float* lse, const int* lens = nullptr) {
-  if (attention_use_mma(dtype, dh)) {
+                                 const void* qkv, void* o, float* lse, const int* lens = nullptr,
+                                 const DropArgs& da = DropArgs{0u, 0u, 0u, 0u, 0u, 1.0f}) {
+  if (attention_use_mma(dtype, dh) && da.thr == 0u) {
     if (gemm_tc_init() == 0 && attn_tc_eligible(dh, qkv, H)) {        // tcgen05 kernel
       attn_tc_fwd_launch(st, B, S, H, dh, causal, qkv, o, lse, lens);
       return;
@@ -115,15 +118,16 @@ inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H
     return;
   }
 #define CALL_F(D)                                                              \
-  if (dtype == 0) attention_fwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, lens); \
-  else attention_fwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, lens)
+  if (dtype == 0) attention_fwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, lens, da); \
+  else attention_fwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, lens, da)
   HIFT_DH_SWITCH(dh, CALL_F)
 #undef CALL_F
 }
 inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
                                  const void* qkv, const void* o, const float* lse, const void* dout,
-                                 void* dqkv, float* dsum, const int* lens = nullptr) {
-  if (attention_use_mma(dtype, dh)) {
+                                 void* dqkv, float* dsum, const int* lens = nullptr,
+                                 const DropArgs& da = DropArgs{0u, 0u, 0u, 0u, 0u, 1.0f}) {
+  if (attention_use_mma(dtype, dh) && da.thr == 0u) {
     if (gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv) && (((uintptr_t)o) & 15) == 0) {   // tcgen05 kernels
       launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
       attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv, lens);
@@ -134,8 +138,8 @@ inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H
     return;
   }
 #define CALL_B(D)                                                                              \
-  if (dtype == 0) attention_bwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens); \
-  else attention_bwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens)
+  if (dtype == 0) attention_bwd_inst<float, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens, da); \
+  else attention_bwd_inst<bf16, D>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens, da)
   HIFT_DH_SWITCH(dh, CALL_B)
 #undef CALL_B
 }

@@ -685,6 +685,29 @@ def test_dropout_masks_match_the_oracle(arch, dtype):
              resync=True)
 
 
+@pytest.mark.parametrize("arch,dtype", [(0, synth.DTYPE_FP32), (1, synth.DTYPE_FP32), (2, synth.DTYPE_FP32),
+                                        (0, synth.DTYPE_BF16), (1, synth.DTYPE_BF16), (2, synth.DTYPE_BF16)])
+@pytest.mark.parametrize("both", [0, 1])
+def test_attention_probability_dropout_matches_the_oracle(arch, dtype, both):
+    """Dropout on the attention probabilities (after the softmax, own rate, site 1000 + block, elements numbered with
+    rows padded to a multiple of four), alone and together with the dropout of the residual branches: a full cycle
+    in lockstep with the oracle.  The fp32 miniature has sequence length 40 with ragged key lengths and head size
+    16; the bf16 configurations have head sizes 64 and 128, whose attention leaves the tensor-core kernels when
+    this rate is above 0."""
+    fp32 = dtype == synth.DTYPE_FP32
+    extra = dict(attn_dropout=0.2, dropout_seed=0xABCDEF0123, dropout=0.1 if both else 0.0)
+    if fp32:
+        cfg = mini(arch, dtype, **extra)
+    else:
+        cfg = synth.ModelCfg(arch=arch, n_blocks=2, d_model=256, n_heads=2 if arch == 2 else 4, d_ffn=512, vocab=1001, max_pos=128,
+                             n_classes=2 if arch == 1 else 0, causal=0 if arch == 1 else 1, norm_eps=1e-6 if arch == 2 else 1e-5,
+                             dtype=dtype, batch=2, seq=128, init_std=0.05, **extra)
+    oc = synth.OptCfg(kind=0, lr=1e-3, offload_state=1, prefetch_groups=1)
+    lens = (lambda t: [cfg.seq - (3 * t + 5 * b) % (cfg.seq // 2) for b in range(cfg.batch)]) if fp32 and not both else None
+    lockstep(cfg, synth.GroupCfg(1), oc, cfg.n_units + 1, "zipf", FP32_LOSS if fp32 else BF16_LOSS, FP32_GRAD if fp32 else BF16_GRAD,
+             resync=True, lens=lens)
+
+
 def test_dropout_is_reproducible_and_recompute_redraws_the_same_masks():
     import torch
     from paper_2401_15207_b200 import HiFT
@@ -711,6 +734,10 @@ def test_dropout_is_reproducible_and_recompute_redraws_the_same_masks():
     b, pb = run(dropout=0.2, dropout_seed=5)
     c, _ = run(dropout=0.2, dropout_seed=6)
     r, pr = run(recompute=1, dropout=0.2, dropout_seed=5)
+    ad, pad = run(attn_dropout=0.2, dropout_seed=5)
+    adr, padr = run(recompute=1, attn_dropout=0.2, dropout_seed=5)
+    assert ad != plain and ad != a            # the probabilities' masks act, and are not the branches' masks
+    assert ad == adr and all(np.array_equal(x, y) for x, y in zip(pad, padr))
     assert plain == zero                      # p = 0 is the plain model, whatever the seed
     assert a == b and all(np.array_equal(x, y) for x, y in zip(pa, pb))
     assert a != plain and a != c              # the masks act, and follow the seed
