@@ -74,9 +74,9 @@ typedef struct {
   double  attn_dropout; /* probability in [0, 1) of dropping an attention probability, after the softmax and
                           before the product with V (kept ones scaled by 1/(1-p)); 0 = none.  Same seed;
                           site 1000 + i for block i; the probabilities are numbered ((b H + h) S + q) S' + k
-                          with S' = seq rounded up to a multiple of 4.  The CUDA-core attention kernels
-                          apply it for every type and head size, so a bf16 configuration with this rate
-                          above 0 does not run its attention on the tensor cores.                    */
+                          with S' = seq rounded up to a multiple of 4.  The tensor-core (tcgen05) and the
+                          CUDA-core attention kernels apply it; the warp-level fallback kernels do not, so a
+                          bf16 launch they would have taken goes to the CUDA-core kernels.            */
 } hift_model_cfg;
 
 /* Grouping and order (paper: Notation paragraph; Algorithm 1 "UpdateStrategy"). */

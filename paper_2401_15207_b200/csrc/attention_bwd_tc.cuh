@@ -66,13 +66,19 @@ __device__ __forceinline__ void tmem_ld_wait16(uint32_t (&v)[16]) {
 //   MODE 1   : row_l2 / row_d are this thread's own
 //   MASKED   : the block touches the diagonal or the end of the sequence (decided per step, so the
 //              common case carries no comparisons)
-template <int MODE, bool MASKED>
+//   DROP     : dropout on the probabilities: with keep = 0 or 1 / (1 - p) per (query, key), the P that feeds dV is
+//              P o keep and dS = P o (dP o keep - D).  MODE 1 draws one generator block per four of its keys; MODE 0
+//              has one key and sixteen queries, so one block per element.
+template <int MODE, bool MASKED, bool DROP>
 __device__ __forceinline__ void ab_p_ds16(const uint32_t (&sv)[16], const uint32_t (&pv)[16], float col_l2, float col_d,
                                           int lane_base, float row_l2, float row_d, float sl2, int S, int klen, int causal,
-                                          int frow, int x_first, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8]) {
+                                          int frow, int x_first, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8],
+                                          const DropArgs& da, int bh) {
+  uint4 w4 = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
     float pp[2], dd[2];
+    if (DROP && MODE == 1 && (i & 3) == 0) w4 = attn_drop_words(da, bh, S, min(frow, S - 1), x_first + i);
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const float l2 = MODE == 0 ? __shfl_sync(0xffffffffu, col_l2, lane_base + i + e) : row_l2;
@@ -83,8 +89,17 @@ __device__ __forceinline__ void ab_p_ds16(const uint32_t (&sv)[16], const uint32
         const int key = MODE == 0 ? frow : xi, qry = MODE == 0 ? xi : frow;
         if (key >= klen || qry >= S || (causal && key > qry)) p = 0.f;
       }
-      pp[e] = p;
-      dd[e] = p * (__uint_as_float(pv[i + e]) - dv);
+      if (DROP) {
+        uint32_t word;
+        if (MODE == 1) word = word_of(w4, (i + e) & 3);
+        else word = word_of(attn_drop_words(da, bh, S, min(x_first + i + e, S - 1), frow & ~3), frow & 3);
+        const float keep = word < da.thr ? 0.f : da.scale;
+        pp[e] = p * keep;
+        dd[e] = p * (__uint_as_float(pv[i + e]) * keep - dv);
+      } else {
+        pp[e] = p;
+        dd[e] = p * (__uint_as_float(pv[i + e]) - dv);
+      }
     }
     __nv_bfloat162 hp = __floats2bfloat162_rn(pp[0], pp[1]), hd = __floats2bfloat162_rn(dd[0], dd[1]);
     pk_p[i >> 1] = *reinterpret_cast<uint32_t*>(&hp);
@@ -92,14 +107,14 @@ __device__ __forceinline__ void ab_p_ds16(const uint32_t (&sv)[16], const uint32
   }
 }
 
-template <int DH, int MODE>
+template <int DH, int MODE, bool DROP>
 __global__ void __launch_bounds__(kAbThreads, 1)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_constant__ CUtensorMap map_f1,
                    const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1,
                    int col_f0, int col_f1, int col_x0, int col_x1,      // column of head 0 in each tensor
                    const float* __restrict__ lse, const float* __restrict__ dsum,
                    __nv_bfloat16* __restrict__ dqkv, int B, int S, int H, int causal, float scale,
-                   const int* __restrict__ lens) {
+                   const int* __restrict__ lens, DropArgs da) {
   typedef AttnBwdCfg<DH, MODE> Cfg;
   constexpr int SP = DH / 64;                            // 64-column swizzle spans per tile row
   constexpr int FSPAN = kAbF * 128, XSPAN = kAbX * 128;  // bytes of one span of a fixed / streamed tile
@@ -381,8 +396,14 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_f0, const __grid_cons
             if (lane == 0) mbar_arrive(s_free(u));        // the tensor core may overwrite tS / tP [u]
           }
           uint32_t pk_p[8], pk_ds[8];
-          if (masked) ab_p_ds16<MODE, true>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds);
-          else ab_p_ds16<MODE, false>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds);
+          const int bh = it.b * H + it.h;
+          if (DROP) {              // with dropout every step takes the instance with the mask tests
+            ab_p_ds16<MODE, true, true>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds, da, bh);
+          } else if (masked) {
+            ab_p_ds16<MODE, true, false>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds, da, bh);
+          } else {
+            ab_p_ds16<MODE, false, false>(sv, pv, col_l2, d_raw, hf * 16, row_l2, row_d, sl2, S, klen, causal, frow, xb0 + cb, pk_p, pk_ds, da, bh);
+          }
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             const int chunk = hc * 4 + hf * 2 + c;

@@ -96,11 +96,12 @@ __device__ __forceinline__ int tc_key_len(const int* __restrict__ lens, int b, i
   return lens != nullptr ? max(1, min(lens[b], S)) : S;
 }
 
-template <int DH>
+// DROP: dropout on the probabilities (its own instance, so that the plain kernel carries none of the generator's code)
+template <int DH, bool DROP>
 __global__ void __launch_bounds__(kAttThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* __restrict__ o,
                    float* __restrict__ lse, int B, int S, int H, int causal, float scale,
-                   const int* __restrict__ lens) {
+                   const int* __restrict__ lens, DropArgs da) {
   typedef AttnTcCfg<DH> Cfg;
   constexpr int SP = Cfg::kSpans;
   constexpr int SPAN_BYTES = 128 * 128;                 // 128 rows x 64 elements x 2 bytes
@@ -400,6 +401,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
           for (int e = 0; e < 4; ++e) { sc[i + e] = ex2_approx(fmaf(sc[i + e], sl2, nmuse)); sum4[e] += sc[i + e]; }
         }
         l = l * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+        // dropout on the probabilities (uniform across the CTA): the sum above runs over all of them, the product with
+        // V over the kept ones; 1 / (1 - p) goes into the final scaling.  One generator block per four keys.
+        if (DROP) {
+          const int bh = it.b * H + it.h, qd = min(qrow, S - 1), kfirst = j * kAttBK + half * HB;
+#pragma unroll
+          for (int i = 0; i < HB; i += 4) {
+            const uint4 w = attn_drop_words(da, bh, S, qd, kfirst + i);
+            if (w.x < da.thr) sc[i] = 0.f;
+            if (w.y < da.thr) sc[i + 1] = 0.f;
+            if (w.z < da.thr) sc[i + 2] = 0.f;
+            if (w.w < da.thr) sc[i + 3] = 0.f;
+          }
+        }
         if (pend_n >= 0) {                              // the previous item's output (uniform across the CTA)
           ok = finish_item();
           if (!ok) { pair_release(); break; }
@@ -443,7 +457,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* 
       pair_sync();
       if (half == 0 && qrow < S) lse[((int64_t)it.b * H + it.h) * S + qrow] = (m + log2f(ltot)) * 0.6931471805599453f;
       pend_n = n;
-      pend_inv = 1.0f / ltot;
+      pend_inv = (DROP ? da.scale : 1.0f) / ltot;
       pend_row = row_g0 + qrow;
       pend_end = row_g0 + S;
       pend_col = it.h * DH + half * OC;

@@ -1079,7 +1079,10 @@ int g_attn_tc = 1;       // tcgen05 attention forward (switch 2; 0 falls back to
 int g_attn_bwd_tc = 1;   // tcgen05 attention backward (switch 3; 0 falls back to the mma.sync kernels)
 template <int DH, int MODE>
 cudaError_t set_smem_attr_ab() {
-  return cudaFuncSetAttribute(attn_bwd_tc_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attn_bwd_tc_kernel<DH, MODE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AttnBwdCfg<DH, MODE>::kSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_bwd_tc_kernel<DH, MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               AttnBwdCfg<DH, MODE>::kSmem);
 }
 int g_pair_mode = 1;     // CTA-pair kernel for 256-wide tiles (switch 0; 0 falls back to one CTA per tile)
@@ -1124,8 +1127,10 @@ int gemm_tc_init() {
   if (e == cudaSuccess) e = set_smem_attr2<false, true, true>();
   if (e == cudaSuccess) e = set_smem_attr2<true, true, true>();
   if (e == cudaSuccess) e = set_smem_attr2<true, true, false>();
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::kSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_tc_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::kSmem);
   if (e == cudaSuccess) e = set_smem_attr_ab<64, 0>();
   if (e == cudaSuccess) e = set_smem_attr_ab<64, 1>();
   if (e == cudaSuccess) e = set_smem_attr_ab<128, 0>();
@@ -1239,16 +1244,17 @@ bool attn_tc_eligible(int dh, const void* qkv, int H) {
   return g_init_state == 0 && g_attn_tc && (dh == 128 || dh == 64) && (((uintptr_t)qkv) & 15) == 0 && ((3 * H * dh) % 8) == 0;
 }
 cudaError_t attn_tc_fwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, void* o, float* lse,
-                               const int* lens) {
+                               const int* lens, const DropArgs& da) {
   CUtensorMap tm;
   const uint64_t d3 = 3ull * H * dh;
   if (!get_map(qkv, d3, (uint64_t)B * S, d3, 128, &tm)) return cudaErrorInvalidValue;
   const int nitems = ((S + kAttBQ - 1) / kAttBQ) * H * B;
   const int grid = nitems < g_num_sms ? nitems : g_num_sms;          // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)dh);
-  if (dh == 64)
-    return launch_pdl_tc(attn_fwd_tc_kernel<64>, dim3(grid), dim3(kAttThreads), AttnTcCfg<64>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale, lens);
-  return launch_pdl_tc(attn_fwd_tc_kernel<128>, dim3(grid), dim3(kAttThreads), AttnTcCfg<128>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale, lens);
+#define HIFT_ATTN_FWD(D, DR) launch_pdl_tc(attn_fwd_tc_kernel<D, DR>, dim3(grid), dim3(kAttThreads), AttnTcCfg<D>::kSmem, st, tm, (__nv_bfloat16*)o, lse, B, S, H, causal, scale, lens, da)
+  if (da.thr != 0u) return dh == 64 ? HIFT_ATTN_FWD(64, true) : HIFT_ATTN_FWD(128, true);
+  return dh == 64 ? HIFT_ATTN_FWD(64, false) : HIFT_ATTN_FWD(128, false);
+#undef HIFT_ATTN_FWD
 }
 
 bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, const void* dqkv) {
@@ -1257,7 +1263,7 @@ bool attn_tc_bwd_eligible(int dh, int H, const void* qkv, const void* dout, cons
 }
 template <int DH>
 static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int causal, const void* qkv, const void* dout,
-                                    const float* lse, const float* dsum, void* dqkv, const int* lens) {
+                                    const float* lse, const float* dsum, void* dqkv, const int* lens, const DropArgs& da) {
   const uint64_t d = (uint64_t)H * DH, d3 = 3 * d, rows = (uint64_t)B * S;
   CUtensorMap qkv_f, qkv_x, do_f, do_x;
   if (!get_map(qkv, d3, rows, d3, kAbF, &qkv_f) || !get_map(qkv, d3, rows, d3, kAbX, &qkv_x) ||
@@ -1267,17 +1273,22 @@ static cudaError_t attn_tc_bwd_inst(cudaStream_t st, int B, int S, int H, int ca
   const int grid = nitems < g_num_sms ? nitems : g_num_sms;       // persistent: one CTA per SM
   const float scale = 1.0f / sqrtf((float)DH);
   // dK, dV: fixed K, V; streamed Q, dO
-  cudaError_t e = launch_pdl_tc(attn_bwd_tc_kernel<DH, 0>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 0>::kSmem, st,
-      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale, lens);
+#define HIFT_ATTN_BWD0(DR) launch_pdl_tc(attn_bwd_tc_kernel<DH, 0, DR>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 0>::kSmem, st, \
+      qkv_f, qkv_f, qkv_x, do_x, (int)d, (int)(2 * d), 0, 0, lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale, lens, da)
+#define HIFT_ATTN_BWD1(DR) launch_pdl_tc(attn_bwd_tc_kernel<DH, 1, DR>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 1>::kSmem, st, \
+      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale, lens, da)
+  const bool drop = da.thr != 0u;
+  cudaError_t e = drop ? HIFT_ATTN_BWD0(true) : HIFT_ATTN_BWD0(false);
   if (e != cudaSuccess) return e;
   // dQ: fixed Q, dO; streamed K, V
-  return launch_pdl_tc(attn_bwd_tc_kernel<DH, 1>, dim3(grid), dim3(kAbThreads), AttnBwdCfg<DH, 1>::kSmem, st,
-      qkv_f, do_f, qkv_x, qkv_x, 0, 0, (int)d, (int)(2 * d), lse, dsum, (__nv_bfloat16*)dqkv, B, S, H, causal, scale, lens);
+  return drop ? HIFT_ATTN_BWD1(true) : HIFT_ATTN_BWD1(false);
+#undef HIFT_ATTN_BWD0
+#undef HIFT_ATTN_BWD1
 }
 cudaError_t attn_tc_bwd_launch(cudaStream_t st, int B, int S, int H, int dh, int causal, const void* qkv, const void* dout,
-                               const float* lse, const float* dsum, void* dqkv, const int* lens) {
-  if (dh == 64) return attn_tc_bwd_inst<64>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv, lens);
-  return attn_tc_bwd_inst<128>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv, lens);
+                               const float* lse, const float* dsum, void* dqkv, const int* lens, const DropArgs& da) {
+  if (dh == 64) return attn_tc_bwd_inst<64>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv, lens, da);
+  return attn_tc_bwd_inst<128>(st, B, S, H, causal, qkv, dout, lse, dsum, dqkv, lens, da);
 }
 
 int gemm_tc_set_error(int v) {

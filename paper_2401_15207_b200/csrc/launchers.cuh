@@ -104,15 +104,16 @@ inline void attention_mma_bwd(cudaStream_t st, int B, int S, int H, int causal, 
                                                                            (bf16*)dqkv, S, H, causal, scale, lens);
 }
 // `da` (thr != 0): dropout on the probabilities (dropout_rng.cuh).  The CUDA-core kernels take it for every type and
-// head size; the warp-level kernels do not, so a dropped bf16 launch they would have got goes to the CUDA-core kernels.
+// head size, the tcgen05 kernels for theirs; the warp-level kernels do not, so a dropped bf16 launch they would have
+// got (tcgen05 switched off, or operands that are not 16-byte aligned) goes to the CUDA-core kernels.
 inline void launch_attention_fwd(cudaStream_t st, int dtype, int B, int S, int H, int dh, int causal,
                                  const void* qkv, void* o, float* lse, const int* lens = nullptr,
                                  const DropArgs& da = DropArgs{0u, 0u, 0u, 0u, 0u, 1.0f}) {
+  if (attention_use_mma(dtype, dh) && gemm_tc_init() == 0 && attn_tc_eligible(dh, qkv, H)) {        // tcgen05 kernel
+    attn_tc_fwd_launch(st, B, S, H, dh, causal, qkv, o, lse, lens, da);
+    return;
+  }
   if (attention_use_mma(dtype, dh) && da.thr == 0u) {
-    if (gemm_tc_init() == 0 && attn_tc_eligible(dh, qkv, H)) {        // tcgen05 kernel
-      attn_tc_fwd_launch(st, B, S, H, dh, causal, qkv, o, lse, lens);
-      return;
-    }
     if (dh == 64) attention_mma_fwd<64>(st, B, S, H, causal, qkv, o, lse, lens);
     else attention_mma_fwd<128>(st, B, S, H, causal, qkv, o, lse, lens);
     return;
@@ -127,12 +128,13 @@ inline void launch_attention_bwd(cudaStream_t st, int dtype, int B, int S, int H
                                  const void* qkv, const void* o, const float* lse, const void* dout,
                                  void* dqkv, float* dsum, const int* lens = nullptr,
                                  const DropArgs& da = DropArgs{0u, 0u, 0u, 0u, 0u, 1.0f}) {
+  if (attention_use_mma(dtype, dh) && gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv) &&
+      (((uintptr_t)o) & 15) == 0) {                                                                   // tcgen05 kernels
+    launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
+    attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv, lens, da);
+    return;
+  }
   if (attention_use_mma(dtype, dh) && da.thr == 0u) {
-    if (gemm_tc_init() == 0 && attn_tc_bwd_eligible(dh, H, qkv, dout, dqkv) && (((uintptr_t)o) & 15) == 0) {   // tcgen05 kernels
-      launch_attn_dsum(st, (const bf16*)o, (const bf16*)dout, dsum, B, S, H, dh);
-      attn_tc_bwd_launch(st, B, S, H, dh, causal, qkv, dout, lse, dsum, dqkv, lens);
-      return;
-    }
     if (dh == 64) attention_mma_bwd<64>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens);
     else attention_mma_bwd<128>(st, B, S, H, causal, qkv, o, lse, dout, dqkv, dsum, lens);
     return;
