@@ -911,7 +911,7 @@ hift_status enqueue_forward_backward(hift_ctx* c, const int32_t* tok, const int3
     norm_fwd(c, c->x_final, c->t_fg, c->t_fb, c->xf, nullptr, c->stf);
     const int tw = m.tie_head ? c->t_tok : c->t_wh;
     linear_fwd(c, T, V, d, c->xf, d, c->P(tw), c->logits, Vp, nullptr, nullptr, 0, false);
-    LAUNCH(HIFT_K_CE, 4.0 * T * (double)V * c->es,
+    LAUNCH(HIFT_K_CE, 2.0 * T * (double)Vp * c->es,       // one read of the logits, one write of their gradient
            launch_cross_entropy(c->st, c->mixed, T, V, Vp, c->logits, lab, c->rowloss, nvalid, bad, c->scal));
     c->step_launches += 2;
   }

@@ -195,10 +195,14 @@ inline void launch_cross_entropy(cudaStream_t st, int dtype, int64_t rows, int64
                                  int* bad, float* loss) {
   count_valid_kernel<<<1, 256, 0, st>>>(labels, rows, nvalid);
   const int th = vocab >= 4096 ? 512 : (vocab >= 256 ? 128 : 32);
-  if (dtype == 0)
-    cross_entropy_kernel<float><<<(unsigned)rows, th, 0, st>>>((float*)logits, labels, rowloss, nvalid, bad, vocab, ld);
-  else
-    cross_entropy_kernel<bf16><<<(unsigned)rows, th, 0, st>>>((bf16*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+  const bool vec = (((uintptr_t)logits) & 15) == 0 && ld % (dtype == 0 ? 4 : 8) == 0;     // 16-byte rows
+  if (dtype == 0) {
+    if (vec) cross_entropy_vec_kernel<float><<<(unsigned)rows, th, 0, st>>>((float*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+    else cross_entropy_kernel<float><<<(unsigned)rows, th, 0, st>>>((float*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+  } else {
+    if (vec) cross_entropy_vec_kernel<bf16><<<(unsigned)rows, th, 0, st>>>((bf16*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+    else cross_entropy_kernel<bf16><<<(unsigned)rows, th, 0, st>>>((bf16*)logits, labels, rowloss, nvalid, bad, vocab, ld);
+  }
   loss_reduce_kernel<<<1, 256, 0, st>>>(rowloss, rows, nvalid, loss);
 }
 
