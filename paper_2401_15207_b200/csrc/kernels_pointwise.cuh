@@ -212,6 +212,75 @@ __global__ void norm_fwd_kernel(const float* __restrict__ x, const P* __restrict
   }
 }
 
+// The same with the row held in registers: every thread loads its NC chunks of 8 once (cols <= 8 * NC * blockDim.x) and the
+// two reductions and the output run from registers; per-thread and block summation orders are those of the kernel above,
+// so the results are the same bits.
+template <typename P, int KIND, int NC>
+__global__ void norm_fwd_reg_kernel(const float* __restrict__ x, const P* __restrict__ gain,
+                                    const P* __restrict__ bias, P* __restrict__ y_a,
+                                    float* __restrict__ y_r, float* __restrict__ stats, int64_t rows,
+                                    int cols, float eps) {
+  pdl_launch_next();
+  pdl_wait_prior();
+  __shared__ float red[33];
+  const int64_t row = blockIdx.x;
+  const float* xr = x + row * cols;
+  float v[NC][8];
+#pragma unroll
+  for (int k = 0; k < NC; ++k) {
+    const int c = (threadIdx.x + k * blockDim.x) * 8;
+    if (c < cols) load8(xr + c, v[k]);
+    else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[k][i] = 0.f;
+    }
+  }
+  float mean = 0.f;
+  if (KIND == 0) {
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < NC; ++k) {
+      if ((threadIdx.x + k * blockDim.x) * 8 < cols) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s += v[k][i];
+      }
+    }
+    mean = block_sum(s, red) / cols;
+  }
+  float q = 0.f;
+#pragma unroll
+  for (int k = 0; k < NC; ++k) {
+    if ((threadIdx.x + k * blockDim.x) * 8 < cols) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q += (v[k][i] - mean) * (v[k][i] - mean);
+    }
+  }
+  const float var = block_sum(q, red) / cols;
+  const float rstd = 1.0f / sqrtf(var + eps);
+  if (threadIdx.x == 0) {
+    stats[row] = mean;
+    stats[rows + row] = rstd;
+  }
+#pragma unroll
+  for (int k = 0; k < NC; ++k) {
+    const int c = (threadIdx.x + k * blockDim.x) * 8;
+    if (c >= cols) continue;
+    float g[8];
+    load8(gain + c, g);
+    if (KIND == 0) {
+      float b[8];
+      load8(bias + c, b);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[k][i] = (v[k][i] - mean) * rstd * g[i] + b[i];
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[k][i] = v[k][i] * rstd * g[i];
+    }
+    store8(y_a + row * cols + c, v[k]);
+    if (y_r) store8(y_r + row * cols + c, v[k]);
+  }
+}
+
 // dx = norm_bwd(dy; x, stats, gain) (+ add).  One block per row.  dy is either a GEMM
 // output (type P) or a residual-stream gradient (fp32).  dx_r: fp32 stream gradient;
 // dx_a (optional): the same values rounded once to the GEMM-operand type.

@@ -152,10 +152,17 @@ inline void launch_norm_fwd(cudaStream_t st, int dtype, int kind, int64_t rows, 
                             const float* x, const void* gain, const void* bias, void* y_a, float* y_r,
                             float* stats) {
   const int th = norm_threads(cols);
-#define NF(P, K) launch_pdl(norm_fwd_kernel<P, K>, dim3((unsigned)rows), dim3(th), 0, st, x, (const P*)gain, (const P*)bias, (P*)y_a, y_r, stats, rows, cols, eps)
+  const int nc = (cols / 8 + th - 1) / th;            // chunks of 8 per thread: rows up to 8192 wide stay in registers
+#define NFR(P, K, NC) launch_pdl(norm_fwd_reg_kernel<P, K, NC>, dim3((unsigned)rows), dim3(th), 0, st, x, (const P*)gain, (const P*)bias, (P*)y_a, y_r, stats, rows, cols, eps)
+#define NF(P, K)                                                                                                   \
+  do {                                                                                                             \
+    if (nc <= 1) NFR(P, K, 1); else if (nc == 2) NFR(P, K, 2); else if (nc <= 4) NFR(P, K, 4);                      \
+    else launch_pdl(norm_fwd_kernel<P, K>, dim3((unsigned)rows), dim3(th), 0, st, x, (const P*)gain, (const P*)bias, (P*)y_a, y_r, stats, rows, cols, eps); \
+  } while (0)
   if (dtype == 0) { if (kind == 0) NF(float, 0); else NF(float, 1); }
   else { if (kind == 0) NF(bf16, 0); else NF(bf16, 1); }
 #undef NF
+#undef NFR
 }
 // dy_f32: dy is an fp32 stream gradient (else it has the operand type)
 inline void launch_norm_bwd_dx(cudaStream_t st, int dtype, int kind, bool dy_f32, int64_t rows, int cols,
