@@ -162,11 +162,22 @@ def run_reference(args, cfg, gcfg, ocfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    times = []
-    for _ in range(args.warmup_ref + args.steps_ref):
+    # --steps K --warmup W as for the other arm, each step one bounded sample of the workload; the run is kept to about
+    # three minutes: once the first sample has shown what a step costs, W and K are cut to what fits (the line reports
+    # the steps that ran and the steps that were asked for).  --steps-ref / --warmup-ref > 0 override K and W.
+    K_req = args.steps_ref if args.steps_ref > 0 else args.steps
+    W_req = args.warmup_ref if args.steps_ref > 0 else args.warmup
+    budget_s = 180.0
+    t_start = time.perf_counter()
+    dt, desc, flops, threads = oracle_sample(cfg, gcfg, ocfg)
+    fit = max(1, int((budget_s - (time.perf_counter() - t_start)) / max(dt, 1e-3)))
+    W_run = min(W_req, max(0, fit - 1), 1 if fit < W_req + K_req else W_req)
+    K_run = max(1, min(K_req, fit + 1 - W_run))
+    times = [dt]
+    for _ in range(W_run + K_run - 1):
         dt, desc, flops, threads = oracle_sample(cfg, gcfg, ocfg)
         times.append(dt)
-    times = times[args.warmup_ref:]
+    times = times[W_run:]
     dt = float(np.mean(times))
     groups = [(g[0], g[-1]) for g in __import__("oracle.hift_oracle", fromlist=["x"]).build_groups(
         cfg.n_units, gcfg.layers_per_group, gcfg.split_emb_head)]
@@ -174,7 +185,8 @@ def run_reference(args, cfg, gcfg, ocfg):
     value = cfg.tokens_per_step / (dt * full / flops)
     line = {
         "impl": "reference", "metric": "HiFT step tokens/s", "value": value, "unit": "tokens/s",
-        "n_gpus": args.gpus, "steps": args.steps_ref, "warmup": args.warmup_ref, "ms_per_step": dt * full / flops * 1e3,
+        "n_gpus": args.gpus, "steps": K_run, "warmup": W_run, "steps_requested": K_req, "warmup_requested": W_req,
+        "ms_per_step": dt * full / flops * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "note": "CPU oracle on a bounded sample, extrapolated by flops"},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
@@ -816,7 +828,7 @@ def main():
                     help="single kernels at the workload's shapes, a few launches each (small enough for an ncu capture)")
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--only", default=None, help="--micro gemm: only shapes whose name contains this")
-    ap.add_argument("--steps-ref", type=int, default=2)
+    ap.add_argument("--steps-ref", type=int, default=0, help="--impl reference: overrides --steps / --warmup when > 0")
     ap.add_argument("--warmup-ref", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
@@ -832,7 +844,6 @@ def main():
         gcfg = synth.GroupCfg(layers_per_group=cfg.n_units, split_emb_head=0, order=synth.ORDER_BOTTOM2UP)
         args.offload, args.prefetch = 0, 0
     if args.impl == "reference":
-        args.steps_ref = max(1, min(args.steps, args.steps_ref))
         run_reference(args, cfg, gcfg, ocfg)
     else:
         run_ours(args, cfg, gcfg, ocfg)
