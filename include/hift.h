@@ -419,6 +419,17 @@ hift_status hift_k_attention_bwd(int32_t dtype, int32_t batch, int32_t seq, int3
                                  const void *o_dev, const float *lse_dev, const void *do_dev,
                                  void *dqkv_dev, float *dsum_dev, const int32_t *key_lens_dev,
                                  void *cuda_stream);
+/* The same two with dropout on the probabilities (hift_model_cfg.attn_dropout): rate p in [0, 1), the generator's
+ * seed, site and step as the step would pass them (site 1000 + block, step t).  p = 0 is the plain kernel. */
+hift_status hift_k_attention_fwd_drop(int32_t dtype, int32_t batch, int32_t seq, int32_t n_heads,
+                                      int32_t d_head, int32_t causal, const void *qkv_dev, void *o_dev,
+                                      float *lse_dev, const int32_t *key_lens_dev, double p, uint64_t seed,
+                                      int32_t site, int64_t step, void *cuda_stream);
+hift_status hift_k_attention_bwd_drop(int32_t dtype, int32_t batch, int32_t seq, int32_t n_heads,
+                                      int32_t d_head, int32_t causal, const void *qkv_dev,
+                                      const void *o_dev, const float *lse_dev, const void *do_dev,
+                                      void *dqkv_dev, float *dsum_dev, const int32_t *key_lens_dev, double p,
+                                      uint64_t seed, int32_t site, int64_t step, void *cuda_stream);
 /* Rotary models (RoPE on q and k, as in the LLaMA-shaped configuration the paper profiles) on the
  * tensor-core path: the rotation is fused into the epilogue of the qkv projection, and this hook
  * exposes exactly that kernel: out[M,N] = rope(x[M,K] w[N,K]^T + bias) on columns [0, rope_cols),

@@ -120,6 +120,8 @@ def _prototypes():
         "hift_k_linear": (C.c_int, [i32, i32, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_attention_fwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
         "hift_k_attention_bwd": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
+        "hift_k_attention_fwd_drop": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, f64, C.c_uint64, i32, i64, vp]),
+        "hift_k_attention_bwd_drop": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, f64, C.c_uint64, i32, i64, vp]),
         "hift_k_linear_rope": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, i64, vp]),
         "hift_k_linear_swiglu": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp, vp]),
         "hift_k_linear_dx_swiglu_bwd": (C.c_int, [i64, i64, i64, vp, vp, vp, vp, vp]),
@@ -510,6 +512,19 @@ def k_attention_fwd(dtype, B, S, H, dh, causal, qkv, o, lse, stream=None, key_le
 def k_attention_bwd(dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, stream=None, key_lens=None):
     _check(lib().hift_k_attention_bwd(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout),
                                       _ptr(dqkv), _ptr(dsum), _ptr(key_lens), _st(stream)), "hift_k_attention_bwd")
+
+
+def k_attention_fwd_drop(dtype, B, S, H, dh, causal, qkv, o, lse, p, seed, site, step, stream=None, key_lens=None):
+    _check(lib().hift_k_attention_fwd_drop(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(key_lens),
+                                           float(p), int(seed), int(site), int(step), _st(stream)),
+           "hift_k_attention_fwd_drop")
+
+
+def k_attention_bwd_drop(dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, p, seed, site, step, stream=None,
+                         key_lens=None):
+    _check(lib().hift_k_attention_bwd_drop(dtype, B, S, H, dh, causal, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout),
+                                           _ptr(dqkv), _ptr(dsum), _ptr(key_lens), float(p), int(seed),
+                                           int(site), int(step), _st(stream)), "hift_k_attention_bwd_drop")
 
 
 def k_linear_rope(M, N, K, a, b, out, bias, cs, seq, d_head, rope_cols, stream=None):

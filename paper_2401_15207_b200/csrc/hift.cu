@@ -2158,6 +2158,28 @@ hift_status hift_k_attention_bwd(int32_t dtype, int32_t B, int32_t S, int32_t H,
   launch_attention_bwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, key_lens);
   return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
 }
+static DropArgs attn_drop_of(double p, uint64_t seed, int32_t site, int64_t step) {
+  DropArgs a;
+  a.k0 = (uint32_t)seed; a.k1 = (uint32_t)(seed >> 32); a.site = (uint32_t)site; a.step = (uint32_t)step;
+  a.thr = (uint32_t)floor(p * 4294967296.0); a.scale = (float)(1.0 / (1.0 - p));
+  return a;
+}
+hift_status hift_k_attention_fwd_drop(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
+                                      const void* qkv, void* o, float* lse, const int32_t* key_lens, double p,
+                                      uint64_t seed, int32_t site, int64_t step, void* stream) {
+  if (!attention_head_ok(dh) || dtype < 0 || dtype > 1 || !(p >= 0.0 && p < 1.0)) return HIFT_ERR_CFG;
+  launch_attention_fwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, key_lens, attn_drop_of(p, seed, site, step));
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
+hift_status hift_k_attention_bwd_drop(int32_t dtype, int32_t B, int32_t S, int32_t H, int32_t dh, int32_t causal,
+                                      const void* qkv, const void* o, const float* lse, const void* dout,
+                                      void* dqkv, float* dsum, const int32_t* key_lens, double p, uint64_t seed,
+                                      int32_t site, int64_t step, void* stream) {
+  if (!attention_head_ok(dh) || dtype < 0 || dtype > 1 || !(p >= 0.0 && p < 1.0)) return HIFT_ERR_CFG;
+  launch_attention_bwd((cudaStream_t)stream, dtype, B, S, H, dh, causal, qkv, o, lse, dout, dqkv, dsum, key_lens,
+                       attn_drop_of(p, seed, site, step));
+  return cudaGetLastError() == cudaSuccess ? HIFT_OK : HIFT_ERR_CUDA;
+}
 hift_status hift_k_linear_rope(int64_t M, int64_t N, int64_t K, const void* a, const void* b, void* out, const void* bias,
                                const float* cs, int32_t seq, int32_t d_head, int64_t rope_cols, void* stream) {
   if (M < 1 || N < 1 || K < 1 || !cs || seq < 1) return HIFT_ERR_CFG;

@@ -242,6 +242,50 @@ def test_attention_tensor_core_edge_lengths(dh, B, S, H, causal):
         assert_elem(got[:, i * d:(i + 1) * d], r, U_BF16, sl[1 + i].reshape(B * S, d) + 1e-12, "dq dk dv"[3 * i:3 * i + 2])
 
 
+@pytest.mark.parametrize("dtype,dh,B,S,H", [(1, 128, 6, 300, 26), (1, 64, 5, 200, 32), (0, 32, 2, 75, 3), (1, 16, 2, 130, 2)])
+@pytest.mark.parametrize("causal", [0, 1])
+def test_attention_with_probability_dropout(dtype, dh, B, S, H, causal):
+    """Attention with dropout on the probabilities, kernel by kernel against the oracle with the same mask: the
+    tcgen05 kernels at more work items than SMs with ragged tails (sequence lengths that are no multiple of the
+    tile or of four, ragged key lengths on top), and the CUDA-core kernels in fp32 and bf16."""
+    import torch
+    from paper_2401_15207_b200 import k_attention_fwd_drop, k_attention_bwd_drop
+    p_drop, seed, site, step = 0.3, 0x5EED_0123_4567, 1003, 17
+    d = H * dh
+    rng = np.random.default_rng(100 * dh + S + causal)
+    qkv = rng.standard_normal((B * S, 3 * d)).astype(np.float32)
+    do = rng.standard_normal((B * S, d)).astype(np.float32)
+    lens = [S - (7 * b) % (S // 2) for b in range(B)]
+    bf = dtype == 1
+    cvt = _bf if bf else (lambda a: a.astype(np.float64))
+    q, k, v = (cvt(qkv)[:, i * d:(i + 1) * d].reshape(B, S, H, dh) for i in range(3))
+    Sp = (S + 3) // 4 * 4
+    pm = O.dropout_mask(B * H * S * Sp, p_drop, seed, site, step).reshape(B, H, S, Sp)[..., :S]
+    o_ref, p = O.attention_fwd(q, k, v, bool(causal), lens, pm)
+    td = torch.bfloat16 if bf else torch.float32
+    tq = _t(qkv, td)
+    tl = _t(np.asarray(lens, dtype=np.int32))
+    o = torch.full((B * S, d), 9.0, dtype=td, device="cuda")
+    lse = torch.full((B, H, S), 9.0, dtype=torch.float32, device="cuda")
+    k_attention_fwd_drop(dtype, B, S, H, dh, causal, tq, o, lse, p_drop, seed, site, step, key_lens=tl)
+    got_o = o.float().cpu().numpy()
+    u = U_BF16 if bf else 4 * U_F32
+    sl = attention_slack(q, k, v, p * pm, cvt(do).reshape(B, S, H, dh), u)
+    assert rel_l2(got_o, o_ref.reshape(B * S, d)) <= (6e-3 if bf else 3e-6)
+    assert_elem(got_o, o_ref.reshape(B * S, d), u, sl[0].reshape(B * S, d) * (1.0 / (1.0 - p_drop)) + 1e-12, "o")
+    dqkv = torch.full((B * S, 3 * d), 9.0, dtype=td, device="cuda")
+    dsum = torch.empty(B * S * H, dtype=torch.float32, device="cuda")
+    k_attention_bwd_drop(dtype, B, S, H, dh, causal, tq, o, lse, _t(do, td), dqkv, dsum, p_drop, seed, site, step, key_lens=tl)
+    dq, dk, dv = O.attention_bwd(cvt(do).reshape(B, S, H, dh), q, k, v, p, pm)
+    ref = np.concatenate([t.reshape(B * S, d) for t in (dq, dk, dv)], axis=1)
+    got = dqkv.float().cpu().numpy()
+    for i in range(3):
+        assert rel_l2(got[:, i * d:(i + 1) * d], ref[:, i * d:(i + 1) * d]) <= (1.5e-2 if bf else 1e-5), i
+    # the mask really is the oracle's: without it the output differs by far more than any tolerance
+    o2, _ = O.attention_fwd(q, k, v, bool(causal), lens)
+    assert rel_l2(got_o, o2.reshape(B * S, d)) > 0.1
+
+
 @pytest.mark.parametrize("dtype,dh", [(0, 32), (1, 64), (1, 128)])
 @pytest.mark.parametrize("causal", [0, 1])
 def test_attention_key_lengths(dtype, dh, causal):
