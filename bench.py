@@ -163,11 +163,11 @@ def run_reference(args, cfg, gcfg, ocfg):
     if rank != 0:
         return
     # --steps K --warmup W as for the other arm, each step one bounded sample of the workload; the run is kept to about
-    # three minutes: once the first sample has shown what a step costs, W and K are cut to what fits (the line reports
+    # two and a half minutes: once the first sample has shown what a step costs, W and K are cut to what fits (the line reports
     # the steps that ran and the steps that were asked for).  --steps-ref / --warmup-ref > 0 override K and W.
     K_req = args.steps_ref if args.steps_ref > 0 else args.steps
     W_req = args.warmup_ref if args.steps_ref > 0 else args.warmup
-    budget_s = 180.0
+    budget_s = 150.0
     t_start = time.perf_counter()
     dt, desc, flops, threads = oracle_sample(cfg, gcfg, ocfg)
     fit = max(1, int((budget_s - (time.perf_counter() - t_start)) / max(dt, 1e-3)))
