@@ -78,4 +78,30 @@ gemm_simt_kernel(int M, int N, int K, const TIN* __restrict__ a, int64_t sam, in
   }
 }
 
+// The same contraction for products with few outputs and a long k (the 2-class head: 16 x 2 outputs over k = 768):
+// one warp per output element, lanes strided over k, a fixed shuffle tree at the end.  The tiled kernel above would
+// run such a product in one block, k-step by k-step.
+template <typename TIN, typename TOUT>
+__global__ void __launch_bounds__(256)
+gemm_few_outputs_kernel(int M, int N, int K, const TIN* __restrict__ a, int64_t sam, int64_t sak,
+                        const TIN* __restrict__ b, int64_t sbk, int64_t sbn, TOUT* __restrict__ c,
+                        int64_t ldc, const TIN* __restrict__ bias, const float* __restrict__ residual,
+                        int64_t ldr) {
+  const int lane = threadIdx.x & 31;
+  const int64_t out = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (out >= (int64_t)M * N) return;
+  const int m = (int)(out / N), n = (int)(out % N);
+  const TIN* ap = a + (int64_t)m * sam;
+  const TIN* bp = b + (int64_t)n * sbn;
+  float acc = 0.f;
+  for (int k = lane; k < K; k += 32) acc = fmaf(to_f(ap[(int64_t)k * sak]), to_f(bp[(int64_t)k * sbk]), acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    if (bias) acc += to_f(bias[n]);
+    if (residual) acc += residual[(int64_t)m * ldr + n];
+    c[(int64_t)m * ldc + n] = from_f<TOUT>(acc);
+  }
+}
+
 }  // namespace hift

@@ -25,6 +25,17 @@ inline int norm_threads(int cols) {
 
 // ---- GEMM (CUDA cores) ----------------------------------------------------------
 inline void launch_gemm_simt(cudaStream_t st, int dtype, const GemmArgs& g) {
+  if ((int64_t)g.M * g.N <= 1024 && g.K >= 256) {      // few outputs, long k: one warp per output
+    const unsigned blocks = (unsigned)(((int64_t)g.M * g.N + 7) / 8);
+#define HIFT_FEW(TI, TO, BIAS, RES, LDR)                                                                                  \
+  gemm_few_outputs_kernel<TI, TO><<<blocks, 256, 0, st>>>(g.M, g.N, g.K, (const TI*)g.a, g.sam, g.sak, (const TI*)g.b, g.sbk, \
+                                                          g.sbn, (TO*)g.c, g.ldc, (const TI*)BIAS, RES, LDR)
+    if (dtype == 0) HIFT_FEW(float, float, g.bias, g.residual, g.ldr);
+    else if (g.out_f32) HIFT_FEW(bf16, float, g.bias, g.residual, g.ldr);
+    else HIFT_FEW(bf16, bf16, g.bias, nullptr, 0);
+#undef HIFT_FEW
+    return;
+  }
   dim3 grid((g.N + 63) / 64, (g.M + 63) / 64);
   if (dtype == 0) {
     gemm_simt_kernel<float, float><<<grid, 256, 0, st>>>(
